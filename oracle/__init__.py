@@ -1,0 +1,1 @@
+"""Float64 CPU oracle: test infrastructure, never imported by the product package."""

@@ -1,0 +1,346 @@
+/*
+ * kopref — float64 CPU oracle for the fused pointwise+reduction segments.
+ *
+ * TEST INFRASTRUCTURE ONLY. This file is the slow, plain definition of what each
+ * segment computes. It is used by the tests, by the smoke check and by the
+ * benchmark's cpu_baseline / reference legs; the product path (the CUDA library)
+ * never links, loads or calls it, and it shares no code, header, table or
+ * constant with that path.
+ *
+ * The paper names these segment classes (planner strategies 8-9, the codegen
+ * agent's "beating Inductor" list and the fusion agent's technique list:
+ * fused softmax, single-pass LayerNorm / RMSNorm, activation+bias fusion,
+ * residual+norm, reduction+pointwise, LogSumExp reductions) but never prints
+ * their formulas, so each function below writes out the textbook definition in
+ * the most direct form: two passes where the definition has two passes, no
+ * online recurrences, no blocking, no reordering. The fast methods the CUDA
+ * path uses (row in registers, online max/sum) reach the same real number up
+ * to rounding order, so the plain definition is the reference.
+ *
+ * Conventions
+ *   - data tensors come in as fp32, bf16 bit patterns (uint16) or fp64, chosen
+ *     by a dtype tag; they are widened exactly to double. Parameter vectors
+ *     (bias, gamma, beta, scale, shift, weight) are fp32 and widened exactly.
+ *   - every output is double, never rounded back.
+ *   - strides are in elements; the innermost stride is 1.
+ *   - `threads` > 1 splits the outer (row / plane) loop with OpenMP; each row is
+ *     still computed by one thread in index order, so results do not depend on it.
+ *   - return value 0 = ok, negative = bad argument.
+ *
+ * All parity pins live in tests/test_oracle_pins.py; every function is pinned.
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { KOPREF_F32 = 0, KOPREF_BF16 = 1, KOPREF_F64 = 2 };
+
+/* ---- exact widening / narrowing helpers ------------------------------------ */
+
+/* bf16 is the upper 16 bits of an IEEE binary32, so widening is exact. */
+double kopref_bf16_to_f64(uint16_t bits)
+{
+    uint32_t u = ((uint32_t)bits) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/* Round a double directly to bf16 (round to nearest, ties to even) without
+ * passing through fp32, so there is no double rounding. bf16 has 8 significant
+ * bits (1 implicit + 7 stored) and the fp32 exponent range. */
+uint16_t kopref_f64_to_bf16_rne(double v)
+{
+    if (v != v) return 0x7FC0u;                          /* quiet NaN */
+    uint16_t sign = signbit(v) ? 0x8000u : 0u;
+    double a = fabs(v);
+    if (a == 0.0) return sign;
+    if (isinf(a)) return (uint16_t)(sign | 0x7F80u);
+    int e;
+    (void)frexp(a, &e);                                  /* a = m * 2^e, m in [0.5, 1) */
+    int exp_unbiased = e - 1;                            /* a = (2m) * 2^(e-1), 2m in [1,2) */
+    if (exp_unbiased < -126) exp_unbiased = -126;        /* subnormal range: fixed quantum */
+    /* quantum of the bf16 grid at this exponent: 2^(exp_unbiased - 7) */
+    double q = ldexp(1.0, exp_unbiased - 7);
+    double n = a / q;                                    /* exact: power-of-two division */
+    double fl = floor(n);
+    double frac = n - fl;
+    if (frac > 0.5 || (frac == 0.5 && fmod(fl, 2.0) == 1.0)) fl += 1.0;
+    double r = fl * q;                                   /* rounded magnitude */
+    if (r >= ldexp(1.0, 128)) return (uint16_t)(sign | 0x7F80u);   /* overflow to inf */
+    float rf = (float)r;                                 /* exact: r is on the bf16 grid */
+    uint32_t u;
+    memcpy(&u, &rf, sizeof u);
+    return (uint16_t)(sign | (uint16_t)(u >> 16));
+}
+
+static inline double load_elem(const void* base, int64_t idx, int dtype)
+{
+    switch (dtype) {
+    case KOPREF_F32:  return (double)((const float*)base)[idx];
+    case KOPREF_BF16: return kopref_bf16_to_f64(((const uint16_t*)base)[idx]);
+    default:          return ((const double*)base)[idx];
+    }
+}
+
+static int bad_dtype(int dtype) { return dtype < KOPREF_F32 || dtype > KOPREF_F64; }
+
+static int pick_threads(int threads)
+{
+#ifdef _OPENMP
+    if (threads < 1) threads = 1;
+    return threads;
+#else
+    (void)threads;
+    return 1;
+#endif
+}
+
+int kopref_has_openmp(void)
+{
+#ifdef _OPENMP
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+/* ---- softmax(x * s + b) over each row ---------------------------------------
+ * z_j = x_j * s + b_j ; m = max_j z_j ; e_j = exp(z_j - m) ; S = sum_j e_j ;
+ * y_j = e_j / S.   ("fused softmax", planner strategy 9.)  bias may be NULL (= 0).
+ * A row whose z are all -inf gives NaN, as the definition's 0/0 does. */
+int kopref_softmax_scale_bias(const void* x, const float* bias, double* y,
+                              int64_t rows, int64_t cols, int64_t x_row_stride,
+                              int64_t y_row_stride, double scale, int dtype, int threads)
+{
+    if (!x || !y || rows < 0 || cols <= 0 || bad_dtype(dtype)) return -1;
+    int nt = pick_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t i = 0; i < rows; ++i) {
+        double* yr = y + i * y_row_stride;
+        double m = -INFINITY;
+        for (int64_t j = 0; j < cols; ++j) {
+            double z = load_elem(x, i * x_row_stride + j, dtype) * scale
+                     + (bias ? (double)bias[j] : 0.0);
+            yr[j] = z;
+            if (z > m) m = z;
+        }
+        double S = 0.0;
+        for (int64_t j = 0; j < cols; ++j) {
+            double e = exp(yr[j] - m);
+            yr[j] = e;
+            S += e;
+        }
+        for (int64_t j = 0; j < cols; ++j) yr[j] = yr[j] / S;
+    }
+    return 0;
+}
+
+/* ---- tanh-form GELU --------------------------------------------------------
+ * g(u) = 0.5 u (1 + tanh( sqrt(2/pi) (u + 0.044715 u^3) )). */
+double kopref_gelu_tanh(double u)
+{
+    const double k = sqrt(2.0 / 3.14159265358979323846264338327950288);
+    return 0.5 * u * (1.0 + tanh(k * (u + 0.044715 * u * u * u)));
+}
+
+/* ---- bias + GELU + residual + LayerNorm --------------------------------------
+ * v_j = r_j + g(x_j + b_j) ; mu = (1/H) sum v ; var = (1/H) sum (v - mu)^2 (biased) ;
+ * rstd = 1 / sqrt(var + eps) ; y_j = (v_j - mu) rstd gamma_j + beta_j.
+ * ("residual + norm" and "normalization fusion" in the fusion agent's list,
+ * "activation + bias fusion" for the prologue.)  v is never rounded.
+ * mean / rstd may be NULL. */
+int kopref_bias_gelu_residual_layernorm(const void* x, const void* residual,
+        const float* bias, const float* gamma, const float* beta,
+        double* y, double* mean, double* rstd,
+        int64_t rows, int64_t hidden, int64_t x_row_stride, int64_t res_row_stride,
+        int64_t y_row_stride, double eps, int dtype, int threads)
+{
+    if (!x || !residual || !bias || !gamma || !beta || !y) return -1;
+    if (rows < 0 || hidden <= 0 || bad_dtype(dtype)) return -1;
+    int nt = pick_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t i = 0; i < rows; ++i) {
+        double* yr = y + i * y_row_stride;
+        double sum = 0.0;
+        for (int64_t j = 0; j < hidden; ++j) {
+            double u = load_elem(x, i * x_row_stride + j, dtype) + (double)bias[j];
+            double v = load_elem(residual, i * res_row_stride + j, dtype) + kopref_gelu_tanh(u);
+            yr[j] = v;
+            sum += v;
+        }
+        double mu = sum / (double)hidden;
+        double ss = 0.0;
+        for (int64_t j = 0; j < hidden; ++j) {
+            double d = yr[j] - mu;
+            ss += d * d;
+        }
+        double var = ss / (double)hidden;
+        double rs = 1.0 / sqrt(var + eps);
+        for (int64_t j = 0; j < hidden; ++j)
+            yr[j] = (yr[j] - mu) * rs * (double)gamma[j] + (double)beta[j];
+        if (mean) mean[i] = mu;
+        if (rstd) rstd[i] = rs;
+    }
+    return 0;
+}
+
+/* ---- inference BatchNorm affine + ReLU + global average pool (NCHW) ----------
+ * a[n,c,h,w] = relu(x[n,c,h,w] * scale[c] + shift[c]) ; p[n,c] = mean_{h,w} a.
+ * relu(v) = v if v > 0, 0 otherwise, and NaN stays NaN.  ("reduction +
+ * pointwise"; BN / pooling epilogues of the CNN models.)  x and y are
+ * contiguous NCHW. y may be NULL (only the pooled output is produced). */
+int kopref_bn_relu_avgpool(const void* x, const float* scale, const float* shift,
+        double* y, double* pooled, int64_t N, int64_t C, int64_t H, int64_t W,
+        int dtype, int threads)
+{
+    if (!x || !scale || !shift || !pooled) return -1;
+    if (N < 0 || C <= 0 || H <= 0 || W <= 0 || bad_dtype(dtype)) return -1;
+    int64_t plane = H * W;
+    int64_t planes = N * C;
+    int nt = pick_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t p = 0; p < planes; ++p) {
+        int64_t c = p % C;
+        double sc = (double)scale[c], sh = (double)shift[c];
+        double sum = 0.0;
+        for (int64_t k = 0; k < plane; ++k) {
+            double v = load_elem(x, p * plane + k, dtype) * sc + sh;
+            double a = (v != v) ? v : (v > 0.0 ? v : 0.0);
+            if (y) y[p * plane + k] = a;
+            sum += a;
+        }
+        pooled[p] = sum / (double)plane;
+    }
+    return 0;
+}
+
+/* ---- row-wise cross-entropy ---------------------------------------------------
+ * m = max_j z_j ; lse = m + ln sum_j exp(z_j - m) ; loss_i = lse - z[i, label_i] ;
+ * mean = (1/M) sum_i loss_i (row order).  ("LogSumExp reductions"; the loss is
+ * logsumexp minus the label logit.)  A label outside [0, V) gives loss NaN and
+ * is counted in *bad_label_count. mean_loss / bad_label_count may be NULL. */
+int kopref_ce_loss_rowwise(const void* logits, const int32_t* labels,
+        double* loss, double* mean_loss, int64_t* bad_label_count,
+        int64_t rows, int64_t vocab, int64_t row_stride, int dtype, int threads)
+{
+    if (!logits || !labels || !loss) return -1;
+    if (rows < 0 || vocab <= 0 || bad_dtype(dtype)) return -1;
+    int nt = pick_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t i = 0; i < rows; ++i) {
+        double m = -INFINITY;
+        for (int64_t j = 0; j < vocab; ++j) {
+            double z = load_elem(logits, i * row_stride + j, dtype);
+            if (z > m) m = z;
+        }
+        double S = 0.0;
+        for (int64_t j = 0; j < vocab; ++j)
+            S += exp(load_elem(logits, i * row_stride + j, dtype) - m);
+        double lse = m + log(S);
+        int32_t lab = labels[i];
+        if (lab < 0 || (int64_t)lab >= vocab) loss[i] = NAN;
+        else loss[i] = lse - load_elem(logits, i * row_stride + lab, dtype);
+    }
+    int64_t bad = 0;
+    double total = 0.0;
+    for (int64_t i = 0; i < rows; ++i) {
+        int32_t lab = labels[i];
+        if (lab < 0 || (int64_t)lab >= vocab) ++bad;
+        total += loss[i];
+    }
+    if (mean_loss) *mean_loss = rows > 0 ? total / (double)rows : NAN;
+    if (bad_label_count) *bad_label_count = bad;
+    return 0;
+}
+
+/* ---- RMSNorm -------------------------------------------------------------------
+ * y_j = x_j / sqrt( (1/H) sum_k x_k^2 + eps ) * w_j.  ("RMSNorm sequences".) */
+int kopref_rmsnorm(const void* x, const float* weight, double* y,
+        int64_t rows, int64_t hidden, int64_t x_row_stride, int64_t y_row_stride,
+        double eps, int dtype, int threads)
+{
+    if (!x || !weight || !y || rows < 0 || hidden <= 0 || bad_dtype(dtype)) return -1;
+    int nt = pick_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t i = 0; i < rows; ++i) {
+        double ss = 0.0;
+        for (int64_t j = 0; j < hidden; ++j) {
+            double v = load_elem(x, i * x_row_stride + j, dtype);
+            ss += v * v;
+        }
+        double r = 1.0 / sqrt(ss / (double)hidden + eps);
+        for (int64_t j = 0; j < hidden; ++j)
+            y[i * y_row_stride + j] =
+                load_elem(x, i * x_row_stride + j, dtype) * r * (double)weight[j];
+    }
+    return 0;
+}
+
+/* ---- SiLU(gate) * up -------------------------------------------------------------
+ * Row layout [gate(0..I) | up(I..2I)]; out_j = gate_j / (1 + exp(-gate_j)) * up_j.
+ * ("activation fusion (GELU/SiLU/ReLU)"; only the epilogue is fused.) */
+int kopref_silu_mul(const void* gate_up, double* out, int64_t rows, int64_t inter,
+        int64_t in_row_stride, int64_t out_row_stride, int dtype, int threads)
+{
+    if (!gate_up || !out || rows < 0 || inter <= 0 || bad_dtype(dtype)) return -1;
+    int nt = pick_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t i = 0; i < rows; ++i) {
+        for (int64_t j = 0; j < inter; ++j) {
+            double g = load_elem(gate_up, i * in_row_stride + j, dtype);
+            double u = load_elem(gate_up, i * in_row_stride + inter + j, dtype);
+            out[i * out_row_stride + j] = g / (1.0 + exp(-g)) * u;
+        }
+    }
+    return 0;
+}
+
+/* ---- residual add ---------------------------------------------------------------
+ * out = a + b ("pointwise + pointwise: load once, store once"). */
+int kopref_residual_add(const void* a, const void* b, double* out, int64_t rows, int64_t cols,
+        int64_t a_row_stride, int64_t b_row_stride, int64_t out_row_stride,
+        int dtype, int threads)
+{
+    if (!a || !b || !out || rows < 0 || cols <= 0 || bad_dtype(dtype)) return -1;
+    int nt = pick_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t i = 0; i < rows; ++i)
+        for (int64_t j = 0; j < cols; ++j)
+            out[i * out_row_stride + j] = load_elem(a, i * a_row_stride + j, dtype)
+                                        + load_elem(b, i * b_row_stride + j, dtype);
+    return 0;
+}
+
+/* ---- C = A * W^T (the preserved vendor GEMM, written as the triple loop) -----------
+ * A [M,K] and W [N,K] row-major with their own dtype tags, C [M,N] double.
+ * Used only for the chained-segment check. */
+int kopref_gemm_nt(const void* A, int a_dtype, const void* Wt, int w_dtype, double* Cout,
+        int64_t M, int64_t N, int64_t K, int threads)
+{
+    if (!A || !Wt || !Cout || M < 0 || N <= 0 || K <= 0) return -1;
+    if (bad_dtype(a_dtype) || bad_dtype(w_dtype)) return -1;
+    int nt = pick_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t i = 0; i < M; ++i)
+        for (int64_t n = 0; n < N; ++n) {
+            double acc = 0.0;
+            for (int64_t k = 0; k < K; ++k)
+                acc += load_elem(A, i * K + k, a_dtype) * load_elem(Wt, n * K + k, w_dtype);
+            Cout[i * N + n] = acc;
+        }
+    return 0;
+}

@@ -1,0 +1,224 @@
+"""ctypes front end of the float64 CPU oracle (oracle/kopref.c).
+
+TEST INFRASTRUCTURE ONLY: imported by tests/, by the smoke check and by the
+benchmark's cpu_baseline / reference legs. The product package never imports it,
+and this module imports nothing from the product package.
+
+Data tensors may be numpy arrays (float32, float64, or uint16 holding bf16 bit
+patterns) or CPU torch tensors (float32, float64, bfloat16); they must be
+contiguous in their last dimension. Every result is a float64 numpy array.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+from . import build as _build
+
+F32, BF16, F64 = 0, 1, 2
+_lib = None
+
+
+def lib() -> C.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(_build.build())
+        i64, dbl, vp = C.c_int64, C.c_double, C.c_void_p
+        _lib.kopref_bf16_to_f64.restype = dbl
+        _lib.kopref_bf16_to_f64.argtypes = [C.c_uint16]
+        _lib.kopref_f64_to_bf16_rne.restype = C.c_uint16
+        _lib.kopref_f64_to_bf16_rne.argtypes = [dbl]
+        _lib.kopref_gelu_tanh.restype = dbl
+        _lib.kopref_gelu_tanh.argtypes = [dbl]
+        _lib.kopref_softmax_scale_bias.argtypes = [vp, vp, vp, i64, i64, i64, i64, dbl, C.c_int, C.c_int]
+        _lib.kopref_bias_gelu_residual_layernorm.argtypes = [vp] * 8 + [i64] * 5 + [dbl, C.c_int, C.c_int]
+        _lib.kopref_bn_relu_avgpool.argtypes = [vp] * 5 + [i64] * 4 + [C.c_int, C.c_int]
+        _lib.kopref_ce_loss_rowwise.argtypes = [vp] * 5 + [i64] * 3 + [C.c_int, C.c_int]
+        _lib.kopref_rmsnorm.argtypes = [vp] * 3 + [i64] * 4 + [dbl, C.c_int, C.c_int]
+        _lib.kopref_silu_mul.argtypes = [vp] * 2 + [i64] * 4 + [C.c_int, C.c_int]
+        _lib.kopref_residual_add.argtypes = [vp] * 3 + [i64] * 5 + [C.c_int, C.c_int]
+        _lib.kopref_gemm_nt.argtypes = [vp, C.c_int, vp, C.c_int, vp, i64, i64, i64, C.c_int]
+    return _lib
+
+
+def host_threads() -> int:
+    """Host cores this process may use (what `threads=None` resolves to)."""
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:  # pragma: no cover
+        return os.cpu_count() or 1
+
+
+def _nt(threads) -> int:
+    return host_threads() if threads is None else int(threads)
+
+
+def as_data(a):
+    """Return (numpy array, dtype tag) for a data tensor without changing any bit."""
+    if hasattr(a, "detach"):  # torch tensor
+        import torch
+        a = a.detach()
+        assert a.device.type == "cpu", "oracle inputs live on the host"
+        if a.dtype == torch.bfloat16:
+            return a.contiguous().view(torch.int16).numpy().view(np.uint16), BF16
+        a = a.contiguous().numpy()
+    a = np.asarray(a)
+    if a.dtype == np.float32:
+        return np.ascontiguousarray(a), F32
+    if a.dtype == np.uint16:
+        return np.ascontiguousarray(a), BF16
+    if a.dtype == np.float64:
+        return np.ascontiguousarray(a), F64
+    raise TypeError(f"unsupported oracle data dtype {a.dtype}")
+
+
+def as_param(a):
+    """fp32 parameter vector as a contiguous numpy array (None stays None)."""
+    if a is None:
+        return None
+    if hasattr(a, "detach"):
+        a = a.detach().cpu().numpy()
+    a = np.ascontiguousarray(a)
+    assert a.dtype == np.float32, "parameter vectors are fp32"
+    return a
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _check(rc, name):
+    if rc != 0:
+        raise ValueError(f"{name}: bad argument (rc={rc})")
+
+
+def bf16_to_f64(bits) -> np.ndarray:
+    bits = np.asarray(bits, dtype=np.uint16)
+    f = lib().kopref_bf16_to_f64
+    return np.array([f(int(b)) for b in bits.ravel()], dtype=np.float64).reshape(bits.shape)
+
+
+def f64_to_bf16_rne(v) -> np.ndarray:
+    v = np.asarray(v, dtype=np.float64)
+    f = lib().kopref_f64_to_bf16_rne
+    return np.array([f(float(t)) for t in v.ravel()], dtype=np.uint16).reshape(v.shape)
+
+
+def gelu_tanh(u: float) -> float:
+    return lib().kopref_gelu_tanh(float(u))
+
+
+def softmax_scale_bias(x, bias, scale, threads=1) -> np.ndarray:
+    xa, dt = as_data(x)
+    rows, cols = xa.shape
+    b = as_param(bias)
+    y = np.empty((rows, cols), dtype=np.float64)
+    _check(lib().kopref_softmax_scale_bias(_p(xa), _p(b), _p(y), rows, cols, cols, cols,
+                                           float(scale), dt, _nt(threads)), "softmax_scale_bias")
+    return y
+
+
+def bias_gelu_residual_layernorm(x, residual, bias, gamma, beta, eps, threads=1):
+    """Returns (y, mean, rstd)."""
+    xa, dt = as_data(x)
+    ra, dt2 = as_data(residual)
+    assert dt == dt2 and xa.shape == ra.shape
+    rows, hidden = xa.shape
+    b, g, be = as_param(bias), as_param(gamma), as_param(beta)
+    y = np.empty((rows, hidden), dtype=np.float64)
+    mean = np.empty(rows, dtype=np.float64)
+    rstd = np.empty(rows, dtype=np.float64)
+    _check(lib().kopref_bias_gelu_residual_layernorm(
+        _p(xa), _p(ra), _p(b), _p(g), _p(be), _p(y), _p(mean), _p(rstd),
+        rows, hidden, hidden, hidden, hidden, float(eps), dt, _nt(threads)),
+        "bias_gelu_residual_layernorm")
+    return y, mean, rstd
+
+
+def bn_relu_avgpool(x, scale, shift, threads=1, want_y=True):
+    """x is NCHW contiguous. Returns (y or None, pooled[N,C])."""
+    xa, dt = as_data(x)
+    N, Cc, H, W = xa.shape
+    sc, sh = as_param(scale), as_param(shift)
+    y = np.empty((N, Cc, H, W), dtype=np.float64) if want_y else None
+    pooled = np.empty((N, Cc), dtype=np.float64)
+    _check(lib().kopref_bn_relu_avgpool(_p(xa), _p(sc), _p(sh), _p(y), _p(pooled),
+                                        N, Cc, H, W, dt, _nt(threads)), "bn_relu_avgpool")
+    return y, pooled
+
+
+def ce_loss_rowwise(logits, labels, threads=1):
+    """Returns (loss[rows], mean, bad_label_count)."""
+    za, dt = as_data(logits)
+    rows, vocab = za.shape
+    if hasattr(labels, "detach"):
+        labels = labels.detach().cpu().numpy()
+    lab = np.ascontiguousarray(labels, dtype=np.int32)
+    loss = np.empty(rows, dtype=np.float64)
+    mean = C.c_double(0.0)
+    bad = C.c_int64(0)
+    _check(lib().kopref_ce_loss_rowwise(_p(za), _p(lab), _p(loss), C.addressof(mean),
+                                        C.addressof(bad), rows, vocab, vocab, dt, _nt(threads)),
+           "ce_loss_rowwise")
+    return loss, mean.value, bad.value
+
+
+def rmsnorm(x, weight, eps, threads=1) -> np.ndarray:
+    xa, dt = as_data(x)
+    rows, hidden = xa.shape
+    w = as_param(weight)
+    y = np.empty((rows, hidden), dtype=np.float64)
+    _check(lib().kopref_rmsnorm(_p(xa), _p(w), _p(y), rows, hidden, hidden, hidden,
+                                float(eps), dt, _nt(threads)), "rmsnorm")
+    return y
+
+
+def silu_mul(gate_up, threads=1) -> np.ndarray:
+    ga, dt = as_data(gate_up)
+    rows, two_i = ga.shape
+    assert two_i % 2 == 0
+    inter = two_i // 2
+    out = np.empty((rows, inter), dtype=np.float64)
+    _check(lib().kopref_silu_mul(_p(ga), _p(out), rows, inter, two_i, inter, dt, _nt(threads)),
+           "silu_mul")
+    return out
+
+
+def residual_add(a, b, threads=1) -> np.ndarray:
+    aa, dt = as_data(a)
+    ba, dt2 = as_data(b)
+    assert dt == dt2 and aa.shape == ba.shape
+    rows, cols = aa.shape
+    out = np.empty((rows, cols), dtype=np.float64)
+    _check(lib().kopref_residual_add(_p(aa), _p(ba), _p(out), rows, cols, cols, cols, cols,
+                                     dt, _nt(threads)), "residual_add")
+    return out
+
+
+def gemm_nt(a, w, threads=1) -> np.ndarray:
+    """C = A @ W^T with A [M,K], W [N,K]; triple loop in float64."""
+    aa, adt = as_data(a)
+    wa, wdt = as_data(w)
+    M, K = aa.shape
+    N, K2 = wa.shape
+    assert K == K2
+    out = np.empty((M, N), dtype=np.float64)
+    _check(lib().kopref_gemm_nt(_p(aa), adt, _p(wa), wdt, _p(out), M, N, K, _nt(threads)), "gemm_nt")
+    return out
+
+
+def mlp_segment(h, rms_weight, w_gate_up, w_down, eps, threads=1) -> np.ndarray:
+    """The chained segment in pure float64, no intermediate rounding:
+    out = h + (silu(gate) * up) @ W2^T with [gate|up] = rmsnorm(h) @ W1^T."""
+    n = rmsnorm(h, rms_weight, eps, threads)
+    gu = gemm_nt(n, w_gate_up, threads)
+    act = silu_mul(gu, threads)
+    d = gemm_nt(act, w_down, threads)
+    ha, _ = as_data(h)
+    if ha.dtype == np.uint16:
+        hd = (ha.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    else:
+        hd = ha.astype(np.float64)
+    return residual_add(hd, d, threads)

@@ -1,0 +1,491 @@
+"""Pins for the float64 CPU oracle: every oracle function is checked against something
+other than itself — closed forms, invariants, special cases that reduce to a library
+routine (torch / scipy in float64), and 50-digit mpmath brute force on tiny inputs.
+
+The paper prints no worked numeric example for any of these segments (it only names the
+segment classes), so there are no paper-printed golden values; the pins are what the
+mathematics fixes.
+"""
+import math
+
+import mpmath as mp
+import numpy as np
+import pytest
+import scipy.special
+import torch
+import torch.nn.functional as F
+
+from oracle import kopref
+
+mp.mp.dps = 50
+RNG = np.random.default_rng(20260930)
+
+
+def f32(a):
+    return np.asarray(a, dtype=np.float32)
+
+
+def to_bf16_bits(a):
+    """fp32 -> bf16 bit patterns through torch (an independent RNE implementation)."""
+    t = torch.from_numpy(np.asarray(a, dtype=np.float32)).to(torch.bfloat16)
+    return t.view(torch.int16).numpy().view(np.uint16).copy()
+
+
+# --------------------------------------------------------------------------- bf16 helpers
+
+def test_bf16_widening_exhaustive_round_trip():
+    bits = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    wide = kopref.bf16_to_f64(bits)
+    via_torch = torch.from_numpy(bits.view(np.int16).copy()).view(torch.bfloat16).to(torch.float64).numpy()
+    finite = np.isfinite(via_torch)
+    assert np.array_equal(wide[finite], via_torch[finite])
+    assert np.array_equal(np.isnan(wide), np.isnan(via_torch))
+    back = kopref.f64_to_bf16_rne(wide)
+    keep = ~np.isnan(wide)
+    assert np.array_equal(back[keep], bits[keep])
+
+
+def test_bf16_rne_ties_and_against_torch():
+    # 1 + 2^-8 lies exactly between 1 (even mantissa) and 1 + 2^-7: ties-to-even gives 1.
+    assert kopref.f64_to_bf16_rne([1.0 + 2.0 ** -8])[0] == 0x3F80
+    # 1 + 3*2^-8 lies between 1+2^-7 (odd) and 1+2^-6 (even): rounds up.
+    assert kopref.f64_to_bf16_rne([1.0 + 3 * 2.0 ** -8])[0] == 0x3F82
+    # just above / below a tie (not representable in fp32: shows there is no double rounding)
+    assert kopref.f64_to_bf16_rne([1.0 + 2.0 ** -8 + 2.0 ** -40])[0] == 0x3F81
+    assert kopref.f64_to_bf16_rne([1.0 + 2.0 ** -8 - 2.0 ** -40])[0] == 0x3F80
+    assert kopref.f64_to_bf16_rne([-0.0])[0] == 0x8000
+    assert kopref.f64_to_bf16_rne([1e40])[0] == 0x7F80
+    v = RNG.standard_normal(4096).astype(np.float32) * np.float32(37.0)
+    assert np.array_equal(kopref.f64_to_bf16_rne(v.astype(np.float64)), to_bf16_bits(v))
+    tiny = (RNG.standard_normal(512) * 1e-39).astype(np.float32)      # bf16 subnormals
+    assert np.array_equal(kopref.f64_to_bf16_rne(tiny.astype(np.float64)), to_bf16_bits(tiny))
+
+
+# --------------------------------------------------------------------------- softmax
+
+def mp_softmax_row(x, b, s):
+    z = [mp.mpf(float(xi)) * mp.mpf(float(s)) + mp.mpf(float(bi)) for xi, bi in zip(x, b)]
+    e = [mp.exp(t) for t in z]
+    S = mp.fsum(e)
+    return [float(t / S) for t in e]
+
+
+def test_softmax_invariants():
+    x = f32(RNG.standard_normal((37, 513)))
+    b = f32(RNG.standard_normal(513) * 0.1)
+    y = kopref.softmax_scale_bias(x, b, 0.125)
+    assert np.all(np.abs(y.sum(axis=1) - 1.0) <= 1e-13)
+    assert np.all((y >= 0.0) & (y <= 1.0))
+    # shift invariance: adding a constant to every bias entry changes nothing
+    y2 = kopref.softmax_scale_bias(x, f32(b + np.float32(3.0)), 0.125)
+    assert np.max(np.abs(y - y2)) <= 1e-7     # b+3 is re-rounded to fp32: not bit-exact
+    # constant row -> exactly uniform; one column -> 1
+    yc = kopref.softmax_scale_bias(f32(np.full((3, 16), 2.5)), None, 0.125)
+    assert np.array_equal(yc, np.full((3, 16), 1.0 / 16))
+    assert np.array_equal(kopref.softmax_scale_bias(f32([[7.0]]), None, 0.125), [[1.0]])
+    # scale 0 and no bias -> uniform whatever x is
+    assert np.array_equal(kopref.softmax_scale_bias(x[:2, :8], None, 0.0), np.full((2, 8), 0.125))
+
+
+def test_softmax_scale_before_bias_and_two_element_closed_form():
+    # z = x*s + b (scale applies to x only): with x=(8,0), s=0.125, b=(0,2): z=(1,2)
+    y = kopref.softmax_scale_bias(f32([[8.0, 0.0]]), f32([0.0, 2.0]), 0.125)
+    assert y[0, 0] == pytest.approx(1.0 / (1.0 + math.e), rel=1e-15)
+    assert y[0, 1] == pytest.approx(math.e / (1.0 + math.e), rel=1e-15)
+
+
+def test_softmax_masked_column_and_all_masked_row():
+    x = f32(RNG.standard_normal((2, 6)))
+    b = f32([0, -np.inf, 0, 0, -np.inf, 0])
+    y = kopref.softmax_scale_bias(x, b, 1.0)
+    assert np.all(y[:, [1, 4]] == 0.0)
+    keep = [0, 2, 3, 5]
+    assert np.allclose(y[:, keep], kopref.softmax_scale_bias(x[:, keep], None, 1.0), rtol=0, atol=1e-16)
+    ynan = kopref.softmax_scale_bias(x, f32([-np.inf] * 6), 1.0)
+    assert np.all(np.isnan(ynan))
+
+
+def test_softmax_matches_library_and_mpmath():
+    x = f32(RNG.standard_normal((5, 8)) * 3)
+    b = f32(RNG.standard_normal(8))
+    y = kopref.softmax_scale_bias(x, b, 0.125)
+    lib = scipy.special.softmax(x.astype(np.float64) * 0.125 + b.astype(np.float64), axis=1)
+    assert np.max(np.abs(y - lib)) <= 1e-15
+    for i in range(5):
+        assert np.max(np.abs(y[i] - np.array(mp_softmax_row(x[i], b, 0.125)))) <= 1e-15
+    # bf16 data path: values are widened exactly
+    xb = to_bf16_bits(x)
+    yb = kopref.softmax_scale_bias(xb, b, 0.125)
+    xw = torch.from_numpy(x).to(torch.bfloat16).to(torch.float64).numpy()
+    assert np.max(np.abs(yb - scipy.special.softmax(xw * 0.125 + b.astype(np.float64), axis=1))) <= 1e-15
+
+
+# --------------------------------------------------------------------------- GELU (tanh form)
+
+def mp_gelu(u):
+    u = mp.mpf(u)
+    return 0.5 * u * (1 + mp.tanh(mp.sqrt(2 / mp.pi) * (u + mp.mpf("0.044715") * u ** 3)))
+
+
+def test_gelu_tanh_points_identity_limits():
+    assert kopref.gelu_tanh(0.0) == 0.0
+    for u in [-6.0, -2.5, -1.0, -0.3, 0.1, 0.5, 1.0, 2.0, 3.7, 8.0]:
+        assert kopref.gelu_tanh(u) == pytest.approx(float(mp_gelu(u)), rel=2e-15, abs=1e-15)  # 1 + tanh cancels near -1
+        # g(u) - g(-u) = u exactly in real arithmetic (tanh is odd)
+        assert kopref.gelu_tanh(u) - kopref.gelu_tanh(-u) == pytest.approx(u, rel=1e-15)
+    assert kopref.gelu_tanh(12.0) == 12.0
+    assert abs(kopref.gelu_tanh(-12.0)) <= 1e-30
+    # library: torch's tanh-approximate GELU in float64
+    u = torch.linspace(-5, 5, 41, dtype=torch.float64)
+    ref = F.gelu(u, approximate="tanh").numpy()
+    got = np.array([kopref.gelu_tanh(float(t)) for t in u])
+    assert np.max(np.abs(got - ref)) <= 1e-15
+
+
+# --------------------------------------------------------------------------- bias+GELU+residual+LayerNorm
+
+def test_layernorm_zero_mean_unit_variance_before_affine():
+    H = 96
+    x = f32(RNG.standard_normal((9, H)))
+    r = f32(RNG.standard_normal((9, H)))
+    b = f32(RNG.standard_normal(H) * 0.1)
+    eps = 1e-5
+    y, mu, rstd = kopref.bias_gelu_residual_layernorm(x, r, b, f32(np.ones(H)), f32(np.zeros(H)), eps)
+    assert np.all(np.abs(y.mean(axis=1)) <= 1e-12)
+    var = 1.0 / rstd ** 2 - eps                       # sigma^2 recovered from rstd
+    assert np.allclose(y.var(axis=1), var / (var + eps), rtol=1e-12, atol=0)
+    # mean output is the mean of v = r + gelu(x + b)
+    v = r.astype(np.float64) + F.gelu(torch.from_numpy(x.astype(np.float64) + b.astype(np.float64)),
+                                      approximate="tanh").numpy()
+    assert np.allclose(mu, v.mean(axis=1), rtol=0, atol=1e-14)
+    assert np.allclose(rstd, 1.0 / np.sqrt(v.var(axis=1) + eps), rtol=1e-13, atol=0)
+
+
+def test_layernorm_closed_forms():
+    # x = 0, bias = 0 -> gelu term vanishes, so v = r: plain LayerNorm of r.
+    H = 64
+    zeros = f32(np.zeros((1, H)))
+    ones, nul = f32(np.ones(H)), f32(np.zeros(H))
+    r = f32(np.arange(H, dtype=np.float64)[None, :])              # arithmetic progression
+    y, mu, rstd = kopref.bias_gelu_residual_layernorm(zeros, r, nul, ones, nul, 1e-5)
+    assert mu[0] == pytest.approx((H - 1) / 2, rel=1e-15)
+    assert rstd[0] == pytest.approx(1.0 / math.sqrt((H * H - 1) / 12.0 + 1e-5), rel=1e-14)
+    # two-element row [-1, 1]: mu = 0, var = 1 -> y = -+ 1/sqrt(1+eps)
+    y2, _, _ = kopref.bias_gelu_residual_layernorm(f32(np.zeros((1, 2))), f32([[-1.0, 1.0]]),
+                                                   f32([0, 0]), f32([1, 1]), f32([0, 0]), 1e-5)
+    assert y2[0, 0] == pytest.approx(-1.0 / math.sqrt(1 + 1e-5), rel=1e-15)
+    assert y2[0, 1] == pytest.approx(+1.0 / math.sqrt(1 + 1e-5), rel=1e-15)
+    # affine step is elementwise: gamma, beta applied per column
+    g = f32(RNG.standard_normal(H))
+    be = f32(RNG.standard_normal(H))
+    ya, _, _ = kopref.bias_gelu_residual_layernorm(zeros, r, nul, g, be, 1e-5)
+    assert np.allclose(ya, y * g.astype(np.float64) + be.astype(np.float64), rtol=1e-14, atol=1e-14)
+
+
+def test_layernorm_op_order_and_library():
+    # distinguishes bias->gelu->residual->LN from any other order: compare with torch float64
+    H = 40
+    x = f32(RNG.standard_normal((6, H)) * 2)
+    r = f32(RNG.standard_normal((6, H)))
+    b = f32(RNG.standard_normal(H))
+    g = f32(1 + 0.02 * RNG.standard_normal(H))
+    be = f32(0.02 * RNG.standard_normal(H))
+    y, mu, rstd = kopref.bias_gelu_residual_layernorm(x, r, b, g, be, 1e-5)
+    tx, tr, tb, tg, tbe = (torch.from_numpy(a.astype(np.float64)) for a in (x, r, b, g, be))
+    v = tr + F.gelu(tx + tb, approximate="tanh")
+    ref = F.layer_norm(v, (H,), tg, tbe, 1e-5).numpy()
+    assert np.max(np.abs(y - ref)) <= 1e-13
+    # bf16 inputs are widened exactly and v is not rounded
+    xb, rb = to_bf16_bits(x), to_bf16_bits(r)
+    yb, _, _ = kopref.bias_gelu_residual_layernorm(xb, rb, b, g, be, 1e-5)
+    txb = torch.from_numpy(x).to(torch.bfloat16).to(torch.float64)
+    trb = torch.from_numpy(r).to(torch.bfloat16).to(torch.float64)
+    refb = F.layer_norm(trb + F.gelu(txb + tb, approximate="tanh"), (H,), tg, tbe, 1e-5).numpy()
+    assert np.max(np.abs(yb - refb)) <= 1e-13
+
+
+def test_layernorm_mpmath_tiny():
+    x = f32([[0.5, -1.25, 2.0, 0.0]])
+    r = f32([[1.0, 0.25, -0.5, 3.0]])
+    b = f32([0.1, -0.2, 0.3, 0.0])
+    g = f32([1.0, 0.5, 2.0, -1.0])
+    be = f32([0.0, 0.1, -0.1, 0.2])
+    y, mu, rstd = kopref.bias_gelu_residual_layernorm(x, r, b, g, be, 1e-5)
+    v = [mp.mpf(float(r[0, j])) + mp_gelu(mp.mpf(float(x[0, j])) + mp.mpf(float(b[j]))) for j in range(4)]
+    m = mp.fsum(v) / 4
+    var = mp.fsum([(t - m) ** 2 for t in v]) / 4
+    rs = 1 / mp.sqrt(var + mp.mpf(1e-5))
+    ref = [float((v[j] - m) * rs * mp.mpf(float(g[j])) + mp.mpf(float(be[j]))) for j in range(4)]
+    assert np.max(np.abs(y[0] - np.array(ref))) <= 1e-14
+    assert mu[0] == pytest.approx(float(m), rel=1e-15)
+    assert rstd[0] == pytest.approx(float(rs), rel=1e-14)
+
+
+def test_welford_chan_merge_equals_two_pass():
+    # The merge formula a single-pass method relies on, checked against the oracle's
+    # two-pass statistics: delta = mu_b - mu_a; mu = mu_a + delta n_b/n;
+    # M2 = M2_a + M2_b + delta^2 n_a n_b / n.
+    H = 200
+    r = f32(RNG.standard_normal((1, H)) * 3 + 5)
+    _, mu, rstd = kopref.bias_gelu_residual_layernorm(f32(np.zeros((1, H))), r, f32(np.zeros(H)),
+                                                     f32(np.ones(H)), f32(np.zeros(H)), 0.0)
+    v = r[0].astype(np.float64)
+    for cut in (1, 37, 100, 199):
+        a, b = v[:cut], v[cut:]
+        na, nb = len(a), len(b)
+        mua, mub = a.mean(), b.mean()
+        M2a, M2b = ((a - mua) ** 2).sum(), ((b - mub) ** 2).sum()
+        d = mub - mua
+        n = na + nb
+        m = mua + d * nb / n
+        M2 = M2a + M2b + d * d * na * nb / n
+        assert m == pytest.approx(mu[0], rel=1e-14)
+        assert 1.0 / math.sqrt(M2 / n) == pytest.approx(rstd[0], rel=1e-13)
+
+
+# --------------------------------------------------------------------------- BN + ReLU + avgpool
+
+def test_bn_relu_avgpool_special_cases():
+    N, Cc, H, W = 2, 3, 5, 4
+    x = f32(RNG.standard_normal((N, Cc, H, W)))
+    one, nul = f32(np.ones(Cc)), f32(np.zeros(Cc))
+    y, p = kopref.bn_relu_avgpool(x, one, nul)
+    assert np.array_equal(y, np.maximum(x.astype(np.float64), 0.0))      # scale 1, shift 0 = ReLU
+    assert np.allclose(p, y.mean(axis=(2, 3)), rtol=1e-15, atol=0)
+    # all-positive plane: pooling is linear, p = scale * mean(x) + shift
+    xp = f32(np.abs(x) + 0.5)
+    sc, sh = f32([0.5, 1.0, 1.5]), f32([0.1, 0.2, 0.3])
+    _, pp = kopref.bn_relu_avgpool(xp, sc, sh)
+    expect = xp.astype(np.float64).mean(axis=(2, 3)) * sc.astype(np.float64) + sh.astype(np.float64)
+    assert np.allclose(pp, expect, rtol=1e-14, atol=0)
+    # all-negative after affine -> zeros
+    yn, pn = kopref.bn_relu_avgpool(f32(-xp), sc, f32(-sh))
+    assert np.all(yn == 0.0) and np.all(pn == 0.0)
+    # constant plane
+    yc, pc = kopref.bn_relu_avgpool(f32(np.full((1, 3, 2, 2), 2.0)), sc, sh)
+    assert np.allclose(pc[0], 2.0 * sc.astype(np.float64) + sh.astype(np.float64), rtol=1e-15)
+    # channel index is the second axis (a transposed-operand mistake fails here)
+    xs = f32(np.ones((2, 3, 2, 2)))
+    _, ps = kopref.bn_relu_avgpool(xs, f32([1, 2, 3]), nul)
+    assert np.array_equal(ps, np.array([[1.0, 2.0, 3.0], [1.0, 2.0, 3.0]]))
+
+
+def test_bn_relu_nan_propagates_and_library():
+    x = f32(RNG.standard_normal((2, 4, 3, 3)))
+    x[0, 1, 1, 1] = np.nan
+    sc = f32(RNG.uniform(0.5, 1.5, 4))
+    sh = f32(RNG.standard_normal(4) * 0.1)
+    y, p = kopref.bn_relu_avgpool(x, sc, sh)
+    assert np.isnan(y[0, 1, 1, 1]) and np.isnan(p[0, 1])
+    assert not np.isnan(p[1]).any()
+    # library: eval-mode batch_norm with mean 0 / var 1-eps folded, then relu, then adaptive pool
+    xc = torch.from_numpy(np.nan_to_num(x).astype(np.float64))
+    ref_y = F.relu(xc * torch.from_numpy(sc.astype(np.float64))[None, :, None, None]
+                   + torch.from_numpy(sh.astype(np.float64))[None, :, None, None])
+    ref_p = F.adaptive_avg_pool2d(ref_y, 1)[:, :, 0, 0].numpy()
+    yy, ppp = kopref.bn_relu_avgpool(np.nan_to_num(x), sc, sh)
+    assert np.max(np.abs(yy - ref_y.numpy())) <= 1e-15
+    assert np.max(np.abs(ppp - ref_p)) <= 1e-15
+
+
+# --------------------------------------------------------------------------- cross-entropy
+
+def test_ce_closed_forms():
+    V = 32000
+    z = f32(np.full((3, V), -1.75))
+    loss, mean, bad = kopref.ce_loss_rowwise(z, np.array([0, 17, V - 1], dtype=np.int32))
+    assert np.all(np.abs(loss - math.log(V)) <= 1e-12)                  # uniform row -> ln V
+    assert mean == pytest.approx(math.log(V), rel=1e-14) and bad == 0
+    # two classes: loss = log1p(exp(z_other - z_label))
+    z2 = f32([[1.5, -0.25], [1.5, -0.25]])
+    l2, m2, _ = kopref.ce_loss_rowwise(z2, np.array([0, 1], dtype=np.int32))
+    assert l2[0] == pytest.approx(math.log1p(math.exp(-1.75)), rel=1e-14)
+    assert l2[1] == pytest.approx(math.log1p(math.exp(+1.75)), rel=1e-14)
+    assert m2 == pytest.approx((l2[0] + l2[1]) / 2, rel=1e-15)          # mean divides by M
+
+
+def test_ce_invariants_and_library():
+    M, V = 11, 257
+    z = f32(RNG.standard_normal((M, V)) * 2)
+    lab = RNG.integers(0, V, M).astype(np.int32)
+    loss, mean, bad = kopref.ce_loss_rowwise(z, lab)
+    assert np.all(loss >= 0) and bad == 0
+    # loss = logsumexp - label logit
+    lse = scipy.special.logsumexp(z.astype(np.float64), axis=1)
+    assert np.allclose(loss, lse - z[np.arange(M), lab].astype(np.float64), rtol=0, atol=1e-13)
+    # library
+    ref = F.cross_entropy(torch.from_numpy(z.astype(np.float64)), torch.from_numpy(lab.astype(np.int64)),
+                          reduction="none").numpy()
+    assert np.max(np.abs(loss - ref)) <= 1e-13
+    assert mean == pytest.approx(ref.mean(), rel=1e-14)
+    # sum over all possible labels of exp(-loss) is 1 (the softmax is a distribution)
+    row = np.repeat(z[:1], V, axis=0)
+    lall, _, _ = kopref.ce_loss_rowwise(row, np.arange(V, dtype=np.int32))
+    assert abs(np.exp(-lall).sum() - 1.0) <= 1e-13
+    # shift invariance (power-of-two shift keeps fp32 exact enough: use exact small ints)
+    zi = f32(RNG.integers(-8, 8, (4, 33)))
+    li = RNG.integers(0, 33, 4).astype(np.int32)
+    a, _, _ = kopref.ce_loss_rowwise(zi, li)
+    b, _, _ = kopref.ce_loss_rowwise(f32(zi + 100.0), li)
+    assert np.max(np.abs(a - b)) <= 1e-12
+    # large logits do not overflow (max subtraction)
+    big, _, _ = kopref.ce_loss_rowwise(f32([[1000.0, 999.0]]), np.array([1], dtype=np.int32))
+    assert big[0] == pytest.approx(math.log1p(math.exp(-1.0)) + 1.0, rel=1e-14)
+
+
+def test_ce_online_merge_equals_two_pass_and_mpmath():
+    V = 300
+    z = f32(RNG.standard_normal((1, V)) * 4)
+    lab = np.array([123], dtype=np.int32)
+    loss, _, _ = kopref.ce_loss_rowwise(z, lab)
+    zz = z[0].astype(np.float64)
+    for cut in (1, 64, 299):
+        # (m, s) (+) (m', s') = (max, s e^{m - max} + s' e^{m' - max})
+        ma, mb = zz[:cut].max(), zz[cut:].max()
+        sa, sb = np.exp(zz[:cut] - ma).sum(), np.exp(zz[cut:] - mb).sum()
+        m = max(ma, mb)
+        s = sa * math.exp(ma - m) + sb * math.exp(mb - m)
+        assert m + math.log(s) - zz[123] == pytest.approx(loss[0], rel=1e-13)
+    ref = mp.log(mp.fsum([mp.exp(mp.mpf(float(t))) for t in z[0]])) - mp.mpf(float(z[0, 123]))
+    assert loss[0] == pytest.approx(float(ref), rel=1e-14)
+
+
+def test_ce_bad_labels_and_bf16():
+    z = f32(RNG.standard_normal((4, 10)))
+    loss, mean, bad = kopref.ce_loss_rowwise(z, np.array([0, -1, 10, 9], dtype=np.int32))
+    assert bad == 2 and np.isnan(loss[1]) and np.isnan(loss[2]) and np.isnan(mean)
+    assert np.isfinite(loss[0]) and np.isfinite(loss[3])
+    zb = to_bf16_bits(z)
+    lb, _, _ = kopref.ce_loss_rowwise(zb, np.array([0, 1, 2, 3], dtype=np.int32))
+    zw = torch.from_numpy(z).to(torch.bfloat16).to(torch.float64)
+    ref = F.cross_entropy(zw, torch.tensor([0, 1, 2, 3]), reduction="none").numpy()
+    assert np.max(np.abs(lb - ref)) <= 1e-14
+
+
+# --------------------------------------------------------------------------- RMSNorm
+
+def test_rmsnorm_closed_forms_and_library():
+    H = 48
+    one = f32(np.ones(H))
+    eps = 1e-6
+    x = f32(RNG.standard_normal((7, H)))
+    y = kopref.rmsnorm(x, one, eps)
+    ms = (x.astype(np.float64) ** 2).mean(axis=1)
+    assert np.allclose((y ** 2).mean(axis=1), ms / (ms + eps), rtol=1e-13, atol=0)
+    c = 3.0
+    yc = kopref.rmsnorm(f32(np.full((1, H), c)), one, eps)
+    assert np.allclose(yc, c / math.sqrt(c * c + eps), rtol=1e-15, atol=0)
+    alt = f32([[1.0, -1.0] * (H // 2)])
+    ya = kopref.rmsnorm(alt, one, eps)
+    assert np.allclose(ya, alt.astype(np.float64) / math.sqrt(1 + eps), rtol=1e-15, atol=0)
+    # f(a x) = sign(a) f(x) when eps = 0
+    y0 = kopref.rmsnorm(x, one, 0.0)
+    ym = kopref.rmsnorm(f32(x * np.float32(-4.0)), one, 0.0)
+    assert np.allclose(ym, -y0, rtol=1e-14, atol=0)
+    # weight is applied per column; library rms_norm in float64
+    w = f32(1 + 0.02 * RNG.standard_normal(H))
+    yw = kopref.rmsnorm(x, w, eps)
+    ref = F.rms_norm(torch.from_numpy(x.astype(np.float64)), (H,),
+                     torch.from_numpy(w.astype(np.float64)), eps).numpy()
+    assert np.max(np.abs(yw - ref)) <= 1e-14
+    # mpmath on one row
+    row = x[0]
+    msq = mp.fsum([mp.mpf(float(t)) ** 2 for t in row]) / H
+    refm = [float(mp.mpf(float(row[j])) / mp.sqrt(msq + mp.mpf(eps)) * mp.mpf(float(w[j]))) for j in range(H)]
+    assert np.max(np.abs(yw[0] - np.array(refm))) <= 1e-14
+
+
+# --------------------------------------------------------------------------- SiLU * up, residual add
+
+def test_silu_mul_identities_layout_library():
+    inter = 6
+    g = f32(RNG.standard_normal((3, inter)) * 3)
+    u = f32(RNG.standard_normal((3, inter)))
+    gu = np.concatenate([g, u], axis=1)                         # [gate | up] halves
+    out = kopref.silu_mul(gu)
+    ref = (F.silu(torch.from_numpy(g.astype(np.float64))) * torch.from_numpy(u.astype(np.float64))).numpy()
+    assert np.max(np.abs(out - ref)) <= 1e-15
+    # up = 1 -> silu(gate); silu(0) = 0; silu(g) - silu(-g) = g
+    ones = f32(np.ones((3, inter)))
+    s_pos = kopref.silu_mul(np.concatenate([g, ones], axis=1))
+    s_neg = kopref.silu_mul(np.concatenate([-g, ones], axis=1))
+    assert np.allclose(s_pos - s_neg, g.astype(np.float64), rtol=1e-14, atol=1e-15)
+    assert kopref.silu_mul(f32([[0.0, 5.0]]))[0, 0] == 0.0
+    # large gate -> gate * up
+    big = kopref.silu_mul(f32([[40.0, 0.5]]))
+    assert big[0, 0] == pytest.approx(20.0, rel=1e-15)
+    # swapping the halves changes the answer (SiLU applies to the first half)
+    assert np.max(np.abs(kopref.silu_mul(np.concatenate([u, g], axis=1)) - out)) > 1e-3
+    for gv, uv in [(0.5, 2.0), (-3.0, 1.5), (7.25, -0.125)]:
+        refm = mp.mpf(gv) / (1 + mp.exp(-mp.mpf(gv))) * mp.mpf(uv)
+        assert kopref.silu_mul(f32([[gv, uv]]))[0, 0] == pytest.approx(float(refm), rel=1e-15)
+
+
+def test_residual_add_exact():
+    a = f32(RNG.standard_normal((5, 9)))
+    b = f32(RNG.standard_normal((5, 9)))
+    assert np.array_equal(kopref.residual_add(a, b), a.astype(np.float64) + b.astype(np.float64))
+    ab, bb = to_bf16_bits(a), to_bf16_bits(b)
+    wa = torch.from_numpy(a).to(torch.bfloat16).to(torch.float64).numpy()
+    wb = torch.from_numpy(b).to(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(kopref.residual_add(ab, bb), wa + wb)
+
+
+# --------------------------------------------------------------------------- GEMM helper and the chain
+
+def test_gemm_nt_exact_cases():
+    M, K, N = 4, 6, 5
+    A = f32(RNG.integers(-5, 6, (M, K)))
+    Wm = f32(RNG.integers(-5, 6, (N, K)))
+    Cm = kopref.gemm_nt(A, Wm)
+    assert np.array_equal(Cm, A.astype(np.float64) @ Wm.astype(np.float64).T)   # small ints: exact
+    eye = f32(np.eye(K))
+    assert np.array_equal(kopref.gemm_nt(A, eye), A.astype(np.float64))
+    perm = f32(np.eye(K)[[2, 0, 1, 5, 4, 3]])           # row n of W selects column perm[n] of A
+    assert np.array_equal(kopref.gemm_nt(A, perm), A.astype(np.float64)[:, [2, 0, 1, 5, 4, 3]])
+    Ar = RNG.standard_normal((M, K))
+    Wr = RNG.standard_normal((N, K))
+    assert np.allclose(kopref.gemm_nt(Ar, Wr), Ar @ Wr.T, rtol=1e-14, atol=1e-14)
+
+
+def test_mlp_chain_selector_weights_collapse_to_elementwise():
+    # W1 = [I; I] (gate and up both copy the normed row), W2 = I:
+    # out_j = h_j + silu(n_j) * n_j with n = rmsnorm(h).
+    Hd = 16
+    h = f32(RNG.standard_normal((5, Hd)))
+    w = f32(1 + 0.02 * RNG.standard_normal(Hd))
+    W1 = f32(np.concatenate([np.eye(Hd), np.eye(Hd)], axis=0))
+    W2 = f32(np.eye(Hd))
+    out = kopref.mlp_segment(h, w, W1, W2, 1e-6)
+    hd = h.astype(np.float64)
+    n = hd / np.sqrt((hd ** 2).mean(axis=1, keepdims=True) + 1e-6) * w.astype(np.float64)
+    assert np.allclose(out, hd + n / (1 + np.exp(-n)) * n, rtol=1e-13, atol=1e-14)
+
+
+def test_mlp_chain_reduced_shape_vs_numpy():
+    M, Hd, I = 12, 32, 56
+    h = to_bf16_bits(RNG.standard_normal((M, Hd)))
+    w = f32(1 + 0.02 * RNG.standard_normal(Hd))
+    W1 = to_bf16_bits(RNG.standard_normal((2 * I, Hd)) * 0.02)
+    W2 = to_bf16_bits(RNG.standard_normal((Hd, I)) * 0.02)
+    out = kopref.mlp_segment(h, w, W1, W2, 1e-6)
+
+    def wide(bits):
+        return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    hd, W1d, W2d = wide(h), wide(W1), wide(W2)
+    n = hd / np.sqrt((hd ** 2).mean(axis=1, keepdims=True) + 1e-6) * w.astype(np.float64)
+    gu = n @ W1d.T
+    act = gu[:, :I] / (1 + np.exp(-gu[:, :I])) * gu[:, I:]
+    ref = hd + act @ W2d.T
+    assert np.allclose(out, ref, rtol=1e-12, atol=1e-14)
+
+
+def test_threads_do_not_change_results():
+    x = f32(RNG.standard_normal((64, 100)))
+    b = f32(RNG.standard_normal(100))
+    assert np.array_equal(kopref.softmax_scale_bias(x, b, 0.125, threads=1),
+                          kopref.softmax_scale_bias(x, b, 0.125, threads=4))
+    lab = RNG.integers(0, 100, 64).astype(np.int32)
+    l1, m1, _ = kopref.ce_loss_rowwise(x, lab, threads=1)
+    l4, m4, _ = kopref.ce_loss_rowwise(x, lab, threads=4)
+    assert np.array_equal(l1, l4) and m1 == m4
