@@ -1,0 +1,220 @@
+/*
+ * libkop — fused pointwise+reduction segments for NVIDIA B200 (sm_100a), C ABI.
+ *
+ * These are the memory-bound sub-kernels a model compiler emits between vendor
+ * GEMM / convolution calls: bias / scale / activation / residual chains that end in a
+ * row- or channel-wise reduction. The paper's problem formulation (Definition 1)
+ * keeps the vendor calls fixed and speeds up exactly these sub-kernels; its fusion
+ * agent's technique list and planner strategies 8-9 name the classes implemented
+ * here (fused softmax, single-pass LayerNorm / RMSNorm, activation + bias fusion,
+ * residual + norm, reduction + pointwise, LogSumExp reductions). The paper never
+ * prints their formulas; each entry point below states the one it computes.
+ *
+ * Conventions shared by every entry point
+ *   pointers   All data / parameter / output / workspace pointers are DEVICE pointers
+ *              on the current device, owned by the caller. Shape arrays passed by
+ *              pointer (strides of kop_bn_relu_avgpool) are HOST pointers.
+ *   dtype      `dtype` is the element type of the data tensors (inputs and the main
+ *              output): KOP_F32 or KOP_BF16. Parameter vectors (bias, gamma, beta,
+ *              scale, shift, weight) and statistics outputs (mean, rstd, pooled,
+ *              loss) are always fp32. All arithmetic is fp32; the only rounding to
+ *              bf16 is the final store (round to nearest even), as the paper's
+ *              numerics rule requires (accumulate in fp32, cast only at the store).
+ *   strides    In elements. The innermost stride is 1 by contract; a row stride
+ *              must be >= the row length.
+ *   alignment  16-byte-aligned bases, row strides and row lengths take the 128-bit
+ *              vector kernels; anything else runs a scalar-load GPU kernel of the
+ *              same arithmetic. There is no CPU path.
+ *   aliasing   Where stated, the output may be exactly the input (same pointer and
+ *              stride). Any other overlap returns KOP_ERR_BAD_ALIAS when detectable
+ *              and is undefined otherwise.
+ *   stream     Work is enqueued on `stream`; nothing synchronises, allocates or frees,
+ *              and the library keeps no state between calls (kop_mlp_handle_* aside,
+ *              which only wrap cuBLAS handle creation).
+ *   errors     Static validation (the paper's Gate 1: structural checks before any
+ *              numerics) runs first and touches no CUDA API: a call that fails
+ *              validation launches nothing. rows == 0 (or N == 0) returns KOP_OK
+ *              without a launch. Launch failures are reported as KOP_ERR_CUDA.
+ *              Device code never traps or asserts.
+ */
+#ifndef KOP_H_
+#define KOP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Same type as the CUDA runtime's cudaStream_t (a pointer to CUstream_st). */
+typedef struct CUstream_st* kop_stream_t;
+
+typedef enum {
+    KOP_OK = 0,
+    KOP_ERR_NULL_POINTER = 1,
+    KOP_ERR_BAD_SHAPE = 2,
+    KOP_ERR_BAD_STRIDE = 3,
+    KOP_ERR_UNSUPPORTED_DTYPE = 4,
+    KOP_ERR_MISALIGNED = 5,
+    KOP_ERR_BAD_ALIAS = 6,
+    KOP_ERR_WORKSPACE_TOO_SMALL = 7,
+    KOP_ERR_UNSUPPORTED_DEVICE = 8,
+    KOP_ERR_CUDA = 9,
+    KOP_ERR_CUBLAS = 10
+} kop_status_t;
+
+typedef enum { KOP_F32 = 0, KOP_BF16 = 1 } kop_dtype_t;
+
+/* Library version as major * 10000 + minor * 100 + patch. */
+int kop_version(void);
+
+/* Static, NUL-terminated name of a status code ("KOP_OK", ...); never NULL. */
+const char* kop_status_string(kop_status_t status);
+
+/*
+ * Row softmax of a scaled, biased matrix ("fused softmax", planner strategy 9):
+ *   z[i,j] = x[i,j] * scale + bias[j];  y[i,j] = exp(z[i,j] - max_j z) / sum_j exp(z[i,j] - max_j z)
+ * x, y: [rows, cols] of `dtype`, row strides x_row_stride / y_row_stride.
+ * bias: fp32 [cols], or NULL for no bias; -inf entries mask a column (output 0);
+ *       a row whose z are all -inf yields NaN (the definition's 0/0).
+ * y may alias x exactly. Element size must divide the alignment of x / y
+ * (else KOP_ERR_MISALIGNED).
+ */
+kop_status_t kop_softmax_scale_bias(const void* x, const float* bias, void* y,
+                                    int64_t rows, int64_t cols,
+                                    int64_t x_row_stride, int64_t y_row_stride,
+                                    float scale, kop_dtype_t dtype, kop_stream_t stream);
+
+/*
+ * Bias-add, tanh-form GELU, residual add and LayerNorm in one pass (fusion agent:
+ * "activation + bias fusion" and "residual + norm: one kernel, one memory pass";
+ * codegen agent: "single-pass LayerNorm instead of 3 kernels"):
+ *   u = x + bias;  g = 0.5 u (1 + tanh(sqrt(2/pi) (u + 0.044715 u^3)));  v = residual + g
+ *   mu = mean_j v;  var = mean_j (v - mu)^2 (biased);  r = 1 / sqrt(var + eps)
+ *   y = (v - mu) * r * gamma + beta;   mean[i] = mu;  rstd[i] = r
+ * x, residual, y: [rows, hidden] of `dtype`; bias, gamma, beta: fp32 [hidden];
+ * mean, rstd: fp32 [rows], each may be NULL. v is kept in fp32 (never rounded).
+ * y may alias x or residual exactly.
+ */
+kop_status_t kop_bias_gelu_residual_layernorm(const void* x, const void* residual,
+                                              const float* bias, const float* gamma,
+                                              const float* beta, void* y,
+                                              float* mean, float* rstd,
+                                              int64_t rows, int64_t hidden,
+                                              int64_t x_row_stride, int64_t res_row_stride,
+                                              int64_t y_row_stride, float eps,
+                                              kop_dtype_t dtype, kop_stream_t stream);
+
+/*
+ * Inference BatchNorm (pre-folded per-channel affine), ReLU and global average pool
+ * (fusion agent: "reduction + pointwise"; the BN / pooling epilogues of the paper's
+ * CNN models, next to preserved cuDNN convolutions):
+ *   a[n,c,h,w] = max(x[n,c,h,w] * scale[c] + shift[c], 0)   (NaN stays NaN)
+ *   pooled[n,c] = (1 / (H W)) sum_{h,w} a[n,c,h,w]          (sum of unrounded fp32 a)
+ * x, y: NCHW of `dtype`; x_strides / y_strides are HOST arrays of 4 element strides
+ * and must describe a contiguous NCHW tensor ({C*H*W, H*W, W, 1}), anything else
+ * returns KOP_ERR_BAD_STRIDE. scale, shift: fp32 [C]; pooled: fp32 [N, C].
+ * y may alias x exactly.
+ */
+kop_status_t kop_bn_relu_avgpool(const void* x, const float* scale, const float* shift,
+                                 void* y, float* pooled,
+                                 int64_t N, int64_t C, int64_t H, int64_t W,
+                                 const int64_t x_strides[4], const int64_t y_strides[4],
+                                 kop_dtype_t dtype, kop_stream_t stream);
+
+/*
+ * Row-wise cross-entropy in a single pass over the logits ("LogSumExp reductions";
+ * planner strategy 8 "single-pass reductions"; "online softmax"):
+ *   loss[i] = ln sum_j exp(z[i,j]) - z[i, labels[i]];   *mean_loss = (1/rows) sum_i loss[i]
+ * logits: [rows, vocab] of `dtype`, row stride row_stride; labels: int32 [rows];
+ * loss: fp32 [rows]; mean_loss: fp32 [1] or NULL; bad_label_count: int32 [1] or NULL.
+ * A label outside [0, vocab) gives loss NaN for that row and is counted in
+ * *bad_label_count (then *mean_loss is NaN). The mean is summed in a fixed order:
+ * results are bit-identical run to run.
+ * workspace: device scratch of at least kop_ce_loss_rowwise_workspace_bytes() bytes,
+ * 16-byte aligned, contents irrelevant on entry (the call clears what it needs on
+ * `stream`); calls sharing one workspace must not overlap on the GPU.
+ */
+kop_status_t kop_ce_loss_rowwise(const void* logits, const int32_t* labels,
+                                 float* loss, float* mean_loss, int32_t* bad_label_count,
+                                 int64_t rows, int64_t vocab, int64_t row_stride,
+                                 void* workspace, size_t workspace_bytes,
+                                 kop_dtype_t dtype, kop_stream_t stream);
+
+/* Scratch bytes kop_ce_loss_rowwise needs for this shape (0 on invalid arguments). */
+size_t kop_ce_loss_rowwise_workspace_bytes(int64_t rows, int64_t vocab, kop_dtype_t dtype);
+
+/*
+ * RMSNorm (fusion agent: "normalization fusion (LayerNorm/RMSNorm sequences)"):
+ *   y[i,j] = x[i,j] / sqrt(mean_j x[i,j]^2 + eps) * weight[j]
+ * x, y: [rows, hidden] of `dtype`; weight: fp32 [hidden]. y may alias x exactly.
+ */
+kop_status_t kop_rmsnorm(const void* x, const float* weight, void* y,
+                         int64_t rows, int64_t hidden,
+                         int64_t x_row_stride, int64_t y_row_stride,
+                         float eps, kop_dtype_t dtype, kop_stream_t stream);
+
+/*
+ * SwiGLU epilogue of a preserved GEMM (fusion agent: "activation fusion
+ * (GELU/SiLU/ReLU)"; codegen agent: keep the matmul as a library call and fuse only
+ * the epilogue):
+ *   out[i,j] = gate / (1 + exp(-gate)) * up,  gate = gate_up[i,j],  up = gate_up[i, inter + j]
+ * gate_up: [rows, 2*inter] of `dtype` (two contiguous halves per row), row stride
+ * in_row_stride; out: [rows, inter], row stride out_row_stride. No aliasing.
+ */
+kop_status_t kop_silu_mul(const void* gate_up, void* out, int64_t rows, int64_t inter,
+                          int64_t in_row_stride, int64_t out_row_stride,
+                          kop_dtype_t dtype, kop_stream_t stream);
+
+/*
+ * Residual add (fusion agent: "pointwise + pointwise: load once, store once"):
+ *   out[i,j] = a[i,j] + b[i,j]
+ * a, b, out: [rows, cols] of `dtype`. out may alias a or b exactly.
+ */
+kop_status_t kop_residual_add(const void* a, const void* b, void* out,
+                              int64_t rows, int64_t cols,
+                              int64_t a_row_stride, int64_t b_row_stride,
+                              int64_t out_row_stride, kop_dtype_t dtype, kop_stream_t stream);
+
+/*
+ * Transformer MLP segment with the vendor GEMMs preserved between the fused kernels
+ * (problem formulation: extern library calls stay fixed; codegen agent: "do not
+ * replace cuBLAS"): five operations enqueued on `stream`,
+ *   n = rmsnorm(h; rms_weight, eps)            kop_rmsnorm
+ *   gu = n * w_gate_up^T                       cuBLAS, [rows, 2*inter]
+ *   act = silu(gu[:, :inter]) * gu[:, inter:]  kop_silu_mul
+ *   d = act * w_down^T                         cuBLAS, [rows, hidden]
+ *   out = h + d                                kop_residual_add
+ * h, out: [rows, hidden] contiguous; w_gate_up: [2*inter, hidden]; w_down:
+ * [hidden, inter], both row-major (out_features, in_features), all of `dtype`;
+ * rms_weight: fp32 [hidden]. GEMMs accumulate in fp32 and store `dtype`.
+ * handle: from kop_mlp_handle_create, used by one call at a time.
+ * workspace: device scratch of at least kop_rmsnorm_swiglu_residual_workspace_bytes()
+ * bytes, 256-byte aligned; holds n, gu, act, d and the cuBLAS workspace, so the call
+ * allocates nothing and can be captured into a CUDA graph. out may alias h exactly.
+ */
+kop_status_t kop_rmsnorm_swiglu_residual(void* handle, const void* h, const float* rms_weight,
+                                         const void* w_gate_up, const void* w_down, void* out,
+                                         int64_t rows, int64_t hidden, int64_t inter, float eps,
+                                         void* workspace, size_t workspace_bytes,
+                                         kop_dtype_t dtype, kop_stream_t stream);
+
+/* Scratch bytes kop_rmsnorm_swiglu_residual needs (0 on invalid arguments). */
+size_t kop_rmsnorm_swiglu_residual_workspace_bytes(int64_t rows, int64_t hidden, int64_t inter,
+                                                   kop_dtype_t dtype);
+
+/*
+ * Create / destroy the vendor-GEMM handle used by kop_rmsnorm_swiglu_residual (a
+ * cuBLAS handle made by the same cuBLAS this library is linked against, on the current
+ * device). Creation allocates; do it outside stream capture. (Part of the preserved
+ * vendor-call boundary; the paper has no counterpart beyond "extern_kernels".)
+ */
+kop_status_t kop_mlp_handle_create(void** handle);
+kop_status_t kop_mlp_handle_destroy(void* handle);
+
+#ifdef __cplusplus
+}
+#endif
+
+#endif /* KOP_H_ */

@@ -1,0 +1,210 @@
+// kop_ce_loss_rowwise: loss[i] = logsumexp_j z[i,j] - z[i, label_i] and the mean over rows, with a
+// single pass over the logits.
+//
+// One CTA streams one row. Each thread pulls a batch of 16-byte vectors into registers (all loads
+// issued before first use), takes the batch maximum on the packed values, and then adds
+// 2^(z*log2e - M) for every element with M the thread's running offset (the online-softmax
+// recurrence, applied once per batch rather than once per element: one ex2 per element). The
+// per-thread (M, S) pairs are merged across the CTA, lse = (M + log2 S) * ln 2, and thread 0
+// subtracts the label logit. The last CTA to finish (a ticket counter in the workspace; nobody
+// waits on it) sums loss[] in a fixed order, so the mean is bit-identical run to run.
+#include "kop_common.cuh"
+
+namespace kop {
+namespace {
+
+struct CeWorkspace {
+    unsigned int ticket;
+    unsigned int pad[3];
+};
+
+template <typename T>
+__device__ __forceinline__ float vec_max(const Vec16& v);
+
+template <>
+__device__ __forceinline__ float vec_max<float>(const Vec16& v)
+{
+    return fmaxf(fmaxf(__uint_as_float(v.w[0]), __uint_as_float(v.w[1])),
+                 fmaxf(__uint_as_float(v.w[2]), __uint_as_float(v.w[3])));
+}
+template <>
+__device__ __forceinline__ float vec_max<__nv_bfloat16>(const Vec16& v)
+{
+    // max.bf16x2: two elements per instruction.
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(v.w);
+    const __nv_bfloat162 m = __hmax2(__hmax2(h[0], h[1]), __hmax2(h[2], h[3]));
+    return fmaxf(__low2float(m), __high2float(m));
+}
+
+// Merge the per-thread (M, S) pairs, finish the row, and let the last CTA reduce the mean.
+template <typename T>
+__device__ __forceinline__ void ce_finish(float M, float S, const T* zr, const int32_t* labels,
+                                          float* loss, float* mean_loss, int32_t* bad_label_count,
+                                          CeWorkspace* ws, int64_t row, int64_t rows, int64_t vocab)
+{
+    __shared__ float red_a[32], red_b[32], red_c[32];
+    __shared__ int is_last, bad_total;
+    const float Mb = block_max(M, red_a);
+    // A thread that saw nothing has M = -inf and S = 0; keep its term at 0 rather than 0 * 2^nan.
+    const float Sb = block_sum(M == -INFINITY ? 0.0f : S * ex2_approx(M - Mb), red_b);
+    if (threadIdx.x == 0) {
+        const float lse = (Mb + log2f(Sb)) * kLn2;
+        const int32_t lab = labels[row];
+        float l;
+        if (lab < 0 || (int64_t)lab >= vocab) l = __int_as_float(0x7FC00000);
+        else l = lse - Elem<T>::load1(zr + lab);
+        loss[row] = l;
+        __threadfence();
+        const unsigned t = atomicAdd(&ws->ticket, 1u);
+        is_last = (t == gridDim.x - 1);
+        bad_total = 0;
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    float acc = 0.0f;
+    int bad = 0;
+    for (int64_t i = threadIdx.x; i < rows; i += blockDim.x) {
+        acc += __ldcg(loss + i);
+        const int32_t lab = __ldg(labels + i);
+        bad += (lab < 0 || (int64_t)lab >= vocab) ? 1 : 0;
+    }
+    if (bad != 0) atomicAdd(&bad_total, bad);           // integer: order does not matter
+    acc = block_sum(acc, red_c);                        // contains the barrier bad_total needs
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        if (mean_loss != nullptr) *mean_loss = acc / (float)rows;
+        if (bad_label_count != nullptr) *bad_label_count = bad_total;
+        ws->ticket = 0;
+    }
+}
+
+template <typename T, int VPT>
+__global__ void __launch_bounds__(512)
+ce_row_kernel(const T* __restrict__ z, const int32_t* __restrict__ labels, float* __restrict__ loss,
+              float* __restrict__ mean_loss, int32_t* __restrict__ bad_label_count,
+              CeWorkspace* __restrict__ ws, int64_t rows, int nvec, int64_t row_stride, int64_t vocab)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    const int64_t row = blockIdx.x;
+    const T* zr = z + row * row_stride;
+    float M = -INFINITY, S = 0.0f;
+    for (int base = 0; base < nvec; base += VPT * blockDim.x) {
+        Vec16 raw[VPT];
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            const int v = base + k * blockDim.x + threadIdx.x;
+            raw[k] = Elem<T>::fill_neg_inf();
+            if (v < nvec) raw[k] = ld_stream(zr + (int64_t)v * E);
+        }
+        float cm = vec_max<T>(raw[0]);
+#pragma unroll
+        for (int k = 1; k < VPT; ++k) cm = fmaxf(cm, vec_max<T>(raw[k]));
+        const float cm2 = cm * kLog2e;
+        if (cm2 > -INFINITY) {
+            const float newM = fmaxf(M, cm2);
+            float s = S * ex2_approx(M - newM);          // M = -inf on the first batch: S * 0
+            const float neg = -newM;
+#pragma unroll
+            for (int k = 0; k < VPT; ++k) {
+                float f[E];
+                Elem<T>::unpack(raw[k], f);
+#pragma unroll
+                for (int e = 0; e < E; ++e) s += ex2_approx(fmaf(f[e], kLog2e, neg));
+            }
+            S = s;
+            M = newM;
+        }
+    }
+    ce_finish<T>(M, S, zr, labels, loss, mean_loss, bad_label_count, ws, row, rows, vocab);
+}
+
+// Any vocab / alignment: scalar loads, element-wise online recurrence.
+template <typename T>
+__global__ void __launch_bounds__(256)
+ce_row_scalar_kernel(const T* __restrict__ z, const int32_t* __restrict__ labels,
+                     float* __restrict__ loss, float* __restrict__ mean_loss,
+                     int32_t* __restrict__ bad_label_count, CeWorkspace* __restrict__ ws,
+                     int64_t rows, int64_t row_stride, int64_t vocab)
+{
+    const int64_t row = blockIdx.x;
+    const T* zr = z + row * row_stride;
+    float M = -INFINITY, S = 0.0f;
+    for (int64_t j = threadIdx.x; j < vocab; j += blockDim.x) {
+        const float x2 = Elem<T>::load1(zr + j) * kLog2e;
+        if (x2 == -INFINITY) continue;
+        if (x2 > M) {
+            S = S * ex2_approx(M - x2) + 1.0f;
+            M = x2;
+        } else {
+            S += ex2_approx(x2 - M);
+        }
+    }
+    ce_finish<T>(M, S, zr, labels, loss, mean_loss, bad_label_count, ws, row, rows, vocab);
+}
+
+template <typename T>
+kop_status_t launch_ce(const void* zv, const int32_t* labels, float* loss, float* mean_loss,
+                       int32_t* bad, int64_t rows, int64_t vocab, int64_t stride, void* workspace,
+                       cudaStream_t stream)
+{
+    const T* z = static_cast<const T*>(zv);
+    constexpr int E = Elem<T>::kPerVec;
+    CeWorkspace* ws = static_cast<CeWorkspace*>(workspace);
+    if (cudaMemsetAsync(ws, 0, sizeof(CeWorkspace), stream) != cudaSuccess) return KOP_ERR_CUDA;
+    const bool vec = vec_ok(z, vocab, stride, sizeof(T));
+    const int64_t nvec64 = vocab / E;
+    if (vec && nvec64 <= 0x7FFFFFFF) {
+        const int nvec = (int)nvec64;
+        const int threads = 256;
+        const int per = (nvec + threads - 1) / threads;
+#define KOP_CE(V) ce_row_kernel<T, V><<<(unsigned)rows, threads, 0, stream>>>(z, labels, loss, mean_loss, bad, ws, rows, nvec, stride, vocab)
+        if (per <= 1) KOP_CE(1);
+        else if (per <= 2) KOP_CE(2);
+        else if (per <= 4) KOP_CE(4);
+        else if (per <= 8) KOP_CE(8);
+        else KOP_CE(16);
+#undef KOP_CE
+        return launch_status();
+    }
+    ce_row_scalar_kernel<T><<<(unsigned)rows, 256, 0, stream>>>(z, labels, loss, mean_loss, bad, ws, rows, stride, vocab);
+    return launch_status();
+}
+
+}  // namespace
+}  // namespace kop
+
+extern "C" size_t kop_ce_loss_rowwise_workspace_bytes(int64_t rows, int64_t vocab, kop_dtype_t dtype)
+{
+    if (rows < 0 || vocab <= 0 || !kop::dtype_ok(dtype)) return 0;
+    return sizeof(kop::CeWorkspace);
+}
+
+extern "C" kop_status_t kop_ce_loss_rowwise(const void* logits, const int32_t* labels, float* loss,
+                                            float* mean_loss, int32_t* bad_label_count, int64_t rows,
+                                            int64_t vocab, int64_t row_stride, void* workspace,
+                                            size_t workspace_bytes, kop_dtype_t dtype,
+                                            kop_stream_t stream)
+{
+    using namespace kop;
+    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    if (!logits || !labels || !loss || !workspace) return KOP_ERR_NULL_POINTER;
+    kop_status_t st = check_rows_cols(rows, vocab);
+    if (st != KOP_OK) return st;
+    if (vocab > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;            // labels are int32
+    if (rows > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;             // one CTA per row
+    if ((st = check_row_stride(row_stride, vocab, rows)) != KOP_OK) return st;
+    const int esz = elem_size(dtype);
+    if (!aligned_to(logits, esz) || !aligned_to(labels, 4) || !aligned_to(loss, 4) ||
+        (mean_loss && !aligned_to(mean_loss, 4)) || (bad_label_count && !aligned_to(bad_label_count, 4)) ||
+        !aligned_to(workspace, 16))
+        return KOP_ERR_MISALIGNED;
+    if (workspace_bytes < kop_ce_loss_rowwise_workspace_bytes(rows, vocab, dtype))
+        return KOP_ERR_WORKSPACE_TOO_SMALL;
+    if (rows == 0) return KOP_OK;
+    if ((st = check_device()) != KOP_OK) return st;
+    cudaStream_t s = as_stream(stream);
+    return dtype == KOP_F32
+               ? launch_ce<float>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s)
+               : launch_ce<__nv_bfloat16>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s);
+}

@@ -1,0 +1,253 @@
+// Shared host validation helpers and device building blocks of libkop (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kop.h"
+
+namespace kop {
+
+// ------------------------------------------------------------------------------------------
+// Host side: static validation (the paper's Gate 1 analogue). Pure integer checks, no CUDA call.
+// ------------------------------------------------------------------------------------------
+
+inline bool dtype_ok(kop_dtype_t d) { return d == KOP_F32 || d == KOP_BF16; }
+inline int elem_size(kop_dtype_t d) { return d == KOP_F32 ? 4 : 2; }
+inline bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// Largest product / offset we accept: keeps every byte offset inside int64.
+constexpr int64_t kMaxElems = (int64_t)1 << 46;
+
+inline kop_status_t check_rows_cols(int64_t rows, int64_t cols)
+{
+    if (rows < 0 || cols <= 0) return KOP_ERR_BAD_SHAPE;
+    if (rows > kMaxElems || cols > kMaxElems) return KOP_ERR_BAD_SHAPE;
+    return KOP_OK;
+}
+
+inline kop_status_t check_row_stride(int64_t stride, int64_t cols, int64_t rows)
+{
+    if (stride < cols) return KOP_ERR_BAD_STRIDE;
+    if (stride > kMaxElems) return KOP_ERR_BAD_STRIDE;
+    // rows * stride must not overflow what we can address
+    if (rows > 0 && stride > kMaxElems / (rows > 0 ? rows : 1)) return KOP_ERR_BAD_SHAPE;
+    return KOP_OK;
+}
+
+// Byte span [lo, hi) touched by a strided 2-D tensor.
+inline void span_of(const void* base, int64_t rows, int64_t cols, int64_t stride, int esz,
+                    uintptr_t* lo, uintptr_t* hi)
+{
+    *lo = reinterpret_cast<uintptr_t>(base);
+    *hi = *lo + (rows > 0 ? (uintptr_t)(((rows - 1) * stride + cols) * esz) : 0);
+}
+
+// Output `out` may be exactly `in` (same base and stride) or disjoint from it.
+inline bool alias_ok(const void* in, int64_t in_stride, const void* out, int64_t out_stride,
+                     int64_t rows, int64_t cols, int esz, bool exact_allowed)
+{
+    if (rows == 0) return true;
+    if (in == out) return exact_allowed && in_stride == out_stride;
+    uintptr_t a0, a1, b0, b1;
+    span_of(in, rows, cols, in_stride, esz, &a0, &a1);
+    span_of(out, rows, cols, out_stride, esz, &b0, &b1);
+    return a1 <= b0 || b1 <= a0;
+}
+
+// True when a [rows, cols] tensor can be read with 16-byte vectors row by row.
+inline bool vec_ok(const void* base, int64_t cols, int64_t stride, int esz)
+{
+    const int per = 16 / esz;
+    return aligned_to(base, 16) && (cols % per) == 0 && (stride % per) == 0;
+}
+
+// Checks that the current device is a B200-class part (compute capability 10.x); the library is
+// compiled for sm_100a only. Result is cached per device ordinal.
+kop_status_t check_device();
+
+// SM count of the current device (valid after check_device() succeeded on it; 148 otherwise).
+int sm_count();
+
+// Maps the last launch error (non-sticky peek) to a status.
+inline kop_status_t launch_status()
+{
+    return cudaGetLastError() == cudaSuccess ? KOP_OK : KOP_ERR_CUDA;
+}
+
+inline cudaStream_t as_stream(kop_stream_t s) { return reinterpret_cast<cudaStream_t>(s); }
+
+// ------------------------------------------------------------------------------------------
+// Device side
+// ------------------------------------------------------------------------------------------
+#ifdef __CUDACC__
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// Row-in-registers kernels keep `vals` fp32 values per thread; the CTA size they may be launched
+// with shrinks as that count grows so the row always fits the register file without spills.
+constexpr int max_threads_for(int vals) { return vals <= 16 ? 1024 : (vals <= 32 ? 512 : 256); }
+// Longest row (in elements) a single CTA can hold in registers under max_threads_for().
+constexpr int64_t kMaxRegisterRow = 16384;
+
+struct __align__(16) Vec16 {
+    uint32_t w[4];
+};
+
+// Streaming 128-bit global load: data tensors are touched exactly once, so they bypass L1
+// allocation and leave L1 to the small parameter vectors that every row re-reads.
+// (Not .nc: outputs may alias inputs exactly, so the location is not read-only.)
+__device__ __forceinline__ Vec16 ld_stream(const void* p)
+{
+    Vec16 v;
+    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.w[0]), "=r"(v.w[1]), "=r"(v.w[2]), "=r"(v.w[3])
+                 : "l"(p));
+    return v;
+}
+
+// 128-bit global store of a result that this kernel never reads back.
+__device__ __forceinline__ void st_stream(void* p, const Vec16& v)
+{
+    asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};"
+                 :: "l"(p), "r"(v.w[0]), "r"(v.w[1]), "r"(v.w[2]), "r"(v.w[3])
+                 : "memory");
+}
+
+__device__ __forceinline__ float4 ldg_f4(const float* p)
+{
+    return __ldg(reinterpret_cast<const float4*>(p));
+}
+
+__device__ __forceinline__ float ex2_approx(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float lg2_approx(float x)
+{
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float rcp_approx(float x)
+{
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float tanh_approx(float x)
+{
+    float y;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Element traits: how many elements a 16-byte vector holds and how to widen / narrow them.
+template <typename T>
+struct Elem;
+
+template <>
+struct Elem<float> {
+    static constexpr int kPerVec = 4;
+    __device__ __forceinline__ static void unpack(const Vec16& v, float (&f)[4])
+    {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) f[i] = __uint_as_float(v.w[i]);
+    }
+    __device__ __forceinline__ static Vec16 pack(const float (&f)[4])
+    {
+        Vec16 v;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) v.w[i] = __float_as_uint(f[i]);
+        return v;
+    }
+    __device__ __forceinline__ static float load1(const float* p) { return *p; }
+    __device__ __forceinline__ static void store1(float* p, float f) { *p = f; }
+    __device__ __forceinline__ static Vec16 fill_neg_inf()
+    {
+        Vec16 v;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) v.w[i] = 0xFF800000u;
+        return v;
+    }
+};
+
+template <>
+struct Elem<__nv_bfloat16> {
+    static constexpr int kPerVec = 8;
+    // bf16 is the top half of an fp32: widening is a shift / mask of the packed word.
+    __device__ __forceinline__ static void unpack(const Vec16& v, float (&f)[8])
+    {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            f[2 * i] = __uint_as_float(v.w[i] << 16);
+            f[2 * i + 1] = __uint_as_float(v.w[i] & 0xFFFF0000u);
+        }
+    }
+    // Round to nearest even, two values per cvt.
+    __device__ __forceinline__ static Vec16 pack(const float (&f)[8])
+    {
+        Vec16 v;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+            v.w[i] = *reinterpret_cast<uint32_t*>(&h);
+        }
+        return v;
+    }
+    __device__ __forceinline__ static float load1(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+    __device__ __forceinline__ static void store1(__nv_bfloat16* p, float f) { *p = __float2bfloat16_rn(f); }
+    __device__ __forceinline__ static Vec16 fill_neg_inf()
+    {
+        Vec16 v;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) v.w[i] = 0xFF80FF80u;
+        return v;
+    }
+};
+
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+    return v;
+}
+
+// Block-wide sum / max with ONE barrier: every warp publishes its partial in `slots` (>= 32
+// floats of shared memory, a different array for each back-to-back reduction so no second
+// barrier is needed), then every thread folds the published partials in slot order. The
+// result is identical in all threads and does not depend on scheduling.
+__device__ __forceinline__ float block_sum(float v, float* slots)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+    v = warp_sum(v);
+    if (nw == 1) return v;
+    if (lane == 0) slots[warp] = v;
+    __syncthreads();
+    float t = lane < nw ? slots[lane] : 0.0f;
+    return warp_sum(t);
+}
+__device__ __forceinline__ float block_max(float v, float* slots)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+    v = warp_max(v);
+    if (nw == 1) return v;
+    if (lane == 0) slots[warp] = v;
+    __syncthreads();
+    float t = lane < nw ? slots[lane] : -INFINITY;
+    return warp_max(t);
+}
+
+#endif  // __CUDACC__
+
+}  // namespace kop

@@ -1,0 +1,217 @@
+// kop_bias_gelu_residual_layernorm: v = residual + gelu_tanh(x + bias); y = LayerNorm(v) in one
+// HBM pass. A CTA owns a row; each thread keeps its share of v in fp32 registers, so the mean
+// and the centred second moment are both exact two-sweep sums over registers (no E[v^2]-mu^2
+// cancellation, no Welford merge needed) while x and residual are read from HBM once.
+#include "kop_common.cuh"
+
+namespace kop {
+namespace {
+
+// 0.5 u (1 + tanh(k0 (u + 0.044715 u^3))). bf16 rows use the hardware tanh (abs error ~2^-11,
+// below the 2^-9 relative step of the bf16 store); fp32 rows use the accurate tanhf.
+template <bool kFastTanh>
+__device__ __forceinline__ float gelu_tanh(float u)
+{
+    const float k0 = 0.7978845608028654f;          // sqrt(2/pi)
+    const float k1 = 0.7978845608028654f * 0.044715f;
+    const float inner = u * fmaf(k1, u * u, k0);
+    const float t = kFastTanh ? tanh_approx(inner) : tanhf(inner);
+    const float hu = 0.5f * u;
+    return fmaf(hu, t, hu);
+}
+
+template <typename T, int VPT>
+__global__ void __launch_bounds__(max_threads_for(VPT * Elem<T>::kPerVec))
+ln_block_kernel(const T* __restrict__ x, const T* __restrict__ res, const float* __restrict__ bias,
+                const float* __restrict__ gamma, const float* __restrict__ beta, T* __restrict__ y,
+                float* __restrict__ mean, float* __restrict__ rstd, int nvec, int64_t x_stride,
+                int64_t r_stride, int64_t y_stride, float eps, float inv_hidden)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    constexpr bool kFast = sizeof(T) == 2;
+    __shared__ float red_a[32], red_b[32];
+    const int64_t row = blockIdx.x;
+    const T* xr = x + row * x_stride;
+    const T* rr = res + row * r_stride;
+    T* yr = y + row * y_stride;
+
+    Vec16 rx[VPT], rres[VPT];
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+        const int v = k * blockDim.x + threadIdx.x;
+        if (v < nvec) {
+            rx[k] = ld_stream(xr + (int64_t)v * E);
+            rres[k] = ld_stream(rr + (int64_t)v * E);
+        }
+    }
+    float val[VPT][E];
+    float sum = 0.0f;
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+        const int v = k * blockDim.x + threadIdx.x;
+        float fx[E], fr[E];
+        Elem<T>::unpack(rx[k], fx);
+        Elem<T>::unpack(rres[k], fr);
+#pragma unroll
+        for (int q = 0; q < E / 4; ++q) {
+            float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (v < nvec) b = ldg_f4(bias + (int64_t)v * E + 4 * q);
+            const float bb[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int e = 4 * q + c;
+                const float t = fr[e] + gelu_tanh<kFast>(fx[e] + bb[c]);
+                val[k][e] = v < nvec ? t : 0.0f;
+                sum += val[k][e];
+            }
+        }
+    }
+    const float mu = block_sum(sum, red_a) * inv_hidden;
+    float ss = 0.0f;
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+        const int v = k * blockDim.x + threadIdx.x;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            val[k][e] -= mu;
+            ss = v < nvec ? fmaf(val[k][e], val[k][e], ss) : ss;
+        }
+    }
+    const float var = block_sum(ss, red_b) * inv_hidden;
+    const float rs = rsqrtf(var + eps);
+    if (threadIdx.x == 0) {
+        if (mean != nullptr) mean[row] = mu;
+        if (rstd != nullptr) rstd[row] = rs;
+    }
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+        const int v = k * blockDim.x + threadIdx.x;
+        if (v < nvec) {
+            float o[E];
+#pragma unroll
+            for (int q = 0; q < E / 4; ++q) {
+                const float4 g = ldg_f4(gamma + (int64_t)v * E + 4 * q);
+                const float4 b = ldg_f4(beta + (int64_t)v * E + 4 * q);
+                o[4 * q + 0] = fmaf(val[k][4 * q + 0] * rs, g.x, b.x);
+                o[4 * q + 1] = fmaf(val[k][4 * q + 1] * rs, g.y, b.y);
+                o[4 * q + 2] = fmaf(val[k][4 * q + 2] * rs, g.z, b.z);
+                o[4 * q + 3] = fmaf(val[k][4 * q + 3] * rs, g.w, b.w);
+            }
+            st_stream(yr + (int64_t)v * E, Elem<T>::pack(o));
+        }
+    }
+}
+
+// Any hidden size / alignment: scalar loads, v recomputed in each of three sweeps.
+template <typename T>
+__global__ void __launch_bounds__(256)
+ln_generic_kernel(const T* __restrict__ x, const T* __restrict__ res, const float* __restrict__ bias,
+                  const float* __restrict__ gamma, const float* __restrict__ beta, T* __restrict__ y,
+                  float* __restrict__ mean, float* __restrict__ rstd, int64_t hidden, int64_t x_stride,
+                  int64_t r_stride, int64_t y_stride, float eps, float inv_hidden)
+{
+    constexpr bool kFast = sizeof(T) == 2;
+    __shared__ float red_a[32], red_b[32];
+    const int64_t row = blockIdx.x;
+    const T* xr = x + row * x_stride;
+    const T* rr = res + row * r_stride;
+    T* yr = y + row * y_stride;
+    float sum = 0.0f;
+    for (int64_t j = threadIdx.x; j < hidden; j += blockDim.x)
+        sum += Elem<T>::load1(rr + j) + gelu_tanh<kFast>(Elem<T>::load1(xr + j) + __ldg(bias + j));
+    const float mu = block_sum(sum, red_a) * inv_hidden;
+    float ss = 0.0f;
+    for (int64_t j = threadIdx.x; j < hidden; j += blockDim.x) {
+        const float d =
+            Elem<T>::load1(rr + j) + gelu_tanh<kFast>(Elem<T>::load1(xr + j) + __ldg(bias + j)) - mu;
+        ss = fmaf(d, d, ss);
+    }
+    const float rs = rsqrtf(block_sum(ss, red_b) * inv_hidden + eps);
+    if (threadIdx.x == 0) {
+        if (mean != nullptr) mean[row] = mu;
+        if (rstd != nullptr) rstd[row] = rs;
+    }
+    for (int64_t j = threadIdx.x; j < hidden; j += blockDim.x) {
+        const float d =
+            Elem<T>::load1(rr + j) + gelu_tanh<kFast>(Elem<T>::load1(xr + j) + __ldg(bias + j)) - mu;
+        Elem<T>::store1(yr + j, fmaf(d * rs, __ldg(gamma + j), __ldg(beta + j)));
+    }
+}
+
+template <typename T>
+kop_status_t launch_ln(const void* xv, const void* rv, const float* bias, const float* gamma,
+                       const float* beta, void* yv, float* mean, float* rstd, int64_t rows,
+                       int64_t hidden, int64_t xs, int64_t rs, int64_t ys, float eps,
+                       cudaStream_t stream)
+{
+    const T* x = static_cast<const T*>(xv);
+    const T* r = static_cast<const T*>(rv);
+    T* y = static_cast<T*>(yv);
+    constexpr int E = Elem<T>::kPerVec;
+    const float inv_hidden = (float)(1.0 / (double)hidden);
+    if (rows > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+    const bool vec = vec_ok(x, hidden, xs, sizeof(T)) && vec_ok(r, hidden, rs, sizeof(T)) &&
+                     vec_ok(y, hidden, ys, sizeof(T)) && aligned_to(bias, 16) &&
+                     aligned_to(gamma, 16) && aligned_to(beta, 16);
+    const int64_t nvec64 = hidden / E;
+    if (vec && hidden <= kMaxRegisterRow) {
+        const int nvec = (int)nvec64;
+        // 32 values per thread (hidden 4096 -> 128-thread CTAs, eight 16-byte loads in flight per
+        // thread and ~8 CTAs per SM); short rows use fewer, rows beyond 512 threads' worth use 64.
+        int vals = 32;
+        if (hidden <= 1024) vals = 16;
+        if (hidden <= 256) vals = 8;
+        if ((nvec + vals / E - 1) / (vals / E) > max_threads_for(vals)) vals = 64;
+        const int vpt = vals / E;
+        const int threads = ((nvec + vpt - 1) / vpt + 31) / 32 * 32;
+#define KOP_LN(V)                                                                               \
+    ln_block_kernel<T, V><<<(unsigned)rows, threads, 0, stream>>>(x, r, bias, gamma, beta, y, mean, \
+                                                                  rstd, nvec, xs, rs, ys, eps, inv_hidden)
+        switch (vals) {
+        case 8: KOP_LN(8 / E); break;
+        case 16: KOP_LN(16 / E); break;
+        case 32: KOP_LN(32 / E); break;
+        default: KOP_LN(64 / E); break;
+        }
+#undef KOP_LN
+        return launch_status();
+    }
+    ln_generic_kernel<T><<<(unsigned)rows, 256, 0, stream>>>(x, r, bias, gamma, beta, y, mean, rstd,
+                                                             hidden, xs, rs, ys, eps, inv_hidden);
+    return launch_status();
+}
+
+}  // namespace
+}  // namespace kop
+
+extern "C" kop_status_t kop_bias_gelu_residual_layernorm(
+    const void* x, const void* residual, const float* bias, const float* gamma, const float* beta,
+    void* y, float* mean, float* rstd, int64_t rows, int64_t hidden, int64_t x_row_stride,
+    int64_t res_row_stride, int64_t y_row_stride, float eps, kop_dtype_t dtype, kop_stream_t stream)
+{
+    using namespace kop;
+    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    if (!x || !residual || !bias || !gamma || !beta || !y) return KOP_ERR_NULL_POINTER;
+    kop_status_t st = check_rows_cols(rows, hidden);
+    if (st != KOP_OK) return st;
+    if ((st = check_row_stride(x_row_stride, hidden, rows)) != KOP_OK) return st;
+    if ((st = check_row_stride(res_row_stride, hidden, rows)) != KOP_OK) return st;
+    if ((st = check_row_stride(y_row_stride, hidden, rows)) != KOP_OK) return st;
+    if (!(eps >= 0.0f)) return KOP_ERR_BAD_SHAPE;
+    const int esz = elem_size(dtype);
+    if (!aligned_to(x, esz) || !aligned_to(residual, esz) || !aligned_to(y, esz) ||
+        !aligned_to(bias, 4) || !aligned_to(gamma, 4) || !aligned_to(beta, 4) ||
+        (mean && !aligned_to(mean, 4)) || (rstd && !aligned_to(rstd, 4)))
+        return KOP_ERR_MISALIGNED;
+    if (!alias_ok(x, x_row_stride, y, y_row_stride, rows, hidden, esz, true) ||
+        !alias_ok(residual, res_row_stride, y, y_row_stride, rows, hidden, esz, true))
+        return KOP_ERR_BAD_ALIAS;
+    if (rows == 0) return KOP_OK;
+    if ((st = check_device()) != KOP_OK) return st;
+    cudaStream_t s = as_stream(stream);
+    return dtype == KOP_F32
+               ? launch_ln<float>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
+                                  x_row_stride, res_row_stride, y_row_stride, eps, s)
+               : launch_ln<__nv_bfloat16>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
+                                          x_row_stride, res_row_stride, y_row_stride, eps, s);
+}

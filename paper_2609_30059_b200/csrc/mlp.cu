@@ -1,0 +1,465 @@
+// The transformer-MLP segment: kop_rmsnorm, kop_silu_mul, kop_residual_add, and the driver
+// kop_rmsnorm_swiglu_residual that enqueues them around two preserved cuBLAS GEMMs.
+#include <cublas_v2.h>
+
+#include "kop_common.cuh"
+
+namespace kop {
+namespace {
+
+// ---- RMSNorm: CTA per row, row in registers -----------------------------------------------------
+template <typename T, int VPT>
+__global__ void __launch_bounds__(max_threads_for(VPT * Elem<T>::kPerVec))
+rmsnorm_block_kernel(const T* __restrict__ x, const float* __restrict__ w, T* __restrict__ y, int nvec,
+                     int64_t x_stride, int64_t y_stride, float eps, float inv_hidden)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    __shared__ float red[32];
+    const int64_t row = blockIdx.x;
+    const T* xr = x + row * x_stride;
+    T* yr = y + row * y_stride;
+    Vec16 raw[VPT];
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+        const int v = k * blockDim.x + threadIdx.x;
+        if (v < nvec) raw[k] = ld_stream(xr + (int64_t)v * E);
+    }
+    float val[VPT][E];
+    float ss = 0.0f;
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+        const int v = k * blockDim.x + threadIdx.x;
+        Elem<T>::unpack(raw[k], val[k]);
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            val[k][e] = v < nvec ? val[k][e] : 0.0f;
+            ss = fmaf(val[k][e], val[k][e], ss);
+        }
+    }
+    const float r = rsqrtf(block_sum(ss, red) * inv_hidden + eps);
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+        const int v = k * blockDim.x + threadIdx.x;
+        if (v < nvec) {
+            float o[E];
+#pragma unroll
+            for (int q = 0; q < E / 4; ++q) {
+                const float4 g = ldg_f4(w + (int64_t)v * E + 4 * q);
+                o[4 * q + 0] = val[k][4 * q + 0] * r * g.x;
+                o[4 * q + 1] = val[k][4 * q + 1] * r * g.y;
+                o[4 * q + 2] = val[k][4 * q + 2] * r * g.z;
+                o[4 * q + 3] = val[k][4 * q + 3] * r * g.w;
+            }
+            st_stream(yr + (int64_t)v * E, Elem<T>::pack(o));
+        }
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+rmsnorm_generic_kernel(const T* __restrict__ x, const float* __restrict__ w, T* __restrict__ y,
+                       int64_t hidden, int64_t x_stride, int64_t y_stride, float eps, float inv_hidden)
+{
+    __shared__ float red[32];
+    const int64_t row = blockIdx.x;
+    const T* xr = x + row * x_stride;
+    T* yr = y + row * y_stride;
+    float ss = 0.0f;
+    for (int64_t j = threadIdx.x; j < hidden; j += blockDim.x) {
+        const float v = Elem<T>::load1(xr + j);
+        ss = fmaf(v, v, ss);
+    }
+    const float r = rsqrtf(block_sum(ss, red) * inv_hidden + eps);
+    for (int64_t j = threadIdx.x; j < hidden; j += blockDim.x)
+        Elem<T>::store1(yr + j, Elem<T>::load1(xr + j) * r * __ldg(w + j));
+}
+
+// ---- SiLU(gate) * up ------------------------------------------------------------------------------
+// silu(g) = g / (1 + 2^(-g log2e)): one ex2 and one reciprocal. bf16 rows use the approximate
+// reciprocal (relative error ~2^-23, far below the bf16 store step); fp32 rows divide exactly.
+template <bool kFast>
+__device__ __forceinline__ float silu(float g)
+{
+    const float d = 1.0f + ex2_approx(-g * kLog2e);
+    return kFast ? g * rcp_approx(d) : g / d;
+}
+
+// A CTA covers `U * blockDim.x` consecutive output vectors of one row (tile index = blockIdx.x).
+template <typename T, int U>
+__global__ void __launch_bounds__(256)
+silu_mul_kernel(const T* __restrict__ gu, T* __restrict__ out, int nvec, int tiles_per_row,
+                int64_t inter, int64_t in_stride, int64_t out_stride)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    constexpr bool kFast = sizeof(T) == 2;
+    const int64_t row = blockIdx.x / tiles_per_row;
+    const int tile = (int)(blockIdx.x - row * tiles_per_row);
+    const T* g = gu + row * in_stride;
+    const T* u = g + inter;
+    T* o = out + row * out_stride;
+    const int v0 = tile * (U * blockDim.x) + threadIdx.x;
+    Vec16 rg[U], ru[U];
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+        const int v = v0 + k * blockDim.x;
+        if (v < nvec) {
+            rg[k] = ld_stream(g + (int64_t)v * E);
+            ru[k] = ld_stream(u + (int64_t)v * E);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+        const int v = v0 + k * blockDim.x;
+        if (v < nvec) {
+            float fg[E], fu[E];
+            Elem<T>::unpack(rg[k], fg);
+            Elem<T>::unpack(ru[k], fu);
+#pragma unroll
+            for (int e = 0; e < E; ++e) fg[e] = silu<kFast>(fg[e]) * fu[e];
+            st_stream(o + (int64_t)v * E, Elem<T>::pack(fg));
+        }
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+silu_mul_scalar_kernel(const T* __restrict__ gu, T* __restrict__ out, int64_t rows, int64_t inter,
+                       int64_t in_stride, int64_t out_stride)
+{
+    constexpr bool kFast = sizeof(T) == 2;
+    const int64_t total = rows * inter;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / inter, j = i - r * inter;
+        const float g = Elem<T>::load1(gu + r * in_stride + j);
+        const float u = Elem<T>::load1(gu + r * in_stride + inter + j);
+        Elem<T>::store1(out + r * out_stride + j, silu<kFast>(g) * u);
+    }
+}
+
+// ---- residual add -----------------------------------------------------------------------------------
+template <typename T, int U>
+__global__ void __launch_bounds__(256)
+residual_add_kernel(const T* __restrict__ a, const T* __restrict__ b, T* __restrict__ out, int64_t nvec,
+                    int64_t tiles_per_row, int64_t a_stride, int64_t b_stride, int64_t o_stride)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    const int64_t row = blockIdx.x / tiles_per_row;
+    const int64_t tile = blockIdx.x - row * tiles_per_row;
+    const T* ar = a + row * a_stride;
+    const T* br = b + row * b_stride;
+    T* orow = out + row * o_stride;
+    const int64_t v0 = tile * (U * blockDim.x) + threadIdx.x;
+    Vec16 ra[U], rb[U];
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+        const int64_t v = v0 + k * blockDim.x;
+        if (v < nvec) {
+            ra[k] = ld_stream(ar + v * E);
+            rb[k] = ld_stream(br + v * E);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+        const int64_t v = v0 + k * blockDim.x;
+        if (v < nvec) {
+            float fa[E], fb[E];
+            Elem<T>::unpack(ra[k], fa);
+            Elem<T>::unpack(rb[k], fb);
+#pragma unroll
+            for (int e = 0; e < E; ++e) fa[e] += fb[e];
+            st_stream(orow + v * E, Elem<T>::pack(fa));
+        }
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+residual_add_scalar_kernel(const T* __restrict__ a, const T* __restrict__ b, T* __restrict__ out,
+                           int64_t rows, int64_t cols, int64_t a_stride, int64_t b_stride,
+                           int64_t o_stride)
+{
+    const int64_t total = rows * cols;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / cols, j = i - r * cols;
+        Elem<T>::store1(out + r * o_stride + j,
+                        Elem<T>::load1(a + r * a_stride + j) + Elem<T>::load1(b + r * b_stride + j));
+    }
+}
+
+// ---- launchers ------------------------------------------------------------------------------------
+template <typename T>
+kop_status_t launch_rmsnorm(const void* xv, const float* w, void* yv, int64_t rows, int64_t hidden,
+                            int64_t xs, int64_t ys, float eps, cudaStream_t stream)
+{
+    const T* x = static_cast<const T*>(xv);
+    T* y = static_cast<T*>(yv);
+    constexpr int E = Elem<T>::kPerVec;
+    if (rows > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+    const float inv_hidden = (float)(1.0 / (double)hidden);
+    const bool vec = vec_ok(x, hidden, xs, sizeof(T)) && vec_ok(y, hidden, ys, sizeof(T)) && aligned_to(w, 16);
+    const int64_t nvec64 = hidden / E;
+    if (vec && hidden <= kMaxRegisterRow) {
+        const int nvec = (int)nvec64;
+        int vals = 32;
+        if (hidden <= 1024) vals = 16;
+        if (hidden <= 256) vals = 8;
+        if ((nvec + vals / E - 1) / (vals / E) > max_threads_for(vals)) vals = 64;
+        const int vpt = vals / E;
+        const int threads = ((nvec + vpt - 1) / vpt + 31) / 32 * 32;
+#define KOP_RMS(V) rmsnorm_block_kernel<T, V><<<(unsigned)rows, threads, 0, stream>>>(x, w, y, nvec, xs, ys, eps, inv_hidden)
+        switch (vals) {
+        case 8: KOP_RMS(8 / E); break;
+        case 16: KOP_RMS(16 / E); break;
+        case 32: KOP_RMS(32 / E); break;
+        default: KOP_RMS(64 / E); break;
+        }
+#undef KOP_RMS
+        return launch_status();
+    }
+    rmsnorm_generic_kernel<T><<<(unsigned)rows, 256, 0, stream>>>(x, w, y, hidden, xs, ys, eps, inv_hidden);
+    return launch_status();
+}
+
+inline unsigned scalar_grid(int64_t total)
+{
+    const int64_t want = (total + 255) / 256;
+    const int64_t cap = (int64_t)sm_count() * 32;
+    return (unsigned)(want < cap ? (want > 0 ? want : 1) : cap);
+}
+
+template <typename T>
+kop_status_t launch_silu_mul(const void* guv, void* outv, int64_t rows, int64_t inter, int64_t is,
+                             int64_t os, cudaStream_t stream)
+{
+    const T* gu = static_cast<const T*>(guv);
+    T* out = static_cast<T*>(outv);
+    constexpr int E = Elem<T>::kPerVec;
+    const bool vec = aligned_to(gu, 16) && aligned_to(out, 16) && (inter % E) == 0 && (is % E) == 0 &&
+                     (os % E) == 0;
+    const int64_t nvec64 = inter / E;
+    if (vec && nvec64 <= 0x7FFFFFFF) {
+        const int nvec = (int)nvec64;
+        const int threads = 128;
+        // Two gate and two up vectors in flight per thread; the tile divides inter = 14336 bf16
+        // (1792 vectors = 7 tiles of 256) exactly.
+        constexpr int U = 2;
+        const int tiles = (nvec + threads * U - 1) / (threads * U);
+        const int64_t grid = rows * tiles;
+        if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+        silu_mul_kernel<T, U><<<(unsigned)grid, threads, 0, stream>>>(gu, out, nvec, tiles, inter, is, os);
+        return launch_status();
+    }
+    silu_mul_scalar_kernel<T><<<scalar_grid(rows * inter), 256, 0, stream>>>(gu, out, rows, inter, is, os);
+    return launch_status();
+}
+
+template <typename T>
+kop_status_t launch_residual_add(const void* av, const void* bv, void* ov, int64_t rows, int64_t cols,
+                                 int64_t as, int64_t bs, int64_t os, cudaStream_t stream)
+{
+    const T* a = static_cast<const T*>(av);
+    const T* b = static_cast<const T*>(bv);
+    T* out = static_cast<T*>(ov);
+    constexpr int E = Elem<T>::kPerVec;
+    // Fully contiguous tensors collapse to one long row.
+    if (as == cols && bs == cols && os == cols) {
+        cols = rows * cols;
+        rows = 1;
+        as = bs = os = cols;
+    }
+    const bool vec = vec_ok(a, cols, as, sizeof(T)) && vec_ok(b, cols, bs, sizeof(T)) &&
+                     vec_ok(out, cols, os, sizeof(T));
+    if (vec) {
+        const int64_t nvec = cols / E;
+        const int threads = 128;
+        constexpr int U = 4;
+        const int64_t tiles = (nvec + threads * U - 1) / (threads * U);
+        const int64_t grid = rows * tiles;
+        if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+        residual_add_kernel<T, U><<<(unsigned)grid, threads, 0, stream>>>(a, b, out, nvec, tiles, as, bs, os);
+        return launch_status();
+    }
+    residual_add_scalar_kernel<T><<<scalar_grid(rows * cols), 256, 0, stream>>>(a, b, out, rows, cols, as, bs, os);
+    return launch_status();
+}
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+constexpr size_t kCublasWorkspace = (size_t)32 << 20;   // recommended size for Hopper-class and later
+
+struct MlpLayout {
+    size_t n_off, gu_off, act_off, d_off, cublas_off, total;
+};
+inline MlpLayout mlp_layout(int64_t rows, int64_t hidden, int64_t inter, int esz)
+{
+    MlpLayout L;
+    size_t off = 0;
+    L.n_off = off;      off = align_up(off + (size_t)rows * hidden * esz, 256);
+    L.gu_off = off;     off = align_up(off + (size_t)rows * 2 * inter * esz, 256);
+    L.act_off = off;    off = align_up(off + (size_t)rows * inter * esz, 256);
+    L.d_off = off;      off = align_up(off + (size_t)rows * hidden * esz, 256);
+    L.cublas_off = off; off += kCublasWorkspace;
+    L.total = off;
+    return L;
+}
+
+// Row-major C[M,N] = A[M,K] * W[N,K]^T  ==  column-major C^T[N,M] = W(KxN col-major)^T * A^T.
+kop_status_t gemm_nt(cublasHandle_t h, const void* A, const void* Wt, void* Cout, int64_t M, int64_t N,
+                     int64_t K, kop_dtype_t dtype)
+{
+    const float alpha = 1.0f, beta = 0.0f;
+    const cudaDataType_t t = dtype == KOP_F32 ? CUDA_R_32F : CUDA_R_16BF;
+    if (M > 0x7FFFFFFFLL || N > 0x7FFFFFFFLL || K > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+    cublasStatus_t st = cublasGemmEx(h, CUBLAS_OP_T, CUBLAS_OP_N, (int)N, (int)M, (int)K, &alpha, Wt, t,
+                                     (int)K, A, t, (int)K, &beta, Cout, t, (int)N, CUBLAS_COMPUTE_32F,
+                                     CUBLAS_GEMM_DEFAULT);
+    return st == CUBLAS_STATUS_SUCCESS ? KOP_OK : KOP_ERR_CUBLAS;
+}
+
+}  // namespace
+}  // namespace kop
+
+extern "C" kop_status_t kop_rmsnorm(const void* x, const float* weight, void* y, int64_t rows,
+                                    int64_t hidden, int64_t x_row_stride, int64_t y_row_stride,
+                                    float eps, kop_dtype_t dtype, kop_stream_t stream)
+{
+    using namespace kop;
+    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    if (!x || !weight || !y) return KOP_ERR_NULL_POINTER;
+    kop_status_t st = check_rows_cols(rows, hidden);
+    if (st != KOP_OK) return st;
+    if ((st = check_row_stride(x_row_stride, hidden, rows)) != KOP_OK) return st;
+    if ((st = check_row_stride(y_row_stride, hidden, rows)) != KOP_OK) return st;
+    if (!(eps >= 0.0f)) return KOP_ERR_BAD_SHAPE;
+    const int esz = elem_size(dtype);
+    if (!aligned_to(x, esz) || !aligned_to(y, esz) || !aligned_to(weight, 4)) return KOP_ERR_MISALIGNED;
+    if (!alias_ok(x, x_row_stride, y, y_row_stride, rows, hidden, esz, true)) return KOP_ERR_BAD_ALIAS;
+    if (rows == 0) return KOP_OK;
+    if ((st = check_device()) != KOP_OK) return st;
+    cudaStream_t s = as_stream(stream);
+    return dtype == KOP_F32
+               ? launch_rmsnorm<float>(x, weight, y, rows, hidden, x_row_stride, y_row_stride, eps, s)
+               : launch_rmsnorm<__nv_bfloat16>(x, weight, y, rows, hidden, x_row_stride, y_row_stride, eps, s);
+}
+
+extern "C" kop_status_t kop_silu_mul(const void* gate_up, void* out, int64_t rows, int64_t inter,
+                                     int64_t in_row_stride, int64_t out_row_stride, kop_dtype_t dtype,
+                                     kop_stream_t stream)
+{
+    using namespace kop;
+    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    if (!gate_up || !out) return KOP_ERR_NULL_POINTER;
+    kop_status_t st = check_rows_cols(rows, inter);
+    if (st != KOP_OK) return st;
+    if (inter > kMaxElems / 2) return KOP_ERR_BAD_SHAPE;
+    if ((st = check_row_stride(in_row_stride, 2 * inter, rows)) != KOP_OK) return st;
+    if ((st = check_row_stride(out_row_stride, inter, rows)) != KOP_OK) return st;
+    const int esz = elem_size(dtype);
+    if (!aligned_to(gate_up, esz) || !aligned_to(out, esz)) return KOP_ERR_MISALIGNED;
+    if (rows > 0) {
+        uintptr_t a0, a1, b0, b1;
+        span_of(gate_up, rows, 2 * inter, in_row_stride, esz, &a0, &a1);
+        span_of(out, rows, inter, out_row_stride, esz, &b0, &b1);
+        if (!(a1 <= b0 || b1 <= a0)) return KOP_ERR_BAD_ALIAS;
+    }
+    if (rows == 0) return KOP_OK;
+    if ((st = check_device()) != KOP_OK) return st;
+    cudaStream_t s = as_stream(stream);
+    return dtype == KOP_F32
+               ? launch_silu_mul<float>(gate_up, out, rows, inter, in_row_stride, out_row_stride, s)
+               : launch_silu_mul<__nv_bfloat16>(gate_up, out, rows, inter, in_row_stride, out_row_stride, s);
+}
+
+extern "C" kop_status_t kop_residual_add(const void* a, const void* b, void* out, int64_t rows,
+                                         int64_t cols, int64_t a_row_stride, int64_t b_row_stride,
+                                         int64_t out_row_stride, kop_dtype_t dtype, kop_stream_t stream)
+{
+    using namespace kop;
+    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    if (!a || !b || !out) return KOP_ERR_NULL_POINTER;
+    kop_status_t st = check_rows_cols(rows, cols);
+    if (st != KOP_OK) return st;
+    if ((st = check_row_stride(a_row_stride, cols, rows)) != KOP_OK) return st;
+    if ((st = check_row_stride(b_row_stride, cols, rows)) != KOP_OK) return st;
+    if ((st = check_row_stride(out_row_stride, cols, rows)) != KOP_OK) return st;
+    const int esz = elem_size(dtype);
+    if (!aligned_to(a, esz) || !aligned_to(b, esz) || !aligned_to(out, esz)) return KOP_ERR_MISALIGNED;
+    if (!alias_ok(a, a_row_stride, out, out_row_stride, rows, cols, esz, true) ||
+        !alias_ok(b, b_row_stride, out, out_row_stride, rows, cols, esz, true))
+        return KOP_ERR_BAD_ALIAS;
+    if (rows == 0) return KOP_OK;
+    if ((st = check_device()) != KOP_OK) return st;
+    cudaStream_t s = as_stream(stream);
+    return dtype == KOP_F32
+               ? launch_residual_add<float>(a, b, out, rows, cols, a_row_stride, b_row_stride, out_row_stride, s)
+               : launch_residual_add<__nv_bfloat16>(a, b, out, rows, cols, a_row_stride, b_row_stride, out_row_stride, s);
+}
+
+extern "C" size_t kop_rmsnorm_swiglu_residual_workspace_bytes(int64_t rows, int64_t hidden,
+                                                              int64_t inter, kop_dtype_t dtype)
+{
+    using namespace kop;
+    if (rows < 0 || hidden <= 0 || inter <= 0 || !dtype_ok(dtype)) return 0;
+    if (hidden > 0x7FFFFFFFLL || inter > 0x3FFFFFFFLL || rows > 0x7FFFFFFFLL) return 0;
+    return mlp_layout(rows, hidden, inter, elem_size(dtype)).total;
+}
+
+extern "C" kop_status_t kop_mlp_handle_create(void** handle)
+{
+    if (handle == nullptr) return KOP_ERR_NULL_POINTER;
+    kop_status_t st = kop::check_device();
+    if (st != KOP_OK) return st;
+    cublasHandle_t h = nullptr;
+    if (cublasCreate(&h) != CUBLAS_STATUS_SUCCESS) return KOP_ERR_CUBLAS;
+    *handle = h;
+    return KOP_OK;
+}
+
+extern "C" kop_status_t kop_mlp_handle_destroy(void* handle)
+{
+    if (handle == nullptr) return KOP_ERR_NULL_POINTER;
+    return cublasDestroy(static_cast<cublasHandle_t>(handle)) == CUBLAS_STATUS_SUCCESS ? KOP_OK
+                                                                                       : KOP_ERR_CUBLAS;
+}
+
+extern "C" kop_status_t kop_rmsnorm_swiglu_residual(void* handle, const void* h, const float* rms_weight,
+                                                    const void* w_gate_up, const void* w_down, void* out,
+                                                    int64_t rows, int64_t hidden, int64_t inter, float eps,
+                                                    void* workspace, size_t workspace_bytes,
+                                                    kop_dtype_t dtype, kop_stream_t stream)
+{
+    using namespace kop;
+    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    if (!handle || !h || !rms_weight || !w_gate_up || !w_down || !out || !workspace)
+        return KOP_ERR_NULL_POINTER;
+    if (rows < 0 || hidden <= 0 || inter <= 0) return KOP_ERR_BAD_SHAPE;
+    if (hidden > 0x7FFFFFFFLL || inter > 0x3FFFFFFFLL || rows > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+    const int esz = elem_size(dtype);
+    if (!aligned_to(h, esz) || !aligned_to(out, esz) || !aligned_to(w_gate_up, esz) ||
+        !aligned_to(w_down, esz) || !aligned_to(rms_weight, 4) || !aligned_to(workspace, 256))
+        return KOP_ERR_MISALIGNED;
+    if (!(eps >= 0.0f)) return KOP_ERR_BAD_SHAPE;
+    if (!alias_ok(h, hidden, out, hidden, rows, hidden, esz, true)) return KOP_ERR_BAD_ALIAS;
+    const MlpLayout L = mlp_layout(rows, hidden, inter, esz);
+    if (workspace_bytes < L.total) return KOP_ERR_WORKSPACE_TOO_SMALL;
+    if (rows == 0) return KOP_OK;
+    kop_status_t st = check_device();
+    if (st != KOP_OK) return st;
+
+    char* ws = static_cast<char*>(workspace);
+    void* n = ws + L.n_off;
+    void* gu = ws + L.gu_off;
+    void* act = ws + L.act_off;
+    void* d = ws + L.d_off;
+    cublasHandle_t cb = static_cast<cublasHandle_t>(handle);
+    if (cublasSetStream(cb, as_stream(stream)) != CUBLAS_STATUS_SUCCESS) return KOP_ERR_CUBLAS;
+    if (cublasSetWorkspace(cb, ws + L.cublas_off, kCublasWorkspace) != CUBLAS_STATUS_SUCCESS)
+        return KOP_ERR_CUBLAS;
+
+    if ((st = kop_rmsnorm(h, rms_weight, n, rows, hidden, hidden, hidden, eps, dtype, stream)) != KOP_OK) return st;
+    if ((st = gemm_nt(cb, n, w_gate_up, gu, rows, 2 * inter, hidden, dtype)) != KOP_OK) return st;
+    if ((st = kop_silu_mul(gu, act, rows, inter, 2 * inter, inter, dtype, stream)) != KOP_OK) return st;
+    if ((st = gemm_nt(cb, act, w_down, d, rows, hidden, inter, dtype)) != KOP_OK) return st;
+    return kop_residual_add(h, d, out, rows, hidden, hidden, hidden, hidden, dtype, stream);
+}

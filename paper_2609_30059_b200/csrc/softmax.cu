@@ -1,0 +1,266 @@
+// kop_softmax_scale_bias: y = softmax_j(x * scale + bias) per row, one HBM pass.
+//
+// The row lives in registers between the load and the store: a warp owns a row when it is short
+// (each lane holds VPL 16-byte vectors), a whole CTA owns it when it is long. The exponent runs
+// in the base-2 domain: t = x * (scale*log2e) + bias*log2e is one FMA, the row max is taken on t,
+// and exp(z - max z) = 2^(t - max t) is one ex2.approx. Rows that cannot be read with 16-byte
+// vectors go to a scalar three-sweep kernel with the same arithmetic.
+#include "kop_common.cuh"
+
+namespace kop {
+namespace {
+
+// ---- warp per row, grid-stride over rows, bias kept in registers ------------------------------
+template <typename T, int VPL, bool kBiasInRegs>
+__global__ void __launch_bounds__(256)
+softmax_warp_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* __restrict__ y,
+                    int64_t rows, int nvec, int64_t x_stride, int64_t y_stride, float scale)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    const int lane = threadIdx.x & 31;
+    const int64_t warps_per_cta = blockDim.x >> 5;
+    const int64_t warp0 = (int64_t)blockIdx.x * warps_per_cta + (threadIdx.x >> 5);
+    const int64_t nwarps = (int64_t)gridDim.x * warps_per_cta;
+    const float s2 = scale * kLog2e;
+
+    // Short rows keep the (pre-scaled) bias in registers across the rows a warp visits; wider
+    // rows re-read it through L1, where the streaming data loads never allocate.
+    float b2[kBiasInRegs ? VPL : 1][E];
+#pragma unroll
+    for (int k = 0; k < (kBiasInRegs ? VPL : 0); ++k) {
+        const int v = k * 32 + lane;
+#pragma unroll
+        for (int e = 0; e < E; ++e) b2[k][e] = 0.0f;
+        if (bias != nullptr && v < nvec) {
+#pragma unroll
+            for (int q = 0; q < E / 4; ++q) {
+                float4 t = ldg_f4(bias + (int64_t)v * E + 4 * q);
+                b2[k][4 * q + 0] = t.x * kLog2e;
+                b2[k][4 * q + 1] = t.y * kLog2e;
+                b2[k][4 * q + 2] = t.z * kLog2e;
+                b2[k][4 * q + 3] = t.w * kLog2e;
+            }
+        }
+    }
+
+    for (int64_t row = warp0; row < rows; row += nwarps) {
+        const T* xr = x + row * x_stride;
+        T* yr = y + row * y_stride;
+        Vec16 raw[VPL];
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+            const int v = k * 32 + lane;
+            if (v < nvec) raw[k] = ld_stream(xr + (int64_t)v * E);
+        }
+        float t[VPL][E];
+        float m = -INFINITY;
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+            const int v = k * 32 + lane;
+            float f[E];
+            Elem<T>::unpack(raw[k], f);
+            float bk[E];
+            if (kBiasInRegs) {
+#pragma unroll
+                for (int e = 0; e < E; ++e) bk[e] = b2[k][e];
+            } else {
+#pragma unroll
+                for (int q = 0; q < E / 4; ++q) {
+                    float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (bias != nullptr && v < nvec) b = ldg_f4(bias + (int64_t)v * E + 4 * q);
+                    bk[4 * q + 0] = b.x * kLog2e;
+                    bk[4 * q + 1] = b.y * kLog2e;
+                    bk[4 * q + 2] = b.z * kLog2e;
+                    bk[4 * q + 3] = b.w * kLog2e;
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                t[k][e] = v < nvec ? fmaf(f[e], s2, bk[e]) : -INFINITY;
+                m = fmaxf(m, t[k][e]);
+            }
+        }
+        m = warp_max(m);
+        float s = 0.0f;
+#pragma unroll
+        for (int k = 0; k < VPL; ++k)
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                t[k][e] = ex2_approx(t[k][e] - m);
+                s += t[k][e];
+            }
+        s = warp_sum(s);
+        const float inv = 1.0f / s;
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+            const int v = k * 32 + lane;
+            float o[E];
+#pragma unroll
+            for (int e = 0; e < E; ++e) o[e] = t[k][e] * inv;
+            if (v < nvec) st_stream(yr + (int64_t)v * E, Elem<T>::pack(o));
+        }
+    }
+}
+
+// ---- CTA per row, row in registers ---------------------------------------------------------------
+template <typename T, int VPT>
+__global__ void __launch_bounds__(max_threads_for(VPT * Elem<T>::kPerVec))
+softmax_block_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* __restrict__ y,
+                     int nvec, int64_t x_stride, int64_t y_stride, float scale)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    __shared__ float red_a[32], red_b[32];
+    const int64_t row = blockIdx.x;
+    const T* xr = x + row * x_stride;
+    T* yr = y + row * y_stride;
+    const float s2 = scale * kLog2e;
+
+    Vec16 raw[VPT];
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+        const int v = k * blockDim.x + threadIdx.x;
+        if (v < nvec) raw[k] = ld_stream(xr + (int64_t)v * E);
+    }
+    float t[VPT][E];
+    float m = -INFINITY;
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+        const int v = k * blockDim.x + threadIdx.x;
+        float f[E];
+        Elem<T>::unpack(raw[k], f);
+#pragma unroll
+        for (int q = 0; q < E / 4; ++q) {
+            float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (bias != nullptr && v < nvec) b = ldg_f4(bias + (int64_t)v * E + 4 * q);
+            const float bb[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int e = 4 * q + c;
+                t[k][e] = v < nvec ? fmaf(f[e], s2, bb[c] * kLog2e) : -INFINITY;
+                m = fmaxf(m, t[k][e]);
+            }
+        }
+    }
+    m = block_max(m, red_a);
+    float s = 0.0f;
+#pragma unroll
+    for (int k = 0; k < VPT; ++k)
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            t[k][e] = ex2_approx(t[k][e] - m);
+            s += t[k][e];
+        }
+    s = block_sum(s, red_b);
+    const float inv = 1.0f / s;
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+        const int v = k * blockDim.x + threadIdx.x;
+        float o[E];
+#pragma unroll
+        for (int e = 0; e < E; ++e) o[e] = t[k][e] * inv;
+        if (v < nvec) st_stream(yr + (int64_t)v * E, Elem<T>::pack(o));
+    }
+}
+
+// ---- any length, any alignment: scalar loads, three sweeps over the row ----------------------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+softmax_generic_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* __restrict__ y,
+                       int64_t cols, int64_t x_stride, int64_t y_stride, float scale)
+{
+    __shared__ float red_a[32], red_b[32];
+    const int64_t row = blockIdx.x;
+    const T* xr = x + row * x_stride;
+    T* yr = y + row * y_stride;
+    const float s2 = scale * kLog2e;
+    float m = -INFINITY;
+    for (int64_t j = threadIdx.x; j < cols; j += blockDim.x) {
+        const float b = bias != nullptr ? __ldg(bias + j) * kLog2e : 0.0f;
+        m = fmaxf(m, fmaf(Elem<T>::load1(xr + j), s2, b));
+    }
+    m = block_max(m, red_a);
+    float s = 0.0f;
+    for (int64_t j = threadIdx.x; j < cols; j += blockDim.x) {
+        const float b = bias != nullptr ? __ldg(bias + j) * kLog2e : 0.0f;
+        s += ex2_approx(fmaf(Elem<T>::load1(xr + j), s2, b) - m);
+    }
+    s = block_sum(s, red_b);
+    const float inv = 1.0f / s;
+    // The last sweep reads x[j] and writes y[j] in the same thread, so exact aliasing stays safe.
+    for (int64_t j = threadIdx.x; j < cols; j += blockDim.x) {
+        const float b = bias != nullptr ? __ldg(bias + j) * kLog2e : 0.0f;
+        Elem<T>::store1(yr + j, ex2_approx(fmaf(Elem<T>::load1(xr + j), s2, b) - m) * inv);
+    }
+}
+
+template <typename T>
+kop_status_t launch_softmax(const void* xv, const float* bias, void* yv, int64_t rows, int64_t cols,
+                            int64_t xs, int64_t ys, float scale, cudaStream_t stream)
+{
+    const T* x = static_cast<const T*>(xv);
+    T* y = static_cast<T*>(yv);
+    constexpr int E = Elem<T>::kPerVec;
+    const bool vec = vec_ok(x, cols, xs, sizeof(T)) && vec_ok(y, cols, ys, sizeof(T)) &&
+                     (bias == nullptr || aligned_to(bias, 16));
+    const int64_t nvec64 = cols / E;
+    if (vec && nvec64 <= 32 * 4) {
+        const int nvec = (int)nvec64;
+        const int vpl = (nvec + 31) / 32;
+        const int threads = 256;
+        const int64_t ctas_needed = (rows + 7) / 8;
+        const int64_t cap = (int64_t)sm_count() * 8;   // 8 CTAs of 256 threads fill an SM
+        const unsigned grid = (unsigned)(ctas_needed < cap ? ctas_needed : cap);
+#define KOP_SM_WARP(V, B) softmax_warp_kernel<T, V, B><<<grid, threads, 0, stream>>>(x, bias, y, rows, nvec, xs, ys, scale)
+        if (vpl <= 1) KOP_SM_WARP(1, true);
+        else if (vpl <= 2) KOP_SM_WARP(2, true);
+        else KOP_SM_WARP(4, false);
+#undef KOP_SM_WARP
+        return launch_status();
+    }
+    if (rows > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+    if (vec && cols <= kMaxRegisterRow) {
+        const int nvec = (int)nvec64;
+        // Per-thread vector count: 16 values per thread while the CTA stays within 1024 threads
+        // keeps many CTAs resident; longer rows double the count (and halve the CTA limit).
+        int vpt = 16 / E;
+        while (vpt * E < 64 && (nvec + vpt - 1) / vpt > max_threads_for(vpt * E)) vpt *= 2;
+        const int threads = ((nvec + vpt - 1) / vpt + 31) / 32 * 32;
+#define KOP_SM_BLOCK(V) softmax_block_kernel<T, V><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, nvec, xs, ys, scale)
+        switch (vpt * E) {
+        case 16: KOP_SM_BLOCK(16 / E); break;
+        case 32: KOP_SM_BLOCK(32 / E); break;
+        default: KOP_SM_BLOCK(64 / E); break;
+        }
+#undef KOP_SM_BLOCK
+        return launch_status();
+    }
+    softmax_generic_kernel<T><<<(unsigned)rows, 256, 0, stream>>>(x, bias, y, cols, xs, ys, scale);
+    return launch_status();
+}
+
+}  // namespace
+}  // namespace kop
+
+extern "C" kop_status_t kop_softmax_scale_bias(const void* x, const float* bias, void* y,
+                                               int64_t rows, int64_t cols, int64_t x_row_stride,
+                                               int64_t y_row_stride, float scale,
+                                               kop_dtype_t dtype, kop_stream_t stream)
+{
+    using namespace kop;
+    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    if (x == nullptr || y == nullptr) return KOP_ERR_NULL_POINTER;
+    kop_status_t st = check_rows_cols(rows, cols);
+    if (st != KOP_OK) return st;
+    if ((st = check_row_stride(x_row_stride, cols, rows)) != KOP_OK) return st;
+    if ((st = check_row_stride(y_row_stride, cols, rows)) != KOP_OK) return st;
+    const int esz = elem_size(dtype);
+    if (!aligned_to(x, esz) || !aligned_to(y, esz) || (bias != nullptr && !aligned_to(bias, 4)))
+        return KOP_ERR_MISALIGNED;
+    if (!alias_ok(x, x_row_stride, y, y_row_stride, rows, cols, esz, true)) return KOP_ERR_BAD_ALIAS;
+    if (rows == 0) return KOP_OK;
+    if ((st = check_device()) != KOP_OK) return st;
+    cudaStream_t s = as_stream(stream);
+    return dtype == KOP_F32
+               ? launch_softmax<float>(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale, s)
+               : launch_softmax<__nv_bfloat16>(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale, s);
+}

@@ -1,0 +1,259 @@
+"""Thin Python binding of libkop's C ABI (include/kop.h): argument marshalling only.
+
+Every function has the name of the C entry point it calls, takes torch CUDA tensors (used purely as
+device memory) and passes raw device pointers, shapes, element strides, the dtype tag and the
+current CUDA stream to the library. Output tensors are allocated here when the caller passes none;
+all arithmetic happens inside the CUDA kernels. There is no fallback: if libkop.so has not been
+built (python -m paper_2609_30059_b200.build) importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libkop.so")
+
+KOP_OK = 0
+KOP_F32, KOP_BF16 = 0, 1
+STATUS_NAMES = [
+    "KOP_OK", "KOP_ERR_NULL_POINTER", "KOP_ERR_BAD_SHAPE", "KOP_ERR_BAD_STRIDE",
+    "KOP_ERR_UNSUPPORTED_DTYPE", "KOP_ERR_MISALIGNED", "KOP_ERR_BAD_ALIAS",
+    "KOP_ERR_WORKSPACE_TOO_SMALL", "KOP_ERR_UNSUPPORTED_DEVICE", "KOP_ERR_CUDA", "KOP_ERR_CUBLAS",
+]
+
+
+class KopError(RuntimeError):
+    """A libkop call returned a status other than KOP_OK."""
+
+    def __init__(self, status: int, where: str):
+        self.status = int(status)
+        name = lib().kop_status_string(self.status).decode()
+        super().__init__(f"{where}: {name} ({self.status})")
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """The loaded shared library with argument types declared (raw C-ABI access)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_30059_b200.build`; "
+                          "libkop has no fallback path")
+    L = C.CDLL(LIB_PATH)
+    vp, i64, f32, i32, sz = C.c_void_p, C.c_int64, C.c_float, C.c_int, C.c_size_t
+    L.kop_version.restype = C.c_int
+    L.kop_version.argtypes = []
+    L.kop_status_string.restype = C.c_char_p
+    L.kop_status_string.argtypes = [i32]
+    L.kop_softmax_scale_bias.argtypes = [vp, vp, vp, i64, i64, i64, i64, f32, i32, vp]
+    L.kop_bias_gelu_residual_layernorm.argtypes = [vp] * 8 + [i64] * 5 + [f32, i32, vp]
+    L.kop_bn_relu_avgpool.argtypes = [vp] * 5 + [i64] * 4 + [C.POINTER(i64), C.POINTER(i64), i32, vp]
+    L.kop_ce_loss_rowwise.argtypes = [vp] * 5 + [i64] * 3 + [vp, sz, i32, vp]
+    L.kop_ce_loss_rowwise_workspace_bytes.restype = sz
+    L.kop_ce_loss_rowwise_workspace_bytes.argtypes = [i64, i64, i32]
+    L.kop_rmsnorm.argtypes = [vp, vp, vp, i64, i64, i64, i64, f32, i32, vp]
+    L.kop_silu_mul.argtypes = [vp, vp, i64, i64, i64, i64, i32, vp]
+    L.kop_residual_add.argtypes = [vp, vp, vp, i64, i64, i64, i64, i64, i32, vp]
+    L.kop_rmsnorm_swiglu_residual.argtypes = [vp] * 6 + [i64] * 3 + [f32, vp, sz, i32, vp]
+    L.kop_rmsnorm_swiglu_residual_workspace_bytes.restype = sz
+    L.kop_rmsnorm_swiglu_residual_workspace_bytes.argtypes = [i64, i64, i64, i32]
+    L.kop_mlp_handle_create.argtypes = [C.POINTER(vp)]
+    L.kop_mlp_handle_destroy.argtypes = [vp]
+    for name in ("kop_softmax_scale_bias", "kop_bias_gelu_residual_layernorm", "kop_bn_relu_avgpool",
+                 "kop_ce_loss_rowwise", "kop_rmsnorm", "kop_silu_mul", "kop_residual_add",
+                 "kop_rmsnorm_swiglu_residual", "kop_mlp_handle_create", "kop_mlp_handle_destroy"):
+        getattr(L, name).restype = i32
+    _lib = L
+    return L
+
+
+def _dtype_tag(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return KOP_F32
+    if t.dtype == torch.bfloat16:
+        return KOP_BF16
+    raise TypeError(f"libkop data tensors are float32 or bfloat16, got {t.dtype}")
+
+
+def _rows2d(t: torch.Tensor, name: str):
+    if t.dim() != 2 or (t.shape[1] > 1 and t.stride(1) != 1):
+        raise ValueError(f"{name}: expected a 2-D tensor with unit inner stride")
+    if not t.is_cuda:
+        raise ValueError(f"{name}: expected a CUDA tensor")
+    return t.shape[0], t.shape[1], t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1])
+
+
+def _param(t, name: str, n: int):
+    if t is None:
+        return None
+    if t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous() or t.numel() != n:
+        raise ValueError(f"{name}: expected a contiguous fp32 CUDA vector of {n} elements")
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _check(st: int, where: str):
+    if st != KOP_OK:
+        raise KopError(st, where)
+
+
+def kop_version() -> int:
+    return lib().kop_version()
+
+
+def kop_softmax_scale_bias(x, bias, scale, out=None, stream=None):
+    rows, cols, xs = _rows2d(x, "x")
+    out = torch.empty_like(x) if out is None else out
+    _, _, ys = _rows2d(out, "out")
+    assert out.shape == x.shape and out.dtype == x.dtype
+    _check(lib().kop_softmax_scale_bias(x.data_ptr(), _param(bias, "bias", cols), out.data_ptr(), rows,
+                                        cols, xs, ys, float(scale), _dtype_tag(x), _stream(stream)),
+           "kop_softmax_scale_bias")
+    return out
+
+
+def kop_bias_gelu_residual_layernorm(x, residual, bias, gamma, beta, eps, out=None, mean=None,
+                                     rstd=None, want_stats=True, stream=None):
+    rows, hidden, xs = _rows2d(x, "x")
+    _, _, rs = _rows2d(residual, "residual")
+    assert residual.shape == x.shape and residual.dtype == x.dtype
+    out = torch.empty_like(x) if out is None else out
+    _, _, ys = _rows2d(out, "out")
+    if want_stats:
+        mean = torch.empty(rows, dtype=torch.float32, device=x.device) if mean is None else mean
+        rstd = torch.empty(rows, dtype=torch.float32, device=x.device) if rstd is None else rstd
+    _check(lib().kop_bias_gelu_residual_layernorm(
+        x.data_ptr(), residual.data_ptr(), _param(bias, "bias", hidden), _param(gamma, "gamma", hidden),
+        _param(beta, "beta", hidden), out.data_ptr(),
+        None if mean is None else mean.data_ptr(), None if rstd is None else rstd.data_ptr(),
+        rows, hidden, xs, rs, ys, float(eps), _dtype_tag(x), _stream(stream)),
+        "kop_bias_gelu_residual_layernorm")
+    return out, mean, rstd
+
+
+def kop_bn_relu_avgpool(x, scale, shift, out=None, pooled=None, stream=None):
+    if x.dim() != 4 or not x.is_cuda:
+        raise ValueError("x: expected a 4-D NCHW CUDA tensor")
+    N, Cc, H, W = x.shape
+    out = torch.empty_like(x) if out is None else out
+    pooled = torch.empty((N, Cc), dtype=torch.float32, device=x.device) if pooled is None else pooled
+    xs = (C.c_int64 * 4)(*x.stride())
+    ys = (C.c_int64 * 4)(*out.stride())
+    _check(lib().kop_bn_relu_avgpool(x.data_ptr(), _param(scale, "scale", Cc), _param(shift, "shift", Cc),
+                                     out.data_ptr(), pooled.data_ptr(), N, Cc, H, W, xs, ys,
+                                     _dtype_tag(x), _stream(stream)), "kop_bn_relu_avgpool")
+    return out, pooled
+
+
+def kop_ce_loss_rowwise_workspace_bytes(rows: int, vocab: int, dtype_tag: int) -> int:
+    return lib().kop_ce_loss_rowwise_workspace_bytes(rows, vocab, dtype_tag)
+
+
+def kop_ce_loss_rowwise(logits, labels, loss=None, mean_loss=None, bad_label_count=None,
+                        workspace=None, stream=None):
+    """Returns (loss[rows], mean_loss[1], bad_label_count[1]) as device tensors."""
+    rows, vocab, zs = _rows2d(logits, "logits")
+    if labels.dtype != torch.int32 or not labels.is_cuda or not labels.is_contiguous() or labels.numel() != rows:
+        raise ValueError("labels: expected a contiguous int32 CUDA vector of `rows` elements")
+    dev = logits.device
+    loss = torch.empty(rows, dtype=torch.float32, device=dev) if loss is None else loss
+    mean_loss = torch.empty(1, dtype=torch.float32, device=dev) if mean_loss is None else mean_loss
+    bad_label_count = (torch.empty(1, dtype=torch.int32, device=dev)
+                       if bad_label_count is None else bad_label_count)
+    need = kop_ce_loss_rowwise_workspace_bytes(rows, vocab, _dtype_tag(logits))
+    if workspace is None:
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
+    _check(lib().kop_ce_loss_rowwise(logits.data_ptr(), labels.data_ptr(), loss.data_ptr(),
+                                     mean_loss.data_ptr(), bad_label_count.data_ptr(), rows, vocab, zs,
+                                     workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                     _dtype_tag(logits), _stream(stream)), "kop_ce_loss_rowwise")
+    return loss, mean_loss, bad_label_count
+
+
+def kop_rmsnorm(x, weight, eps, out=None, stream=None):
+    rows, hidden, xs = _rows2d(x, "x")
+    out = torch.empty_like(x) if out is None else out
+    _, _, ys = _rows2d(out, "out")
+    _check(lib().kop_rmsnorm(x.data_ptr(), _param(weight, "weight", hidden), out.data_ptr(), rows, hidden,
+                             xs, ys, float(eps), _dtype_tag(x), _stream(stream)), "kop_rmsnorm")
+    return out
+
+
+def kop_silu_mul(gate_up, out=None, stream=None):
+    rows, two_i, is_ = _rows2d(gate_up, "gate_up")
+    if two_i % 2:
+        raise ValueError("gate_up: the row length must be even ([gate | up])")
+    inter = two_i // 2
+    out = torch.empty((rows, inter), dtype=gate_up.dtype, device=gate_up.device) if out is None else out
+    _, _, os_ = _rows2d(out, "out")
+    _check(lib().kop_silu_mul(gate_up.data_ptr(), out.data_ptr(), rows, inter, is_, os_,
+                              _dtype_tag(gate_up), _stream(stream)), "kop_silu_mul")
+    return out
+
+
+def kop_residual_add(a, b, out=None, stream=None):
+    rows, cols, as_ = _rows2d(a, "a")
+    _, _, bs = _rows2d(b, "b")
+    assert a.shape == b.shape and a.dtype == b.dtype
+    out = torch.empty_like(a) if out is None else out
+    _, _, os_ = _rows2d(out, "out")
+    _check(lib().kop_residual_add(a.data_ptr(), b.data_ptr(), out.data_ptr(), rows, cols, as_, bs, os_,
+                                  _dtype_tag(a), _stream(stream)), "kop_residual_add")
+    return out
+
+
+class MlpHandle:
+    """Owner of the vendor-GEMM handle (kop_mlp_handle_create / kop_mlp_handle_destroy)."""
+
+    def __init__(self):
+        h = C.c_void_p()
+        _check(lib().kop_mlp_handle_create(C.byref(h)), "kop_mlp_handle_create")
+        self.ptr = h.value
+
+    def close(self):
+        if self.ptr:
+            lib().kop_mlp_handle_destroy(self.ptr)
+            self.ptr = None
+
+    def __del__(self):  # pragma: no cover
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def kop_rmsnorm_swiglu_residual_workspace_bytes(rows, hidden, inter, dtype_tag) -> int:
+    return lib().kop_rmsnorm_swiglu_residual_workspace_bytes(rows, hidden, inter, dtype_tag)
+
+
+def kop_rmsnorm_swiglu_residual(handle: MlpHandle, h, rms_weight, w_gate_up, w_down, eps, out=None,
+                                workspace=None, stream=None):
+    rows, hidden, _ = _rows2d(h, "h")
+    two_i, hid2, _ = _rows2d(w_gate_up, "w_gate_up")
+    hid3, inter, _ = _rows2d(w_down, "w_down")
+    if not (h.is_contiguous() and w_gate_up.is_contiguous() and w_down.is_contiguous()):
+        raise ValueError("h, w_gate_up and w_down must be contiguous")
+    if hid2 != hidden or hid3 != hidden or two_i != 2 * inter:
+        raise ValueError("weight shapes must be [2*inter, hidden] and [hidden, inter]")
+    out = torch.empty_like(h) if out is None else out
+    tag = _dtype_tag(h)
+    need = kop_rmsnorm_swiglu_residual_workspace_bytes(rows, hidden, inter, tag)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=h.device)
+    _check(lib().kop_rmsnorm_swiglu_residual(handle.ptr, h.data_ptr(), _param(rms_weight, "rms_weight", hidden),
+                                             w_gate_up.data_ptr(), w_down.data_ptr(), out.data_ptr(),
+                                             rows, hidden, inter, float(eps), workspace.data_ptr(),
+                                             workspace.numel(), tag, _stream(stream)),
+           "kop_rmsnorm_swiglu_residual")
+    return out

@@ -1,0 +1,96 @@
+"""Seeded synthetic inputs for the fused segments: shapes and value distributions only.
+
+This module holds none of the segments' arithmetic; it only draws tensors. Values are drawn in
+fp32 with torch's generator on the requested device, in a fixed order per segment, and then cast
+to the data dtype, so the CUDA path and the CPU oracle see identical bit patterns (the oracle gets
+a host copy). In N(a, b) the second parameter is the standard deviation.
+"""
+from __future__ import annotations
+
+import torch
+
+SEEDS = (0, 42, 123, 1337, 2609)
+
+# Full-size workloads (the benchmark configurations).
+CONFIGS = {
+    "softmax_small": dict(rows=128, cols=512, dtype=torch.float32, scale=0.125),
+    "softmax_large": dict(rows=131072, cols=512, dtype=torch.float32, scale=0.125),
+    "layernorm": dict(rows=8192, hidden=4096, dtype=torch.bfloat16, eps=1e-5),
+    "bn_pool": dict(N=64, C=256, H=56, W=56, dtype=torch.float32),
+    "ce_loss": dict(rows=32768, vocab=32000, dtype=torch.bfloat16),
+    "mlp": dict(rows=16384, hidden=4096, inter=14336, dtype=torch.bfloat16, eps=1e-6),
+}
+
+
+def _gen(seed: int, device) -> torch.Generator:
+    g = torch.Generator(device=device)
+    g.manual_seed(int(seed))
+    return g
+
+
+def _normal(shape, mean, std, g, device):
+    return torch.randn(shape, generator=g, device=device, dtype=torch.float32) * std + mean
+
+
+def _uniform(shape, lo, hi, g, device):
+    return torch.rand(shape, generator=g, device=device, dtype=torch.float32) * (hi - lo) + lo
+
+
+def softmax_inputs(rows, cols, dtype=torch.float32, seed=0, device="cpu"):
+    """x ~ N(0,1) [rows, cols]; bias fp32 ~ N(0,0.1) [cols]."""
+    g = _gen(seed, device)
+    x = _normal((rows, cols), 0.0, 1.0, g, device).to(dtype)
+    bias = _normal((cols,), 0.0, 0.1, g, device)
+    return x, bias
+
+
+def layernorm_inputs(rows, hidden, dtype=torch.bfloat16, seed=0, device="cpu"):
+    """x, residual ~ N(0,1); bias ~ N(0,0.1); gamma ~ N(1,0.02); beta ~ N(0,0.02) (params fp32)."""
+    g = _gen(seed, device)
+    x = _normal((rows, hidden), 0.0, 1.0, g, device).to(dtype)
+    residual = _normal((rows, hidden), 0.0, 1.0, g, device).to(dtype)
+    bias = _normal((hidden,), 0.0, 0.1, g, device)
+    gamma = _normal((hidden,), 1.0, 0.02, g, device)
+    beta = _normal((hidden,), 0.0, 0.02, g, device)
+    return x, residual, bias, gamma, beta
+
+
+def bn_pool_inputs(N, C, H, W, dtype=torch.float32, seed=0, device="cpu"):
+    """x ~ N(0,1) NCHW; scale ~ U(0.5,1.5); shift ~ N(0,0.1) (params fp32)."""
+    g = _gen(seed, device)
+    x = _normal((N, C, H, W), 0.0, 1.0, g, device).to(dtype)
+    scale = _uniform((C,), 0.5, 1.5, g, device)
+    shift = _normal((C,), 0.0, 0.1, g, device)
+    return x, scale, shift
+
+
+def ce_inputs(rows, vocab, dtype=torch.bfloat16, seed=0, device="cpu"):
+    """logits ~ N(0,2) [rows, vocab]; labels int32 ~ U[0, vocab)."""
+    g = _gen(seed, device)
+    logits = _normal((rows, vocab), 0.0, 2.0, g, device).to(dtype)
+    labels = torch.randint(0, vocab, (rows,), generator=g, device=device, dtype=torch.int64).to(torch.int32)
+    return logits, labels
+
+
+def mlp_inputs(rows, hidden, inter, dtype=torch.bfloat16, seed=0, device="cpu"):
+    """h ~ N(0,1); rms weight fp32 ~ N(1,0.02); W_gate_up [2*inter, hidden], W_down [hidden, inter] ~ N(0,0.02)."""
+    g = _gen(seed, device)
+    h = _normal((rows, hidden), 0.0, 1.0, g, device).to(dtype)
+    rms_weight = _normal((hidden,), 1.0, 0.02, g, device)
+    w_gate_up = _normal((2 * inter, hidden), 0.0, 0.02, g, device).to(dtype)
+    w_down = _normal((hidden, inter), 0.0, 0.02, g, device).to(dtype)
+    return h, rms_weight, w_gate_up, w_down
+
+
+def gate_up_inputs(rows, inter, dtype=torch.bfloat16, seed=0, device="cpu", std=1.0):
+    """A stand-in [rows, 2*inter] GEMM output ~ N(0, std) for testing the SwiGLU epilogue alone."""
+    g = _gen(seed, device)
+    return _normal((rows, 2 * inter), 0.0, std, g, device).to(dtype)
+
+
+def pair_inputs(rows, cols, dtype=torch.bfloat16, seed=0, device="cpu"):
+    """Two ~N(0,1) tensors for the residual add."""
+    g = _gen(seed, device)
+    a = _normal((rows, cols), 0.0, 1.0, g, device).to(dtype)
+    b = _normal((rows, cols), 0.0, 1.0, g, device).to(dtype)
+    return a, b

@@ -1,0 +1,437 @@
+"""GPU parity: every libkop segment, called through the C ABI, against the float64 CPU oracle on
+the same seeded inputs. Five seeds at sizes that span several CTAs / tiles plus ragged tails, the
+full benchmark shapes on seed 0, edge cases (empty, one element, odd lengths, misaligned bases,
+strided rows, in-place, masked columns, bad labels), guard bands around every output, and
+run-to-run bit equality.
+
+Tolerance: |got - ref| <= tol * max(1, |ref|), tol = 1e-5 for fp32 data and 2e-2 for bf16 data;
+bf16 outputs are additionally held to about two bf16 steps of the float64 value."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import kopref
+from paper_2609_30059_b200 import build as kbuild
+from paper_2609_30059_b200 import synth
+from tests._util import Guarded, assert_bf16_tight, assert_close, to_f64, tol_of
+
+pytestmark = pytest.mark.gpu
+
+SEEDS = synth.SEEDS
+F32, BF16 = torch.float32, torch.bfloat16
+
+
+@pytest.fixture(scope="module")
+def kop():
+    kbuild.build()
+    from paper_2609_30059_b200 import kop as K
+    return K
+
+
+def host(t):
+    return t.detach().cpu()
+
+
+# ------------------------------------------------------------------------------------------ softmax
+
+SOFTMAX_SHAPES = [
+    (128, 512, F32),       # benchmark small config: warp-per-row
+    (1000, 512, F32),
+    (333, 96, F32),        # partial last vector group in the warp
+    (257, 2048, F32),      # CTA-per-row, row in registers
+    (19, 16384, F32),      # longest register-resident row
+    (7, 20000, F32),       # beyond registers: generic
+    (37, 513, F32),        # odd length: scalar
+    (64, 1, F32),
+    (515, 1000, BF16),
+    (129, 4096, BF16),
+    (33, 777, BF16),
+]
+
+
+@pytest.mark.parametrize("rows,cols,dtype", SOFTMAX_SHAPES)
+@pytest.mark.parametrize("seed", SEEDS)
+def test_softmax_parity(kop, rows, cols, dtype, seed):
+    x, bias = synth.softmax_inputs(rows, cols, dtype, seed, "cuda")
+    out = Guarded((rows, cols), dtype)
+    kop.kop_softmax_scale_bias(x, bias, 0.125, out=out.t)
+    ref = kopref.softmax_scale_bias(host(x), host(bias), 0.125, threads=None)
+    assert_close(out.t, ref, tol_of(dtype), "softmax")
+    out.check("softmax")
+    sums = to_f64(out.t).sum(axis=1)
+    assert np.all(np.abs(sums - 1.0) <= (1e-5 if dtype == F32 else 2e-2))
+
+
+def test_softmax_large_config_seed0(kop):
+    c = synth.CONFIGS["softmax_large"]
+    x, bias = synth.softmax_inputs(c["rows"], c["cols"], c["dtype"], 0, "cuda")
+    y = kop.kop_softmax_scale_bias(x, bias, c["scale"])
+    ref = kopref.softmax_scale_bias(host(x), host(bias), c["scale"], threads=None)
+    assert_close(y, ref, 1e-5, "softmax large")
+
+
+def test_softmax_options(kop):
+    x, bias = synth.softmax_inputs(300, 512, F32, 1, "cuda")
+    # no bias
+    y = kop.kop_softmax_scale_bias(x, None, 0.5)
+    assert_close(y, kopref.softmax_scale_bias(host(x), None, 0.5), 1e-5, "no bias")
+    # masked columns (-inf bias) give exact zeros
+    b2 = bias.clone()
+    b2[::3] = float("-inf")
+    y = kop.kop_softmax_scale_bias(x, b2, 0.125)
+    assert_close(y, kopref.softmax_scale_bias(host(x), host(b2), 0.125), 1e-5, "masked")
+    assert bool((y[:, ::3] == 0).all())
+    # in place
+    ref = kopref.softmax_scale_bias(host(x), host(bias), 0.125)
+    xi = x.clone()
+    kop.kop_softmax_scale_bias(xi, bias, 0.125, out=xi)
+    assert_close(xi, ref, 1e-5, "in place")
+    # strided rows (a column slice of a wider matrix), vector-aligned and not
+    wide = torch.zeros((300, 1024), dtype=F32, device="cuda")
+    wide[:, 256:768] = x
+    ow = torch.full((300, 640), 7.0, dtype=F32, device="cuda")
+    kop.kop_softmax_scale_bias(wide[:, 256:768], bias, 0.125, out=ow[:, 64:576])
+    assert_close(ow[:, 64:576], ref, 1e-5, "strided")
+    assert bool((ow[:, :64] == 7.0).all()) and bool((ow[:, 576:] == 7.0).all())
+    wide[:, 257:769] = x
+    y = kop.kop_softmax_scale_bias(wide[:, 257:769], bias, 0.125)         # misaligned base: scalar path
+    assert_close(y, ref, 1e-5, "misaligned")
+    # empty
+    e = torch.empty((0, 512), dtype=F32, device="cuda")
+    assert kop.kop_softmax_scale_bias(e, bias, 0.125).shape == (0, 512)
+    # determinism
+    a = kop.kop_softmax_scale_bias(x, bias, 0.125)
+    b = kop.kop_softmax_scale_bias(x, bias, 0.125)
+    assert torch.equal(a, b)
+
+
+# ------------------------------------------------------------------------------------------ LayerNorm
+
+LN_SHAPES = [
+    (2048, 4096, BF16),    # benchmark row length, >= 4 waves of CTAs
+    (300, 4096, F32),
+    (129, 1024, BF16),
+    (65, 256, BF16),
+    (33, 8192, BF16),
+    (17, 16384, F32),      # longest register-resident row
+    (9, 20480, BF16),      # generic
+    (21, 513, F32),        # scalar
+    (40, 1000, BF16),      # 125 vectors: ragged CTA
+    (5, 1, F32),
+]
+
+
+@pytest.mark.parametrize("rows,hidden,dtype", LN_SHAPES)
+@pytest.mark.parametrize("seed", SEEDS)
+def test_layernorm_parity(kop, rows, hidden, dtype, seed):
+    x, r, b, g, be = synth.layernorm_inputs(rows, hidden, dtype, seed, "cuda")
+    out = Guarded((rows, hidden), dtype)
+    mean = Guarded((rows,), F32)
+    rstd = Guarded((rows,), F32)
+    kop.kop_bias_gelu_residual_layernorm(x, r, b, g, be, 1e-5, out=out.t, mean=mean.t, rstd=rstd.t)
+    ry, rm, rr = kopref.bias_gelu_residual_layernorm(host(x), host(r), host(b), host(g), host(be), 1e-5,
+                                                     threads=None)
+    tol = tol_of(dtype)
+    if hidden == 1:
+        # var = 0: y = beta exactly, rstd = 1/sqrt(eps) ~ 316: only the relative rule applies there
+        assert_close(out.t, ry, tol, "ln y (hidden 1)")
+    else:
+        assert_close(out.t, ry, tol, "ln y")
+    assert_close(mean.t, rm, tol, "ln mean")
+    assert_close(rstd.t, rr, tol, "ln rstd")
+    # statistics are fp32 whatever the data dtype: hold them to a tighter, informational-grade bound
+    assert_close(mean.t, rm, 1e-3 if dtype == BF16 else 1e-5, "ln mean (tight)")
+    assert_close(rstd.t, rr, 1e-3 if dtype == BF16 else 1e-5, "ln rstd (tight)")
+    if dtype == BF16:
+        assert_bf16_tight(out.t, ry, "ln y", floor=8e-3)
+    for gd in (out, mean, rstd):
+        gd.check("ln")
+
+
+def test_layernorm_full_config_seed0(kop):
+    c = synth.CONFIGS["layernorm"]
+    x, r, b, g, be = synth.layernorm_inputs(c["rows"], c["hidden"], c["dtype"], 0, "cuda")
+    y, mean, rstd = kop.kop_bias_gelu_residual_layernorm(x, r, b, g, be, c["eps"])
+    ry, rm, rr = kopref.bias_gelu_residual_layernorm(host(x), host(r), host(b), host(g), host(be), c["eps"],
+                                                     threads=None)
+    assert_close(y, ry, 2e-2, "ln full y")
+    assert_close(mean, rm, 2e-2, "ln full mean")
+    assert_close(rstd, rr, 2e-2, "ln full rstd")
+    assert_bf16_tight(y, ry, "ln full y", floor=8e-3)
+    y2, m2, r2 = kop.kop_bias_gelu_residual_layernorm(x, r, b, g, be, c["eps"])
+    assert torch.equal(y, y2) and torch.equal(mean, m2) and torch.equal(rstd, r2)
+
+
+def test_layernorm_options(kop):
+    x, r, b, g, be = synth.layernorm_inputs(100, 4096, BF16, 3, "cuda")
+    ry, rm, rr = kopref.bias_gelu_residual_layernorm(host(x), host(r), host(b), host(g), host(be), 1e-5)
+    # no statistics outputs
+    y, m, s = kop.kop_bias_gelu_residual_layernorm(x, r, b, g, be, 1e-5, want_stats=False)
+    assert m is None and s is None
+    assert_close(y, ry, 2e-2, "no stats")
+    # in place over x, and over the residual
+    xi = x.clone()
+    kop.kop_bias_gelu_residual_layernorm(xi, r, b, g, be, 1e-5, out=xi)
+    assert_close(xi, ry, 2e-2, "in place x")
+    ri = r.clone()
+    kop.kop_bias_gelu_residual_layernorm(x, ri, b, g, be, 1e-5, out=ri)
+    assert_close(ri, ry, 2e-2, "in place residual")
+    # strided inputs and output
+    wx = torch.zeros((100, 8192), dtype=BF16, device="cuda")
+    wx[:, 4096:] = x
+    wr = torch.zeros((100, 4104), dtype=BF16, device="cuda")
+    wr[:, :4096] = r
+    wo = torch.zeros((100, 4096 + 64), dtype=BF16, device="cuda")
+    kop.kop_bias_gelu_residual_layernorm(wx[:, 4096:], wr[:, :4096], b, g, be, 1e-5, out=wo[:, 64:])
+    assert_close(wo[:, 64:], ry, 2e-2, "strided")
+    assert bool((wo[:, :64] == 0).all())
+    # misaligned base -> scalar kernel
+    wx2 = torch.zeros((100, 4099), dtype=BF16, device="cuda")
+    wx2[:, 3:] = x
+    y, _, _ = kop.kop_bias_gelu_residual_layernorm(wx2[:, 3:], r, b, g, be, 1e-5)
+    assert_close(y, ry, 2e-2, "misaligned")
+    e = torch.empty((0, 4096), dtype=BF16, device="cuda")
+    y, _, _ = kop.kop_bias_gelu_residual_layernorm(e, e, b, g, be, 1e-5)
+    assert y.shape == (0, 4096)
+
+
+# ------------------------------------------------------------------------------------------ BN + ReLU + pool
+
+BN_SHAPES = [
+    (8, 256, 56, 56, F32),     # benchmark plane
+    (3, 5, 56, 56, BF16),
+    (4, 16, 7, 7, F32),        # small odd plane: warp, scalar
+    (4, 16, 14, 14, F32),      # small plane: warp, vector
+    (2, 3, 112, 112, F32),     # multi-trip plane
+    (2, 7, 33, 35, F32),       # large odd plane: scalar CTA
+    (5, 3, 1, 1, F32),
+    (2, 8, 64, 64, BF16),
+]
+
+
+@pytest.mark.parametrize("N,C,H,W,dtype", BN_SHAPES)
+@pytest.mark.parametrize("seed", SEEDS)
+def test_bn_relu_avgpool_parity(kop, N, C, H, W, dtype, seed):
+    x, scale, shift = synth.bn_pool_inputs(N, C, H, W, dtype, seed, "cuda")
+    out = Guarded((N, C, H, W), dtype)
+    pooled = Guarded((N, C), F32)
+    kop.kop_bn_relu_avgpool(x, scale, shift, out=out.t, pooled=pooled.t)
+    ry, rp = kopref.bn_relu_avgpool(host(x), host(scale), host(shift), threads=None)
+    tol = tol_of(dtype)
+    assert_close(out.t, ry, tol, "bn y")
+    assert_close(pooled.t, rp, tol, "bn pooled")
+    assert_close(pooled.t, rp, 1e-5, "bn pooled (fp32-grade: pooled sums unrounded activations)")
+    if dtype == BF16:
+        assert_bf16_tight(out.t, ry, "bn y", floor=1e-6)
+    out.check("bn y")
+    pooled.check("bn pooled")
+
+
+def test_bn_full_config_seed0_and_options(kop):
+    c = synth.CONFIGS["bn_pool"]
+    x, scale, shift = synth.bn_pool_inputs(c["N"], c["C"], c["H"], c["W"], c["dtype"], 0, "cuda")
+    y, p = kop.kop_bn_relu_avgpool(x, scale, shift)
+    ry, rp = kopref.bn_relu_avgpool(host(x), host(scale), host(shift), threads=None)
+    assert_close(y, ry, 1e-5, "bn full y")
+    assert_close(p, rp, 1e-5, "bn full pooled")
+    y2, p2 = kop.kop_bn_relu_avgpool(x, scale, shift)
+    assert torch.equal(y, y2) and torch.equal(p, p2)
+    # in place
+    xi = x[:4].clone()
+    _, pi = kop.kop_bn_relu_avgpool(xi, scale, shift, out=xi)
+    assert_close(xi, ry[:4], 1e-5, "bn in place")
+    assert_close(pi, rp[:4], 1e-5, "bn in place pooled")
+    # NaN propagates through ReLU into the activation and the pooled mean
+    xn = x[:1].clone()
+    xn[0, 3, 5, 7] = float("nan")
+    yn, pn = kop.kop_bn_relu_avgpool(xn, scale, shift)
+    assert bool(torch.isnan(yn[0, 3, 5, 7])) and bool(torch.isnan(pn[0, 3]))
+    assert int(torch.isnan(pn).sum()) == 1
+    # channels-last strides are rejected, not misread
+    with pytest.raises(kop.KopError) as ei:
+        kop.kop_bn_relu_avgpool(x[:2].contiguous(memory_format=torch.channels_last), scale, shift,
+                                out=torch.empty_like(x[:2]))
+    assert ei.value.status == 3
+    e = torch.empty((0, 256, 56, 56), dtype=F32, device="cuda")
+    ye, pe = kop.kop_bn_relu_avgpool(e, scale, shift)
+    assert ye.shape == e.shape and pe.shape == (0, 256)
+
+
+# ------------------------------------------------------------------------------------------ cross-entropy
+
+CE_SHAPES = [
+    (2048, 32000, BF16),   # benchmark row length
+    (300, 32000, F32),
+    (257, 4096, BF16),
+    (100, 50264, BF16),    # multi-batch rows (more than 16 vectors per thread)
+    (64, 131072, BF16),
+    (33, 1000, F32),
+    (21, 32001, BF16),     # odd vocab: scalar
+    (9, 1, F32),
+    (5, 8, BF16),
+]
+
+
+@pytest.mark.parametrize("rows,vocab,dtype", CE_SHAPES)
+@pytest.mark.parametrize("seed", SEEDS)
+def test_ce_parity(kop, rows, vocab, dtype, seed):
+    if rows * vocab > 40_000_000 and seed not in (0, 42):
+        pytest.skip("large shape: two seeds keep the CPU oracle time bounded")
+    z, lab = synth.ce_inputs(rows, vocab, dtype, seed, "cuda")
+    loss = Guarded((rows,), F32)
+    mean = Guarded((1,), F32)
+    bad = Guarded((1,), torch.int32)
+    kop.kop_ce_loss_rowwise(z, lab, loss=loss.t, mean_loss=mean.t, bad_label_count=bad.t)
+    rl, rmean, rbad = kopref.ce_loss_rowwise(host(z), host(lab), threads=None)
+    tol = tol_of(dtype)
+    assert_close(loss.t, rl, tol, "ce loss")
+    assert_close(mean.t, np.array([rmean]), tol, "ce mean")
+    # the kernel computes in fp32 whatever the logits' dtype: hold it to fp32-grade accuracy too
+    assert_close(loss.t, rl, 2e-5, "ce loss (fp32-grade)")
+    assert_close(mean.t, np.array([rmean]), 2e-5, "ce mean (fp32-grade)")
+    assert int(bad.t.item()) == rbad == 0
+    for gd in (loss, mean, bad):
+        gd.check("ce")
+
+
+def test_ce_full_config_sampled_rows_and_mean(kop):
+    c = synth.CONFIGS["ce_loss"]
+    z, lab = synth.ce_inputs(c["rows"], c["vocab"], c["dtype"], 0, "cuda")
+    loss, mean, bad = kop.kop_ce_loss_rowwise(z, lab)
+    idx = torch.from_numpy(np.random.default_rng(0).choice(c["rows"], 1024, replace=False)).to("cuda")
+    idx = torch.cat([idx, torch.tensor([0, c["rows"] - 1], device="cuda")])
+    rl, _, _ = kopref.ce_loss_rowwise(host(z[idx]), host(lab[idx]), threads=None)
+    assert_close(loss[idx], rl, 2e-2, "ce full sampled rows")
+    assert_close(loss[idx], rl, 2e-5, "ce full sampled rows (fp32-grade)")
+    # property that holds at any size: the mean output is the mean of the per-row losses
+    assert abs(float(mean.item()) - to_f64(loss).mean()) <= 1e-5 * 13
+    assert int(bad.item()) == 0
+    # loss >= 0 and close to ln V + sigma^2/2 on average for N(0,2) logits
+    assert float(loss.min().item()) >= 0.0
+    assert abs(float(mean.item()) - (np.log(c["vocab"]) + 2.0)) < 0.1
+    l2, m2, _ = kop.kop_ce_loss_rowwise(z, lab)
+    assert torch.equal(loss, l2) and torch.equal(mean, m2)
+
+
+def test_ce_options(kop):
+    z, lab = synth.ce_inputs(200, 4096, BF16, 5, "cuda")
+    # bad labels: NaN loss for those rows, counted, mean NaN
+    lab2 = lab.clone()
+    lab2[3] = -1
+    lab2[77] = 4096
+    loss, mean, bad = kop.kop_ce_loss_rowwise(z, lab2)
+    rl, rmean, rbad = kopref.ce_loss_rowwise(host(z), host(lab2))
+    assert int(bad.item()) == rbad == 2
+    assert bool(torch.isnan(loss[3])) and bool(torch.isnan(loss[77])) and bool(torch.isnan(mean[0]))
+    assert_close(loss, rl, 2e-5, "ce with bad labels")
+    # strided rows; workspace reuse across calls without clearing it
+    wide = torch.zeros((200, 8192), dtype=BF16, device="cuda")
+    wide[:, 4096:] = z
+    ws = torch.full((64,), 0xFF, dtype=torch.uint8, device="cuda")     # garbage on entry
+    for _ in range(3):
+        loss, mean, bad = kop.kop_ce_loss_rowwise(wide[:, 4096:], lab, workspace=ws)
+        rl, rmean, _ = kopref.ce_loss_rowwise(host(z), host(lab))
+        assert_close(loss, rl, 2e-5, "ce strided")
+        assert_close(mean, np.array([rmean]), 2e-5, "ce strided mean")
+    # extreme logits: no overflow, -inf entries allowed
+    zz = z.clone().float()
+    zz[:, 0] = 3.0e4
+    zz[:, 1] = float("-inf")
+    zz = zz.to(BF16)
+    lab_e = lab.clamp(min=2)                       # keep the label off the -inf column
+    loss, _, _ = kop.kop_ce_loss_rowwise(zz, lab_e)
+    rl, _, _ = kopref.ce_loss_rowwise(host(zz), host(lab_e))
+    assert_close(loss, rl, 2e-2, "ce extreme")
+    # uniform row -> ln V
+    u = torch.full((4, 32000), -1.75, dtype=BF16, device="cuda")
+    loss, mean, _ = kop.kop_ce_loss_rowwise(u, torch.tensor([0, 5, 31999, 16000], dtype=torch.int32, device="cuda"))
+    assert torch.allclose(loss, torch.full_like(loss, float(np.log(32000))), rtol=0, atol=2e-5)
+    e = torch.empty((0, 4096), dtype=BF16, device="cuda")
+    l0, _, _ = kop.kop_ce_loss_rowwise(e, torch.empty((0,), dtype=torch.int32, device="cuda"))
+    assert l0.shape == (0,)
+
+
+# ------------------------------------------------------------------------------------------ MLP pieces
+
+RMS_SHAPES = [(2048, 4096, BF16), (300, 4096, F32), (65, 512, BF16), (17, 16384, BF16),
+              (9, 20480, F32), (21, 1001, BF16), (7, 1, F32)]
+
+
+@pytest.mark.parametrize("rows,hidden,dtype", RMS_SHAPES)
+@pytest.mark.parametrize("seed", SEEDS)
+def test_rmsnorm_parity(kop, rows, hidden, dtype, seed):
+    h, w, _, _ = synth.mlp_inputs(rows, hidden, 8, dtype, seed, "cuda")
+    out = Guarded((rows, hidden), dtype)
+    kop.kop_rmsnorm(h, w, 1e-6, out=out.t)
+    ref = kopref.rmsnorm(host(h), host(w), 1e-6, threads=None)
+    assert_close(out.t, ref, tol_of(dtype), "rmsnorm")
+    if dtype == BF16:
+        assert_bf16_tight(out.t, ref, "rmsnorm", floor=1e-6)
+    out.check("rmsnorm")
+
+
+SILU_SHAPES = [(512, 14336, BF16), (100, 14336, F32), (33, 1000, BF16), (17, 1001, F32),
+               (64, 8, BF16), (5, 1, F32)]
+
+
+@pytest.mark.parametrize("rows,inter,dtype", SILU_SHAPES)
+@pytest.mark.parametrize("seed", SEEDS)
+def test_silu_mul_parity(kop, rows, inter, dtype, seed):
+    gu = synth.gate_up_inputs(rows, inter, dtype, seed, "cuda", std=3.0)
+    out = Guarded((rows, inter), dtype)
+    kop.kop_silu_mul(gu, out=out.t)
+    ref = kopref.silu_mul(host(gu), threads=None)
+    assert_close(out.t, ref, tol_of(dtype), "silu_mul")
+    if dtype == BF16:
+        assert_bf16_tight(out.t, ref, "silu_mul", floor=1e-6)
+    out.check("silu_mul")
+
+
+ADD_SHAPES = [(2048, 4096, BF16), (100, 4096, F32), (33, 1001, BF16), (1, 7, F32)]
+
+
+@pytest.mark.parametrize("rows,cols,dtype", ADD_SHAPES)
+@pytest.mark.parametrize("seed", SEEDS)
+def test_residual_add_parity(kop, rows, cols, dtype, seed):
+    a, b = synth.pair_inputs(rows, cols, dtype, seed, "cuda")
+    out = Guarded((rows, cols), dtype)
+    kop.kop_residual_add(a, b, out=out.t)
+    ref = kopref.residual_add(host(a), host(b), threads=None)
+    if dtype == F32:
+        # one fp32 add, correctly rounded: equal to the float64 sum rounded to fp32
+        assert np.array_equal(to_f64(out.t), ref.astype(np.float32).astype(np.float64))
+    else:
+        assert_close(out.t, ref, 2e-2, "residual_add")
+        assert_bf16_tight(out.t, ref, "residual_add", floor=1e-6)
+    out.check("residual_add")
+
+
+def test_mlp_pieces_options(kop):
+    h, w, _, _ = synth.mlp_inputs(64, 4096, 8, BF16, 9, "cuda")
+    ref = kopref.rmsnorm(host(h), host(w), 1e-6)
+    hi = h.clone()
+    kop.kop_rmsnorm(hi, w, 1e-6, out=hi)
+    assert_close(hi, ref, 2e-2, "rmsnorm in place")
+    wide = torch.zeros((64, 4096 + 72), dtype=BF16, device="cuda")
+    wide[:, 72:] = h
+    assert_close(kop.kop_rmsnorm(wide[:, 72:], w, 1e-6), ref, 2e-2, "rmsnorm strided")
+    wide2 = torch.zeros((64, 4097), dtype=BF16, device="cuda")
+    wide2[:, 1:] = h
+    assert_close(kop.kop_rmsnorm(wide2[:, 1:], w, 1e-6), ref, 2e-2, "rmsnorm misaligned")
+    # silu_mul on a strided view and residual add in place, with strided operands
+    gu = synth.gate_up_inputs(50, 1024, BF16, 2, "cuda", std=3.0)
+    wg = torch.zeros((50, 4096), dtype=BF16, device="cuda")
+    wg[:, 1024:3072] = gu
+    assert_close(kop.kop_silu_mul(wg[:, 1024:3072]), kopref.silu_mul(host(gu)), 2e-2, "silu strided")
+    a, b = synth.pair_inputs(50, 1024, BF16, 2, "cuda")
+    rs = kopref.residual_add(host(a), host(b))
+    ai = a.clone()
+    kop.kop_residual_add(ai, b, out=ai)
+    assert_close(ai, rs, 2e-2, "add in place")
+    wa = torch.zeros((50, 2048), dtype=BF16, device="cuda")
+    wa[:, 8:1032] = a
+    assert_close(kop.kop_residual_add(wa[:, 8:1032], b), rs, 2e-2, "add strided")
+    for fn, args in ((kop.kop_rmsnorm, (torch.empty((0, 64), dtype=BF16, device="cuda"), w[:64].contiguous(), 1e-6)),
+                     (kop.kop_silu_mul, (torch.empty((0, 64), dtype=BF16, device="cuda"),)),
+                     (kop.kop_residual_add, (torch.empty((0, 64), dtype=BF16, device="cuda"),) * 2)):
+        assert fn(*args).shape[0] == 0
