@@ -1,0 +1,620 @@
+#!/usr/bin/env python
+"""Benchmark of libkop's fused segments on B200.
+
+One STEP is one pass of the whole fused hot path over one batch of seeded synthetic input:
+  softmax (small + large), bias+GELU+residual+LayerNorm, BN+ReLU+avgpool, row-wise cross-entropy,
+  RMSNorm, SiLU*up, residual add — each launched through the C ABI on its benchmark shape with
+  inputs resident in HBM (the SiLU*up and residual inputs are the actual cuBLAS outputs of the MLP
+  chain) and bracketed by CUDA events.
+
+value (GB/s) = algorithmic bytes of the fused kernels (every input read once, every output written
+once) / the time those kernels took inside the K timed steps. Every kernel's working set is far
+larger than L2 except the small softmax, and consecutive kernels evict each other, so all launches
+run cold. After the timed region the whole transformer-MLP segment (RMSNorm -> cuBLAS -> SiLU*up ->
+cuBLAS -> residual) is replayed as one CUDA graph and reported under "mlp_segment_graph", together
+with the fused kernels' numbers when they alternate with that graph: the preserved vendor GEMMs
+drive the GPU into its power cap, so those show the same kernels at the lower SM clock they see
+inside a model. The vendor GEMMs themselves are not part of `value`.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+With N > 1 (launched by torch.distributed.run) every rank runs an independent replica on its own
+GPU (the path has no exchange step): weak scaling, value = sum of bytes / max time over ranks.
+--impl reference times the float64 CPU oracle, as it stands, on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2609_30059_b200 import synth  # noqa: E402
+
+METRIC = "achieved HBM GB/s over the fused segments (algorithmic bytes / device time)"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+# ----------------------------------------------------------------------------- workload description
+
+def segment_bytes():
+    """Algorithmic bytes and element counts per fused kernel at the benchmark shapes."""
+    c = synth.CONFIGS
+    out = {}
+    s, L = c["softmax_small"], c["softmax_large"]
+    out["softmax_small"] = dict(bytes=2 * s["rows"] * s["cols"] * 4 + s["cols"] * 4, elems=s["rows"] * s["cols"])
+    out["softmax_large"] = dict(bytes=2 * L["rows"] * L["cols"] * 4 + L["cols"] * 4, elems=L["rows"] * L["cols"])
+    n = c["layernorm"]
+    out["layernorm"] = dict(bytes=3 * n["rows"] * n["hidden"] * 2 + 3 * n["hidden"] * 4 + 2 * n["rows"] * 4,
+                            elems=n["rows"] * n["hidden"])
+    b = c["bn_pool"]
+    e = b["N"] * b["C"] * b["H"] * b["W"]
+    out["bn_pool"] = dict(bytes=2 * e * 4 + 2 * b["C"] * 4 + b["N"] * b["C"] * 4, elems=e)
+    z = c["ce_loss"]
+    out["ce_loss"] = dict(bytes=z["rows"] * z["vocab"] * 2 + 2 * z["rows"] * 4 + 4, elems=z["rows"] * z["vocab"])
+    m = c["mlp"]
+    out["rmsnorm"] = dict(bytes=2 * m["rows"] * m["hidden"] * 2 + m["hidden"] * 4, elems=m["rows"] * m["hidden"])
+    out["silu_mul"] = dict(bytes=3 * m["rows"] * m["inter"] * 2, elems=m["rows"] * m["inter"])
+    out["residual_add"] = dict(bytes=3 * m["rows"] * m["hidden"] * 2, elems=m["rows"] * m["hidden"])
+    return out
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+# ----------------------------------------------------------------------------- clocks sampling
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device: int):
+        self.proc = None
+        self.path = None
+        try:
+            uuid = str(torch.cuda.get_device_properties(device).uuid)
+            self.sel = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+        except Exception:
+            self.sel = str(device)
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", self.sel, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "20"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                p = [t.strip() for t in line.split(",")]
+                if len(p) < 7:
+                    continue
+                try:
+                    sm.append(float(p[0]))
+                    mx.append(float(p[1]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[3:7]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.remove(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ----------------------------------------------------------------------------- our arm
+
+class Workload:
+    """All benchmark inputs and outputs resident on one GPU, plus the MLP-segment CUDA graph."""
+
+    ORDER = ["softmax_small", "softmax_large", "layernorm", "bn_pool", "ce_loss", "rmsnorm", "silu_mul", "residual_add"]
+
+    def __init__(self, kop, device, seed, only=None, rows_div=1):
+        """only: build just these segments (None = all, plus the MLP segment); rows_div cuts the row
+        (or image) count of every segment, for small profiler captures."""
+        self.kop = kop
+        c = synth.CONFIGS
+        dev = device
+        want = set(self.ORDER) | {"mlp"} if only is None else set(only)
+        cut = lambda r: max(1, r // rows_div)  # noqa: E731
+        self.c = c
+        self.graph = None
+        if "softmax_small" in want:
+            s = c["softmax_small"]
+            self.sx, self.sb = synth.softmax_inputs(s["rows"], s["cols"], s["dtype"], seed, dev)
+            self.sy = torch.empty_like(self.sx)
+        if "softmax_large" in want:
+            L = c["softmax_large"]
+            self.lx, self.lb = synth.softmax_inputs(cut(L["rows"]), L["cols"], L["dtype"], seed, dev)
+            self.ly = torch.empty_like(self.lx)
+        if "layernorm" in want:
+            n = c["layernorm"]
+            self.nx, self.nr, self.nb, self.ng, self.nbe = synth.layernorm_inputs(cut(n["rows"]), n["hidden"], n["dtype"], seed, dev)
+            self.ny = torch.empty_like(self.nx)
+            self.nmean = torch.empty(self.nx.shape[0], dtype=torch.float32, device=dev)
+            self.nrstd = torch.empty(self.nx.shape[0], dtype=torch.float32, device=dev)
+        if "bn_pool" in want:
+            b = c["bn_pool"]
+            self.bx, self.bscale, self.bshift = synth.bn_pool_inputs(cut(b["N"]), b["C"], b["H"], b["W"], b["dtype"], seed, dev)
+            self.by = torch.empty_like(self.bx)
+            self.bp = torch.empty((self.bx.shape[0], b["C"]), dtype=torch.float32, device=dev)
+        if "ce_loss" in want:
+            z = c["ce_loss"]
+            self.cz, self.clab = synth.ce_inputs(cut(z["rows"]), z["vocab"], z["dtype"], seed, dev)
+            self.closs = torch.empty(self.cz.shape[0], dtype=torch.float32, device=dev)
+            self.cmean = torch.empty(1, dtype=torch.float32, device=dev)
+            self.cbad = torch.empty(1, dtype=torch.int32, device=dev)
+            need = kop.kop_ce_loss_rowwise_workspace_bytes(self.cz.shape[0], z["vocab"], kop.KOP_BF16)
+            self.cws = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
+        m = c["mlp"]
+        self.eps = m["eps"]
+        rows = cut(m["rows"])
+        if want & {"rmsnorm", "residual_add", "silu_mul", "mlp"}:
+            g = torch.Generator(device=dev)
+            g.manual_seed(seed)
+            if "mlp" in want:
+                self.h, self.rw, self.W1, self.W2 = synth.mlp_inputs(rows, m["hidden"], m["inter"], m["dtype"], seed, dev)
+                self.handle = kop.MlpHandle()
+                need = kop.kop_rmsnorm_swiglu_residual_workspace_bytes(rows, m["hidden"], m["inter"], kop.KOP_BF16)
+                self.mws = torch.empty(need, dtype=torch.uint8, device=dev)
+                self.mout = torch.empty_like(self.h)
+                # stand-alone inputs of the MLP's fused kernels: the actual GEMM outputs of this chain
+                self.n = kop.kop_rmsnorm(self.h, self.rw, self.eps)
+                self.gu = self.n @ self.W1.t()
+                self.act = kop.kop_silu_mul(self.gu)
+                self.d = self.act @ self.W2.t()
+            else:
+                # profiler captures of one kernel: stand-in tensors of the same shape and spread
+                self.h, self.rw, _, _ = synth.mlp_inputs(rows, m["hidden"], 8, m["dtype"], seed, dev)
+                self.n = torch.empty_like(self.h)
+                if "silu_mul" in want:
+                    self.gu = synth.gate_up_inputs(rows, m["inter"], m["dtype"], seed, dev)
+                    self.act = torch.empty((rows, m["inter"]), dtype=m["dtype"], device=dev)
+                if "residual_add" in want:
+                    _, self.d = synth.pair_inputs(rows, m["hidden"], m["dtype"], seed, dev)
+            self.res = torch.empty_like(self.h)
+
+    def launch(self, name):
+        k, c = self.kop, self.c
+        if name == "softmax_small":
+            k.kop_softmax_scale_bias(self.sx, self.sb, c["softmax_small"]["scale"], out=self.sy)
+        elif name == "softmax_large":
+            k.kop_softmax_scale_bias(self.lx, self.lb, c["softmax_large"]["scale"], out=self.ly)
+        elif name == "layernorm":
+            k.kop_bias_gelu_residual_layernorm(self.nx, self.nr, self.nb, self.ng, self.nbe, c["layernorm"]["eps"],
+                                               out=self.ny, mean=self.nmean, rstd=self.nrstd)
+        elif name == "bn_pool":
+            k.kop_bn_relu_avgpool(self.bx, self.bscale, self.bshift, out=self.by, pooled=self.bp)
+        elif name == "ce_loss":
+            k.kop_ce_loss_rowwise(self.cz, self.clab, loss=self.closs, mean_loss=self.cmean,
+                                  bad_label_count=self.cbad, workspace=self.cws)
+        elif name == "rmsnorm":
+            k.kop_rmsnorm(self.h, self.rw, self.eps, out=self.n)
+        elif name == "silu_mul":
+            k.kop_silu_mul(self.gu, out=self.act)
+        elif name == "residual_add":
+            k.kop_residual_add(self.h, self.d, out=self.res)
+        else:
+            raise KeyError(name)
+
+    def mlp_segment(self):
+        self.kop.kop_rmsnorm_swiglu_residual(self.handle, self.h, self.rw, self.W1, self.W2, self.eps,
+                                             out=self.mout, workspace=self.mws)
+
+    def capture_graph(self):
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            self.mlp_segment()
+            side.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                self.mlp_segment()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        self.graph = g
+
+
+def run_ours(args, rank, world, local_rank):
+    from paper_2609_30059_b200 import build as kbuild
+    if rank == 0:
+        kbuild.build()
+    if world > 1:
+        torch.distributed.barrier()
+    from paper_2609_30059_b200 import kop
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    wl = Workload(kop, dev, seed=rank)
+    wl.capture_graph()
+    wl.graph.replay()
+    segs = segment_bytes()
+    names = Workload.ORDER
+
+    def step(events, with_graph=False):
+        for i, nm in enumerate(names):
+            events[i][0].record()
+            wl.launch(nm)
+            events[i][1].record()
+        if with_graph:
+            events[len(names)][0].record()
+            wl.graph.replay()
+            events[len(names)][1].record()
+
+    def new_events():
+        return [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                for _ in range(len(names) + 1)]
+
+    def timed(n_steps, with_graph):
+        all_events = [new_events() for _ in range(n_steps)]
+        t0 = torch.cuda.Event(enable_timing=True)
+        t1 = torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        if world > 1:
+            torch.distributed.barrier()
+        t0.record()
+        for ev in all_events:
+            step(ev, with_graph)
+        t1.record()
+        torch.cuda.synchronize()
+        if world > 1:
+            torch.distributed.barrier()
+        per = {nm: [ev[i][0].elapsed_time(ev[i][1]) for ev in all_events] for i, nm in enumerate(names)}
+        g = [ev[len(names)][0].elapsed_time(ev[len(names)][1]) for ev in all_events] if with_graph else []
+        return t0.elapsed_time(t1), per, g
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    for _ in range(max(args.warmup, 3)):
+        step(new_events())
+    # ---- the timed region: K steps of the fused kernels ------------------------------------------
+    total_ms, per, _ = timed(args.steps, with_graph=False)
+    clocks = sampler.stop()
+    # ---- the MLP segment as a CUDA graph (our three kernels + the two preserved cuBLAS GEMMs), and
+    # the fused kernels again when they alternate with it: the GEMMs pull the GPU into its power cap,
+    # so this second set shows the same kernels at the lower clocks they see inside a model.
+    sampler2 = ClockSampler(local_rank)
+    sampler2.start()
+    situ_steps = max(3, min(args.steps, 20))
+    for _ in range(3):
+        step(new_events(), with_graph=True)
+    _, per_situ, graph_ms = timed(situ_steps, with_graph=True)
+    clocks_situ = sampler2.stop()
+
+    fused_ms_step = sum(statistics.mean(per[nm]) for nm in names)
+    fused_bytes = sum(segs[nm]["bytes"] for nm in names)
+    # max over ranks of the timed quantities
+    if world > 1:
+        t = torch.tensor([total_ms, fused_ms_step], dtype=torch.float64, device=dev)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        total_ms, fused_ms_step_max = float(t[0]), float(t[1])
+    else:
+        fused_ms_step_max = fused_ms_step
+    value = world * fused_bytes / (fused_ms_step_max * 1e-3) / 1e9
+
+    peak, peak_src = measured_peak()
+
+    def report(per_kernel):
+        out = {}
+        for nm in names:
+            ms = statistics.mean(per_kernel[nm])
+            gbs = segs[nm]["bytes"] / (ms * 1e-3) / 1e9
+            out[nm] = dict(us=round(ms * 1e3, 2), us_min=round(min(per_kernel[nm]) * 1e3, 2), gbs=round(gbs, 1),
+                           frac_measured=round(gbs / peak, 4), frac_nominal=round(gbs / NOMINAL_HBM_GBS, 4),
+                           gelems_per_s=round(segs[nm]["elems"] / (ms * 1e-3) / 1e9, 2), bytes=segs[nm]["bytes"])
+        return out
+
+    seg_report = report(per)
+    dom = max(names, key=lambda nm: statistics.mean(per[nm]))
+    dom_ms = statistics.mean(per[dom])
+    achieved = segs[dom]["bytes"] / (dom_ms * 1e-3) / 1e9
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if os.path.exists(tpath):
+        try:
+            traffic = json.load(open(tpath)).get(dom)
+        except Exception:
+            traffic = None
+    roofline = dict(bound="hbm", kernel=dom, achieved=round(achieved, 1), peak=peak, unit="GB/s",
+                    frac=round(achieved / peak, 4), traffic=traffic, peak_source=peak_src,
+                    algorithmic_bytes=segs[dom]["bytes"], avg_launch_us=round(dom_ms * 1e3, 2))
+
+    e2e = run_e2e(args, wl, kop, dev, segs, names, world)
+    cpu = None
+    if rank == 0 and world == 1:
+        cpu = cpu_baseline(budget_s=args.cpu_seconds)
+
+    if rank == 0:
+        situ_ms = sum(statistics.mean(per_situ[nm]) for nm in names)
+        line = {
+            "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": round(total_ms / args.steps, 4),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic (seeded; shapes and distributions of the five benchmark configs)",
+            "config": {"workload": "all fused segments at full benchmark shapes: softmax fp32 [128,512] and "
+                                   "[131072,512]; bias+GELU+residual+LayerNorm bf16 [8192,4096]; BN+ReLU+avgpool "
+                                   "fp32 [64,256,56,56]; cross-entropy bf16 [32768,32000]; RMSNorm bf16 "
+                                   "[16384,4096]; SiLU*up bf16 [16384,2x14336]; residual add bf16 [16384,4096]",
+                       "l2": "inputs larger than L2: each step streams > 5 GB through a 126 MB L2",
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "fused_ms_per_step": round(fused_ms_step_max, 4),
+            "gpu_launches": args.steps * len(names),
+            "segments": seg_report,
+            "roofline": roofline,
+            "frac_of_nominal_8TBs": round(value / world / NOMINAL_HBM_GBS, 4),
+            "clocks": clocks,
+            "mlp_segment_graph": {
+                "ms_per_replay": round(statistics.mean(graph_ms), 4), "replays": situ_steps,
+                "nodes": "rmsnorm, cuBLAS GEMM [16384,4096]x[4096,28672], silu_mul, cuBLAS GEMM "
+                         "[16384,14336]x[14336,4096], residual_add", "gemm_tflop": 5.772,
+                "clocks": clocks_situ,
+                "fused_segments_alternating_with_graph": report(per_situ),
+                "fused_gbs_alternating_with_graph": round(fused_bytes / (situ_ms * 1e-3) / 1e9, 1),
+            },
+            "e2e": e2e,
+            "paper_context": "torch.compile geomean speedups 1.40x/1.15x/1.07x on one H200 (context only)",
+        }
+        if cpu is not None:
+            line["cpu_baseline"] = cpu
+        print(json.dumps(line), flush=True)
+
+
+def run_e2e(args, wl, kop, dev, segs, names, world):
+    """Same metric end to end: every step copies the step's inputs from pinned host memory, runs the
+    segments through the C ABI (MLP via the segment driver) and reads every result back."""
+    pin = lambda t: torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t)  # noqa: E731
+    ins = [(wl.sx, pin(wl.sx)), (wl.lx, pin(wl.lx)), (wl.nx, pin(wl.nx)), (wl.nr, pin(wl.nr)),
+           (wl.bx, pin(wl.bx)), (wl.cz, pin(wl.cz)), (wl.clab, pin(wl.clab)), (wl.h, pin(wl.h))]
+    outs = [wl.sy, wl.ly, wl.ny, wl.nmean, wl.nrstd, wl.by, wl.bp, wl.closs, wl.cmean, wl.cbad, wl.mout]
+    houts = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in outs]
+    h2d = sum(h.numel() * h.element_size() for _, h in ins)
+    d2h = sum(h.numel() * h.element_size() for h in houts)
+
+    def step():
+        for d, h in ins:
+            d.copy_(h, non_blocking=True)
+        for nm in ("softmax_small", "softmax_large", "layernorm", "bn_pool", "ce_loss"):
+            wl.launch(nm)
+        wl.mlp_segment()
+        for d, h in zip(outs, houts):
+            h.copy_(d, non_blocking=True)
+
+    steps = max(2, min(args.steps, 5))
+    step()
+    torch.cuda.synchronize()
+    if world > 1:
+        torch.distributed.barrier()
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    wall0 = time.perf_counter()
+    t0.record()
+    for _ in range(steps):
+        step()
+    t1.record()
+    torch.cuda.synchronize()
+    wall = (time.perf_counter() - wall0) * 1e3
+    ms = max(t0.elapsed_time(t1), wall) / steps
+    if world > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        ms = float(t[0])
+    fused_bytes = sum(segs[nm]["bytes"] for nm in names)
+    return {"value": round(world * fused_bytes / (ms * 1e-3) / 1e9, 2), "unit": UNIT, "ms_per_step": round(ms, 3),
+            "steps": steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "includes": "pinned-host H2D of all data inputs, all fused kernels, both cuBLAS GEMMs, D2H of all outputs"}
+
+
+# ----------------------------------------------------------------------------- CPU oracle arm
+
+def oracle_sample_plan():
+    """A bounded sample of the same workload: each segment at its benchmark row length with the row
+    count cut (where needed) so that one pass is about a second of CPU work on a few cores."""
+    return {"softmax_large": 131072, "layernorm": 4096, "bn_pool": 32, "ce_loss": 2048, "rmsnorm": 16384,
+            "silu_mul": 2048, "residual_add": 16384}
+
+
+def oracle_pass(inputs, threads):
+    from oracle import kopref
+    c = synth.CONFIGS
+    t = {}
+    t0 = time.perf_counter()
+    kopref.softmax_scale_bias(inputs["sx"], inputs["sb"], c["softmax_large"]["scale"], threads)
+    t["softmax_large"] = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    kopref.bias_gelu_residual_layernorm(*inputs["ln"], c["layernorm"]["eps"], threads)
+    t["layernorm"] = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    kopref.bn_relu_avgpool(*inputs["bn"], threads=threads)
+    t["bn_pool"] = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    kopref.ce_loss_rowwise(*inputs["ce"], threads=threads)
+    t["ce_loss"] = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    kopref.rmsnorm(inputs["h"], inputs["rw"], c["mlp"]["eps"], threads)
+    t["rmsnorm"] = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    kopref.silu_mul(inputs["gu"], threads)
+    t["silu_mul"] = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    kopref.residual_add(inputs["a"], inputs["b"], threads)
+    t["residual_add"] = time.perf_counter() - t0
+    return t
+
+
+def oracle_inputs(plan):
+    c = synth.CONFIGS
+    sx, sb = synth.softmax_inputs(plan["softmax_large"], c["softmax_large"]["cols"], torch.float32, 0)
+    ln = synth.layernorm_inputs(plan["layernorm"], c["layernorm"]["hidden"], torch.bfloat16, 0)
+    b = c["bn_pool"]
+    bn = synth.bn_pool_inputs(plan["bn_pool"], b["C"], b["H"], b["W"], torch.float32, 0)
+    ce = synth.ce_inputs(plan["ce_loss"], c["ce_loss"]["vocab"], torch.bfloat16, 0)
+    m = c["mlp"]
+    h, rw, _, _ = synth.mlp_inputs(plan["rmsnorm"], m["hidden"], 8, torch.bfloat16, 0)
+    gu = synth.gate_up_inputs(plan["silu_mul"], m["inter"], torch.bfloat16, 0, std=1.0)
+    a, bb = synth.pair_inputs(plan["residual_add"], m["hidden"], torch.bfloat16, 0)
+    return dict(sx=sx, sb=sb, ln=ln, bn=bn, ce=ce, h=h, rw=rw, gu=gu, a=a, b=bb)
+
+
+def oracle_sample_bytes(plan):
+    """Algorithmic bytes of the sample, by the same rule as the GPU arm."""
+    c = synth.CONFIGS
+    full = segment_bytes()
+    rows_full = {"softmax_large": c["softmax_large"]["rows"], "layernorm": c["layernorm"]["rows"],
+                 "bn_pool": c["bn_pool"]["N"], "ce_loss": c["ce_loss"]["rows"], "rmsnorm": c["mlp"]["rows"],
+                 "silu_mul": c["mlp"]["rows"], "residual_add": c["mlp"]["rows"]}
+    return {k: full[k]["bytes"] * plan[k] / rows_full[k] for k in plan}
+
+
+def cpu_baseline(budget_s=15.0, repeats=None):
+    """Times the oracle, as it stands, on the host cores over a bounded sample of the workload."""
+    from oracle import kopref
+    threads = kopref.host_threads()
+    plan = oracle_sample_plan()
+    inputs = oracle_inputs(plan)
+    nbytes = oracle_sample_bytes(plan)
+    oracle_pass(inputs, threads)                       # warm-up (builds the library, touches memory)
+    times = []
+    t_start = time.perf_counter()
+    while True:
+        times.append(oracle_pass(inputs, threads))
+        if repeats is not None and len(times) >= repeats:
+            break
+        if repeats is None and (time.perf_counter() - t_start > budget_s or len(times) >= 20):
+            break
+    tot = sum(sum(t.values()) for t in times) / len(times)
+    per = {k: round(nbytes[k] / (sum(t[k] for t in times) / len(times)) / 1e9, 3) for k in plan}
+    return {"value": round(sum(nbytes.values()) / tot / 1e9, 3), "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": "one pass per repeat over " + ", ".join(f"{k}:{v} rows" for k, v in plan.items())
+                      + " at the benchmark row lengths (bn_pool rows = images)",
+            "seconds_per_pass": round(tot, 3), "passes": len(times), "per_segment_gbs": per}
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    from oracle import kopref
+    threads = kopref.host_threads()
+    plan = oracle_sample_plan()
+    inputs = oracle_inputs(plan)
+    nbytes = sum(oracle_sample_bytes(plan).values())
+    for _ in range(min(args.warmup, 2) or 1):
+        oracle_pass(inputs, threads)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_pass(inputs, threads)
+    ms = (time.perf_counter() - t0) * 1e3 / args.steps
+    val = round(nbytes / (ms * 1e-3) / 1e9, 3)
+    sample = "each step = one oracle pass over " + ", ".join(f"{k}:{v} rows" for k, v in plan.items())
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms, 3), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic (seeded)",
+        "config": {"workload": "bounded sample of the fused-segment workload at the benchmark row lengths", "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }), flush=True)
+
+
+def run_profile(args):
+    """Launch the named segments alone a few times (for ncu captures and quick timing). Only their
+    tensors are allocated; --rows-div shrinks the row count so a multi-pass capture stays small."""
+    from paper_2609_30059_b200 import build as kbuild
+    kbuild.build()
+    from paper_2609_30059_b200 import kop
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    names = args.profile.split(",")
+    wl = Workload(kop, dev, seed=0, only=names, rows_div=args.rows_div)
+    segs = segment_bytes()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    report = {}
+    for nm in names:
+        if nm == "mlp":
+            wl.mlp_segment()
+            continue
+        ts = []
+        for i in range(args.launches + 1):
+            flush.zero_()                                   # evict L2 between launches
+            e0 = torch.cuda.Event(enable_timing=True)
+            e1 = torch.cuda.Event(enable_timing=True)
+            e0.record()
+            wl.launch(nm)
+            e1.record()
+            torch.cuda.synchronize()
+            if i:
+                ts.append(e0.elapsed_time(e1))
+        ms = statistics.median(ts)
+        nb = segs[nm]["bytes"] / (1 if nm == "softmax_small" else args.rows_div)
+        report[nm] = {"us": round(ms * 1e3, 2), "gbs": round(nb / (ms * 1e-3) / 1e9, 1)}
+    print(json.dumps({"profile": report, "rows_div": args.rows_div, "launches": args.launches}), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cpu-seconds", type=float, default=15.0, help="CPU time budget of the cpu_baseline leg")
+    ap.add_argument("--profile", default=None, help="comma list of segments to launch alone (ncu / quick timing)")
+    ap.add_argument("--rows-div", type=int, default=1, help="with --profile: divide every row count by this")
+    ap.add_argument("--launches", type=int, default=3, help="with --profile: timed launches per segment")
+    args = ap.parse_args()
+    if args.profile:
+        run_profile(args)
+        return
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libkop has no CPU path")
+    if world > 1:
+        torch.cuda.set_device(local_rank)
+        torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    try:
+        run_ours(args, rank, world, local_rank)
+    finally:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

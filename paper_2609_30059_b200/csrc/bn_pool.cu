@@ -159,8 +159,9 @@ extern "C" kop_status_t kop_bn_relu_avgpool(const void* x, const float* scale, c
 {
     using namespace kop;
     if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
-    if (!x || !scale || !shift || !y || !pooled || !x_strides || !y_strides) return KOP_ERR_NULL_POINTER;
     if (N < 0 || C <= 0 || H <= 0 || W <= 0) return KOP_ERR_BAD_SHAPE;
+    if (N == 0) return KOP_OK;
+    if (!x || !scale || !shift || !y || !pooled || !x_strides || !y_strides) return KOP_ERR_NULL_POINTER;
     if (C > 0x7FFFFFFF || H > kMaxElems || W > kMaxElems || N > kMaxElems) return KOP_ERR_BAD_SHAPE;
     if (H > kMaxElems / W) return KOP_ERR_BAD_SHAPE;
     const int64_t plane = H * W;
@@ -174,7 +175,6 @@ extern "C" kop_status_t kop_bn_relu_avgpool(const void* x, const float* scale, c
         !aligned_to(pooled, 4))
         return KOP_ERR_MISALIGNED;
     if (!alias_ok(x, C * plane, y, C * plane, N, C * plane, esz, true)) return KOP_ERR_BAD_ALIAS;
-    if (N == 0) return KOP_OK;
     kop_status_t st = check_device();
     if (st != KOP_OK) return st;
     cudaStream_t s = as_stream(stream);

@@ -121,6 +121,40 @@ __device__ __forceinline__ float4 ldg_f4(const float* p)
     return __ldg(reinterpret_cast<const float4*>(p));
 }
 
+// Read-only 256-bit load (sm_100): eight consecutive floats per lane in one request. `p` must be
+// 32-byte aligned.
+struct __align__(32) Float8 {
+    float f[8];
+};
+__device__ __forceinline__ Float8 ldg_f8(const float* p)
+{
+    Float8 r;
+    asm volatile("ld.global.nc.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(r.f[0]), "=f"(r.f[1]), "=f"(r.f[2]), "=f"(r.f[3]), "=f"(r.f[4]), "=f"(r.f[5]),
+                   "=f"(r.f[6]), "=f"(r.f[7])
+                 : "l"(p));
+    return r;
+}
+
+// The E fp32 parameters that belong to one data vector, as E/2 packed pairs. kWide (E == 8 only)
+// uses one 256-bit load; otherwise E/4 128-bit loads.
+template <int E, bool kWide>
+__device__ __forceinline__ void load_params(const float* p, float2 (&out)[E / 2])
+{
+    if constexpr (kWide && E == 8) {
+        const Float8 t = ldg_f8(p);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) out[q] = make_float2(t.f[2 * q], t.f[2 * q + 1]);
+    } else {
+#pragma unroll
+        for (int q = 0; q < E / 4; ++q) {
+            const float4 t = ldg_f4(p + 4 * q);
+            out[2 * q] = make_float2(t.x, t.y);
+            out[2 * q + 1] = make_float2(t.z, t.w);
+        }
+    }
+}
+
 __device__ __forceinline__ float ex2_approx(float x)
 {
     float y;
@@ -165,6 +199,20 @@ struct Elem<float> {
         for (int i = 0; i < 4; ++i) v.w[i] = __float_as_uint(f[i]);
         return v;
     }
+    __device__ __forceinline__ static void unpack2(const Vec16& v, float2 (&f)[2])
+    {
+        f[0] = make_float2(__uint_as_float(v.w[0]), __uint_as_float(v.w[1]));
+        f[1] = make_float2(__uint_as_float(v.w[2]), __uint_as_float(v.w[3]));
+    }
+    __device__ __forceinline__ static Vec16 pack2(const float2 (&f)[2])
+    {
+        Vec16 v;
+        v.w[0] = __float_as_uint(f[0].x);
+        v.w[1] = __float_as_uint(f[0].y);
+        v.w[2] = __float_as_uint(f[1].x);
+        v.w[3] = __float_as_uint(f[1].y);
+        return v;
+    }
     __device__ __forceinline__ static float load1(const float* p) { return *p; }
     __device__ __forceinline__ static void store1(float* p, float f) { *p = f; }
     __device__ __forceinline__ static Vec16 fill_neg_inf()
@@ -195,6 +243,22 @@ struct Elem<__nv_bfloat16> {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+            v.w[i] = *reinterpret_cast<uint32_t*>(&h);
+        }
+        return v;
+    }
+    __device__ __forceinline__ static void unpack2(const Vec16& v, float2 (&f)[4])
+    {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            f[i] = make_float2(__uint_as_float(v.w[i] << 16), __uint_as_float(v.w[i] & 0xFFFF0000u));
+    }
+    __device__ __forceinline__ static Vec16 pack2(const float2 (&f)[4])
+    {
+        Vec16 v;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            __nv_bfloat162 h = __floats2bfloat162_rn(f[i].x, f[i].y);
             v.w[i] = *reinterpret_cast<uint32_t*>(&h);
         }
         return v;

@@ -20,7 +20,26 @@ __device__ __forceinline__ float gelu_tanh(float u)
     return fmaf(hu, t, hu);
 }
 
-template <typename T, int VPT>
+// Two-wide version on packed fp32 pairs (fma.rn.f32x2 and friends: one issue slot per two
+// elements), returning residual + gelu(x + bias).
+template <bool kFastTanh>
+__device__ __forceinline__ float2 gelu_residual2(float2 x, float2 b, float2 r)
+{
+    const float k0 = 0.7978845608028654f, k1 = 0.7978845608028654f * 0.044715f;
+    const float2 u = __fadd2_rn(x, b);
+    const float2 p = __ffma2_rn(make_float2(k1, k1), __fmul2_rn(u, u), make_float2(k0, k0));
+    const float2 inner = __fmul2_rn(u, p);
+    const float2 t = kFastTanh ? make_float2(tanh_approx(inner.x), tanh_approx(inner.y))
+                               : make_float2(tanhf(inner.x), tanhf(inner.y));
+    const float2 hu = __fmul2_rn(make_float2(0.5f, 0.5f), u);
+    return __ffma2_rn(hu, t, __fadd2_rn(hu, r));
+}
+
+// CTA per row, row in registers as fp32 pairs. kFull: the row is exactly blockDim.x * VPT vectors
+// (no tail predicates). kWide: the eight fp32 parameters that go with a bf16 vector are fetched
+// with one 256-bit load per lane, so a warp touches each 128-byte line once (two 128-bit loads
+// per lane would walk every line twice and double the L1 wavefronts, which bound this kernel).
+template <typename T, int VPT, bool kFull, bool kWide>
 __global__ void __launch_bounds__(max_threads_for(VPT * Elem<T>::kPerVec))
 ln_block_kernel(const T* __restrict__ x, const T* __restrict__ res, const float* __restrict__ bias,
                 const float* __restrict__ gamma, const float* __restrict__ beta, T* __restrict__ y,
@@ -28,6 +47,7 @@ ln_block_kernel(const T* __restrict__ x, const T* __restrict__ res, const float*
                 int64_t r_stride, int64_t y_stride, float eps, float inv_hidden)
 {
     constexpr int E = Elem<T>::kPerVec;
+    constexpr int P = E / 2;                       // fp32 pairs per vector
     constexpr bool kFast = sizeof(T) == 2;
     __shared__ float red_a[32], red_b[32];
     const int64_t row = blockIdx.x;
@@ -39,65 +59,66 @@ ln_block_kernel(const T* __restrict__ x, const T* __restrict__ res, const float*
 #pragma unroll
     for (int k = 0; k < VPT; ++k) {
         const int v = k * blockDim.x + threadIdx.x;
-        if (v < nvec) {
+        if (kFull || v < nvec) {
             rx[k] = ld_stream(xr + (int64_t)v * E);
             rres[k] = ld_stream(rr + (int64_t)v * E);
+        } else {
+            rx[k] = Vec16{{0u, 0u, 0u, 0u}};
+            rres[k] = Vec16{{0u, 0u, 0u, 0u}};
         }
     }
-    float val[VPT][E];
-    float sum = 0.0f;
+    float2 val[VPT][P];
+    float2 sum2 = make_float2(0.0f, 0.0f);
 #pragma unroll
     for (int k = 0; k < VPT; ++k) {
         const int v = k * blockDim.x + threadIdx.x;
-        float fx[E], fr[E];
-        Elem<T>::unpack(rx[k], fx);
-        Elem<T>::unpack(rres[k], fr);
+        float2 bb[P], fx[P], fr[P];
+        if (kFull || v < nvec) load_params<E, kWide>(bias + (int64_t)v * E, bb);
+        else {
 #pragma unroll
-        for (int q = 0; q < E / 4; ++q) {
-            float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (v < nvec) b = ldg_f4(bias + (int64_t)v * E + 4 * q);
-            const float bb[4] = {b.x, b.y, b.z, b.w};
+            for (int q = 0; q < P; ++q) bb[q] = make_float2(0.0f, 0.0f);
+        }
+        Elem<T>::unpack2(rx[k], fx);
+        Elem<T>::unpack2(rres[k], fr);
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const int e = 4 * q + c;
-                const float t = fr[e] + gelu_tanh<kFast>(fx[e] + bb[c]);
-                val[k][e] = v < nvec ? t : 0.0f;
-                sum += val[k][e];
-            }
+        for (int q = 0; q < P; ++q) {
+            float2 t = gelu_residual2<kFast>(fx[q], bb[q], fr[q]);
+            if (!kFull && v >= nvec) t = make_float2(0.0f, 0.0f);
+            val[k][q] = t;
+            sum2 = __fadd2_rn(sum2, t);
         }
     }
-    const float mu = block_sum(sum, red_a) * inv_hidden;
-    float ss = 0.0f;
+    const float mu = block_sum(sum2.x + sum2.y, red_a) * inv_hidden;
+    const float2 nmu = make_float2(-mu, -mu);
+    float2 ss2 = make_float2(0.0f, 0.0f);
 #pragma unroll
     for (int k = 0; k < VPT; ++k) {
         const int v = k * blockDim.x + threadIdx.x;
 #pragma unroll
-        for (int e = 0; e < E; ++e) {
-            val[k][e] -= mu;
-            ss = v < nvec ? fmaf(val[k][e], val[k][e], ss) : ss;
+        for (int q = 0; q < P; ++q) {
+            float2 d = __fadd2_rn(val[k][q], nmu);
+            if (!kFull && v >= nvec) d = make_float2(0.0f, 0.0f);
+            val[k][q] = d;
+            ss2 = __ffma2_rn(d, d, ss2);
         }
     }
-    const float var = block_sum(ss, red_b) * inv_hidden;
+    const float var = block_sum(ss2.x + ss2.y, red_b) * inv_hidden;
     const float rs = rsqrtf(var + eps);
     if (threadIdx.x == 0) {
         if (mean != nullptr) mean[row] = mu;
         if (rstd != nullptr) rstd[row] = rs;
     }
+    const float2 rs2 = make_float2(rs, rs);
 #pragma unroll
     for (int k = 0; k < VPT; ++k) {
         const int v = k * blockDim.x + threadIdx.x;
-        if (v < nvec) {
-            float o[E];
+        if (kFull || v < nvec) {
+            float2 g[P], b[P], o[P];
+            load_params<E, kWide>(gamma + (int64_t)v * E, g);
+            load_params<E, kWide>(beta + (int64_t)v * E, b);
 #pragma unroll
-            for (int q = 0; q < E / 4; ++q) {
-                const float4 g = ldg_f4(gamma + (int64_t)v * E + 4 * q);
-                const float4 b = ldg_f4(beta + (int64_t)v * E + 4 * q);
-                o[4 * q + 0] = fmaf(val[k][4 * q + 0] * rs, g.x, b.x);
-                o[4 * q + 1] = fmaf(val[k][4 * q + 1] * rs, g.y, b.y);
-                o[4 * q + 2] = fmaf(val[k][4 * q + 2] * rs, g.z, b.z);
-                o[4 * q + 3] = fmaf(val[k][4 * q + 3] * rs, g.w, b.w);
-            }
-            st_stream(yr + (int64_t)v * E, Elem<T>::pack(o));
+            for (int q = 0; q < P; ++q) o[q] = __ffma2_rn(__fmul2_rn(val[k][q], rs2), g[q], b[q]);
+            st_stream(yr + (int64_t)v * E, Elem<T>::pack2(o));
         }
     }
 }
@@ -164,15 +185,25 @@ kop_status_t launch_ln(const void* xv, const void* rv, const float* bias, const 
         if ((nvec + vals / E - 1) / (vals / E) > max_threads_for(vals)) vals = 64;
         const int vpt = vals / E;
         const int threads = ((nvec + vpt - 1) / vpt + 31) / 32 * 32;
-#define KOP_LN(V)                                                                               \
-    ln_block_kernel<T, V><<<(unsigned)rows, threads, 0, stream>>>(x, r, bias, gamma, beta, y, mean, \
-                                                                  rstd, nvec, xs, rs, ys, eps, inv_hidden)
+        const bool full = (nvec % vpt) == 0 && (nvec / vpt) == threads;
+        const bool wide = E == 8 && aligned_to(bias, 32) && aligned_to(gamma, 32) && aligned_to(beta, 32);
+#define KOP_LN_LAUNCH(V, F, W)                                                                    \
+    ln_block_kernel<T, V, F, W><<<(unsigned)rows, threads, 0, stream>>>(x, r, bias, gamma, beta, y, mean, \
+                                                                        rstd, nvec, xs, rs, ys, eps, inv_hidden)
+#define KOP_LN(V)                                             \
+    do {                                                      \
+        if (full && wide) KOP_LN_LAUNCH(V, true, true);       \
+        else if (full) KOP_LN_LAUNCH(V, true, false);         \
+        else if (wide) KOP_LN_LAUNCH(V, false, true);         \
+        else KOP_LN_LAUNCH(V, false, false);                  \
+    } while (0)
         switch (vals) {
         case 8: KOP_LN(8 / E); break;
         case 16: KOP_LN(16 / E); break;
         case 32: KOP_LN(32 / E); break;
         default: KOP_LN(64 / E); break;
         }
+#undef KOP_LN_LAUNCH
 #undef KOP_LN
         return launch_status();
     }
@@ -191,9 +222,10 @@ extern "C" kop_status_t kop_bias_gelu_residual_layernorm(
 {
     using namespace kop;
     if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
-    if (!x || !residual || !bias || !gamma || !beta || !y) return KOP_ERR_NULL_POINTER;
     kop_status_t st = check_rows_cols(rows, hidden);
     if (st != KOP_OK) return st;
+    if (rows == 0) return KOP_OK;
+    if (!x || !residual || !bias || !gamma || !beta || !y) return KOP_ERR_NULL_POINTER;
     if ((st = check_row_stride(x_row_stride, hidden, rows)) != KOP_OK) return st;
     if ((st = check_row_stride(res_row_stride, hidden, rows)) != KOP_OK) return st;
     if ((st = check_row_stride(y_row_stride, hidden, rows)) != KOP_OK) return st;
@@ -206,7 +238,6 @@ extern "C" kop_status_t kop_bias_gelu_residual_layernorm(
     if (!alias_ok(x, x_row_stride, y, y_row_stride, rows, hidden, esz, true) ||
         !alias_ok(residual, res_row_stride, y, y_row_stride, rows, hidden, esz, true))
         return KOP_ERR_BAD_ALIAS;
-    if (rows == 0) return KOP_OK;
     if ((st = check_device()) != KOP_OK) return st;
     cudaStream_t s = as_stream(stream);
     return dtype == KOP_F32

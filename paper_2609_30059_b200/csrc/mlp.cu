@@ -8,12 +8,15 @@ namespace kop {
 namespace {
 
 // ---- RMSNorm: CTA per row, row in registers -----------------------------------------------------
-template <typename T, int VPT>
+// kFull: the row is exactly blockDim.x * VPT vectors (no tail predicates). kWide: the eight fp32
+// weights of a bf16 vector come in one 256-bit load per lane (each 128-byte line touched once).
+template <typename T, int VPT, bool kFull, bool kWide>
 __global__ void __launch_bounds__(max_threads_for(VPT * Elem<T>::kPerVec))
 rmsnorm_block_kernel(const T* __restrict__ x, const float* __restrict__ w, T* __restrict__ y, int nvec,
                      int64_t x_stride, int64_t y_stride, float eps, float inv_hidden)
 {
     constexpr int E = Elem<T>::kPerVec;
+    constexpr int P = E / 2;
     __shared__ float red[32];
     const int64_t row = blockIdx.x;
     const T* xr = x + row * x_stride;
@@ -22,35 +25,28 @@ rmsnorm_block_kernel(const T* __restrict__ x, const float* __restrict__ w, T* __
 #pragma unroll
     for (int k = 0; k < VPT; ++k) {
         const int v = k * blockDim.x + threadIdx.x;
-        if (v < nvec) raw[k] = ld_stream(xr + (int64_t)v * E);
+        if (kFull || v < nvec) raw[k] = ld_stream(xr + (int64_t)v * E);
+        else raw[k] = Vec16{{0u, 0u, 0u, 0u}};
     }
-    float val[VPT][E];
-    float ss = 0.0f;
+    float2 val[VPT][P];
+    float2 ss2 = make_float2(0.0f, 0.0f);
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+        Elem<T>::unpack2(raw[k], val[k]);
+#pragma unroll
+        for (int q = 0; q < P; ++q) ss2 = __ffma2_rn(val[k][q], val[k][q], ss2);
+    }
+    const float r = rsqrtf(block_sum(ss2.x + ss2.y, red) * inv_hidden + eps);
+    const float2 r2 = make_float2(r, r);
 #pragma unroll
     for (int k = 0; k < VPT; ++k) {
         const int v = k * blockDim.x + threadIdx.x;
-        Elem<T>::unpack(raw[k], val[k]);
+        if (kFull || v < nvec) {
+            float2 g[P], o[P];
+            load_params<E, kWide>(w + (int64_t)v * E, g);
 #pragma unroll
-        for (int e = 0; e < E; ++e) {
-            val[k][e] = v < nvec ? val[k][e] : 0.0f;
-            ss = fmaf(val[k][e], val[k][e], ss);
-        }
-    }
-    const float r = rsqrtf(block_sum(ss, red) * inv_hidden + eps);
-#pragma unroll
-    for (int k = 0; k < VPT; ++k) {
-        const int v = k * blockDim.x + threadIdx.x;
-        if (v < nvec) {
-            float o[E];
-#pragma unroll
-            for (int q = 0; q < E / 4; ++q) {
-                const float4 g = ldg_f4(w + (int64_t)v * E + 4 * q);
-                o[4 * q + 0] = val[k][4 * q + 0] * r * g.x;
-                o[4 * q + 1] = val[k][4 * q + 1] * r * g.y;
-                o[4 * q + 2] = val[k][4 * q + 2] * r * g.z;
-                o[4 * q + 3] = val[k][4 * q + 3] * r * g.w;
-            }
-            st_stream(yr + (int64_t)v * E, Elem<T>::pack(o));
+            for (int q = 0; q < P; ++q) o[q] = __fmul2_rn(__fmul2_rn(val[k][q], r2), g[q]);
+            st_stream(yr + (int64_t)v * E, Elem<T>::pack2(o));
         }
     }
 }
@@ -208,13 +204,24 @@ kop_status_t launch_rmsnorm(const void* xv, const float* w, void* yv, int64_t ro
         if ((nvec + vals / E - 1) / (vals / E) > max_threads_for(vals)) vals = 64;
         const int vpt = vals / E;
         const int threads = ((nvec + vpt - 1) / vpt + 31) / 32 * 32;
-#define KOP_RMS(V) rmsnorm_block_kernel<T, V><<<(unsigned)rows, threads, 0, stream>>>(x, w, y, nvec, xs, ys, eps, inv_hidden)
+        const bool full = (nvec % vpt) == 0 && (nvec / vpt) == threads;
+        const bool wide = E == 8 && aligned_to(w, 32);
+#define KOP_RMS_LAUNCH(V, F, W) \
+    rmsnorm_block_kernel<T, V, F, W><<<(unsigned)rows, threads, 0, stream>>>(x, w, y, nvec, xs, ys, eps, inv_hidden)
+#define KOP_RMS(V)                                             \
+    do {                                                       \
+        if (full && wide) KOP_RMS_LAUNCH(V, true, true);       \
+        else if (full) KOP_RMS_LAUNCH(V, true, false);         \
+        else if (wide) KOP_RMS_LAUNCH(V, false, true);         \
+        else KOP_RMS_LAUNCH(V, false, false);                  \
+    } while (0)
         switch (vals) {
         case 8: KOP_RMS(8 / E); break;
         case 16: KOP_RMS(16 / E); break;
         case 32: KOP_RMS(32 / E); break;
         default: KOP_RMS(64 / E); break;
         }
+#undef KOP_RMS_LAUNCH
 #undef KOP_RMS
         return launch_status();
     }
@@ -326,16 +333,16 @@ extern "C" kop_status_t kop_rmsnorm(const void* x, const float* weight, void* y,
 {
     using namespace kop;
     if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
-    if (!x || !weight || !y) return KOP_ERR_NULL_POINTER;
     kop_status_t st = check_rows_cols(rows, hidden);
     if (st != KOP_OK) return st;
+    if (rows == 0) return KOP_OK;
+    if (!x || !weight || !y) return KOP_ERR_NULL_POINTER;
     if ((st = check_row_stride(x_row_stride, hidden, rows)) != KOP_OK) return st;
     if ((st = check_row_stride(y_row_stride, hidden, rows)) != KOP_OK) return st;
     if (!(eps >= 0.0f)) return KOP_ERR_BAD_SHAPE;
     const int esz = elem_size(dtype);
     if (!aligned_to(x, esz) || !aligned_to(y, esz) || !aligned_to(weight, 4)) return KOP_ERR_MISALIGNED;
     if (!alias_ok(x, x_row_stride, y, y_row_stride, rows, hidden, esz, true)) return KOP_ERR_BAD_ALIAS;
-    if (rows == 0) return KOP_OK;
     if ((st = check_device()) != KOP_OK) return st;
     cudaStream_t s = as_stream(stream);
     return dtype == KOP_F32
@@ -349,9 +356,10 @@ extern "C" kop_status_t kop_silu_mul(const void* gate_up, void* out, int64_t row
 {
     using namespace kop;
     if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
-    if (!gate_up || !out) return KOP_ERR_NULL_POINTER;
     kop_status_t st = check_rows_cols(rows, inter);
     if (st != KOP_OK) return st;
+    if (rows == 0) return KOP_OK;
+    if (!gate_up || !out) return KOP_ERR_NULL_POINTER;
     if (inter > kMaxElems / 2) return KOP_ERR_BAD_SHAPE;
     if ((st = check_row_stride(in_row_stride, 2 * inter, rows)) != KOP_OK) return st;
     if ((st = check_row_stride(out_row_stride, inter, rows)) != KOP_OK) return st;
@@ -363,7 +371,6 @@ extern "C" kop_status_t kop_silu_mul(const void* gate_up, void* out, int64_t row
         span_of(out, rows, inter, out_row_stride, esz, &b0, &b1);
         if (!(a1 <= b0 || b1 <= a0)) return KOP_ERR_BAD_ALIAS;
     }
-    if (rows == 0) return KOP_OK;
     if ((st = check_device()) != KOP_OK) return st;
     cudaStream_t s = as_stream(stream);
     return dtype == KOP_F32
@@ -377,9 +384,10 @@ extern "C" kop_status_t kop_residual_add(const void* a, const void* b, void* out
 {
     using namespace kop;
     if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
-    if (!a || !b || !out) return KOP_ERR_NULL_POINTER;
     kop_status_t st = check_rows_cols(rows, cols);
     if (st != KOP_OK) return st;
+    if (rows == 0) return KOP_OK;
+    if (!a || !b || !out) return KOP_ERR_NULL_POINTER;
     if ((st = check_row_stride(a_row_stride, cols, rows)) != KOP_OK) return st;
     if ((st = check_row_stride(b_row_stride, cols, rows)) != KOP_OK) return st;
     if ((st = check_row_stride(out_row_stride, cols, rows)) != KOP_OK) return st;
@@ -388,7 +396,6 @@ extern "C" kop_status_t kop_residual_add(const void* a, const void* b, void* out
     if (!alias_ok(a, a_row_stride, out, out_row_stride, rows, cols, esz, true) ||
         !alias_ok(b, b_row_stride, out, out_row_stride, rows, cols, esz, true))
         return KOP_ERR_BAD_ALIAS;
-    if (rows == 0) return KOP_OK;
     if ((st = check_device()) != KOP_OK) return st;
     cudaStream_t s = as_stream(stream);
     return dtype == KOP_F32
@@ -431,10 +438,11 @@ extern "C" kop_status_t kop_rmsnorm_swiglu_residual(void* handle, const void* h,
 {
     using namespace kop;
     if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
-    if (!handle || !h || !rms_weight || !w_gate_up || !w_down || !out || !workspace)
-        return KOP_ERR_NULL_POINTER;
     if (rows < 0 || hidden <= 0 || inter <= 0) return KOP_ERR_BAD_SHAPE;
     if (hidden > 0x7FFFFFFFLL || inter > 0x3FFFFFFFLL || rows > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+    if (rows == 0) return KOP_OK;
+    if (!handle || !h || !rms_weight || !w_gate_up || !w_down || !out || !workspace)
+        return KOP_ERR_NULL_POINTER;
     const int esz = elem_size(dtype);
     if (!aligned_to(h, esz) || !aligned_to(out, esz) || !aligned_to(w_gate_up, esz) ||
         !aligned_to(w_down, esz) || !aligned_to(rms_weight, 4) || !aligned_to(workspace, 256))
@@ -443,7 +451,6 @@ extern "C" kop_status_t kop_rmsnorm_swiglu_residual(void* handle, const void* h,
     if (!alias_ok(h, hidden, out, hidden, rows, hidden, esz, true)) return KOP_ERR_BAD_ALIAS;
     const MlpLayout L = mlp_layout(rows, hidden, inter, esz);
     if (workspace_bytes < L.total) return KOP_ERR_WORKSPACE_TOO_SMALL;
-    if (rows == 0) return KOP_OK;
     kop_status_t st = check_device();
     if (st != KOP_OK) return st;
 

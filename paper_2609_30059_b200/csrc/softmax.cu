@@ -248,16 +248,16 @@ extern "C" kop_status_t kop_softmax_scale_bias(const void* x, const float* bias,
 {
     using namespace kop;
     if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
-    if (x == nullptr || y == nullptr) return KOP_ERR_NULL_POINTER;
     kop_status_t st = check_rows_cols(rows, cols);
     if (st != KOP_OK) return st;
+    if (rows == 0) return KOP_OK;                       // empty: nothing to validate further or launch
+    if (x == nullptr || y == nullptr) return KOP_ERR_NULL_POINTER;
     if ((st = check_row_stride(x_row_stride, cols, rows)) != KOP_OK) return st;
     if ((st = check_row_stride(y_row_stride, cols, rows)) != KOP_OK) return st;
     const int esz = elem_size(dtype);
     if (!aligned_to(x, esz) || !aligned_to(y, esz) || (bias != nullptr && !aligned_to(bias, 4)))
         return KOP_ERR_MISALIGNED;
     if (!alias_ok(x, x_row_stride, y, y_row_stride, rows, cols, esz, true)) return KOP_ERR_BAD_ALIAS;
-    if (rows == 0) return KOP_OK;
     if ((st = check_device()) != KOP_OK) return st;
     cudaStream_t s = as_stream(stream);
     return dtype == KOP_F32
