@@ -146,6 +146,39 @@ kop_status_t kop_ce_loss_rowwise(const void* logits, const int32_t* labels,
 size_t kop_ce_loss_rowwise_workspace_bytes(int64_t rows, int64_t vocab, kop_dtype_t dtype);
 
 /*
+ * kop_ce_loss_rowwise for callers that cannot allocate. (The paper has no counterpart: this is a
+ * packaging variant of the entry point above, same arithmetic, same kernels.)
+ *
+ * Who needs it: code that has no allocator to turn to at the point of the call — a plug-in inside
+ * another runtime's operator that cannot reach that runtime's memory pool (and where a raw
+ * cudaMalloc would synchronise the device and take memory the pool does not know about), a server
+ * whose memory plan is frozen after start-up, a C caller on a latency-critical path. Instead of a
+ * caller-supplied workspace, the scratch of the mean reduction (tickets and per-group partials) is
+ * a fixed device array inside the library: 49,168 bytes that every GPU which loads the library
+ * holds until the process exits.
+ *
+ * Arguments, outputs, results and error behaviour are those of kop_ce_loss_rowwise without the
+ * workspace pair, with these additions:
+ *   limit     rows <= kop_ce_loss_rowwise_static_max_rows() (1,048,576). More rows return
+ *             KOP_ERR_WORKSPACE_TOO_SMALL before anything is launched; use the workspace variant.
+ *   set-up    The first call on each device looks up the device address of the built-in array
+ *             (once per device, with that device current). Make that first call outside any
+ *             stream capture. The call itself never calls cudaMalloc, cudaFree or any allocating
+ *             library routine; it clears the tickets it needs on `stream`.
+ *   sharing   Every call on a device uses the same array, which keeps the previous call's
+ *             contents. Calls that may overlap on the GPU (different streams, different threads)
+ *             race on it and give wrong means: serialise them, or use kop_ce_loss_rowwise with
+ *             one workspace per concurrent call.
+ */
+kop_status_t kop_ce_loss_rowwise_static(const void* logits, const int32_t* labels,
+                                        float* loss, float* mean_loss, int32_t* bad_label_count,
+                                        int64_t rows, int64_t vocab, int64_t row_stride,
+                                        kop_dtype_t dtype, kop_stream_t stream);
+
+/* Largest `rows` kop_ce_loss_rowwise_static accepts. */
+int64_t kop_ce_loss_rowwise_static_max_rows(void);
+
+/*
  * RMSNorm (fusion agent: "normalization fusion (LayerNorm/RMSNorm sequences)"):
  *   y[i,j] = x[i,j] / sqrt(mean_j x[i,j]^2 + eps) * weight[j]
  * x, y: [rows, hidden] of `dtype`; weight: fp32 [hidden]. y may alias x exactly.

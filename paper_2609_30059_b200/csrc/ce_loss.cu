@@ -263,3 +263,72 @@ extern "C" kop_status_t kop_ce_loss_rowwise(const void* logits, const int32_t* l
                ? launch_ce<float>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s)
                : launch_ce<__nv_bfloat16>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s);
 }
+
+// ------------------------------------------------------------------------------------------------
+// kop_ce_loss_rowwise_static: the same cross-entropy, for callers that cannot allocate.
+//
+// Some callers have no way to get scratch memory at the point of the call: a plug-in running inside
+// another runtime's operator has no handle on that runtime's memory pool, and a raw cudaMalloc there
+// would synchronise the whole device and grow memory behind the pool's back; a serving process that
+// fixed its memory plan at start-up may forbid driver allocations afterwards; C callers on a
+// latency-critical path cannot afford an allocator round trip per call. For them the ticket / partial
+// scratch of the mean reduction lives in a file-scope device array that every GPU loading this
+// library holds until the process exits. Its size fixes the largest problem this entry point takes.
+namespace kop {
+namespace {
+
+constexpr int64_t kStaticMaxRows = (int64_t)1 << 20;                       // 1,048,576 rows
+constexpr int64_t kStaticScratchWords = 4 + 3 * (kStaticMaxRows / kGroupRows);   // 12,292 words = 49,168 B
+static __device__ __align__(256) unsigned int g_ce_static_scratch[kStaticScratchWords];
+
+// In host code the array's name is only a stand-in for the symbol, not a device address: the address
+// the kernel needs comes from cudaGetSymbolAddress, asked once per device with that device current.
+constexpr int kStaticMaxDevices = 64;
+void* g_ce_static_ptr[kStaticMaxDevices];      // benign race: every writer stores the same value
+
+kop_status_t ce_static_scratch(void** out)
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return KOP_ERR_CUDA;
+    }
+    if (dev < 0 || dev >= kStaticMaxDevices) return KOP_ERR_UNSUPPORTED_DEVICE;
+    if (g_ce_static_ptr[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_ce_static_scratch) != cudaSuccess || p == nullptr) {
+            (void)cudaGetLastError();
+            return KOP_ERR_CUDA;
+        }
+        g_ce_static_ptr[dev] = p;
+    }
+    *out = g_ce_static_ptr[dev];
+    return KOP_OK;
+}
+
+}  // namespace
+}  // namespace kop
+
+extern "C" int64_t kop_ce_loss_rowwise_static_max_rows(void) { return kop::kStaticMaxRows; }
+
+extern "C" kop_status_t kop_ce_loss_rowwise_static(const void* logits, const int32_t* labels,
+                                                   float* loss, float* mean_loss,
+                                                   int32_t* bad_label_count, int64_t rows, int64_t vocab,
+                                                   int64_t row_stride, kop_dtype_t dtype,
+                                                   kop_stream_t stream)
+{
+    using namespace kop;
+    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    kop_status_t st = check_rows_cols(rows, vocab);
+    if (st != KOP_OK) return st;
+    if (rows == 0) return KOP_OK;
+    // Beyond the built-in scratch: refuse, loudly, before touching the device.
+    if (rows > kStaticMaxRows) return KOP_ERR_WORKSPACE_TOO_SMALL;
+    if ((st = check_device()) != KOP_OK) return st;
+    void* scratch = nullptr;
+    if ((st = ce_static_scratch(&scratch)) != KOP_OK) return st;
+    // Same validation, same clearing of the tickets on `stream`, same kernels as the caller-workspace
+    // entry point; only the scratch pointer differs.
+    return kop_ce_loss_rowwise(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride,
+                               scratch, (size_t)kStaticScratchWords * sizeof(unsigned int), dtype, stream);
+}

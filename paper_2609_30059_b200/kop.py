@@ -57,6 +57,10 @@ def lib() -> C.CDLL:
     L.kop_ce_loss_rowwise.argtypes = [vp] * 5 + [i64] * 3 + [vp, sz, i32, vp]
     L.kop_ce_loss_rowwise_workspace_bytes.restype = sz
     L.kop_ce_loss_rowwise_workspace_bytes.argtypes = [i64, i64, i32]
+    L.kop_ce_loss_rowwise_static.argtypes = [vp] * 5 + [i64] * 3 + [i32, vp]
+    L.kop_ce_loss_rowwise_static.restype = i32
+    L.kop_ce_loss_rowwise_static_max_rows.restype = i64
+    L.kop_ce_loss_rowwise_static_max_rows.argtypes = []
     L.kop_rmsnorm.argtypes = [vp, vp, vp, i64, i64, i64, i64, f32, i32, vp]
     L.kop_silu_mul.argtypes = [vp, vp, i64, i64, i64, i64, i32, vp]
     L.kop_residual_add.argtypes = [vp, vp, vp, i64, i64, i64, i64, i64, i32, vp]
@@ -178,6 +182,26 @@ def kop_ce_loss_rowwise(logits, labels, loss=None, mean_loss=None, bad_label_cou
                                      mean_loss.data_ptr(), bad_label_count.data_ptr(), rows, vocab, zs,
                                      workspace.data_ptr(), workspace.numel() * workspace.element_size(),
                                      _dtype_tag(logits), _stream(stream)), "kop_ce_loss_rowwise")
+    return loss, mean_loss, bad_label_count
+
+
+def kop_ce_loss_rowwise_static_max_rows() -> int:
+    return lib().kop_ce_loss_rowwise_static_max_rows()
+
+
+def kop_ce_loss_rowwise_static(logits, labels, loss, mean_loss, bad_label_count, stream=None):
+    """kop_ce_loss_rowwise without a workspace argument, for callers that cannot allocate: the
+    scratch is a fixed array inside the library (see include/kop.h for the row limit, the one-time
+    per-device set-up on the first call, and why overlapping calls race). This wrapper allocates
+    nothing either: the caller passes every output tensor."""
+    rows, vocab, zs = _rows2d(logits, "logits")
+    if labels.dtype != torch.int32 or not labels.is_cuda or not labels.is_contiguous() or labels.numel() != rows:
+        raise ValueError("labels: expected a contiguous int32 CUDA vector of `rows` elements")
+    _check(lib().kop_ce_loss_rowwise_static(
+        logits.data_ptr(), labels.data_ptr(), loss.data_ptr(),
+        None if mean_loss is None else mean_loss.data_ptr(),
+        None if bad_label_count is None else bad_label_count.data_ptr(),
+        rows, vocab, zs, _dtype_tag(logits), _stream(stream)), "kop_ce_loss_rowwise_static")
     return loss, mean_loss, bad_label_count
 
 
