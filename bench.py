@@ -94,6 +94,25 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
 
 
+# ----------------------------------------------------------------------------- multi-rank aggregation
+
+def max_over_ranks(values, world, device="cpu"):
+    """Element-wise max of a list of floats over all ranks (identity when world == 1). The path has no
+    data exchange: replicas run independently and only these timings cross ranks."""
+    if world <= 1:
+        return [float(v) for v in values]
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def aggregate_throughput(bytes_per_rank, ms_local, world, device="cpu"):
+    """Whole-job GB/s of `world` independent replicas: every rank moves bytes_per_rank in ms_local;
+    the job takes as long as its slowest rank."""
+    (ms,) = max_over_ranks([ms_local], world, device)
+    return world * bytes_per_rank / (ms * 1e-3) / 1e9, ms
+
+
 # ----------------------------------------------------------------------------- clocks sampling
 
 class ClockSampler:
@@ -333,13 +352,8 @@ def run_ours(args, rank, world, local_rank):
     fused_ms_step = sum(statistics.mean(per[nm]) for nm in names)
     fused_bytes = sum(segs[nm]["bytes"] for nm in names)
     # max over ranks of the timed quantities
-    if world > 1:
-        t = torch.tensor([total_ms, fused_ms_step], dtype=torch.float64, device=dev)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        total_ms, fused_ms_step_max = float(t[0]), float(t[1])
-    else:
-        fused_ms_step_max = fused_ms_step
-    value = world * fused_bytes / (fused_ms_step_max * 1e-3) / 1e9
+    (total_ms,) = max_over_ranks([total_ms], world, dev)
+    value, fused_ms_step_max = aggregate_throughput(fused_bytes, fused_ms_step, world, dev)
 
     peak, peak_src = measured_peak()
 
@@ -437,12 +451,9 @@ def run_e2e(args, wl, kop, dev, segs, names, world):
     torch.cuda.synchronize()
     wall = (time.perf_counter() - wall0) * 1e3
     ms = max(t0.elapsed_time(t1), wall) / steps
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        ms = float(t[0])
     fused_bytes = sum(segs[nm]["bytes"] for nm in names)
-    return {"value": round(world * fused_bytes / (ms * 1e-3) / 1e9, 2), "unit": UNIT, "ms_per_step": round(ms, 3),
+    e2e_value, ms = aggregate_throughput(fused_bytes, ms, world, dev)
+    return {"value": round(e2e_value, 2), "unit": UNIT, "ms_per_step": round(ms, 3),
             "steps": steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
             "includes": "pinned-host H2D of all data inputs, all fused kernels, both cuBLAS GEMMs, D2H of all outputs"}
 

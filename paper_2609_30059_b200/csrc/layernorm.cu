@@ -123,6 +123,113 @@ ln_block_kernel(const T* __restrict__ x, const T* __restrict__ res, const float*
     }
 }
 
+// Two rows per CTA. The fp32 parameter vectors are three times the bytes of a bf16 row, and at
+// one row per CTA their L1 wavefronts (not HBM) bound the kernel (with the parameter loads stubbed
+// out the kernel runs at the speed of a plain two-reads-one-write stream). Each thread therefore
+// fetches its bias / gamma / beta once and applies them to the same columns of two rows, which
+// halves that traffic; both rows' reductions share the two barriers. The row must be exactly
+// blockDim.x * VPT vectors; `rows` may be odd (the last CTA then skips its second row).
+template <typename T, int VPT, bool kWide, int kMaxThreads>
+__global__ void __launch_bounds__(kMaxThreads, 768 / kMaxThreads)
+ln_pair_kernel(const T* __restrict__ x, const T* __restrict__ res, const float* __restrict__ bias,
+               const float* __restrict__ gamma, const float* __restrict__ beta, T* __restrict__ y,
+               float* __restrict__ mean, float* __restrict__ rstd, int64_t rows, int64_t x_stride,
+               int64_t r_stride, int64_t y_stride, float eps, float inv_hidden)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    constexpr int P = E / 2;
+    constexpr bool kFast = sizeof(T) == 2;
+    __shared__ float red_a[2][32], red_b[2][32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    const int64_t row0 = (int64_t)blockIdx.x * 2;
+    const bool two = row0 + 1 < rows;
+
+    Vec16 rx[2][VPT], rres[2][VPT];
+#pragma unroll
+    for (int r = 0; r < 2; ++r)
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            const int64_t v = (int64_t)k * blockDim.x + threadIdx.x;
+            if (r == 0 || two) {
+                rx[r][k] = ld_stream(x + (row0 + r) * x_stride + v * E);
+                rres[r][k] = ld_stream(res + (row0 + r) * r_stride + v * E);
+            } else {
+                rx[r][k] = Vec16{{0u, 0u, 0u, 0u}};
+                rres[r][k] = Vec16{{0u, 0u, 0u, 0u}};
+            }
+        }
+    float2 val[2][VPT][P];
+    float2 sum2[2] = {make_float2(0.0f, 0.0f), make_float2(0.0f, 0.0f)};
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+        const int64_t v = (int64_t)k * blockDim.x + threadIdx.x;
+        float2 bb[P];
+        load_params<E, kWide>(bias + v * E, bb);
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            float2 fx[P], fr[P];
+            Elem<T>::unpack2(rx[r][k], fx);
+            Elem<T>::unpack2(rres[r][k], fr);
+#pragma unroll
+            for (int q = 0; q < P; ++q) {
+                const float2 t = gelu_residual2<kFast>(fx[q], bb[q], fr[q]);
+                val[r][k][q] = t;
+                sum2[r] = __fadd2_rn(sum2[r], t);
+            }
+        }
+    }
+    float mu[2], rs[2];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const float s = warp_sum(sum2[r].x + sum2[r].y);
+        if (lane == 0) red_a[r][warp] = s;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < 2; ++r) mu[r] = warp_sum(lane < nw ? red_a[r][lane] : 0.0f) * inv_hidden;
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const float2 nmu = make_float2(-mu[r], -mu[r]);
+        float2 ss2 = make_float2(0.0f, 0.0f);
+#pragma unroll
+        for (int k = 0; k < VPT; ++k)
+#pragma unroll
+            for (int q = 0; q < P; ++q) {
+                const float2 d = __fadd2_rn(val[r][k][q], nmu);
+                val[r][k][q] = d;
+                ss2 = __ffma2_rn(d, d, ss2);
+            }
+        const float s = warp_sum(ss2.x + ss2.y);
+        if (lane == 0) red_b[r][warp] = s;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        rs[r] = rsqrtf(warp_sum(lane < nw ? red_b[r][lane] : 0.0f) * inv_hidden + eps);
+        if (threadIdx.x == 0 && (r == 0 || two)) {
+            if (mean != nullptr) mean[row0 + r] = mu[r];
+            if (rstd != nullptr) rstd[row0 + r] = rs[r];
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+        const int64_t v = (int64_t)k * blockDim.x + threadIdx.x;
+        float2 g[P], b[P];
+        load_params<E, kWide>(gamma + v * E, g);
+        load_params<E, kWide>(beta + v * E, b);
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            if (r == 0 || two) {
+                const float2 rs2 = make_float2(rs[r], rs[r]);
+                float2 o[P];
+#pragma unroll
+                for (int q = 0; q < P; ++q) o[q] = __ffma2_rn(__fmul2_rn(val[r][k][q], rs2), g[q], b[q]);
+                st_stream(y + (row0 + r) * y_stride + v * E, Elem<T>::pack2(o));
+            }
+        }
+    }
+}
+
 // Any hidden size / alignment: scalar loads, v recomputed in each of three sweeps.
 template <typename T>
 __global__ void __launch_bounds__(256)
@@ -179,6 +286,24 @@ kop_status_t launch_ln(const void* xv, const void* rv, const float* bias, const 
         const int nvec = (int)nvec64;
         // 32 values per thread (hidden 4096 -> 128-thread CTAs, eight 16-byte loads in flight per
         // thread and ~8 CTAs per SM); short rows use fewer, rows beyond 512 threads' worth use 64.
+        const bool wide = E == 8 && aligned_to(bias, 32) && aligned_to(gamma, 32) && aligned_to(beta, 32);
+        // Rows of 2048..8192 elements that split evenly into 16 values per thread go two per CTA
+        // (parameters fetched once per pair) once there are enough pairs to fill the GPU.
+        {
+            const int vpt2 = 16 / E;
+            const int threads2 = nvec / vpt2;
+            if (nvec % vpt2 == 0 && threads2 % 32 == 0 && threads2 >= 128 && threads2 <= 512 &&
+                rows >= 8 * (int64_t)sm_count()) {
+                const unsigned grid = (unsigned)((rows + 1) / 2);
+#define KOP_LN_PAIR(W, MT)                                                                              \
+    ln_pair_kernel<T, 16 / E, W, MT><<<grid, threads2, 0, stream>>>(x, r, bias, gamma, beta, y, mean, rstd, \
+                                                                    rows, xs, rs, ys, eps, inv_hidden)
+                if (threads2 <= 256) { if (wide) KOP_LN_PAIR(true, 256); else KOP_LN_PAIR(false, 256); }
+                else { if (wide) KOP_LN_PAIR(true, 512); else KOP_LN_PAIR(false, 512); }
+#undef KOP_LN_PAIR
+                return launch_status();
+            }
+        }
         int vals = 32;
         if (hidden <= 1024) vals = 16;
         if (hidden <= 256) vals = 8;
@@ -186,7 +311,6 @@ kop_status_t launch_ln(const void* xv, const void* rv, const float* bias, const 
         const int vpt = vals / E;
         const int threads = ((nvec + vpt - 1) / vpt + 31) / 32 * 32;
         const bool full = (nvec % vpt) == 0 && (nvec / vpt) == threads;
-        const bool wide = E == 8 && aligned_to(bias, 32) && aligned_to(gamma, 32) && aligned_to(beta, 32);
 #define KOP_LN_LAUNCH(V, F, W)                                                                    \
     ln_block_kernel<T, V, F, W><<<(unsigned)rows, threads, 0, stream>>>(x, r, bias, gamma, beta, y, mean, \
                                                                         rstd, nvec, xs, rs, ys, eps, inv_hidden)

@@ -108,7 +108,9 @@ def test_softmax_options(kop):
 # ------------------------------------------------------------------------------------------ LayerNorm
 
 LN_SHAPES = [
-    (2048, 4096, BF16),    # benchmark row length, >= 4 waves of CTAs
+    (2048, 4096, BF16),    # benchmark row length, >= 4 waves of CTAs (two rows per CTA)
+    (1185, 4096, BF16),    # odd row count on the two-rows-per-CTA kernel
+    (1301, 2048, F32),     # the same kernel on fp32 rows
     (300, 4096, F32),
     (129, 1024, BF16),
     (65, 256, BF16),
