@@ -116,20 +116,57 @@ def aggregate_throughput(bytes_per_rank, ms_local, world, device="cpu"):
 # ----------------------------------------------------------------------------- clocks sampling
 
 class ClockSampler:
+    """Samples the SM clock, power and throttle reasons of one GPU while the timed region runs: NVML
+    from a background thread every few milliseconds (read-only queries), or an `nvidia-smi -lms` child
+    process when NVML cannot be loaded."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, device: int):
-        self.proc = None
-        self.path = None
+    def __init__(self, device: int, period_s: float = 0.004):
+        self.period = period_s
+        self.proc = self.path = self.thread = self.handle = None
+        self.sm, self.power, self.reasons, self.max_mhz = [], [], set(), None
+        self.stop_flag = False
         try:
             uuid = str(torch.cuda.get_device_properties(device).uuid)
             self.sel = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
         except Exception:
             self.sel = str(device)
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nvml = pynvml
+            try:
+                self.handle = pynvml.nvmlDeviceGetHandleByUUID(self.sel.encode())
+            except Exception:
+                self.handle = pynvml.nvmlDeviceGetHandleByUUID(self.sel)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.handle = None
+
+    def _loop(self):
+        n = self.nvml
+        while not self.stop_flag:
+            try:
+                self.sm.append(float(n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM)))
+                self.power.append(n.nvmlDeviceGetPowerUsage(self.handle) / 1000.0)
+                bits = int(n.nvmlDeviceGetCurrentClocksEventReasons(self.handle))
+                for bit, name in self.REASONS.items():
+                    if bits & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
 
     def start(self):
+        if self.handle is not None:
+            import threading
+            self.thread = threading.Thread(target=self._loop, daemon=True)
+            self.thread.start()
+            return
         try:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
@@ -140,7 +177,16 @@ class ClockSampler:
             self.proc = None
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "source": None}
+        if self.thread is not None:
+            self.stop_flag = True
+            self.thread.join(timeout=2)
+            if self.sm:
+                out.update(sm_mhz=statistics.median(self.sm), sm_min_mhz=min(self.sm), sm_max_mhz=self.max_mhz,
+                           power_w_max=round(max(self.power), 1) if self.power else None, samples=len(self.sm))
+            out["reasons"] = sorted(self.reasons)
+            out["source"] = "nvml"
+            return out
         if self.proc is None:
             return out
         self.proc.terminate()
@@ -168,6 +214,7 @@ class ClockSampler:
         if sm:
             out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
         out["reasons"] = sorted(reasons)
+        out["source"] = "nvidia-smi"
         return out
 
 
@@ -331,7 +378,7 @@ def run_ours(args, rank, world, local_rank):
         g = [ev[len(names)][0].elapsed_time(ev[len(names)][1]) for ev in all_events] if with_graph else []
         return t0.elapsed_time(t1), per, g
 
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(local_rank, args.clock_sample_ms * 1e-3)
     sampler.start()
     for _ in range(max(args.warmup, 3)):
         step(new_events())
@@ -341,7 +388,7 @@ def run_ours(args, rank, world, local_rank):
     # ---- the MLP segment as a CUDA graph (our three kernels + the two preserved cuBLAS GEMMs), and
     # the fused kernels again when they alternate with it: the GEMMs pull the GPU into its power cap,
     # so this second set shows the same kernels at the lower clocks they see inside a model.
-    sampler2 = ClockSampler(local_rank)
+    sampler2 = ClockSampler(local_rank, args.clock_sample_ms * 1e-3)
     sampler2.start()
     situ_steps = max(3, min(args.steps, 20))
     for _ in range(3):
@@ -609,6 +656,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--clock-sample-ms", type=float, default=4.0, help="period of the SM-clock sampler")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="CPU time budget of the cpu_baseline leg")
     ap.add_argument("--profile", default=None, help="comma list of segments to launch alone (ncu / quick timing)")
     ap.add_argument("--rows-div", type=int, default=1, help="with --profile: divide every row count by this")

@@ -50,7 +50,7 @@ bn_plane_block_kernel(const T* __restrict__ x, const float* __restrict__ scale,
     if (threadIdx.x == 0) pooled[p] = sum * inv_plane;
 }
 
-// One warp per plane (small planes), scalar or vector by template flag; grid-stride over planes.
+// One warp per plane (small planes), scalar or vector by template flag.
 template <typename T, bool kVec>
 __global__ void __launch_bounds__(256)
 bn_plane_warp_kernel(const T* __restrict__ x, const float* __restrict__ scale,
@@ -59,9 +59,8 @@ bn_plane_warp_kernel(const T* __restrict__ x, const float* __restrict__ scale,
 {
     constexpr int E = Elem<T>::kPerVec;
     const int lane = threadIdx.x & 31;
-    const int64_t wpc = blockDim.x >> 5;
-    const int64_t nwarps = (int64_t)gridDim.x * wpc;
-    for (int64_t p = (int64_t)blockIdx.x * wpc + (threadIdx.x >> 5); p < planes; p += nwarps) {
+    const int64_t p = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (p < planes) {
         const int c = (int)(p % C);
         const float sc = __ldg(scale + c), sh = __ldg(shift + c);
         const T* xp = x + p * plane_elems;
@@ -127,8 +126,8 @@ kop_status_t launch_bn(const void* xv, const float* scale, const float* shift, v
     const int64_t nvec64 = plane / E;
     if (plane <= 1024 || planes > 0x7FFFFFFFLL) {
         const int64_t ctas = (planes + 7) / 8;
-        const int64_t cap = (int64_t)sm_count() * 8;
-        const unsigned grid = (unsigned)(ctas < cap ? ctas : cap);
+        if (ctas > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+        const unsigned grid = (unsigned)ctas;
         if (vec)
             bn_plane_warp_kernel<T, true><<<grid, 256, 0, stream>>>(x, scale, shift, y, pooled, planes, plane, (int)C, inv_plane);
         else

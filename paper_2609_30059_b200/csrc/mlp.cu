@@ -81,7 +81,8 @@ __device__ __forceinline__ float silu(float g)
 }
 
 // A CTA covers `U * blockDim.x` consecutive output vectors of one row (tile index = blockIdx.x).
-template <typename T, int U>
+// kFull: the row is a whole number of tiles (no bounds predicates).
+template <typename T, int U, bool kFull>
 __global__ void __launch_bounds__(256)
 silu_mul_kernel(const T* __restrict__ gu, T* __restrict__ out, int nvec, int tiles_per_row,
                 int64_t inter, int64_t in_stride, int64_t out_stride)
@@ -98,7 +99,7 @@ silu_mul_kernel(const T* __restrict__ gu, T* __restrict__ out, int nvec, int til
 #pragma unroll
     for (int k = 0; k < U; ++k) {
         const int v = v0 + k * blockDim.x;
-        if (v < nvec) {
+        if (kFull || v < nvec) {
             rg[k] = ld_stream(g + (int64_t)v * E);
             ru[k] = ld_stream(u + (int64_t)v * E);
         }
@@ -106,7 +107,7 @@ silu_mul_kernel(const T* __restrict__ gu, T* __restrict__ out, int nvec, int til
 #pragma unroll
     for (int k = 0; k < U; ++k) {
         const int v = v0 + k * blockDim.x;
-        if (v < nvec) {
+        if (kFull || v < nvec) {
             float fg[E], fu[E];
             Elem<T>::unpack(rg[k], fg);
             Elem<T>::unpack(ru[k], fu);
@@ -134,7 +135,7 @@ silu_mul_scalar_kernel(const T* __restrict__ gu, T* __restrict__ out, int64_t ro
 }
 
 // ---- residual add -----------------------------------------------------------------------------------
-template <typename T, int U>
+template <typename T, int U, bool kFull>
 __global__ void __launch_bounds__(256)
 residual_add_kernel(const T* __restrict__ a, const T* __restrict__ b, T* __restrict__ out, int64_t nvec,
                     int64_t tiles_per_row, int64_t a_stride, int64_t b_stride, int64_t o_stride)
@@ -150,7 +151,7 @@ residual_add_kernel(const T* __restrict__ a, const T* __restrict__ b, T* __restr
 #pragma unroll
     for (int k = 0; k < U; ++k) {
         const int64_t v = v0 + k * blockDim.x;
-        if (v < nvec) {
+        if (kFull || v < nvec) {
             ra[k] = ld_stream(ar + v * E);
             rb[k] = ld_stream(br + v * E);
         }
@@ -158,7 +159,7 @@ residual_add_kernel(const T* __restrict__ a, const T* __restrict__ b, T* __restr
 #pragma unroll
     for (int k = 0; k < U; ++k) {
         const int64_t v = v0 + k * blockDim.x;
-        if (v < nvec) {
+        if (kFull || v < nvec) {
             float fa[E], fb[E];
             Elem<T>::unpack(ra[k], fa);
             Elem<T>::unpack(rb[k], fb);
@@ -255,7 +256,10 @@ kop_status_t launch_silu_mul(const void* guv, void* outv, int64_t rows, int64_t 
         const int tiles = (nvec + threads * U - 1) / (threads * U);
         const int64_t grid = rows * tiles;
         if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
-        silu_mul_kernel<T, U><<<(unsigned)grid, threads, 0, stream>>>(gu, out, nvec, tiles, inter, is, os);
+        if (nvec % (threads * U) == 0)
+            silu_mul_kernel<T, U, true><<<(unsigned)grid, threads, 0, stream>>>(gu, out, nvec, tiles, inter, is, os);
+        else
+            silu_mul_kernel<T, U, false><<<(unsigned)grid, threads, 0, stream>>>(gu, out, nvec, tiles, inter, is, os);
         return launch_status();
     }
     silu_mul_scalar_kernel<T><<<scalar_grid(rows * inter), 256, 0, stream>>>(gu, out, rows, inter, is, os);
@@ -285,7 +289,10 @@ kop_status_t launch_residual_add(const void* av, const void* bv, void* ov, int64
         const int64_t tiles = (nvec + threads * U - 1) / (threads * U);
         const int64_t grid = rows * tiles;
         if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
-        residual_add_kernel<T, U><<<(unsigned)grid, threads, 0, stream>>>(a, b, out, nvec, tiles, as, bs, os);
+        if (nvec % (threads * U) == 0)
+            residual_add_kernel<T, U, true><<<(unsigned)grid, threads, 0, stream>>>(a, b, out, nvec, tiles, as, bs, os);
+        else
+            residual_add_kernel<T, U, false><<<(unsigned)grid, threads, 0, stream>>>(a, b, out, nvec, tiles, as, bs, os);
         return launch_status();
     }
     residual_add_scalar_kernel<T><<<scalar_grid(rows * cols), 256, 0, stream>>>(a, b, out, rows, cols, as, bs, os);

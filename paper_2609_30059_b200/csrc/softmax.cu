@@ -10,95 +10,68 @@
 namespace kop {
 namespace {
 
-// ---- warp per row, grid-stride over rows, bias kept in registers ------------------------------
-template <typename T, int VPL, bool kBiasInRegs>
+// ---- warp per row, one row per warp ---------------------------------------------------------------
+// (A grid-stride version with the bias held in registers across rows measured 8 % slower on
+// [131072, 512] fp32: many short-lived CTAs at different phases overlap loads, math and stores better
+// than a few resident warps that each serialise them.)
+// kFull: the row is exactly 32 * VPL vectors (no tail predicates); kBias: bias != NULL.
+template <typename T, int VPL, bool kFull, bool kBias>
 __global__ void __launch_bounds__(256)
 softmax_warp_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* __restrict__ y,
                     int64_t rows, int nvec, int64_t x_stride, int64_t y_stride, float scale)
 {
     constexpr int E = Elem<T>::kPerVec;
     const int lane = threadIdx.x & 31;
-    const int64_t warps_per_cta = blockDim.x >> 5;
-    const int64_t warp0 = (int64_t)blockIdx.x * warps_per_cta + (threadIdx.x >> 5);
-    const int64_t nwarps = (int64_t)gridDim.x * warps_per_cta;
+    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= rows) return;
     const float s2 = scale * kLog2e;
-
-    // Short rows keep the (pre-scaled) bias in registers across the rows a warp visits; wider
-    // rows re-read it through L1, where the streaming data loads never allocate.
-    float b2[kBiasInRegs ? VPL : 1][E];
+    const T* xr = x + row * x_stride;
+    T* yr = y + row * y_stride;
+    Vec16 raw[VPL];
 #pragma unroll
-    for (int k = 0; k < (kBiasInRegs ? VPL : 0); ++k) {
+    for (int k = 0; k < VPL; ++k) {
         const int v = k * 32 + lane;
-#pragma unroll
-        for (int e = 0; e < E; ++e) b2[k][e] = 0.0f;
-        if (bias != nullptr && v < nvec) {
-#pragma unroll
-            for (int q = 0; q < E / 4; ++q) {
-                float4 t = ldg_f4(bias + (int64_t)v * E + 4 * q);
-                b2[k][4 * q + 0] = t.x * kLog2e;
-                b2[k][4 * q + 1] = t.y * kLog2e;
-                b2[k][4 * q + 2] = t.z * kLog2e;
-                b2[k][4 * q + 3] = t.w * kLog2e;
-            }
-        }
+        if (kFull || v < nvec) raw[k] = ld_stream(xr + (int64_t)v * E);
+        else raw[k] = Vec16{{0u, 0u, 0u, 0u}};
     }
-
-    for (int64_t row = warp0; row < rows; row += nwarps) {
-        const T* xr = x + row * x_stride;
-        T* yr = y + row * y_stride;
-        Vec16 raw[VPL];
+    float t[VPL][E];
+    float m = -INFINITY;
 #pragma unroll
-        for (int k = 0; k < VPL; ++k) {
-            const int v = k * 32 + lane;
-            if (v < nvec) raw[k] = ld_stream(xr + (int64_t)v * E);
-        }
-        float t[VPL][E];
-        float m = -INFINITY;
+    for (int k = 0; k < VPL; ++k) {
+        const int v = k * 32 + lane;
+        float f[E];
+        Elem<T>::unpack(raw[k], f);
 #pragma unroll
-        for (int k = 0; k < VPL; ++k) {
-            const int v = k * 32 + lane;
-            float f[E];
-            Elem<T>::unpack(raw[k], f);
-            float bk[E];
-            if (kBiasInRegs) {
+        for (int q = 0; q < E / 4; ++q) {
+            float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (kBias && (kFull || v < nvec)) b = ldg_f4(bias + (int64_t)v * E + 4 * q);
+            const float bb[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
-                for (int e = 0; e < E; ++e) bk[e] = b2[k][e];
-            } else {
-#pragma unroll
-                for (int q = 0; q < E / 4; ++q) {
-                    float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (bias != nullptr && v < nvec) b = ldg_f4(bias + (int64_t)v * E + 4 * q);
-                    bk[4 * q + 0] = b.x * kLog2e;
-                    bk[4 * q + 1] = b.y * kLog2e;
-                    bk[4 * q + 2] = b.z * kLog2e;
-                    bk[4 * q + 3] = b.w * kLog2e;
-                }
-            }
-#pragma unroll
-            for (int e = 0; e < E; ++e) {
-                t[k][e] = v < nvec ? fmaf(f[e], s2, bk[e]) : -INFINITY;
+            for (int c = 0; c < 4; ++c) {
+                const int e = 4 * q + c;
+                t[k][e] = (kFull || v < nvec) ? fmaf(f[e], s2, bb[c] * kLog2e) : -INFINITY;
                 m = fmaxf(m, t[k][e]);
             }
         }
-        m = warp_max(m);
-        float s = 0.0f;
+    }
+    m = warp_max(m);
+    float s = 0.0f;
 #pragma unroll
-        for (int k = 0; k < VPL; ++k)
+    for (int k = 0; k < VPL; ++k)
 #pragma unroll
-            for (int e = 0; e < E; ++e) {
-                t[k][e] = ex2_approx(t[k][e] - m);
-                s += t[k][e];
-            }
-        s = warp_sum(s);
-        const float inv = 1.0f / s;
-#pragma unroll
-        for (int k = 0; k < VPL; ++k) {
-            const int v = k * 32 + lane;
-            float o[E];
-#pragma unroll
-            for (int e = 0; e < E; ++e) o[e] = t[k][e] * inv;
-            if (v < nvec) st_stream(yr + (int64_t)v * E, Elem<T>::pack(o));
+        for (int e = 0; e < E; ++e) {
+            t[k][e] = ex2_approx(t[k][e] - m);
+            s += t[k][e];
         }
+    s = warp_sum(s);
+    const float inv = 1.0f / s;
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) {
+        const int v = k * 32 + lane;
+        float o[E];
+#pragma unroll
+        for (int e = 0; e < E; ++e) o[e] = t[k][e] * inv;
+        if (kFull || v < nvec) st_stream(yr + (int64_t)v * E, Elem<T>::pack(o));
     }
 }
 
@@ -207,13 +180,23 @@ kop_status_t launch_softmax(const void* xv, const float* bias, void* yv, int64_t
         const int nvec = (int)nvec64;
         const int vpl = (nvec + 31) / 32;
         const int threads = 256;
-        const int64_t ctas_needed = (rows + 7) / 8;
-        const int64_t cap = (int64_t)sm_count() * 8;   // 8 CTAs of 256 threads fill an SM
-        const unsigned grid = (unsigned)(ctas_needed < cap ? ctas_needed : cap);
-#define KOP_SM_WARP(V, B) softmax_warp_kernel<T, V, B><<<grid, threads, 0, stream>>>(x, bias, y, rows, nvec, xs, ys, scale)
-        if (vpl <= 1) KOP_SM_WARP(1, true);
-        else if (vpl <= 2) KOP_SM_WARP(2, true);
-        else KOP_SM_WARP(4, false);
+        const int64_t ctas = (rows + 7) / 8;
+        if (ctas > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+        const unsigned grid = (unsigned)ctas;
+        const int vp = vpl <= 1 ? 1 : (vpl <= 2 ? 2 : 4);
+        const bool full = nvec == 32 * vp;
+#define KOP_SM_WARP_L(V, F, B) softmax_warp_kernel<T, V, F, B><<<grid, threads, 0, stream>>>(x, bias, y, rows, nvec, xs, ys, scale)
+#define KOP_SM_WARP(V)                                                         \
+    do {                                                                       \
+        if (full && bias != nullptr) KOP_SM_WARP_L(V, true, true);             \
+        else if (full) KOP_SM_WARP_L(V, true, false);                          \
+        else if (bias != nullptr) KOP_SM_WARP_L(V, false, true);               \
+        else KOP_SM_WARP_L(V, false, false);                                   \
+    } while (0)
+        if (vp == 1) KOP_SM_WARP(1);
+        else if (vp == 2) KOP_SM_WARP(2);
+        else KOP_SM_WARP(4);
+#undef KOP_SM_WARP_L
 #undef KOP_SM_WARP
         return launch_status();
     }
