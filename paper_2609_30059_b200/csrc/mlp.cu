@@ -89,8 +89,10 @@ silu_mul_kernel(const T* __restrict__ gu, T* __restrict__ out, int nvec, int til
 {
     constexpr int E = Elem<T>::kPerVec;
     constexpr bool kFast = sizeof(T) == 2;
-    const int64_t row = blockIdx.x / tiles_per_row;
-    const int tile = (int)(blockIdx.x - row * tiles_per_row);
+    // blockIdx.x = row * tiles_per_row + tile; both factors fit 31 bits, so one 32-bit division.
+    const unsigned urow = blockIdx.x / (unsigned)tiles_per_row;
+    const int tile = (int)(blockIdx.x - urow * (unsigned)tiles_per_row);
+    const int64_t row = urow;
     const T* g = gu + row * in_stride;
     const T* u = g + inter;
     T* o = out + row * out_stride;
@@ -141,8 +143,10 @@ residual_add_kernel(const T* __restrict__ a, const T* __restrict__ b, T* __restr
                     int64_t tiles_per_row, int64_t a_stride, int64_t b_stride, int64_t o_stride)
 {
     constexpr int E = Elem<T>::kPerVec;
-    const int64_t row = blockIdx.x / tiles_per_row;
-    const int64_t tile = blockIdx.x - row * tiles_per_row;
+    // A contiguous tensor arrives as one long row (tiles_per_row == gridDim.x): no division at all.
+    const unsigned urow = tiles_per_row == (int64_t)gridDim.x ? 0u : blockIdx.x / (unsigned)tiles_per_row;
+    const int64_t row = urow;
+    const int64_t tile = blockIdx.x - urow * (unsigned)tiles_per_row;
     const T* ar = a + row * a_stride;
     const T* br = b + row * b_stride;
     T* orow = out + row * o_stride;
