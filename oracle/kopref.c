@@ -344,3 +344,39 @@ int kopref_gemm_nt(const void* A, int a_dtype, const void* Wt, int w_dtype, doub
         }
     return 0;
 }
+
+/* ---- row scale ("diag(a) * B" written as the O(N^2) product the paper's L1-012 case study reaches) ----
+ * out[i,j] = a[i] * B[i,j].  a has the data dtype of B. */
+int kopref_row_scale(const void* a, const void* B, double* out, int64_t rows, int64_t cols,
+        int64_t b_row_stride, int64_t out_row_stride, int dtype, int threads)
+{
+    if (!a || !B || !out || rows < 0 || cols <= 0 || bad_dtype(dtype)) return -1;
+    int nt = pick_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t i = 0; i < rows; ++i) {
+        double ai = load_elem(a, i, dtype);
+        for (int64_t j = 0; j < cols; ++j)
+            out[i * out_row_stride + j] = ai * load_elem(B, i * b_row_stride + j, dtype);
+    }
+    return 0;
+}
+
+/* ---- mat-vec with a bias sum (the form the paper's L2-018 case study reduces Linear -> Sum to) ----------
+ * out[i] = sum_k X[i,k] * w[k] + b_sum, with w[k] = sum_j W[j,k] and b_sum = sum_j b[j] precomputed by the
+ * caller (w fp32).  The later max / mean / logsumexp of that chain act on a single element per row and
+ * are identities. */
+int kopref_matvec_bias(const void* X, const float* w, double b_sum, double* out, int64_t M, int64_t K,
+        int64_t x_row_stride, int dtype, int threads)
+{
+    if (!X || !w || !out || M < 0 || K <= 0 || bad_dtype(dtype)) return -1;
+    int nt = pick_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t i = 0; i < M; ++i) {
+        double acc = 0.0;
+        for (int64_t k = 0; k < K; ++k) acc += load_elem(X, i * x_row_stride + k, dtype) * (double)w[k];
+        out[i] = acc + b_sum;
+    }
+    return 0;
+}

@@ -40,6 +40,8 @@ def lib() -> C.CDLL:
         _lib.kopref_silu_mul.argtypes = [vp] * 2 + [i64] * 4 + [C.c_int, C.c_int]
         _lib.kopref_residual_add.argtypes = [vp] * 3 + [i64] * 5 + [C.c_int, C.c_int]
         _lib.kopref_gemm_nt.argtypes = [vp, C.c_int, vp, C.c_int, vp, i64, i64, i64, C.c_int]
+        _lib.kopref_row_scale.argtypes = [vp, vp, vp, i64, i64, i64, i64, C.c_int, C.c_int]
+        _lib.kopref_matvec_bias.argtypes = [vp, vp, dbl, vp, i64, i64, i64, C.c_int, C.c_int]
     return _lib
 
 
@@ -206,6 +208,28 @@ def gemm_nt(a, w, threads=1) -> np.ndarray:
     assert K == K2
     out = np.empty((M, N), dtype=np.float64)
     _check(lib().kopref_gemm_nt(_p(aa), adt, _p(wa), wdt, _p(out), M, N, K, _nt(threads)), "gemm_nt")
+    return out
+
+
+def row_scale(a, b, threads=1) -> np.ndarray:
+    """out[i, :] = a[i] * b[i, :]."""
+    aa, adt = as_data(a)
+    ba, bdt = as_data(b)
+    assert adt == bdt and aa.ndim == 1 and aa.shape[0] == ba.shape[0]
+    rows, cols = ba.shape
+    out = np.empty((rows, cols), dtype=np.float64)
+    _check(lib().kopref_row_scale(_p(aa), _p(ba), _p(out), rows, cols, cols, cols, bdt, _nt(threads)), "row_scale")
+    return out
+
+
+def matvec_bias(x, w, b_sum, threads=1) -> np.ndarray:
+    """out[i] = sum_k x[i, k] * w[k] + b_sum (w fp32)."""
+    xa, dt = as_data(x)
+    M, K = xa.shape
+    wa = as_param(w)
+    assert wa.shape == (K,)
+    out = np.empty(M, dtype=np.float64)
+    _check(lib().kopref_matvec_bias(_p(xa), _p(wa), float(b_sum), _p(out), M, K, K, dt, _nt(threads)), "matvec_bias")
     return out
 
 

@@ -480,6 +480,48 @@ def test_mlp_chain_reduced_shape_vs_numpy():
     assert np.allclose(out, ref, rtol=1e-12, atol=1e-14)
 
 
+# --------------------------------------------------------------------------- row scale, mat-vec + bias sum
+
+def test_row_scale_is_diag_times_matrix():
+    n = 7
+    a = f32(RNG.standard_normal(n))
+    B = f32(RNG.standard_normal((n, 5)))
+    out = kopref.row_scale(a, B)
+    # the O(N^3) form the case study starts from: diag(a) @ B, in float64
+    assert np.array_equal(out, np.diag(a.astype(np.float64)) @ B.astype(np.float64))
+    assert np.array_equal(kopref.row_scale(f32(np.ones(n)), B), B.astype(np.float64))
+    ai = f32(RNG.integers(-4, 5, n))
+    Bi = f32(RNG.integers(-4, 5, (n, 5)))
+    assert np.array_equal(kopref.row_scale(ai, Bi), ai[:, None].astype(np.float64) * Bi)      # exact on integers
+    ab, Bb = to_bf16_bits(a), to_bf16_bits(B)
+    wa = torch.from_numpy(a).to(torch.bfloat16).to(torch.float64).numpy()
+    wB = torch.from_numpy(B).to(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(kopref.row_scale(ab, Bb), wa[:, None] * wB)
+
+
+def test_matvec_bias_equals_linear_then_sum_and_later_reductions_are_identities():
+    # sum_j (sum_k X_ik W_jk + b_j) = sum_k X_ik (sum_j W_jk) + sum_j b_j
+    M, K, N = 9, 13, 6
+    X = f32(RNG.standard_normal((M, K)))
+    Wm = f32(RNG.standard_normal((N, K)))
+    b = f32(RNG.standard_normal(N))
+    w_colsum = f32(Wm.astype(np.float64).sum(axis=0))           # rounded to fp32 as the caller would pass it
+    b_sum = float(b.astype(np.float64).sum())
+    out = kopref.matvec_bias(X, w_colsum, b_sum)
+    lin = kopref.gemm_nt(X, Wm) + b.astype(np.float64)[None, :]
+    assert np.allclose(out, lin.sum(axis=1), rtol=0, atol=1e-5)      # fp32 rounding of the column sums only
+    exact = X.astype(np.float64) @ w_colsum.astype(np.float64) + b_sum
+    assert np.allclose(out, exact, rtol=1e-14, atol=1e-14)
+    # max, mean and logsumexp over a singleton dimension return the element itself
+    col = out[:, None]
+    assert np.array_equal(col.max(axis=1), out) and np.array_equal(col.mean(axis=1), out)
+    assert np.allclose(scipy.special.logsumexp(col, axis=1), out, rtol=1e-15, atol=1e-15)
+    # integer case is exact; a transposed weight would fail it
+    Xi = f32(RNG.integers(-3, 4, (4, 5)))
+    wi = f32([1, -2, 3, 0, 5])
+    assert np.array_equal(kopref.matvec_bias(Xi, wi, 2.0), Xi.astype(np.float64) @ wi.astype(np.float64) + 2.0)
+
+
 def test_threads_do_not_change_results():
     x = f32(RNG.standard_normal((64, 100)))
     b = f32(RNG.standard_normal(100))
