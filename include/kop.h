@@ -211,6 +211,27 @@ kop_status_t kop_residual_add(const void* a, const void* b, void* out,
                               int64_t out_row_stride, kop_dtype_t dtype, kop_stream_t stream);
 
 /*
+ * Row scaling, the O(N^2) form of diag(a) * B that the paper's L1-012 case study (Appendix "Generated
+ * Kernel Examples", diagonal matrix multiply) replaces a cuBLAS GEMM with:
+ *   out[i,j] = a[i] * b[i,j]
+ * a: [rows] of `dtype`; b, out: [rows, cols] of `dtype`. out may alias b exactly; a must not overlap out.
+ */
+kop_status_t kop_row_scale(const void* a, const void* b, void* out, int64_t rows, int64_t cols,
+                           int64_t b_row_stride, int64_t out_row_stride, kop_dtype_t dtype,
+                           kop_stream_t stream);
+
+/*
+ * Mat-vec with a bias sum, the form the paper's L2-018 case study reduces Linear -> Sum -> Max -> Mean ->
+ * LogSumExp -> LogSumExp to (sum_j (x W^T + b)_j = x . colsum(W) + sum(b); the later reductions act on a
+ * single element per row and are identities):
+ *   out[i] = sum_k x[i,k] * w[k] + b_sum
+ * x: [rows, k] of `dtype`; w: fp32 [k] (the caller's precomputed column sums); out: fp32 [rows]. x is read
+ * once; products and sums are fp32.
+ */
+kop_status_t kop_matvec_bias(const void* x, const float* w, float b_sum, float* out, int64_t rows,
+                             int64_t k, int64_t x_row_stride, kop_dtype_t dtype, kop_stream_t stream);
+
+/*
  * Transformer MLP segment with the vendor GEMMs preserved between the fused kernels
  * (problem formulation: extern library calls stay fixed; codegen agent: "do not
  * replace cuBLAS"): five operations enqueued on `stream`,

@@ -64,6 +64,10 @@ def lib() -> C.CDLL:
     L.kop_rmsnorm.argtypes = [vp, vp, vp, i64, i64, i64, i64, f32, i32, vp]
     L.kop_silu_mul.argtypes = [vp, vp, i64, i64, i64, i64, i32, vp]
     L.kop_residual_add.argtypes = [vp, vp, vp, i64, i64, i64, i64, i64, i32, vp]
+    L.kop_row_scale.argtypes = [vp, vp, vp, i64, i64, i64, i64, i32, vp]
+    L.kop_row_scale.restype = i32
+    L.kop_matvec_bias.argtypes = [vp, vp, f32, vp, i64, i64, i64, i32, vp]
+    L.kop_matvec_bias.restype = i32
     L.kop_rmsnorm_swiglu_residual.argtypes = [vp] * 6 + [i64] * 3 + [f32, vp, sz, i32, vp]
     L.kop_rmsnorm_swiglu_residual_workspace_bytes.restype = sz
     L.kop_rmsnorm_swiglu_residual_workspace_bytes.argtypes = [i64, i64, i64, i32]
@@ -234,6 +238,25 @@ def kop_residual_add(a, b, out=None, stream=None):
     _, _, os_ = _rows2d(out, "out")
     _check(lib().kop_residual_add(a.data_ptr(), b.data_ptr(), out.data_ptr(), rows, cols, as_, bs, os_,
                                   _dtype_tag(a), _stream(stream)), "kop_residual_add")
+    return out
+
+
+def kop_row_scale(a, b, out=None, stream=None):
+    rows, cols, bs = _rows2d(b, "b")
+    if a.dtype != b.dtype or not a.is_cuda or not a.is_contiguous() or a.numel() != rows:
+        raise ValueError("a: expected a contiguous CUDA vector of `rows` elements with b's dtype")
+    out = torch.empty_like(b) if out is None else out
+    _, _, os_ = _rows2d(out, "out")
+    _check(lib().kop_row_scale(a.data_ptr(), b.data_ptr(), out.data_ptr(), rows, cols, bs, os_,
+                               _dtype_tag(b), _stream(stream)), "kop_row_scale")
+    return out
+
+
+def kop_matvec_bias(x, w, b_sum, out=None, stream=None):
+    rows, k, xs = _rows2d(x, "x")
+    out = torch.empty(rows, dtype=torch.float32, device=x.device) if out is None else out
+    _check(lib().kop_matvec_bias(x.data_ptr(), _param(w, "w", k), float(b_sum), out.data_ptr(), rows, k, xs,
+                                 _dtype_tag(x), _stream(stream)), "kop_matvec_bias")
     return out
 
 

@@ -19,6 +19,9 @@ CONFIGS = {
     "bn_pool": dict(N=64, C=256, H=56, W=56, dtype=torch.float32),
     "ce_loss": dict(rows=32768, vocab=32000, dtype=torch.bfloat16),
     "mlp": dict(rows=16384, hidden=4096, inter=14336, dtype=torch.bfloat16, eps=1e-6),
+    # beyond the five benchmark configs: the two kernels the paper's case studies print
+    "row_scale": dict(rows=4096, cols=4096, dtype=torch.float32),          # the paper's 4096 x 4096 shape
+    "matvec_bias": dict(rows=32768, k=4096, dtype=torch.bfloat16),         # shape not given in the paper
 }
 
 
@@ -94,3 +97,21 @@ def pair_inputs(rows, cols, dtype=torch.bfloat16, seed=0, device="cpu"):
     a = _normal((rows, cols), 0.0, 1.0, g, device).to(dtype)
     b = _normal((rows, cols), 0.0, 1.0, g, device).to(dtype)
     return a, b
+
+
+def row_scale_inputs(rows, cols, dtype=torch.float32, seed=0, device="cpu"):
+    """a ~ N(0,1) [rows]; b ~ N(0,1) [rows, cols], both of the data dtype."""
+    g = _gen(seed, device)
+    a = _normal((rows,), 0.0, 1.0, g, device).to(dtype)
+    b = _normal((rows, cols), 0.0, 1.0, g, device).to(dtype)
+    return a, b
+
+
+def matvec_inputs(rows, k, dtype=torch.bfloat16, seed=0, device="cpu"):
+    """x ~ N(0,1) [rows, k]; w fp32 ~ N(0,0.16) [k] and b_sum ~ N(0,0.8) (a Python float): the spread
+    that column sums over 64 outputs of a N(0,0.02) weight and a N(0,0.1) bias would have."""
+    g = _gen(seed, device)
+    x = _normal((rows, k), 0.0, 1.0, g, device).to(dtype)
+    w = _normal((k,), 0.0, 0.16, g, device)
+    b_sum = _normal((1,), 0.0, 0.8, g, device)
+    return x, w, float(b_sum.item())

@@ -142,6 +142,22 @@ def test_mlp_pieces_validation(L):
     assert L.kop_residual_add(P, Q, R, 4, -3, 64, 64, 64, 0, None) == SHAPE
 
 
+def test_row_ops_validation(L):
+    assert L.kop_row_scale(P, Q, R, 0, 64, 64, 64, 0, None) == OK
+    assert L.kop_row_scale(None, Q, R, 4, 64, 64, 64, 0, None) == NULLP
+    assert L.kop_row_scale(P, Q, R, 4, 64, 63, 64, 0, None) == STRIDE
+    assert L.kop_row_scale(P, Q, Q + 8, 4, 64, 64, 64, 0, None) == ALIAS       # out overlaps b
+    assert L.kop_row_scale(R + 16, Q, R, 4, 64, 64, 64, 0, None) == ALIAS      # a overlaps out
+    assert L.kop_row_scale(P, Q, R, 4, 64, 64, 64, 2, None) == DTYPE
+    assert L.kop_row_scale(P + 1, Q, R, 4, 64, 64, 64, 1, None) == MISAL
+    assert L.kop_matvec_bias(P, Q, 0.5, R, 0, 64, 64, 1, None) == OK
+    assert L.kop_matvec_bias(P, None, 0.5, R, 4, 64, 64, 1, None) == NULLP
+    assert L.kop_matvec_bias(P, Q, 0.5, R, 4, 0, 64, 1, None) == SHAPE
+    assert L.kop_matvec_bias(P, Q, 0.5, R, 4, 64, 32, 1, None) == STRIDE
+    assert L.kop_matvec_bias(P, Q, 0.5, P + 64, 4, 64, 64, 1, None) == ALIAS
+    assert L.kop_matvec_bias(P, Q + 2, 0.5, R, 4, 64, 64, 1, None) == MISAL
+
+
 def test_mlp_driver_validation(L):
     f = L.kop_rmsnorm_swiglu_residual
     wsb = L.kop_rmsnorm_swiglu_residual_workspace_bytes(16, 64, 128, 1)

@@ -437,3 +437,65 @@ def test_mlp_pieces_options(kop):
                      (kop.kop_silu_mul, (torch.empty((0, 64), dtype=BF16, device="cuda"),)),
                      (kop.kop_residual_add, (torch.empty((0, 64), dtype=BF16, device="cuda"),) * 2)):
         assert fn(*args).shape[0] == 0
+
+
+# ------------------------------------------------------------------------------------------ row scale, mat-vec
+
+ROW_SCALE_SHAPES = [(4096, 4096, F32), (1000, 4096, BF16), (33, 1001, F32), (257, 520, BF16), (1, 1, F32)]
+
+
+@pytest.mark.parametrize("rows,cols,dtype", ROW_SCALE_SHAPES)
+@pytest.mark.parametrize("seed", SEEDS)
+def test_row_scale_parity(kop, rows, cols, dtype, seed):
+    a, b = synth.row_scale_inputs(rows, cols, dtype, seed, "cuda")
+    out = Guarded((rows, cols), dtype)
+    kop.kop_row_scale(a, b, out=out.t)
+    ref = kopref.row_scale(host(a), host(b), threads=None)
+    if dtype == F32:
+        assert np.array_equal(to_f64(out.t), ref.astype(np.float32).astype(np.float64))    # one fp32 product
+    else:
+        assert_close(out.t, ref, 2e-2, "row_scale")
+        assert_bf16_tight(out.t, ref, "row_scale", floor=1e-6)
+    out.check("row_scale")
+
+
+MATVEC_SHAPES = [(4096, 4096, BF16), (1000, 4096, F32), (37, 1000, BF16), (129, 257, F32), (9, 8, BF16), (3, 1, F32)]
+
+
+@pytest.mark.parametrize("rows,k,dtype", MATVEC_SHAPES)
+@pytest.mark.parametrize("seed", SEEDS)
+def test_matvec_bias_parity(kop, rows, k, dtype, seed):
+    x, w, b_sum = synth.matvec_inputs(rows, k, dtype, seed, "cuda")
+    out = Guarded((rows,), F32)
+    kop.kop_matvec_bias(x, w, b_sum, out=out.t)
+    ref = kopref.matvec_bias(host(x), host(w), np.float32(b_sum), threads=None)
+    assert_close(out.t, ref, tol_of(dtype), "matvec_bias")
+    assert_close(out.t, ref, 2e-5, "matvec_bias (fp32-grade: fp32 products and sums)")
+    out.check("matvec_bias")
+
+
+def test_row_ops_options_and_full_configs(kop):
+    c = synth.CONFIGS["matvec_bias"]
+    x, w, b_sum = synth.matvec_inputs(c["rows"], c["k"], c["dtype"], 0, "cuda")
+    out = kop.kop_matvec_bias(x, w, b_sum)
+    ref = kopref.matvec_bias(host(x), host(w), np.float32(b_sum), threads=None)
+    assert_close(out, ref, 2e-5, "matvec full config")
+    assert torch.equal(out, kop.kop_matvec_bias(x, w, b_sum))
+    # strided rows
+    wide = torch.zeros((100, 8192), dtype=BF16, device="cuda")
+    wide[:, 4096:] = x[:100]
+    assert_close(kop.kop_matvec_bias(wide[:, 4096:], w, b_sum), ref[:100], 2e-5, "matvec strided")
+    wide2 = torch.zeros((100, 4097), dtype=BF16, device="cuda")
+    wide2[:, 1:] = x[:100]
+    assert_close(kop.kop_matvec_bias(wide2[:, 1:], w, b_sum), ref[:100], 2e-5, "matvec misaligned")
+    # row scale in place and strided
+    a, b = synth.row_scale_inputs(300, 4096, F32, 1, "cuda")
+    rs = kopref.row_scale(host(a), host(b))
+    bi = b.clone()
+    kop.kop_row_scale(a, bi, out=bi)
+    assert np.array_equal(to_f64(bi), rs.astype(np.float32).astype(np.float64))
+    wb = torch.zeros((300, 8192), dtype=F32, device="cuda")
+    wb[:, 1024:5120] = b
+    assert np.array_equal(to_f64(kop.kop_row_scale(a, wb[:, 1024:5120])), rs.astype(np.float32).astype(np.float64))
+    assert kop.kop_row_scale(a[:0], b[:0]).shape == (0, 4096)
+    assert kop.kop_matvec_bias(x[:0], w, b_sum).shape == (0,)
