@@ -380,3 +380,104 @@ int kopref_matvec_bias(const void* X, const float* w, double b_sum, double* out,
     }
     return 0;
 }
+
+/* ---- residual add + LayerNorm, and plain LayerNorm ----------------------------------------------------
+ * v_j = x_j + r_j (r may be NULL: v = x) ; then LayerNorm exactly as above: biased variance, eps inside
+ * the square root, y = (v - mu) rstd gamma + beta.  This is the fusion agent's "residual + norm" pattern
+ * without the bias / activation prologue. */
+int kopref_residual_layernorm(const void* x, const void* residual, const float* gamma, const float* beta,
+        double* y, double* mean, double* rstd, int64_t rows, int64_t hidden, int64_t x_row_stride,
+        int64_t res_row_stride, int64_t y_row_stride, double eps, int dtype, int threads)
+{
+    if (!x || !gamma || !beta || !y || rows < 0 || hidden <= 0 || bad_dtype(dtype)) return -1;
+    int nt = pick_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t i = 0; i < rows; ++i) {
+        double* yr = y + i * y_row_stride;
+        double sum = 0.0;
+        for (int64_t j = 0; j < hidden; ++j) {
+            double v = load_elem(x, i * x_row_stride + j, dtype);
+            if (residual) v += load_elem(residual, i * res_row_stride + j, dtype);
+            yr[j] = v;
+            sum += v;
+        }
+        double mu = sum / (double)hidden;
+        double ss = 0.0;
+        for (int64_t j = 0; j < hidden; ++j) {
+            double d = yr[j] - mu;
+            ss += d * d;
+        }
+        double rs = 1.0 / sqrt(ss / (double)hidden + eps);
+        for (int64_t j = 0; j < hidden; ++j)
+            yr[j] = (yr[j] - mu) * rs * (double)gamma[j] + (double)beta[j];
+        if (mean) mean[i] = mu;
+        if (rstd) rstd[i] = rs;
+    }
+    return 0;
+}
+
+/* ---- SiLU(gate) * up with interleaved columns ---------------------------------------------------------------
+ * Row layout [g0, u0, g1, u1, ...]; out_j = g_j / (1 + exp(-g_j)) * u_j. */
+int kopref_silu_mul_interleaved(const void* gate_up, double* out, int64_t rows, int64_t inter,
+        int64_t in_row_stride, int64_t out_row_stride, int dtype, int threads)
+{
+    if (!gate_up || !out || rows < 0 || inter <= 0 || bad_dtype(dtype)) return -1;
+    int nt = pick_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t i = 0; i < rows; ++i)
+        for (int64_t j = 0; j < inter; ++j) {
+            double g = load_elem(gate_up, i * in_row_stride + 2 * j, dtype);
+            double u = load_elem(gate_up, i * in_row_stride + 2 * j + 1, dtype);
+            out[i * out_row_stride + j] = g / (1.0 + exp(-g)) * u;
+        }
+    return 0;
+}
+
+/* ---- cross-entropy with ignore_index and label smoothing --------------------------------------------------
+ * lse_i = logsumexp_j z_ij.  With smoothing s in [0,1):
+ *   loss_i = (1 - s) (lse_i - z[i, label_i]) + s (lse_i - (1/V) sum_j z_ij)
+ * Rows whose label equals ignore_index give loss 0 and do not count; mean = sum of counted losses /
+ * number of counted rows (NaN when none is counted).  A label outside [0, V) that is not ignore_index
+ * gives NaN and is counted in *bad_label_count. */
+int kopref_ce_loss_opts(const void* logits, const int32_t* labels, double* loss, double* mean_loss,
+        int64_t* bad_label_count, int64_t* counted_rows, int64_t rows, int64_t vocab, int64_t row_stride,
+        int32_t ignore_index, double smoothing, int dtype, int threads)
+{
+    if (!logits || !labels || !loss || rows < 0 || vocab <= 0 || bad_dtype(dtype)) return -1;
+    if (!(smoothing >= 0.0 && smoothing < 1.0)) return -1;
+    int nt = pick_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t i = 0; i < rows; ++i) {
+        int32_t lab = labels[i];
+        if (lab == ignore_index) { loss[i] = 0.0; continue; }
+        double m = -INFINITY, zsum = 0.0;
+        for (int64_t j = 0; j < vocab; ++j) {
+            double z = load_elem(logits, i * row_stride + j, dtype);
+            if (z > m) m = z;
+            zsum += z;
+        }
+        double S = 0.0;
+        for (int64_t j = 0; j < vocab; ++j) S += exp(load_elem(logits, i * row_stride + j, dtype) - m);
+        double lse = m + log(S);
+        if (lab < 0 || (int64_t)lab >= vocab) { loss[i] = NAN; continue; }
+        double nll = lse - load_elem(logits, i * row_stride + lab, dtype);
+        double smooth = lse - zsum / (double)vocab;
+        loss[i] = (1.0 - smoothing) * nll + smoothing * smooth;
+    }
+    int64_t bad = 0, counted = 0;
+    double total = 0.0;
+    for (int64_t i = 0; i < rows; ++i) {
+        int32_t lab = labels[i];
+        if (lab == ignore_index) continue;
+        if (lab < 0 || (int64_t)lab >= vocab) ++bad;
+        ++counted;
+        total += loss[i];
+    }
+    if (mean_loss) *mean_loss = counted > 0 ? total / (double)counted : NAN;
+    if (bad_label_count) *bad_label_count = bad;
+    if (counted_rows) *counted_rows = counted;
+    return 0;
+}

@@ -40,6 +40,9 @@ def lib() -> C.CDLL:
         _lib.kopref_silu_mul.argtypes = [vp] * 2 + [i64] * 4 + [C.c_int, C.c_int]
         _lib.kopref_residual_add.argtypes = [vp] * 3 + [i64] * 5 + [C.c_int, C.c_int]
         _lib.kopref_gemm_nt.argtypes = [vp, C.c_int, vp, C.c_int, vp, i64, i64, i64, C.c_int]
+        _lib.kopref_residual_layernorm.argtypes = [vp] * 7 + [i64] * 5 + [dbl, C.c_int, C.c_int]
+        _lib.kopref_silu_mul_interleaved.argtypes = [vp] * 2 + [i64] * 4 + [C.c_int, C.c_int]
+        _lib.kopref_ce_loss_opts.argtypes = [vp] * 6 + [i64] * 3 + [C.c_int32, dbl, C.c_int, C.c_int]
         _lib.kopref_row_scale.argtypes = [vp, vp, vp, i64, i64, i64, i64, C.c_int, C.c_int]
         _lib.kopref_matvec_bias.argtypes = [vp, vp, dbl, vp, i64, i64, i64, C.c_int, C.c_int]
     return _lib
@@ -209,6 +212,51 @@ def gemm_nt(a, w, threads=1) -> np.ndarray:
     out = np.empty((M, N), dtype=np.float64)
     _check(lib().kopref_gemm_nt(_p(aa), adt, _p(wa), wdt, _p(out), M, N, K, _nt(threads)), "gemm_nt")
     return out
+
+
+def residual_layernorm(x, residual, gamma, beta, eps, threads=1):
+    """LayerNorm(x + residual) (residual may be None). Returns (y, mean, rstd)."""
+    xa, dt = as_data(x)
+    ra = None
+    if residual is not None:
+        ra, dt2 = as_data(residual)
+        assert dt == dt2 and ra.shape == xa.shape
+    rows, hidden = xa.shape
+    g, be = as_param(gamma), as_param(beta)
+    y = np.empty((rows, hidden), dtype=np.float64)
+    mean = np.empty(rows, dtype=np.float64)
+    rstd = np.empty(rows, dtype=np.float64)
+    _check(lib().kopref_residual_layernorm(_p(xa), _p(ra), _p(g), _p(be), _p(y), _p(mean), _p(rstd), rows, hidden,
+                                           hidden, hidden, hidden, float(eps), dt, _nt(threads)), "residual_layernorm")
+    return y, mean, rstd
+
+
+def silu_mul_interleaved(gate_up, threads=1) -> np.ndarray:
+    ga, dt = as_data(gate_up)
+    rows, two_i = ga.shape
+    assert two_i % 2 == 0
+    inter = two_i // 2
+    out = np.empty((rows, inter), dtype=np.float64)
+    _check(lib().kopref_silu_mul_interleaved(_p(ga), _p(out), rows, inter, two_i, inter, dt, _nt(threads)),
+           "silu_mul_interleaved")
+    return out
+
+
+def ce_loss_opts(logits, labels, ignore_index=-100, smoothing=0.0, threads=1):
+    """Returns (loss[rows], mean over counted rows, bad_label_count, counted_rows)."""
+    za, dt = as_data(logits)
+    rows, vocab = za.shape
+    if hasattr(labels, "detach"):
+        labels = labels.detach().cpu().numpy()
+    lab = np.ascontiguousarray(labels, dtype=np.int32)
+    loss = np.empty(rows, dtype=np.float64)
+    mean = C.c_double(0.0)
+    bad = C.c_int64(0)
+    cnt = C.c_int64(0)
+    _check(lib().kopref_ce_loss_opts(_p(za), _p(lab), _p(loss), C.addressof(mean), C.addressof(bad),
+                                     C.addressof(cnt), rows, vocab, vocab, int(ignore_index), float(smoothing),
+                                     dt, _nt(threads)), "ce_loss_opts")
+    return loss, mean.value, bad.value, cnt.value
 
 
 def row_scale(a, b, threads=1) -> np.ndarray:

@@ -480,6 +480,70 @@ def test_mlp_chain_reduced_shape_vs_numpy():
     assert np.allclose(out, ref, rtol=1e-12, atol=1e-14)
 
 
+# --------------------------------------------------------------------------- residual+LN, interleaved SwiGLU, CE options
+
+def test_residual_layernorm_library_and_invariants():
+    H = 72
+    x = f32(RNG.standard_normal((8, H)) * 2 + 1)
+    r = f32(RNG.standard_normal((8, H)))
+    g = f32(1 + 0.1 * RNG.standard_normal(H))
+    be = f32(0.1 * RNG.standard_normal(H))
+    tx, tr, tg, tbe = (torch.from_numpy(a.astype(np.float64)) for a in (x, r, g, be))
+    y, mu, rstd = kopref.residual_layernorm(x, r, g, be, 1e-5)
+    assert np.max(np.abs(y - F.layer_norm(tx + tr, (H,), tg, tbe, 1e-5).numpy())) <= 1e-13
+    assert np.allclose(mu, (tx + tr).mean(dim=1).numpy(), rtol=0, atol=1e-14)
+    # no residual: plain LayerNorm; zero mean and sigma^2/(sigma^2+eps) variance before the affine step
+    y0, mu0, rstd0 = kopref.residual_layernorm(x, None, f32(np.ones(H)), f32(np.zeros(H)), 1e-5)
+    assert np.max(np.abs(y0 - F.layer_norm(tx, (H,), None, None, 1e-5).numpy())) <= 1e-13
+    assert np.all(np.abs(y0.mean(axis=1)) <= 1e-12)
+    var = x.astype(np.float64).var(axis=1)
+    assert np.allclose(y0.var(axis=1), var / (var + 1e-5), rtol=1e-12, atol=0)
+    # consistent with the full bias+GELU+residual oracle when the GELU term is switched off by x = 0, b = 0
+    yf, _, _ = kopref.bias_gelu_residual_layernorm(f32(np.zeros((8, H))), r, f32(np.zeros(H)), g, be, 1e-5)
+    yr, _, _ = kopref.residual_layernorm(r, None, g, be, 1e-5)
+    assert np.array_equal(yf, yr)
+
+
+def test_silu_mul_interleaved_is_a_column_permutation_of_the_split_layout():
+    inter = 7
+    g = f32(RNG.standard_normal((4, inter)) * 3)
+    u = f32(RNG.standard_normal((4, inter)))
+    inter_l = np.empty((4, 2 * inter), dtype=np.float32)
+    inter_l[:, 0::2] = g
+    inter_l[:, 1::2] = u
+    assert np.array_equal(kopref.silu_mul_interleaved(inter_l), kopref.silu_mul(np.concatenate([g, u], axis=1)))
+    ref = (F.silu(torch.from_numpy(g.astype(np.float64))) * torch.from_numpy(u.astype(np.float64))).numpy()
+    assert np.max(np.abs(kopref.silu_mul_interleaved(inter_l) - ref)) <= 1e-15
+
+
+def test_ce_options_against_library_and_base_oracle():
+    M, V = 13, 101
+    z = f32(RNG.standard_normal((M, V)) * 2)
+    lab = RNG.integers(0, V, M).astype(np.int32)
+    lab[[2, 7]] = -100
+    tz, tl = torch.from_numpy(z.astype(np.float64)), torch.from_numpy(lab.astype(np.int64))
+    for s in (0.0, 0.1, 0.35):
+        loss, mean, bad, cnt = kopref.ce_loss_opts(z, lab, ignore_index=-100, smoothing=s)
+        ref = F.cross_entropy(tz, tl, reduction="none", ignore_index=-100, label_smoothing=s).numpy()
+        assert np.max(np.abs(loss - ref)) <= 1e-13
+        assert mean == pytest.approx(float(F.cross_entropy(tz, tl, ignore_index=-100, label_smoothing=s)), rel=1e-13)
+        assert bad == 0 and cnt == M - 2 and loss[2] == 0.0 and loss[7] == 0.0
+    # no ignored rows and no smoothing: identical to the plain oracle
+    lab2 = RNG.integers(0, V, M).astype(np.int32)
+    a, ma, _, c = kopref.ce_loss_opts(z, lab2, ignore_index=-100, smoothing=0.0)
+    b, mb, _ = kopref.ce_loss_rowwise(z, lab2)
+    assert np.array_equal(a, b) and ma == mb and c == M
+    # smoothing on a uniform row changes nothing (both terms equal ln V); all rows ignored -> NaN mean
+    zu = f32(np.full((2, V), 0.5))
+    lu, mu_, _, _ = kopref.ce_loss_opts(zu, np.array([3, 4], dtype=np.int32), smoothing=0.3)
+    assert np.all(np.abs(lu - math.log(V)) <= 1e-13)
+    _, mn, _, cn = kopref.ce_loss_opts(zu, np.array([-100, -100], dtype=np.int32))
+    assert cn == 0 and math.isnan(mn)
+    # an out-of-range label that is not ignore_index is bad, not ignored
+    l3, m3, b3, c3 = kopref.ce_loss_opts(zu, np.array([V, 1], dtype=np.int32))
+    assert b3 == 1 and c3 == 2 and math.isnan(l3[0]) and math.isnan(m3)
+
+
 # --------------------------------------------------------------------------- row scale, mat-vec + bias sum
 
 def test_row_scale_is_diag_times_matrix():
