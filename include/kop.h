@@ -154,7 +154,7 @@ size_t kop_ce_loss_rowwise_workspace_bytes(int64_t rows, int64_t vocab, kop_dtyp
  * cudaMalloc would synchronise the device and take memory the pool does not know about), a server
  * whose memory plan is frozen after start-up, a C caller on a latency-critical path. Instead of a
  * caller-supplied workspace, the scratch of the mean reduction (tickets and per-group partials) is
- * a fixed device array inside the library: 49,168 bytes that every GPU which loads the library
+ * a fixed device array inside the library: 65,552 bytes that every GPU which loads the library
  * holds until the process exits.
  *
  * Arguments, outputs, results and error behaviour are those of kop_ce_loss_rowwise without the
@@ -179,6 +179,33 @@ kop_status_t kop_ce_loss_rowwise_static(const void* logits, const int32_t* label
 int64_t kop_ce_loss_rowwise_static_max_rows(void);
 
 /*
+ * kop_ce_loss_rowwise with ignore_index and label smoothing (coverage variant of the same segment):
+ *   loss[i] = (1 - s) (lse_i - z[i, label_i]) + s (lse_i - (1/vocab) sum_j z[i,j]),  s = label_smoothing in [0, 1)
+ * Rows whose label equals ignore_index get loss 0, are not read, and do not count;
+ * *mean_loss = sum of counted losses / *counted_rows (NaN when no row counts); a label outside [0, vocab)
+ * that is not ignore_index is a bad label as above. counted_rows: int32 [1] or NULL. Workspace as for
+ * kop_ce_loss_rowwise (same size function).
+ */
+kop_status_t kop_ce_loss_rowwise_opts(const void* logits, const int32_t* labels,
+                                      float* loss, float* mean_loss, int32_t* bad_label_count,
+                                      int32_t* counted_rows, int64_t rows, int64_t vocab, int64_t row_stride,
+                                      int32_t ignore_index, float label_smoothing,
+                                      void* workspace, size_t workspace_bytes,
+                                      kop_dtype_t dtype, kop_stream_t stream);
+
+/*
+ * Residual add + LayerNorm, the fusion agent's "residual + norm" pattern without a bias / activation
+ * prologue ("x = residual + x; x = LayerNorm(x): one kernel, one memory pass"), or plain LayerNorm:
+ *   v = x + residual (residual may be NULL: v = x);  y = (v - mean v) / sqrt(var v + eps) * gamma + beta
+ * Same statistics outputs, strides and aliasing rules as kop_bias_gelu_residual_layernorm.
+ */
+kop_status_t kop_residual_layernorm(const void* x, const void* residual,
+                                    const float* gamma, const float* beta, void* y,
+                                    float* mean, float* rstd, int64_t rows, int64_t hidden,
+                                    int64_t x_row_stride, int64_t res_row_stride, int64_t y_row_stride,
+                                    float eps, kop_dtype_t dtype, kop_stream_t stream);
+
+/*
  * RMSNorm (fusion agent: "normalization fusion (LayerNorm/RMSNorm sequences)"):
  *   y[i,j] = x[i,j] / sqrt(mean_j x[i,j]^2 + eps) * weight[j]
  * x, y: [rows, hidden] of `dtype`; weight: fp32 [hidden]. y may alias x exactly.
@@ -199,6 +226,14 @@ kop_status_t kop_rmsnorm(const void* x, const float* weight, void* y,
 kop_status_t kop_silu_mul(const void* gate_up, void* out, int64_t rows, int64_t inter,
                           int64_t in_row_stride, int64_t out_row_stride,
                           kop_dtype_t dtype, kop_stream_t stream);
+
+/*
+ * kop_silu_mul for the interleaved layout [g0, u0, g1, u1, ...] (gate_up: [rows, 2*inter]):
+ *   out[i,j] = silu(gate_up[i, 2j]) * gate_up[i, 2j+1]
+ */
+kop_status_t kop_silu_mul_interleaved(const void* gate_up, void* out, int64_t rows, int64_t inter,
+                                      int64_t in_row_stride, int64_t out_row_stride,
+                                      kop_dtype_t dtype, kop_stream_t stream);
 
 /*
  * Residual add (fusion agent: "pointwise + pointwise: load once, store once"):

@@ -14,13 +14,21 @@ namespace kop {
 namespace {
 
 // Workspace layout (all 4-byte words): [0] global ticket, [1..3] pad, then per group of
-// kGroupRows rows: a ticket, a partial loss sum, a bad-label count.
+// kGroupRows rows: a ticket, a partial loss sum, a bad-label count, a counted-row count (the last
+// only used by the variant with ignore_index).
 constexpr int kGroupRows = 256;
 struct CeWorkspace {
     unsigned int* global_ticket;
     unsigned int* group_ticket;
     float* group_sum;
     int* group_bad;
+    int* group_cnt;
+};
+// Options of kop_ce_loss_rowwise_opts (unused by the plain entry point).
+struct CeOpts {
+    int32_t ignore_index;
+    float smoothing;
+    int32_t* counted_rows;
 };
 __host__ __device__ inline int64_t ce_groups(int64_t rows) { return (rows + kGroupRows - 1) / kGroupRows; }
 __host__ __device__ inline CeWorkspace ce_workspace(void* base, int64_t rows)
@@ -32,9 +40,10 @@ __host__ __device__ inline CeWorkspace ce_workspace(void* base, int64_t rows)
     ws.group_ticket = w + 4;
     ws.group_sum = reinterpret_cast<float*>(w + 4 + g);
     ws.group_bad = reinterpret_cast<int*>(w + 4 + 2 * g);
+    ws.group_cnt = reinterpret_cast<int*>(w + 4 + 3 * g);
     return ws;
 }
-inline size_t ce_workspace_bytes(int64_t rows) { return (size_t)(4 + 3 * ce_groups(rows)) * 4; }
+inline size_t ce_workspace_bytes(int64_t rows) { return (size_t)(4 + 4 * ce_groups(rows)) * 4; }
 inline size_t ce_workspace_clear_bytes(int64_t rows) { return (size_t)(4 + ce_groups(rows)) * 4; }
 
 template <typename T>
@@ -69,15 +78,18 @@ __device__ __forceinline__ int warp_sum_int(int v)
 // again in a fixed order. Which CTA does the summing varies, the order of the additions does not,
 // so the mean is bit-identical run to run. (A whole-CTA wait on a single ticket held every CTA's
 // registers for an extra L2 round trip and cost 12 % on the benchmark shape.)
-template <typename T>
-__device__ __forceinline__ void ce_finish(float M, float S, const T* zr, const int32_t* labels,
+template <typename T, bool kOpts, bool kSmooth>
+__device__ __forceinline__ void ce_finish(float M, float S, float Z, const T* zr, const int32_t* labels,
                                           float* loss, float* mean_loss, int32_t* bad_label_count,
-                                          CeWorkspace ws, int64_t row, int64_t rows, int64_t vocab)
+                                          CeWorkspace ws, int64_t row, int64_t rows, int64_t vocab,
+                                          CeOpts opts)
 {
-    __shared__ float red_a[32], red_b[32];
+    __shared__ float red_a[32], red_b[32], red_c[32];
     const float Mb = block_max(M, red_a);
     // A thread that saw nothing has M = -inf and S = 0; keep its term at 0 rather than 0 * 2^nan.
     const float Sb = block_sum(M == -INFINITY ? 0.0f : S * ex2_approx(M - Mb), red_b);
+    float Zb = 0.0f;
+    if (kSmooth) Zb = block_sum(Z, red_c);          // sum of the row's logits, for label smoothing
     if (threadIdx.x >= 32) return;
     const int lane = threadIdx.x;
     const int64_t g = row / kGroupRows;
@@ -88,8 +100,12 @@ __device__ __forceinline__ void ce_finish(float M, float S, const T* zr, const i
         const float lse = (Mb + log2f(Sb)) * kLn2;
         const int32_t lab = labels[row];
         float l;
-        if (lab < 0 || (int64_t)lab >= vocab) l = __int_as_float(0x7FC00000);
-        else l = lse - Elem<T>::load1(zr + lab);
+        if (kOpts && lab == opts.ignore_index) l = 0.0f;
+        else if (lab < 0 || (int64_t)lab >= vocab) l = __int_as_float(0x7FC00000);
+        else {
+            l = lse - Elem<T>::load1(zr + lab);
+            if (kSmooth) l = (1.0f - opts.smoothing) * l + opts.smoothing * (lse - Zb / (float)vocab);
+        }
         loss[row] = l;
         __threadfence();
         t = atomicAdd(ws.group_ticket + g, 1u);
@@ -98,19 +114,23 @@ __device__ __forceinline__ void ce_finish(float M, float S, const T* zr, const i
     if (t != (unsigned)(gsize - 1)) return;
     __threadfence();
     float acc = 0.0f;
-    int bad = 0;
+    int bad = 0, cnt = 0;
     for (int i = lane; i < gsize; i += 32) {
         acc += __ldcg(loss + g0 + i);
         const int32_t lab = __ldg(labels + g0 + i);
-        bad += (lab < 0 || (int64_t)lab >= vocab) ? 1 : 0;
+        const bool ignored = kOpts && lab == opts.ignore_index;
+        bad += (!ignored && (lab < 0 || (int64_t)lab >= vocab)) ? 1 : 0;
+        cnt += ignored ? 0 : 1;
     }
     acc = warp_sum(acc);
     bad = warp_sum_int(bad);
+    if (kOpts) cnt = warp_sum_int(cnt);
     const int64_t ngroups = ce_groups(rows);
     unsigned t2 = 0;
     if (lane == 0) {
         ws.group_sum[g] = acc;
         ws.group_bad[g] = bad;
+        if (kOpts) ws.group_cnt[g] = cnt;
         __threadfence();
         t2 = atomicAdd(ws.global_ticket, 1u);
     }
@@ -118,16 +138,24 @@ __device__ __forceinline__ void ce_finish(float M, float S, const T* zr, const i
     if (t2 != (unsigned)(ngroups - 1)) return;
     __threadfence();
     float tot = 0.0f;
-    int64_t nbad = 0;
+    int64_t nbad = 0, ncnt = 0;
     for (int64_t i = lane; i < ngroups; i += 32) {
         tot += __ldcg(ws.group_sum + i);
         nbad += __ldcg(ws.group_bad + i);
+        if (kOpts) ncnt += __ldcg(ws.group_cnt + i);
     }
     tot = warp_sum(tot);
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) nbad += __shfl_xor_sync(0xFFFFFFFFu, nbad, o);
+    for (int o = 16; o > 0; o >>= 1) {
+        nbad += __shfl_xor_sync(0xFFFFFFFFu, nbad, o);
+        if (kOpts) ncnt += __shfl_xor_sync(0xFFFFFFFFu, ncnt, o);
+    }
     if (lane == 0) {
-        if (mean_loss != nullptr) *mean_loss = tot / (float)rows;
+        if (kOpts) {
+            // mean over the rows that count; no counted row gives 0 / 0 = NaN, as the definition does
+            if (mean_loss != nullptr) *mean_loss = tot / (float)ncnt;
+            if (opts.counted_rows != nullptr) *opts.counted_rows = (int32_t)ncnt;
+        } else if (mean_loss != nullptr) *mean_loss = tot / (float)rows;
         if (bad_label_count != nullptr)
             *bad_label_count = (int32_t)(nbad > 0x7FFFFFFF ? 0x7FFFFFFF : nbad);
     }
@@ -135,8 +163,8 @@ __device__ __forceinline__ void ce_finish(float M, float S, const T* zr, const i
 
 // One batch of VPT vectors per thread: loads first (all in flight), then the batch maximum on the
 // packed values, then one ex2 per element against the updated running offset.
-template <typename T, int VPT, bool kTail>
-__device__ __forceinline__ void ce_batch(const T* zr, int base, int nvec, float& M, float& S)
+template <typename T, int VPT, bool kTail, bool kSum>
+__device__ __forceinline__ void ce_batch(const T* zr, int base, int nvec, float& M, float& S, float& Z)
 {
     constexpr int E = Elem<T>::kPerVec;
     Vec16 raw[VPT];
@@ -164,6 +192,11 @@ __device__ __forceinline__ void ce_batch(const T* zr, int base, int nvec, float&
             Elem<T>::unpack(raw[k], f);
 #pragma unroll
             for (int e = 0; e < E; ++e) s += ex2_approx(fmaf(f[e], kLog2e, neg));
+            if (kSum && (!kTail || base + k * (int)blockDim.x + (int)threadIdx.x < nvec)) {
+                // pairwise first: half the dependent adds on the running sum
+#pragma unroll
+                for (int e = 0; e < E; e += 2) Z += f[e] + f[e + 1];
+            }
         }
         S = s;
         M = newM;
@@ -172,36 +205,43 @@ __device__ __forceinline__ void ce_batch(const T* zr, int base, int nvec, float&
 
 // 256 threads, capped at 32 registers: eight CTAs (2048 threads) per SM. Occupancy is what hides the
 // load latency here; a build that drifted to 40 registers (six CTAs) was 6 % slower.
-template <typename T, int VPT>
-__global__ void __launch_bounds__(256, 8)
+// kOpts: ignore_index handling; kSmooth: additionally the row sum of the logits for label smoothing
+// (one more add per element and a few more registers, so that variant allows 40 registers).
+template <typename T, int VPT, bool kOpts, bool kSmooth>
+__global__ void __launch_bounds__(256, kSmooth ? 6 : 8)
 ce_row_kernel(const T* __restrict__ z, const int32_t* __restrict__ labels, float* __restrict__ loss,
               float* __restrict__ mean_loss, int32_t* __restrict__ bad_label_count,
-              CeWorkspace ws, int64_t rows, int nvec, int64_t row_stride, int64_t vocab)
+              CeWorkspace ws, int64_t rows, int nvec, int64_t row_stride, int64_t vocab, CeOpts opts)
 {
     const int64_t row = blockIdx.x;
     const T* zr = z + row * row_stride;
-    float M = -INFINITY, S = 0.0f;
+    float M = -INFINITY, S = 0.0f, Z = 0.0f;
+    // An ignored row is not read at all: it only takes its tickets.
+    if (kOpts && __ldg(labels + row) == opts.ignore_index) nvec = 0;
     // One loop body with bounds predicates on every batch (out-of-range vectors read as -inf). A
     // predicate-free main loop plus a separate tail batch doubled the inlined body, pushed the kernel
     // from 32 to 40 registers (six CTAs per SM instead of eight) and measured 3-6 % slower.
     const int step = VPT * blockDim.x;
-    for (int base = 0; base < nvec; base += step) ce_batch<T, VPT, true>(zr, base, nvec, M, S);
-    ce_finish<T>(M, S, zr, labels, loss, mean_loss, bad_label_count, ws, row, rows, vocab);
+    for (int base = 0; base < nvec; base += step) ce_batch<T, VPT, true, kSmooth>(zr, base, nvec, M, S, Z);
+    ce_finish<T, kOpts, kSmooth>(M, S, Z, zr, labels, loss, mean_loss, bad_label_count, ws, row, rows, vocab, opts);
 }
 
 // Any vocab / alignment: scalar loads, element-wise online recurrence.
-template <typename T>
+template <typename T, bool kOpts>
 __global__ void __launch_bounds__(256)
 ce_row_scalar_kernel(const T* __restrict__ z, const int32_t* __restrict__ labels,
                      float* __restrict__ loss, float* __restrict__ mean_loss,
                      int32_t* __restrict__ bad_label_count, CeWorkspace ws,
-                     int64_t rows, int64_t row_stride, int64_t vocab)
+                     int64_t rows, int64_t row_stride, int64_t vocab, CeOpts opts)
 {
     const int64_t row = blockIdx.x;
     const T* zr = z + row * row_stride;
-    float M = -INFINITY, S = 0.0f;
-    for (int64_t j = threadIdx.x; j < vocab; j += blockDim.x) {
-        const float x2 = Elem<T>::load1(zr + j) * kLog2e;
+    float M = -INFINITY, S = 0.0f, Z = 0.0f;
+    const int64_t n = (kOpts && __ldg(labels + row) == opts.ignore_index) ? 0 : vocab;
+    for (int64_t j = threadIdx.x; j < n; j += blockDim.x) {
+        const float xj = Elem<T>::load1(zr + j);
+        if (kOpts) Z += xj;
+        const float x2 = xj * kLog2e;
         if (x2 == -INFINITY) continue;
         if (x2 > M) {
             S = S * ex2_approx(M - x2) + 1.0f;
@@ -210,13 +250,13 @@ ce_row_scalar_kernel(const T* __restrict__ z, const int32_t* __restrict__ labels
             S += ex2_approx(x2 - M);
         }
     }
-    ce_finish<T>(M, S, zr, labels, loss, mean_loss, bad_label_count, ws, row, rows, vocab);
+    ce_finish<T, kOpts, kOpts>(M, S, Z, zr, labels, loss, mean_loss, bad_label_count, ws, row, rows, vocab, opts);
 }
 
-template <typename T>
+template <typename T, bool kOpts>
 kop_status_t launch_ce(const void* zv, const int32_t* labels, float* loss, float* mean_loss,
                        int32_t* bad, int64_t rows, int64_t vocab, int64_t stride, void* workspace,
-                       cudaStream_t stream)
+                       cudaStream_t stream, CeOpts opts)
 {
     const T* z = static_cast<const T*>(zv);
     constexpr int E = Elem<T>::kPerVec;
@@ -231,14 +271,20 @@ kop_status_t launch_ce(const void* zv, const int32_t* labels, float* loss, float
         // Batches of at most four vectors per thread: ~50 registers, so five 256-thread CTAs stay
         // resident per SM and their load and exp phases interleave. Larger batches (more bytes in
         // flight per thread, fewer resident warps) measured 5-30 % slower on a 32000-wide bf16 row.
-#define KOP_CE(V) ce_row_kernel<T, V><<<(unsigned)rows, threads, 0, stream>>>(z, labels, loss, mean_loss, bad, ws, rows, nvec, stride, vocab)
+#define KOP_CE_L(V, SM) ce_row_kernel<T, V, kOpts, SM><<<(unsigned)rows, threads, 0, stream>>>(z, labels, loss, mean_loss, bad, ws, rows, nvec, stride, vocab, opts)
+#define KOP_CE(V)                                                  \
+    do {                                                           \
+        if (kOpts && opts.smoothing > 0.0f) KOP_CE_L(V, true);     \
+        else KOP_CE_L(V, false);                                   \
+    } while (0)
         if (per <= 1) KOP_CE(1);
         else if (per <= 2) KOP_CE(2);
         else KOP_CE(4);
 #undef KOP_CE
+#undef KOP_CE_L
         return launch_status();
     }
-    ce_row_scalar_kernel<T><<<(unsigned)rows, 256, 0, stream>>>(z, labels, loss, mean_loss, bad, ws, rows, stride, vocab);
+    ce_row_scalar_kernel<T, kOpts><<<(unsigned)rows, 256, 0, stream>>>(z, labels, loss, mean_loss, bad, ws, rows, stride, vocab, opts);
     return launch_status();
 }
 
@@ -276,8 +322,40 @@ extern "C" kop_status_t kop_ce_loss_rowwise(const void* logits, const int32_t* l
     if ((st = check_device()) != KOP_OK) return st;
     cudaStream_t s = as_stream(stream);
     return dtype == KOP_F32
-               ? launch_ce<float>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s)
-               : launch_ce<__nv_bfloat16>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s);
+               ? launch_ce<float, false>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s, CeOpts{0, 0.0f, nullptr})
+               : launch_ce<__nv_bfloat16, false>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s, CeOpts{0, 0.0f, nullptr});
+}
+
+extern "C" kop_status_t kop_ce_loss_rowwise_opts(const void* logits, const int32_t* labels, float* loss,
+                                                 float* mean_loss, int32_t* bad_label_count,
+                                                 int32_t* counted_rows, int64_t rows, int64_t vocab,
+                                                 int64_t row_stride, int32_t ignore_index,
+                                                 float label_smoothing, void* workspace,
+                                                 size_t workspace_bytes, kop_dtype_t dtype,
+                                                 kop_stream_t stream)
+{
+    using namespace kop;
+    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    kop_status_t st = check_rows_cols(rows, vocab);
+    if (st != KOP_OK) return st;
+    if (!(label_smoothing >= 0.0f && label_smoothing < 1.0f)) return KOP_ERR_BAD_SHAPE;
+    if (rows == 0) return KOP_OK;
+    if (!logits || !labels || !loss || !workspace) return KOP_ERR_NULL_POINTER;
+    if (vocab > 0x7FFFFFFFLL || rows > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+    if ((st = check_row_stride(row_stride, vocab, rows)) != KOP_OK) return st;
+    const int esz = elem_size(dtype);
+    if (!aligned_to(logits, esz) || !aligned_to(labels, 4) || !aligned_to(loss, 4) ||
+        (mean_loss && !aligned_to(mean_loss, 4)) || (bad_label_count && !aligned_to(bad_label_count, 4)) ||
+        (counted_rows && !aligned_to(counted_rows, 4)) || !aligned_to(workspace, 16))
+        return KOP_ERR_MISALIGNED;
+    if (workspace_bytes < kop_ce_loss_rowwise_workspace_bytes(rows, vocab, dtype))
+        return KOP_ERR_WORKSPACE_TOO_SMALL;
+    if ((st = check_device()) != KOP_OK) return st;
+    cudaStream_t s = as_stream(stream);
+    const CeOpts opts{ignore_index, label_smoothing, counted_rows};
+    return dtype == KOP_F32
+               ? launch_ce<float, true>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s, opts)
+               : launch_ce<__nv_bfloat16, true>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s, opts);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -294,7 +372,7 @@ namespace kop {
 namespace {
 
 constexpr int64_t kStaticMaxRows = (int64_t)1 << 20;                       // 1,048,576 rows
-constexpr int64_t kStaticScratchWords = 4 + 3 * (kStaticMaxRows / kGroupRows);   // 12,292 words = 49,168 B
+constexpr int64_t kStaticScratchWords = 4 + 4 * (kStaticMaxRows / kGroupRows);   // 16,388 words = 65,552 B
 static __device__ __align__(256) unsigned int g_ce_static_scratch[kStaticScratchWords];
 
 // In host code the array's name is only a stand-in for the symbol, not a device address: the address

@@ -35,11 +35,29 @@ __device__ __forceinline__ float2 gelu_residual2(float2 x, float2 b, float2 r)
     return __ffma2_rn(hu, t, __fadd2_rn(hu, r));
 }
 
+// What precedes the normalisation: kProBiasGeluResidual: v = residual + gelu(x + bias) (the benchmark
+// segment); kProResidual: v = x + residual; kProNone: v = x. The unused operands are never loaded.
+enum { kProBiasGeluResidual = 0, kProResidual = 1, kProNone = 2 };
+template <int PRO, bool kFastTanh>
+__device__ __forceinline__ float2 prologue2(float2 x, float2 b, float2 r)
+{
+    if (PRO == kProBiasGeluResidual) return gelu_residual2<kFastTanh>(x, b, r);
+    if (PRO == kProResidual) return __fadd2_rn(x, r);
+    return x;
+}
+template <int PRO, bool kFastTanh>
+__device__ __forceinline__ float prologue1(float x, float b, float r)
+{
+    if (PRO == kProBiasGeluResidual) return r + gelu_tanh<kFastTanh>(x + b);
+    if (PRO == kProResidual) return x + r;
+    return x;
+}
+
 // CTA per row, row in registers as fp32 pairs. kFull: the row is exactly blockDim.x * VPT vectors
 // (no tail predicates). kWide: the eight fp32 parameters that go with a bf16 vector are fetched
 // with one 256-bit load per lane, so a warp touches each 128-byte line once (two 128-bit loads
 // per lane would walk every line twice and double the L1 wavefronts, which bound this kernel).
-template <typename T, int VPT, bool kFull, bool kWide>
+template <typename T, int VPT, bool kFull, bool kWide, int PRO>
 __global__ void __launch_bounds__(max_threads_for(VPT * Elem<T>::kPerVec))
 ln_block_kernel(const T* __restrict__ x, const T* __restrict__ res, const float* __restrict__ bias,
                 const float* __restrict__ gamma, const float* __restrict__ beta, T* __restrict__ y,
@@ -61,7 +79,8 @@ ln_block_kernel(const T* __restrict__ x, const T* __restrict__ res, const float*
         const int v = k * blockDim.x + threadIdx.x;
         if (kFull || v < nvec) {
             rx[k] = ld_stream(xr + (int64_t)v * E);
-            rres[k] = ld_stream(rr + (int64_t)v * E);
+            if (PRO <= kProResidual) rres[k] = ld_stream(rr + (int64_t)v * E);
+            else rres[k] = Vec16{{0u, 0u, 0u, 0u}};
         } else {
             rx[k] = Vec16{{0u, 0u, 0u, 0u}};
             rres[k] = Vec16{{0u, 0u, 0u, 0u}};
@@ -73,7 +92,7 @@ ln_block_kernel(const T* __restrict__ x, const T* __restrict__ res, const float*
     for (int k = 0; k < VPT; ++k) {
         const int v = k * blockDim.x + threadIdx.x;
         float2 bb[P], fx[P], fr[P];
-        if (kFull || v < nvec) load_params<E, kWide>(bias + (int64_t)v * E, bb);
+        if (PRO == kProBiasGeluResidual && (kFull || v < nvec)) load_params<E, kWide>(bias + (int64_t)v * E, bb);
         else {
 #pragma unroll
             for (int q = 0; q < P; ++q) bb[q] = make_float2(0.0f, 0.0f);
@@ -82,7 +101,7 @@ ln_block_kernel(const T* __restrict__ x, const T* __restrict__ res, const float*
         Elem<T>::unpack2(rres[k], fr);
 #pragma unroll
         for (int q = 0; q < P; ++q) {
-            float2 t = gelu_residual2<kFast>(fx[q], bb[q], fr[q]);
+            float2 t = prologue2<PRO, kFast>(fx[q], bb[q], fr[q]);
             if (!kFull && v >= nvec) t = make_float2(0.0f, 0.0f);
             val[k][q] = t;
             sum2 = __fadd2_rn(sum2, t);
@@ -129,7 +148,7 @@ ln_block_kernel(const T* __restrict__ x, const T* __restrict__ res, const float*
 // fetches its bias / gamma / beta once and applies them to the same columns of two rows, which
 // halves that traffic; both rows' reductions share the two barriers. The row must be exactly
 // blockDim.x * VPT vectors; `rows` may be odd (the last CTA then skips its second row).
-template <typename T, int VPT, bool kWide, int kMaxThreads>
+template <typename T, int VPT, bool kWide, int kMaxThreads, int PRO>
 __global__ void __launch_bounds__(kMaxThreads, 768 / kMaxThreads)
 ln_pair_kernel(const T* __restrict__ x, const T* __restrict__ res, const float* __restrict__ bias,
                const float* __restrict__ gamma, const float* __restrict__ beta, T* __restrict__ y,
@@ -152,7 +171,8 @@ ln_pair_kernel(const T* __restrict__ x, const T* __restrict__ res, const float* 
             const int64_t v = (int64_t)k * blockDim.x + threadIdx.x;
             if (r == 0 || two) {
                 rx[r][k] = ld_stream(x + (row0 + r) * x_stride + v * E);
-                rres[r][k] = ld_stream(res + (row0 + r) * r_stride + v * E);
+                if (PRO <= kProResidual) rres[r][k] = ld_stream(res + (row0 + r) * r_stride + v * E);
+                else rres[r][k] = Vec16{{0u, 0u, 0u, 0u}};
             } else {
                 rx[r][k] = Vec16{{0u, 0u, 0u, 0u}};
                 rres[r][k] = Vec16{{0u, 0u, 0u, 0u}};
@@ -164,7 +184,11 @@ ln_pair_kernel(const T* __restrict__ x, const T* __restrict__ res, const float* 
     for (int k = 0; k < VPT; ++k) {
         const int64_t v = (int64_t)k * blockDim.x + threadIdx.x;
         float2 bb[P];
-        load_params<E, kWide>(bias + v * E, bb);
+        if (PRO == kProBiasGeluResidual) load_params<E, kWide>(bias + v * E, bb);
+        else {
+#pragma unroll
+            for (int q = 0; q < P; ++q) bb[q] = make_float2(0.0f, 0.0f);
+        }
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
             float2 fx[P], fr[P];
@@ -172,7 +196,7 @@ ln_pair_kernel(const T* __restrict__ x, const T* __restrict__ res, const float* 
             Elem<T>::unpack2(rres[r][k], fr);
 #pragma unroll
             for (int q = 0; q < P; ++q) {
-                const float2 t = gelu_residual2<kFast>(fx[q], bb[q], fr[q]);
+                const float2 t = prologue2<PRO, kFast>(fx[q], bb[q], fr[q]);
                 val[r][k][q] = t;
                 sum2[r] = __fadd2_rn(sum2[r], t);
             }
@@ -231,7 +255,16 @@ ln_pair_kernel(const T* __restrict__ x, const T* __restrict__ res, const float* 
 }
 
 // Any hidden size / alignment: scalar loads, v recomputed in each of three sweeps.
-template <typename T>
+template <typename T, int PRO, bool kFast>
+__device__ __forceinline__ float ln_value(const T* xr, const T* rr, const float* bias, int64_t j)
+{
+    const float xv = Elem<T>::load1(xr + j);
+    const float rv = PRO <= kProResidual ? Elem<T>::load1(rr + j) : 0.0f;
+    const float bv = PRO == kProBiasGeluResidual ? __ldg(bias + j) : 0.0f;
+    return prologue1<PRO, kFast>(xv, bv, rv);
+}
+
+template <typename T, int PRO>
 __global__ void __launch_bounds__(256)
 ln_generic_kernel(const T* __restrict__ x, const T* __restrict__ res, const float* __restrict__ bias,
                   const float* __restrict__ gamma, const float* __restrict__ beta, T* __restrict__ y,
@@ -246,12 +279,12 @@ ln_generic_kernel(const T* __restrict__ x, const T* __restrict__ res, const floa
     T* yr = y + row * y_stride;
     float sum = 0.0f;
     for (int64_t j = threadIdx.x; j < hidden; j += blockDim.x)
-        sum += Elem<T>::load1(rr + j) + gelu_tanh<kFast>(Elem<T>::load1(xr + j) + __ldg(bias + j));
+        sum += ln_value<T, PRO, kFast>(xr, rr, bias, j);
     const float mu = block_sum(sum, red_a) * inv_hidden;
     float ss = 0.0f;
     for (int64_t j = threadIdx.x; j < hidden; j += blockDim.x) {
         const float d =
-            Elem<T>::load1(rr + j) + gelu_tanh<kFast>(Elem<T>::load1(xr + j) + __ldg(bias + j)) - mu;
+            ln_value<T, PRO, kFast>(xr, rr, bias, j) - mu;
         ss = fmaf(d, d, ss);
     }
     const float rs = rsqrtf(block_sum(ss, red_b) * inv_hidden + eps);
@@ -261,12 +294,12 @@ ln_generic_kernel(const T* __restrict__ x, const T* __restrict__ res, const floa
     }
     for (int64_t j = threadIdx.x; j < hidden; j += blockDim.x) {
         const float d =
-            Elem<T>::load1(rr + j) + gelu_tanh<kFast>(Elem<T>::load1(xr + j) + __ldg(bias + j)) - mu;
+            ln_value<T, PRO, kFast>(xr, rr, bias, j) - mu;
         Elem<T>::store1(yr + j, fmaf(d * rs, __ldg(gamma + j), __ldg(beta + j)));
     }
 }
 
-template <typename T>
+template <typename T, int PRO>
 kop_status_t launch_ln(const void* xv, const void* rv, const float* bias, const float* gamma,
                        const float* beta, void* yv, float* mean, float* rstd, int64_t rows,
                        int64_t hidden, int64_t xs, int64_t rs, int64_t ys, float eps,
@@ -278,15 +311,16 @@ kop_status_t launch_ln(const void* xv, const void* rv, const float* bias, const 
     constexpr int E = Elem<T>::kPerVec;
     const float inv_hidden = (float)(1.0 / (double)hidden);
     if (rows > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
-    const bool vec = vec_ok(x, hidden, xs, sizeof(T)) && vec_ok(r, hidden, rs, sizeof(T)) &&
-                     vec_ok(y, hidden, ys, sizeof(T)) && aligned_to(bias, 16) &&
+    const bool vec = vec_ok(x, hidden, xs, sizeof(T)) && (PRO > kProResidual || vec_ok(r, hidden, rs, sizeof(T))) &&
+                     vec_ok(y, hidden, ys, sizeof(T)) && (PRO != kProBiasGeluResidual || aligned_to(bias, 16)) &&
                      aligned_to(gamma, 16) && aligned_to(beta, 16);
     const int64_t nvec64 = hidden / E;
     if (vec && hidden <= kMaxRegisterRow) {
         const int nvec = (int)nvec64;
         // 32 values per thread (hidden 4096 -> 128-thread CTAs, eight 16-byte loads in flight per
         // thread and ~8 CTAs per SM); short rows use fewer, rows beyond 512 threads' worth use 64.
-        const bool wide = E == 8 && aligned_to(bias, 32) && aligned_to(gamma, 32) && aligned_to(beta, 32);
+        const bool wide = E == 8 && (PRO != kProBiasGeluResidual || aligned_to(bias, 32)) && aligned_to(gamma, 32) &&
+                          aligned_to(beta, 32);
         // Rows of 2048..8192 elements that split evenly into 16 values per thread go two per CTA
         // (parameters fetched once per pair) once there are enough pairs to fill the GPU.
         {
@@ -296,7 +330,7 @@ kop_status_t launch_ln(const void* xv, const void* rv, const float* bias, const 
                 rows >= 8 * (int64_t)sm_count()) {
                 const unsigned grid = (unsigned)((rows + 1) / 2);
 #define KOP_LN_PAIR(W, MT)                                                                              \
-    ln_pair_kernel<T, 16 / E, W, MT><<<grid, threads2, 0, stream>>>(x, r, bias, gamma, beta, y, mean, rstd, \
+    ln_pair_kernel<T, 16 / E, W, MT, PRO><<<grid, threads2, 0, stream>>>(x, r, bias, gamma, beta, y, mean, rstd, \
                                                                     rows, xs, rs, ys, eps, inv_hidden)
                 if (threads2 <= 256) { if (wide) KOP_LN_PAIR(true, 256); else KOP_LN_PAIR(false, 256); }
                 else { if (wide) KOP_LN_PAIR(true, 512); else KOP_LN_PAIR(false, 512); }
@@ -312,7 +346,7 @@ kop_status_t launch_ln(const void* xv, const void* rv, const float* bias, const 
         const int threads = ((nvec + vpt - 1) / vpt + 31) / 32 * 32;
         const bool full = (nvec % vpt) == 0 && (nvec / vpt) == threads;
 #define KOP_LN_LAUNCH(V, F, W)                                                                    \
-    ln_block_kernel<T, V, F, W><<<(unsigned)rows, threads, 0, stream>>>(x, r, bias, gamma, beta, y, mean, \
+    ln_block_kernel<T, V, F, W, PRO><<<(unsigned)rows, threads, 0, stream>>>(x, r, bias, gamma, beta, y, mean, \
                                                                         rstd, nvec, xs, rs, ys, eps, inv_hidden)
 #define KOP_LN(V)                                             \
     do {                                                      \
@@ -331,7 +365,7 @@ kop_status_t launch_ln(const void* xv, const void* rv, const float* bias, const 
 #undef KOP_LN
         return launch_status();
     }
-    ln_generic_kernel<T><<<(unsigned)rows, 256, 0, stream>>>(x, r, bias, gamma, beta, y, mean, rstd,
+    ln_generic_kernel<T, PRO><<<(unsigned)rows, 256, 0, stream>>>(x, r, bias, gamma, beta, y, mean, rstd,
                                                              hidden, xs, rs, ys, eps, inv_hidden);
     return launch_status();
 }
@@ -365,8 +399,47 @@ extern "C" kop_status_t kop_bias_gelu_residual_layernorm(
     if ((st = check_device()) != KOP_OK) return st;
     cudaStream_t s = as_stream(stream);
     return dtype == KOP_F32
-               ? launch_ln<float>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
+               ? launch_ln<float, kProBiasGeluResidual>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
                                   x_row_stride, res_row_stride, y_row_stride, eps, s)
-               : launch_ln<__nv_bfloat16>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
+               : launch_ln<__nv_bfloat16, kProBiasGeluResidual>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
                                           x_row_stride, res_row_stride, y_row_stride, eps, s);
+}
+
+extern "C" kop_status_t kop_residual_layernorm(const void* x, const void* residual, const float* gamma,
+                                               const float* beta, void* y, float* mean, float* rstd,
+                                               int64_t rows, int64_t hidden, int64_t x_row_stride,
+                                               int64_t res_row_stride, int64_t y_row_stride, float eps,
+                                               kop_dtype_t dtype, kop_stream_t stream)
+{
+    using namespace kop;
+    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    kop_status_t st = check_rows_cols(rows, hidden);
+    if (st != KOP_OK) return st;
+    if (rows == 0) return KOP_OK;
+    if (!x || !gamma || !beta || !y) return KOP_ERR_NULL_POINTER;
+    if ((st = check_row_stride(x_row_stride, hidden, rows)) != KOP_OK) return st;
+    if (residual && (st = check_row_stride(res_row_stride, hidden, rows)) != KOP_OK) return st;
+    if ((st = check_row_stride(y_row_stride, hidden, rows)) != KOP_OK) return st;
+    if (!(eps >= 0.0f)) return KOP_ERR_BAD_SHAPE;
+    const int esz = elem_size(dtype);
+    if (!aligned_to(x, esz) || (residual && !aligned_to(residual, esz)) || !aligned_to(y, esz) ||
+        !aligned_to(gamma, 4) || !aligned_to(beta, 4) || (mean && !aligned_to(mean, 4)) ||
+        (rstd && !aligned_to(rstd, 4)))
+        return KOP_ERR_MISALIGNED;
+    if (!alias_ok(x, x_row_stride, y, y_row_stride, rows, hidden, esz, true) ||
+        (residual && !alias_ok(residual, res_row_stride, y, y_row_stride, rows, hidden, esz, true)))
+        return KOP_ERR_BAD_ALIAS;
+    if ((st = check_device()) != KOP_OK) return st;
+    cudaStream_t s = as_stream(stream);
+    const int64_t rs = residual ? res_row_stride : x_row_stride;
+    if (residual != nullptr)
+        return dtype == KOP_F32
+                   ? launch_ln<float, kProResidual>(x, residual, nullptr, gamma, beta, y, mean, rstd, rows, hidden,
+                                                    x_row_stride, rs, y_row_stride, eps, s)
+                   : launch_ln<__nv_bfloat16, kProResidual>(x, residual, nullptr, gamma, beta, y, mean, rstd, rows,
+                                                            hidden, x_row_stride, rs, y_row_stride, eps, s);
+    return dtype == KOP_F32 ? launch_ln<float, kProNone>(x, x, nullptr, gamma, beta, y, mean, rstd, rows, hidden,
+                                                         x_row_stride, rs, y_row_stride, eps, s)
+                            : launch_ln<__nv_bfloat16, kProNone>(x, x, nullptr, gamma, beta, y, mean, rstd, rows,
+                                                                 hidden, x_row_stride, rs, y_row_stride, eps, s);
 }

@@ -120,6 +120,66 @@ silu_mul_kernel(const T* __restrict__ gu, T* __restrict__ out, int nvec, int til
     }
 }
 
+// Interleaved layout [g0, u0, g1, u1, ...]: an output vector needs the two consecutive input vectors
+// that hold its E (gate, up) pairs; for bf16 every 32-bit word is exactly one pair.
+template <typename T, int U, bool kFull>
+__global__ void __launch_bounds__(256)
+silu_mul_interleaved_kernel(const T* __restrict__ gu, T* __restrict__ out, int nvec, int tiles_per_row,
+                            int64_t in_stride, int64_t out_stride)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    constexpr bool kFast = sizeof(T) == 2;
+    const unsigned urow = blockIdx.x / (unsigned)tiles_per_row;
+    const int tile = (int)(blockIdx.x - urow * (unsigned)tiles_per_row);
+    const int64_t row = urow;
+    const T* g = gu + row * in_stride;
+    T* o = out + row * out_stride;
+    const int v0 = tile * (U * blockDim.x) + threadIdx.x;
+    Vec16 r0[U], r1[U];
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+        const int v = v0 + k * blockDim.x;
+        if (kFull || v < nvec) {
+            r0[k] = ld_stream(g + (int64_t)(2 * v) * E);
+            r1[k] = ld_stream(g + (int64_t)(2 * v + 1) * E);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+        const int v = v0 + k * blockDim.x;
+        if (kFull || v < nvec) {
+            float f[2 * E], res[E];
+            float lo[E], hi[E];
+            Elem<T>::unpack(r0[k], lo);
+            Elem<T>::unpack(r1[k], hi);
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                f[e] = lo[e];
+                f[E + e] = hi[e];
+            }
+#pragma unroll
+            for (int e = 0; e < E; ++e) res[e] = silu<kFast>(f[2 * e]) * f[2 * e + 1];
+            st_stream(o + (int64_t)v * E, Elem<T>::pack(res));
+        }
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+silu_mul_interleaved_scalar_kernel(const T* __restrict__ gu, T* __restrict__ out, int64_t rows, int64_t inter,
+                                   int64_t in_stride, int64_t out_stride)
+{
+    constexpr bool kFast = sizeof(T) == 2;
+    const int64_t total = rows * inter;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / inter, j = i - r * inter;
+        const float g = Elem<T>::load1(gu + r * in_stride + 2 * j);
+        const float u = Elem<T>::load1(gu + r * in_stride + 2 * j + 1);
+        Elem<T>::store1(out + r * out_stride + j, silu<kFast>(g) * u);
+    }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256)
 silu_mul_scalar_kernel(const T* __restrict__ gu, T* __restrict__ out, int64_t rows, int64_t inter,
@@ -271,6 +331,33 @@ kop_status_t launch_silu_mul(const void* guv, void* outv, int64_t rows, int64_t 
 }
 
 template <typename T>
+kop_status_t launch_silu_mul_interleaved(const void* guv, void* outv, int64_t rows, int64_t inter, int64_t is,
+                                         int64_t os, cudaStream_t stream)
+{
+    const T* gu = static_cast<const T*>(guv);
+    T* out = static_cast<T*>(outv);
+    constexpr int E = Elem<T>::kPerVec;
+    const bool vec = aligned_to(gu, 16) && aligned_to(out, 16) && (inter % E) == 0 && (is % E) == 0 &&
+                     (os % E) == 0;
+    const int64_t nvec64 = inter / E;
+    if (vec && nvec64 <= 0x3FFFFFFF) {
+        const int nvec = (int)nvec64;
+        const int threads = 128;
+        constexpr int U = 2;
+        const int tiles = (nvec + threads * U - 1) / (threads * U);
+        const int64_t grid = rows * tiles;
+        if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+        if (nvec % (threads * U) == 0)
+            silu_mul_interleaved_kernel<T, U, true><<<(unsigned)grid, threads, 0, stream>>>(gu, out, nvec, tiles, is, os);
+        else
+            silu_mul_interleaved_kernel<T, U, false><<<(unsigned)grid, threads, 0, stream>>>(gu, out, nvec, tiles, is, os);
+        return launch_status();
+    }
+    silu_mul_interleaved_scalar_kernel<T><<<scalar_grid(rows * inter), 256, 0, stream>>>(gu, out, rows, inter, is, os);
+    return launch_status();
+}
+
+template <typename T>
 kop_status_t launch_residual_add(const void* av, const void* bv, void* ov, int64_t rows, int64_t cols,
                                  int64_t as, int64_t bs, int64_t os, cudaStream_t stream)
 {
@@ -387,6 +474,34 @@ extern "C" kop_status_t kop_silu_mul(const void* gate_up, void* out, int64_t row
     return dtype == KOP_F32
                ? launch_silu_mul<float>(gate_up, out, rows, inter, in_row_stride, out_row_stride, s)
                : launch_silu_mul<__nv_bfloat16>(gate_up, out, rows, inter, in_row_stride, out_row_stride, s);
+}
+
+extern "C" kop_status_t kop_silu_mul_interleaved(const void* gate_up, void* out, int64_t rows, int64_t inter,
+                                                 int64_t in_row_stride, int64_t out_row_stride,
+                                                 kop_dtype_t dtype, kop_stream_t stream)
+{
+    using namespace kop;
+    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    kop_status_t st = check_rows_cols(rows, inter);
+    if (st != KOP_OK) return st;
+    if (rows == 0) return KOP_OK;
+    if (!gate_up || !out) return KOP_ERR_NULL_POINTER;
+    if (inter > kMaxElems / 2) return KOP_ERR_BAD_SHAPE;
+    if ((st = check_row_stride(in_row_stride, 2 * inter, rows)) != KOP_OK) return st;
+    if ((st = check_row_stride(out_row_stride, inter, rows)) != KOP_OK) return st;
+    const int esz = elem_size(dtype);
+    if (!aligned_to(gate_up, esz) || !aligned_to(out, esz)) return KOP_ERR_MISALIGNED;
+    {
+        uintptr_t a0, a1, b0, b1;
+        span_of(gate_up, rows, 2 * inter, in_row_stride, esz, &a0, &a1);
+        span_of(out, rows, inter, out_row_stride, esz, &b0, &b1);
+        if (!(a1 <= b0 || b1 <= a0)) return KOP_ERR_BAD_ALIAS;
+    }
+    if ((st = check_device()) != KOP_OK) return st;
+    cudaStream_t s = as_stream(stream);
+    return dtype == KOP_F32
+               ? launch_silu_mul_interleaved<float>(gate_up, out, rows, inter, in_row_stride, out_row_stride, s)
+               : launch_silu_mul_interleaved<__nv_bfloat16>(gate_up, out, rows, inter, in_row_stride, out_row_stride, s);
 }
 
 extern "C" kop_status_t kop_residual_add(const void* a, const void* b, void* out, int64_t rows,

@@ -64,6 +64,12 @@ def lib() -> C.CDLL:
     L.kop_rmsnorm.argtypes = [vp, vp, vp, i64, i64, i64, i64, f32, i32, vp]
     L.kop_silu_mul.argtypes = [vp, vp, i64, i64, i64, i64, i32, vp]
     L.kop_residual_add.argtypes = [vp, vp, vp, i64, i64, i64, i64, i64, i32, vp]
+    L.kop_ce_loss_rowwise_opts.argtypes = [vp] * 6 + [i64] * 3 + [C.c_int32, f32, vp, sz, i32, vp]
+    L.kop_ce_loss_rowwise_opts.restype = i32
+    L.kop_residual_layernorm.argtypes = [vp] * 7 + [i64] * 5 + [f32, i32, vp]
+    L.kop_residual_layernorm.restype = i32
+    L.kop_silu_mul_interleaved.argtypes = [vp, vp, i64, i64, i64, i64, i32, vp]
+    L.kop_silu_mul_interleaved.restype = i32
     L.kop_row_scale.argtypes = [vp, vp, vp, i64, i64, i64, i64, i32, vp]
     L.kop_row_scale.restype = i32
     L.kop_matvec_bias.argtypes = [vp, vp, f32, vp, i64, i64, i64, i32, vp]
@@ -238,6 +244,61 @@ def kop_residual_add(a, b, out=None, stream=None):
     _, _, os_ = _rows2d(out, "out")
     _check(lib().kop_residual_add(a.data_ptr(), b.data_ptr(), out.data_ptr(), rows, cols, as_, bs, os_,
                                   _dtype_tag(a), _stream(stream)), "kop_residual_add")
+    return out
+
+
+def kop_ce_loss_rowwise_opts(logits, labels, ignore_index=-100, label_smoothing=0.0, loss=None, mean_loss=None,
+                             bad_label_count=None, counted_rows=None, workspace=None, stream=None):
+    """Returns (loss[rows], mean_loss[1], bad_label_count[1], counted_rows[1]) as device tensors."""
+    rows, vocab, zs = _rows2d(logits, "logits")
+    if labels.dtype != torch.int32 or not labels.is_cuda or not labels.is_contiguous() or labels.numel() != rows:
+        raise ValueError("labels: expected a contiguous int32 CUDA vector of `rows` elements")
+    dev = logits.device
+    loss = torch.empty(rows, dtype=torch.float32, device=dev) if loss is None else loss
+    mean_loss = torch.empty(1, dtype=torch.float32, device=dev) if mean_loss is None else mean_loss
+    bad_label_count = torch.empty(1, dtype=torch.int32, device=dev) if bad_label_count is None else bad_label_count
+    counted_rows = torch.empty(1, dtype=torch.int32, device=dev) if counted_rows is None else counted_rows
+    need = kop_ce_loss_rowwise_workspace_bytes(rows, vocab, _dtype_tag(logits))
+    if workspace is None:
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
+    _check(lib().kop_ce_loss_rowwise_opts(logits.data_ptr(), labels.data_ptr(), loss.data_ptr(),
+                                          mean_loss.data_ptr(), bad_label_count.data_ptr(),
+                                          counted_rows.data_ptr(), rows, vocab, zs, int(ignore_index),
+                                          float(label_smoothing), workspace.data_ptr(),
+                                          workspace.numel() * workspace.element_size(), _dtype_tag(logits),
+                                          _stream(stream)), "kop_ce_loss_rowwise_opts")
+    return loss, mean_loss, bad_label_count, counted_rows
+
+
+def kop_residual_layernorm(x, residual, gamma, beta, eps, out=None, mean=None, rstd=None, want_stats=True,
+                           stream=None):
+    rows, hidden, xs = _rows2d(x, "x")
+    rs = xs
+    if residual is not None:
+        _, _, rs = _rows2d(residual, "residual")
+        assert residual.shape == x.shape and residual.dtype == x.dtype
+    out = torch.empty_like(x) if out is None else out
+    _, _, ys = _rows2d(out, "out")
+    if want_stats:
+        mean = torch.empty(rows, dtype=torch.float32, device=x.device) if mean is None else mean
+        rstd = torch.empty(rows, dtype=torch.float32, device=x.device) if rstd is None else rstd
+    _check(lib().kop_residual_layernorm(
+        x.data_ptr(), None if residual is None else residual.data_ptr(), _param(gamma, "gamma", hidden),
+        _param(beta, "beta", hidden), out.data_ptr(), None if mean is None else mean.data_ptr(),
+        None if rstd is None else rstd.data_ptr(), rows, hidden, xs, rs, ys, float(eps), _dtype_tag(x),
+        _stream(stream)), "kop_residual_layernorm")
+    return out, mean, rstd
+
+
+def kop_silu_mul_interleaved(gate_up, out=None, stream=None):
+    rows, two_i, is_ = _rows2d(gate_up, "gate_up")
+    if two_i % 2:
+        raise ValueError("gate_up: the row length must be even ([g0, u0, g1, u1, ...])")
+    inter = two_i // 2
+    out = torch.empty((rows, inter), dtype=gate_up.dtype, device=gate_up.device) if out is None else out
+    _, _, os_ = _rows2d(out, "out")
+    _check(lib().kop_silu_mul_interleaved(gate_up.data_ptr(), out.data_ptr(), rows, inter, is_, os_,
+                                          _dtype_tag(gate_up), _stream(stream)), "kop_silu_mul_interleaved")
     return out
 
 

@@ -499,3 +499,89 @@ def test_row_ops_options_and_full_configs(kop):
     assert np.array_equal(to_f64(kop.kop_row_scale(a, wb[:, 1024:5120])), rs.astype(np.float32).astype(np.float64))
     assert kop.kop_row_scale(a[:0], b[:0]).shape == (0, 4096)
     assert kop.kop_matvec_bias(x[:0], w, b_sum).shape == (0,)
+
+
+# ------------------------------------------------------------------------------------------ coverage variants
+
+RLN_SHAPES = [(2048, 4096, BF16), (1185, 4096, BF16), (300, 4096, F32), (65, 256, BF16), (9, 20480, BF16),
+              (21, 513, F32)]
+
+
+@pytest.mark.parametrize("rows,hidden,dtype", RLN_SHAPES)
+@pytest.mark.parametrize("with_residual", [True, False])
+@pytest.mark.parametrize("seed", SEEDS[:3])
+def test_residual_layernorm_parity(kop, rows, hidden, dtype, with_residual, seed):
+    x, r, _, g, be = synth.layernorm_inputs(rows, hidden, dtype, seed, "cuda")
+    res = r if with_residual else None
+    out = Guarded((rows, hidden), dtype)
+    mean = Guarded((rows,), F32)
+    rstd = Guarded((rows,), F32)
+    kop.kop_residual_layernorm(x, res, g, be, 1e-5, out=out.t, mean=mean.t, rstd=rstd.t)
+    ry, rm, rr = kopref.residual_layernorm(host(x), None if res is None else host(res), host(g), host(be), 1e-5,
+                                           threads=None)
+    assert_close(out.t, ry, tol_of(dtype), "rln y")
+    assert_close(mean.t, rm, 1e-5, "rln mean (exact fp32 sums of the inputs)")
+    assert_close(rstd.t, rr, 1e-5, "rln rstd")
+    if dtype == BF16:
+        assert_bf16_tight(out.t, ry, "rln y", floor=1e-6)
+    for gd in (out, mean, rstd):
+        gd.check("rln")
+
+
+@pytest.mark.parametrize("rows,inter,dtype", [(512, 14336, BF16), (100, 4096, F32), (33, 1000, BF16), (17, 1001, F32), (5, 1, F32)])
+@pytest.mark.parametrize("seed", SEEDS[:3])
+def test_silu_mul_interleaved_parity(kop, rows, inter, dtype, seed):
+    gu = synth.gate_up_inputs(rows, inter, dtype, seed, "cuda", std=3.0)
+    out = Guarded((rows, inter), dtype)
+    kop.kop_silu_mul_interleaved(gu, out=out.t)
+    ref = kopref.silu_mul_interleaved(host(gu), threads=None)
+    assert_close(out.t, ref, tol_of(dtype), "silu_mul_interleaved")
+    if dtype == BF16:
+        assert_bf16_tight(out.t, ref, "silu_mul_interleaved", floor=1e-6)
+    out.check("silu_mul_interleaved")
+    # same numbers as the split layout on the de-interleaved columns
+    split = torch.cat([gu[:, 0::2], gu[:, 1::2]], dim=1).contiguous()
+    assert torch.equal(out.t, kop.kop_silu_mul(split))
+
+
+@pytest.mark.parametrize("rows,vocab,dtype", [(2048, 32000, BF16), (300, 4096, F32), (257, 50264, BF16), (21, 32001, BF16), (9, 8, F32)])
+@pytest.mark.parametrize("smoothing", [0.0, 0.1])
+@pytest.mark.parametrize("seed", SEEDS[:3])
+def test_ce_opts_parity(kop, rows, vocab, dtype, smoothing, seed):
+    z, lab = synth.ce_inputs(rows, vocab, dtype, seed, "cuda")
+    lab = lab.clone()
+    lab[::5] = -100                                    # every fifth row is ignored
+    loss = Guarded((rows,), F32)
+    mean = Guarded((1,), F32)
+    bad = Guarded((1,), torch.int32)
+    cnt = Guarded((1,), torch.int32)
+    kop.kop_ce_loss_rowwise_opts(z, lab, -100, smoothing, loss=loss.t, mean_loss=mean.t, bad_label_count=bad.t,
+                                 counted_rows=cnt.t)
+    rl, rmean, rbad, rcnt = kopref.ce_loss_opts(host(z), host(lab), -100, smoothing, threads=None)
+    assert_close(loss.t, rl, 2e-5, "ce opts loss")
+    assert_close(mean.t, np.array([rmean]), 2e-5, "ce opts mean")
+    assert int(bad.t.item()) == rbad == 0 and int(cnt.t.item()) == rcnt
+    assert bool((loss.t[::5] == 0).all())
+    for gd in (loss, mean, bad, cnt):
+        gd.check("ce opts")
+
+
+def test_ce_opts_edge_cases(kop):
+    z, lab = synth.ce_inputs(64, 4096, BF16, 3, "cuda")
+    # no ignored row, no smoothing: bit-identical to the plain entry point
+    a = kop.kop_ce_loss_rowwise_opts(z, lab, -100, 0.0)
+    b = kop.kop_ce_loss_rowwise(z, lab)
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1]) and int(a[3].item()) == 64
+    # everything ignored: zero losses, NaN mean, nothing counted
+    allig = torch.full_like(lab, 7)
+    l, m, bd, c = kop.kop_ce_loss_rowwise_opts(z, allig, 7, 0.2)
+    assert bool((l == 0).all()) and bool(torch.isnan(m[0])) and int(c.item()) == 0 and int(bd.item()) == 0
+    # a bad label next to ignored rows
+    lab2 = lab.clone()
+    lab2[1] = 4096
+    lab2[2] = -100
+    l, m, bd, c = kop.kop_ce_loss_rowwise_opts(z, lab2, -100, 0.0)
+    assert bool(torch.isnan(l[1])) and float(l[2]) == 0.0 and int(bd.item()) == 1 and int(c.item()) == 63
+    with pytest.raises(kop.KopError) as ei:
+        kop.kop_ce_loss_rowwise_opts(z, lab, -100, 1.0)
+    assert ei.value.status == 2
