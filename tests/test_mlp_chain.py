@@ -1,5 +1,5 @@
 """The chained transformer-MLP segment (RMSNorm -> vendor GEMM -> SiLU*up -> vendor GEMM -> residual)
-against the pure-float64 oracle chain, judged with the paper's model-level rule (Gate 3): strict
+against the pure-float64 oracle chain, checked with the paper's model-level rule (Gate 3): strict
 comparison first, else the float64 disambiguation with an unfused same-dtype chain as the
 baseline (rho = d_opt / d_ref <= 10, scale-relative check when the baseline is exact, absolute
 escape bound). Also: per-kernel parity on the actual device intermediates, CUDA-graph capture of
