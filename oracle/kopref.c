@@ -481,3 +481,43 @@ int kopref_ce_loss_opts(const void* logits, const int32_t* labels, double* loss,
     if (counted_rows) *counted_rows = counted;
     return 0;
 }
+
+/* ---- GroupNorm (InstanceNorm when groups == C) + activation, NCHW -------------------------------------------
+ * For every image n and group g (C/groups consecutive channels): mu, var (biased) over the group's
+ * (C/groups) * H * W elements; y = (x - mu) / sqrt(var + eps) * gamma[c] + beta[c] (gamma / beta may be NULL:
+ * 1 and 0); then act: 0 = none, 1 = ReLU (NaN kept), 2 = SiLU.  mean / rstd: [N, groups], may be NULL. */
+int kopref_groupnorm_act(const void* x, const float* gamma, const float* beta, double* y, double* mean,
+        double* rstd, int64_t N, int64_t C, int64_t H, int64_t W, int64_t groups, double eps, int act,
+        int dtype, int threads)
+{
+    if (!x || !y || N < 0 || C <= 0 || H <= 0 || W <= 0 || groups <= 0 || C % groups || bad_dtype(dtype)) return -1;
+    if (act < 0 || act > 2) return -1;
+    const int64_t cpg = C / groups, plane = H * W, chunk = cpg * plane;
+    int nt = pick_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t ng = 0; ng < N * groups; ++ng) {
+        const int64_t g = ng % groups;
+        const int64_t base = ng * chunk;
+        double sum = 0.0;
+        for (int64_t k = 0; k < chunk; ++k) sum += load_elem(x, base + k, dtype);
+        const double mu = sum / (double)chunk;
+        double ss = 0.0;
+        for (int64_t k = 0; k < chunk; ++k) {
+            double d = load_elem(x, base + k, dtype) - mu;
+            ss += d * d;
+        }
+        const double rs = 1.0 / sqrt(ss / (double)chunk + eps);
+        for (int64_t k = 0; k < chunk; ++k) {
+            const int64_t c = g * cpg + k / plane;
+            double v = (load_elem(x, base + k, dtype) - mu) * rs;
+            v = v * (gamma ? (double)gamma[c] : 1.0) + (beta ? (double)beta[c] : 0.0);
+            if (act == 1) v = (v != v) ? v : (v > 0.0 ? v : 0.0);
+            else if (act == 2) v = v / (1.0 + exp(-v));
+            y[base + k] = v;
+        }
+        if (mean) mean[ng] = mu;
+        if (rstd) rstd[ng] = rs;
+    }
+    return 0;
+}

@@ -43,6 +43,7 @@ def lib() -> C.CDLL:
         _lib.kopref_residual_layernorm.argtypes = [vp] * 7 + [i64] * 5 + [dbl, C.c_int, C.c_int]
         _lib.kopref_silu_mul_interleaved.argtypes = [vp] * 2 + [i64] * 4 + [C.c_int, C.c_int]
         _lib.kopref_ce_loss_opts.argtypes = [vp] * 6 + [i64] * 3 + [C.c_int32, dbl, C.c_int, C.c_int]
+        _lib.kopref_groupnorm_act.argtypes = [vp] * 6 + [i64] * 5 + [dbl, C.c_int, C.c_int, C.c_int]
         _lib.kopref_row_scale.argtypes = [vp, vp, vp, i64, i64, i64, i64, C.c_int, C.c_int]
         _lib.kopref_matvec_bias.argtypes = [vp, vp, dbl, vp, i64, i64, i64, C.c_int, C.c_int]
     return _lib
@@ -257,6 +258,19 @@ def ce_loss_opts(logits, labels, ignore_index=-100, smoothing=0.0, threads=1):
                                      C.addressof(cnt), rows, vocab, vocab, int(ignore_index), float(smoothing),
                                      dt, _nt(threads)), "ce_loss_opts")
     return loss, mean.value, bad.value, cnt.value
+
+
+def groupnorm_act(x, gamma, beta, groups, eps, act=0, threads=1):
+    """x is NCHW contiguous; act 0 none / 1 relu / 2 silu. Returns (y, mean[N,groups], rstd[N,groups])."""
+    xa, dt = as_data(x)
+    N, Cc, H, W = xa.shape
+    g, be = as_param(gamma), as_param(beta)
+    y = np.empty((N, Cc, H, W), dtype=np.float64)
+    mean = np.empty((N, groups), dtype=np.float64)
+    rstd = np.empty((N, groups), dtype=np.float64)
+    _check(lib().kopref_groupnorm_act(_p(xa), _p(g), _p(be), _p(y), _p(mean), _p(rstd), N, Cc, H, W, int(groups),
+                                      float(eps), int(act), dt, _nt(threads)), "groupnorm_act")
+    return y, mean, rstd
 
 
 def row_scale(a, b, threads=1) -> np.ndarray:

@@ -544,6 +544,47 @@ def test_ce_options_against_library_and_base_oracle():
     assert b3 == 1 and c3 == 2 and math.isnan(l3[0]) and math.isnan(m3)
 
 
+# --------------------------------------------------------------------------- GroupNorm / InstanceNorm + activation
+
+def test_groupnorm_library_invariants_and_instance_norm():
+    N, Cc, H, W, G = 3, 12, 5, 7, 4
+    x = f32(RNG.standard_normal((N, Cc, H, W)) * 2 + 0.5)
+    g = f32(1 + 0.1 * RNG.standard_normal(Cc))
+    b = f32(0.1 * RNG.standard_normal(Cc))
+    tx, tg, tb = (torch.from_numpy(a.astype(np.float64)) for a in (x, g, b))
+    y, mu, rstd = kopref.groupnorm_act(x, g, b, G, 1e-5)
+    assert np.max(np.abs(y - F.group_norm(tx, G, tg, tb, 1e-5).numpy())) <= 1e-13
+    xs = x.astype(np.float64).reshape(N, G, -1)
+    assert np.allclose(mu, xs.mean(axis=2), rtol=0, atol=1e-14)
+    assert np.allclose(rstd, 1 / np.sqrt(xs.var(axis=2) + 1e-5), rtol=1e-13, atol=0)
+    # no affine: every group has zero mean and variance var/(var+eps)
+    y0, _, _ = kopref.groupnorm_act(x, None, None, G, 1e-5)
+    ys = y0.reshape(N, G, -1)
+    assert np.all(np.abs(ys.mean(axis=2)) <= 1e-12)
+    assert np.allclose(ys.var(axis=2), xs.var(axis=2) / (xs.var(axis=2) + 1e-5), rtol=1e-12, atol=0)
+    # groups == C is InstanceNorm; groups == 1 normalises the whole image (LayerNorm over C,H,W)
+    yi, _, _ = kopref.groupnorm_act(x, None, None, Cc, 1e-5)
+    assert np.max(np.abs(yi - F.instance_norm(tx, eps=1e-5).numpy())) <= 1e-13
+    y1, _, _ = kopref.groupnorm_act(x, None, None, 1, 1e-5)
+    assert np.max(np.abs(y1 - F.layer_norm(tx, (Cc, H, W), eps=1e-5).numpy())) <= 1e-13
+    # the affine step indexes the channel, not the group (a group-indexed gamma fails this)
+    gsel = f32(np.arange(1, Cc + 1))
+    ysel, _, _ = kopref.groupnorm_act(x, gsel, None, G, 1e-5)
+    assert np.allclose(ysel, y0 * gsel.astype(np.float64)[None, :, None, None], rtol=1e-14, atol=1e-14)
+    # activations act on the normalised, affine-transformed value
+    yr, _, _ = kopref.groupnorm_act(x, g, b, G, 1e-5, act=1)
+    ysl, _, _ = kopref.groupnorm_act(x, g, b, G, 1e-5, act=2)
+    assert np.array_equal(yr, np.maximum(y, 0.0))
+    assert np.max(np.abs(ysl - F.silu(torch.from_numpy(y)).numpy())) <= 1e-14
+    # bf16 input widened exactly; constant group -> zeros (var 0, rstd = 1/sqrt(eps))
+    xb = to_bf16_bits(x)
+    yb, _, _ = kopref.groupnorm_act(xb, g, b, G, 1e-5)
+    txb = torch.from_numpy(x).to(torch.bfloat16).to(torch.float64)
+    assert np.max(np.abs(yb - F.group_norm(txb, G, tg, tb, 1e-5).numpy())) <= 1e-13
+    yc, muc, rc = kopref.groupnorm_act(f32(np.full((1, 4, 2, 2), 3.0)), None, None, 2, 1e-5)
+    assert np.all(yc == 0.0) and np.all(muc == 3.0) and np.allclose(rc, 1 / math.sqrt(1e-5), rtol=1e-15)
+
+
 # --------------------------------------------------------------------------- row scale, mat-vec + bias sum
 
 def test_row_scale_is_diag_times_matrix():
