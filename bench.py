@@ -91,6 +91,9 @@ def segment_bytes():
     out["silu_mul_interleaved"] = dict(out["silu_mul"])
     kept = z["rows"] - (z["rows"] + 4) // 5            # every fifth row is ignored and never read
     out["ce_loss_opts"] = dict(bytes=kept * z["vocab"] * 2 + 2 * z["rows"] * 4 + 8, elems=kept * z["vocab"])
+    q = c["groupnorm"]
+    e = q["N"] * q["C"] * q["H"] * q["W"]
+    out["groupnorm"] = dict(bytes=2 * e * 4 + 2 * q["C"] * 4 + 2 * q["N"] * q["groups"] * 4, elems=e)
     return out
 
 
@@ -234,7 +237,7 @@ class Workload:
 
     ORDER = ["softmax_small", "softmax_large", "layernorm", "bn_pool", "ce_loss", "rmsnorm", "silu_mul", "residual_add"]
     # Beyond the benchmark configs (not part of `value`): the two kernels the paper's case studies print.
-    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "silu_mul_interleaved", "ce_loss_opts"]
+    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "silu_mul_interleaved", "ce_loss_opts", "groupnorm"]
 
     def __init__(self, kop, device, seed, only=None, rows_div=1):
         """only: build just these segments (None = all, plus the MLP segment); rows_div cuts the row
@@ -284,6 +287,12 @@ class Workload:
             v = c["matvec_bias"]
             self.vx, self.vw, self.vb = synth.matvec_inputs(cut(v["rows"]), v["k"], v["dtype"], seed, dev)
             self.vo = torch.empty(self.vx.shape[0], dtype=torch.float32, device=dev)
+        if "groupnorm" in want:
+            q = c["groupnorm"]
+            self.qx, self.qg, self.qb = synth.groupnorm_inputs(cut(q["N"]), q["C"], q["H"], q["W"], q["dtype"], seed, dev)
+            self.qy = torch.empty_like(self.qx)
+            self.qmean = torch.empty((self.qx.shape[0], q["groups"]), dtype=torch.float32, device=dev)
+            self.qrstd = torch.empty_like(self.qmean)
         m = c["mlp"]
         self.eps = m["eps"]
         rows = cut(m["rows"])
@@ -344,6 +353,10 @@ class Workload:
         elif name == "ce_loss_opts":             # the CE config with every fifth row ignored, smoothing 0.1
             k.kop_ce_loss_rowwise_opts(self.cz, self.clab_ig, -100, 0.1, loss=self.closs, mean_loss=self.cmean,
                                        bad_label_count=self.cbad, counted_rows=self.ccnt, workspace=self.cws)
+        elif name == "groupnorm":                # GroupNorm(32) + SiLU over [64, 256, 56, 56] fp32
+            q = c["groupnorm"]
+            k.kop_groupnorm_act(self.qx, self.qg, self.qb, q["groups"], q["eps"], q["act"], out=self.qy,
+                                mean=self.qmean, rstd=self.qrstd)
         else:
             raise KeyError(name)
 

@@ -267,6 +267,32 @@ kop_status_t kop_matvec_bias(const void* x, const float* w, float b_sum, float* 
                              int64_t k, int64_t x_row_stride, kop_dtype_t dtype, kop_stream_t stream);
 
 /*
+ * GroupNorm with optional per-channel affine and activation (the per-kernel results table's InstanceNorm
+ * row, L1-034, and GroupNorm row, L1-035, which the paper's system left at its fallback; fusion agent:
+ * normalisation followed by a pointwise op is one load and one store). For image n and group g over the
+ * (C / groups) * H * W elements of that group:
+ *   mu = mean(x), var = mean((x - mu)^2)              (biased variance)
+ *   y[n,c,h,w] = act((x[n,c,h,w] - mu) / sqrt(var + eps) * gamma[c] + beta[c])
+ * groups == C is InstanceNorm; groups == 1 normalises whole images. act: 0 identity, 1 ReLU (NaN passes),
+ * 2 SiLU v / (1 + exp(-v)).
+ * x, y: [N, C, H, W] contiguous NCHW of `dtype`; y may be x exactly. gamma, beta: fp32 [C], each may be NULL
+ * (1 and 0). mean, rstd: fp32 [N, groups] outputs, each may be NULL. Statistics are fp32, accumulated as
+ * (count, mean, M2) triples merged pairwise in a fixed order, so results do not depend on scheduling.
+ * Errors: groups must divide C; act outside 0..2 or eps < 0 or NaN is KOP_ERR_BAD_SHAPE. N == 0 is KOP_OK.
+ */
+kop_status_t kop_groupnorm_act(const void* x, const float* gamma, const float* beta, void* y,
+                               float* mean, float* rstd, int64_t N, int64_t C, int64_t H, int64_t W,
+                               int64_t groups, float eps, int act, kop_dtype_t dtype, kop_stream_t stream);
+
+/*
+ * Diagnostic for kop_groupnorm_act (no counterpart in the paper): its staged kernel waits for its bulk
+ * copies with a bounded number of polls; a CTA whose wait runs out writes nothing, and counts itself here.
+ * host_count: HOST pointer, receives the count for the current device since the library was loaded (always
+ * 0 on healthy hardware). Blocks until the device is idle (a synchronous copy); not for hot paths.
+ */
+kop_status_t kop_groupnorm_wait_timeouts(unsigned int* host_count);
+
+/*
  * Transformer MLP segment with the vendor GEMMs preserved between the fused kernels
  * (problem formulation: extern library calls stay fixed; codegen agent: "do not
  * replace cuBLAS"): five operations enqueued on `stream`,

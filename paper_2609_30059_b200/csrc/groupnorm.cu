@@ -1,0 +1,521 @@
+// kop_groupnorm_act: GroupNorm (InstanceNorm when groups == C) with optional per-channel affine and an
+// activation, NCHW, in one HBM pass.
+//
+// A CTA owns one (image, group) chunk: (C / groups) * H * W contiguous elements. The chunk is far too
+// long for registers (100 KB for 8 channels of 56x56 fp32) but fits the 227 KB of shared memory a
+// Blackwell CTA can have, so the chunk is fetched into shared memory once (bulk asynchronous copies
+// requested up front), the statistics are accumulated as the parts land, and the normalising sweep
+// re-reads the chunk from shared memory instead of HBM.
+// Mean and variance come from one sweep without the E[x^2] - mean^2 cancellation: every thread keeps
+// a (count, mean, M2) triple, updated per batch of vectors with an exact two-sweep computation over
+// the batch held in registers and merged with the pairwise (Chan) formula; triples are merged across
+// the CTA the same way. Chunks beyond the shared-memory budget take two sweeps over global memory
+// (the second mostly from L2).
+#include "kop_common.cuh"
+
+#include <atomic>
+
+namespace kop {
+namespace {
+
+struct Moments {
+    float n, mean, m2;
+};
+
+// Pairwise merge: delta = mean_b - mean_a; mean = mean_a + delta n_b / n; M2 = M2_a + M2_b + delta^2 n_a n_b / n.
+__device__ __forceinline__ Moments merge(Moments a, Moments b)
+{
+    const float n = a.n + b.n;
+    if (n == 0.0f) return Moments{0.0f, 0.0f, 0.0f};
+    const float f = b.n / n;
+    const float d = b.mean - a.mean;
+    return Moments{n, fmaf(d, f, a.mean), a.m2 + b.m2 + d * d * a.n * f};
+}
+
+__device__ __forceinline__ Moments warp_merge(Moments m)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        Moments other;
+        other.n = __shfl_xor_sync(0xFFFFFFFFu, m.n, o);
+        other.mean = __shfl_xor_sync(0xFFFFFFFFu, m.mean, o);
+        other.m2 = __shfl_xor_sync(0xFFFFFFFFu, m.m2, o);
+        // both lanes of a pair must combine in the same order to agree bit for bit
+        const bool low = (threadIdx.x & o) == 0;
+        m = low ? merge(m, other) : merge(other, m);
+    }
+    return m;
+}
+
+enum { kActNone = 0, kActRelu = 1, kActSilu = 2 };
+
+// SiLU through ex2.approx and rcp.approx: about 3e-7 relative error, far inside the fp32 gate of 1e-5,
+// and a third of the instructions of an IEEE division (this kernel is close to issue-bound on fp32 data).
+template <int ACT>
+__device__ __forceinline__ float activate(float v)
+{
+    if (ACT == kActRelu) return v > 0.0f ? v : (v <= 0.0f ? 0.0f : v);       // NaN passes through
+    if (ACT == kActSilu) return v * rcp_approx(1.0f + ex2_approx(-v * kLog2e));
+    return v;
+}
+
+// v / d for 0 <= v < 2^22 without the 20-instruction integer division: float estimate, one-step fix-up.
+__device__ __forceinline__ int div_small(int v, int d, float inv_d)
+{
+    int q = (int)((float)v * inv_d);
+    const int r = v - q * d;
+    q += (r >= d) ? 1 : 0;
+    q -= (r < 0) ? 1 : 0;
+    return q;
+}
+
+constexpr int kGnThreads = 512;
+constexpr int kGnUnroll = 4;
+constexpr int kGnPartVecs = kGnUnroll * kGnThreads;      // 32 KB: one bulk copy, one barrier, one trip
+constexpr int kGnMaxParts = 7;                           // covers the 200 KB staging budget
+
+// Moments of up to kGnUnroll vectors held in registers (exact two-sweep), merged into `acc`.
+// Slots k >= cnt hold zeros: they add nothing to the sum and are skipped in the second sweep.
+template <typename T>
+__device__ __forceinline__ void accumulate_batch(const Vec16 (&raw)[kGnUnroll], int cnt, Moments& acc)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    if (cnt == 0) return;
+    float f[kGnUnroll][E];
+    float s = 0.0f;
+#pragma unroll
+    for (int k = 0; k < kGnUnroll; ++k) {
+        Elem<T>::unpack(raw[k], f[k]);
+#pragma unroll
+        for (int e = 0; e < E; ++e) s += f[k][e];
+    }
+    const float bn = (float)(cnt * E);
+    const float bmean = s / bn;
+    float m2 = 0.0f;
+#pragma unroll
+    for (int k = 0; k < kGnUnroll; ++k) {
+        if (k < cnt) {
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                const float d = f[k][e] - bmean;
+                m2 = fmaf(d, d, m2);
+            }
+        }
+    }
+    acc = merge(acc, Moments{bn, bmean, m2});
+}
+
+// CTA-wide merge in a fixed order (lanes by butterfly, warps by index); thread 0 of warp 0 publishes
+// mean and rstd. `ok` is and-reduced over the CTA by the same barrier and returned.
+struct GnShared {
+    float n[32], mean[32], m2[32];
+    float bc_mean, bc_rstd;
+};
+
+__device__ __forceinline__ bool cta_moments(Moments acc, GnShared& sh, float eps, float* mean, float* rstd,
+                                            int64_t chunk, bool ok, float& mu, float& rs)
+{
+    acc = warp_merge(acc);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    if (lane == 0) {
+        sh.n[warp] = acc.n;
+        sh.mean[warp] = acc.mean;
+        sh.m2[warp] = acc.m2;
+    }
+    const bool all_ok = __syncthreads_and(ok) != 0;
+    if (warp == 0) {
+        Moments t = lane < nw ? Moments{sh.n[lane], sh.mean[lane], sh.m2[lane]} : Moments{0.0f, 0.0f, 0.0f};
+        t = warp_merge(t);
+        if (lane == 0) {
+            const float r = rsqrtf(t.m2 / t.n + eps);
+            sh.bc_mean = t.mean;
+            sh.bc_rstd = r;
+            if (all_ok) {
+                if (mean != nullptr) mean[chunk] = t.mean;
+                if (rstd != nullptr) rstd[chunk] = r;
+            }
+        }
+    }
+    __syncthreads();
+    mu = sh.bc_mean;
+    rs = sh.bc_rstd;
+    return all_ok;
+}
+
+// y = act((x - mu) * rstd * gamma[c] + beta[c]) for one vector; a vector never straddles two channels.
+template <typename T, int ACT>
+__device__ __forceinline__ void normalize_store(const Vec16& raw, T* dst, int c, const float* gamma,
+                                                const float* beta, float mu, float rs)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    const float sc = rs * (gamma != nullptr ? __ldg(gamma + c) : 1.0f);
+    const float be = beta != nullptr ? __ldg(beta + c) : 0.0f;
+    float f[E];
+    Elem<T>::unpack(raw, f);
+    // (x - mu) first: folding mu into a shift would cost |mu| * rstd ulps when the spread is small
+#pragma unroll
+    for (int e = 0; e < E; ++e) f[e] = activate<ACT>(fmaf(f[e] - mu, sc, be));
+    st_stream(dst, Elem<T>::pack(f));
+}
+
+// Chunks beyond the staging budget: two sweeps over global memory (the second mostly served by L2).
+// Self-contained on purpose (it shares only merge / warp_merge / activate with the staged kernel).
+template <typename T, int ACT>
+__global__ void __launch_bounds__(kGnThreads)
+groupnorm_twosweep_kernel(const T* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
+                          T* __restrict__ y, float* __restrict__ mean, float* __restrict__ rstd, int nvec,
+                          int vec_per_plane, int cpg, int groups, float eps)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    __shared__ float red_n[32], red_mean[32], red_m2[32];
+    __shared__ float bc_mean, bc_rstd;
+
+    const int64_t chunk = blockIdx.x;                       // image * groups + group
+    const int g = (int)(chunk % groups);
+    const T* xc = x + chunk * (int64_t)nvec * E;
+    T* yc = y + chunk * (int64_t)nvec * E;
+
+    Moments acc{0.0f, 0.0f, 0.0f};
+    for (int base = 0; base < nvec; base += kGnUnroll * kGnThreads) {
+        Vec16 raw[kGnUnroll];
+        int cnt = 0;
+#pragma unroll
+        for (int k = 0; k < kGnUnroll; ++k) {
+            const int v = base + k * kGnThreads + threadIdx.x;
+            if (v < nvec) {
+                raw[k] = ld_stream(xc + (int64_t)v * E);
+                ++cnt;
+            } else {
+                raw[k] = Vec16{{0u, 0u, 0u, 0u}};
+            }
+        }
+        if (cnt > 0) {
+            // exact two-sweep moments of this batch (zero padding adds 0 to the sum and is masked below)
+            float f[kGnUnroll][E];
+            float s = 0.0f;
+#pragma unroll
+            for (int k = 0; k < kGnUnroll; ++k) {
+                Elem<T>::unpack(raw[k], f[k]);
+#pragma unroll
+                for (int e = 0; e < E; ++e) s += f[k][e];
+            }
+            const float bn = (float)(cnt * E);
+            const float bmean = s / bn;
+            float m2 = 0.0f;
+#pragma unroll
+            for (int k = 0; k < kGnUnroll; ++k) {
+                if (k < cnt) {
+#pragma unroll
+                    for (int e = 0; e < E; ++e) {
+                        const float d = f[k][e] - bmean;
+                        m2 = fmaf(d, d, m2);
+                    }
+                }
+            }
+            acc = merge(acc, Moments{bn, bmean, m2});
+        }
+    }
+    // CTA-wide merge in a fixed order: lanes by butterfly, warps by index
+    acc = warp_merge(acc);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) {
+        red_n[warp] = acc.n;
+        red_mean[warp] = acc.mean;
+        red_m2[warp] = acc.m2;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        constexpr int NW = kGnThreads / 32;
+        Moments t = lane < NW ? Moments{red_n[lane], red_mean[lane], red_m2[lane]} : Moments{0.0f, 0.0f, 0.0f};
+        t = warp_merge(t);
+        if (lane == 0) {
+            const float rs = rsqrtf(t.m2 / t.n + eps);
+            bc_mean = t.mean;
+            bc_rstd = rs;
+            if (mean != nullptr) mean[chunk] = t.mean;
+            if (rstd != nullptr) rstd[chunk] = rs;
+        }
+    }
+    __syncthreads();
+    const float mu = bc_mean, rs = bc_rstd;
+
+    for (int base = 0; base < nvec; base += kGnUnroll * kGnThreads) {
+        Vec16 raw[kGnUnroll];
+#pragma unroll
+        for (int k = 0; k < kGnUnroll; ++k) {
+            const int v = base + k * kGnThreads + threadIdx.x;
+            if (v < nvec) raw[k] = ld_stream(xc + (int64_t)v * E);
+        }
+#pragma unroll
+        for (int k = 0; k < kGnUnroll; ++k) {
+            const int v = base + k * kGnThreads + threadIdx.x;
+            if (v < nvec) {
+                const int c = g * cpg + v / vec_per_plane;           // a vector never straddles two channels
+                const float ga = gamma != nullptr ? __ldg(gamma + c) : 1.0f;
+                const float be = beta != nullptr ? __ldg(beta + c) : 0.0f;
+                const float sc = rs * ga;
+                float f[E];
+                Elem<T>::unpack(raw[k], f);
+                // (x - mu) first: folding mu into a shift would cost |mu| * rstd ulps when the spread is small
+#pragma unroll
+                for (int e = 0; e < E; ++e) f[e] = activate<ACT>(fmaf(f[e] - mu, sc, be));
+                st_stream(yc + (int64_t)v * E, Elem<T>::pack(f));
+            }
+        }
+    }
+}
+
+// ---- staged kernel: the chunk is fetched into shared memory by bulk asynchronous copies --------------
+// One thread requests the whole chunk up front as 32 KB copies (cp.async.bulk, global -> shared), each
+// completing on its own mbarrier, so the CTA has its entire input in flight from its first cycles and
+// the memory system, not the loop structure, sets the pace. All threads then consume the parts in
+// order (moments from shared memory as each part lands), merge, and normalise out of shared memory.
+__device__ unsigned int g_gn_wait_timeouts;              // CTAs that gave up waiting for a copy
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
+{
+    uint32_t done;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(done)
+        : "r"(smem_addr(bar)), "r"(parity)
+        : "memory");
+    return done != 0;
+}
+
+// Bounded wait: a copy that never lands (it cannot, short of a hardware fault) must not hang the GPU.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity)
+{
+    for (int spin = 0; spin < (1 << 22); ++spin)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+
+__device__ __forceinline__ void bulk_load(void* dst_smem, const void* src, uint32_t bytes, uint64_t* bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_addr(dst_smem)),
+                 "l"(src), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
+}
+
+template <typename T, int ACT>
+__global__ void __launch_bounds__(kGnThreads)
+groupnorm_staged_kernel(const T* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
+                        T* __restrict__ y, float* __restrict__ mean, float* __restrict__ rstd, int nvec,
+                        int vec_per_plane, int cpg, int groups, float eps)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    extern __shared__ __align__(128) unsigned char gn_smem[];
+    Vec16* stage = reinterpret_cast<Vec16*>(gn_smem);
+    __shared__ GnShared sh;
+    __shared__ __align__(8) uint64_t bars[kGnMaxParts];
+
+    const int64_t chunk = blockIdx.x;                       // image * groups + group
+    const int g = (int)(chunk % groups);
+    const T* xc = x + chunk * (int64_t)nvec * E;
+    T* yc = y + chunk * (int64_t)nvec * E;
+    const int nparts = (nvec + kGnPartVecs - 1) / kGnPartVecs;      // <= kGnMaxParts by the launch rule
+
+    if (threadIdx.x == 0) {
+        for (int p = 0; p < nparts; ++p) mbar_init(bars + p, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        for (int p = 0; p < nparts; ++p) {
+            const int v0 = p * kGnPartVecs;
+            const uint32_t bytes = (uint32_t)min(kGnPartVecs, nvec - v0) * 16u;
+            mbar_expect_tx(bars + p, bytes);
+            bulk_load(stage + v0, xc + (int64_t)v0 * E, bytes, bars + p);
+        }
+    }
+    __syncthreads();                                        // barriers initialised before anyone polls them
+
+    Moments acc{0.0f, 0.0f, 0.0f};
+    bool ok = true;
+    for (int p = 0; p < nparts; ++p) {
+        ok = mbar_wait_bounded(bars + p, 0) && ok;
+        Vec16 raw[kGnUnroll];
+        int cnt = 0;
+#pragma unroll
+        for (int k = 0; k < kGnUnroll; ++k) {
+            const int v = p * kGnPartVecs + k * kGnThreads + threadIdx.x;
+            if (v < nvec) {
+                raw[k] = stage[v];
+                ++cnt;
+            } else {
+                raw[k] = Vec16{{0u, 0u, 0u, 0u}};
+            }
+        }
+        accumulate_batch<T>(raw, cnt, acc);
+    }
+    float mu, rs;
+    if (!cta_moments(acc, sh, eps, mean, rstd, chunk, ok, mu, rs)) {
+        // give the copies one more bounded chance to drain before this CTA's shared memory is released
+        for (int p = 0; p < nparts; ++p) mbar_wait_bounded(bars + p, 0);
+        if (threadIdx.x == 0) atomicAdd(&g_gn_wait_timeouts, 1u);
+        return;
+    }
+    const float inv_vpp = 1.0f / (float)vec_per_plane;
+    for (int base = 0; base < nvec; base += kGnPartVecs) {
+#pragma unroll
+        for (int k = 0; k < kGnUnroll; ++k) {
+            const int v = base + k * kGnThreads + threadIdx.x;
+            if (v < nvec)
+                normalize_store<T, ACT>(stage[v], yc + (int64_t)v * E, g * cpg + div_small(v, vec_per_plane, inv_vpp),
+                                        gamma, beta, mu, rs);
+        }
+    }
+}
+
+// Any plane size / alignment: scalar loads, two sweeps over global memory, same moment arithmetic.
+template <typename T, int ACT>
+__global__ void __launch_bounds__(256)
+groupnorm_scalar_kernel(const T* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
+                        T* __restrict__ y, float* __restrict__ mean, float* __restrict__ rstd,
+                        int64_t chunk_elems, int64_t plane, int cpg, int groups, float eps)
+{
+    __shared__ float red_n[32], red_mean[32], red_m2[32];
+    __shared__ float bc_mean, bc_rstd;
+    const int64_t chunk = blockIdx.x;
+    const int g = (int)(chunk % groups);
+    const T* xc = x + chunk * chunk_elems;
+    T* yc = y + chunk * chunk_elems;
+    Moments acc{0.0f, 0.0f, 0.0f};
+    for (int64_t j = threadIdx.x; j < chunk_elems; j += blockDim.x)
+        acc = merge(acc, Moments{1.0f, Elem<T>::load1(xc + j), 0.0f});
+    acc = warp_merge(acc);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    if (lane == 0) {
+        red_n[warp] = acc.n;
+        red_mean[warp] = acc.mean;
+        red_m2[warp] = acc.m2;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        Moments t = lane < nw ? Moments{red_n[lane], red_mean[lane], red_m2[lane]} : Moments{0.0f, 0.0f, 0.0f};
+        t = warp_merge(t);
+        if (lane == 0) {
+            const float rs = rsqrtf(t.m2 / t.n + eps);
+            bc_mean = t.mean;
+            bc_rstd = rs;
+            if (mean != nullptr) mean[chunk] = t.mean;
+            if (rstd != nullptr) rstd[chunk] = rs;
+        }
+    }
+    __syncthreads();
+    const float mu = bc_mean, rs = bc_rstd;
+    for (int64_t j = threadIdx.x; j < chunk_elems; j += blockDim.x) {
+        const int c = g * cpg + (int)(j / plane);
+        const float sc = rs * (gamma != nullptr ? __ldg(gamma + c) : 1.0f);
+        const float be = beta != nullptr ? __ldg(beta + c) : 0.0f;
+        Elem<T>::store1(yc + j, activate<ACT>(fmaf(Elem<T>::load1(xc + j) - mu, sc, be)));
+    }
+}
+
+constexpr size_t kGnStageLimit = 200 * 1024;     // leaves room for the static reduction slots
+static_assert(kGnStageLimit <= (size_t)kGnMaxParts * kGnPartVecs * 16, "one barrier per 32 KB part");
+constexpr int kMaxDevices = 64;
+
+template <typename T, int ACT>
+kop_status_t launch_gn_act(const T* x, const float* gamma, const float* beta, T* y, float* mean, float* rstd,
+                           int64_t chunks, int64_t chunk_elems, int64_t plane, int cpg, int groups, float eps,
+                           cudaStream_t stream)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    const bool vec = aligned_to(x, 16) && aligned_to(y, 16) && (plane % E) == 0 && chunk_elems / E <= 0x7FFFFFFF;
+    if (vec) {
+        const int nvec = (int)(chunk_elems / E);
+        const int vpp = (int)(plane / E);
+        const size_t bytes = (size_t)nvec * 16;
+        if (bytes <= kGnStageLimit) {
+            // the opt-in above 48 KB is per function and per device; one flag per template instance
+            static std::atomic<bool> configured[kMaxDevices];
+            int dev = 0;
+            if (cudaGetDevice(&dev) != cudaSuccess) return KOP_ERR_CUDA;
+            if (dev < 0 || dev >= kMaxDevices || !configured[dev].load(std::memory_order_acquire)) {
+                if (cudaFuncSetAttribute(groupnorm_staged_kernel<T, ACT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)kGnStageLimit) != cudaSuccess)
+                    return KOP_ERR_CUDA;
+                if (dev >= 0 && dev < kMaxDevices) configured[dev].store(true, std::memory_order_release);
+            }
+            groupnorm_staged_kernel<T, ACT><<<(unsigned)chunks, kGnThreads, bytes, stream>>>(
+                x, gamma, beta, y, mean, rstd, nvec, vpp, cpg, groups, eps);
+        } else {
+            groupnorm_twosweep_kernel<T, ACT><<<(unsigned)chunks, kGnThreads, 0, stream>>>(
+                x, gamma, beta, y, mean, rstd, nvec, vpp, cpg, groups, eps);
+        }
+        return launch_status();
+    }
+    groupnorm_scalar_kernel<T, ACT><<<(unsigned)chunks, 256, 0, stream>>>(x, gamma, beta, y, mean, rstd, chunk_elems,
+                                                                          plane, cpg, groups, eps);
+    return launch_status();
+}
+
+template <typename T>
+kop_status_t launch_gn(const void* x, const float* gamma, const float* beta, void* y, float* mean, float* rstd,
+                       int64_t chunks, int64_t chunk_elems, int64_t plane, int cpg, int groups, float eps, int act,
+                       cudaStream_t stream)
+{
+    const T* xt = static_cast<const T*>(x);
+    T* yt = static_cast<T*>(y);
+    switch (act) {
+    case kActRelu: return launch_gn_act<T, kActRelu>(xt, gamma, beta, yt, mean, rstd, chunks, chunk_elems, plane, cpg, groups, eps, stream);
+    case kActSilu: return launch_gn_act<T, kActSilu>(xt, gamma, beta, yt, mean, rstd, chunks, chunk_elems, plane, cpg, groups, eps, stream);
+    default: return launch_gn_act<T, kActNone>(xt, gamma, beta, yt, mean, rstd, chunks, chunk_elems, plane, cpg, groups, eps, stream);
+    }
+}
+
+}  // namespace
+}  // namespace kop
+
+extern "C" kop_status_t kop_groupnorm_act(const void* x, const float* gamma, const float* beta, void* y,
+                                          float* mean, float* rstd, int64_t N, int64_t C, int64_t H, int64_t W,
+                                          int64_t groups, float eps, int act, kop_dtype_t dtype,
+                                          kop_stream_t stream)
+{
+    using namespace kop;
+    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    if (N < 0 || C <= 0 || H <= 0 || W <= 0 || groups <= 0 || groups > C || C % groups != 0) return KOP_ERR_BAD_SHAPE;
+    if (act < 0 || act > 2 || !(eps >= 0.0f)) return KOP_ERR_BAD_SHAPE;
+    if (C > 0x7FFFFFFF || H > kMaxElems || W > kMaxElems || N > kMaxElems || H > kMaxElems / W) return KOP_ERR_BAD_SHAPE;
+    const int64_t plane = H * W;
+    if (C > kMaxElems / plane) return KOP_ERR_BAD_SHAPE;
+    if (N == 0) return KOP_OK;
+    if (C * plane > kMaxElems / N) return KOP_ERR_BAD_SHAPE;
+    if (N * groups > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;           // one CTA per (image, group)
+    if (!x || !y) return KOP_ERR_NULL_POINTER;
+    const int esz = elem_size(dtype);
+    if (!aligned_to(x, esz) || !aligned_to(y, esz) || (gamma && !aligned_to(gamma, 4)) ||
+        (beta && !aligned_to(beta, 4)) || (mean && !aligned_to(mean, 4)) || (rstd && !aligned_to(rstd, 4)))
+        return KOP_ERR_MISALIGNED;
+    if (!alias_ok(x, C * plane, y, C * plane, N, C * plane, esz, true)) return KOP_ERR_BAD_ALIAS;
+    kop_status_t st = check_device();
+    if (st != KOP_OK) return st;
+    const int cpg = (int)(C / groups);
+    const int64_t chunk_elems = (int64_t)cpg * plane;
+    cudaStream_t s = as_stream(stream);
+    return dtype == KOP_F32
+               ? launch_gn<float>(x, gamma, beta, y, mean, rstd, N * groups, chunk_elems, plane, cpg, (int)groups, eps, act, s)
+               : launch_gn<__nv_bfloat16>(x, gamma, beta, y, mean, rstd, N * groups, chunk_elems, plane, cpg, (int)groups, eps, act, s);
+}
+
+extern "C" kop_status_t kop_groupnorm_wait_timeouts(unsigned int* host_count)
+{
+    using namespace kop;
+    if (!host_count) return KOP_ERR_NULL_POINTER;
+    kop_status_t st = check_device();
+    if (st != KOP_OK) return st;
+    return cudaMemcpyFromSymbol(host_count, g_gn_wait_timeouts, sizeof(unsigned int)) == cudaSuccess ? KOP_OK
+                                                                                                      : KOP_ERR_CUDA;
+}

@@ -74,6 +74,10 @@ def lib() -> C.CDLL:
     L.kop_row_scale.restype = i32
     L.kop_matvec_bias.argtypes = [vp, vp, f32, vp, i64, i64, i64, i32, vp]
     L.kop_matvec_bias.restype = i32
+    L.kop_groupnorm_act.argtypes = [vp] * 6 + [i64] * 5 + [f32, i32, i32, vp]
+    L.kop_groupnorm_act.restype = i32
+    L.kop_groupnorm_wait_timeouts.argtypes = [C.POINTER(C.c_uint)]
+    L.kop_groupnorm_wait_timeouts.restype = i32
     L.kop_rmsnorm_swiglu_residual.argtypes = [vp] * 6 + [i64] * 3 + [f32, vp, sz, i32, vp]
     L.kop_rmsnorm_swiglu_residual_workspace_bytes.restype = sz
     L.kop_rmsnorm_swiglu_residual_workspace_bytes.argtypes = [i64, i64, i64, i32]
@@ -319,6 +323,31 @@ def kop_matvec_bias(x, w, b_sum, out=None, stream=None):
     _check(lib().kop_matvec_bias(x.data_ptr(), _param(w, "w", k), float(b_sum), out.data_ptr(), rows, k, xs,
                                  _dtype_tag(x), _stream(stream)), "kop_matvec_bias")
     return out
+
+
+def kop_groupnorm_act(x, gamma, beta, groups, eps, act=0, out=None, mean=None, rstd=None, want_stats=True,
+                      stream=None):
+    """act: 0 identity, 1 ReLU, 2 SiLU. groups == C is InstanceNorm. Returns (y, mean[N, groups], rstd[N, groups])."""
+    if x.dim() != 4 or not x.is_cuda or not x.is_contiguous():
+        raise ValueError("x: expected a contiguous 4-D NCHW CUDA tensor")
+    N, Cc, H, W = x.shape
+    out = torch.empty_like(x) if out is None else out
+    if out.shape != x.shape or out.dtype != x.dtype or not out.is_contiguous():
+        raise ValueError("out: expected a contiguous tensor of x's shape and dtype")
+    if want_stats:
+        mean = torch.empty((N, groups), dtype=torch.float32, device=x.device) if mean is None else mean
+        rstd = torch.empty((N, groups), dtype=torch.float32, device=x.device) if rstd is None else rstd
+    _check(lib().kop_groupnorm_act(x.data_ptr(), _param(gamma, "gamma", Cc), _param(beta, "beta", Cc),
+                                   out.data_ptr(), None if mean is None else mean.data_ptr(),
+                                   None if rstd is None else rstd.data_ptr(), N, Cc, H, W, int(groups),
+                                   float(eps), int(act), _dtype_tag(x), _stream(stream)), "kop_groupnorm_act")
+    return out, mean, rstd
+
+
+def kop_groupnorm_wait_timeouts() -> int:
+    n = C.c_uint(0)
+    _check(lib().kop_groupnorm_wait_timeouts(C.byref(n)), "kop_groupnorm_wait_timeouts")
+    return int(n.value)
 
 
 class MlpHandle:

@@ -22,6 +22,8 @@ CONFIGS = {
     # beyond the five benchmark configs: the two kernels the paper's case studies print
     "row_scale": dict(rows=4096, cols=4096, dtype=torch.float32),          # the paper's 4096 x 4096 shape
     "matvec_bias": dict(rows=32768, k=4096, dtype=torch.bfloat16),         # shape not given in the paper
+    # GroupNorm + SiLU as in a diffusion U-Net residual block: 32 groups over 256 channels of a 56 x 56 map
+    "groupnorm": dict(N=64, C=256, H=56, W=56, groups=32, dtype=torch.float32, eps=1e-5, act=2),
 }
 
 
@@ -115,3 +117,15 @@ def matvec_inputs(rows, k, dtype=torch.bfloat16, seed=0, device="cpu"):
     w = _normal((k,), 0.0, 0.16, g, device)
     b_sum = _normal((1,), 0.0, 0.8, g, device)
     return x, w, float(b_sum.item())
+
+
+def groupnorm_inputs(N, C, H, W, dtype=torch.float32, seed=0, device="cpu"):
+    """x NCHW with a per-channel offset and spread (x = m_c + s_c * N(0,1), m_c ~ N(0,1), s_c ~ U(0.5,2)), so the
+    groups have non-zero means; gamma ~ N(1,0.02); beta ~ N(0,0.02) (params fp32)."""
+    g = _gen(seed, device)
+    m = _normal((1, C, 1, 1), 0.0, 1.0, g, device)
+    s = _uniform((1, C, 1, 1), 0.5, 2.0, g, device)
+    x = (_normal((N, C, H, W), 0.0, 1.0, g, device) * s + m).to(dtype)
+    gamma = _normal((C,), 1.0, 0.02, g, device)
+    beta = _normal((C,), 0.0, 0.02, g, device)
+    return x, gamma, beta

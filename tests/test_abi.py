@@ -158,6 +158,29 @@ def test_row_ops_validation(L):
     assert L.kop_matvec_bias(P, Q + 2, 0.5, R, 4, 64, 64, 1, None) == MISAL
 
 
+def test_groupnorm_validation(L):
+    f = L.kop_groupnorm_act
+    G, B, M, S = 0x600000, 0x610000, 0x620000, 0x630000
+    ok = (P, G, B, Q, M, S)
+    assert f(*ok, 0, 8, 4, 4, 2, 1e-5, 0, 0, None) == OK                       # empty batch: no CUDA call
+    assert f(None, G, B, Q, M, S, 2, 8, 4, 4, 2, 1e-5, 0, 0, None) == NULLP
+    assert f(P, G, B, None, M, S, 2, 8, 4, 4, 2, 1e-5, 0, 0, None) == NULLP
+    assert f(*ok, 2, 8, 4, 4, 3, 1e-5, 0, 0, None) == SHAPE                    # groups must divide C
+    assert f(*ok, 2, 8, 4, 4, 0, 1e-5, 0, 0, None) == SHAPE
+    assert f(*ok, 2, 8, 4, 4, 16, 1e-5, 0, 0, None) == SHAPE
+    assert f(*ok, 2, 8, 0, 4, 2, 1e-5, 0, 0, None) == SHAPE
+    assert f(*ok, -1, 8, 4, 4, 2, 1e-5, 0, 0, None) == SHAPE
+    assert f(*ok, 2, 8, 4, 4, 2, 1e-5, 3, 0, None) == SHAPE                    # unknown activation
+    assert f(*ok, 2, 8, 4, 4, 2, -1.0, 0, 0, None) == SHAPE                    # negative eps
+    assert f(*ok, 2, 8, 4, 4, 2, float("nan"), 0, 0, None) == SHAPE
+    assert f(*ok, 2, 8, 4, 4, 2, 1e-5, 0, 5, None) == DTYPE
+    assert f(P + 2, G, B, Q, M, S, 2, 8, 4, 4, 2, 1e-5, 0, 0, None) == MISAL
+    assert f(P, G + 2, B, Q, M, S, 2, 8, 4, 4, 2, 1e-5, 0, 0, None) == MISAL
+    assert f(P, G, B, Q, M + 1, S, 2, 8, 4, 4, 2, 1e-5, 0, 0, None) == MISAL
+    assert f(P, G, B, P + 64, M, S, 2, 8, 4, 4, 2, 1e-5, 0, 0, None) == ALIAS  # partial overlap of x and y
+    assert L.kop_groupnorm_wait_timeouts(None) == NULLP
+
+
 def test_mlp_driver_validation(L):
     f = L.kop_rmsnorm_swiglu_residual
     wsb = L.kop_rmsnorm_swiglu_residual_workspace_bytes(16, 64, 128, 1)
