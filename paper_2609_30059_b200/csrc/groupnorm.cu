@@ -6,13 +6,14 @@
 // Blackwell CTA can have, so the chunk is fetched into shared memory once (bulk asynchronous copies
 // requested up front), the statistics are accumulated as the parts land, and the normalising sweep
 // re-reads the chunk from shared memory instead of HBM.
-// Mean and variance come from one sweep without the E[x^2] - mean^2 cancellation: every thread keeps
-// a (count, mean, M2) triple, updated per batch of vectors with an exact two-sweep computation over
-// the batch held in registers and merged with the pairwise (Chan) formula; triples are merged across
-// the CTA the same way. Chunks beyond the shared-memory budget take two sweeps over global memory
-// (the second mostly from L2).
+// With the chunk on chip the statistics are the exact two-pass ones (mean, then squared deviations from
+// it). Chunks beyond the shared-memory budget take two sweeps over global memory (the second mostly from
+// L2); there, and in the scalar kernel, mean and variance come from one sweep without the
+// E[x^2] - mean^2 cancellation: every thread keeps a (count, mean, M2) triple, updated per batch with an
+// exact two-sweep computation in registers and merged with the pairwise (Chan) formula.
 #include "kop_common.cuh"
 
+#include <algorithm>
 #include <atomic>
 
 namespace kop {
@@ -71,91 +72,34 @@ __device__ __forceinline__ int div_small(int v, int d, float inv_d)
 
 constexpr int kGnThreads = 512;
 constexpr int kGnUnroll = 4;
-constexpr int kGnPartVecs = kGnUnroll * kGnThreads;      // 32 KB: one bulk copy, one barrier, one trip
+constexpr int kGnCopyVecs = 2048;                        // 32 KB: one bulk copy, one barrier
 constexpr int kGnMaxParts = 7;                           // covers the 200 KB staging budget
 
-// Moments of up to kGnUnroll vectors held in registers (exact two-sweep), merged into `acc`.
-// Slots k >= cnt hold zeros: they add nothing to the sum and are skipped in the second sweep.
-template <typename T>
-__device__ __forceinline__ void accumulate_batch(const Vec16 (&raw)[kGnUnroll], int cnt, Moments& acc)
-{
-    constexpr int E = Elem<T>::kPerVec;
-    if (cnt == 0) return;
-    float f[kGnUnroll][E];
-    float s = 0.0f;
-#pragma unroll
-    for (int k = 0; k < kGnUnroll; ++k) {
-        Elem<T>::unpack(raw[k], f[k]);
-#pragma unroll
-        for (int e = 0; e < E; ++e) s += f[k][e];
-    }
-    const float bn = (float)(cnt * E);
-    const float bmean = s / bn;
-    float m2 = 0.0f;
-#pragma unroll
-    for (int k = 0; k < kGnUnroll; ++k) {
-        if (k < cnt) {
-#pragma unroll
-            for (int e = 0; e < E; ++e) {
-                const float d = f[k][e] - bmean;
-                m2 = fmaf(d, d, m2);
-            }
-        }
-    }
-    acc = merge(acc, Moments{bn, bmean, m2});
-}
-
-// CTA-wide merge in a fixed order (lanes by butterfly, warps by index); thread 0 of warp 0 publishes
-// mean and rstd. `ok` is and-reduced over the CTA by the same barrier and returned.
-struct GnShared {
-    float n[32], mean[32], m2[32];
-    float bc_mean, bc_rstd;
-};
-
-__device__ __forceinline__ bool cta_moments(Moments acc, GnShared& sh, float eps, float* mean, float* rstd,
-                                            int64_t chunk, bool ok, float& mu, float& rs)
-{
-    acc = warp_merge(acc);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
-    if (lane == 0) {
-        sh.n[warp] = acc.n;
-        sh.mean[warp] = acc.mean;
-        sh.m2[warp] = acc.m2;
-    }
-    const bool all_ok = __syncthreads_and(ok) != 0;
-    if (warp == 0) {
-        Moments t = lane < nw ? Moments{sh.n[lane], sh.mean[lane], sh.m2[lane]} : Moments{0.0f, 0.0f, 0.0f};
-        t = warp_merge(t);
-        if (lane == 0) {
-            const float r = rsqrtf(t.m2 / t.n + eps);
-            sh.bc_mean = t.mean;
-            sh.bc_rstd = r;
-            if (all_ok) {
-                if (mean != nullptr) mean[chunk] = t.mean;
-                if (rstd != nullptr) rstd[chunk] = r;
-            }
-        }
-    }
-    __syncthreads();
-    mu = sh.bc_mean;
-    rs = sh.bc_rstd;
-    return all_ok;
-}
-
 // y = act((x - mu) * rstd * gamma[c] + beta[c]) for one vector; a vector never straddles two channels.
+// (x - mu) first: folding mu into a shift would cost |mu| * rstd ulps when the spread is small.
 template <typename T, int ACT>
 __device__ __forceinline__ void normalize_store(const Vec16& raw, T* dst, int c, const float* gamma,
                                                 const float* beta, float mu, float rs)
 {
-    constexpr int E = Elem<T>::kPerVec;
+    constexpr int P = Elem<T>::kPerVec / 2;
     const float sc = rs * (gamma != nullptr ? __ldg(gamma + c) : 1.0f);
     const float be = beta != nullptr ? __ldg(beta + c) : 0.0f;
-    float f[E];
-    Elem<T>::unpack(raw, f);
-    // (x - mu) first: folding mu into a shift would cost |mu| * rstd ulps when the spread is small
+    const float2 nmu = make_float2(-mu, -mu), sc2 = make_float2(sc, sc), be2 = make_float2(be, be);
+    float2 f[P];
+    Elem<T>::unpack2(raw, f);
 #pragma unroll
-    for (int e = 0; e < E; ++e) f[e] = activate<ACT>(fmaf(f[e] - mu, sc, be));
-    st_stream(dst, Elem<T>::pack(f));
+    for (int e = 0; e < P; ++e) {
+        float2 u = __ffma2_rn(__fadd2_rn(f[e], nmu), sc2, be2);
+        if (ACT == kActSilu) {
+            const float2 a = __fmul2_rn(u, make_float2(-kLog2e, -kLog2e));
+            const float2 d = __fadd2_rn(make_float2(ex2_approx(a.x), ex2_approx(a.y)), make_float2(1.0f, 1.0f));
+            u = __fmul2_rn(u, make_float2(rcp_approx(d.x), rcp_approx(d.y)));
+        } else {
+            u = make_float2(activate<ACT>(u.x), activate<ACT>(u.y));
+        }
+        f[e] = u;
+    }
+    st_stream(dst, Elem<T>::pack2(f));
 }
 
 // Chunks beyond the staging budget: two sweeps over global memory (the second mostly served by L2).
@@ -284,22 +228,25 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes)
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
 }
 
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
+// One poll: the thread is suspended until the phase completes or about `hint_ns` nanoseconds pass, so a
+// waiting warp costs the SM's schedulers next to nothing.
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity, uint32_t hint_ns)
 {
     uint32_t done;
     asm volatile(
-        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
         : "=r"(done)
-        : "r"(smem_addr(bar)), "r"(parity)
+        : "r"(smem_addr(bar)), "r"(parity), "r"(hint_ns)
         : "memory");
     return done != 0;
 }
 
-// Bounded wait: a copy that never lands (it cannot, short of a hardware fault) must not hang the GPU.
+// Bounded wait (at most about two seconds): a copy that never lands (it cannot, short of a hardware
+// fault) must not hang the GPU.
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity)
 {
-    for (int spin = 0; spin < (1 << 22); ++spin)
-        if (mbar_try_wait(bar, parity)) return true;
+    for (int spin = 0; spin < (1 << 18); ++spin)
+        if (mbar_try_wait(bar, parity, 8000u)) return true;
     return false;
 }
 
@@ -311,66 +258,99 @@ __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src, uint3
                  : "memory");
 }
 
-template <typename T, int ACT>
-__global__ void __launch_bounds__(kGnThreads)
+// NT threads per CTA (128, 256 or 512, chosen from the chunk length so short chunks do not pay for idle
+// warps). With the chunk in shared memory the statistics are the textbook two-pass ones: the sum is
+// accumulated part by part as the copies land, the squared deviations from the exact mean in a second
+// sweep over shared memory; both CTA reductions are plain sums (one barrier each, fixed order).
+template <typename T, int ACT, int NT>
+__global__ void __launch_bounds__(NT)
 groupnorm_staged_kernel(const T* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
                         T* __restrict__ y, float* __restrict__ mean, float* __restrict__ rstd, int nvec,
-                        int vec_per_plane, int cpg, int groups, float eps)
+                        int vec_per_plane, int cpg, int groups, float eps, float inv_count)
 {
     constexpr int E = Elem<T>::kPerVec;
+    constexpr int P = E / 2;
+    constexpr int kPartVecs = kGnUnroll * NT;
     extern __shared__ __align__(128) unsigned char gn_smem[];
     Vec16* stage = reinterpret_cast<Vec16*>(gn_smem);
-    __shared__ GnShared sh;
+    __shared__ float slots_a[32], slots_b[32];
     __shared__ __align__(8) uint64_t bars[kGnMaxParts];
 
     const int64_t chunk = blockIdx.x;                       // image * groups + group
     const int g = (int)(chunk % groups);
     const T* xc = x + chunk * (int64_t)nvec * E;
     T* yc = y + chunk * (int64_t)nvec * E;
-    const int nparts = (nvec + kGnPartVecs - 1) / kGnPartVecs;      // <= kGnMaxParts by the launch rule
+    // copies of kGnCopyVecs vectors, one barrier each; kGnMaxParts of them cover the staging budget
+    const int nparts = (nvec + kGnCopyVecs - 1) / kGnCopyVecs;
 
     if (threadIdx.x == 0) {
         for (int p = 0; p < nparts; ++p) mbar_init(bars + p, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         for (int p = 0; p < nparts; ++p) {
-            const int v0 = p * kGnPartVecs;
-            const uint32_t bytes = (uint32_t)min(kGnPartVecs, nvec - v0) * 16u;
+            const int v0 = p * kGnCopyVecs;
+            const uint32_t bytes = (uint32_t)min(kGnCopyVecs, nvec - v0) * 16u;
             mbar_expect_tx(bars + p, bytes);
             bulk_load(stage + v0, xc + (int64_t)v0 * E, bytes, bars + p);
         }
     }
     __syncthreads();                                        // barriers initialised before anyone polls them
 
-    Moments acc{0.0f, 0.0f, 0.0f};
-    bool ok = true;
+    float2 s2 = make_float2(0.0f, 0.0f);
     for (int p = 0; p < nparts; ++p) {
-        ok = mbar_wait_bounded(bars + p, 0) && ok;
-        Vec16 raw[kGnUnroll];
-        int cnt = 0;
+        // One thread polls the copy's barrier; the rest sleep in the CTA barrier instead of burning the
+        // issue slots that co-resident CTAs need for their arithmetic. The vote makes a timeout uniform.
+        bool landed = true;
+        if (threadIdx.x == 0) landed = mbar_wait_bounded(bars + p, 0);
+        if (!__syncthreads_and(landed)) {
+            // give the copies one more bounded chance to drain before this CTA's shared memory is released
+            if (threadIdx.x == 0) {
+                for (int q = p; q < nparts; ++q) mbar_wait_bounded(bars + q, 0);
+                atomicAdd(&g_gn_wait_timeouts, 1u);
+            }
+            return;
+        }
+        const int end = min(nvec, (p + 1) * kGnCopyVecs);
+        for (int base = p * kGnCopyVecs; base < end; base += kPartVecs) {
 #pragma unroll
-        for (int k = 0; k < kGnUnroll; ++k) {
-            const int v = p * kGnPartVecs + k * kGnThreads + threadIdx.x;
-            if (v < nvec) {
-                raw[k] = stage[v];
-                ++cnt;
-            } else {
-                raw[k] = Vec16{{0u, 0u, 0u, 0u}};
+            for (int k = 0; k < kGnUnroll; ++k) {
+                const int v = base + k * NT + threadIdx.x;
+                if (v < end) {
+                    float2 f[P];
+                    Elem<T>::unpack2(stage[v], f);
+#pragma unroll
+                    for (int e = 0; e < P; ++e) s2 = __fadd2_rn(s2, f[e]);
+                }
             }
         }
-        accumulate_batch<T>(raw, cnt, acc);
     }
-    float mu, rs;
-    if (!cta_moments(acc, sh, eps, mean, rstd, chunk, ok, mu, rs)) {
-        // give the copies one more bounded chance to drain before this CTA's shared memory is released
-        for (int p = 0; p < nparts; ++p) mbar_wait_bounded(bars + p, 0);
-        if (threadIdx.x == 0) atomicAdd(&g_gn_wait_timeouts, 1u);
-        return;
-    }
-    const float inv_vpp = 1.0f / (float)vec_per_plane;
-    for (int base = 0; base < nvec; base += kGnPartVecs) {
+    const float mu = block_sum(s2.x + s2.y, slots_a) * inv_count;
+    const float2 nmu = make_float2(-mu, -mu);
+    float2 q2 = make_float2(0.0f, 0.0f);
+    for (int base = 0; base < nvec; base += kPartVecs) {
 #pragma unroll
         for (int k = 0; k < kGnUnroll; ++k) {
-            const int v = base + k * kGnThreads + threadIdx.x;
+            const int v = base + k * NT + threadIdx.x;
+            if (v < nvec) {
+                float2 f[P];
+                Elem<T>::unpack2(stage[v], f);
+#pragma unroll
+                for (int e = 0; e < P; ++e) {
+                    const float2 d = __fadd2_rn(f[e], nmu);
+                    q2 = __ffma2_rn(d, d, q2);
+                }
+            }
+        }
+    }
+    const float rs = rsqrtf(block_sum(q2.x + q2.y, slots_b) * inv_count + eps);
+    if (threadIdx.x == 0) {
+        if (mean != nullptr) mean[chunk] = mu;
+        if (rstd != nullptr) rstd[chunk] = rs;
+    }
+    const float inv_vpp = 1.0f / (float)vec_per_plane;
+    for (int base = 0; base < nvec; base += kPartVecs) {
+#pragma unroll
+        for (int k = 0; k < kGnUnroll; ++k) {
+            const int v = base + k * NT + threadIdx.x;
             if (v < nvec)
                 normalize_store<T, ACT>(stage[v], yc + (int64_t)v * E, g * cpg + div_small(v, vec_per_plane, inv_vpp),
                                         gamma, beta, mu, rs);
@@ -424,7 +404,7 @@ groupnorm_scalar_kernel(const T* __restrict__ x, const float* __restrict__ gamma
 }
 
 constexpr size_t kGnStageLimit = 200 * 1024;     // leaves room for the static reduction slots
-static_assert(kGnStageLimit <= (size_t)kGnMaxParts * kGnPartVecs * 16, "one barrier per 32 KB part");
+static_assert(kGnStageLimit <= (size_t)kGnMaxParts * kGnCopyVecs * 16, "one barrier per 32 KB part");
 constexpr int kMaxDevices = 64;
 
 template <typename T, int ACT>
@@ -444,13 +424,23 @@ kop_status_t launch_gn_act(const T* x, const float* gamma, const float* beta, T*
             int dev = 0;
             if (cudaGetDevice(&dev) != cudaSuccess) return KOP_ERR_CUDA;
             if (dev < 0 || dev >= kMaxDevices || !configured[dev].load(std::memory_order_acquire)) {
-                if (cudaFuncSetAttribute(groupnorm_staged_kernel<T, ACT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                // only the 512-thread instance ever needs more than the default 48 KB (chunks beyond 32 KB)
+                if (cudaFuncSetAttribute(groupnorm_staged_kernel<T, ACT, 512>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)kGnStageLimit) != cudaSuccess)
                     return KOP_ERR_CUDA;
                 if (dev >= 0 && dev < kMaxDevices) configured[dev].store(true, std::memory_order_release);
             }
-            groupnorm_staged_kernel<T, ACT><<<(unsigned)chunks, kGnThreads, bytes, stream>>>(
-                x, gamma, beta, y, mean, rstd, nvec, vpp, cpg, groups, eps);
+            const float inv_count = (float)(1.0 / (double)chunk_elems);
+            if (nvec <= 512)
+                groupnorm_staged_kernel<T, ACT, 128><<<(unsigned)chunks, 128, bytes, stream>>>(
+                    x, gamma, beta, y, mean, rstd, nvec, vpp, cpg, groups, eps, inv_count);
+            else if (nvec <= 2048)
+                groupnorm_staged_kernel<T, ACT, 256><<<(unsigned)chunks, 256, bytes, stream>>>(
+                    x, gamma, beta, y, mean, rstd, nvec, vpp, cpg, groups, eps, inv_count);
+            else
+                groupnorm_staged_kernel<T, ACT, 512><<<(unsigned)chunks, 512, bytes, stream>>>(
+                    x, gamma, beta, y, mean, rstd, nvec, vpp, cpg, groups, eps, inv_count);
         } else {
             groupnorm_twosweep_kernel<T, ACT><<<(unsigned)chunks, kGnThreads, 0, stream>>>(
                 x, gamma, beta, y, mean, rstd, nvec, vpp, cpg, groups, eps);

@@ -1,6 +1,6 @@
 """GPU parity of kop_groupnorm_act (GroupNorm / InstanceNorm with optional affine and activation)
 against the float64 CPU oracle: five seeds over shapes that hit the shared-memory-staged kernel
-(one and several trips, ragged last trip), the unstaged kernel (chunks beyond the staging budget)
+(one and several parts, ragged last part, several waves of CTAs), the two-sweep kernel (chunks beyond the staging budget)
 and the scalar kernel (planes that do not split into 16-byte vectors, misaligned bases), all three
 activations, missing affine parameters, in-place use, guard bands and run-to-run bit equality.
 
@@ -45,6 +45,8 @@ GN_SHAPES = [
     (2, 8, 2, 2, 4, F32, 1),           # plane of one vector, chunk shorter than a warp's worth
     (5, 3, 1, 1, 3, F32, 0),           # one element per group: variance 0, y = beta
     (1, 16, 4, 4, 2, BF16, 2),
+    (10, 256, 56, 56, 32, F32, 0),     # 320 chunks of 100 KB: more CTAs than fit the GPU at once
+    (80, 64, 56, 56, 8, BF16, 1),      # 640 chunks of 50 KB
 ]
 
 
