@@ -496,7 +496,7 @@ def run_ours(args, rank, world, local_rank):
                     frac=round(achieved / peak, 4), traffic=traffic, peak_source=peak_src,
                     algorithmic_bytes=segs[dom]["bytes"], avg_launch_us=round(dom_ms * 1e3, 2))
 
-    gate = perf_gate(wl, names) if (rank == 0 and not args.no_perf_gate) else None
+    gate = perf_gate(wl, names, inductor=args.inductor) if (rank == 0 and not args.no_perf_gate) else None
     e2e = run_e2e(args, wl, kop, dev, segs, names, world)
     cpu = None
     if rank == 0 and world == 1:
@@ -573,10 +573,12 @@ def unfused_torch_chain(wl, name):
     raise KeyError(name)
 
 
-def perf_gate(wl, names, reps=10):
+def perf_gate(wl, names, reps=10, inductor=False):
     """Gate 4 of the paper's cascade (Eq. 5): tau(new) <= gamma * tau(baseline), gamma = 1.03, with the
     unfused stock-torch chain as the baseline. Both sides are timed the same way on this GPU in this
-    run: `reps` back-to-back launches between one pair of events."""
+    run: `reps` back-to-back launches between one pair of events. With `inductor`, the same chain is
+    also compiled with torch.compile (default mode): the baseline the paper's speed-ups are quoted
+    against; a compile failure is recorded, not raised."""
     def back_to_back(f):
         f()
         f()
@@ -597,6 +599,16 @@ def perf_gate(wl, names, reps=10):
         ours_us = back_to_back(lambda: wl.launch(nm))
         out[nm] = {"unfused_torch_us": round(base_us, 1), "libkop_us": round(ours_us, 1),
                    "speedup": round(base_us / ours_us, 2), "passes_gamma_1.03": bool(ours_us <= 1.03 * base_us)}
+        if inductor:
+            try:
+                cf = torch.compile(f)
+                ind_us = back_to_back(cf)
+                out[nm].update({"torch_compile_us": round(ind_us, 1),
+                                "speedup_vs_torch_compile": round(ind_us / ours_us, 2),
+                                "passes_gamma_1.03_vs_torch_compile": bool(ours_us <= 1.03 * ind_us)})
+                del cf
+            except Exception as e:  # noqa: BLE001
+                out[nm]["torch_compile_error"] = f"{type(e).__name__}: {str(e)[:200]}"
         del f
         torch.cuda.empty_cache()
     return out
@@ -796,6 +808,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-perf-gate", action="store_true", help="skip the comparison with the unfused torch chains")
+    ap.add_argument("--inductor", action="store_true",
+                    help="perf gate: also time each chain compiled with torch.compile (adds compile time)")
     ap.add_argument("--clock-sample-ms", type=float, default=4.0, help="period of the SM-clock sampler")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="CPU time budget of the cpu_baseline leg")
     ap.add_argument("--profile", default=None, help="comma list of segments to launch alone (ncu / quick timing)")
