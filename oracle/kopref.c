@@ -521,3 +521,37 @@ int kopref_groupnorm_act(const void* x, const float* gamma, const float* beta, d
     }
     return 0;
 }
+
+/* ---- row-wise cumulative sum (the CumSum rows of the paper's per-kernel results table, L1-089..093: plain,
+ * reverse, exclusive and masked running sums along the last dimension) ---------------------------------
+ * m[i,k] = 1 when mask is NULL, else (mask[i,k] != 0).
+ *   inclusive, forward : y[i,j] = sum_{k <= j} x[i,k] m[i,k]
+ *   exclusive, forward : y[i,j] = sum_{k <  j} x[i,k] m[i,k]
+ *   inclusive, reverse : y[i,j] = sum_{k >= j} x[i,k] m[i,k]
+ *   exclusive, reverse : y[i,j] = sum_{k >  j} x[i,k] m[i,k]
+ * The running sum is carried in double, in index order. */
+int kopref_cumsum_rows(const void* x, const unsigned char* mask, double* y, int64_t rows, int64_t cols,
+        int64_t x_row_stride, int64_t mask_row_stride, int64_t y_row_stride, int exclusive, int reverse,
+        int dtype, int threads)
+{
+    if (!x || !y || rows < 0 || cols <= 0 || bad_dtype(dtype)) return -1;
+    int nt = pick_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t i = 0; i < rows; ++i) {
+        double run = 0.0;
+        for (int64_t s = 0; s < cols; ++s) {
+            int64_t j = reverse ? cols - 1 - s : s;
+            double v = load_elem(x, i * x_row_stride + j, dtype);
+            if (mask && mask[i * mask_row_stride + j] == 0) v = 0.0;
+            if (exclusive) {
+                y[i * y_row_stride + j] = run;
+                run += v;
+            } else {
+                run += v;
+                y[i * y_row_stride + j] = run;
+            }
+        }
+    }
+    return 0;
+}

@@ -45,6 +45,7 @@ def lib() -> C.CDLL:
         _lib.kopref_ce_loss_opts.argtypes = [vp] * 6 + [i64] * 3 + [C.c_int32, dbl, C.c_int, C.c_int]
         _lib.kopref_groupnorm_act.argtypes = [vp] * 6 + [i64] * 5 + [dbl, C.c_int, C.c_int, C.c_int]
         _lib.kopref_row_scale.argtypes = [vp, vp, vp, i64, i64, i64, i64, C.c_int, C.c_int]
+        _lib.kopref_cumsum_rows.argtypes = [vp, vp, vp] + [i64] * 5 + [C.c_int] * 4
         _lib.kopref_matvec_bias.argtypes = [vp, vp, dbl, vp, i64, i64, i64, C.c_int, C.c_int]
     return _lib
 
@@ -292,6 +293,22 @@ def matvec_bias(x, w, b_sum, threads=1) -> np.ndarray:
     assert wa.shape == (K,)
     out = np.empty(M, dtype=np.float64)
     _check(lib().kopref_matvec_bias(_p(xa), _p(wa), float(b_sum), _p(out), M, K, K, dt, _nt(threads)), "matvec_bias")
+    return out
+
+
+def cumsum_rows(x, mask=None, exclusive=False, reverse=False, threads=1) -> np.ndarray:
+    """Running sum along each row of x [rows, cols]; mask (uint8 / bool, same shape, nonzero = keep) zeroes
+    elements before they are summed. See kopref_cumsum_rows for the four variants."""
+    xa, dt = as_data(x)
+    rows, cols = xa.shape
+    m = None
+    if mask is not None:
+        m = np.ascontiguousarray(np.asarray(mask.detach().cpu().numpy() if hasattr(mask, "detach") else mask)
+                                 .astype(np.uint8))
+        assert m.shape == (rows, cols)
+    out = np.empty((rows, cols), dtype=np.float64)
+    _check(lib().kopref_cumsum_rows(_p(xa), None if m is None else _p(m), _p(out), rows, cols, cols, cols, cols,
+                                    int(bool(exclusive)), int(bool(reverse)), dt, _nt(threads)), "cumsum_rows")
     return out
 
 

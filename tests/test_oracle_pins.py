@@ -636,3 +636,57 @@ def test_threads_do_not_change_results():
     l1, m1, _ = kopref.ce_loss_rowwise(x, lab, threads=1)
     l4, m4, _ = kopref.ce_loss_rowwise(x, lab, threads=4)
     assert np.array_equal(l1, l4) and m1 == m4
+
+
+# --------------------------------------------------------------------------- row-wise cumulative sums
+
+def test_cumsum_closed_forms_library_and_identities():
+    # closed forms: integers are exact in float64
+    n = 257
+    ones = np.ones((2, n), dtype=np.float32)
+    k = np.arange(1, n + 1, dtype=np.float64)
+    assert np.array_equal(kopref.cumsum_rows(ones)[0], k)                          # 1, 2, ..., n
+    assert np.array_equal(kopref.cumsum_rows(ones, exclusive=True)[1], k - 1)      # 0, 1, ..., n-1
+    assert np.array_equal(kopref.cumsum_rows(ones, reverse=True)[0], k[::-1])      # n, ..., 1
+    assert np.array_equal(kopref.cumsum_rows(ones, exclusive=True, reverse=True)[0], k[::-1] - 1)
+    ramp = np.tile(np.arange(1, n + 1, dtype=np.float32), (3, 1))
+    assert np.array_equal(kopref.cumsum_rows(ramp)[2], k * (k + 1) / 2)            # triangular numbers
+    alt = np.tile(np.where(np.arange(n) % 2 == 0, 1.0, -1.0).astype(np.float32), (1, 1))
+    assert np.array_equal(kopref.cumsum_rows(alt)[0], (np.arange(n) % 2 == 0).astype(np.float64))
+    geo = np.tile((0.5 ** np.arange(40)).astype(np.float32), (1, 1))              # exact powers of two
+    assert np.array_equal(kopref.cumsum_rows(geo)[0], 2.0 - 0.5 ** np.arange(40))
+    # library routine in float64 on random data, every variant, fp32 and bf16 inputs
+    x = f32(RNG.normal(0, 1, (7, 301)))
+    m = RNG.random((7, 301)) < 0.6
+    xd = x.astype(np.float64)
+    inc = np.cumsum(xd, axis=1)
+    np.testing.assert_allclose(kopref.cumsum_rows(x), inc, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(kopref.cumsum_rows(x, exclusive=True), inc - xd, rtol=0, atol=1e-12)
+    rev = np.cumsum(xd[:, ::-1], axis=1)[:, ::-1]
+    np.testing.assert_allclose(kopref.cumsum_rows(x, reverse=True), rev, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(kopref.cumsum_rows(x, exclusive=True, reverse=True), rev - xd, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(kopref.cumsum_rows(x, mask=m), np.cumsum(xd * m, axis=1), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(kopref.cumsum_rows(x, mask=m, reverse=True),
+                               np.cumsum((xd * m)[:, ::-1], axis=1)[:, ::-1], rtol=0, atol=1e-12)
+    tb = torch.from_numpy(x).to(torch.bfloat16)
+    np.testing.assert_allclose(kopref.cumsum_rows(tb), torch.cumsum(tb.to(torch.float64), dim=1).numpy(),
+                               rtol=0, atol=1e-12)
+    # identities: inclusive forward + exclusive reverse = row total; the last column is the row sum;
+    # an all-ones mask changes nothing, an all-zero mask gives zeros; differences recover the input
+    total = xd.sum(axis=1, keepdims=True)
+    np.testing.assert_allclose(kopref.cumsum_rows(x) + kopref.cumsum_rows(x, exclusive=True, reverse=True),
+                               np.broadcast_to(total, x.shape), rtol=0, atol=1e-11)
+    np.testing.assert_allclose(kopref.cumsum_rows(x)[:, -1], math_fsum_rows(xd), rtol=0, atol=1e-12)
+    assert np.array_equal(kopref.cumsum_rows(x, mask=np.ones_like(m)), kopref.cumsum_rows(x))
+    assert np.array_equal(kopref.cumsum_rows(x, mask=np.zeros_like(m)), np.zeros_like(xd))
+    np.testing.assert_allclose(np.diff(kopref.cumsum_rows(x), axis=1), xd[:, 1:], rtol=0, atol=1e-12)
+    # one column: inclusive is x, exclusive is 0
+    c1 = f32(RNG.normal(0, 1, (5, 1)))
+    assert np.array_equal(kopref.cumsum_rows(c1), c1.astype(np.float64))
+    assert np.array_equal(kopref.cumsum_rows(c1, exclusive=True), np.zeros((5, 1)))
+    # threads do not change the result
+    assert np.array_equal(kopref.cumsum_rows(x, mask=m, threads=4), kopref.cumsum_rows(x, mask=m, threads=1))
+
+
+def math_fsum_rows(a):
+    return np.array([math.fsum(r) for r in a])
