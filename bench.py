@@ -94,6 +94,8 @@ def segment_bytes():
     q = c["groupnorm"]
     e = q["N"] * q["C"] * q["H"] * q["W"]
     out["groupnorm"] = dict(bytes=2 * e * 4 + 2 * q["C"] * 4 + 2 * q["N"] * q["groups"] * 4, elems=e)
+    u = c["cumsum"]
+    out["cumsum"] = dict(bytes=2 * u["rows"] * u["cols"] * 4, elems=u["rows"] * u["cols"])
     return out
 
 
@@ -237,7 +239,7 @@ class Workload:
 
     ORDER = ["softmax_small", "softmax_large", "layernorm", "bn_pool", "ce_loss", "rmsnorm", "silu_mul", "residual_add"]
     # Beyond the benchmark configs (not part of `value`): the two kernels the paper's case studies print.
-    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "silu_mul_interleaved", "ce_loss_opts", "groupnorm"]
+    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum"]
 
     def __init__(self, kop, device, seed, only=None, rows_div=1):
         """only: build just these segments (None = all, plus the MLP segment); rows_div cuts the row
@@ -293,6 +295,10 @@ class Workload:
             self.qy = torch.empty_like(self.qx)
             self.qmean = torch.empty((self.qx.shape[0], q["groups"]), dtype=torch.float32, device=dev)
             self.qrstd = torch.empty_like(self.qmean)
+        if "cumsum" in want:
+            u = c["cumsum"]
+            self.ux, _ = synth.cumsum_inputs(cut(u["rows"]), u["cols"], u["dtype"], seed, dev)
+            self.uy = torch.empty_like(self.ux)
         m = c["mlp"]
         self.eps = m["eps"]
         rows = cut(m["rows"])
@@ -357,6 +363,8 @@ class Workload:
             q = c["groupnorm"]
             k.kop_groupnorm_act(self.qx, self.qg, self.qb, q["groups"], q["eps"], q["act"], out=self.qy,
                                 mean=self.qmean, rstd=self.qrstd)
+        elif name == "cumsum":                   # inclusive running sum along rows, fp32 [32768, 4096]
+            k.kop_cumsum_rows(self.ux, out=self.uy)
         else:
             raise KeyError(name)
 

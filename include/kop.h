@@ -285,6 +285,24 @@ kop_status_t kop_groupnorm_act(const void* x, const float* gamma, const float* b
                                int64_t groups, float eps, int act, kop_dtype_t dtype, kop_stream_t stream);
 
 /*
+ * Running sums along each row (the CumSum rows of the paper's per-kernel results table, L1-089 to L1-093:
+ * plain, reverse, exclusive and masked cumulative sums; planner strategy "single-pass reductions" applied
+ * to a scan). With m[i,k] = 1 when mask is NULL, else (mask[i,k] != 0):
+ *   exclusive = 0, reverse = 0:  y[i,j] = sum_{k <= j} x[i,k] m[i,k]
+ *   exclusive = 1, reverse = 0:  y[i,j] = sum_{k <  j} x[i,k] m[i,k]      (y[i,0] = 0)
+ *   exclusive = 0, reverse = 1:  y[i,j] = sum_{k >= j} x[i,k] m[i,k]
+ *   exclusive = 1, reverse = 1:  y[i,j] = sum_{k >  j} x[i,k] m[i,k]      (y[i,cols-1] = 0)
+ * x, y: [rows, cols] of `dtype`; mask: uint8 [rows, cols] with row stride mask_row_stride (bytes =
+ * elements), or NULL. Sums are fp32 (a tree of partial sums, fixed order: results are bit-identical run
+ * to run); a masked-out element contributes 0 even if it is NaN or infinite; a NaN or infinity that is
+ * kept affects exactly the outputs whose sums include it. y may alias x exactly; mask must not overlap y.
+ * rows <= 2^31 - 1. Nonzero `exclusive` / `reverse` mean "on".
+ */
+kop_status_t kop_cumsum_rows(const void* x, const unsigned char* mask, void* y, int64_t rows, int64_t cols,
+                             int64_t x_row_stride, int64_t mask_row_stride, int64_t y_row_stride,
+                             int exclusive, int reverse, kop_dtype_t dtype, kop_stream_t stream);
+
+/*
  * Diagnostic for kop_groupnorm_act (no counterpart in the paper): its staged kernel waits for its bulk
  * copies with a bounded number of polls; a CTA whose wait runs out writes nothing, and counts itself here.
  * host_count: HOST pointer, receives the count for the current device since the library was loaded (always

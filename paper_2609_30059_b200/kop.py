@@ -76,6 +76,8 @@ def lib() -> C.CDLL:
     L.kop_matvec_bias.restype = i32
     L.kop_groupnorm_act.argtypes = [vp] * 6 + [i64] * 5 + [f32, i32, i32, vp]
     L.kop_groupnorm_act.restype = i32
+    L.kop_cumsum_rows.argtypes = [vp, vp, vp] + [i64] * 5 + [i32, i32, i32, vp]
+    L.kop_cumsum_rows.restype = i32
     L.kop_groupnorm_wait_timeouts.argtypes = [C.POINTER(C.c_uint)]
     L.kop_groupnorm_wait_timeouts.restype = i32
     L.kop_rmsnorm_swiglu_residual.argtypes = [vp] * 6 + [i64] * 3 + [f32, vp, sz, i32, vp]
@@ -342,6 +344,25 @@ def kop_groupnorm_act(x, gamma, beta, groups, eps, act=0, out=None, mean=None, r
                                    None if rstd is None else rstd.data_ptr(), N, Cc, H, W, int(groups),
                                    float(eps), int(act), _dtype_tag(x), _stream(stream)), "kop_groupnorm_act")
     return out, mean, rstd
+
+
+def kop_cumsum_rows(x, mask=None, exclusive=False, reverse=False, out=None, stream=None):
+    """mask: uint8 or bool CUDA tensor of x's shape (nonzero = keep), unit inner stride."""
+    rows, cols, xs = _rows2d(x, "x")
+    out = torch.empty_like(x) if out is None else out
+    _, _, ys = _rows2d(out, "out")
+    assert out.shape == x.shape and out.dtype == x.dtype
+    mp, ms = None, cols
+    if mask is not None:
+        if mask.dtype == torch.bool:
+            mask = mask.view(torch.uint8)
+        if mask.dtype != torch.uint8 or mask.shape != x.shape:
+            raise ValueError("mask: expected a uint8 / bool tensor of x's shape")
+        _, _, ms = _rows2d(mask, "mask")
+        mp = mask.data_ptr()
+    _check(lib().kop_cumsum_rows(x.data_ptr(), mp, out.data_ptr(), rows, cols, xs, ms, ys, int(bool(exclusive)),
+                                 int(bool(reverse)), _dtype_tag(x), _stream(stream)), "kop_cumsum_rows")
+    return out
 
 
 def kop_groupnorm_wait_timeouts() -> int:

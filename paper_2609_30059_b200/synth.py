@@ -24,6 +24,8 @@ CONFIGS = {
     "matvec_bias": dict(rows=32768, k=4096, dtype=torch.bfloat16),         # shape not given in the paper
     # GroupNorm + SiLU as in a diffusion U-Net residual block: 32 groups over 256 channels of a 56 x 56 map
     "groupnorm": dict(N=64, C=256, H=56, W=56, groups=32, dtype=torch.float32, eps=1e-5, act=2),
+    # running sum along rows (shape ours; the paper gives none)
+    "cumsum": dict(rows=32768, cols=4096, dtype=torch.float32),
 }
 
 
@@ -129,3 +131,11 @@ def groupnorm_inputs(N, C, H, W, dtype=torch.float32, seed=0, device="cpu"):
     gamma = _normal((C,), 1.0, 0.02, g, device)
     beta = _normal((C,), 0.0, 0.02, g, device)
     return x, gamma, beta
+
+
+def cumsum_inputs(rows, cols, dtype=torch.float32, seed=0, device="cpu", keep=0.7):
+    """x ~ N(0,1) [rows, cols]; mask uint8, 1 with probability `keep`."""
+    g = _gen(seed, device)
+    x = _normal((rows, cols), 0.0, 1.0, g, device).to(dtype)
+    mask = (torch.rand((rows, cols), generator=g, device=device, dtype=torch.float32) < keep).to(torch.uint8)
+    return x, mask

@@ -181,6 +181,25 @@ def test_groupnorm_validation(L):
     assert L.kop_groupnorm_wait_timeouts(None) == NULLP
 
 
+def test_cumsum_validation(L):
+    f = L.kop_cumsum_rows
+    M = 0x600000
+    assert f(P, None, Q, 0, 64, 64, 64, 64, 0, 0, 0, None) == OK
+    assert f(None, None, Q, 4, 64, 64, 64, 64, 0, 0, 0, None) == NULLP
+    assert f(P, None, None, 4, 64, 64, 64, 64, 0, 0, 0, None) == NULLP
+    assert f(P, None, Q, 4, 0, 64, 64, 64, 0, 0, 0, None) == SHAPE
+    assert f(P, None, Q, -1, 64, 64, 64, 64, 0, 0, 0, None) == SHAPE
+    assert f(P, None, Q, 2 ** 31, 64, 64, 64, 64, 0, 0, 0, None) == SHAPE      # one CTA per row
+    assert f(P, None, Q, 4, 64, 63, 64, 64, 0, 0, 0, None) == STRIDE
+    assert f(P, None, Q, 4, 64, 64, 64, 8, 0, 0, 0, None) == STRIDE
+    assert f(P, M, Q, 4, 64, 64, 63, 64, 0, 0, 0, None) == STRIDE              # mask stride checked when given
+    assert f(P, None, Q, 4, 64, 64, 1, 64, 0, 0, 0, None) != STRIDE            # and ignored when not
+    assert f(P, None, Q, 4, 64, 64, 64, 64, 0, 0, 3, None) == DTYPE
+    assert f(P + 2, None, Q, 4, 64, 64, 64, 64, 0, 0, 0, None) == MISAL
+    assert f(P, None, P + 8, 4, 64, 64, 64, 64, 0, 0, 0, None) == ALIAS        # partial overlap of x and y
+    assert f(P, Q + 16, Q, 4, 64, 64, 64, 64, 0, 0, 0, None) == ALIAS          # mask overlaps y
+
+
 def test_mlp_driver_validation(L):
     f = L.kop_rmsnorm_swiglu_residual
     wsb = L.kop_rmsnorm_swiglu_residual_workspace_bytes(16, 64, 128, 1)
