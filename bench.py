@@ -94,6 +94,7 @@ def segment_bytes():
     q = c["groupnorm"]
     e = q["N"] * q["C"] * q["H"] * q["W"]
     out["groupnorm"] = dict(bytes=2 * e * 4 + 2 * q["C"] * 4 + 2 * q["N"] * q["groups"] * 4, elems=e)
+    out["bn_pool_nhwc"] = dict(out["bn_pool"])
     u = c["cumsum"]
     out["cumsum"] = dict(bytes=2 * u["rows"] * u["cols"] * 4, elems=u["rows"] * u["cols"])
     return out
@@ -239,7 +240,7 @@ class Workload:
 
     ORDER = ["softmax_small", "softmax_large", "layernorm", "bn_pool", "ce_loss", "rmsnorm", "silu_mul", "residual_add"]
     # Beyond the benchmark configs (not part of `value`): the two kernels the paper's case studies print.
-    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum"]
+    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc"]
 
     def __init__(self, kop, device, seed, only=None, rows_div=1):
         """only: build just these segments (None = all, plus the MLP segment); rows_div cuts the row
@@ -295,6 +296,13 @@ class Workload:
             self.qy = torch.empty_like(self.qx)
             self.qmean = torch.empty((self.qx.shape[0], q["groups"]), dtype=torch.float32, device=dev)
             self.qrstd = torch.empty_like(self.qmean)
+        if "bn_pool_nhwc" in want:
+            b = c["bn_pool"]
+            hx, self.hscale, self.hshift = synth.bn_pool_inputs(cut(b["N"]), b["C"], b["H"], b["W"], b["dtype"], seed, dev)
+            self.hx = hx.contiguous(memory_format=torch.channels_last)
+            del hx
+            self.hy = torch.empty_like(self.hx)
+            self.hp = torch.empty((self.hx.shape[0], b["C"]), dtype=torch.float32, device=dev)
         if "cumsum" in want:
             u = c["cumsum"]
             self.ux, _ = synth.cumsum_inputs(cut(u["rows"]), u["cols"], u["dtype"], seed, dev)
@@ -363,6 +371,8 @@ class Workload:
             q = c["groupnorm"]
             k.kop_groupnorm_act(self.qx, self.qg, self.qb, q["groups"], q["eps"], q["act"], out=self.qy,
                                 mean=self.qmean, rstd=self.qrstd)
+        elif name == "bn_pool_nhwc":             # the BN + ReLU + pool config in channels-last memory
+            k.kop_bn_relu_avgpool(self.hx, self.hscale, self.hshift, out=self.hy, pooled=self.hp)
         elif name == "cumsum":                   # inclusive running sum along rows, fp32 [32768, 4096]
             k.kop_cumsum_rows(self.ux, out=self.uy)
         else:

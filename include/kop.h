@@ -112,10 +112,12 @@ kop_status_t kop_bias_gelu_residual_layernorm(const void* x, const void* residua
  * CNN models, next to preserved cuDNN convolutions):
  *   a[n,c,h,w] = max(x[n,c,h,w] * scale[c] + shift[c], 0)   (NaN stays NaN)
  *   pooled[n,c] = (1 / (H W)) sum_{h,w} a[n,c,h,w]          (sum of unrounded fp32 a)
- * x, y: NCHW of `dtype`; x_strides / y_strides are HOST arrays of 4 element strides
- * and must describe a contiguous NCHW tensor ({C*H*W, H*W, W, 1}), anything else
+ * x, y: indexed [n,c,h,w], of `dtype`; x_strides / y_strides are HOST arrays of 4 element
+ * strides (for n, c, h, w) and must both describe the same one of two dense layouts:
+ * contiguous NCHW ({C*H*W, H*W, W, 1}) or channels-last, i.e. NHWC memory
+ * ({H*W*C, 1, W*C, C}); strides of extent-1 dimensions are ignored; anything else
  * returns KOP_ERR_BAD_STRIDE. scale, shift: fp32 [C]; pooled: fp32 [N, C].
- * y may alias x exactly.
+ * y may alias x exactly. Each pooled value is summed by one CTA in a fixed order.
  */
 kop_status_t kop_bn_relu_avgpool(const void* x, const float* scale, const float* shift,
                                  void* y, float* pooled,

@@ -1,6 +1,7 @@
 // kop_bn_relu_avgpool: a = relu(x * scale[c] + shift[c]) written once, pooled[n,c] = mean over the
 // (h, w) plane of the unrounded fp32 activations, in the same pass. NCHW planes are contiguous, so
-// a CTA (or a warp, for small planes) streams one plane with 16-byte vectors and reduces it.
+// a CTA (or a warp, for small planes) streams one plane with 16-byte vectors and reduces it; the
+// channels-last kernels are at the end of the file.
 #include "kop_common.cuh"
 
 namespace kop {
@@ -147,6 +148,207 @@ kop_status_t launch_bn(const void* xv, const float* scale, const float* shift, v
     return launch_status();
 }
 
+// ---- channels-last (NHWC memory): x[n][h*w][c] --------------------------------------------------------
+// The channel is the innermost index, so the pooled mean is a column sum. A CTA owns one image, a tile of
+// TV 16-byte vectors of channels (up to 256 contiguous bytes per row) and a slab of rows; thread t keeps
+// column t % TV and walks rows t / TV, t / TV + R, ... of the slab (R = 256 / TV rows per sweep, U of them
+// in flight) with its scale / shift values and running column sums in registers. When an image has too
+// few (tile) CTAs to fill the GPU its rows are split over a thread-block cluster of up to 8 CTAs: each
+// writes its column sums into the first CTA's shared memory (distributed shared memory), one cluster
+// barrier, and the first CTA adds them in rank order. No atomics, no workspace, and for a given call
+// shape a fixed summation order.
+__device__ __forceinline__ uint32_t cluster_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+
+__device__ __forceinline__ void store_to_cluster_cta(float* local_slot, uint32_t cta, float v)
+{
+    const uint32_t la = (uint32_t)__cvta_generic_to_shared(local_slot);
+    uint32_t ra;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(la), "r"(cta));
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(ra), "f"(v) : "memory");
+}
+
+__device__ __forceinline__ void cluster_barrier()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+constexpr int kBnMaxSlabs = 8;      // portable cluster size
+
+template <typename T, int TV, int U, bool kCluster>
+__global__ void __launch_bounds__(256)
+bn_nhwc_kernel(const T* __restrict__ x, const float* __restrict__ scale, const float* __restrict__ shift,
+               T* __restrict__ y, float* __restrict__ pooled, int64_t hw, int cvec, int tiles, int slabs,
+               float inv_hw)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    constexpr int NT = 256, R = NT / TV;
+    __shared__ float part[R][TV * E];
+    __shared__ float from_ranks[kCluster ? kBnMaxSlabs : 1][TV * E];
+    const int col = threadIdx.x % TV, phase = threadIdx.x / TV;
+    const int slab = kCluster ? (int)cluster_rank() : 0;     // consecutive CTAs form a cluster
+    const int64_t unit = blockIdx.x / slabs;                 // (image, channel tile)
+    const int64_t n = unit / tiles;
+    const int tile = (int)(unit - n * tiles);
+    const int cv = tile * TV + col;                          // this thread's channel vector
+    const bool live = cv < cvec;
+    const int64_t C = (int64_t)cvec * E;
+    const int64_t slab_rows = (hw + slabs - 1) / slabs;
+    const int64_t r_begin = slab * slab_rows;
+    const int64_t r_end = r_begin + slab_rows < hw ? r_begin + slab_rows : hw;
+    float sc[E], sh[E], acc[E];
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+        sc[e] = live ? __ldg(scale + (int64_t)cv * E + e) : 0.0f;
+        sh[e] = live ? __ldg(shift + (int64_t)cv * E + e) : 0.0f;
+        acc[e] = 0.0f;
+    }
+    const T* xn = x + n * hw * C + (int64_t)cv * E;
+    T* yn = y + n * hw * C + (int64_t)cv * E;
+    if (live) {
+        for (int64_t r0 = r_begin + phase; r0 < r_end; r0 += (int64_t)R * U) {
+            Vec16 raw[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int64_t r = r0 + (int64_t)u * R;
+                if (r < r_end) raw[u] = ld_stream(xn + r * C);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int64_t r = r0 + (int64_t)u * R;
+                if (r < r_end) {
+                    float f[E];
+                    Elem<T>::unpack(raw[u], f);
+#pragma unroll
+                    for (int e = 0; e < E; ++e) {
+                        f[e] = relu_keep_nan(fmaf(f[e], sc[e], sh[e]));
+                        acc[e] += f[e];
+                    }
+                    st_stream(yn + r * C, Elem<T>::pack(f));
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < E; ++e) part[phase][col * E + e] = acc[e];
+    __syncthreads();
+    float s = 0.0f;
+    if (threadIdx.x < TV * E) {
+#pragma unroll 8
+        for (int r = 0; r < R; ++r) s += part[r][threadIdx.x];
+    }
+    if (kCluster) {
+        if (threadIdx.x < TV * E) store_to_cluster_cta(&from_ranks[slab][threadIdx.x], 0u, s);
+        cluster_barrier();                                   // hardware barrier over the cluster's CTAs
+        if (slab != 0) return;
+        if (threadIdx.x < TV * E) {
+            s = 0.0f;
+            for (int k = 0; k < slabs; ++k) s += from_ranks[k][threadIdx.x];
+        }
+    }
+    if (threadIdx.x < TV * E) {
+        const int64_t c = (int64_t)tile * TV * E + threadIdx.x;
+        if (c < C) pooled[n * C + c] = s * inv_hw;
+    }
+}
+
+// Any channel count / alignment: lanes along channels with scalar loads, warps along rows.
+template <typename T>
+__global__ void __launch_bounds__(256)
+bn_nhwc_scalar_kernel(const T* __restrict__ x, const float* __restrict__ scale, const float* __restrict__ shift,
+                      T* __restrict__ y, float* __restrict__ pooled, int64_t hw, int64_t C, int tiles,
+                      float inv_hw)
+{
+    __shared__ float part[8][32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t n = blockIdx.x / tiles;
+    const int64_t c = (blockIdx.x - n * tiles) * 32 + lane;
+    float acc = 0.0f;
+    if (c < C) {
+        const float sc = __ldg(scale + c), sh = __ldg(shift + c);
+        const T* xn = x + n * hw * C + c;
+        T* yn = y + n * hw * C + c;
+        for (int64_t r = warp; r < hw; r += 8) {
+            const float a = relu_keep_nan(fmaf(Elem<T>::load1(xn + r * C), sc, sh));
+            acc += a;
+            Elem<T>::store1(yn + r * C, a);
+        }
+    }
+    part[warp][lane] = acc;
+    __syncthreads();
+    if (warp == 0 && c < C) {
+        float s = 0.0f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) s += part[w][lane];
+        pooled[n * C + c] = s * inv_hw;
+    }
+}
+
+template <typename T>
+kop_status_t launch_bn_nhwc(const void* xv, const float* scale, const float* shift, void* yv, float* pooled,
+                            int64_t N, int64_t C, int64_t H, int64_t W, cudaStream_t stream)
+{
+    const T* x = static_cast<const T*>(xv);
+    T* y = static_cast<T*>(yv);
+    constexpr int E = Elem<T>::kPerVec;
+    const int64_t hw = H * W;
+    const float inv_hw = (float)(1.0 / (double)hw);
+    const bool vec = aligned_to(x, 16) && aligned_to(y, 16) && (C % E) == 0;
+    if (vec) {
+        const int cvec = (int)(C / E);
+        // a tile as wide as the channel count allows, up to 16 vectors (one 256-byte run per row)
+        int tv = 16;
+        while (tv > 1 && tv / 2 >= cvec) tv >>= 1;
+        const int tiles = (cvec + tv - 1) / tv;
+        // rows split over a cluster until there are ~6 CTAs per SM, each slab keeping at least four sweeps
+        const int64_t want = 6LL * sm_count();
+        const int64_t sweep = (256 / tv) * 4;
+        int slabs = 1;
+        while (slabs < kBnMaxSlabs && N * tiles * slabs < want && hw / (2 * slabs) >= 4 * sweep) slabs <<= 1;
+        const int64_t grid = N * tiles * slabs;
+        if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)grid, 1, 1);
+        cfg.blockDim = dim3(256, 1, 1);
+        cfg.dynamicSmemBytes = 0;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)slabs;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = slabs > 1 ? 1 : 0;
+        cudaError_t err;
+#define KOP_BN_NHWC(TVV)                                                                                         \
+    err = slabs > 1 ? cudaLaunchKernelEx(&cfg, bn_nhwc_kernel<T, TVV, 4, true>, x, scale, shift, y, pooled, hw,   \
+                                         cvec, tiles, slabs, inv_hw)                                              \
+                    : cudaLaunchKernelEx(&cfg, bn_nhwc_kernel<T, TVV, 4, false>, x, scale, shift, y, pooled, hw,  \
+                                         cvec, tiles, slabs, inv_hw)
+        switch (tv) {
+        case 16: KOP_BN_NHWC(16); break;
+        case 8: KOP_BN_NHWC(8); break;
+        case 4: KOP_BN_NHWC(4); break;
+        case 2: KOP_BN_NHWC(2); break;
+        default: KOP_BN_NHWC(1); break;
+        }
+#undef KOP_BN_NHWC
+        if (err != cudaSuccess) {
+            (void)cudaGetLastError();
+            return KOP_ERR_CUDA;
+        }
+        return launch_status();
+    }
+    const int64_t tiles = (C + 31) / 32;
+    if (N * tiles > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+    bn_nhwc_scalar_kernel<T><<<(unsigned)(N * tiles), 256, 0, stream>>>(x, scale, shift, y, pooled, hw, C, (int)tiles, inv_hw);
+    return launch_status();
+}
+
 }  // namespace
 }  // namespace kop
 
@@ -166,9 +368,18 @@ extern "C" kop_status_t kop_bn_relu_avgpool(const void* x, const float* scale, c
     const int64_t plane = H * W;
     if (C > kMaxElems / plane) return KOP_ERR_BAD_SHAPE;
     if (N > 0 && C * plane > kMaxElems / N) return KOP_ERR_BAD_SHAPE;
-    const int64_t want[4] = {C * plane, plane, W, 1};
-    for (int i = 0; i < 4; ++i)
-        if (x_strides[i] != want[i] || y_strides[i] != want[i]) return KOP_ERR_BAD_STRIDE;
+    // Two layouts, the same for x and y: contiguous NCHW, or channels-last (NHWC memory addressed with
+    // NCHW indices). When both descriptions fit (C == 1 or H * W == 1) the layouts coincide.
+    const int64_t nchw[4] = {C * plane, plane, W, 1};
+    const int64_t nhwc[4] = {C * plane, 1, W * C, C};
+    const int64_t dims[4] = {N, C, H, W};
+    bool is_nchw = true, is_nhwc = true;
+    for (int i = 0; i < 4; ++i) {
+        if (dims[i] == 1) continue;                          // the stride of an extent-1 dimension is never used
+        is_nchw = is_nchw && x_strides[i] == nchw[i] && y_strides[i] == nchw[i];
+        is_nhwc = is_nhwc && x_strides[i] == nhwc[i] && y_strides[i] == nhwc[i];
+    }
+    if (!is_nchw && !is_nhwc) return KOP_ERR_BAD_STRIDE;
     const int esz = elem_size(dtype);
     if (!aligned_to(x, esz) || !aligned_to(y, esz) || !aligned_to(scale, 4) || !aligned_to(shift, 4) ||
         !aligned_to(pooled, 4))
@@ -177,6 +388,9 @@ extern "C" kop_status_t kop_bn_relu_avgpool(const void* x, const float* scale, c
     kop_status_t st = check_device();
     if (st != KOP_OK) return st;
     cudaStream_t s = as_stream(stream);
+    if (!is_nchw)
+        return dtype == KOP_F32 ? launch_bn_nhwc<float>(x, scale, shift, y, pooled, N, C, H, W, s)
+                                : launch_bn_nhwc<__nv_bfloat16>(x, scale, shift, y, pooled, N, C, H, W, s);
     return dtype == KOP_F32 ? launch_bn<float>(x, scale, shift, y, pooled, N, C, H, W, s)
                             : launch_bn<__nv_bfloat16>(x, scale, shift, y, pooled, N, C, H, W, s);
 }

@@ -103,6 +103,11 @@ def test_bn_validation(L):
     assert f(P, Q, Q + 64, R, R + 4096, N, Cc, H, -1, good, good, 0, None) == SHAPE
     assert f(P, Q, Q + 64, R, R + 4096, N, Cc, H, W, nhwc, good, 0, None) == STRIDE
     assert f(P, Q, Q + 64, R, R + 4096, N, Cc, H, W, good, nhwc, 0, None) == STRIDE
+    assert f(P, Q, Q + 64, R, R + 4096, N, Cc, H, W, nhwc, nhwc, 0, None) != STRIDE      # channels-last on both sides
+    padded = (C.c_int64 * 4)(Cc * H * W + 4, H * W, W, 1)
+    assert f(P, Q, Q + 64, R, R + 4096, N, Cc, H, W, padded, padded, 0, None) == STRIDE   # neither dense layout
+    one = (C.c_int64 * 4)(Cc, 1, 77, 99)                                                 # H = W = 1: those strides are unused
+    assert f(P, Q, Q + 64, R, R + 4096, N, Cc, 1, 1, one, one, 0, None) != STRIDE
     assert f(P, Q, Q + 64, R, R + 4096, N, Cc, H, W, good, good, 3, None) == DTYPE
     assert f(P, Q, Q + 64, P + 32, R + 4096, N, Cc, H, W, good, good, 0, None) == ALIAS
     assert f(P, Q + 1, Q + 64, R, R + 4096, N, Cc, H, W, good, good, 0, None) == MISAL

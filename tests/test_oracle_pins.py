@@ -690,3 +690,18 @@ def test_cumsum_closed_forms_library_and_identities():
 
 def math_fsum_rows(a):
     return np.array([math.fsum(r) for r in a])
+
+
+def test_bn_oracle_is_layout_agnostic():
+    """The oracle is defined over (n, c, h, w) indices: a channels-last tensor gives the same values, and
+    both agree with torch in float64 evaluated directly on the NHWC-permuted data."""
+    x = torch.from_numpy(f32(RNG.normal(0, 1, (3, 6, 5, 4))))
+    scale = torch.from_numpy(f32(RNG.uniform(0.5, 1.5, 6)))
+    shift = torch.from_numpy(f32(RNG.normal(0, 0.1, 6)))
+    y0, p0 = kopref.bn_relu_avgpool(x, scale, shift)
+    y1, p1 = kopref.bn_relu_avgpool(x.contiguous(memory_format=torch.channels_last), scale, shift)
+    assert np.array_equal(y0, y1) and np.array_equal(p0, p1)
+    nhwc = x.permute(0, 2, 3, 1).to(torch.float64)                       # [n, h, w, c]
+    a = torch.relu(nhwc * scale.to(torch.float64) + shift.to(torch.float64))
+    np.testing.assert_allclose(y0, a.permute(0, 3, 1, 2).numpy(), rtol=0, atol=1e-15)
+    np.testing.assert_allclose(p0, a.mean(dim=(1, 2)).numpy(), rtol=0, atol=1e-15)

@@ -229,6 +229,65 @@ def test_bn_relu_avgpool_parity(kop, N, C, H, W, dtype, seed):
     pooled.check("bn pooled")
 
 
+BN_NHWC_SHAPES = [
+    (8, 256, 56, 56, F32),     # benchmark image, channels last: 16-vector tiles, rows split over a cluster of 8
+    (120, 256, 24, 24, BF16),  # cluster of 2
+    (3, 64, 28, 28, BF16),     # 8 channel vectors
+    (2, 2048, 7, 7, F32),      # wide and shallow: 16-vector tiles
+    (300, 32, 5, 5, BF16),     # many small images
+    (2, 20, 9, 9, F32),        # 5 vectors: ragged tile
+    (3, 24, 6, 6, BF16),       # 3 vectors
+    (2, 7, 33, 35, F32),       # 7 channels: scalar kernel
+    (2, 33, 4, 4, BF16),       # scalar kernel bf16, two lane tiles
+    (5, 4, 1, 1, F32),
+    (2, 1, 3, 3, F32),         # C == 1: both layouts coincide (takes the NCHW path)
+]
+
+
+@pytest.mark.parametrize("N,C,H,W,dtype", BN_NHWC_SHAPES)
+@pytest.mark.parametrize("seed", SEEDS)
+def test_bn_relu_avgpool_channels_last_parity(kop, N, C, H, W, dtype, seed):
+    x, scale, shift = synth.bn_pool_inputs(N, C, H, W, dtype, seed, "cuda")
+    x = x.contiguous(memory_format=torch.channels_last)
+    buf = Guarded((N, H, W, C), dtype)                       # NHWC memory ...
+    out = buf.t.permute(0, 3, 1, 2)                          # ... addressed as NCHW
+    pooled = Guarded((N, C), F32)
+    kop.kop_bn_relu_avgpool(x, scale, shift, out=out, pooled=pooled.t)
+    ry, rp = kopref.bn_relu_avgpool(host(x), host(scale), host(shift), threads=None)
+    tol = tol_of(dtype)
+    assert_close(out, ry, tol, "bn nhwc y")
+    assert_close(pooled.t, rp, 1e-5, "bn nhwc pooled")
+    if dtype == BF16:
+        assert_bf16_tight(out, ry, "bn nhwc y", floor=1e-6)
+    buf.check("bn nhwc y")
+    pooled.check("bn nhwc pooled")
+
+
+def test_bn_channels_last_full_config_in_place_and_nan(kop):
+    c = synth.CONFIGS["bn_pool"]
+    x, scale, shift = synth.bn_pool_inputs(c["N"], c["C"], c["H"], c["W"], c["dtype"], 0, "cuda")
+    xl = x.contiguous(memory_format=torch.channels_last)
+    y, p = kop.kop_bn_relu_avgpool(xl, scale, shift)
+    assert y.is_contiguous(memory_format=torch.channels_last)
+    # the NCHW kernel on the same logical tensor is an independent GPU path: same values up to sum order
+    y0, p0 = kop.kop_bn_relu_avgpool(x, scale, shift)
+    assert torch.equal(y.contiguous(), y0)
+    assert float((p - p0).abs().max()) < 1e-5
+    ry, rp = kopref.bn_relu_avgpool(host(x[:8]), host(scale), host(shift), threads=None)
+    assert_close(y[:8], ry, 1e-5, "bn nhwc full y (first 8 images)")
+    assert_close(p[:8], rp, 1e-5, "bn nhwc full pooled")
+    y2, p2 = kop.kop_bn_relu_avgpool(xl, scale, shift)
+    assert torch.equal(y, y2) and torch.equal(p, p2)
+    xi = xl[:4].clone(memory_format=torch.channels_last)
+    _, pi = kop.kop_bn_relu_avgpool(xi, scale, shift, out=xi)
+    # (the tile width, hence the summation order, may differ with the batch size: values, not bits)
+    assert torch.equal(xi, y[:4]) and float((pi - p[:4]).abs().max()) < 1e-5
+    xn = xl[:1].clone(memory_format=torch.channels_last)
+    xn[0, 3, 5, 7] = float("nan")
+    yn, pn = kop.kop_bn_relu_avgpool(xn, scale, shift)
+    assert bool(torch.isnan(yn[0, 3, 5, 7])) and bool(torch.isnan(pn[0, 3])) and int(torch.isnan(pn).sum()) == 1
+
+
 def test_bn_full_config_seed0_and_options(kop):
     c = synth.CONFIGS["bn_pool"]
     x, scale, shift = synth.bn_pool_inputs(c["N"], c["C"], c["H"], c["W"], c["dtype"], 0, "cuda")
@@ -249,10 +308,14 @@ def test_bn_full_config_seed0_and_options(kop):
     yn, pn = kop.kop_bn_relu_avgpool(xn, scale, shift)
     assert bool(torch.isnan(yn[0, 3, 5, 7])) and bool(torch.isnan(pn[0, 3]))
     assert int(torch.isnan(pn).sum()) == 1
-    # channels-last strides are rejected, not misread
+    # x and y must share one layout: a channels-last input with an NCHW output is rejected, not misread,
+    # and so is a tensor that is neither (a sliced width)
     with pytest.raises(kop.KopError) as ei:
         kop.kop_bn_relu_avgpool(x[:2].contiguous(memory_format=torch.channels_last), scale, shift,
                                 out=torch.empty_like(x[:2]))
+    assert ei.value.status == 3
+    with pytest.raises(kop.KopError) as ei:
+        kop.kop_bn_relu_avgpool(x[:2, :, :, :48], scale, shift, out=torch.empty_like(x[:2, :, :, :48]))
     assert ei.value.status == 3
     e = torch.empty((0, 256, 56, 56), dtype=F32, device="cuda")
     ye, pe = kop.kop_bn_relu_avgpool(e, scale, shift)
