@@ -91,6 +91,71 @@ bn_plane_warp_kernel(const T* __restrict__ x, const float* __restrict__ scale,
     }
 }
 
+// Small planes (7x7, 14x14, ...: the usual input of a global average pool) are shorter than a warp's
+// worth of vectors and often not a whole number of them, but consecutive planes are contiguous. A CTA
+// therefore takes a run of G planes (G a multiple of the vector length, so every run starts on a 16-byte
+// boundary) as one flat array: 16-byte loads and stores across plane boundaries, the plane of each
+// element found by one small division per vector and carried along it, per-plane scale / shift staged in
+// shared memory, the activations parked in shared memory, and the plane sums taken from there by one
+// warp per plane in a fixed order.
+constexpr int kFlatThreads = 256;
+constexpr int kFlatMaxElems = 4096;                       // activations parked per CTA (16 KB)
+
+template <typename T>
+__global__ void __launch_bounds__(kFlatThreads)
+bn_flat_kernel(const T* __restrict__ x, const float* __restrict__ scale, const float* __restrict__ shift,
+               T* __restrict__ y, float* __restrict__ pooled, int64_t planes, int plane, int G, int C,
+               float inv_plane)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    __shared__ __align__(16) float act[kFlatMaxElems];
+    __shared__ float sc_s[kFlatMaxElems / 4], sh_s[kFlatMaxElems / 4];      // G <= chunk / plane, plane >= 1 ...
+    const int64_t p0 = (int64_t)blockIdx.x * G;
+    const int g_here = (int)(planes - p0 < G ? planes - p0 : G);
+    const int elems = g_here * plane;
+    const T* xc = x + p0 * plane;
+    T* yc = y + p0 * plane;
+    for (int g = threadIdx.x; g < g_here; g += kFlatThreads) {
+        const int c = (int)((p0 + g) % C);
+        sc_s[g] = __ldg(scale + c);
+        sh_s[g] = __ldg(shift + c);
+    }
+    __syncthreads();
+    const float inv = 1.0f / (float)plane;
+    const int nvec = elems / E;
+    for (int v = threadIdx.x; v < nvec; v += kFlatThreads) {
+        float f[E];
+        Elem<T>::unpack(ld_stream(xc + (int64_t)v * E), f);
+        const int i0 = v * E;
+        int pl = (int)((float)i0 * inv);                 // i0 / plane: float estimate, one-step fix-up
+        int rem = i0 - pl * plane;
+        if (rem >= plane) { rem -= plane; ++pl; }
+        if (rem < 0) { rem += plane; --pl; }
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            f[e] = relu_keep_nan(fmaf(f[e], sc_s[pl], sh_s[pl]));
+            act[i0 + e] = f[e];
+            if (++rem == plane) { rem = 0; ++pl; }
+        }
+        st_stream(yc + (int64_t)v * E, Elem<T>::pack(f));
+    }
+    // the last run of the tensor may end inside a vector: its tail goes element by element
+    for (int i = nvec * E + threadIdx.x; i < elems; i += kFlatThreads) {
+        const int pl = i / plane;
+        const float a = relu_keep_nan(fmaf(Elem<T>::load1(xc + i), sc_s[pl], sh_s[pl]));
+        act[i] = a;
+        Elem<T>::store1(yc + i, a);
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int g = warp; g < g_here; g += kFlatThreads / 32) {
+        float s = 0.0f;
+        for (int j = lane; j < plane; j += 32) s += act[g * plane + j];
+        s = warp_sum(s);
+        if (lane == 0) pooled[p0 + g] = s * inv_plane;
+    }
+}
+
 // Large planes that cannot be vectorised: one CTA per plane, scalar loads.
 template <typename T>
 __global__ void __launch_bounds__(256)
@@ -125,6 +190,21 @@ kop_status_t launch_bn(const void* xv, const float* scale, const float* shift, v
     const float inv_plane = (float)(1.0 / (double)plane);
     const bool vec = aligned_to(x, 16) && aligned_to(y, 16) && (plane % E) == 0;
     const int64_t nvec64 = plane / E;
+    // (planes that are whole vectors and at least two warp-loads long do better with a warp each: 14x14
+    // fp32 measured 46 us with the warp kernel against 52 us flat; 7x7 52 us against 40 us flat)
+    if (plane <= 1024 && aligned_to(x, 16) && aligned_to(y, 16) && (plane % E != 0 || plane < 64)) {
+        // G planes per CTA: a multiple of the vector length, about 3K elements, at most 1024 planes
+        int64_t G = (3072 / plane) / E * E;
+        if (G < E) G = E;
+        if (G > 1024) G = 1024;
+        if (G * plane <= kFlatMaxElems) {
+            const int64_t ctas = (planes + G - 1) / G;
+            if (ctas > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+            bn_flat_kernel<T><<<(unsigned)ctas, kFlatThreads, 0, stream>>>(x, scale, shift, y, pooled, planes,
+                                                                          (int)plane, (int)G, (int)C, inv_plane);
+            return launch_status();
+        }
+    }
     if (plane <= 1024 || planes > 0x7FFFFFFFLL) {
         const int64_t ctas = (planes + 7) / 8;
         if (ctas > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;

@@ -208,6 +208,11 @@ BN_SHAPES = [
     (2, 7, 33, 35, F32),       # large odd plane: scalar CTA
     (5, 3, 1, 1, F32),
     (2, 8, 64, 64, BF16),
+    (16, 2048, 7, 7, BF16),    # flat small-plane kernel: many runs of 56 planes
+    (3, 5, 7, 7, BF16),        # one partial run whose last vector is incomplete (735 elements)
+    (2, 3, 31, 31, F32),       # 961-element planes, four per run
+    (7, 9, 3, 3, F32),
+    (2, 1100, 1, 1, BF16),     # one element per plane, runs of 1024 planes
 ]
 
 
