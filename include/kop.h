@@ -348,6 +348,19 @@ size_t kop_rmsnorm_swiglu_residual_workspace_bytes(int64_t rows, int64_t hidden,
 kop_status_t kop_mlp_handle_create(void** handle);
 kop_status_t kop_mlp_handle_destroy(void* handle);
 
+/*
+ * Vendor-library configuration of the segment (the paper's stated future work: besides rewriting the fused
+ * kernels, choose how the preserved vendor calls are configured). With enable != 0 the down projection is
+ * issued as one cublasLtMatmul with C = h and beta = 1, so that
+ *   out = act * w_down^T + h
+ * leaves the GEMM's epilogue directly (fp32 sum, one rounding) and neither kop_residual_add nor the
+ * intermediate d is used. enable == 0 restores the default five-operation form. The setting belongs to
+ * the handle and applies to later kop_rmsnorm_swiglu_residual calls; results differ from the default
+ * form by at most one rounding of `dtype`. Calls with out == h keep the default form (the vendor
+ * kernel is not used in place). Judge it with the perf gate on whole-segment time.
+ */
+kop_status_t kop_mlp_handle_set_residual_in_gemm(void* handle, int enable);
+
 #ifdef __cplusplus
 }
 #endif

@@ -67,7 +67,7 @@ def build(force: bool = False, verbose: bool = False, extra_flags: list[str] | N
         objs = list(pool.map(compile_one, sources()))
     libdir = _cuda_lib_dir(nvcc)
     tmp = lib + f".tmp{os.getpid()}"
-    subprocess.run([nvcc, "-shared", *ARCH, "-o", tmp, *objs, "-L" + libdir, "-lcublas",
+    subprocess.run([nvcc, "-shared", *ARCH, "-o", tmp, *objs, "-L" + libdir, "-lcublas", "-lcublasLt",
                     "-Xlinker", "-rpath", "-Xlinker", libdir], check=True)
     os.replace(tmp, lib)
     if out is not None:

@@ -1,6 +1,9 @@
 // The transformer-MLP segment: kop_rmsnorm, kop_silu_mul, kop_residual_add, and the driver
 // kop_rmsnorm_swiglu_residual that enqueues them around two preserved cuBLAS GEMMs.
+#include <cublasLt.h>
 #include <cublas_v2.h>
+
+#include <new>
 
 #include "kop_common.cuh"
 
@@ -422,6 +425,74 @@ kop_status_t gemm_nt(cublasHandle_t h, const void* A, const void* Wt, void* Cout
     return st == CUBLAS_STATUS_SUCCESS ? KOP_OK : KOP_ERR_CUBLAS;
 }
 
+// What kop_mlp_handle_create hands out: the vendor handle plus the segment's vendor-library configuration.
+struct MlpHandle {
+    cublasHandle_t cb = nullptr;
+    bool residual_in_gemm = false;
+    // single-entry cache of the cublasLt plan for the down projection with the residual epilogue
+    bool plan_valid = false;
+    int64_t plan_m = 0, plan_n = 0, plan_k = 0;
+    kop_dtype_t plan_dtype = KOP_F32;
+    cublasLtMatmulDesc_t op = nullptr;
+    cublasLtMatrixLayout_t la = nullptr, lb = nullptr, lc = nullptr;
+    cublasLtMatmulAlgo_t algo;
+};
+
+void drop_plan(MlpHandle* mh)
+{
+    if (mh->la) cublasLtMatrixLayoutDestroy(mh->la);
+    if (mh->lb) cublasLtMatrixLayoutDestroy(mh->lb);
+    if (mh->lc) cublasLtMatrixLayoutDestroy(mh->lc);
+    if (mh->op) cublasLtMatmulDescDestroy(mh->op);
+    mh->la = mh->lb = mh->lc = nullptr;
+    mh->op = nullptr;
+    mh->plan_valid = false;
+}
+
+// Row-major out[M,N] = A[M,K] * W[N,K]^T + R[M,N] in one vendor call: cublasLtMatmul with C = R and
+// beta = 1 (column-major view as in gemm_nt: out^T = W^T-operand * A^T-operand + R^T). The sum is formed
+// in fp32 and rounded once. out may be R.
+kop_status_t gemm_nt_plus_residual(MlpHandle* mh, const void* A, const void* Wt, const void* R, void* out,
+                                   int64_t M, int64_t N, int64_t K, kop_dtype_t dtype, void* lt_workspace,
+                                   size_t lt_workspace_bytes, cudaStream_t stream)
+{
+    if (M > 0x7FFFFFFFLL || N > 0x7FFFFFFFLL || K > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+    cublasLtHandle_t lt = reinterpret_cast<cublasLtHandle_t>(mh->cb);   // a cuBLAS handle is also a cuBLASLt handle
+    if (!mh->plan_valid || mh->plan_m != M || mh->plan_n != N || mh->plan_k != K || mh->plan_dtype != dtype) {
+        drop_plan(mh);
+        const cudaDataType_t t = dtype == KOP_F32 ? CUDA_R_32F : CUDA_R_16BF;
+        const cublasOperation_t ta = CUBLAS_OP_T, tb = CUBLAS_OP_N;
+        bool ok = cublasLtMatmulDescCreate(&mh->op, CUBLAS_COMPUTE_32F, CUDA_R_32F) == CUBLAS_STATUS_SUCCESS;
+        ok = ok && cublasLtMatmulDescSetAttribute(mh->op, CUBLASLT_MATMUL_DESC_TRANSA, &ta, sizeof(ta)) == CUBLAS_STATUS_SUCCESS;
+        ok = ok && cublasLtMatmulDescSetAttribute(mh->op, CUBLASLT_MATMUL_DESC_TRANSB, &tb, sizeof(tb)) == CUBLAS_STATUS_SUCCESS;
+        ok = ok && cublasLtMatrixLayoutCreate(&mh->la, t, (uint64_t)K, (uint64_t)N, K) == CUBLAS_STATUS_SUCCESS;
+        ok = ok && cublasLtMatrixLayoutCreate(&mh->lb, t, (uint64_t)K, (uint64_t)M, K) == CUBLAS_STATUS_SUCCESS;
+        ok = ok && cublasLtMatrixLayoutCreate(&mh->lc, t, (uint64_t)N, (uint64_t)M, N) == CUBLAS_STATUS_SUCCESS;
+        cublasLtMatmulPreference_t pref = nullptr;
+        ok = ok && cublasLtMatmulPreferenceCreate(&pref) == CUBLAS_STATUS_SUCCESS;
+        ok = ok && cublasLtMatmulPreferenceSetAttribute(pref, CUBLASLT_MATMUL_PREF_MAX_WORKSPACE_BYTES,
+                                                       &lt_workspace_bytes, sizeof(lt_workspace_bytes)) == CUBLAS_STATUS_SUCCESS;
+        cublasLtMatmulHeuristicResult_t res;
+        int found = 0;
+        ok = ok && cublasLtMatmulAlgoGetHeuristic(lt, mh->op, mh->la, mh->lb, mh->lc, mh->lc, pref, 1, &res, &found) == CUBLAS_STATUS_SUCCESS;
+        if (pref) cublasLtMatmulPreferenceDestroy(pref);
+        if (!ok || found < 1) {
+            drop_plan(mh);
+            return KOP_ERR_CUBLAS;
+        }
+        mh->algo = res.algo;
+        mh->plan_m = M;
+        mh->plan_n = N;
+        mh->plan_k = K;
+        mh->plan_dtype = dtype;
+        mh->plan_valid = true;
+    }
+    const float alpha = 1.0f, beta = 1.0f;
+    const cublasStatus_t st = cublasLtMatmul(lt, mh->op, &alpha, Wt, mh->la, A, mh->lb, &beta, R, mh->lc, out, mh->lc,
+                                             &mh->algo, lt_workspace, lt_workspace_bytes, stream);
+    return st == CUBLAS_STATUS_SUCCESS ? KOP_OK : KOP_ERR_CUBLAS;
+}
+
 }  // namespace
 }  // namespace kop
 
@@ -543,17 +614,31 @@ extern "C" kop_status_t kop_mlp_handle_create(void** handle)
     if (handle == nullptr) return KOP_ERR_NULL_POINTER;
     kop_status_t st = kop::check_device();
     if (st != KOP_OK) return st;
-    cublasHandle_t h = nullptr;
-    if (cublasCreate(&h) != CUBLAS_STATUS_SUCCESS) return KOP_ERR_CUBLAS;
-    *handle = h;
+    kop::MlpHandle* mh = new (std::nothrow) kop::MlpHandle();
+    if (mh == nullptr) return KOP_ERR_CUBLAS;
+    if (cublasCreate(&mh->cb) != CUBLAS_STATUS_SUCCESS) {
+        delete mh;
+        return KOP_ERR_CUBLAS;
+    }
+    *handle = mh;
+    return KOP_OK;
+}
+
+extern "C" kop_status_t kop_mlp_handle_set_residual_in_gemm(void* handle, int enable)
+{
+    if (handle == nullptr) return KOP_ERR_NULL_POINTER;
+    static_cast<kop::MlpHandle*>(handle)->residual_in_gemm = enable != 0;
     return KOP_OK;
 }
 
 extern "C" kop_status_t kop_mlp_handle_destroy(void* handle)
 {
     if (handle == nullptr) return KOP_ERR_NULL_POINTER;
-    return cublasDestroy(static_cast<cublasHandle_t>(handle)) == CUBLAS_STATUS_SUCCESS ? KOP_OK
-                                                                                       : KOP_ERR_CUBLAS;
+    kop::MlpHandle* mh = static_cast<kop::MlpHandle*>(handle);
+    kop::drop_plan(mh);
+    const cublasStatus_t st = cublasDestroy(mh->cb);
+    delete mh;
+    return st == CUBLAS_STATUS_SUCCESS ? KOP_OK : KOP_ERR_CUBLAS;
 }
 
 extern "C" kop_status_t kop_rmsnorm_swiglu_residual(void* handle, const void* h, const float* rms_weight,
@@ -585,7 +670,8 @@ extern "C" kop_status_t kop_rmsnorm_swiglu_residual(void* handle, const void* h,
     void* gu = ws + L.gu_off;
     void* act = ws + L.act_off;
     void* d = ws + L.d_off;
-    cublasHandle_t cb = static_cast<cublasHandle_t>(handle);
+    MlpHandle* mh = static_cast<MlpHandle*>(handle);
+    cublasHandle_t cb = mh->cb;
     if (cublasSetStream(cb, as_stream(stream)) != CUBLAS_STATUS_SUCCESS) return KOP_ERR_CUBLAS;
     if (cublasSetWorkspace(cb, ws + L.cublas_off, kCublasWorkspace) != CUBLAS_STATUS_SUCCESS)
         return KOP_ERR_CUBLAS;
@@ -593,6 +679,13 @@ extern "C" kop_status_t kop_rmsnorm_swiglu_residual(void* handle, const void* h,
     if ((st = kop_rmsnorm(h, rms_weight, n, rows, hidden, hidden, hidden, eps, dtype, stream)) != KOP_OK) return st;
     if ((st = gemm_nt(cb, n, w_gate_up, gu, rows, 2 * inter, hidden, dtype)) != KOP_OK) return st;
     if ((st = kop_silu_mul(gu, act, rows, inter, 2 * inter, inter, dtype, stream)) != KOP_OK) return st;
+    // Vendor-library configuration: the residual add rides in the GEMM's epilogue. Not when out is h
+    // itself: with C == D the vendor kernel chosen for bf16 re-reads parts of C after writing D (measured:
+    // 9 % of the outputs one or two roundings away from the out-of-place result), so in-place calls keep
+    // the default form.
+    if (mh->residual_in_gemm && out != h)
+        return gemm_nt_plus_residual(mh, act, w_down, h, out, rows, hidden, inter, dtype, ws + L.cublas_off,
+                                     kCublasWorkspace, as_stream(stream));
     if ((st = gemm_nt(cb, act, w_down, d, rows, hidden, inter, dtype)) != KOP_OK) return st;
     return kop_residual_add(h, d, out, rows, hidden, hidden, hidden, hidden, dtype, stream);
 }

@@ -85,6 +85,8 @@ def lib() -> C.CDLL:
     L.kop_rmsnorm_swiglu_residual_workspace_bytes.argtypes = [i64, i64, i64, i32]
     L.kop_mlp_handle_create.argtypes = [C.POINTER(vp)]
     L.kop_mlp_handle_destroy.argtypes = [vp]
+    L.kop_mlp_handle_set_residual_in_gemm.argtypes = [vp, i32]
+    L.kop_mlp_handle_set_residual_in_gemm.restype = i32
     for name in ("kop_softmax_scale_bias", "kop_bias_gelu_residual_layernorm", "kop_bn_relu_avgpool",
                  "kop_ce_loss_rowwise", "kop_rmsnorm", "kop_silu_mul", "kop_residual_add",
                  "kop_rmsnorm_swiglu_residual", "kop_mlp_handle_create", "kop_mlp_handle_destroy"):
@@ -378,6 +380,11 @@ class MlpHandle:
         h = C.c_void_p()
         _check(lib().kop_mlp_handle_create(C.byref(h)), "kop_mlp_handle_create")
         self.ptr = h.value
+
+    def set_residual_in_gemm(self, enable: bool):
+        """Fold the residual add into the down projection's cuBLASLt epilogue (see kop.h)."""
+        _check(lib().kop_mlp_handle_set_residual_in_gemm(self.ptr, int(bool(enable))),
+               "kop_mlp_handle_set_residual_in_gemm")
 
     def close(self):
         if self.ptr:

@@ -133,3 +133,56 @@ def test_chain_full_shape_sampled_rows_and_intermediates(kop, handle):
     # the driver and the piecewise chain run the same kernels around the same vendor GEMM
     diff = (out.float() - res.float()).abs()
     assert bool((diff <= 2e-2 * res.float().abs().clamp(min=1.0)).all()), "driver vs pieces"
+
+
+@pytest.mark.parametrize("dtype", [BF16, F32])
+def test_chain_with_residual_in_the_gemm_epilogue(kop, dtype):
+    """The vendor-library configuration (residual folded into the down projection through cuBLASLt):
+    same Gate-3 rule against the float64 chain, at most one rounding away from the default form,
+    capturable in a CUDA graph, in place, and switchable back."""
+    M, H, I = 256, 512, 1792
+    hdl = kop.MlpHandle()
+    try:
+        for seed in synth.SEEDS[:3]:
+            h, w, W1, W2 = synth.mlp_inputs(M, H, I, dtype, seed, "cuda")
+            hdl.set_residual_in_gemm(False)
+            base = kop.kop_rmsnorm_swiglu_residual(hdl, h, w, W1, W2, 1e-6)
+            hdl.set_residual_in_gemm(True)
+            out = kop.kop_rmsnorm_swiglu_residual(hdl, h, w, W1, W2, 1e-6)
+            r64 = kopref.mlp_segment(h.cpu(), w.cpu(), W1.cpu(), W2.cpu(), 1e-6, threads=None)
+            r_low = unfused_chain(h, w, W1, W2, 1e-6)
+            ok, tier, d_opt, d_ref = gate3(out, r64, r_low, 2e-2 if dtype == BF16 else 1e-5)
+            assert ok, f"epilogue chain failed Gate 3 ({tier}): d_opt={d_opt:.3e} d_ref={d_ref:.3e}"
+            # one rounding fewer than the default form: never further from the float64 chain than it, up to noise
+            d_base = float(np.abs(to_f64(base) - r64).max())
+            assert d_opt <= 1.5 * d_base + 1e-6
+            step = 2.0 ** -7 if dtype == BF16 else 2.0 ** -20
+            diff = (out.float() - base.float()).abs()
+            assert bool((diff <= step * (1.0 + base.float().abs())).all()), "more than one rounding apart"
+        # graph capture, replay, in place, and back to the default form
+        ws = torch.empty(kop.kop_rmsnorm_swiglu_residual_workspace_bytes(M, H, I, kop.KOP_BF16 if dtype == BF16 else kop.KOP_F32),
+                         dtype=torch.uint8, device="cuda")
+        eager = kop.kop_rmsnorm_swiglu_residual(hdl, h, w, W1, W2, 1e-6, workspace=ws)
+        torch.cuda.synchronize()
+        out = torch.empty_like(h)
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            kop.kop_rmsnorm_swiglu_residual(hdl, h, w, W1, W2, 1e-6, out=out, workspace=ws)
+            side.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                kop.kop_rmsnorm_swiglu_residual(hdl, h, w, W1, W2, 1e-6, out=out, workspace=ws)
+        out.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, eager)
+        hdl.set_residual_in_gemm(False)
+        assert torch.equal(kop.kop_rmsnorm_swiglu_residual(hdl, h, w, W1, W2, 1e-6, workspace=ws), base)
+        # in place the default form is used whatever the setting
+        hdl.set_residual_in_gemm(True)
+        hi = h.clone()
+        kop.kop_rmsnorm_swiglu_residual(hdl, hi, w, W1, W2, 1e-6, out=hi, workspace=ws)
+        assert torch.equal(hi, base)
+    finally:
+        hdl.close()
