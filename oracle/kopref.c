@@ -555,3 +555,52 @@ int kopref_cumsum_rows(const void* x, const unsigned char* mask, double* y, int6
     }
     return 0;
 }
+
+/* ---- per-channel affine + ReLU + windowed 2-D pooling (NCHW): the BatchNorm -> ReLU -> Pool epilogues that
+ * follow the preserved convolutions in the paper's CNN problems ("Pool" is the most frequent non-vendor
+ * operation of its level-2 / level-3 tables). --------------------------------------------------------------
+ *   a[n,c,i,j] = x[n,c,i,j] * scale[c] + shift[c]   (scale / shift NULL: a = x), then ReLU if relu != 0
+ *                (ReLU keeps NaN)
+ *   OH = floor((H + 2 ph - kh) / sh) + 1,  OW likewise
+ *   window of output (oi, oj): rows oi*sh - ph + di, di in [0, kh); columns oj*sw - pw + dj, dj in [0, kw)
+ *   mode 0 (max): y = max of a over the window positions inside the image (padding never wins);
+ *                 a NaN inside the window gives NaN
+ *   mode 1 (avg): y = (sum of a over the window positions inside the image) / (kh * kw)
+ *                 (padding counts as zeros in the divisor)
+ * Requires ph <= kh / 2 and pw <= kw / 2, so that every window touches the image. */
+int kopref_affine_relu_pool2d(const void* x, const float* scale, const float* shift, double* y, int64_t N,
+        int64_t C, int64_t H, int64_t W, int kh, int kw, int sh, int sw, int ph, int pw, int mode, int relu,
+        int dtype, int threads)
+{
+    if (!x || !y || N < 0 || C <= 0 || H <= 0 || W <= 0 || bad_dtype(dtype)) return -1;
+    if (kh <= 0 || kw <= 0 || sh <= 0 || sw <= 0 || ph < 0 || pw < 0 || ph > kh / 2 || pw > kw / 2) return -1;
+    if (H + 2 * ph < kh || W + 2 * pw < kw || (mode != 0 && mode != 1)) return -1;
+    if ((scale == NULL) != (shift == NULL)) return -1;
+    int64_t OH = (H + 2 * ph - kh) / sh + 1, OW = (W + 2 * pw - kw) / sw + 1;
+    int nt = pick_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t p = 0; p < N * C; ++p) {
+        int64_t c = p % C;
+        double sc = scale ? (double)scale[c] : 1.0, sf = shift ? (double)shift[c] : 0.0;
+        for (int64_t oi = 0; oi < OH; ++oi)
+            for (int64_t oj = 0; oj < OW; ++oj) {
+                double best = -INFINITY, sum = 0.0;
+                int saw_nan = 0;
+                for (int di = 0; di < kh; ++di)
+                    for (int dj = 0; dj < kw; ++dj) {
+                        int64_t i = oi * sh - ph + di, j = oj * sw - pw + dj;
+                        if (i < 0 || i >= H || j < 0 || j >= W) continue;
+                        double a = load_elem(x, (p * H + i) * W + j, dtype);
+                        if (scale) a = a * sc + sf;
+                        if (relu) a = (a != a) ? a : (a > 0.0 ? a : 0.0);
+                        if (a != a) saw_nan = 1;
+                        if (a > best) best = a;
+                        sum += a;
+                    }
+                double out = mode == 0 ? (saw_nan ? NAN : best) : sum / (double)(kh * kw);
+                y[(p * OH + oi) * OW + oj] = out;
+            }
+    }
+    return 0;
+}

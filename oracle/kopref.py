@@ -45,6 +45,7 @@ def lib() -> C.CDLL:
         _lib.kopref_ce_loss_opts.argtypes = [vp] * 6 + [i64] * 3 + [C.c_int32, dbl, C.c_int, C.c_int]
         _lib.kopref_groupnorm_act.argtypes = [vp] * 6 + [i64] * 5 + [dbl, C.c_int, C.c_int, C.c_int]
         _lib.kopref_row_scale.argtypes = [vp, vp, vp, i64, i64, i64, i64, C.c_int, C.c_int]
+        _lib.kopref_affine_relu_pool2d.argtypes = [vp] * 4 + [i64] * 4 + [C.c_int] * 10
         _lib.kopref_cumsum_rows.argtypes = [vp, vp, vp] + [i64] * 5 + [C.c_int] * 4
         _lib.kopref_matvec_bias.argtypes = [vp, vp, dbl, vp, i64, i64, i64, C.c_int, C.c_int]
     return _lib
@@ -294,6 +295,21 @@ def matvec_bias(x, w, b_sum, threads=1) -> np.ndarray:
     out = np.empty(M, dtype=np.float64)
     _check(lib().kopref_matvec_bias(_p(xa), _p(wa), float(b_sum), _p(out), M, K, K, dt, _nt(threads)), "matvec_bias")
     return out
+
+
+def affine_relu_pool2d(x, scale, shift, kernel, stride, padding, mode="max", relu=True, threads=1) -> np.ndarray:
+    """Per-channel affine (scale / shift both None: none) + optional ReLU + max / avg pooling over windows.
+    kernel, stride, padding: (h, w) pairs. x is NCHW contiguous. Returns y[N, C, OH, OW]."""
+    xa, dt = as_data(x)
+    N, Cc, H, W = xa.shape
+    sc, sh = as_param(scale), as_param(shift)
+    (kh, kw), (sth, stw), (ph, pw) = kernel, stride, padding
+    OH, OW = (H + 2 * ph - kh) // sth + 1, (W + 2 * pw - kw) // stw + 1
+    y = np.empty((N, Cc, OH, OW), dtype=np.float64)
+    _check(lib().kopref_affine_relu_pool2d(_p(xa), _p(sc), _p(sh), _p(y), N, Cc, H, W, kh, kw, sth, stw, ph, pw,
+                                           {"max": 0, "avg": 1}[mode], int(bool(relu)), dt, _nt(threads)),
+           "affine_relu_pool2d")
+    return y
 
 
 def cumsum_rows(x, mask=None, exclusive=False, reverse=False, threads=1) -> np.ndarray:

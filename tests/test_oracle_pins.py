@@ -705,3 +705,55 @@ def test_bn_oracle_is_layout_agnostic():
     a = torch.relu(nhwc * scale.to(torch.float64) + shift.to(torch.float64))
     np.testing.assert_allclose(y0, a.permute(0, 3, 1, 2).numpy(), rtol=0, atol=1e-15)
     np.testing.assert_allclose(p0, a.mean(dim=(1, 2)).numpy(), rtol=0, atol=1e-15)
+
+
+# --------------------------------------------------------------------------- affine + ReLU + windowed pooling
+
+def test_pool2d_library_closed_forms_and_special_cases():
+    x = torch.from_numpy(f32(RNG.normal(0, 1, (2, 3, 11, 13))))
+    scale = torch.from_numpy(f32(RNG.uniform(0.5, 1.5, 3)))
+    shift = torch.from_numpy(f32(RNG.normal(0, 0.3, 3)))
+    xd = x.to(torch.float64)
+    a = torch.relu(xd * scale.to(torch.float64)[None, :, None, None] + shift.to(torch.float64)[None, :, None, None])
+    for k, s, p in [((3, 3), (2, 2), (1, 1)), ((2, 2), (2, 2), (0, 0)), ((3, 2), (1, 3), (1, 0)), ((5, 5), (1, 1), (2, 2)),
+                    ((1, 1), (1, 1), (0, 0)), ((11, 13), (1, 1), (0, 0))]:
+        # library routines in float64 (torch pads max pooling with -inf and averages with padding counted)
+        np.testing.assert_allclose(kopref.affine_relu_pool2d(x, scale, shift, k, s, p, "max", True),
+                                   F.max_pool2d(a, k, s, p).numpy(), rtol=0, atol=1e-15)
+        np.testing.assert_allclose(kopref.affine_relu_pool2d(x, scale, shift, k, s, p, "avg", True),
+                                   F.avg_pool2d(a, k, s, p, count_include_pad=True).numpy(), rtol=0, atol=1e-14)
+        # no affine, no ReLU: plain pooling of x
+        np.testing.assert_allclose(kopref.affine_relu_pool2d(x, None, None, k, s, p, "max", False),
+                                   F.max_pool2d(xd, k, s, p).numpy(), rtol=0, atol=0)
+        np.testing.assert_allclose(kopref.affine_relu_pool2d(x, None, None, k, s, p, "avg", False),
+                                   F.avg_pool2d(xd, k, s, p, count_include_pad=True).numpy(), rtol=0, atol=1e-14)
+    # special cases: a 1x1 window is the activation itself; a window covering the image is the global pool
+    one = kopref.affine_relu_pool2d(x, scale, shift, (1, 1), (1, 1), (0, 0), "max", True)
+    np.testing.assert_allclose(one, a.numpy(), rtol=0, atol=1e-15)
+    _, pooled = kopref.bn_relu_avgpool(x, scale, shift)
+    full = kopref.affine_relu_pool2d(x, scale, shift, (11, 13), (1, 1), (0, 0), "avg", True)
+    np.testing.assert_allclose(full[:, :, 0, 0], pooled, rtol=0, atol=1e-14)
+    # closed forms: a ramp along w, 2x2 windows of stride 2: max picks the right column, avg the midpoint
+    ramp = torch.arange(16, dtype=torch.float32).repeat(1, 1, 4, 1)                  # [1,1,4,16], value = column
+    assert np.array_equal(kopref.affine_relu_pool2d(ramp, None, None, (2, 2), (2, 2), (0, 0), "max", False)[0, 0, 0],
+                          np.arange(1, 16, 2, dtype=np.float64))
+    assert np.array_equal(kopref.affine_relu_pool2d(ramp, None, None, (2, 2), (2, 2), (0, 0), "avg", False)[0, 0, 1],
+                          np.arange(0.5, 16, 2))
+    # padding never wins a max (all-negative input keeps its own maximum) and counts as zeros in an average
+    neg = torch.full((1, 1, 4, 4), -3.0)
+    assert np.array_equal(kopref.affine_relu_pool2d(neg, None, None, (3, 3), (2, 2), (1, 1), "max", False),
+                          np.full((1, 1, 2, 2), -3.0))
+    corner = kopref.affine_relu_pool2d(torch.ones((1, 1, 4, 4)), None, None, (3, 3), (2, 2), (1, 1), "avg", False)
+    assert corner[0, 0, 0, 0] == 4.0 / 9.0 and corner[0, 0, 1, 1] == 1.0
+    # NaN: poisons exactly the windows that contain it
+    xn = x.clone()
+    xn[0, 1, 4, 6] = float("nan")
+    ym = kopref.affine_relu_pool2d(xn, scale, shift, (3, 3), (2, 2), (1, 1), "max", True)
+    assert {tuple(t) for t in np.argwhere(np.isnan(ym))} == {(0, 1, 2, 3)}      # rows 3..5, columns 5..7
+    ref_nan = torch.isnan(F.max_pool2d(torch.relu(xn.double() * scale.double()[None, :, None, None]
+                                                  + shift.double()[None, :, None, None]), 3, 2, 1)).numpy()
+    assert np.array_equal(np.isnan(ym), ref_nan)
+    # bf16 input and threads
+    xb = x.to(torch.bfloat16)
+    np.testing.assert_allclose(kopref.affine_relu_pool2d(xb, None, None, (3, 3), (2, 2), (1, 1), "max", False, threads=3),
+                               F.max_pool2d(xb.double(), 3, 2, 1).numpy(), rtol=0, atol=0)
