@@ -95,6 +95,11 @@ def segment_bytes():
     e = q["N"] * q["C"] * q["H"] * q["W"]
     out["groupnorm"] = dict(bytes=2 * e * 4 + 2 * q["C"] * 4 + 2 * q["N"] * q["groups"] * 4, elems=e)
     out["bn_pool_nhwc"] = dict(out["bn_pool"])
+    q = c["pool2d"]
+    e_in = q["N"] * q["C"] * q["H"] * q["W"]
+    e_out = q["N"] * q["C"] * ((q["H"] + 2 * q["padding"][0] - q["kernel"][0]) // q["stride"][0] + 1) * \
+        ((q["W"] + 2 * q["padding"][1] - q["kernel"][1]) // q["stride"][1] + 1)
+    out["pool2d"] = dict(bytes=(e_in + e_out) * 4 + 2 * q["C"] * 4, elems=e_in)
     u = c["cumsum"]
     out["cumsum"] = dict(bytes=2 * u["rows"] * u["cols"] * 4, elems=u["rows"] * u["cols"])
     return out
@@ -240,7 +245,7 @@ class Workload:
 
     ORDER = ["softmax_small", "softmax_large", "layernorm", "bn_pool", "ce_loss", "rmsnorm", "silu_mul", "residual_add"]
     # Beyond the benchmark configs (not part of `value`): the two kernels the paper's case studies print.
-    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc"]
+    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc", "pool2d"]
 
     def __init__(self, kop, device, seed, only=None, rows_div=1):
         """only: build just these segments (None = all, plus the MLP segment); rows_div cuts the row
@@ -303,6 +308,12 @@ class Workload:
             del hx
             self.hy = torch.empty_like(self.hx)
             self.hp = torch.empty((self.hx.shape[0], b["C"]), dtype=torch.float32, device=dev)
+        if "pool2d" in want:
+            q = c["pool2d"]
+            self.px, self.pscale, self.pshift = synth.bn_pool_inputs(cut(q["N"]), q["C"], q["H"], q["W"], q["dtype"], seed, dev)
+            oh = (q["H"] + 2 * q["padding"][0] - q["kernel"][0]) // q["stride"][0] + 1
+            ow = (q["W"] + 2 * q["padding"][1] - q["kernel"][1]) // q["stride"][1] + 1
+            self.py = torch.empty((self.px.shape[0], q["C"], oh, ow), dtype=q["dtype"], device=dev)
         if "cumsum" in want:
             u = c["cumsum"]
             self.ux, _ = synth.cumsum_inputs(cut(u["rows"]), u["cols"], u["dtype"], seed, dev)
@@ -373,6 +384,10 @@ class Workload:
                                 mean=self.qmean, rstd=self.qrstd)
         elif name == "bn_pool_nhwc":             # the BN + ReLU + pool config in channels-last memory
             k.kop_bn_relu_avgpool(self.hx, self.hscale, self.hshift, out=self.hy, pooled=self.hp)
+        elif name == "pool2d":                   # BN affine + ReLU + 3x3 / stride-2 max pool, fp32 [64,64,112,112]
+            q = c["pool2d"]
+            k.kop_affine_relu_pool2d(self.px, self.pscale, self.pshift, q["kernel"], q["stride"], q["padding"],
+                                     q["mode"], True, out=self.py)
         elif name == "cumsum":                   # inclusive running sum along rows, fp32 [32768, 4096]
             k.kop_cumsum_rows(self.ux, out=self.uy)
         else:

@@ -287,6 +287,24 @@ kop_status_t kop_groupnorm_act(const void* x, const float* gamma, const float* b
                                int64_t groups, float eps, int act, kop_dtype_t dtype, kop_stream_t stream);
 
 /*
+ * Per-channel affine, optional ReLU and windowed 2-D pooling in one pass over NCHW planes (the BatchNorm ->
+ * ReLU -> Pool epilogues after the preserved convolutions of the paper's CNN problems; "Pool" is the most
+ * frequent non-vendor operation of its level-2 / level-3 result tables; fusion agent: pointwise + reduction):
+ *   a[n,c,i,j] = x[n,c,i,j] * scale[c] + shift[c]  (scale and shift both NULL: a = x), ReLU if relu != 0
+ *   OH = floor((H + 2 ph - kh) / sh) + 1,  OW = floor((W + 2 pw - kw) / sw) + 1
+ *   mode 0: y[n,c,oi,oj] = max of a over rows oi*sh - ph + [0, kh), columns oj*sw - pw + [0, kw) that lie
+ *           inside the image (padding never wins; a NaN inside the window gives NaN)
+ *   mode 1: y = (sum of a over the same positions) / (kh * kw)      (padding counts in the divisor)
+ * x: [N, C, H, W] contiguous, y: [N, C, OH, OW] contiguous, both of `dtype`; scale, shift: fp32 [C] or both
+ * NULL. Requires ph <= kh / 2 and pw <= kw / 2 (every window touches the image), H + 2 ph >= kh,
+ * W + 2 pw >= kw; otherwise KOP_ERR_BAD_SHAPE. The activation a is never written to memory. y must not
+ * overlap x.
+ */
+kop_status_t kop_affine_relu_pool2d(const void* x, const float* scale, const float* shift, void* y,
+                                    int64_t N, int64_t C, int64_t H, int64_t W, int kh, int kw, int sh, int sw,
+                                    int ph, int pw, int mode, int relu, kop_dtype_t dtype, kop_stream_t stream);
+
+/*
  * Running sums along each row (the CumSum rows of the paper's per-kernel results table, L1-089 to L1-093:
  * plain, reverse, exclusive and masked cumulative sums; planner strategy "single-pass reductions" applied
  * to a scan). With m[i,k] = 1 when mask is NULL, else (mask[i,k] != 0):

@@ -1,0 +1,283 @@
+// kop_affine_relu_pool2d: per-channel affine (folded BatchNorm), optional ReLU and windowed max / average
+// pooling over NCHW planes in one pass: the activation is never written to memory, only the pooled map is.
+//
+// A CTA owns a band of output rows of one (n, c) plane. The input rows the band needs are contiguous in
+// memory, so they are fetched once with flat 16-byte loads, turned into fp32 activations and parked in a
+// shared-memory tile that already contains the padding (-inf for max, 0 for average): the windows are then
+// read from shared memory without bounds checks, and overlapping windows cost no extra HBM traffic (only
+// the kh - sh halo rows between bands are read twice). Bands are sized to about 24 KB of tile so that
+// several CTAs share an SM and overlap their phases.
+#include "kop_common.cuh"
+
+namespace kop {
+namespace {
+
+constexpr int kPoolThreads = 256;
+constexpr int kPoolTileBytes = 24 * 1024;       // preferred tile size
+constexpr int kPoolTileMax = 46 * 1024;         // static + dynamic shared memory stays under the 48 KB default
+
+// max that returns NaN when either operand is NaN: one instruction
+__device__ __forceinline__ float max_keep_nan(float m, float a)
+{
+    float r;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(m), "f"(a));
+    return r;
+}
+
+// i / d for 0 <= i < 2^22 without an integer division: float estimate, one-step fix-up
+__device__ __forceinline__ int div_small(int i, int d, float inv_d)
+{
+    int q = (int)((float)i * inv_d);
+    const int r = i - q * d;
+    q += (r >= d) ? 1 : 0;
+    q -= (r < 0) ? 1 : 0;
+    return q;
+}
+
+__device__ __forceinline__ float act_of(float v, float sc, float sf, int relu)
+{
+    v = fmaf(v, sc, sf);
+    return relu ? (v > 0.0f ? v : (v <= 0.0f ? 0.0f : v)) : v;
+}
+
+// Tile geometry shared by host and device: image column 0 sits at tile column `lead` (the left padding
+// rounded up to four floats, so that staged rows start 16-byte aligned and take 128-bit shared-memory
+// stores); a tile row holds lead + W + pw floats, rounded up to four.
+__host__ __device__ __forceinline__ int pool_lead(int pw) { return (pw + 3) / 4 * 4; }
+__host__ __device__ __forceinline__ int pool_row_floats(int W, int pw) { return (pool_lead(pw) + W + pw + 3) / 4 * 4; }
+
+// MODE 0 max, 1 average. KS / ST: compile-time square window and stride (0 = use the runtime values).
+// Consecutive threads take consecutive outputs: their windows start sw floats apart in shared memory (a
+// 2-way bank conflict at stride 2 instead of the 8-way one of a vector of outputs per thread), and a warp's
+// 32 scalar stores still make one contiguous run.
+template <typename T, int MODE, int KS, int ST, bool kVecIn>
+__global__ void __launch_bounds__(kPoolThreads)
+pool2d_tile_kernel(const T* __restrict__ x, const float* __restrict__ scale, const float* __restrict__ shift,
+                   T* __restrict__ y, int C, int H, int W, int OH, int OW, int kh_, int kw_, int sh_, int sw_,
+                   int ph, int pw, int band_rows, int bands, int relu, float inv_area)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    extern __shared__ __align__(16) float tile[];
+    const int kh = KS ? KS : kh_, kw = KS ? KS : kw_, sh = ST ? ST : sh_, sw = ST ? ST : sw_;
+    const int64_t plane = blockIdx.x / bands;
+    const int band = (int)(blockIdx.x - plane * bands);
+    const int c = (int)(plane % C);
+    const float sc = scale != nullptr ? __ldg(scale + c) : 1.0f;
+    const float sf = shift != nullptr ? __ldg(shift + c) : 0.0f;
+    const float pad = MODE == 0 ? -INFINITY : 0.0f;
+
+    const int oh0 = band * band_rows;
+    const int oh1 = min(OH, oh0 + band_rows);
+    const int t0 = oh0 * sh - ph;                            // first tile row, in image coordinates (may be < 0)
+    const int trows = (oh1 - 1 - oh0) * sh + kh;             // tile rows
+    const int lead = pool_lead(pw), Ws = pool_row_floats(W, pw);
+    const int i0 = max(t0, 0), i1 = min(t0 + trows, H);      // image rows present in the tile
+
+    // 1. padding cells only: whole rows above / below the image, then the pw cells left and right of the rest
+    const int top = i0 - t0, bottom = t0 + trows - i1;       // padding rows in the tile (each 0 .. ph)
+    for (int k = threadIdx.x; k < (top + bottom) * Ws; k += kPoolThreads) {
+        const int r = k < top * Ws ? 0 : (i1 - t0) - top;    // rows [0, top) and [i1 - t0, trows)
+        tile[r * Ws + k] = pad;
+    }
+    for (int k = threadIdx.x; k < (i1 - i0) * 2 * pw; k += kPoolThreads) {
+        const int r = k / (2 * pw), m = k - r * 2 * pw;
+        tile[(top + r) * Ws + (m < pw ? lead - pw + m : lead + W + m - pw)] = pad;
+    }
+    // 2. the band's input rows: one contiguous run of (i1 - i0) * W elements
+    const T* xp = x + (plane * H + i0) * (int64_t)W;
+    const int n_in = (i1 - i0) * W;
+    if (kVecIn) {
+        const float inv_w = 1.0f / (float)W;
+        for (int v = threadIdx.x; v < n_in / E; v += kPoolThreads) {
+            float f[E];
+            Elem<T>::unpack(ld_stream(xp + (int64_t)v * E), f);
+            const int idx = v * E;
+            const int r = div_small(idx, W, inv_w), cc = idx - r * W;   // W % E == 0: a vector stays inside one row
+            float4* dst = reinterpret_cast<float4*>(tile + (top + r) * Ws + lead + cc);     // 16-byte aligned
+#pragma unroll
+            for (int q = 0; q < E / 4; ++q)
+                dst[q] = make_float4(act_of(f[4 * q], sc, sf, relu), act_of(f[4 * q + 1], sc, sf, relu),
+                                     act_of(f[4 * q + 2], sc, sf, relu), act_of(f[4 * q + 3], sc, sf, relu));
+        }
+    } else {
+        for (int idx = threadIdx.x; idx < n_in; idx += kPoolThreads) {
+            const int r = idx / W, cc = idx - r * W;
+            tile[(top + r) * Ws + lead + cc] = act_of(Elem<T>::load1(xp + idx), sc, sf, relu);
+        }
+    }
+    __syncthreads();
+    // 3. windows out of the tile; the band's outputs are one contiguous run of (oh1 - oh0) * OW elements
+    T* yp = y + (plane * OH + oh0) * (int64_t)OW;
+    const int n_out = (oh1 - oh0) * OW;
+    const float inv_ow = 1.0f / (float)OW;
+    const float* origin = tile + (lead - pw);
+    for (int o = threadIdx.x; o < n_out; o += kPoolThreads) {
+        const int orow = div_small(o, OW, inv_ow), ocol = o - orow * OW;
+        const float* win = origin + orow * sh * Ws + ocol * sw;
+        float res = MODE == 0 ? -INFINITY : 0.0f;
+        if (KS) {
+#pragma unroll
+            for (int di = 0; di < (KS ? KS : 1); ++di)
+#pragma unroll
+                for (int dj = 0; dj < (KS ? KS : 1); ++dj) {
+                    const float a = win[di * Ws + dj];
+                    res = MODE == 0 ? max_keep_nan(res, a) : res + a;
+                }
+        } else {
+            for (int di = 0; di < kh; ++di)
+                for (int dj = 0; dj < kw; ++dj) {
+                    const float a = win[di * Ws + dj];
+                    res = MODE == 0 ? max_keep_nan(res, a) : res + a;
+                }
+        }
+        Elem<T>::store1(yp + o, MODE == 1 ? res * inv_area : res);
+    }
+}
+
+// Any geometry (rows too wide for the tile): one thread per output, window read from global memory.
+template <typename T>
+__global__ void __launch_bounds__(256)
+pool2d_direct_kernel(const T* __restrict__ x, const float* __restrict__ scale, const float* __restrict__ shift,
+                     T* __restrict__ y, int64_t total, int C, int H, int W, int OH, int OW, int kh, int kw, int sh,
+                     int sw, int ph, int pw, int mode, int relu, float inv_area)
+{
+    for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
+        const int oj = (int)(o % OW);
+        const int oi = (int)((o / OW) % OH);
+        const int64_t plane = o / ((int64_t)OW * OH);
+        const int c = (int)(plane % C);
+        const float sc = scale != nullptr ? __ldg(scale + c) : 1.0f;
+        const float sf = shift != nullptr ? __ldg(shift + c) : 0.0f;
+        const T* xp = x + plane * H * (int64_t)W;
+        float res = mode == 0 ? -INFINITY : 0.0f;
+        for (int di = 0; di < kh; ++di) {
+            const int i = oi * sh - ph + di;
+            if (i < 0 || i >= H) continue;
+            for (int dj = 0; dj < kw; ++dj) {
+                const int j = oj * sw - pw + dj;
+                if (j < 0 || j >= W) continue;
+                const float a = act_of(Elem<T>::load1(xp + (int64_t)i * W + j), sc, sf, relu);
+                res = mode == 0 ? max_keep_nan(res, a) : res + a;
+            }
+        }
+        Elem<T>::store1(y + o, mode == 0 ? res : res * inv_area);
+    }
+}
+
+template <typename T, int MODE, int KS, int ST>
+void launch_tile(bool vin, unsigned grid, size_t smem, cudaStream_t stream, const T* x, const float* scale,
+                 const float* shift, T* y, int C, int H, int W, int OH, int OW, int kh, int kw, int sh, int sw, int ph,
+                 int pw, int band_rows, int bands, int relu, float inv_area)
+{
+    if (vin)
+        pool2d_tile_kernel<T, MODE, KS, ST, true><<<grid, kPoolThreads, smem, stream>>>(
+            x, scale, shift, y, C, H, W, OH, OW, kh, kw, sh, sw, ph, pw, band_rows, bands, relu, inv_area);
+    else
+        pool2d_tile_kernel<T, MODE, KS, ST, false><<<grid, kPoolThreads, smem, stream>>>(
+            x, scale, shift, y, C, H, W, OH, OW, kh, kw, sh, sw, ph, pw, band_rows, bands, relu, inv_area);
+}
+
+template <typename T>
+kop_status_t launch_pool(const void* xv, const float* scale, const float* shift, void* yv, int64_t N, int64_t C,
+                         int H, int W, int OH, int OW, int kh, int kw, int sh, int sw, int ph, int pw, int mode,
+                         int relu, cudaStream_t stream)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    const T* x = static_cast<const T*>(xv);
+    T* y = static_cast<T*>(yv);
+    const float inv_area = (float)(1.0 / ((double)kh * kw));
+    const int64_t planes = N * C;
+    const int64_t row_bytes = (int64_t)pool_row_floats(W, pw) * 4;
+    if ((int64_t)kh * row_bytes <= kPoolTileMax) {
+        // output rows per band: about kPoolTileBytes of tile, at least one row, then evened out
+        int64_t br = ((int64_t)kPoolTileBytes / row_bytes - kh) / sh + 1;
+        if (br < 1) br = 1;
+        while (br > 1 && ((br - 1) * sh + kh) * row_bytes > kPoolTileMax) --br;
+        if (br > OH) br = OH;
+        {
+            // among band heights down to half of that, take the one whose outputs fill the CTA's passes best
+            const int64_t per_row = OW;
+            int64_t best = br;
+            double best_util = 0.0;
+            for (int64_t cand = br; cand >= 1 && cand * 2 >= br; --cand) {
+                const int64_t n = cand * per_row;
+                const double util = (double)n / (double)((n + kPoolThreads - 1) / kPoolThreads * kPoolThreads);
+                if (util > best_util + 1e-9) {
+                    best_util = util;
+                    best = cand;
+                }
+            }
+            br = best;
+        }
+        const int bands = (int)((OH + br - 1) / br);
+        const size_t smem = (size_t)(((br - 1) * sh + kh) * row_bytes);
+        const int64_t grid = planes * bands;
+        if (grid <= 0x7FFFFFFFLL && smem <= (size_t)kPoolTileMax) {
+            // flat vector loads need every band to start on a 16-byte boundary: rows that are whole vectors
+            const bool vin = aligned_to(x, 16) && W % E == 0;
+            const unsigned g = (unsigned)grid;
+#define KOP_POOL_ARGS vin, g, smem, stream, x, scale, shift, y, (int)C, H, W, OH, OW, kh, kw, sh, sw, ph, pw, (int)br, bands, relu, inv_area
+            const bool square = kh == kw && sh == sw;
+            if (mode == 0) {
+                if (square && kh == 3 && sh == 2) launch_tile<T, 0, 3, 2>(KOP_POOL_ARGS);
+                else if (square && kh == 2 && sh == 2) launch_tile<T, 0, 2, 2>(KOP_POOL_ARGS);
+                else if (square && kh == 3 && sh == 1) launch_tile<T, 0, 3, 1>(KOP_POOL_ARGS);
+                else launch_tile<T, 0, 0, 0>(KOP_POOL_ARGS);
+            } else {
+                if (square && kh == 3 && sh == 2) launch_tile<T, 1, 3, 2>(KOP_POOL_ARGS);
+                else if (square && kh == 2 && sh == 2) launch_tile<T, 1, 2, 2>(KOP_POOL_ARGS);
+                else if (square && kh == 3 && sh == 1) launch_tile<T, 1, 3, 1>(KOP_POOL_ARGS);
+                else launch_tile<T, 1, 0, 0>(KOP_POOL_ARGS);
+            }
+#undef KOP_POOL_ARGS
+            return launch_status();
+        }
+    }
+    const int64_t total = planes * OH * OW;
+    int64_t blocks = (total + 255) / 256;
+    const int64_t cap = 32LL * sm_count();
+    if (blocks > cap) blocks = cap;
+    pool2d_direct_kernel<T><<<(unsigned)blocks, 256, 0, stream>>>(x, scale, shift, y, total, (int)C, H, W, OH, OW, kh,
+                                                                   kw, sh, sw, ph, pw, mode, relu, inv_area);
+    return launch_status();
+}
+
+}  // namespace
+}  // namespace kop
+
+extern "C" kop_status_t kop_affine_relu_pool2d(const void* x, const float* scale, const float* shift, void* y,
+                                               int64_t N, int64_t C, int64_t H, int64_t W, int kh, int kw, int sh,
+                                               int sw, int ph, int pw, int mode, int relu, kop_dtype_t dtype,
+                                               kop_stream_t stream)
+{
+    using namespace kop;
+    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    if (N < 0 || C <= 0 || H <= 0 || W <= 0) return KOP_ERR_BAD_SHAPE;
+    if (kh <= 0 || kw <= 0 || sh <= 0 || sw <= 0 || ph < 0 || pw < 0 || ph > kh / 2 || pw > kw / 2)
+        return KOP_ERR_BAD_SHAPE;
+    if (mode != 0 && mode != 1) return KOP_ERR_BAD_SHAPE;
+    if (C > 0x7FFFFFFF || H > 0x3FFFFFFF || W > 0x3FFFFFFF || N > kMaxElems) return KOP_ERR_BAD_SHAPE;
+    if (kh > 0xFFFF || kw > 0xFFFF || H + 2 * (int64_t)ph < kh || W + 2 * (int64_t)pw < kw) return KOP_ERR_BAD_SHAPE;
+    if (H > kMaxElems / W || C > kMaxElems / (H * W)) return KOP_ERR_BAD_SHAPE;
+    if (N == 0) return KOP_OK;
+    if (C * H * W > kMaxElems / N) return KOP_ERR_BAD_SHAPE;
+    if (!x || !y) return KOP_ERR_NULL_POINTER;
+    if ((scale == nullptr) != (shift == nullptr)) return KOP_ERR_NULL_POINTER;      // both or neither
+    const int esz = elem_size(dtype);
+    if (!aligned_to(x, esz) || !aligned_to(y, esz) || (scale && !aligned_to(scale, 4)) || (shift && !aligned_to(shift, 4)))
+        return KOP_ERR_MISALIGNED;
+    const int64_t OH = (H + 2 * (int64_t)ph - kh) / sh + 1, OW = (W + 2 * (int64_t)pw - kw) / sw + 1;
+    {
+        // the output has another shape: it must not overlap the input at all
+        const uintptr_t a0 = reinterpret_cast<uintptr_t>(x), a1 = a0 + (uintptr_t)(N * C * H * W * esz);
+        const uintptr_t b0 = reinterpret_cast<uintptr_t>(y), b1 = b0 + (uintptr_t)(N * C * OH * OW * esz);
+        if (!(a1 <= b0 || b1 <= a0)) return KOP_ERR_BAD_ALIAS;
+    }
+    kop_status_t st = check_device();
+    if (st != KOP_OK) return st;
+    cudaStream_t s = as_stream(stream);
+    return dtype == KOP_F32 ? launch_pool<float>(x, scale, shift, y, N, C, (int)H, (int)W, (int)OH, (int)OW, kh, kw, sh,
+                                                 sw, ph, pw, mode, relu != 0, s)
+                            : launch_pool<__nv_bfloat16>(x, scale, shift, y, N, C, (int)H, (int)W, (int)OH, (int)OW, kh,
+                                                         kw, sh, sw, ph, pw, mode, relu != 0, s);
+}

@@ -76,6 +76,8 @@ def lib() -> C.CDLL:
     L.kop_matvec_bias.restype = i32
     L.kop_groupnorm_act.argtypes = [vp] * 6 + [i64] * 5 + [f32, i32, i32, vp]
     L.kop_groupnorm_act.restype = i32
+    L.kop_affine_relu_pool2d.argtypes = [vp] * 4 + [i64] * 4 + [i32] * 9 + [vp]
+    L.kop_affine_relu_pool2d.restype = i32
     L.kop_cumsum_rows.argtypes = [vp, vp, vp] + [i64] * 5 + [i32, i32, i32, vp]
     L.kop_cumsum_rows.restype = i32
     L.kop_groupnorm_wait_timeouts.argtypes = [C.POINTER(C.c_uint)]
@@ -346,6 +348,23 @@ def kop_groupnorm_act(x, gamma, beta, groups, eps, act=0, out=None, mean=None, r
                                    None if rstd is None else rstd.data_ptr(), N, Cc, H, W, int(groups),
                                    float(eps), int(act), _dtype_tag(x), _stream(stream)), "kop_groupnorm_act")
     return out, mean, rstd
+
+
+def kop_affine_relu_pool2d(x, scale, shift, kernel, stride, padding, mode="max", relu=True, out=None, stream=None):
+    """kernel, stride, padding: (h, w) pairs; mode "max" or "avg"; scale / shift both None for plain pooling."""
+    if x.dim() != 4 or not x.is_cuda or not x.is_contiguous():
+        raise ValueError("x: expected a contiguous 4-D NCHW CUDA tensor")
+    N, Cc, H, W = x.shape
+    (kh, kw), (sh, sw), (ph, pw) = kernel, stride, padding
+    OH, OW = (H + 2 * ph - kh) // sh + 1, (W + 2 * pw - kw) // sw + 1
+    out = torch.empty((N, Cc, max(OH, 0), max(OW, 0)), dtype=x.dtype, device=x.device) if out is None else out
+    if out.dtype != x.dtype or not out.is_contiguous():
+        raise ValueError("out: expected a contiguous tensor of x's dtype")
+    _check(lib().kop_affine_relu_pool2d(x.data_ptr(), _param(scale, "scale", Cc), _param(shift, "shift", Cc),
+                                        out.data_ptr(), N, Cc, H, W, kh, kw, sh, sw, ph, pw,
+                                        {"max": 0, "avg": 1}[mode], int(bool(relu)), _dtype_tag(x), _stream(stream)),
+           "kop_affine_relu_pool2d")
+    return out
 
 
 def kop_cumsum_rows(x, mask=None, exclusive=False, reverse=False, out=None, stream=None):

@@ -26,6 +26,9 @@ CONFIGS = {
     "groupnorm": dict(N=64, C=256, H=56, W=56, groups=32, dtype=torch.float32, eps=1e-5, act=2),
     # running sum along rows (shape ours; the paper gives none)
     "cumsum": dict(rows=32768, cols=4096, dtype=torch.float32),
+    # BatchNorm + ReLU + 3x3 / stride-2 max pool on a 112 x 112 map with 64 channels (a CNN stem)
+    "pool2d": dict(N=64, C=64, H=112, W=112, kernel=(3, 3), stride=(2, 2), padding=(1, 1), mode="max",
+                   dtype=torch.float32),
 }
 
 

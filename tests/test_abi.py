@@ -205,6 +205,25 @@ def test_cumsum_validation(L):
     assert f(P, Q + 16, Q, 4, 64, 64, 64, 64, 0, 0, 0, None) == ALIAS          # mask overlaps y
 
 
+def test_pool2d_validation(L):
+    f = L.kop_affine_relu_pool2d
+    S, T = 0x600000, 0x610000
+    g = (2, 3, 8, 8)
+    assert f(P, S, T, Q, 0, 3, 8, 8, 3, 3, 2, 2, 1, 1, 0, 1, 0, None) == OK
+    assert f(None, S, T, Q, *g, 3, 3, 2, 2, 1, 1, 0, 1, 0, None) == NULLP
+    assert f(P, S, None, Q, *g, 3, 3, 2, 2, 1, 1, 0, 1, 0, None) == NULLP      # scale without shift
+    assert f(P, S, T, Q, *g, 0, 3, 2, 2, 1, 1, 0, 1, 0, None) == SHAPE
+    assert f(P, S, T, Q, *g, 3, 3, 0, 2, 1, 1, 0, 1, 0, None) == SHAPE
+    assert f(P, S, T, Q, *g, 3, 3, 2, 2, 2, 1, 0, 1, 0, None) == SHAPE         # padding > kernel / 2
+    assert f(P, S, T, Q, *g, 3, 3, 2, 2, 1, -1, 0, 1, 0, None) == SHAPE
+    assert f(P, S, T, Q, *g, 11, 3, 2, 2, 1, 1, 0, 1, 0, None) == SHAPE        # window taller than the padded image
+    assert f(P, S, T, Q, *g, 3, 3, 2, 2, 1, 1, 2, 1, 0, None) == SHAPE         # unknown mode
+    assert f(P, S, T, Q, *g, 3, 3, 2, 2, 1, 1, 0, 1, 9, None) == DTYPE
+    assert f(P + 2, S, T, Q, *g, 3, 3, 2, 2, 1, 1, 0, 1, 0, None) == MISAL
+    assert f(P, S + 1, T, Q, *g, 3, 3, 2, 2, 1, 1, 0, 1, 0, None) == MISAL
+    assert f(P, S, T, P + 64, *g, 3, 3, 2, 2, 1, 1, 0, 1, 0, None) == ALIAS    # y inside x
+
+
 def test_mlp_driver_validation(L):
     f = L.kop_rmsnorm_swiglu_residual
     wsb = L.kop_rmsnorm_swiglu_residual_workspace_bytes(16, 64, 128, 1)

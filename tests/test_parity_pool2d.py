@@ -1,0 +1,112 @@
+"""GPU parity of kop_affine_relu_pool2d against the float64 CPU oracle: five seeds over max / average, with
+and without the affine + ReLU prologue, the compile-time window shapes (3x3 s2, 2x2 s2, 3x3 s1) and generic
+ones (rectangular, large, stride > kernel), planes that split into several bands, widths that are not whole
+16-byte vectors (scalar staging and / or scalar stores), rows too wide for a shared-memory tile (direct
+kernel), guard bands, NaN placement and run-to-run bit equality.
+
+Tolerance: |got - ref| <= tol * max(1, |ref|), tol = 1e-5 for fp32 data and 2e-2 for bf16 data. Max pooling
+of unmodified fp32 input must be bit-exact (it only selects)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import kopref
+from paper_2609_30059_b200 import build as kbuild
+from paper_2609_30059_b200 import synth
+from tests._util import Guarded, assert_bf16_tight, assert_close, tol_of
+
+pytestmark = pytest.mark.gpu
+
+SEEDS = synth.SEEDS
+F32, BF16 = torch.float32, torch.bfloat16
+
+
+@pytest.fixture(scope="module")
+def kop():
+    kbuild.build()
+    from paper_2609_30059_b200 import kop as K
+    return K
+
+
+def host(t):
+    return None if t is None else t.detach().cpu()
+
+
+POOL_CASES = [
+    # N, C, H, W, kernel, stride, padding, dtype
+    (2, 8, 112, 112, (3, 3), (2, 2), (1, 1), F32),     # benchmark plane: two bands per plane
+    (3, 5, 56, 56, (3, 3), (2, 2), (1, 1), BF16),
+    (2, 6, 64, 64, (2, 2), (2, 2), (0, 0), F32),
+    (2, 4, 32, 32, (3, 3), (1, 1), (1, 1), BF16),
+    (2, 3, 224, 224, (3, 3), (2, 2), (1, 1), F32),     # eight bands per plane
+    (2, 3, 30, 44, (5, 3), (2, 1), (2, 1), F32),       # rectangular generic window
+    (2, 3, 17, 19, (3, 3), (2, 2), (1, 1), F32),       # odd sizes: scalar staging and scalar stores
+    (2, 2, 16, 16, (2, 2), (3, 3), (0, 0), BF16),      # stride larger than the window
+    (3, 4, 7, 7, (7, 7), (1, 1), (0, 0), F32),         # window = image (global pooling)
+    (2, 2, 9, 8, (1, 1), (1, 1), (0, 0), BF16),        # identity window
+    (1, 2, 6, 5000, (3, 3), (2, 2), (1, 1), F32),      # rows too wide for a tile: direct kernel
+]
+
+
+@pytest.mark.parametrize("N,C,H,W,kernel,stride,padding,dtype", POOL_CASES)
+@pytest.mark.parametrize("seed", SEEDS)
+def test_pool2d_parity(kop, N, C, H, W, kernel, stride, padding, dtype, seed):
+    x, scale, shift = synth.bn_pool_inputs(N, C, H, W, dtype, seed, "cuda")
+    tol = tol_of(dtype)
+    OH = (H + 2 * padding[0] - kernel[0]) // stride[0] + 1
+    OW = (W + 2 * padding[1] - kernel[1]) // stride[1] + 1
+    for mode in ("max", "avg"):
+        for affine, relu in ((True, True), (False, False), (True, False)):
+            sc, sf = (scale, shift) if affine else (None, None)
+            y = Guarded((N, C, OH, OW), dtype)
+            kop.kop_affine_relu_pool2d(x, sc, sf, kernel, stride, padding, mode, relu, out=y.t)
+            ref = kopref.affine_relu_pool2d(host(x), host(sc), host(sf), kernel, stride, padding, mode, relu, threads=None)
+            what = f"pool2d {mode} affine={affine} relu={relu}"
+            assert_close(y.t, ref, tol, what)
+            if dtype == BF16:
+                assert_bf16_tight(y.t, ref, what, floor=1e-6)
+            if mode == "max" and not affine:
+                assert np.array_equal(y.t.cpu().to(torch.float64).numpy(), ref), what + " (selection is exact)"
+            y.check(what)
+
+
+def test_pool2d_full_config_seed0(kop):
+    c = synth.CONFIGS["pool2d"]
+    x, scale, shift = synth.bn_pool_inputs(c["N"], c["C"], c["H"], c["W"], c["dtype"], 0, "cuda")
+    y = kop.kop_affine_relu_pool2d(x, scale, shift, c["kernel"], c["stride"], c["padding"], c["mode"], True)
+    ref = kopref.affine_relu_pool2d(host(x), host(scale), host(shift), c["kernel"], c["stride"], c["padding"],
+                                    c["mode"], True, threads=None)
+    assert_close(y, ref, 1e-5, "pool2d full")
+    assert torch.equal(y, kop.kop_affine_relu_pool2d(x, scale, shift, c["kernel"], c["stride"], c["padding"], c["mode"], True))
+    # a second GPU path for the same definition: the global-pool entry point equals a window covering the image
+    xs = x[:4, :, :14, :14].contiguous()
+    g = kop.kop_affine_relu_pool2d(xs, scale, shift, (14, 14), (1, 1), (0, 0), "avg", True)
+    _, pooled = kop.kop_bn_relu_avgpool(xs, scale, shift)
+    assert float((g[:, :, 0, 0] - pooled).abs().max()) < 1e-5
+
+
+def test_pool2d_options(kop):
+    x, scale, shift = synth.bn_pool_inputs(2, 4, 20, 24, F32, 5, "cuda")
+    # NaN poisons exactly the windows that contain it, in both modes
+    xn = x.clone()
+    xn[1, 2, 9, 13] = float("nan")
+    for mode in ("max", "avg"):
+        y = kop.kop_affine_relu_pool2d(xn, scale, shift, (3, 3), (2, 2), (1, 1), mode, True)
+        ref = kopref.affine_relu_pool2d(host(xn), host(scale), host(shift), (3, 3), (2, 2), (1, 1), mode, True)
+        assert np.array_equal(np.isnan(y.cpu().numpy()), np.isnan(ref)) and np.isnan(ref).sum() >= 1
+    # all-negative input: padding (-inf) never wins a max; averages count the padding as zeros
+    neg = -torch.rand((1, 2, 8, 8), device="cuda") - 1.0
+    ym = kop.kop_affine_relu_pool2d(neg, None, None, (3, 3), (2, 2), (1, 1), "max", False)
+    assert bool(torch.isfinite(ym).all()) and bool((ym <= -1.0).all())
+    ones = torch.ones((1, 1, 4, 4), device="cuda")
+    ya = kop.kop_affine_relu_pool2d(ones, None, None, (3, 3), (2, 2), (1, 1), "avg", False)
+    assert abs(float(ya[0, 0, 0, 0]) - 4.0 / 9.0) < 1e-7 and abs(float(ya[0, 0, 1, 1]) - 1.0) < 1e-7
+    # empty batch; bad geometry
+    e = torch.empty((0, 4, 20, 24), dtype=F32, device="cuda")
+    assert kop.kop_affine_relu_pool2d(e, scale, shift, (3, 3), (2, 2), (1, 1)).shape == (0, 4, 10, 12)
+    with pytest.raises(kop.KopError) as ei:
+        kop.kop_affine_relu_pool2d(x, scale, shift, (3, 3), (2, 2), (2, 2))       # padding > kernel / 2
+    assert ei.value.status == 2
+    with pytest.raises(kop.KopError) as ei:
+        kop.kop_affine_relu_pool2d(x, scale, None, (3, 3), (2, 2), (1, 1))        # scale without shift
+    assert ei.value.status == 1
