@@ -34,10 +34,10 @@ __device__ __forceinline__ int div_small(int i, int d, float inv_d)
     return q;
 }
 
-__device__ __forceinline__ float act_of(float v, float sc, float sf, int relu)
+// affine, then ReLU as one NaN-propagating max (relu_floor = 0) or nothing (relu_floor = -inf)
+__device__ __forceinline__ float act_of(float v, float sc, float sf, float relu_floor)
 {
-    v = fmaf(v, sc, sf);
-    return relu ? (v > 0.0f ? v : (v <= 0.0f ? 0.0f : v)) : v;
+    return max_keep_nan(fmaf(v, sc, sf), relu_floor);
 }
 
 // Tile geometry shared by host and device: image column 0 sits at tile column `lead` (the left padding
@@ -50,14 +50,17 @@ __host__ __device__ __forceinline__ int pool_row_floats(int W, int pw) { return 
 // Consecutive threads take consecutive outputs: their windows start sw floats apart in shared memory (a
 // 2-way bank conflict at stride 2 instead of the 8-way one of a vector of outputs per thread), and a warp's
 // 32 scalar stores still make one contiguous run.
-template <typename T, int MODE, int KS, int ST, bool kVecIn>
+// kRowMap: a warp takes whole rows (lanes along the row), so no index is ever divided; used when rows are
+// long enough to keep most lanes busy. Otherwise threads walk the band's flat index range.
+template <typename T, int MODE, int KS, int ST, bool kVecIn, bool kRowMap>
 __global__ void __launch_bounds__(kPoolThreads)
 pool2d_tile_kernel(const T* __restrict__ x, const float* __restrict__ scale, const float* __restrict__ shift,
                    T* __restrict__ y, int C, int H, int W, int OH, int OW, int kh_, int kw_, int sh_, int sw_,
-                   int ph, int pw, int band_rows, int bands, int relu, float inv_area)
+                   int ph, int pw, int band_rows, int bands, int relu_flag, float inv_area)
 {
     constexpr int E = Elem<T>::kPerVec;
     extern __shared__ __align__(16) float tile[];
+    const float relu = relu_flag ? 0.0f : -INFINITY;
     const int kh = KS ? KS : kh_, kw = KS ? KS : kw_, sh = ST ? ST : sh_, sw = ST ? ST : sw_;
     const int64_t plane = blockIdx.x / bands;
     const int band = (int)(blockIdx.x - plane * bands);
@@ -86,7 +89,25 @@ pool2d_tile_kernel(const T* __restrict__ x, const float* __restrict__ scale, con
     // 2. the band's input rows: one contiguous run of (i1 - i0) * W elements
     const T* xp = x + (plane * H + i0) * (int64_t)W;
     const int n_in = (i1 - i0) * W;
-    if (kVecIn) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (kVecIn && kRowMap) {
+        const int wv = W / E, nrows = i1 - i0;
+        constexpr int NW = kPoolThreads / 32;
+        for (int cv = lane; cv < wv; cv += 32) {
+            const T* src = xp + warp * W + cv * E;
+            float* dst_f = tile + (top + warp) * Ws + lead + cv * E;
+#pragma unroll 2
+            for (int r = warp; r < nrows; r += NW, src += NW * W, dst_f += NW * Ws) {
+                float f[E];
+                Elem<T>::unpack(ld_stream(src), f);
+                float4* dst = reinterpret_cast<float4*>(dst_f);
+#pragma unroll
+                for (int q = 0; q < E / 4; ++q)
+                    dst[q] = make_float4(act_of(f[4 * q], sc, sf, relu), act_of(f[4 * q + 1], sc, sf, relu),
+                                         act_of(f[4 * q + 2], sc, sf, relu), act_of(f[4 * q + 3], sc, sf, relu));
+            }
+        }
+    } else if (kVecIn) {
         const float inv_w = 1.0f / (float)W;
         for (int v = threadIdx.x; v < n_in / E; v += kPoolThreads) {
             float f[E];
@@ -111,6 +132,35 @@ pool2d_tile_kernel(const T* __restrict__ x, const float* __restrict__ scale, con
     const int n_out = (oh1 - oh0) * OW;
     const float inv_ow = 1.0f / (float)OW;
     const float* origin = tile + (lead - pw);
+    if (kRowMap) {
+        constexpr int NW = kPoolThreads / 32;
+        const int orows = oh1 - oh0;
+        for (int ocol = lane; ocol < OW; ocol += 32) {
+            const float* win = origin + warp * sh * Ws + ocol * sw;
+            T* dst = yp + warp * OW + ocol;
+#pragma unroll 2
+            for (int orow = warp; orow < orows; orow += NW, win += NW * sh * Ws, dst += NW * OW) {
+                float res = MODE == 0 ? -INFINITY : 0.0f;
+                if (KS) {
+#pragma unroll
+                    for (int di = 0; di < (KS ? KS : 1); ++di)
+#pragma unroll
+                        for (int dj = 0; dj < (KS ? KS : 1); ++dj) {
+                            const float a = win[di * Ws + dj];
+                            res = MODE == 0 ? max_keep_nan(res, a) : res + a;
+                        }
+                } else {
+                    for (int di = 0; di < kh; ++di)
+                        for (int dj = 0; dj < kw; ++dj) {
+                            const float a = win[di * Ws + dj];
+                            res = MODE == 0 ? max_keep_nan(res, a) : res + a;
+                        }
+                }
+                Elem<T>::store1(dst, MODE == 1 ? res * inv_area : res);
+            }
+        }
+        return;
+    }
     for (int o = threadIdx.x; o < n_out; o += kPoolThreads) {
         const int orow = div_small(o, OW, inv_ow), ocol = o - orow * OW;
         const float* win = origin + orow * sh * Ws + ocol * sw;
@@ -156,7 +206,7 @@ pool2d_direct_kernel(const T* __restrict__ x, const float* __restrict__ scale, c
             for (int dj = 0; dj < kw; ++dj) {
                 const int j = oj * sw - pw + dj;
                 if (j < 0 || j >= W) continue;
-                const float a = act_of(Elem<T>::load1(xp + (int64_t)i * W + j), sc, sf, relu);
+                const float a = act_of(Elem<T>::load1(xp + (int64_t)i * W + j), sc, sf, relu ? 0.0f : -INFINITY);
                 res = mode == 0 ? max_keep_nan(res, a) : res + a;
             }
         }
@@ -165,16 +215,18 @@ pool2d_direct_kernel(const T* __restrict__ x, const float* __restrict__ scale, c
 }
 
 template <typename T, int MODE, int KS, int ST>
-void launch_tile(bool vin, unsigned grid, size_t smem, cudaStream_t stream, const T* x, const float* scale,
-                 const float* shift, T* y, int C, int H, int W, int OH, int OW, int kh, int kw, int sh, int sw, int ph,
-                 int pw, int band_rows, int bands, int relu, float inv_area)
+void launch_tile(bool vin, bool rowmap, unsigned grid, size_t smem, cudaStream_t stream, const T* x,
+                 const float* scale, const float* shift, T* y, int C, int H, int W, int OH, int OW, int kh, int kw,
+                 int sh, int sw, int ph, int pw, int band_rows, int bands, int relu, float inv_area)
 {
-    if (vin)
-        pool2d_tile_kernel<T, MODE, KS, ST, true><<<grid, kPoolThreads, smem, stream>>>(
-            x, scale, shift, y, C, H, W, OH, OW, kh, kw, sh, sw, ph, pw, band_rows, bands, relu, inv_area);
-    else
-        pool2d_tile_kernel<T, MODE, KS, ST, false><<<grid, kPoolThreads, smem, stream>>>(
-            x, scale, shift, y, C, H, W, OH, OW, kh, kw, sh, sw, ph, pw, band_rows, bands, relu, inv_area);
+#define KOP_POOL_GO(VI, RM)                                                                                         \
+    pool2d_tile_kernel<T, MODE, KS, ST, VI, RM><<<grid, kPoolThreads, smem, stream>>>(                               \
+        x, scale, shift, y, C, H, W, OH, OW, kh, kw, sh, sw, ph, pw, band_rows, bands, relu, inv_area)
+    if (vin && rowmap) KOP_POOL_GO(true, true);
+    else if (vin) KOP_POOL_GO(true, false);
+    else if (rowmap) KOP_POOL_GO(false, true);
+    else KOP_POOL_GO(false, false);
+#undef KOP_POOL_GO
 }
 
 template <typename T>
@@ -196,12 +248,14 @@ kop_status_t launch_pool(const void* xv, const float* scale, const float* shift,
         if (br > OH) br = OH;
         {
             // among band heights down to half of that, take the one whose outputs fill the CTA's passes best
-            const int64_t per_row = OW;
+            // (row mapping: whole rows per warp, 8 warps; flat mapping: outputs per pass of 256 threads)
+            const bool by_rows = ((aligned_to(x, 16) && W % E == 0) ? W / E : W) >= 20 && OW >= 20;
+            const int64_t unit = by_rows ? 1 : OW, pass = by_rows ? kPoolThreads / 32 : kPoolThreads;
             int64_t best = br;
             double best_util = 0.0;
             for (int64_t cand = br; cand >= 1 && cand * 2 >= br; --cand) {
-                const int64_t n = cand * per_row;
-                const double util = (double)n / (double)((n + kPoolThreads - 1) / kPoolThreads * kPoolThreads);
+                const int64_t n = cand * unit;
+                const double util = (double)n / (double)((n + pass - 1) / pass * pass);
                 if (util > best_util + 1e-9) {
                     best_util = util;
                     best = cand;
@@ -215,8 +269,10 @@ kop_status_t launch_pool(const void* xv, const float* scale, const float* shift,
         if (grid <= 0x7FFFFFFFLL && smem <= (size_t)kPoolTileMax) {
             // flat vector loads need every band to start on a 16-byte boundary: rows that are whole vectors
             const bool vin = aligned_to(x, 16) && W % E == 0;
+            // a warp per row pays off when rows keep most of its lanes busy on both sides
+            const bool rowmap = (vin ? W / E : W) >= 20 && OW >= 20;
             const unsigned g = (unsigned)grid;
-#define KOP_POOL_ARGS vin, g, smem, stream, x, scale, shift, y, (int)C, H, W, OH, OW, kh, kw, sh, sw, ph, pw, (int)br, bands, relu, inv_area
+#define KOP_POOL_ARGS vin, rowmap, g, smem, stream, x, scale, shift, y, (int)C, H, W, OH, OW, kh, kw, sh, sw, ph, pw, (int)br, bands, relu, inv_area
             const bool square = kh == kw && sh == sw;
             if (mode == 0) {
                 if (square && kh == 3 && sh == 2) launch_tile<T, 0, 3, 2>(KOP_POOL_ARGS);
