@@ -1,0 +1,169 @@
+"""Randomised GPU parity sweep: for every entry point, a few hundred small random shapes (seeded, so the
+sweep is reproducible) with random dtypes, strides, alignments and options, each compared with the
+float64 oracle under the usual rule |got - ref| <= tol * max(1, |ref|) (1e-5 fp32 data, 2e-2 bf16 data).
+The hand-picked cases in the other parity files aim at known kernel boundaries; this sweep is for the
+ones nobody thought of (odd lengths next to vector multiples, one-row and one-column tensors, sizes that
+straddle the kernels' dispatch thresholds)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import kopref
+from paper_2609_30059_b200 import build as kbuild
+from paper_2609_30059_b200 import synth
+from tests._util import assert_close, to_f64, tol_of
+
+pytestmark = pytest.mark.gpu
+F32, BF16 = torch.float32, torch.bfloat16
+
+
+@pytest.fixture(scope="module")
+def kop():
+    kbuild.build()
+    from paper_2609_30059_b200 import kop as K
+    return K
+
+
+def host(t):
+    return None if t is None else t.detach().cpu()
+
+
+def pick_len(rng, hi):
+    """Lengths biased towards the interesting neighbourhoods: tiny, around multiples of 4 / 8 / 32 / 256."""
+    kind = rng.integers(0, 5)
+    if kind == 0:
+        return int(rng.integers(1, 12))
+    if kind == 1:
+        return int(min(hi, max(1, 8 * rng.integers(1, hi // 8 + 1) + rng.integers(-1, 2))))
+    if kind == 2:
+        return int(min(hi, max(1, 256 * rng.integers(1, max(2, hi // 256 + 1)) + rng.integers(-2, 3))))
+    return int(rng.integers(1, hi + 1))
+
+
+def strided(rng, t):
+    """Sometimes re-home a 2-D tensor inside a wider buffer (row stride > cols) or at an odd offset."""
+    mode = rng.integers(0, 4)
+    rows, cols = t.shape
+    if mode == 0:
+        pad = int(rng.integers(1, 9)) * (8 if rng.integers(0, 2) else 1)
+        big = torch.zeros((rows, cols + pad), dtype=t.dtype, device=t.device)
+        big[:, :cols] = t
+        return big[:, :cols]
+    if mode == 1:
+        flat = torch.zeros(rows * cols + 1, dtype=t.dtype, device=t.device)
+        flat[1:] = t.reshape(-1)
+        return flat[1:].view(rows, cols)
+    return t
+
+
+def test_fuzz_row_kernels(kop):
+    rng = np.random.default_rng(2609_30059)
+    for it in range(120):
+        dtype = BF16 if rng.integers(0, 2) else F32
+        tol = tol_of(dtype)
+        rows, cols = pick_len(rng, 70), pick_len(rng, 3000)
+        seed = int(rng.integers(0, 1 << 30))
+        what = f"it={it} rows={rows} cols={cols} {dtype}"
+        # softmax
+        x, bias = synth.softmax_inputs(rows, cols, dtype, seed, "cuda")
+        xs = strided(rng, x)
+        scale = float(rng.uniform(0.05, 2.0))
+        use_bias = bool(rng.integers(0, 2))
+        y = kop.kop_softmax_scale_bias(xs, bias if use_bias else None, scale)
+        assert_close(y, kopref.softmax_scale_bias(host(x), host(bias) if use_bias else None, scale), tol, "softmax " + what)
+        # bias + GELU + residual + LayerNorm and the plain / residual LayerNorm
+        if cols >= 2:
+            x, r, b, g, be = synth.layernorm_inputs(rows, cols, dtype, seed, "cuda")
+            xs, rs_ = strided(rng, x), strided(rng, r)
+            y, mu, rstd = kop.kop_bias_gelu_residual_layernorm(xs, rs_, b, g, be, 1e-5)
+            ry, rm, rr = kopref.bias_gelu_residual_layernorm(host(x), host(r), host(b), host(g), host(be), 1e-5)
+            assert_close(y, ry, tol, "layernorm y " + what)
+            assert_close(mu, rm, 1e-3, "layernorm mean " + what)
+            with_res = bool(rng.integers(0, 2))
+            y, mu, rstd = kop.kop_residual_layernorm(xs, rs_ if with_res else None, g, be, 1e-5)
+            ry, rm, rr = kopref.residual_layernorm(host(x), host(r) if with_res else None, host(g), host(be), 1e-5)
+            assert_close(y, ry, tol, "residual layernorm y " + what)
+        # RMSNorm
+        h, w, _, _ = synth.mlp_inputs(rows, cols, 1, dtype, seed, "cuda")
+        hs = strided(rng, h)
+        assert_close(kop.kop_rmsnorm(hs, w, 1e-6), kopref.rmsnorm(host(h), host(w), 1e-6), tol, "rmsnorm " + what)
+        # cross-entropy (plain and with options)
+        z, lab = synth.ce_inputs(rows, cols, dtype, seed, "cuda")
+        zs = strided(rng, z)
+        loss, mean, bad = kop.kop_ce_loss_rowwise(zs, lab)
+        rl, rmean, rbad = kopref.ce_loss_rowwise(host(z), host(lab))
+        assert_close(loss, rl, max(tol, 2e-5), "ce loss " + what)
+        assert abs(float(mean) - rmean) <= max(tol, 2e-5) * max(1.0, abs(rmean)) and int(bad) == rbad, "ce mean " + what
+        lab2 = lab.clone()
+        lab2[rng.random(rows) < 0.3] = -100
+        sm = float(rng.choice([0.0, 0.1, 0.3]))
+        loss, mean, bad, cnt = kop.kop_ce_loss_rowwise_opts(zs, lab2, -100, sm)
+        rl, rmean, rbad, rcnt = kopref.ce_loss_opts(host(z), host(lab2), -100, sm)
+        assert_close(loss, rl, max(tol, 2e-5), "ce opts loss " + what)
+        assert int(cnt) == rcnt and int(bad) == rbad, "ce opts counts " + what
+        if rcnt > 0:
+            assert abs(float(mean) - rmean) <= max(tol, 2e-5) * max(1.0, abs(rmean)), "ce opts mean " + what
+        # SwiGLU epilogues, residual add, row scale, mat-vec
+        gu = synth.gate_up_inputs(rows, cols, dtype, seed, "cuda")
+        assert_close(kop.kop_silu_mul(strided(rng, gu)), kopref.silu_mul(host(gu)), tol, "silu_mul " + what)
+        assert_close(kop.kop_silu_mul_interleaved(strided(rng, gu)), kopref.silu_mul_interleaved(host(gu)), tol,
+                     "silu_mul_interleaved " + what)
+        a, b2 = synth.pair_inputs(rows, cols, dtype, seed, "cuda")
+        assert_close(kop.kop_residual_add(strided(rng, a), strided(rng, b2)), kopref.residual_add(host(a), host(b2)), tol,
+                     "residual_add " + what)
+        av, bm = synth.row_scale_inputs(rows, cols, dtype, seed, "cuda")
+        assert_close(kop.kop_row_scale(av, strided(rng, bm)), kopref.row_scale(host(av), host(bm)), tol, "row_scale " + what)
+        xv, wv, bs = synth.matvec_inputs(rows, cols, dtype, seed, "cuda")
+        ref = kopref.matvec_bias(host(xv), host(wv), bs)
+        got = to_f64(kop.kop_matvec_bias(strided(rng, xv), wv, bs))
+        # fp32 accumulation of `cols` products against a float64 sum: scale by the sum of magnitudes
+        mag = (host(xv).double().abs() @ host(wv).double().abs()).numpy() + abs(bs)
+        assert np.all(np.abs(got - ref) <= 1e-5 * np.maximum(1.0, mag)), "matvec " + what
+        # running sums
+        xc, mask = synth.cumsum_inputs(rows, cols, dtype, seed, "cuda")
+        ex, rv, um = bool(rng.integers(0, 2)), bool(rng.integers(0, 2)), bool(rng.integers(0, 2))
+        got = to_f64(kop.kop_cumsum_rows(strided(rng, xc), mask if um else None, ex, rv))
+        ref = kopref.cumsum_rows(host(xc), host(mask) if um else None, ex, rv)
+        scale_rows = np.maximum(1.0, np.abs(ref).max(axis=1, keepdims=True))
+        assert np.all(np.abs(got - ref) <= tol * scale_rows), "cumsum " + what
+
+
+def test_fuzz_image_kernels(kop):
+    rng = np.random.default_rng(30059_2609)
+    for it in range(100):
+        dtype = BF16 if rng.integers(0, 2) else F32
+        tol = tol_of(dtype)
+        N, H, W = int(rng.integers(1, 5)), pick_len(rng, 40), pick_len(rng, 40)
+        groups = int(rng.choice([1, 2, 3, 4, 8]))
+        C = groups * int(rng.integers(1, 9))
+        seed = int(rng.integers(0, 1 << 30))
+        what = f"it={it} N={N} C={C} H={H} W={W} G={groups} {dtype}"
+        x, scale, shift = synth.bn_pool_inputs(N, C, H, W, dtype, seed, "cuda")
+        # BN + ReLU + global pool, NCHW and channels-last
+        y, p = kop.kop_bn_relu_avgpool(x, scale, shift)
+        ry, rp = kopref.bn_relu_avgpool(host(x), host(scale), host(shift))
+        assert_close(y, ry, tol, "bn y " + what)
+        assert_close(p, rp, 1e-5, "bn pooled " + what)
+        xl = x.contiguous(memory_format=torch.channels_last)
+        yl, pl = kop.kop_bn_relu_avgpool(xl, scale, shift)
+        assert_close(yl, ry, tol, "bn nhwc y " + what)
+        assert_close(pl, rp, 1e-5, "bn nhwc pooled " + what)
+        # GroupNorm + activation
+        xg, gamma, beta = synth.groupnorm_inputs(N, C, H, W, dtype, seed, "cuda")
+        act = int(rng.integers(0, 3))
+        aff = bool(rng.integers(0, 4))
+        y, mu, rs = kop.kop_groupnorm_act(xg, gamma if aff else None, beta if aff else None, groups, 1e-5, act)
+        ry, rm, rr = kopref.groupnorm_act(host(xg), host(gamma) if aff else None, host(beta) if aff else None, groups, 1e-5, act)
+        assert_close(y, ry, tol, "groupnorm y " + what)
+        assert_close(mu, rm, 1e-5, "groupnorm mean " + what)
+        # windowed pooling with a random legal geometry
+        kh, kw = int(rng.integers(1, min(H, 5) + 1)), int(rng.integers(1, min(W, 5) + 1))
+        sh, sw = int(rng.integers(1, 4)), int(rng.integers(1, 4))
+        ph, pw = int(rng.integers(0, kh // 2 + 1)), int(rng.integers(0, kw // 2 + 1))
+        mode = "max" if rng.integers(0, 2) else "avg"
+        aff, relu = bool(rng.integers(0, 2)), bool(rng.integers(0, 2))
+        y = kop.kop_affine_relu_pool2d(x, scale if aff else None, shift if aff else None, (kh, kw), (sh, sw), (ph, pw), mode, relu)
+        ref = kopref.affine_relu_pool2d(host(x), host(scale) if aff else None, host(shift) if aff else None, (kh, kw),
+                                        (sh, sw), (ph, pw), mode, relu)
+        assert_close(y, ref, tol, f"pool2d k=({kh},{kw}) s=({sh},{sw}) p=({ph},{pw}) {mode} " + what)
+    assert kop.kop_groupnorm_wait_timeouts() == 0
