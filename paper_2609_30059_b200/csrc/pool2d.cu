@@ -184,6 +184,124 @@ pool2d_tile_kernel(const T* __restrict__ x, const float* __restrict__ scale, con
     }
 }
 
+// ---- strip kernel: the two stride-2 windows CNNs use (3x3 pad 1, 2x2 pad 0), no shared memory ----------
+// A thread owns eight input columns (four outputs) of a band of output rows and walks down the rows: per
+// input row two 16-byte loads (one for bf16) plus, for 3x3, the single halo element to its left (a scalar
+// load that hits L1), the affine / ReLU on the nine values, the four horizontal window reductions, and per
+// output row the vertical combination of three (two) such rows, the lowest of which is carried over to
+// the next output row. About four instructions per input element, no index arithmetic inside the loop,
+// every load and store of a warp a contiguous run.
+template <typename T, int MODE>
+__device__ __forceinline__ float pool_op(float a, float b) { return MODE == 0 ? max_keep_nan(a, b) : a + b; }
+
+// Eight consecutive elements of the data type as floats: one 256-bit load for fp32 (a lane then uses whole
+// 32-byte sectors; two 128-bit loads would fetch every sector twice, L1 allocation being off), one 128-bit
+// load for bf16.
+__device__ __forceinline__ void load8(const float* p, float (&f)[8])
+{
+    uint32_t w[8];
+    asm volatile("ld.global.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+                 : "l"(p));
+#pragma unroll
+    for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(w[e]);
+}
+__device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&f)[8])
+{
+    Elem<__nv_bfloat16>::unpack(ld_stream(p), f);
+}
+
+// Horizontal reductions of one input row for this thread's four outputs. KS == 3: windows of columns
+// (2j-1, 2j, 2j+1) relative to the thread's first column, v[0] being the halo, which is the left
+// neighbour lane's last column (a shuffle; lane 0 of a warp loads it); KS == 2: (2j, 2j+1). Rows outside
+// the image are loaded from a clamped row and overridden with padding, so the warp stays converged for
+// the shuffle. Called by all 32 lanes.
+template <typename T, int MODE, int KS>
+__device__ __forceinline__ void strip_row(const T* __restrict__ row, bool row_ok, int seg, int lane, float sc,
+                                          float sf, float relu, float (&h)[4])
+{
+    const float pad = MODE == 0 ? -INFINITY : 0.0f;
+    float v[9], f[8];
+    load8(row, f);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[1 + e] = row_ok ? act_of(f[e], sc, sf, relu) : pad;
+    if (KS == 3) {
+        float left = __shfl_up_sync(0xFFFFFFFFu, v[8], 1);
+        if (lane == 0 && seg > 0) left = row_ok ? act_of(Elem<T>::load1(row - 1), sc, sf, relu) : pad;
+        v[0] = seg > 0 ? left : pad;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) h[j] = pool_op<T, MODE>(pool_op<T, MODE>(v[2 * j], v[2 * j + 1]), v[2 * j + 2]);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) h[j] = pool_op<T, MODE>(v[2 * j + 1], v[2 * j + 2]);
+    }
+}
+
+template <typename T>
+__device__ __forceinline__ void store4(T* dst, const float (&o)[4]);
+template <>
+__device__ __forceinline__ void store4<float>(float* dst, const float (&o)[4])
+{
+    st_stream(dst, Elem<float>::pack(o));
+}
+template <>
+__device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16* dst, const float (&o)[4])
+{
+    const __nv_bfloat162 a = __floats2bfloat162_rn(o[0], o[1]), b = __floats2bfloat162_rn(o[2], o[3]);
+    uint2 w;
+    w.x = *reinterpret_cast<const uint32_t*>(&a);
+    w.y = *reinterpret_cast<const uint32_t*>(&b);
+    *reinterpret_cast<uint2*>(dst) = w;                   // four outputs = 8 bytes, 8-byte aligned (OW % 4 == 0)
+}
+
+template <typename T, int MODE, int KS>
+__global__ void __launch_bounds__(256)
+pool2d_strip_kernel(const T* __restrict__ x, const float* __restrict__ scale, const float* __restrict__ shift,
+                    T* __restrict__ y, int64_t strips, int C, int H, int W, int OH, int OW, int segs, int bands,
+                    int band_rows, int relu_flag, float inv_area)
+{
+    const int64_t g_raw = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const bool live = g_raw < strips;                       // surplus threads of the last CTA shadow the last strip
+    const int64_t g = live ? g_raw : strips - 1;
+    const int lane = threadIdx.x & 31;
+    const int seg = (int)(g % segs);
+    const int64_t rest = g / segs;
+    const int band = (int)(rest % bands);
+    const int64_t plane = rest / bands;
+    const int c = (int)(plane % C);
+    const float sc = scale != nullptr ? __ldg(scale + c) : 1.0f;
+    const float sf = shift != nullptr ? __ldg(shift + c) : 0.0f;
+    const float relu = relu_flag ? 0.0f : -INFINITY;
+    constexpr int P = KS == 3 ? 1 : 0;
+    const int oh0 = band * band_rows, oh1 = min(OH, oh0 + band_rows);
+    const T* col = x + plane * H * (int64_t)W + seg * 8;            // this strip's first column, row 0
+    T* out = y + (plane * OH + oh0) * (int64_t)OW + seg * 4;
+
+    float carry[4];
+    if (KS == 3) {
+        const int i = 2 * oh0 - P;
+        strip_row<T, MODE, KS>(col + (int64_t)max(i, 0) * W, i >= 0, seg, lane, sc, sf, relu, carry);
+    }
+    // every lane runs band_rows trips so that the shuffles stay warp-wide; trips past a short last band are idle
+    for (int t = 0; t < band_rows; ++t, out += OW) {
+        const int oi = min(oh0 + t, OH - 1);
+        float a[4], b[4], o[4];
+        const int i1 = 2 * oi - P + (KS == 3 ? 1 : 0), i2 = i1 + 1;   // the two rows first needed by this output row
+        strip_row<T, MODE, KS>(col + (int64_t)i1 * W, true, seg, lane, sc, sf, relu, a);
+        strip_row<T, MODE, KS>(col + (int64_t)min(i2, H - 1) * W, i2 < H, seg, lane, sc, sf, relu, b);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float r = pool_op<T, MODE>(a[j], b[j]);
+            if (KS == 3) {
+                r = pool_op<T, MODE>(carry[j], r);
+                carry[j] = b[j];
+            }
+            o[j] = MODE == 1 ? r * inv_area : r;
+        }
+        if (live && oh0 + t < oh1) store4<T>(out, o);
+    }
+}
+
 // Any geometry (rows too wide for the tile): one thread per output, window read from global memory.
 template <typename T>
 __global__ void __launch_bounds__(256)
@@ -239,6 +357,32 @@ kop_status_t launch_pool(const void* xv, const float* scale, const float* shift,
     T* y = static_cast<T*>(yv);
     const float inv_area = (float)(1.0 / ((double)kh * kw));
     const int64_t planes = N * C;
+    // the strip kernel: stride-2 3x3 (pad 1) or 2x2 (pad 0) windows over rows of whole 8-column segments
+    const bool k3 = kh == 3 && kw == 3 && ph == 1 && pw == 1, k2 = kh == 2 && kw == 2 && ph == 0 && pw == 0;
+    if ((k3 || k2) && sh == 2 && sw == 2 && W % 8 == 0 && H % 2 == 0 && aligned_to(x, 32) && aligned_to(y, 16)) {
+        const int segs = W / 8;
+        // bands of output rows: enough strips for a full complement of resident warps per SM, at least 4 output rows each
+        int band_rows = OH;
+        const int64_t want = 64LL * 32 * sm_count();
+        while (band_rows > 4 && planes * segs * ((OH + band_rows - 1) / band_rows) < want) band_rows = (band_rows + 1) / 2;
+        const int bands = (OH + band_rows - 1) / band_rows;
+        const int64_t strips = planes * segs * bands;
+        const int64_t blocks = (strips + 255) / 256;
+        if (blocks <= 0x7FFFFFFFLL) {
+#define KOP_STRIP(MODE, KS)                                                                                       \
+    pool2d_strip_kernel<T, MODE, KS><<<(unsigned)blocks, 256, 0, stream>>>(x, scale, shift, y, strips, (int)C, H, W, \
+                                                                            OH, OW, segs, bands, band_rows, relu, inv_area)
+            if (mode == 0) {
+                if (k3) KOP_STRIP(0, 3);
+                else KOP_STRIP(0, 2);
+            } else {
+                if (k3) KOP_STRIP(1, 3);
+                else KOP_STRIP(1, 2);
+            }
+#undef KOP_STRIP
+            return launch_status();
+        }
+    }
     const int64_t row_bytes = (int64_t)pool_row_floats(W, pw) * 4;
     if ((int64_t)kh * row_bytes <= kPoolTileMax) {
         // output rows per band: about kPoolTileBytes of tile, at least one row, then evened out
