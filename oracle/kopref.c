@@ -38,7 +38,7 @@
 #include <omp.h>
 #endif
 
-enum { KOPREF_F32 = 0, KOPREF_BF16 = 1, KOPREF_F64 = 2 };
+enum { KOPREF_F32 = 0, KOPREF_BF16 = 1, KOPREF_F64 = 2, KOPREF_F16 = 3 };
 
 /* ---- exact widening / narrowing helpers ------------------------------------ */
 
@@ -49,6 +49,19 @@ double kopref_bf16_to_f64(uint16_t bits)
     float f;
     memcpy(&f, &u, sizeof f);
     return (double)f;
+}
+
+/* IEEE binary16 (1 sign, 5 exponent, 10 fraction bits) widened exactly, from its fields:
+ * exponent 0: (-1)^s * fraction * 2^-24 (zero and subnormals); exponent 31: infinity or NaN;
+ * otherwise (-1)^s * (1024 + fraction) * 2^(exponent - 25). */
+double kopref_f16_to_f64(uint16_t bits)
+{
+    int s = bits >> 15, e = (bits >> 10) & 0x1F, f = bits & 0x3FF;
+    double v;
+    if (e == 0) v = ldexp((double)f, -24);
+    else if (e == 31) v = f ? NAN : INFINITY;
+    else v = ldexp((double)(1024 + f), e - 25);
+    return s ? -v : v;
 }
 
 /* Round a double directly to bf16 (round to nearest, ties to even) without
@@ -84,11 +97,12 @@ static inline double load_elem(const void* base, int64_t idx, int dtype)
     switch (dtype) {
     case KOPREF_F32:  return (double)((const float*)base)[idx];
     case KOPREF_BF16: return kopref_bf16_to_f64(((const uint16_t*)base)[idx]);
+    case KOPREF_F16:  return kopref_f16_to_f64(((const uint16_t*)base)[idx]);
     default:          return ((const double*)base)[idx];
     }
 }
 
-static int bad_dtype(int dtype) { return dtype < KOPREF_F32 || dtype > KOPREF_F64; }
+static int bad_dtype(int dtype) { return dtype < KOPREF_F32 || dtype > KOPREF_F16; }
 
 static int pick_threads(int threads)
 {

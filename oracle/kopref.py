@@ -4,8 +4,8 @@ TEST INFRASTRUCTURE ONLY: imported by tests/, by the smoke check and by the
 benchmark's cpu_baseline / reference legs. The product package never imports it,
 and this module imports nothing from the product package.
 
-Data tensors may be numpy arrays (float32, float64, or uint16 holding bf16 bit
-patterns) or CPU torch tensors (float32, float64, bfloat16); they must be
+Data tensors may be numpy arrays (float32, float64, float16, or uint16 holding bf16
+bit patterns) or CPU torch tensors (float32, float64, bfloat16, float16); they must be
 contiguous in their last dimension. Every result is a float64 numpy array.
 """
 from __future__ import annotations
@@ -17,7 +17,7 @@ import numpy as np
 
 from . import build as _build
 
-F32, BF16, F64 = 0, 1, 2
+F32, BF16, F64, F16 = 0, 1, 2, 3
 _lib = None
 
 
@@ -28,6 +28,8 @@ def lib() -> C.CDLL:
         i64, dbl, vp = C.c_int64, C.c_double, C.c_void_p
         _lib.kopref_bf16_to_f64.restype = dbl
         _lib.kopref_bf16_to_f64.argtypes = [C.c_uint16]
+        _lib.kopref_f16_to_f64.restype = dbl
+        _lib.kopref_f16_to_f64.argtypes = [C.c_uint16]
         _lib.kopref_f64_to_bf16_rne.restype = C.c_uint16
         _lib.kopref_f64_to_bf16_rne.argtypes = [dbl]
         _lib.kopref_gelu_tanh.restype = dbl
@@ -71,12 +73,16 @@ def as_data(a):
         assert a.device.type == "cpu", "oracle inputs live on the host"
         if a.dtype == torch.bfloat16:
             return a.contiguous().view(torch.int16).numpy().view(np.uint16), BF16
+        if a.dtype == torch.float16:
+            return a.contiguous().view(torch.int16).numpy().view(np.uint16), F16
         a = a.contiguous().numpy()
     a = np.asarray(a)
     if a.dtype == np.float32:
         return np.ascontiguousarray(a), F32
     if a.dtype == np.uint16:
         return np.ascontiguousarray(a), BF16
+    if a.dtype == np.float16:
+        return np.ascontiguousarray(a).view(np.uint16), F16
     if a.dtype == np.float64:
         return np.ascontiguousarray(a), F64
     raise TypeError(f"unsupported oracle data dtype {a.dtype}")
@@ -105,6 +111,12 @@ def _check(rc, name):
 def bf16_to_f64(bits) -> np.ndarray:
     bits = np.asarray(bits, dtype=np.uint16)
     f = lib().kopref_bf16_to_f64
+    return np.array([f(int(b)) for b in bits.ravel()], dtype=np.float64).reshape(bits.shape)
+
+
+def f16_to_f64(bits) -> np.ndarray:
+    bits = np.asarray(bits, dtype=np.uint16)
+    f = lib().kopref_f16_to_f64
     return np.array([f(int(b)) for b in bits.ravel()], dtype=np.float64).reshape(bits.shape)
 
 
@@ -335,9 +347,11 @@ def mlp_segment(h, rms_weight, w_gate_up, w_down, eps, threads=1) -> np.ndarray:
     gu = gemm_nt(n, w_gate_up, threads)
     act = silu_mul(gu, threads)
     d = gemm_nt(act, w_down, threads)
-    ha, _ = as_data(h)
-    if ha.dtype == np.uint16:
+    ha, tag = as_data(h)
+    if tag == BF16:
         hd = (ha.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    elif tag == F16:
+        hd = ha.view(np.float16).astype(np.float64)
     else:
         hd = ha.astype(np.float64)
     return residual_add(hd, d, threads)

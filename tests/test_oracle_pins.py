@@ -757,3 +757,27 @@ def test_pool2d_library_closed_forms_and_special_cases():
     xb = x.to(torch.bfloat16)
     np.testing.assert_allclose(kopref.affine_relu_pool2d(xb, None, None, (3, 3), (2, 2), (1, 1), "max", False, threads=3),
                                F.max_pool2d(xb.double(), 3, 2, 1).numpy(), rtol=0, atol=0)
+
+
+# --------------------------------------------------------------------------- fp16 inputs
+
+def test_f16_widening_exhaustive_and_one_function_end_to_end():
+    bits = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    wide = kopref.f16_to_f64(bits)
+    via_numpy = bits.view(np.float16).astype(np.float64)              # an independent implementation
+    finite = np.isfinite(via_numpy)
+    assert np.array_equal(wide[finite], via_numpy[finite])
+    assert np.array_equal(np.isnan(wide), np.isnan(via_numpy)) and np.array_equal(np.isinf(wide), np.isinf(via_numpy))
+    assert np.array_equal(np.signbit(wide[~np.isnan(wide)]), np.signbit(via_numpy[~np.isnan(via_numpy)]))
+    # through a whole oracle function: fp16 tensors are widened exactly, so the result equals the one on
+    # the same values given as float64
+    x = torch.from_numpy(f32(RNG.normal(0, 1, (5, 37)))).to(torch.float16)
+    b = torch.from_numpy(f32(RNG.normal(0, 0.1, 37)))
+    assert np.array_equal(kopref.softmax_scale_bias(x, b, 0.3), kopref.softmax_scale_bias(x.to(torch.float64), b, 0.3))
+    assert np.array_equal(kopref.softmax_scale_bias(x.numpy(), b, 0.3), kopref.softmax_scale_bias(x, b, 0.3))
+    h = torch.from_numpy(f32(RNG.normal(0, 1, (4, 16)))).to(torch.float16)
+    w = torch.from_numpy(f32(RNG.normal(1, 0.02, 16)))
+    W1 = torch.from_numpy(f32(RNG.normal(0, 0.1, (24, 16)))).to(torch.float16)
+    W2 = torch.from_numpy(f32(RNG.normal(0, 0.1, (16, 12)))).to(torch.float16)
+    np.testing.assert_allclose(kopref.mlp_segment(h, w, W1, W2, 1e-6),
+                               kopref.mlp_segment(h.double(), w, W1.double(), W2.double(), 1e-6), rtol=0, atol=1e-15)
