@@ -15,10 +15,11 @@
  *              on the current device, owned by the caller. Shape arrays passed by
  *              pointer (strides of kop_bn_relu_avgpool) are HOST pointers.
  *   dtype      `dtype` is the element type of the data tensors (inputs and the main
- *              output): KOP_F32 or KOP_BF16. Parameter vectors (bias, gamma, beta,
+ *              output): KOP_F32, KOP_BF16 or KOP_F16 (IEEE binary16; results beyond
+ *              65504 in magnitude are stored as infinity). Parameter vectors (bias, gamma, beta,
  *              scale, shift, weight) and statistics outputs (mean, rstd, pooled,
  *              loss) are always fp32. All arithmetic is fp32; the only rounding to
- *              bf16 is the final store (round to nearest even), as the paper's
+ *              bf16 / fp16 is the final store (round to nearest even), as the paper's
  *              numerics rule requires (accumulate in fp32, cast only at the store).
  *   strides    In elements. The innermost stride is 1 by contract; a row stride
  *              must be >= the row length.
@@ -64,7 +65,7 @@ typedef enum {
     KOP_ERR_CUBLAS = 10
 } kop_status_t;
 
-typedef enum { KOP_F32 = 0, KOP_BF16 = 1 } kop_dtype_t;
+typedef enum { KOP_F32 = 0, KOP_BF16 = 1, KOP_F16 = 2 } kop_dtype_t;
 
 /* Library version as major * 10000 + minor * 100 + patch. */
 int kop_version(void);

@@ -470,7 +470,9 @@ extern "C" kop_status_t kop_bn_relu_avgpool(const void* x, const float* scale, c
     cudaStream_t s = as_stream(stream);
     if (!is_nchw)
         return dtype == KOP_F32 ? launch_bn_nhwc<float>(x, scale, shift, y, pooled, N, C, H, W, s)
-                                : launch_bn_nhwc<__nv_bfloat16>(x, scale, shift, y, pooled, N, C, H, W, s);
+                                : dtype == KOP_BF16 ? launch_bn_nhwc<__nv_bfloat16>(x, scale, shift, y, pooled, N, C, H, W, s)
+                                : launch_bn_nhwc<__half>(x, scale, shift, y, pooled, N, C, H, W, s);
     return dtype == KOP_F32 ? launch_bn<float>(x, scale, shift, y, pooled, N, C, H, W, s)
-                            : launch_bn<__nv_bfloat16>(x, scale, shift, y, pooled, N, C, H, W, s);
+                            : dtype == KOP_BF16 ? launch_bn<__nv_bfloat16>(x, scale, shift, y, pooled, N, C, H, W, s)
+                            : launch_bn<__half>(x, scale, shift, y, pooled, N, C, H, W, s);
 }

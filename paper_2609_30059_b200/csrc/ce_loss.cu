@@ -64,6 +64,14 @@ __device__ __forceinline__ float vec_max<__nv_bfloat16>(const Vec16& v)
     return fmaxf(__low2float(m), __high2float(m));
 }
 
+template <>
+__device__ __forceinline__ float vec_max<__half>(const Vec16& v)
+{
+    const __half2* h = reinterpret_cast<const __half2*>(v.w);
+    const __half2 m = __hmax2(__hmax2(h[0], h[1]), __hmax2(h[2], h[3]));
+    return fmaxf(__low2float(m), __high2float(m));
+}
+
 __device__ __forceinline__ int warp_sum_int(int v)
 {
 #pragma unroll
@@ -323,7 +331,8 @@ extern "C" kop_status_t kop_ce_loss_rowwise(const void* logits, const int32_t* l
     cudaStream_t s = as_stream(stream);
     return dtype == KOP_F32
                ? launch_ce<float, false>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s, CeOpts{0, 0.0f, nullptr})
-               : launch_ce<__nv_bfloat16, false>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s, CeOpts{0, 0.0f, nullptr});
+               : dtype == KOP_BF16 ? launch_ce<__nv_bfloat16, false>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s, CeOpts{0, 0.0f, nullptr})
+               : launch_ce<__half, false>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s, CeOpts{0, 0.0f, nullptr});
 }
 
 extern "C" kop_status_t kop_ce_loss_rowwise_opts(const void* logits, const int32_t* labels, float* loss,
@@ -355,7 +364,8 @@ extern "C" kop_status_t kop_ce_loss_rowwise_opts(const void* logits, const int32
     const CeOpts opts{ignore_index, label_smoothing, counted_rows};
     return dtype == KOP_F32
                ? launch_ce<float, true>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s, opts)
-               : launch_ce<__nv_bfloat16, true>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s, opts);
+               : dtype == KOP_BF16 ? launch_ce<__nv_bfloat16, true>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s, opts)
+               : launch_ce<__half, true>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s, opts);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -497,7 +497,8 @@ extern "C" kop_status_t kop_groupnorm_act(const void* x, const float* gamma, con
     cudaStream_t s = as_stream(stream);
     return dtype == KOP_F32
                ? launch_gn<float>(x, gamma, beta, y, mean, rstd, N * groups, chunk_elems, plane, cpg, (int)groups, eps, act, s)
-               : launch_gn<__nv_bfloat16>(x, gamma, beta, y, mean, rstd, N * groups, chunk_elems, plane, cpg, (int)groups, eps, act, s);
+               : dtype == KOP_BF16 ? launch_gn<__nv_bfloat16>(x, gamma, beta, y, mean, rstd, N * groups, chunk_elems, plane, cpg, (int)groups, eps, act, s)
+               : launch_gn<__half>(x, gamma, beta, y, mean, rstd, N * groups, chunk_elems, plane, cpg, (int)groups, eps, act, s);
 }
 
 extern "C" kop_status_t kop_groupnorm_wait_timeouts(unsigned int* host_count)

@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -13,7 +14,7 @@ namespace kop {
 // Host side: static validation (the paper's Gate 1 analogue). Pure integer checks, no CUDA call.
 // ------------------------------------------------------------------------------------------
 
-inline bool dtype_ok(kop_dtype_t d) { return d == KOP_F32 || d == KOP_BF16; }
+inline bool dtype_ok(kop_dtype_t d) { return d == KOP_F32 || d == KOP_BF16 || d == KOP_F16; }
 inline int elem_size(kop_dtype_t d) { return d == KOP_F32 ? 4 : 2; }
 inline bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
@@ -270,6 +271,55 @@ struct Elem<__nv_bfloat16> {
         Vec16 v;
 #pragma unroll
         for (int i = 0; i < 4; ++i) v.w[i] = 0xFF80FF80u;
+        return v;
+    }
+};
+
+template <>
+struct Elem<__half> {
+    static constexpr int kPerVec = 8;
+    __device__ __forceinline__ static void unpack(const Vec16& v, float (&f)[8])
+    {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 t = __half22float2(*reinterpret_cast<const __half2*>(&v.w[i]));
+            f[2 * i] = t.x;
+            f[2 * i + 1] = t.y;
+        }
+    }
+    // Round to nearest even, two values per cvt; values beyond 65504 become infinity, as IEEE requires.
+    __device__ __forceinline__ static Vec16 pack(const float (&f)[8])
+    {
+        Vec16 v;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            __half2 h = __floats2half2_rn(f[2 * i], f[2 * i + 1]);
+            v.w[i] = *reinterpret_cast<uint32_t*>(&h);
+        }
+        return v;
+    }
+    __device__ __forceinline__ static void unpack2(const Vec16& v, float2 (&f)[4])
+    {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) f[i] = __half22float2(*reinterpret_cast<const __half2*>(&v.w[i]));
+    }
+    __device__ __forceinline__ static Vec16 pack2(const float2 (&f)[4])
+    {
+        Vec16 v;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            __half2 h = __floats2half2_rn(f[i].x, f[i].y);
+            v.w[i] = *reinterpret_cast<uint32_t*>(&h);
+        }
+        return v;
+    }
+    __device__ __forceinline__ static float load1(const __half* p) { return __half2float(*p); }
+    __device__ __forceinline__ static void store1(__half* p, float f) { *p = __float2half_rn(f); }
+    __device__ __forceinline__ static Vec16 fill_neg_inf()
+    {
+        Vec16 v;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) v.w[i] = 0xFC00FC00u;
         return v;
     }
 };

@@ -401,7 +401,9 @@ extern "C" kop_status_t kop_bias_gelu_residual_layernorm(
     return dtype == KOP_F32
                ? launch_ln<float, kProBiasGeluResidual>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
                                   x_row_stride, res_row_stride, y_row_stride, eps, s)
-               : launch_ln<__nv_bfloat16, kProBiasGeluResidual>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
+               : dtype == KOP_BF16 ? launch_ln<__nv_bfloat16, kProBiasGeluResidual>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
+                                          x_row_stride, res_row_stride, y_row_stride, eps, s)
+               : launch_ln<__half, kProBiasGeluResidual>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
                                           x_row_stride, res_row_stride, y_row_stride, eps, s);
 }
 
@@ -436,10 +438,14 @@ extern "C" kop_status_t kop_residual_layernorm(const void* x, const void* residu
         return dtype == KOP_F32
                    ? launch_ln<float, kProResidual>(x, residual, nullptr, gamma, beta, y, mean, rstd, rows, hidden,
                                                     x_row_stride, rs, y_row_stride, eps, s)
-                   : launch_ln<__nv_bfloat16, kProResidual>(x, residual, nullptr, gamma, beta, y, mean, rstd, rows,
+                   : dtype == KOP_BF16 ? launch_ln<__nv_bfloat16, kProResidual>(x, residual, nullptr, gamma, beta, y, mean, rstd, rows,
+                                                            hidden, x_row_stride, rs, y_row_stride, eps, s)
+                   : launch_ln<__half, kProResidual>(x, residual, nullptr, gamma, beta, y, mean, rstd, rows,
                                                             hidden, x_row_stride, rs, y_row_stride, eps, s);
     return dtype == KOP_F32 ? launch_ln<float, kProNone>(x, x, nullptr, gamma, beta, y, mean, rstd, rows, hidden,
                                                          x_row_stride, rs, y_row_stride, eps, s)
-                            : launch_ln<__nv_bfloat16, kProNone>(x, x, nullptr, gamma, beta, y, mean, rstd, rows,
+                            : dtype == KOP_BF16 ? launch_ln<__nv_bfloat16, kProNone>(x, x, nullptr, gamma, beta, y, mean, rstd, rows,
+                                                                 hidden, x_row_stride, rs, y_row_stride, eps, s)
+                            : launch_ln<__half, kProNone>(x, x, nullptr, gamma, beta, y, mean, rstd, rows,
                                                                  hidden, x_row_stride, rs, y_row_stride, eps, s);
 }

@@ -417,7 +417,7 @@ kop_status_t gemm_nt(cublasHandle_t h, const void* A, const void* Wt, void* Cout
                      int64_t K, kop_dtype_t dtype)
 {
     const float alpha = 1.0f, beta = 0.0f;
-    const cudaDataType_t t = dtype == KOP_F32 ? CUDA_R_32F : CUDA_R_16BF;
+    const cudaDataType_t t = dtype == KOP_F32 ? CUDA_R_32F : dtype == KOP_BF16 ? CUDA_R_16BF : CUDA_R_16F;
     if (M > 0x7FFFFFFFLL || N > 0x7FFFFFFFLL || K > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
     cublasStatus_t st = cublasGemmEx(h, CUBLAS_OP_T, CUBLAS_OP_N, (int)N, (int)M, (int)K, &alpha, Wt, t,
                                      (int)K, A, t, (int)K, &beta, Cout, t, (int)N, CUBLAS_COMPUTE_32F,
@@ -460,7 +460,7 @@ kop_status_t gemm_nt_plus_residual(MlpHandle* mh, const void* A, const void* Wt,
     cublasLtHandle_t lt = reinterpret_cast<cublasLtHandle_t>(mh->cb);   // a cuBLAS handle is also a cuBLASLt handle
     if (!mh->plan_valid || mh->plan_m != M || mh->plan_n != N || mh->plan_k != K || mh->plan_dtype != dtype) {
         drop_plan(mh);
-        const cudaDataType_t t = dtype == KOP_F32 ? CUDA_R_32F : CUDA_R_16BF;
+        const cudaDataType_t t = dtype == KOP_F32 ? CUDA_R_32F : dtype == KOP_BF16 ? CUDA_R_16BF : CUDA_R_16F;
         const cublasOperation_t ta = CUBLAS_OP_T, tb = CUBLAS_OP_N;
         bool ok = cublasLtMatmulDescCreate(&mh->op, CUBLAS_COMPUTE_32F, CUDA_R_32F) == CUBLAS_STATUS_SUCCESS;
         ok = ok && cublasLtMatmulDescSetAttribute(mh->op, CUBLASLT_MATMUL_DESC_TRANSA, &ta, sizeof(ta)) == CUBLAS_STATUS_SUCCESS;
@@ -516,7 +516,8 @@ extern "C" kop_status_t kop_rmsnorm(const void* x, const float* weight, void* y,
     cudaStream_t s = as_stream(stream);
     return dtype == KOP_F32
                ? launch_rmsnorm<float>(x, weight, y, rows, hidden, x_row_stride, y_row_stride, eps, s)
-               : launch_rmsnorm<__nv_bfloat16>(x, weight, y, rows, hidden, x_row_stride, y_row_stride, eps, s);
+               : dtype == KOP_BF16 ? launch_rmsnorm<__nv_bfloat16>(x, weight, y, rows, hidden, x_row_stride, y_row_stride, eps, s)
+               : launch_rmsnorm<__half>(x, weight, y, rows, hidden, x_row_stride, y_row_stride, eps, s);
 }
 
 extern "C" kop_status_t kop_silu_mul(const void* gate_up, void* out, int64_t rows, int64_t inter,
@@ -544,7 +545,8 @@ extern "C" kop_status_t kop_silu_mul(const void* gate_up, void* out, int64_t row
     cudaStream_t s = as_stream(stream);
     return dtype == KOP_F32
                ? launch_silu_mul<float>(gate_up, out, rows, inter, in_row_stride, out_row_stride, s)
-               : launch_silu_mul<__nv_bfloat16>(gate_up, out, rows, inter, in_row_stride, out_row_stride, s);
+               : dtype == KOP_BF16 ? launch_silu_mul<__nv_bfloat16>(gate_up, out, rows, inter, in_row_stride, out_row_stride, s)
+               : launch_silu_mul<__half>(gate_up, out, rows, inter, in_row_stride, out_row_stride, s);
 }
 
 extern "C" kop_status_t kop_silu_mul_interleaved(const void* gate_up, void* out, int64_t rows, int64_t inter,
@@ -572,7 +574,8 @@ extern "C" kop_status_t kop_silu_mul_interleaved(const void* gate_up, void* out,
     cudaStream_t s = as_stream(stream);
     return dtype == KOP_F32
                ? launch_silu_mul_interleaved<float>(gate_up, out, rows, inter, in_row_stride, out_row_stride, s)
-               : launch_silu_mul_interleaved<__nv_bfloat16>(gate_up, out, rows, inter, in_row_stride, out_row_stride, s);
+               : dtype == KOP_BF16 ? launch_silu_mul_interleaved<__nv_bfloat16>(gate_up, out, rows, inter, in_row_stride, out_row_stride, s)
+               : launch_silu_mul_interleaved<__half>(gate_up, out, rows, inter, in_row_stride, out_row_stride, s);
 }
 
 extern "C" kop_status_t kop_residual_add(const void* a, const void* b, void* out, int64_t rows,
@@ -597,7 +600,8 @@ extern "C" kop_status_t kop_residual_add(const void* a, const void* b, void* out
     cudaStream_t s = as_stream(stream);
     return dtype == KOP_F32
                ? launch_residual_add<float>(a, b, out, rows, cols, a_row_stride, b_row_stride, out_row_stride, s)
-               : launch_residual_add<__nv_bfloat16>(a, b, out, rows, cols, a_row_stride, b_row_stride, out_row_stride, s);
+               : dtype == KOP_BF16 ? launch_residual_add<__nv_bfloat16>(a, b, out, rows, cols, a_row_stride, b_row_stride, out_row_stride, s)
+               : launch_residual_add<__half>(a, b, out, rows, cols, a_row_stride, b_row_stride, out_row_stride, s);
 }
 
 extern "C" size_t kop_rmsnorm_swiglu_residual_workspace_bytes(int64_t rows, int64_t hidden,

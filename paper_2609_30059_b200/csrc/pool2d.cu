@@ -211,6 +211,11 @@ __device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&f)[8])
     Elem<__nv_bfloat16>::unpack(ld_stream(p), f);
 }
 
+__device__ __forceinline__ void load8(const __half* p, float (&f)[8])
+{
+    Elem<__half>::unpack(ld_stream(p), f);
+}
+
 // Horizontal reductions of one input row for this thread's four outputs. KS == 3: windows of columns
 // (2j-1, 2j, 2j+1) relative to the thread's first column, v[0] being the halo, which is the left
 // neighbour lane's last column (a shuffle; lane 0 of a warp loads it); KS == 2: (2j, 2j+1). Rows outside
@@ -252,6 +257,16 @@ __device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16* dst, const 
     w.x = *reinterpret_cast<const uint32_t*>(&a);
     w.y = *reinterpret_cast<const uint32_t*>(&b);
     *reinterpret_cast<uint2*>(dst) = w;                   // four outputs = 8 bytes, 8-byte aligned (OW % 4 == 0)
+}
+
+template <>
+__device__ __forceinline__ void store4<__half>(__half* dst, const float (&o)[4])
+{
+    const __half2 a = __floats2half2_rn(o[0], o[1]), b = __floats2half2_rn(o[2], o[3]);
+    uint2 w;
+    w.x = *reinterpret_cast<const uint32_t*>(&a);
+    w.y = *reinterpret_cast<const uint32_t*>(&b);
+    *reinterpret_cast<uint2*>(dst) = w;
 }
 
 template <typename T, int MODE, int KS>
@@ -478,6 +493,8 @@ extern "C" kop_status_t kop_affine_relu_pool2d(const void* x, const float* scale
     cudaStream_t s = as_stream(stream);
     return dtype == KOP_F32 ? launch_pool<float>(x, scale, shift, y, N, C, (int)H, (int)W, (int)OH, (int)OW, kh, kw, sh,
                                                  sw, ph, pw, mode, relu != 0, s)
-                            : launch_pool<__nv_bfloat16>(x, scale, shift, y, N, C, (int)H, (int)W, (int)OH, (int)OW, kh,
+                            : dtype == KOP_BF16 ? launch_pool<__nv_bfloat16>(x, scale, shift, y, N, C, (int)H, (int)W, (int)OH, (int)OW, kh,
+                                                         kw, sh, sw, ph, pw, mode, relu != 0, s)
+                            : launch_pool<__half>(x, scale, shift, y, N, C, (int)H, (int)W, (int)OH, (int)OW, kh,
                                                          kw, sh, sw, ph, pw, mode, relu != 0, s);
 }

@@ -219,7 +219,8 @@ extern "C" kop_status_t kop_row_scale(const void* a, const void* b, void* out, i
     if ((st = check_device()) != KOP_OK) return st;
     cudaStream_t s = as_stream(stream);
     return dtype == KOP_F32 ? launch_row_scale<float>(a, b, out, rows, cols, b_row_stride, out_row_stride, s)
-                            : launch_row_scale<__nv_bfloat16>(a, b, out, rows, cols, b_row_stride, out_row_stride, s);
+                            : dtype == KOP_BF16 ? launch_row_scale<__nv_bfloat16>(a, b, out, rows, cols, b_row_stride, out_row_stride, s)
+                            : launch_row_scale<__half>(a, b, out, rows, cols, b_row_stride, out_row_stride, s);
 }
 
 extern "C" kop_status_t kop_matvec_bias(const void* x, const float* w, float b_sum, float* out, int64_t rows,
@@ -243,5 +244,6 @@ extern "C" kop_status_t kop_matvec_bias(const void* x, const float* w, float b_s
     if ((st = check_device()) != KOP_OK) return st;
     cudaStream_t s = as_stream(stream);
     return dtype == KOP_F32 ? launch_matvec<float>(x, w, b_sum, out, rows, k, x_row_stride, s)
-                            : launch_matvec<__nv_bfloat16>(x, w, b_sum, out, rows, k, x_row_stride, s);
+                            : dtype == KOP_BF16 ? launch_matvec<__nv_bfloat16>(x, w, b_sum, out, rows, k, x_row_stride, s)
+                            : launch_matvec<__half>(x, w, b_sum, out, rows, k, x_row_stride, s);
 }

@@ -244,5 +244,6 @@ extern "C" kop_status_t kop_cumsum_rows(const void* x, const unsigned char* mask
     const int ex = exclusive != 0, rv = reverse != 0;
     return dtype == KOP_F32
                ? launch_cumsum<float>(x, mask, y, rows, cols, x_row_stride, mask_row_stride, y_row_stride, ex, rv, s)
-               : launch_cumsum<__nv_bfloat16>(x, mask, y, rows, cols, x_row_stride, mask_row_stride, y_row_stride, ex, rv, s);
+               : dtype == KOP_BF16 ? launch_cumsum<__nv_bfloat16>(x, mask, y, rows, cols, x_row_stride, mask_row_stride, y_row_stride, ex, rv, s)
+               : launch_cumsum<__half>(x, mask, y, rows, cols, x_row_stride, mask_row_stride, y_row_stride, ex, rv, s);
 }

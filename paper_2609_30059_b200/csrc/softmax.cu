@@ -245,5 +245,6 @@ extern "C" kop_status_t kop_softmax_scale_bias(const void* x, const float* bias,
     cudaStream_t s = as_stream(stream);
     return dtype == KOP_F32
                ? launch_softmax<float>(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale, s)
-               : launch_softmax<__nv_bfloat16>(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale, s);
+               : dtype == KOP_BF16 ? launch_softmax<__nv_bfloat16>(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale, s)
+               : launch_softmax<__half>(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale, s);
 }

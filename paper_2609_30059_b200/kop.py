@@ -17,7 +17,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libkop.so")
 
 KOP_OK = 0
-KOP_F32, KOP_BF16 = 0, 1
+KOP_F32, KOP_BF16, KOP_F16 = 0, 1, 2
 STATUS_NAMES = [
     "KOP_OK", "KOP_ERR_NULL_POINTER", "KOP_ERR_BAD_SHAPE", "KOP_ERR_BAD_STRIDE",
     "KOP_ERR_UNSUPPORTED_DTYPE", "KOP_ERR_MISALIGNED", "KOP_ERR_BAD_ALIAS",
@@ -102,7 +102,9 @@ def _dtype_tag(t: torch.Tensor) -> int:
         return KOP_F32
     if t.dtype == torch.bfloat16:
         return KOP_BF16
-    raise TypeError(f"libkop data tensors are float32 or bfloat16, got {t.dtype}")
+    if t.dtype == torch.float16:
+        return KOP_F16
+    raise TypeError(f"libkop data tensors are float32, bfloat16 or float16, got {t.dtype}")
 
 
 def _rows2d(t: torch.Tensor, name: str):

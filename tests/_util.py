@@ -6,7 +6,9 @@ import torch
 
 # Tolerances of the comparison against the float64 oracle, by data dtype of the call:
 # pass iff |got - ref| <= tol * max(1, |ref|) for every element (absolute below 1, relative above).
-TOL = {torch.float32: 1e-5, torch.bfloat16: 2e-2}
+# fp16 data (a widening step beyond the benchmark dtypes): the final RNE store alone is 2^-11 = 4.9e-4 relative
+# and the hardware tanh / ex2 approximations add up to about as much, so 2e-3 leaves a factor of two to four.
+TOL = {torch.float32: 1e-5, torch.bfloat16: 2e-2, torch.float16: 2e-3}
 SENTINEL = 0x5A
 
 

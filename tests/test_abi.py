@@ -84,7 +84,7 @@ def test_layernorm_validation(L):
     assert call(a9=0) == SHAPE
     assert call(a8=-2) == SHAPE
     assert call(a10=63) == STRIDE and call(a11=8) == STRIDE and call(a12=1) == STRIDE
-    assert call(a14=2) == DTYPE
+    assert call(a14=3) == DTYPE
     assert call(a13=-1.0) == SHAPE
     assert call(a2=R + 2) == MISAL
     assert call(a5=P + 64) == ALIAS               # y overlaps x without being x
@@ -153,7 +153,7 @@ def test_row_ops_validation(L):
     assert L.kop_row_scale(P, Q, R, 4, 64, 63, 64, 0, None) == STRIDE
     assert L.kop_row_scale(P, Q, Q + 8, 4, 64, 64, 64, 0, None) == ALIAS       # out overlaps b
     assert L.kop_row_scale(R + 16, Q, R, 4, 64, 64, 64, 0, None) == ALIAS      # a overlaps out
-    assert L.kop_row_scale(P, Q, R, 4, 64, 64, 64, 2, None) == DTYPE
+    assert L.kop_row_scale(P, Q, R, 4, 64, 64, 64, 3, None) == DTYPE
     assert L.kop_row_scale(P + 1, Q, R, 4, 64, 64, 64, 1, None) == MISAL
     assert L.kop_matvec_bias(P, Q, 0.5, R, 0, 64, 64, 1, None) == OK
     assert L.kop_matvec_bias(P, None, 0.5, R, 4, 64, 64, 1, None) == NULLP

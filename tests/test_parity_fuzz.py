@@ -1,6 +1,6 @@
 """Randomised GPU parity sweep: for every entry point, a few hundred small random shapes (seeded, so the
 sweep is reproducible) with random dtypes, strides, alignments and options, each compared with the
-float64 oracle under the usual rule |got - ref| <= tol * max(1, |ref|) (1e-5 fp32 data, 2e-2 bf16 data).
+float64 oracle under the usual rule |got - ref| <= tol * max(1, |ref|) (1e-5 fp32 data, 2e-2 bf16 data, 2e-3 fp16 data).
 The hand-picked cases in the other parity files aim at known kernel boundaries; this sweep is for the
 ones nobody thought of (odd lengths next to vector multiples, one-row and one-column tensors, sizes that
 straddle the kernels' dispatch thresholds)."""
@@ -14,7 +14,7 @@ from paper_2609_30059_b200 import synth
 from tests._util import assert_close, to_f64, tol_of
 
 pytestmark = pytest.mark.gpu
-F32, BF16 = torch.float32, torch.bfloat16
+F32, BF16, F16 = torch.float32, torch.bfloat16, torch.float16
 
 
 @pytest.fixture(scope="module")
@@ -59,7 +59,7 @@ def strided(rng, t):
 def test_fuzz_row_kernels(kop):
     rng = np.random.default_rng(2609_30059)
     for it in range(120):
-        dtype = BF16 if rng.integers(0, 2) else F32
+        dtype = (F32, BF16, F16)[int(rng.integers(0, 3))]
         tol = tol_of(dtype)
         rows, cols = pick_len(rng, 70), pick_len(rng, 3000)
         seed = int(rng.integers(0, 1 << 30))
@@ -131,7 +131,7 @@ def test_fuzz_row_kernels(kop):
 def test_fuzz_image_kernels(kop):
     rng = np.random.default_rng(30059_2609)
     for it in range(100):
-        dtype = BF16 if rng.integers(0, 2) else F32
+        dtype = (F32, BF16, F16)[int(rng.integers(0, 3))]
         tol = tol_of(dtype)
         N, H, W = int(rng.integers(1, 5)), pick_len(rng, 40), pick_len(rng, 40)
         groups = int(rng.choice([1, 2, 3, 4, 8]))
