@@ -170,11 +170,14 @@ double kopref_gelu_tanh(double u)
  * ("residual + norm" and "normalization fusion" in the fusion agent's list,
  * "activation + bias fusion" for the prologue.)  v is never rounded.
  * mean / rstd may be NULL. */
-int kopref_bias_gelu_residual_layernorm(const void* x, const void* residual,
+/* The exact (error-function) GELU: 0.5 u (1 + erf(u / sqrt 2)), the form without the tanh approximation. */
+double kopref_gelu_erf(double u) { return 0.5 * u * (1.0 + erf(u * 0.70710678118654752440)); }
+
+static int bias_gelu_residual_layernorm_impl(const void* x, const void* residual,
         const float* bias, const float* gamma, const float* beta,
         double* y, double* mean, double* rstd,
         int64_t rows, int64_t hidden, int64_t x_row_stride, int64_t res_row_stride,
-        int64_t y_row_stride, double eps, int dtype, int threads)
+        int64_t y_row_stride, double eps, int dtype, int threads, int erf_form)
 {
     if (!x || !residual || !bias || !gamma || !beta || !y) return -1;
     if (rows < 0 || hidden <= 0 || bad_dtype(dtype)) return -1;
@@ -186,7 +189,8 @@ int kopref_bias_gelu_residual_layernorm(const void* x, const void* residual,
         double sum = 0.0;
         for (int64_t j = 0; j < hidden; ++j) {
             double u = load_elem(x, i * x_row_stride + j, dtype) + (double)bias[j];
-            double v = load_elem(residual, i * res_row_stride + j, dtype) + kopref_gelu_tanh(u);
+            double v = load_elem(residual, i * res_row_stride + j, dtype)
+                     + (erf_form ? kopref_gelu_erf(u) : kopref_gelu_tanh(u));
             yr[j] = v;
             sum += v;
         }
@@ -204,6 +208,27 @@ int kopref_bias_gelu_residual_layernorm(const void* x, const void* residual,
         if (rstd) rstd[i] = rs;
     }
     return 0;
+}
+
+int kopref_bias_gelu_residual_layernorm(const void* x, const void* residual,
+        const float* bias, const float* gamma, const float* beta,
+        double* y, double* mean, double* rstd,
+        int64_t rows, int64_t hidden, int64_t x_row_stride, int64_t res_row_stride,
+        int64_t y_row_stride, double eps, int dtype, int threads)
+{
+    return bias_gelu_residual_layernorm_impl(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
+                                             x_row_stride, res_row_stride, y_row_stride, eps, dtype, threads, 0);
+}
+
+/* The same segment with the error-function GELU in place of the tanh form. */
+int kopref_bias_erfgelu_residual_layernorm(const void* x, const void* residual,
+        const float* bias, const float* gamma, const float* beta,
+        double* y, double* mean, double* rstd,
+        int64_t rows, int64_t hidden, int64_t x_row_stride, int64_t res_row_stride,
+        int64_t y_row_stride, double eps, int dtype, int threads)
+{
+    return bias_gelu_residual_layernorm_impl(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
+                                             x_row_stride, res_row_stride, y_row_stride, eps, dtype, threads, 1);
 }
 
 /* ---- inference BatchNorm affine + ReLU + global average pool (NCHW) ----------

@@ -36,6 +36,9 @@ def lib() -> C.CDLL:
         _lib.kopref_gelu_tanh.argtypes = [dbl]
         _lib.kopref_softmax_scale_bias.argtypes = [vp, vp, vp, i64, i64, i64, i64, dbl, C.c_int, C.c_int]
         _lib.kopref_bias_gelu_residual_layernorm.argtypes = [vp] * 8 + [i64] * 5 + [dbl, C.c_int, C.c_int]
+        _lib.kopref_bias_erfgelu_residual_layernorm.argtypes = [vp] * 8 + [i64] * 5 + [dbl, C.c_int, C.c_int]
+        _lib.kopref_gelu_erf.restype = dbl
+        _lib.kopref_gelu_erf.argtypes = [dbl]
         _lib.kopref_bn_relu_avgpool.argtypes = [vp] * 5 + [i64] * 4 + [C.c_int, C.c_int]
         _lib.kopref_ce_loss_rowwise.argtypes = [vp] * 5 + [i64] * 3 + [C.c_int, C.c_int]
         _lib.kopref_rmsnorm.argtypes = [vp] * 3 + [i64] * 4 + [dbl, C.c_int, C.c_int]
@@ -140,8 +143,12 @@ def softmax_scale_bias(x, bias, scale, threads=1) -> np.ndarray:
     return y
 
 
-def bias_gelu_residual_layernorm(x, residual, bias, gamma, beta, eps, threads=1):
-    """Returns (y, mean, rstd)."""
+def gelu_erf(u: float) -> float:
+    return lib().kopref_gelu_erf(float(u))
+
+
+def bias_gelu_residual_layernorm(x, residual, bias, gamma, beta, eps, threads=1, erf_form=False):
+    """Returns (y, mean, rstd). erf_form: the error-function GELU instead of the tanh form."""
     xa, dt = as_data(x)
     ra, dt2 = as_data(residual)
     assert dt == dt2 and xa.shape == ra.shape
@@ -150,7 +157,8 @@ def bias_gelu_residual_layernorm(x, residual, bias, gamma, beta, eps, threads=1)
     y = np.empty((rows, hidden), dtype=np.float64)
     mean = np.empty(rows, dtype=np.float64)
     rstd = np.empty(rows, dtype=np.float64)
-    _check(lib().kopref_bias_gelu_residual_layernorm(
+    fn = lib().kopref_bias_erfgelu_residual_layernorm if erf_form else lib().kopref_bias_gelu_residual_layernorm
+    _check(fn(
         _p(xa), _p(ra), _p(b), _p(g), _p(be), _p(y), _p(mean), _p(rstd),
         rows, hidden, hidden, hidden, hidden, float(eps), dt, _nt(threads)),
         "bias_gelu_residual_layernorm")

@@ -781,3 +781,36 @@ def test_f16_widening_exhaustive_and_one_function_end_to_end():
     W2 = torch.from_numpy(f32(RNG.normal(0, 0.1, (16, 12)))).to(torch.float16)
     np.testing.assert_allclose(kopref.mlp_segment(h, w, W1, W2, 1e-6),
                                kopref.mlp_segment(h.double(), w, W1.double(), W2.double(), 1e-6), rtol=0, atol=1e-15)
+
+
+# --------------------------------------------------------------------------- error-function GELU
+
+def test_gelu_erf_and_the_erf_form_of_the_layernorm_segment():
+    # the scalar against 50-digit arithmetic, a library routine and its closed-form points
+    for u in [-8.0, -3.0, -1.0, -0.3, 0.0, 1e-8, 0.5, 1.0, 2.5, 6.0, 12.0]:
+        exact = float(mp.mpf(u) / 2 * (1 + mp.erf(mp.mpf(u) / mp.sqrt(2))))
+        assert kopref.gelu_erf(u) == pytest.approx(exact, rel=1e-14, abs=1e-15)      # 1 + erf cancels for u << 0
+        assert kopref.gelu_erf(u) == pytest.approx(0.5 * u * (1.0 + scipy.special.erf(u / math.sqrt(2.0))), rel=1e-14, abs=1e-15)
+    assert kopref.gelu_erf(0.0) == 0.0
+    assert kopref.gelu_erf(40.0) == 40.0 and kopref.gelu_erf(-40.0) == 0.0          # saturation
+    # gelu(u) - gelu(-u) = u for every u (erf is odd)
+    for u in [0.1, 0.7, 3.3]:
+        assert kopref.gelu_erf(u) - kopref.gelu_erf(-u) == pytest.approx(u, rel=1e-15)
+    # it differs from the tanh form where that approximation is off (about 1e-4..5e-4 around |u| = 2)
+    assert 1e-4 < abs(kopref.gelu_erf(2.0) - kopref.gelu_tanh(2.0)) < 1e-3
+    # the whole segment against torch in float64 (gelu approximate='none' is the erf form)
+    x = torch.from_numpy(f32(RNG.normal(0, 1, (6, 48))))
+    r = torch.from_numpy(f32(RNG.normal(0, 1, (6, 48))))
+    b = torch.from_numpy(f32(RNG.normal(0, 0.1, 48)))
+    g = torch.from_numpy(f32(RNG.normal(1, 0.02, 48)))
+    be = torch.from_numpy(f32(RNG.normal(0, 0.02, 48)))
+    y, mu, rs = kopref.bias_gelu_residual_layernorm(x, r, b, g, be, 1e-5, erf_form=True)
+    v = r.double() + F.gelu(x.double() + b.double(), approximate="none")
+    ref = F.layer_norm(v, (48,), g.double(), be.double(), 1e-5)
+    np.testing.assert_allclose(y, ref.numpy(), rtol=0, atol=1e-13)
+    np.testing.assert_allclose(mu, v.mean(dim=1).numpy(), rtol=0, atol=1e-14)
+    np.testing.assert_allclose(rs, 1.0 / torch.sqrt(v.var(dim=1, unbiased=False) + 1e-5).numpy(), rtol=1e-13)
+    # and the tanh form is untouched by the refactoring
+    y0, _, _ = kopref.bias_gelu_residual_layernorm(x, r, b, g, be, 1e-5)
+    v0 = r.double() + F.gelu(x.double() + b.double(), approximate="tanh")
+    np.testing.assert_allclose(y0, F.layer_norm(v0, (48,), g.double(), be.double(), 1e-5).numpy(), rtol=0, atol=1e-13)
