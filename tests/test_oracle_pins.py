@@ -796,8 +796,8 @@ def test_gelu_erf_and_the_erf_form_of_the_layernorm_segment():
     # gelu(u) - gelu(-u) = u for every u (erf is odd)
     for u in [0.1, 0.7, 3.3]:
         assert kopref.gelu_erf(u) - kopref.gelu_erf(-u) == pytest.approx(u, rel=1e-15)
-    # it differs from the tanh form where that approximation is off (about 1e-4..5e-4 around |u| = 2)
-    assert 1e-4 < abs(kopref.gelu_erf(2.0) - kopref.gelu_tanh(2.0)) < 1e-3
+    # it differs from the tanh form where that approximation is off (about 1e-4 around |u| = 2)
+    assert 5e-5 < abs(kopref.gelu_erf(2.0) - kopref.gelu_tanh(2.0)) < 5e-4
     # the whole segment against torch in float64 (gelu approximate='none' is the erf form)
     x = torch.from_numpy(f32(RNG.normal(0, 1, (6, 48))))
     r = torch.from_numpy(f32(RNG.normal(0, 1, (6, 48))))
