@@ -108,6 +108,20 @@ kop_status_t kop_bias_gelu_residual_layernorm(const void* x, const void* residua
                                               kop_dtype_t dtype, kop_stream_t stream);
 
 /*
+ * The same segment with the error-function GELU (the exact form, as in BERT- and ViT-style blocks; one of
+ * the coverage variants of the benchmark segment):
+ *   g = 0.5 u (1 + erf(u / sqrt 2)),  u = x + bias;  everything else as in kop_bias_gelu_residual_layernorm.
+ */
+kop_status_t kop_bias_erfgelu_residual_layernorm(const void* x, const void* residual,
+                                                 const float* bias, const float* gamma,
+                                                 const float* beta, void* y,
+                                                 float* mean, float* rstd,
+                                                 int64_t rows, int64_t hidden,
+                                                 int64_t x_row_stride, int64_t res_row_stride,
+                                                 int64_t y_row_stride, float eps,
+                                                 kop_dtype_t dtype, kop_stream_t stream);
+
+/*
  * Inference BatchNorm (pre-folded per-channel affine), ReLU and global average pool
  * (fusion agent: "reduction + pointwise"; the BN / pooling epilogues of the paper's
  * CNN models, next to preserved cuDNN convolutions):

@@ -35,13 +35,24 @@ __device__ __forceinline__ float2 gelu_residual2(float2 x, float2 b, float2 r)
     return __ffma2_rn(hu, t, __fadd2_rn(hu, r));
 }
 
-// What precedes the normalisation: kProBiasGeluResidual: v = residual + gelu(x + bias) (the benchmark
-// segment); kProResidual: v = x + residual; kProNone: v = x. The unused operands are never loaded.
-enum { kProBiasGeluResidual = 0, kProResidual = 1, kProNone = 2 };
+// The error-function form, 0.5 u (1 + erf(u / sqrt 2)); erff is accurate to a few ulp, which every data
+// type needs here (there is no hardware erf).
+__device__ __forceinline__ float gelu_erf(float u) { return 0.5f * u * (1.0f + erff(u * 0.7071067811865476f)); }
+
+// What precedes the normalisation: kProBiasGeluResidual: v = residual + gelu(x + bias) with the tanh-form
+// GELU (the benchmark segment); kProBiasErfGeluResidual: the same with the error-function GELU;
+// kProResidual: v = x + residual; kProNone: v = x. The unused operands are never loaded.
+enum { kProBiasGeluResidual = 0, kProResidual = 1, kProNone = 2, kProBiasErfGeluResidual = 3 };
+__host__ __device__ constexpr bool pro_has_residual(int pro) { return pro != kProNone; }
+__host__ __device__ constexpr bool pro_has_bias(int pro) { return pro == kProBiasGeluResidual || pro == kProBiasErfGeluResidual; }
 template <int PRO, bool kFastTanh>
 __device__ __forceinline__ float2 prologue2(float2 x, float2 b, float2 r)
 {
     if (PRO == kProBiasGeluResidual) return gelu_residual2<kFastTanh>(x, b, r);
+    if (PRO == kProBiasErfGeluResidual) {
+        const float2 u = __fadd2_rn(x, b);
+        return __fadd2_rn(r, make_float2(gelu_erf(u.x), gelu_erf(u.y)));
+    }
     if (PRO == kProResidual) return __fadd2_rn(x, r);
     return x;
 }
@@ -49,6 +60,7 @@ template <int PRO, bool kFastTanh>
 __device__ __forceinline__ float prologue1(float x, float b, float r)
 {
     if (PRO == kProBiasGeluResidual) return r + gelu_tanh<kFastTanh>(x + b);
+    if (PRO == kProBiasErfGeluResidual) return r + gelu_erf(x + b);
     if (PRO == kProResidual) return x + r;
     return x;
 }
@@ -79,7 +91,7 @@ ln_block_kernel(const T* __restrict__ x, const T* __restrict__ res, const float*
         const int v = k * blockDim.x + threadIdx.x;
         if (kFull || v < nvec) {
             rx[k] = ld_stream(xr + (int64_t)v * E);
-            if (PRO <= kProResidual) rres[k] = ld_stream(rr + (int64_t)v * E);
+            if (pro_has_residual(PRO)) rres[k] = ld_stream(rr + (int64_t)v * E);
             else rres[k] = Vec16{{0u, 0u, 0u, 0u}};
         } else {
             rx[k] = Vec16{{0u, 0u, 0u, 0u}};
@@ -92,7 +104,7 @@ ln_block_kernel(const T* __restrict__ x, const T* __restrict__ res, const float*
     for (int k = 0; k < VPT; ++k) {
         const int v = k * blockDim.x + threadIdx.x;
         float2 bb[P], fx[P], fr[P];
-        if (PRO == kProBiasGeluResidual && (kFull || v < nvec)) load_params<E, kWide>(bias + (int64_t)v * E, bb);
+        if (pro_has_bias(PRO) && (kFull || v < nvec)) load_params<E, kWide>(bias + (int64_t)v * E, bb);
         else {
 #pragma unroll
             for (int q = 0; q < P; ++q) bb[q] = make_float2(0.0f, 0.0f);
@@ -171,7 +183,7 @@ ln_pair_kernel(const T* __restrict__ x, const T* __restrict__ res, const float* 
             const int64_t v = (int64_t)k * blockDim.x + threadIdx.x;
             if (r == 0 || two) {
                 rx[r][k] = ld_stream(x + (row0 + r) * x_stride + v * E);
-                if (PRO <= kProResidual) rres[r][k] = ld_stream(res + (row0 + r) * r_stride + v * E);
+                if (pro_has_residual(PRO)) rres[r][k] = ld_stream(res + (row0 + r) * r_stride + v * E);
                 else rres[r][k] = Vec16{{0u, 0u, 0u, 0u}};
             } else {
                 rx[r][k] = Vec16{{0u, 0u, 0u, 0u}};
@@ -184,7 +196,7 @@ ln_pair_kernel(const T* __restrict__ x, const T* __restrict__ res, const float* 
     for (int k = 0; k < VPT; ++k) {
         const int64_t v = (int64_t)k * blockDim.x + threadIdx.x;
         float2 bb[P];
-        if (PRO == kProBiasGeluResidual) load_params<E, kWide>(bias + v * E, bb);
+        if (pro_has_bias(PRO)) load_params<E, kWide>(bias + v * E, bb);
         else {
 #pragma unroll
             for (int q = 0; q < P; ++q) bb[q] = make_float2(0.0f, 0.0f);
@@ -259,8 +271,8 @@ template <typename T, int PRO, bool kFast>
 __device__ __forceinline__ float ln_value(const T* xr, const T* rr, const float* bias, int64_t j)
 {
     const float xv = Elem<T>::load1(xr + j);
-    const float rv = PRO <= kProResidual ? Elem<T>::load1(rr + j) : 0.0f;
-    const float bv = PRO == kProBiasGeluResidual ? __ldg(bias + j) : 0.0f;
+    const float rv = pro_has_residual(PRO) ? Elem<T>::load1(rr + j) : 0.0f;
+    const float bv = pro_has_bias(PRO) ? __ldg(bias + j) : 0.0f;
     return prologue1<PRO, kFast>(xv, bv, rv);
 }
 
@@ -311,15 +323,15 @@ kop_status_t launch_ln(const void* xv, const void* rv, const float* bias, const 
     constexpr int E = Elem<T>::kPerVec;
     const float inv_hidden = (float)(1.0 / (double)hidden);
     if (rows > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
-    const bool vec = vec_ok(x, hidden, xs, sizeof(T)) && (PRO > kProResidual || vec_ok(r, hidden, rs, sizeof(T))) &&
-                     vec_ok(y, hidden, ys, sizeof(T)) && (PRO != kProBiasGeluResidual || aligned_to(bias, 16)) &&
+    const bool vec = vec_ok(x, hidden, xs, sizeof(T)) && (!pro_has_residual(PRO) || vec_ok(r, hidden, rs, sizeof(T))) &&
+                     vec_ok(y, hidden, ys, sizeof(T)) && (!pro_has_bias(PRO) || aligned_to(bias, 16)) &&
                      aligned_to(gamma, 16) && aligned_to(beta, 16);
     const int64_t nvec64 = hidden / E;
     if (vec && hidden <= kMaxRegisterRow) {
         const int nvec = (int)nvec64;
         // 32 values per thread (hidden 4096 -> 128-thread CTAs, eight 16-byte loads in flight per
         // thread and ~8 CTAs per SM); short rows use fewer, rows beyond 512 threads' worth use 64.
-        const bool wide = E == 8 && (PRO != kProBiasGeluResidual || aligned_to(bias, 32)) && aligned_to(gamma, 32) &&
+        const bool wide = E == 8 && (!pro_has_bias(PRO) || aligned_to(bias, 32)) && aligned_to(gamma, 32) &&
                           aligned_to(beta, 32);
         // Rows of 2048..8192 elements that split evenly into 16 values per thread go two per CTA
         // (parameters fetched once per pair) once there are enough pairs to fill the GPU.
@@ -373,12 +385,14 @@ kop_status_t launch_ln(const void* xv, const void* rv, const float* bias, const 
 }  // namespace
 }  // namespace kop
 
-extern "C" kop_status_t kop_bias_gelu_residual_layernorm(
+namespace kop {
+namespace {
+template <int PRO>
+kop_status_t bias_gelu_ln_entry(
     const void* x, const void* residual, const float* bias, const float* gamma, const float* beta,
     void* y, float* mean, float* rstd, int64_t rows, int64_t hidden, int64_t x_row_stride,
     int64_t res_row_stride, int64_t y_row_stride, float eps, kop_dtype_t dtype, kop_stream_t stream)
 {
-    using namespace kop;
     if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
     kop_status_t st = check_rows_cols(rows, hidden);
     if (st != KOP_OK) return st;
@@ -399,12 +413,32 @@ extern "C" kop_status_t kop_bias_gelu_residual_layernorm(
     if ((st = check_device()) != KOP_OK) return st;
     cudaStream_t s = as_stream(stream);
     return dtype == KOP_F32
-               ? launch_ln<float, kProBiasGeluResidual>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
+               ? launch_ln<float, PRO>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
                                   x_row_stride, res_row_stride, y_row_stride, eps, s)
-               : dtype == KOP_BF16 ? launch_ln<__nv_bfloat16, kProBiasGeluResidual>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
+               : dtype == KOP_BF16 ? launch_ln<__nv_bfloat16, PRO>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
                                           x_row_stride, res_row_stride, y_row_stride, eps, s)
-               : launch_ln<__half, kProBiasGeluResidual>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
+               : launch_ln<__half, PRO>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
                                           x_row_stride, res_row_stride, y_row_stride, eps, s);
+}
+}  // namespace
+}  // namespace kop
+
+extern "C" kop_status_t kop_bias_gelu_residual_layernorm(
+    const void* x, const void* residual, const float* bias, const float* gamma, const float* beta,
+    void* y, float* mean, float* rstd, int64_t rows, int64_t hidden, int64_t x_row_stride,
+    int64_t res_row_stride, int64_t y_row_stride, float eps, kop_dtype_t dtype, kop_stream_t stream)
+{
+    return kop::bias_gelu_ln_entry<kop::kProBiasGeluResidual>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
+                                                              x_row_stride, res_row_stride, y_row_stride, eps, dtype, stream);
+}
+
+extern "C" kop_status_t kop_bias_erfgelu_residual_layernorm(
+    const void* x, const void* residual, const float* bias, const float* gamma, const float* beta,
+    void* y, float* mean, float* rstd, int64_t rows, int64_t hidden, int64_t x_row_stride,
+    int64_t res_row_stride, int64_t y_row_stride, float eps, kop_dtype_t dtype, kop_stream_t stream)
+{
+    return kop::bias_gelu_ln_entry<kop::kProBiasErfGeluResidual>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
+                                                                 x_row_stride, res_row_stride, y_row_stride, eps, dtype, stream);
 }
 
 extern "C" kop_status_t kop_residual_layernorm(const void* x, const void* residual, const float* gamma,

@@ -53,6 +53,8 @@ def lib() -> C.CDLL:
     L.kop_status_string.argtypes = [i32]
     L.kop_softmax_scale_bias.argtypes = [vp, vp, vp, i64, i64, i64, i64, f32, i32, vp]
     L.kop_bias_gelu_residual_layernorm.argtypes = [vp] * 8 + [i64] * 5 + [f32, i32, vp]
+    L.kop_bias_erfgelu_residual_layernorm.argtypes = [vp] * 8 + [i64] * 5 + [f32, i32, vp]
+    L.kop_bias_erfgelu_residual_layernorm.restype = i32
     L.kop_bn_relu_avgpool.argtypes = [vp] * 5 + [i64] * 4 + [C.POINTER(i64), C.POINTER(i64), i32, vp]
     L.kop_ce_loss_rowwise.argtypes = [vp] * 5 + [i64] * 3 + [vp, sz, i32, vp]
     L.kop_ce_loss_rowwise_workspace_bytes.restype = sz
@@ -150,7 +152,8 @@ def kop_softmax_scale_bias(x, bias, scale, out=None, stream=None):
 
 
 def kop_bias_gelu_residual_layernorm(x, residual, bias, gamma, beta, eps, out=None, mean=None,
-                                     rstd=None, want_stats=True, stream=None):
+                                     rstd=None, want_stats=True, stream=None, erf_form=False):
+    """erf_form=True calls kop_bias_erfgelu_residual_layernorm (error-function GELU)."""
     rows, hidden, xs = _rows2d(x, "x")
     _, _, rs = _rows2d(residual, "residual")
     assert residual.shape == x.shape and residual.dtype == x.dtype
@@ -159,7 +162,8 @@ def kop_bias_gelu_residual_layernorm(x, residual, bias, gamma, beta, eps, out=No
     if want_stats:
         mean = torch.empty(rows, dtype=torch.float32, device=x.device) if mean is None else mean
         rstd = torch.empty(rows, dtype=torch.float32, device=x.device) if rstd is None else rstd
-    _check(lib().kop_bias_gelu_residual_layernorm(
+    fn = lib().kop_bias_erfgelu_residual_layernorm if erf_form else lib().kop_bias_gelu_residual_layernorm
+    _check(fn(
         x.data_ptr(), residual.data_ptr(), _param(bias, "bias", hidden), _param(gamma, "gamma", hidden),
         _param(beta, "beta", hidden), out.data_ptr(),
         None if mean is None else mean.data_ptr(), None if rstd is None else rstd.data_ptr(),

@@ -150,6 +150,33 @@ def test_layernorm_parity(kop, rows, hidden, dtype, seed):
         gd.check("ln")
 
 
+@pytest.mark.parametrize("rows,hidden,dtype", [(2048, 4096, BF16), (1185, 4096, BF16), (300, 4096, F32), (65, 256, BF16),
+                                               (9, 20480, F32), (33, 1001, F32), (7, 1, F32)])
+@pytest.mark.parametrize("seed", SEEDS)
+def test_layernorm_erf_gelu_parity(kop, rows, hidden, dtype, seed):
+    """The error-function GELU variant: same kernels, other prologue."""
+    x, r, b, g, be = synth.layernorm_inputs(rows, hidden, dtype, seed, "cuda")
+    y = Guarded((rows, hidden), dtype)
+    mean = Guarded((rows,), F32)
+    rstd = Guarded((rows,), F32)
+    kop.kop_bias_gelu_residual_layernorm(x, r, b, g, be, 1e-5, out=y.t, mean=mean.t, rstd=rstd.t, erf_form=True)
+    ry, rm, rr = kopref.bias_gelu_residual_layernorm(host(x), host(r), host(b), host(g), host(be), 1e-5, threads=None,
+                                                     erf_form=True)
+    tol = tol_of(dtype)
+    assert_close(y.t, ry, tol, "erf-gelu layernorm y")
+    assert_close(mean.t, rm, 1e-5 if dtype == F32 else 1e-3, "erf-gelu layernorm mean")
+    if hidden > 1:
+        assert_close(rstd.t, rr, 1e-5 if dtype == F32 else 1e-3, "erf-gelu layernorm rstd")
+    if dtype == BF16:
+        assert_bf16_tight(y.t, ry, "erf-gelu layernorm y")
+    for gb in (y, mean, rstd):
+        gb.check("erf-gelu layernorm")
+    # and it is not the tanh form: the two differ by the approximation error of the tanh form
+    if hidden >= 256 and dtype == F32:
+        y0, _, _ = kop.kop_bias_gelu_residual_layernorm(x, r, b, g, be, 1e-5)
+        assert float((y0 - y.t).abs().max()) > 1e-5
+
+
 def test_layernorm_full_config_seed0(kop):
     c = synth.CONFIGS["layernorm"]
     x, r, b, g, be = synth.layernorm_inputs(c["rows"], c["hidden"], c["dtype"], 0, "cuda")
