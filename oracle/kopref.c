@@ -643,3 +643,45 @@ int kopref_affine_relu_pool2d(const void* x, const float* scale, const float* sh
     }
     return 0;
 }
+
+/* ---- row reductions (the "Reduction" rows of the paper's result tables: sum / mean / max / min / argmax /
+ * argmin over the last dimension, and the LogSumExp reduction its planner names) ---------------------------
+ * op 0 sum, 1 mean, 2 max, 3 min, 4 logsumexp = m + ln sum_j exp(x_j - m) with m = max_j x_j.
+ * out[i] is the reduced value; index[i] (may be NULL; used for max / min only) is the position of the first
+ * element equal to the result. NaN: a NaN anywhere in the row makes every result NaN, and for max / min
+ * the index is that of the first NaN (a NaN ranks above every number, and below none, as in torch).
+ * logsumexp of a row of -inf is -inf; a +inf element gives +inf. Sums run in index order in double. */
+int kopref_reduce_rows(const void* x, double* out, int32_t* index, int64_t rows, int64_t cols,
+        int64_t x_row_stride, int op, int dtype, int threads)
+{
+    if (!x || !out || rows < 0 || cols <= 0 || op < 0 || op > 4 || bad_dtype(dtype)) return -1;
+    int nt = pick_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t i = 0; i < rows; ++i) {
+        double sum = 0.0, best = (op == 3) ? INFINITY : -INFINITY;
+        int64_t where = -1, first_nan = -1;
+        for (int64_t j = 0; j < cols; ++j) {
+            double v = load_elem(x, i * x_row_stride + j, dtype);
+            if (v != v) { if (first_nan < 0) first_nan = j; continue; }
+            sum += v;
+            if (where < 0 || (op == 3 ? v < best : v > best)) { best = v; where = j; }
+        }
+        double r;
+        if (first_nan >= 0) { r = NAN; where = first_nan; }
+        else if (op == 0) r = sum;
+        else if (op == 1) r = sum / (double)cols;
+        else if (op == 2 || op == 3) r = best;
+        else {
+            if (isinf(best)) r = best;                    /* all -inf, or a +inf present */
+            else {
+                double S = 0.0;
+                for (int64_t j = 0; j < cols; ++j) S += exp(load_elem(x, i * x_row_stride + j, dtype) - best);
+                r = best + log(S);
+            }
+        }
+        out[i] = r;
+        if (index && (op == 2 || op == 3)) index[i] = (int32_t)where;
+    }
+    return 0;
+}

@@ -51,6 +51,7 @@ def lib() -> C.CDLL:
         _lib.kopref_groupnorm_act.argtypes = [vp] * 6 + [i64] * 5 + [dbl, C.c_int, C.c_int, C.c_int]
         _lib.kopref_row_scale.argtypes = [vp, vp, vp, i64, i64, i64, i64, C.c_int, C.c_int]
         _lib.kopref_affine_relu_pool2d.argtypes = [vp] * 4 + [i64] * 4 + [C.c_int] * 10
+        _lib.kopref_reduce_rows.argtypes = [vp, vp, vp, i64, i64, i64, C.c_int, C.c_int, C.c_int]
         _lib.kopref_cumsum_rows.argtypes = [vp, vp, vp] + [i64] * 5 + [C.c_int] * 4
         _lib.kopref_matvec_bias.argtypes = [vp, vp, dbl, vp, i64, i64, i64, C.c_int, C.c_int]
     return _lib
@@ -330,6 +331,21 @@ def affine_relu_pool2d(x, scale, shift, kernel, stride, padding, mode="max", rel
                                            {"max": 0, "avg": 1}[mode], int(bool(relu)), dt, _nt(threads)),
            "affine_relu_pool2d")
     return y
+
+
+REDUCE_OPS = {"sum": 0, "mean": 1, "max": 2, "min": 3, "logsumexp": 4}
+
+
+def reduce_rows(x, op, threads=1):
+    """Reduction of each row of x [rows, cols]. Returns (values[rows] float64, index[rows] int32 or None);
+    the index (first position of the result) exists for "max" and "min" only."""
+    xa, dt = as_data(x)
+    rows, cols = xa.shape
+    out = np.empty(rows, dtype=np.float64)
+    idx = np.empty(rows, dtype=np.int32) if op in ("max", "min") else None
+    _check(lib().kopref_reduce_rows(_p(xa), _p(out), _p(idx), rows, cols, cols, REDUCE_OPS[op], dt, _nt(threads)),
+           "reduce_rows")
+    return out, idx
 
 
 def cumsum_rows(x, mask=None, exclusive=False, reverse=False, threads=1) -> np.ndarray:

@@ -814,3 +814,49 @@ def test_gelu_erf_and_the_erf_form_of_the_layernorm_segment():
     y0, _, _ = kopref.bias_gelu_residual_layernorm(x, r, b, g, be, 1e-5)
     v0 = r.double() + F.gelu(x.double() + b.double(), approximate="tanh")
     np.testing.assert_allclose(y0, F.layer_norm(v0, (48,), g.double(), be.double(), 1e-5).numpy(), rtol=0, atol=1e-13)
+
+
+# --------------------------------------------------------------------------- row reductions
+
+def test_reduce_rows_library_closed_forms_and_specials():
+    x = f32(RNG.normal(0, 2, (9, 203)))
+    xd = x.astype(np.float64)
+    np.testing.assert_allclose(kopref.reduce_rows(x, "sum")[0], [math.fsum(r) for r in xd], rtol=0, atol=1e-11)
+    np.testing.assert_allclose(kopref.reduce_rows(x, "mean")[0], [math.fsum(r) / 203 for r in xd], rtol=0, atol=1e-13)
+    v, i = kopref.reduce_rows(x, "max")
+    assert np.array_equal(v, xd.max(axis=1)) and np.array_equal(i, xd.argmax(axis=1))
+    v, i = kopref.reduce_rows(x, "min")
+    assert np.array_equal(v, xd.min(axis=1)) and np.array_equal(i, xd.argmin(axis=1))
+    np.testing.assert_allclose(kopref.reduce_rows(x, "logsumexp")[0], scipy.special.logsumexp(xd, axis=1), rtol=1e-14)
+    np.testing.assert_allclose(kopref.reduce_rows(x, "logsumexp")[0],
+                               torch.logsumexp(torch.from_numpy(xd), dim=1).numpy(), rtol=1e-14)
+    # closed forms
+    n = 1000
+    ramp = np.tile(np.arange(1, n + 1, dtype=np.float32), (2, 1))
+    assert kopref.reduce_rows(ramp, "sum")[0][0] == n * (n + 1) / 2 and kopref.reduce_rows(ramp, "mean")[0][1] == (n + 1) / 2
+    const = np.full((1, n), 0.75, dtype=np.float32)
+    assert kopref.reduce_rows(const, "logsumexp")[0][0] == pytest.approx(0.75 + math.log(n), rel=1e-15)
+    # ties: the first position wins; the logsumexp of huge values does not overflow
+    ties = np.array([[1, 5, 5, 2, 5], [3, 0, 0, 3, 3]], dtype=np.float32)
+    assert list(kopref.reduce_rows(ties, "max")[1]) == [1, 0] and list(kopref.reduce_rows(ties, "min")[1]) == [0, 1]
+    big = np.array([[1e30, 1e30]], dtype=np.float32)
+    assert kopref.reduce_rows(big, "logsumexp")[0][0] == pytest.approx(float(np.float32(1e30)) + math.log(2.0), rel=1e-15)
+    # NaN and infinities
+    xn = x.copy()
+    xn[3, 17] = np.nan
+    xn[3, 90] = np.nan
+    for op in ("sum", "mean", "max", "min", "logsumexp"):
+        v, i = kopref.reduce_rows(xn, op)
+        assert np.isnan(v[3]) and not np.isnan(np.delete(v, 3)).any()
+        if i is not None:
+            assert i[3] == 17
+    assert int(torch.from_numpy(xn[3]).argmax()) == 17                  # torch ranks NaN the same way
+    ninf = np.full((1, 8), -np.inf, dtype=np.float32)
+    assert kopref.reduce_rows(ninf, "logsumexp")[0][0] == -np.inf and kopref.reduce_rows(ninf, "max")[1][0] == 0
+    pinf = np.array([[0.0, np.inf, 1.0]], dtype=np.float32)
+    assert kopref.reduce_rows(pinf, "logsumexp")[0][0] == np.inf and kopref.reduce_rows(pinf, "max")[1][0] == 1
+    # bf16 / fp16 inputs and threads
+    tb = torch.from_numpy(x).to(torch.bfloat16)
+    assert np.array_equal(kopref.reduce_rows(tb, "max", threads=3)[0], tb.double().max(dim=1).values.numpy())
+    th = torch.from_numpy(x).to(torch.float16)
+    np.testing.assert_allclose(kopref.reduce_rows(th, "sum")[0], th.double().sum(dim=1).numpy(), rtol=0, atol=1e-11)
