@@ -100,6 +100,9 @@ def segment_bytes():
     e_out = q["N"] * q["C"] * ((q["H"] + 2 * q["padding"][0] - q["kernel"][0]) // q["stride"][0] + 1) * \
         ((q["W"] + 2 * q["padding"][1] - q["kernel"][1]) // q["stride"][1] + 1)
     out["pool2d"] = dict(bytes=(e_in + e_out) * 4 + 2 * q["C"] * 4, elems=e_in)
+    q = c["reduce"]
+    out["reduce_max"] = dict(bytes=q["rows"] * q["cols"] * 2 + q["rows"] * 8, elems=q["rows"] * q["cols"])
+    out["reduce_logsumexp"] = dict(bytes=q["rows"] * q["cols"] * 2 + q["rows"] * 4, elems=q["rows"] * q["cols"])
     u = c["cumsum"]
     out["cumsum"] = dict(bytes=2 * u["rows"] * u["cols"] * 4, elems=u["rows"] * u["cols"])
     return out
@@ -245,7 +248,7 @@ class Workload:
 
     ORDER = ["softmax_small", "softmax_large", "layernorm", "bn_pool", "ce_loss", "rmsnorm", "silu_mul", "residual_add"]
     # Beyond the benchmark configs (not part of `value`): the two kernels the paper's case studies print.
-    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc", "pool2d"]
+    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc", "pool2d", "reduce_max", "reduce_logsumexp"]
 
     def __init__(self, kop, device, seed, only=None, rows_div=1):
         """only: build just these segments (None = all, plus the MLP segment); rows_div cuts the row
@@ -314,6 +317,11 @@ class Workload:
             oh = (q["H"] + 2 * q["padding"][0] - q["kernel"][0]) // q["stride"][0] + 1
             ow = (q["W"] + 2 * q["padding"][1] - q["kernel"][1]) // q["stride"][1] + 1
             self.py = torch.empty((self.px.shape[0], q["C"], oh, ow), dtype=q["dtype"], device=dev)
+        if want & {"reduce_max", "reduce_logsumexp"}:
+            q = c["reduce"]
+            self.rx, _ = synth.softmax_inputs(cut(q["rows"]), q["cols"], q["dtype"], seed, dev)
+            self.rv = torch.empty(self.rx.shape[0], dtype=torch.float32, device=dev)
+            self.ri = torch.empty(self.rx.shape[0], dtype=torch.int32, device=dev)
         if "cumsum" in want:
             u = c["cumsum"]
             self.ux, _ = synth.cumsum_inputs(cut(u["rows"]), u["cols"], u["dtype"], seed, dev)
@@ -388,6 +396,10 @@ class Workload:
             q = c["pool2d"]
             k.kop_affine_relu_pool2d(self.px, self.pscale, self.pshift, q["kernel"], q["stride"], q["padding"],
                                      q["mode"], True, out=self.py)
+        elif name == "reduce_max":               # row max + argmax, bf16 [32768, 8192]
+            k.kop_reduce_rows(self.rx, "max", out=self.rv, index=self.ri)
+        elif name == "reduce_logsumexp":
+            k.kop_reduce_rows(self.rx, "logsumexp", out=self.rv)
         elif name == "cumsum":                   # inclusive running sum along rows, fp32 [32768, 4096]
             k.kop_cumsum_rows(self.ux, out=self.uy)
         else:

@@ -320,6 +320,19 @@ kop_status_t kop_affine_relu_pool2d(const void* x, const float* scale, const flo
                                     int ph, int pw, int mode, int relu, kop_dtype_t dtype, kop_stream_t stream);
 
 /*
+ * Row reductions (the "Reduction" rows of the paper's result tables and its planner's "single-pass
+ * reductions" / "LogSumExp reductions"), one read-only pass:
+ *   op 0 sum, 1 mean, 2 max, 3 min, 4 logsumexp = m + ln sum_j exp(x[i,j] - m), m = max_j x[i,j]
+ * x: [rows, cols] of `dtype`; out: fp32 [rows]; index: int32 [rows] or NULL, written for max / min only: the
+ * position of the first element equal to the result (argmax / argmin). A NaN in a row makes its result NaN;
+ * for max / min the index is then the position of the first NaN (a NaN outranks every number). logsumexp
+ * of a row of -inf is -inf, a +inf element gives +inf. Sums are fp32 trees in a fixed order; max / min
+ * and the indices are exact. cols and rows <= 2^31 - 1. out and index must not overlap x or each other.
+ */
+kop_status_t kop_reduce_rows(const void* x, float* out, int32_t* index, int64_t rows, int64_t cols,
+                             int64_t x_row_stride, int op, kop_dtype_t dtype, kop_stream_t stream);
+
+/*
  * Running sums along each row (the CumSum rows of the paper's per-kernel results table, L1-089 to L1-093:
  * plain, reverse, exclusive and masked cumulative sums; planner strategy "single-pass reductions" applied
  * to a scan). With m[i,k] = 1 when mask is NULL, else (mask[i,k] != 0):

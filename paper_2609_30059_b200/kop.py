@@ -80,6 +80,8 @@ def lib() -> C.CDLL:
     L.kop_groupnorm_act.restype = i32
     L.kop_affine_relu_pool2d.argtypes = [vp] * 4 + [i64] * 4 + [i32] * 9 + [vp]
     L.kop_affine_relu_pool2d.restype = i32
+    L.kop_reduce_rows.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, vp]
+    L.kop_reduce_rows.restype = i32
     L.kop_cumsum_rows.argtypes = [vp, vp, vp] + [i64] * 5 + [i32, i32, i32, vp]
     L.kop_cumsum_rows.restype = i32
     L.kop_groupnorm_wait_timeouts.argtypes = [C.POINTER(C.c_uint)]
@@ -371,6 +373,22 @@ def kop_affine_relu_pool2d(x, scale, shift, kernel, stride, padding, mode="max",
                                         {"max": 0, "avg": 1}[mode], int(bool(relu)), _dtype_tag(x), _stream(stream)),
            "kop_affine_relu_pool2d")
     return out
+
+
+REDUCE_OPS = {"sum": 0, "mean": 1, "max": 2, "min": 3, "logsumexp": 4}
+
+
+def kop_reduce_rows(x, op, out=None, index=None, want_index=True, stream=None):
+    """Returns (values fp32 [rows], index int32 [rows] or None); the index exists for "max" / "min" only."""
+    rows, cols, xs = _rows2d(x, "x")
+    out = torch.empty(rows, dtype=torch.float32, device=x.device) if out is None else out
+    if op in ("max", "min") and want_index and index is None:
+        index = torch.empty(rows, dtype=torch.int32, device=x.device)
+    if op not in ("max", "min"):
+        index = None
+    _check(lib().kop_reduce_rows(x.data_ptr(), out.data_ptr(), None if index is None else index.data_ptr(), rows, cols,
+                                 xs, REDUCE_OPS[op], _dtype_tag(x), _stream(stream)), "kop_reduce_rows")
+    return out, index
 
 
 def kop_cumsum_rows(x, mask=None, exclusive=False, reverse=False, out=None, stream=None):

@@ -29,6 +29,8 @@ CONFIGS = {
     # BatchNorm + ReLU + 3x3 / stride-2 max pool on a 112 x 112 map with 64 channels (a CNN stem)
     "pool2d": dict(N=64, C=64, H=112, W=112, kernel=(3, 3), stride=(2, 2), padding=(1, 1), mode="max",
                    dtype=torch.float32),
+    # row reductions (shape ours)
+    "reduce": dict(rows=32768, cols=8192, dtype=torch.bfloat16),
 }
 
 

@@ -224,6 +224,23 @@ def test_pool2d_validation(L):
     assert f(P, S, T, P + 64, *g, 3, 3, 2, 2, 1, 1, 0, 1, 0, None) == ALIAS    # y inside x
 
 
+def test_reduce_validation(L):
+    f = L.kop_reduce_rows
+    assert f(P, Q, R, 0, 64, 64, 0, 0, None) == OK
+    assert f(None, Q, R, 4, 64, 64, 0, 0, None) == NULLP
+    assert f(P, None, R, 4, 64, 64, 0, 0, None) == NULLP
+    assert f(P, Q, None, 4, 64, 64, 2, 0, None) != NULLP           # the index output is optional
+    assert f(P, Q, R, 4, 0, 64, 0, 0, None) == SHAPE
+    assert f(P, Q, R, 4, 64, 64, 5, 0, None) == SHAPE               # unknown operation
+    assert f(P, Q, R, 4, 64, 64, -1, 0, None) == SHAPE
+    assert f(P, Q, R, 4, 64, 63, 0, 0, None) == STRIDE
+    assert f(P, Q, R, 4, 64, 64, 0, 7, None) == DTYPE
+    assert f(P + 1, Q, R, 4, 64, 64, 0, 1, None) == MISAL
+    assert f(P, Q + 2, R, 4, 64, 64, 0, 0, None) == MISAL
+    assert f(P, P + 16, R, 4, 64, 64, 0, 0, None) == ALIAS          # out inside x
+    assert f(P, Q, Q + 8, 4, 64, 64, 2, 0, None) == ALIAS           # index overlaps out
+
+
 def test_mlp_driver_validation(L):
     f = L.kop_rmsnorm_swiglu_residual
     wsb = L.kop_rmsnorm_swiglu_residual_workspace_bytes(16, 64, 128, 1)

@@ -119,6 +119,15 @@ def test_fuzz_row_kernels(kop):
         # fp32 accumulation of `cols` products against a float64 sum: scale by the sum of magnitudes
         mag = (host(xv).double().abs() @ host(wv).double().abs()).numpy() + abs(bs)
         assert np.all(np.abs(got - ref) <= 1e-5 * np.maximum(1.0, mag)), "matvec " + what
+        # row reductions: extremes and their positions exactly, logsumexp to 1e-5
+        xr = strided(rng, x)
+        for op in ("max", "min"):
+            v, i = kop.kop_reduce_rows(xr, op)
+            rv, ri = kopref.reduce_rows(host(x), op)
+            assert np.array_equal(to_f64(v), rv) and np.array_equal(i.cpu().numpy(), ri), f"reduce {op} " + what
+        v, _ = kop.kop_reduce_rows(xr, "logsumexp")
+        rv, _ = kopref.reduce_rows(host(x), "logsumexp")
+        assert np.all(np.abs(to_f64(v) - rv) <= 1e-5 * np.maximum(1.0, np.abs(rv))), "reduce logsumexp " + what
         # running sums
         xc, mask = synth.cumsum_inputs(rows, cols, dtype, seed, "cuda")
         ex, rv, um = bool(rng.integers(0, 2)), bool(rng.integers(0, 2)), bool(rng.integers(0, 2))
