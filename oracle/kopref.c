@@ -685,3 +685,43 @@ int kopref_reduce_rows(const void* x, double* out, int32_t* index, int64_t rows,
     }
     return 0;
 }
+
+/* ---- bias + activation epilogue (the fusion agent's "activation + bias fusion": the pointwise tail of a
+ * Linear / GEMM call written once) -----------------------------------------------------------------------
+ *   u = x[i,j] + bias[j]  (bias NULL: u = x[i,j]);  y[i,j] = act(u)
+ * act: 0 identity, 1 relu (NaN stays NaN), 2 leaky_relu: u > 0 ? u : alpha u, 3 gelu (tanh form),
+ * 4 gelu (erf form), 5 silu: u / (1 + exp(-u)), 6 sigmoid: 1 / (1 + exp(-u)), 7 tanh,
+ * 8 mish: u tanh(ln(1 + exp(u))), 9 hardswish: u min(max(u + 3, 0), 6) / 6, 10 elu: u > 0 ? u : alpha (exp(u) - 1). */
+static double act_value(double u, int act, double alpha)
+{
+    switch (act) {
+    case 0: return u;
+    case 1: return (u != u) ? u : (u > 0.0 ? u : 0.0);
+    case 2: return u > 0.0 ? u : alpha * u;
+    case 3: return kopref_gelu_tanh(u);
+    case 4: return kopref_gelu_erf(u);
+    case 5: return u / (1.0 + exp(-u));
+    case 6: return 1.0 / (1.0 + exp(-u));
+    case 7: return tanh(u);
+    case 8: return u * tanh(u > 30.0 ? u : log1p(exp(u)));
+    case 9: { double r = u + 3.0; r = r < 0.0 ? 0.0 : (r > 6.0 ? 6.0 : r); return (u != u) ? u : u * r / 6.0; }
+    default: return u > 0.0 ? u : alpha * expm1(u);
+    }
+}
+
+double kopref_act_value(double u, int act, double alpha) { return act_value(u, act, alpha); }
+
+int kopref_bias_act(const void* x, const float* bias, double* y, int64_t rows, int64_t cols,
+        int64_t x_row_stride, int64_t y_row_stride, int act, double alpha, int dtype, int threads)
+{
+    if (!x || !y || rows < 0 || cols <= 0 || act < 0 || act > 10 || bad_dtype(dtype)) return -1;
+    int nt = pick_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t i = 0; i < rows; ++i)
+        for (int64_t j = 0; j < cols; ++j) {
+            double u = load_elem(x, i * x_row_stride + j, dtype) + (bias ? (double)bias[j] : 0.0);
+            y[i * y_row_stride + j] = act_value(u, act, alpha);
+        }
+    return 0;
+}

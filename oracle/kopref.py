@@ -52,6 +52,9 @@ def lib() -> C.CDLL:
         _lib.kopref_row_scale.argtypes = [vp, vp, vp, i64, i64, i64, i64, C.c_int, C.c_int]
         _lib.kopref_affine_relu_pool2d.argtypes = [vp] * 4 + [i64] * 4 + [C.c_int] * 10
         _lib.kopref_reduce_rows.argtypes = [vp, vp, vp, i64, i64, i64, C.c_int, C.c_int, C.c_int]
+        _lib.kopref_bias_act.argtypes = [vp, vp, vp, i64, i64, i64, i64, C.c_int, dbl, C.c_int, C.c_int]
+        _lib.kopref_act_value.restype = dbl
+        _lib.kopref_act_value.argtypes = [dbl, C.c_int, dbl]
         _lib.kopref_cumsum_rows.argtypes = [vp, vp, vp] + [i64] * 5 + [C.c_int] * 4
         _lib.kopref_matvec_bias.argtypes = [vp, vp, dbl, vp, i64, i64, i64, C.c_int, C.c_int]
     return _lib
@@ -346,6 +349,25 @@ def reduce_rows(x, op, threads=1):
     _check(lib().kopref_reduce_rows(_p(xa), _p(out), _p(idx), rows, cols, cols, REDUCE_OPS[op], dt, _nt(threads)),
            "reduce_rows")
     return out, idx
+
+
+ACTS = {"identity": 0, "relu": 1, "leaky_relu": 2, "gelu_tanh": 3, "gelu_erf": 4, "silu": 5, "sigmoid": 6,
+        "tanh": 7, "mish": 8, "hardswish": 9, "elu": 10}
+
+
+def act_value(u: float, act: str, alpha: float = 0.01) -> float:
+    return lib().kopref_act_value(float(u), ACTS[act], float(alpha))
+
+
+def bias_act(x, bias, act, alpha=0.01, threads=1) -> np.ndarray:
+    """y = act(x + bias) (bias None: act(x)); x [rows, cols], bias fp32 [cols]."""
+    xa, dt = as_data(x)
+    rows, cols = xa.shape
+    b = as_param(bias)
+    y = np.empty((rows, cols), dtype=np.float64)
+    _check(lib().kopref_bias_act(_p(xa), _p(b), _p(y), rows, cols, cols, cols, ACTS[act], float(alpha), dt, _nt(threads)),
+           "bias_act")
+    return y
 
 
 def cumsum_rows(x, mask=None, exclusive=False, reverse=False, threads=1) -> np.ndarray:

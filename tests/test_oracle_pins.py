@@ -860,3 +860,41 @@ def test_reduce_rows_library_closed_forms_and_specials():
     assert np.array_equal(kopref.reduce_rows(tb, "max", threads=3)[0], tb.double().max(dim=1).values.numpy())
     th = torch.from_numpy(x).to(torch.float16)
     np.testing.assert_allclose(kopref.reduce_rows(th, "sum")[0], th.double().sum(dim=1).numpy(), rtol=0, atol=1e-11)
+
+
+# --------------------------------------------------------------------------- bias + activation epilogue
+
+def test_bias_act_against_torch_mpmath_and_identities():
+    x = torch.from_numpy(f32(RNG.normal(0, 2.5, (6, 41))))
+    b = torch.from_numpy(f32(RNG.normal(0, 0.5, 41)))
+    u = x.double() + b.double()
+    lib_ref = {
+        "identity": u, "relu": torch.relu(u), "leaky_relu": F.leaky_relu(u, 0.2), "gelu_tanh": F.gelu(u, approximate="tanh"),
+        "gelu_erf": F.gelu(u, approximate="none"), "silu": F.silu(u), "sigmoid": torch.sigmoid(u), "tanh": torch.tanh(u),
+        "mish": F.mish(u), "hardswish": F.hardswish(u), "elu": F.elu(u, 0.2),
+    }
+    for act, ref in lib_ref.items():
+        np.testing.assert_allclose(kopref.bias_act(x, b, act, alpha=0.2), ref.numpy(), rtol=1e-13, atol=1e-14, err_msg=act)
+        # without bias it is the activation of x itself
+        np.testing.assert_allclose(kopref.bias_act(x, None, act, alpha=0.2),
+                                   kopref.bias_act(x.double(), torch.zeros(41), act, alpha=0.2), rtol=0, atol=0, err_msg=act)
+    # 50-digit values of the transcendental ones
+    for v in [-20.0, -3.0, -0.5, 0.0, 0.7, 4.0, 25.0, 60.0]:
+        m = mp.mpf(v)
+        assert kopref.act_value(v, "silu") == pytest.approx(float(m / (1 + mp.exp(-m))), rel=1e-14, abs=1e-300)
+        assert kopref.act_value(v, "sigmoid") == pytest.approx(float(1 / (1 + mp.exp(-m))), rel=1e-14)
+        assert kopref.act_value(v, "mish") == pytest.approx(float(m * mp.tanh(mp.log(1 + mp.exp(m)))), rel=1e-13, abs=1e-300)
+        assert kopref.act_value(v, "elu", 1.5) == pytest.approx(float(m if v > 0 else 1.5 * mp.expm1(m)), rel=1e-14)
+    # identities and closed-form points
+    for v in [0.3, 1.7, 9.0]:
+        assert kopref.act_value(v, "sigmoid") + kopref.act_value(-v, "sigmoid") == pytest.approx(1.0, rel=1e-15)
+        assert kopref.act_value(v, "silu") - kopref.act_value(-v, "silu") == pytest.approx(v, rel=1e-14)
+        assert kopref.act_value(v, "tanh") == -kopref.act_value(-v, "tanh")
+    assert kopref.act_value(-3.0, "hardswish") == 0.0 and kopref.act_value(3.0, "hardswish") == 3.0
+    assert kopref.act_value(1.0, "hardswish") == pytest.approx(4.0 / 6.0, rel=1e-15)
+    assert kopref.act_value(-2.0, "leaky_relu", 0.25) == -0.5 and kopref.act_value(2.0, "leaky_relu", 0.25) == 2.0
+    assert kopref.act_value(0.0, "sigmoid") == 0.5 and kopref.act_value(0.0, "mish") == 0.0
+    assert math.isnan(kopref.act_value(float("nan"), "relu")) and kopref.act_value(-1.0, "relu") == 0.0
+    # bf16 / fp16 inputs are widened exactly
+    xb = x.to(torch.bfloat16)
+    np.testing.assert_allclose(kopref.bias_act(xb, b, "mish"), F.mish(xb.double() + b.double()).numpy(), rtol=1e-13, atol=1e-14)
