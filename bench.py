@@ -103,6 +103,7 @@ def segment_bytes():
     q = c["reduce"]
     out["reduce_max"] = dict(bytes=q["rows"] * q["cols"] * 2 + q["rows"] * 8, elems=q["rows"] * q["cols"])
     out["reduce_logsumexp"] = dict(bytes=q["rows"] * q["cols"] * 2 + q["rows"] * 4, elems=q["rows"] * q["cols"])
+    out["bias_gelu"] = dict(bytes=2 * m["rows"] * m["inter"] * 2 + m["inter"] * 4, elems=m["rows"] * m["inter"])
     u = c["cumsum"]
     out["cumsum"] = dict(bytes=2 * u["rows"] * u["cols"] * 4, elems=u["rows"] * u["cols"])
     return out
@@ -248,7 +249,7 @@ class Workload:
 
     ORDER = ["softmax_small", "softmax_large", "layernorm", "bn_pool", "ce_loss", "rmsnorm", "silu_mul", "residual_add"]
     # Beyond the benchmark configs (not part of `value`): the two kernels the paper's case studies print.
-    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc", "pool2d", "reduce_max", "reduce_logsumexp"]
+    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc", "pool2d", "reduce_max", "reduce_logsumexp", "bias_gelu"]
 
     def __init__(self, kop, device, seed, only=None, rows_div=1):
         """only: build just these segments (None = all, plus the MLP segment); rows_div cuts the row
@@ -322,6 +323,11 @@ class Workload:
             self.rx, _ = synth.softmax_inputs(cut(q["rows"]), q["cols"], q["dtype"], seed, dev)
             self.rv = torch.empty(self.rx.shape[0], dtype=torch.float32, device=dev)
             self.ri = torch.empty(self.rx.shape[0], dtype=torch.int32, device=dev)
+        if "bias_gelu" in want:
+            m_ = c["mlp"]
+            self.ax = synth.gate_up_inputs(cut(m_["rows"]), m_["inter"] // 2, m_["dtype"], seed, dev)
+            self.ab = torch.randn(m_["inter"], device=dev, dtype=torch.float32) * 0.1
+            self.ay = torch.empty_like(self.ax)
         if "cumsum" in want:
             u = c["cumsum"]
             self.ux, _ = synth.cumsum_inputs(cut(u["rows"]), u["cols"], u["dtype"], seed, dev)
@@ -400,6 +406,8 @@ class Workload:
             k.kop_reduce_rows(self.rx, "max", out=self.rv, index=self.ri)
         elif name == "reduce_logsumexp":
             k.kop_reduce_rows(self.rx, "logsumexp", out=self.rv)
+        elif name == "bias_gelu":                # bias + tanh-GELU epilogue, bf16 [16384, 14336]
+            k.kop_bias_act(self.ax, self.ab, "gelu_tanh", out=self.ay)
         elif name == "cumsum":                   # inclusive running sum along rows, fp32 [32768, 4096]
             k.kop_cumsum_rows(self.ux, out=self.uy)
         else:

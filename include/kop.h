@@ -320,6 +320,20 @@ kop_status_t kop_affine_relu_pool2d(const void* x, const float* scale, const flo
                                     int ph, int pw, int mode, int relu, kop_dtype_t dtype, kop_stream_t stream);
 
 /*
+ * Bias + activation epilogue (fusion agent: "activation + bias fusion"; the pointwise tail that follows a
+ * preserved Linear / GEMM call in most of the paper's level-2 problems), one load and one store:
+ *   u = x[i,j] + bias[j]   (bias NULL: u = x[i,j]);   y[i,j] = act(u)
+ * act: 0 identity, 1 relu (NaN stays NaN), 2 leaky_relu (u > 0 ? u : alpha u), 3 gelu, tanh form,
+ *      4 gelu, erf form, 5 silu u / (1 + exp(-u)), 6 sigmoid, 7 tanh, 8 mish u tanh(ln(1 + exp(u))),
+ *      9 hardswish u min(max(u + 3, 0), 6) / 6, 10 elu (u > 0 ? u : alpha (exp(u) - 1)).
+ * alpha is used by leaky_relu and elu only. x, y: [rows, cols] of `dtype`; bias: fp32 [cols] or NULL.
+ * y may alias x exactly.
+ */
+kop_status_t kop_bias_act(const void* x, const float* bias, void* y, int64_t rows, int64_t cols,
+                          int64_t x_row_stride, int64_t y_row_stride, int act, float alpha,
+                          kop_dtype_t dtype, kop_stream_t stream);
+
+/*
  * Row reductions (the "Reduction" rows of the paper's result tables and its planner's "single-pass
  * reductions" / "LogSumExp reductions"), one read-only pass:
  *   op 0 sum, 1 mean, 2 max, 3 min, 4 logsumexp = m + ln sum_j exp(x[i,j] - m), m = max_j x[i,j]

@@ -1,0 +1,183 @@
+// kop_bias_act: y = act(x + bias[j]), the pointwise tail of a Linear / GEMM call written once ("activation +
+// bias fusion"). Pure streaming: 16-byte loads and stores, the bias vector through L1, fp32 arithmetic, one
+// compile-time activation per kernel. fp32 data uses the accurate math functions where the approximate
+// ones would eat into the 1e-5 gate (tanh, erf, expm1); 16-bit data uses the hardware approximations, whose
+// error is far below the output rounding.
+#include "kop_common.cuh"
+
+namespace kop {
+namespace {
+
+enum {
+    kActIdentity = 0, kActRelu, kActLeakyRelu, kActGeluTanh, kActGeluErf, kActSilu, kActSigmoid, kActTanh, kActMish,
+    kActHardswish, kActElu, kActCount
+};
+
+template <int ACT, bool kFast>
+__device__ __forceinline__ float act_dev(float u, float alpha)
+{
+    switch (ACT) {
+    case kActRelu: {
+        float r;
+        asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(u), "f"(0.0f));      // NaN stays NaN
+        return r;
+    }
+    case kActLeakyRelu: return u > 0.0f ? u : alpha * u;
+    case kActGeluTanh: {
+        const float k0 = 0.7978845608028654f, k1 = 0.7978845608028654f * 0.044715f;
+        const float inner = u * fmaf(k1, u * u, k0);
+        const float t = kFast ? tanh_approx(inner) : tanhf(inner);
+        const float hu = 0.5f * u;
+        return fmaf(hu, t, hu);
+    }
+    case kActGeluErf: return 0.5f * u * (1.0f + erff(u * 0.7071067811865476f));
+    case kActSilu: return u * rcp_approx(1.0f + ex2_approx(-u * kLog2e));      // ~3e-7 relative
+    case kActSigmoid: return rcp_approx(1.0f + ex2_approx(-u * kLog2e));
+    case kActTanh: return kFast ? tanh_approx(u) : tanhf(u);
+    case kActMish: {
+        // tanh(ln(1 + e^u)) = n / (n + 2) with n = e^u (e^u + 2); beyond u = 20 the quotient is 1 in fp32
+        const float e = ex2_approx(fminf(u, 20.0f) * kLog2e);
+        const float n = e * (e + 2.0f);
+        return u > 20.0f ? u : u * n * rcp_approx(n + 2.0f);
+    }
+    case kActHardswish: return u * fminf(fmaxf(u + 3.0f, 0.0f), 6.0f) * (1.0f / 6.0f);   // NaN * 0 is NaN
+    case kActElu: return u > 0.0f ? u : alpha * (kFast ? ex2_approx(u * kLog2e) - 1.0f : expm1f(u));
+    default: return u;
+    }
+}
+
+template <typename T, int ACT>
+__global__ void __launch_bounds__(256)
+bias_act_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* __restrict__ y, int nvec,
+                int tiles_per_row, int64_t x_stride, int64_t y_stride, float alpha)
+{
+    constexpr int E = Elem<T>::kPerVec, U = 4;
+    constexpr bool kFast = sizeof(T) == 2;
+    const int64_t row = blockIdx.x / tiles_per_row;
+    const int tile = (int)(blockIdx.x - row * tiles_per_row);
+    const T* xr = x + row * x_stride;
+    T* yr = y + row * y_stride;
+    const int v0 = tile * (U * blockDim.x) + threadIdx.x;
+    Vec16 raw[U];
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+        const int v = v0 + k * blockDim.x;
+        if (v < nvec) raw[k] = ld_stream(xr + (int64_t)v * E);
+    }
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+        const int v = v0 + k * blockDim.x;
+        if (v < nvec) {
+            float f[E];
+            Elem<T>::unpack(raw[k], f);
+            if (bias != nullptr) {
+#pragma unroll
+                for (int q = 0; q < E / 4; ++q) {
+                    const float4 b = ldg_f4(bias + (int64_t)v * E + 4 * q);
+                    f[4 * q] += b.x;
+                    f[4 * q + 1] += b.y;
+                    f[4 * q + 2] += b.z;
+                    f[4 * q + 3] += b.w;
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < E; ++e) f[e] = act_dev<ACT, kFast>(f[e], alpha);
+            st_stream(yr + (int64_t)v * E, Elem<T>::pack(f));
+        }
+    }
+}
+
+template <typename T, int ACT>
+__global__ void __launch_bounds__(256)
+bias_act_scalar_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* __restrict__ y, int64_t rows,
+                       int64_t cols, int64_t x_stride, int64_t y_stride, float alpha)
+{
+    constexpr bool kFast = sizeof(T) == 2;
+    const int64_t total = rows * cols;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / cols, j = i - r * cols;
+        const float u = Elem<T>::load1(x + r * x_stride + j) + (bias != nullptr ? __ldg(bias + j) : 0.0f);
+        Elem<T>::store1(y + r * y_stride + j, act_dev<ACT, kFast>(u, alpha));
+    }
+}
+
+template <typename T, int ACT>
+kop_status_t launch_bias_act_a(const T* x, const float* bias, T* y, int64_t rows, int64_t cols, int64_t xs,
+                               int64_t ys, float alpha, cudaStream_t stream)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    // without a bias a contiguous tensor is one long row (no per-row tail, no row index)
+    if (bias == nullptr && xs == cols && ys == cols && rows * cols / E <= 0x3FFFFFFFLL) {
+        cols = rows * cols;
+        xs = ys = cols;
+        rows = 1;
+    }
+    const bool vec = vec_ok(x, cols, xs, sizeof(T)) && vec_ok(y, cols, ys, sizeof(T)) && cols / E <= 0x3FFFFFFF &&
+                     (bias == nullptr || aligned_to(bias, 16));
+    if (vec) {
+        const int nvec = (int)(cols / E);
+        int threads = ((nvec + 3) / 4 + 31) / 32 * 32;
+        if (threads > 256) threads = 256;
+        const int tiles = (nvec + 4 * threads - 1) / (4 * threads);
+        const int64_t grid = rows * tiles;
+        if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+        bias_act_kernel<T, ACT><<<(unsigned)grid, threads, 0, stream>>>(x, bias, y, nvec, tiles, xs, ys, alpha);
+        return launch_status();
+    }
+    int64_t blocks = (rows * cols + 255) / 256;
+    const int64_t cap = 32LL * sm_count();
+    if (blocks > cap) blocks = cap;
+    bias_act_scalar_kernel<T, ACT><<<(unsigned)blocks, 256, 0, stream>>>(x, bias, y, rows, cols, xs, ys, alpha);
+    return launch_status();
+}
+
+template <typename T>
+kop_status_t launch_bias_act(const void* xv, const float* bias, void* yv, int64_t rows, int64_t cols, int64_t xs,
+                             int64_t ys, int act, float alpha, cudaStream_t stream)
+{
+    const T* x = static_cast<const T*>(xv);
+    T* y = static_cast<T*>(yv);
+#define KOP_ACT_CASE(A) \
+    case A: return launch_bias_act_a<T, A>(x, bias, y, rows, cols, xs, ys, alpha, stream)
+    switch (act) {
+        KOP_ACT_CASE(kActRelu);
+        KOP_ACT_CASE(kActLeakyRelu);
+        KOP_ACT_CASE(kActGeluTanh);
+        KOP_ACT_CASE(kActGeluErf);
+        KOP_ACT_CASE(kActSilu);
+        KOP_ACT_CASE(kActSigmoid);
+        KOP_ACT_CASE(kActTanh);
+        KOP_ACT_CASE(kActMish);
+        KOP_ACT_CASE(kActHardswish);
+        KOP_ACT_CASE(kActElu);
+    default: return launch_bias_act_a<T, kActIdentity>(x, bias, y, rows, cols, xs, ys, alpha, stream);
+    }
+#undef KOP_ACT_CASE
+}
+
+}  // namespace
+}  // namespace kop
+
+extern "C" kop_status_t kop_bias_act(const void* x, const float* bias, void* y, int64_t rows, int64_t cols,
+                                     int64_t x_row_stride, int64_t y_row_stride, int act, float alpha,
+                                     kop_dtype_t dtype, kop_stream_t stream)
+{
+    using namespace kop;
+    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    kop_status_t st = check_rows_cols(rows, cols);
+    if (st != KOP_OK) return st;
+    if (act < 0 || act >= kActCount) return KOP_ERR_BAD_SHAPE;
+    if ((st = check_row_stride(x_row_stride, cols, rows)) != KOP_OK) return st;
+    if ((st = check_row_stride(y_row_stride, cols, rows)) != KOP_OK) return st;
+    if (rows == 0) return KOP_OK;
+    if (!x || !y) return KOP_ERR_NULL_POINTER;
+    const int esz = elem_size(dtype);
+    if (!aligned_to(x, esz) || !aligned_to(y, esz) || (bias && !aligned_to(bias, 4))) return KOP_ERR_MISALIGNED;
+    if (!alias_ok(x, x_row_stride, y, y_row_stride, rows, cols, esz, true)) return KOP_ERR_BAD_ALIAS;
+    if ((st = check_device()) != KOP_OK) return st;
+    cudaStream_t s = as_stream(stream);
+    return dtype == KOP_F32 ? launch_bias_act<float>(x, bias, y, rows, cols, x_row_stride, y_row_stride, act, alpha, s)
+           : dtype == KOP_BF16
+               ? launch_bias_act<__nv_bfloat16>(x, bias, y, rows, cols, x_row_stride, y_row_stride, act, alpha, s)
+               : launch_bias_act<__half>(x, bias, y, rows, cols, x_row_stride, y_row_stride, act, alpha, s);
+}

@@ -82,6 +82,8 @@ def lib() -> C.CDLL:
     L.kop_affine_relu_pool2d.restype = i32
     L.kop_reduce_rows.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, vp]
     L.kop_reduce_rows.restype = i32
+    L.kop_bias_act.argtypes = [vp, vp, vp, i64, i64, i64, i64, i32, f32, i32, vp]
+    L.kop_bias_act.restype = i32
     L.kop_cumsum_rows.argtypes = [vp, vp, vp] + [i64] * 5 + [i32, i32, i32, vp]
     L.kop_cumsum_rows.restype = i32
     L.kop_groupnorm_wait_timeouts.argtypes = [C.POINTER(C.c_uint)]
@@ -372,6 +374,20 @@ def kop_affine_relu_pool2d(x, scale, shift, kernel, stride, padding, mode="max",
                                         out.data_ptr(), N, Cc, H, W, kh, kw, sh, sw, ph, pw,
                                         {"max": 0, "avg": 1}[mode], int(bool(relu)), _dtype_tag(x), _stream(stream)),
            "kop_affine_relu_pool2d")
+    return out
+
+
+ACTS = {"identity": 0, "relu": 1, "leaky_relu": 2, "gelu_tanh": 3, "gelu_erf": 4, "silu": 5, "sigmoid": 6,
+        "tanh": 7, "mish": 8, "hardswish": 9, "elu": 10}
+
+
+def kop_bias_act(x, bias, act, alpha=0.01, out=None, stream=None):
+    rows, cols, xs = _rows2d(x, "x")
+    out = torch.empty_like(x) if out is None else out
+    _, _, ys = _rows2d(out, "out")
+    assert out.shape == x.shape and out.dtype == x.dtype
+    _check(lib().kop_bias_act(x.data_ptr(), _param(bias, "bias", cols), out.data_ptr(), rows, cols, xs, ys, ACTS[act],
+                              float(alpha), _dtype_tag(x), _stream(stream)), "kop_bias_act")
     return out
 
 

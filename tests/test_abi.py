@@ -241,6 +241,18 @@ def test_reduce_validation(L):
     assert f(P, Q, Q + 8, 4, 64, 64, 2, 0, None) == ALIAS           # index overlaps out
 
 
+def test_bias_act_validation(L):
+    f = L.kop_bias_act
+    assert f(P, Q, R, 0, 64, 64, 64, 1, 0.0, 0, None) == OK
+    assert f(None, Q, R, 4, 64, 64, 64, 1, 0.0, 0, None) == NULLP
+    assert f(P, None, R, 4, 64, 64, 64, 1, 0.0, 0, None) != NULLP          # the bias is optional
+    assert f(P, Q, R, 4, 64, 64, 64, 11, 0.0, 0, None) == SHAPE             # unknown activation
+    assert f(P, Q, R, 4, 64, 63, 64, 1, 0.0, 0, None) == STRIDE
+    assert f(P, Q, R, 4, 64, 64, 64, 1, 0.0, 6, None) == DTYPE
+    assert f(P, Q + 2, R, 4, 64, 64, 64, 1, 0.0, 0, None) == MISAL
+    assert f(P, Q, P + 8, 4, 64, 64, 64, 1, 0.0, 0, None) == ALIAS
+
+
 def test_mlp_driver_validation(L):
     f = L.kop_rmsnorm_swiglu_residual
     wsb = L.kop_rmsnorm_swiglu_residual_workspace_bytes(16, 64, 128, 1)

@@ -1,0 +1,79 @@
+"""GPU parity of kop_bias_act against the float64 CPU oracle: the eleven activations, three data types, five
+seeds, with and without bias, vector and scalar paths, strided and in-place use, NaN / infinity behaviour,
+guard bands. Tolerance |got - ref| <= tol * max(1, |ref|), tol = 1e-5 (fp32), 2e-2 (bf16), 2e-3 (fp16)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import kopref
+from paper_2609_30059_b200 import build as kbuild
+from paper_2609_30059_b200 import synth
+from tests._util import Guarded, assert_bf16_tight, assert_close, tol_of
+
+pytestmark = pytest.mark.gpu
+SEEDS = synth.SEEDS
+F32, BF16, F16 = torch.float32, torch.bfloat16, torch.float16
+ACTS = ("identity", "relu", "leaky_relu", "gelu_tanh", "gelu_erf", "silu", "sigmoid", "tanh", "mish", "hardswish", "elu")
+
+
+@pytest.fixture(scope="module")
+def kop():
+    kbuild.build()
+    from paper_2609_30059_b200 import kop as K
+    return K
+
+
+def host(t):
+    return None if t is None else t.detach().cpu()
+
+
+@pytest.mark.parametrize("rows,cols,dtype", [(512, 4096, BF16), (300, 4096, F32), (65, 1000, F16), (33, 1001, F32),
+                                             (9, 20480, BF16), (7, 1, F32)])
+@pytest.mark.parametrize("seed", SEEDS)
+def test_bias_act_parity(kop, rows, cols, dtype, seed):
+    x, bias = synth.softmax_inputs(rows, cols, dtype, seed, "cuda")
+    x = x * 3.0                                            # reach the saturated ends of the activations
+    bias = bias * 5.0
+    tol = tol_of(dtype)
+    for k, act in enumerate(ACTS):
+        use_bias = (k + seed) % 3 != 0
+        y = Guarded((rows, cols), dtype)
+        kop.kop_bias_act(x, bias if use_bias else None, act, alpha=0.2, out=y.t)
+        ref = kopref.bias_act(host(x), host(bias) if use_bias else None, act, alpha=0.2, threads=None)
+        assert_close(y.t, ref, tol, f"bias_act {act} bias={use_bias}")
+        if dtype == BF16:
+            assert_bf16_tight(y.t, ref, f"bias_act {act}")
+        y.check(act)
+
+
+def test_bias_act_options(kop):
+    rows, cols = 40, 2048
+    x, bias = synth.softmax_inputs(rows, cols, F32, 9, "cuda")
+    x = x * 4.0
+    for act in ("gelu_erf", "mish", "elu"):
+        ref = kopref.bias_act(host(x), host(bias), act, alpha=1.0)
+        xi = x.clone()
+        kop.kop_bias_act(xi, bias, act, alpha=1.0, out=xi)                       # in place
+        assert_close(xi, ref, 1e-5, act + " in place")
+        big = torch.zeros((rows, cols + 40), dtype=F32, device="cuda")            # strided rows
+        big[:, :cols] = x
+        outb = torch.full((rows, cols + 8), 5.0, dtype=F32, device="cuda")
+        kop.kop_bias_act(big[:, :cols], bias, act, alpha=1.0, out=outb[:, :cols])
+        assert_close(outb[:, :cols], ref, 1e-5, act + " strided")
+        assert bool((outb[:, cols:] == 5.0).all())
+        flat = torch.zeros(rows * cols + 1, dtype=F32, device="cuda")             # misaligned base: scalar kernel
+        flat[1:] = x.reshape(-1)
+        assert_close(kop.kop_bias_act(flat[1:].view(rows, cols), bias, act, alpha=1.0), ref, 1e-5, act + " misaligned")
+    # special values
+    sp = torch.tensor([[float("nan"), float("inf"), float("-inf"), 0.0, -0.0, 100.0, -100.0, 1e-30]], device="cuda")
+    for act in ACTS:
+        got = kop.kop_bias_act(sp, None, act, alpha=0.5).cpu().double().numpy()
+        ref = kopref.bias_act(host(sp), None, act, alpha=0.5)
+        assert bool(np.isnan(got[0, 0])), act + ": NaN must stay NaN"
+        finite = np.isfinite(ref[0])
+        assert np.allclose(got[0][finite], ref[0][finite], rtol=1e-5, atol=1e-5), act + " special values"
+        both_inf = np.isinf(ref[0])
+        assert np.array_equal(got[0][both_inf], ref[0][both_inf]), act + " infinities"
+    e = torch.empty((0, 8), dtype=F32, device="cuda")
+    assert kop.kop_bias_act(e, None, "relu").shape == (0, 8)
+    assert kop.lib().kop_bias_act(x.data_ptr(), None, x.data_ptr(), 4, 16, 16, 16, 11, 0.0, 0, None) == 2

@@ -128,6 +128,12 @@ def test_fuzz_row_kernels(kop):
         v, _ = kop.kop_reduce_rows(xr, "logsumexp")
         rv, _ = kopref.reduce_rows(host(x), "logsumexp")
         assert np.all(np.abs(to_f64(v) - rv) <= 1e-5 * np.maximum(1.0, np.abs(rv))), "reduce logsumexp " + what
+        # bias + activation epilogue, a random activation
+        act = ("identity", "relu", "leaky_relu", "gelu_tanh", "gelu_erf", "silu", "sigmoid", "tanh", "mish", "hardswish",
+               "elu")[int(rng.integers(0, 11))]
+        xa, ba = synth.softmax_inputs(rows, cols, dtype, seed, "cuda")
+        assert_close(kop.kop_bias_act(strided(rng, xa), ba, act, alpha=0.3), kopref.bias_act(host(xa), host(ba), act, alpha=0.3),
+                     tol, f"bias_act {act} " + what)
         # running sums
         xc, mask = synth.cumsum_inputs(rows, cols, dtype, seed, "cuda")
         ex, rv, um = bool(rng.integers(0, 2)), bool(rng.integers(0, 2)), bool(rng.integers(0, 2))
