@@ -725,3 +725,35 @@ int kopref_bias_act(const void* x, const float* bias, double* y, int64_t rows, i
         }
     return 0;
 }
+
+/* ---- softmax variants ("fused softmax", "online softmax", LogSoftmax) -------------------------------------
+ * z[i,j] = x[i,j] * scale + bias[j] (bias may be NULL). With period > 0 the rows are causal: row i keeps the
+ * columns j <= (i mod period) + (cols - period) (period == cols is the square causal mask of attention scores,
+ * a smaller period leaves a prefix of cols - period columns visible to every row) and the others count as
+ * z = -inf. log_out == 0: y = exp(z - m) / sum_j exp(z_j - m), m = max_j z_j (masked columns give 0);
+ * log_out != 0: y = z - m - ln sum_j exp(z_j - m) (masked columns give -inf). */
+int kopref_softmax_opts(const void* x, const float* bias, double* y, int64_t rows, int64_t cols,
+        int64_t x_row_stride, int64_t y_row_stride, double scale, int log_out, int64_t period, int dtype,
+        int threads)
+{
+    if (!x || !y || rows < 0 || cols <= 0 || period < 0 || period > cols || bad_dtype(dtype)) return -1;
+    int nt = pick_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t i = 0; i < rows; ++i) {
+        double* yr = y + i * y_row_stride;
+        int64_t last = period > 0 ? (i % period) + (cols - period) : cols - 1;   /* last visible column */
+        double m = -INFINITY;
+        for (int64_t j = 0; j < cols; ++j) {
+            double z = j <= last ? load_elem(x, i * x_row_stride + j, dtype) * scale + (bias ? (double)bias[j] : 0.0)
+                                 : -INFINITY;
+            yr[j] = z;
+            if (z > m) m = z;
+        }
+        double S = 0.0;
+        for (int64_t j = 0; j < cols; ++j) S += exp(yr[j] - m);
+        double lnS = log(S);
+        for (int64_t j = 0; j < cols; ++j) yr[j] = log_out ? (yr[j] - m) - lnS : exp(yr[j] - m) / S;
+    }
+    return 0;
+}

@@ -55,6 +55,7 @@ def lib() -> C.CDLL:
         _lib.kopref_bias_act.argtypes = [vp, vp, vp, i64, i64, i64, i64, C.c_int, dbl, C.c_int, C.c_int]
         _lib.kopref_act_value.restype = dbl
         _lib.kopref_act_value.argtypes = [dbl, C.c_int, dbl]
+        _lib.kopref_softmax_opts.argtypes = [vp, vp, vp, i64, i64, i64, i64, dbl, C.c_int, i64, C.c_int, C.c_int]
         _lib.kopref_cumsum_rows.argtypes = [vp, vp, vp] + [i64] * 5 + [C.c_int] * 4
         _lib.kopref_matvec_bias.argtypes = [vp, vp, dbl, vp, i64, i64, i64, C.c_int, C.c_int]
     return _lib
@@ -149,6 +150,17 @@ def softmax_scale_bias(x, bias, scale, threads=1) -> np.ndarray:
 
 def gelu_erf(u: float) -> float:
     return lib().kopref_gelu_erf(float(u))
+
+
+def softmax_opts(x, bias, scale, log_output=False, causal_period=0, threads=1) -> np.ndarray:
+    """Softmax or log-softmax of x * scale + bias per row, optionally causal (see kopref_softmax_opts)."""
+    xa, dt = as_data(x)
+    rows, cols = xa.shape
+    b = as_param(bias)
+    y = np.empty((rows, cols), dtype=np.float64)
+    _check(lib().kopref_softmax_opts(_p(xa), _p(b), _p(y), rows, cols, cols, cols, float(scale), int(bool(log_output)),
+                                     int(causal_period), dt, _nt(threads)), "softmax_opts")
+    return y
 
 
 def bias_gelu_residual_layernorm(x, residual, bias, gamma, beta, eps, threads=1, erf_form=False):

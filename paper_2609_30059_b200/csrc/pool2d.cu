@@ -46,6 +46,29 @@ __device__ __forceinline__ float act_of(float v, float sc, float sf, float relu_
 __host__ __device__ __forceinline__ int pool_lead(int pw) { return (pw + 3) / 4 * 4; }
 __host__ __device__ __forceinline__ int pool_row_floats(int W, int pw) { return (pool_lead(pw) + W + pw + 3) / 4 * 4; }
 
+// One window out of the tile: the max (NaN-propagating) or the average of kh x kw cells starting at `win`.
+template <int MODE, int KS>
+__device__ __forceinline__ float window_value(const float* win, int Ws, int kh, int kw, float inv_area)
+{
+    float res = MODE == 0 ? -INFINITY : 0.0f;
+    if (KS) {
+#pragma unroll
+        for (int di = 0; di < (KS ? KS : 1); ++di)
+#pragma unroll
+            for (int dj = 0; dj < (KS ? KS : 1); ++dj) {
+                const float a = win[di * Ws + dj];
+                res = MODE == 0 ? max_keep_nan(res, a) : res + a;
+            }
+    } else {
+        for (int di = 0; di < kh; ++di)
+            for (int dj = 0; dj < kw; ++dj) {
+                const float a = win[di * Ws + dj];
+                res = MODE == 0 ? max_keep_nan(res, a) : res + a;
+            }
+    }
+    return MODE == 1 ? res * inv_area : res;
+}
+
 // MODE 0 max, 1 average. KS / ST: compile-time square window and stride (0 = use the runtime values).
 // Consecutive threads take consecutive outputs: their windows start sw floats apart in shared memory (a
 // 2-way bank conflict at stride 2 instead of the 8-way one of a vector of outputs per thread), and a warp's
@@ -140,47 +163,14 @@ pool2d_tile_kernel(const T* __restrict__ x, const float* __restrict__ scale, con
             T* dst = yp + warp * OW + ocol;
 #pragma unroll 2
             for (int orow = warp; orow < orows; orow += NW, win += NW * sh * Ws, dst += NW * OW) {
-                float res = MODE == 0 ? -INFINITY : 0.0f;
-                if (KS) {
-#pragma unroll
-                    for (int di = 0; di < (KS ? KS : 1); ++di)
-#pragma unroll
-                        for (int dj = 0; dj < (KS ? KS : 1); ++dj) {
-                            const float a = win[di * Ws + dj];
-                            res = MODE == 0 ? max_keep_nan(res, a) : res + a;
-                        }
-                } else {
-                    for (int di = 0; di < kh; ++di)
-                        for (int dj = 0; dj < kw; ++dj) {
-                            const float a = win[di * Ws + dj];
-                            res = MODE == 0 ? max_keep_nan(res, a) : res + a;
-                        }
-                }
-                Elem<T>::store1(dst, MODE == 1 ? res * inv_area : res);
+                Elem<T>::store1(dst, window_value<MODE, KS>(win, Ws, kh, kw, inv_area));
             }
         }
-        return;
-    }
-    for (int o = threadIdx.x; o < n_out; o += kPoolThreads) {
-        const int orow = div_small(o, OW, inv_ow), ocol = o - orow * OW;
-        const float* win = origin + orow * sh * Ws + ocol * sw;
-        float res = MODE == 0 ? -INFINITY : 0.0f;
-        if (KS) {
-#pragma unroll
-            for (int di = 0; di < (KS ? KS : 1); ++di)
-#pragma unroll
-                for (int dj = 0; dj < (KS ? KS : 1); ++dj) {
-                    const float a = win[di * Ws + dj];
-                    res = MODE == 0 ? max_keep_nan(res, a) : res + a;
-                }
-        } else {
-            for (int di = 0; di < kh; ++di)
-                for (int dj = 0; dj < kw; ++dj) {
-                    const float a = win[di * Ws + dj];
-                    res = MODE == 0 ? max_keep_nan(res, a) : res + a;
-                }
+    } else {
+        for (int o = threadIdx.x; o < n_out; o += kPoolThreads) {
+            const int orow = div_small(o, OW, inv_ow), ocol = o - orow * OW;
+            Elem<T>::store1(yp + o, window_value<MODE, KS>(origin + orow * sh * Ws + ocol * sw, Ws, kh, kw, inv_area));
         }
-        Elem<T>::store1(yp + o, MODE == 1 ? res * inv_area : res);
     }
 }
 

@@ -898,3 +898,41 @@ def test_bias_act_against_torch_mpmath_and_identities():
     # bf16 / fp16 inputs are widened exactly
     xb = x.to(torch.bfloat16)
     np.testing.assert_allclose(kopref.bias_act(xb, b, "mish"), F.mish(xb.double() + b.double()).numpy(), rtol=1e-13, atol=1e-14)
+
+
+# --------------------------------------------------------------------------- softmax variants
+
+def test_softmax_opts_log_and_causal():
+    x = torch.from_numpy(f32(RNG.normal(0, 2, (12, 37))))
+    b = torch.from_numpy(f32(RNG.normal(0, 0.5, 37)))
+    z = x.double() * 0.7 + b.double()
+    # without options it is the plain oracle; the log form is its logarithm and torch's log_softmax
+    assert np.array_equal(kopref.softmax_opts(x, b, 0.7), kopref.softmax_scale_bias(x, b, 0.7))
+    np.testing.assert_allclose(kopref.softmax_opts(x, b, 0.7, log_output=True), F.log_softmax(z, dim=1).numpy(), rtol=0, atol=1e-13)
+    np.testing.assert_allclose(np.exp(kopref.softmax_opts(x, b, 0.7, log_output=True)), kopref.softmax_scale_bias(x, b, 0.7),
+                               rtol=1e-13)
+    # log-softmax of a constant row of n entries is -ln n; it survives huge logits
+    const = torch.full((2, 50), 3.0)
+    np.testing.assert_allclose(kopref.softmax_opts(const, None, 1.0, log_output=True), np.full((2, 50), -math.log(50)), rtol=1e-15)
+    big = torch.tensor([[1000.0, 999.0]])
+    np.testing.assert_allclose(kopref.softmax_opts(big, None, 1.0, log_output=True)[0],
+                               [-math.log1p(math.exp(-1.0)), -1.0 - math.log1p(math.exp(-1.0))], rtol=1e-14)
+    # causal, square (period == cols): equals torch softmax over the masked scores, row by row within each block
+    S = 9
+    sc = torch.from_numpy(f32(RNG.normal(0, 1, (3 * S, S))))
+    mask = torch.tril(torch.ones(S, S, dtype=torch.bool)).repeat(3, 1)
+    zm = (sc.double() * 0.5).masked_fill(~mask, float("-inf"))
+    np.testing.assert_allclose(kopref.softmax_opts(sc, None, 0.5, causal_period=S), torch.softmax(zm, dim=1).numpy(), rtol=0, atol=1e-15)
+    got = kopref.softmax_opts(sc, None, 0.5, log_output=True, causal_period=S)
+    ref = F.log_softmax(zm, dim=1).numpy()
+    assert np.array_equal(np.isneginf(got), np.isneginf(ref)) and np.array_equal(np.isneginf(got), ~mask.numpy())
+    np.testing.assert_allclose(got[mask.numpy()], ref[mask.numpy()], rtol=0, atol=1e-13)
+    # first row of every block sees one column: probability 1 there; the last row sees all: the plain softmax
+    p = kopref.softmax_opts(sc, None, 0.5, causal_period=S)
+    assert np.array_equal(p[0::S, 0], np.ones(3)) and np.array_equal(p[0, 1:], np.zeros(S - 1))
+    np.testing.assert_allclose(p[S - 1::S], kopref.softmax_scale_bias(sc[S - 1::S], None, 0.5), rtol=0, atol=0)
+    # a period shorter than the row leaves a prefix visible to every row (4 queries over 9 keys: 5 + r + 1 visible)
+    q = kopref.softmax_opts(sc[:8], None, 1.0, causal_period=4)
+    for r in range(8):
+        vis = 5 + (r % 4) + 1
+        assert np.all(q[r, vis:] == 0) and q[r, :vis].sum() == pytest.approx(1.0, rel=1e-14) and np.all(q[r, :vis] > 0)
