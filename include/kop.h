@@ -88,6 +88,22 @@ kop_status_t kop_softmax_scale_bias(const void* x, const float* bias, void* y,
                                     float scale, kop_dtype_t dtype, kop_stream_t stream);
 
 /*
+ * Softmax variants (planner strategy 9 "fused softmax" / "online softmax"; the LogSoftmax row of the results
+ * table): the same z = x * scale + bias, then
+ *   log_output == 0:  y = exp(z - m) / sum_j exp(z_j - m)            (as kop_softmax_scale_bias)
+ *   log_output != 0:  y = z - m - ln sum_j exp(z_j - m)               (log-softmax)
+ * with m = max_j z_j, and, when causal_period > 0, causal rows: row i keeps the columns
+ * j <= (i mod causal_period) + (cols - causal_period) and every other column counts as z = -inf (output 0, or
+ * -inf in the log form). causal_period == cols is the square mask of attention scores stored as
+ * [batch * heads * cols, cols]; a smaller period leaves a prefix of cols - causal_period columns visible to every
+ * row (queries behind a cache). 0 <= causal_period <= cols, else KOP_ERR_BAD_SHAPE. Everything else as in
+ * kop_softmax_scale_bias.
+ */
+kop_status_t kop_softmax_opts(const void* x, const float* bias, void* y, int64_t rows, int64_t cols,
+                              int64_t x_row_stride, int64_t y_row_stride, float scale, int log_output,
+                              int64_t causal_period, kop_dtype_t dtype, kop_stream_t stream);
+
+/*
  * Bias-add, tanh-form GELU, residual add and LayerNorm in one pass (fusion agent:
  * "activation + bias fusion" and "residual + norm: one kernel, one memory pass";
  * codegen agent: "single-pass LayerNorm instead of 3 kernels"):

@@ -76,14 +76,27 @@ softmax_warp_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* 
 }
 
 // ---- CTA per row, row in registers ---------------------------------------------------------------
-template <typename T, int VPT>
+// kOpts adds the variants of kop_softmax_opts: `last` is the row's last visible column (causal rows; every
+// later column counts as -inf) and log_out selects z - m - ln(sum) instead of exp(z - m) / sum.
+struct SmOpts {
+    int log_out;
+    int64_t period;      // 0: not causal
+    int64_t cols;
+};
+__device__ __forceinline__ int64_t last_visible(const SmOpts& o, int64_t row)
+{
+    return o.period > 0 ? (row % o.period) + (o.cols - o.period) : o.cols - 1;
+}
+
+template <typename T, int VPT, bool kOpts>
 __global__ void __launch_bounds__(max_threads_for(VPT * Elem<T>::kPerVec))
 softmax_block_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* __restrict__ y,
-                     int nvec, int64_t x_stride, int64_t y_stride, float scale)
+                     int nvec, int64_t x_stride, int64_t y_stride, float scale, SmOpts opts)
 {
     constexpr int E = Elem<T>::kPerVec;
     __shared__ float red_a[32], red_b[32];
     const int64_t row = blockIdx.x;
+    const int64_t last = kOpts ? last_visible(opts, row) : 0;
     const T* xr = x + row * x_stride;
     T* yr = y + row * y_stride;
     const float s2 = scale * kLog2e;
@@ -109,66 +122,76 @@ softmax_block_kernel(const T* __restrict__ x, const float* __restrict__ bias, T*
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 const int e = 4 * q + c;
-                t[k][e] = v < nvec ? fmaf(f[e], s2, bb[c] * kLog2e) : -INFINITY;
+                const bool keep = v < nvec && (!kOpts || (int64_t)v * E + e <= last);
+                t[k][e] = keep ? fmaf(f[e], s2, bb[c] * kLog2e) : -INFINITY;
                 m = fmaxf(m, t[k][e]);
             }
         }
     }
     m = block_max(m, red_a);
     float s = 0.0f;
+    const bool log_out = kOpts && opts.log_out != 0;
 #pragma unroll
     for (int k = 0; k < VPT; ++k)
 #pragma unroll
         for (int e = 0; e < E; ++e) {
-            t[k][e] = ex2_approx(t[k][e] - m);
-            s += t[k][e];
+            const float d = t[k][e] - m;
+            const float p = ex2_approx(d);
+            s += p;
+            t[k][e] = log_out ? d : p;                       // the log form keeps the base-2 exponent
         }
     s = block_sum(s, red_b);
     const float inv = 1.0f / s;
+    const float lg = lg2_approx(s);
 #pragma unroll
     for (int k = 0; k < VPT; ++k) {
         const int v = k * blockDim.x + threadIdx.x;
         float o[E];
 #pragma unroll
-        for (int e = 0; e < E; ++e) o[e] = t[k][e] * inv;
+        for (int e = 0; e < E; ++e) o[e] = log_out ? (t[k][e] - lg) * kLn2 : t[k][e] * inv;
         if (v < nvec) st_stream(yr + (int64_t)v * E, Elem<T>::pack(o));
     }
 }
 
 // ---- any length, any alignment: scalar loads, three sweeps over the row ----------------------------
-template <typename T>
+template <typename T, bool kOpts>
 __global__ void __launch_bounds__(256)
 softmax_generic_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* __restrict__ y,
-                       int64_t cols, int64_t x_stride, int64_t y_stride, float scale)
+                       int64_t cols, int64_t x_stride, int64_t y_stride, float scale, SmOpts opts)
 {
     __shared__ float red_a[32], red_b[32];
     const int64_t row = blockIdx.x;
+    const int64_t last = kOpts ? last_visible(opts, row) : cols - 1;
+    const bool log_out = kOpts && opts.log_out != 0;
     const T* xr = x + row * x_stride;
     T* yr = y + row * y_stride;
     const float s2 = scale * kLog2e;
     float m = -INFINITY;
     for (int64_t j = threadIdx.x; j < cols; j += blockDim.x) {
         const float b = bias != nullptr ? __ldg(bias + j) * kLog2e : 0.0f;
-        m = fmaxf(m, fmaf(Elem<T>::load1(xr + j), s2, b));
+        if (j <= last) m = fmaxf(m, fmaf(Elem<T>::load1(xr + j), s2, b));
     }
     m = block_max(m, red_a);
     float s = 0.0f;
     for (int64_t j = threadIdx.x; j < cols; j += blockDim.x) {
         const float b = bias != nullptr ? __ldg(bias + j) * kLog2e : 0.0f;
-        s += ex2_approx(fmaf(Elem<T>::load1(xr + j), s2, b) - m);
+        if (j <= last) s += ex2_approx(fmaf(Elem<T>::load1(xr + j), s2, b) - m);
     }
     s = block_sum(s, red_b);
     const float inv = 1.0f / s;
+    const float lg = lg2_approx(s);
     // The last sweep reads x[j] and writes y[j] in the same thread, so exact aliasing stays safe.
     for (int64_t j = threadIdx.x; j < cols; j += blockDim.x) {
         const float b = bias != nullptr ? __ldg(bias + j) * kLog2e : 0.0f;
-        Elem<T>::store1(yr + j, ex2_approx(fmaf(Elem<T>::load1(xr + j), s2, b) - m) * inv);
+        const float d = j <= last ? fmaf(Elem<T>::load1(xr + j), s2, b) - m : -INFINITY;
+        Elem<T>::store1(yr + j, log_out ? (d - lg) * kLn2 : ex2_approx(d) * inv);
     }
 }
 
 template <typename T>
 kop_status_t launch_softmax(const void* xv, const float* bias, void* yv, int64_t rows, int64_t cols,
-                            int64_t xs, int64_t ys, float scale, cudaStream_t stream)
+                            int64_t xs, int64_t ys, float scale, cudaStream_t stream, bool with_opts = false,
+                            SmOpts opts = SmOpts{0, 0, 0})
 {
     const T* x = static_cast<const T*>(xv);
     T* y = static_cast<T*>(yv);
@@ -176,7 +199,7 @@ kop_status_t launch_softmax(const void* xv, const float* bias, void* yv, int64_t
     const bool vec = vec_ok(x, cols, xs, sizeof(T)) && vec_ok(y, cols, ys, sizeof(T)) &&
                      (bias == nullptr || aligned_to(bias, 16));
     const int64_t nvec64 = cols / E;
-    if (vec && nvec64 <= 32 * 4) {
+    if (vec && nvec64 <= 32 * 4 && !with_opts) {
         const int nvec = (int)nvec64;
         const int vpl = (nvec + 31) / 32;
         const int threads = 256;
@@ -208,7 +231,11 @@ kop_status_t launch_softmax(const void* xv, const float* bias, void* yv, int64_t
         int vpt = 16 / E;
         while (vpt * E < 64 && (nvec + vpt - 1) / vpt > max_threads_for(vpt * E)) vpt *= 2;
         const int threads = ((nvec + vpt - 1) / vpt + 31) / 32 * 32;
-#define KOP_SM_BLOCK(V) softmax_block_kernel<T, V><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, nvec, xs, ys, scale)
+#define KOP_SM_BLOCK(V)                                                                                              \
+    do {                                                                                                             \
+        if (with_opts) softmax_block_kernel<T, V, true><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, nvec, xs, ys, scale, opts); \
+        else softmax_block_kernel<T, V, false><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, nvec, xs, ys, scale, opts);          \
+    } while (0)
         switch (vpt * E) {
         case 16: KOP_SM_BLOCK(16 / E); break;
         case 32: KOP_SM_BLOCK(32 / E); break;
@@ -217,7 +244,8 @@ kop_status_t launch_softmax(const void* xv, const float* bias, void* yv, int64_t
 #undef KOP_SM_BLOCK
         return launch_status();
     }
-    softmax_generic_kernel<T><<<(unsigned)rows, 256, 0, stream>>>(x, bias, y, cols, xs, ys, scale);
+    if (with_opts) softmax_generic_kernel<T, true><<<(unsigned)rows, 256, 0, stream>>>(x, bias, y, cols, xs, ys, scale, opts);
+    else softmax_generic_kernel<T, false><<<(unsigned)rows, 256, 0, stream>>>(x, bias, y, cols, xs, ys, scale, opts);
     return launch_status();
 }
 
@@ -247,4 +275,30 @@ extern "C" kop_status_t kop_softmax_scale_bias(const void* x, const float* bias,
                ? launch_softmax<float>(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale, s)
                : dtype == KOP_BF16 ? launch_softmax<__nv_bfloat16>(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale, s)
                : launch_softmax<__half>(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale, s);
+}
+
+extern "C" kop_status_t kop_softmax_opts(const void* x, const float* bias, void* y, int64_t rows, int64_t cols,
+                                         int64_t x_row_stride, int64_t y_row_stride, float scale, int log_output,
+                                         int64_t causal_period, kop_dtype_t dtype, kop_stream_t stream)
+{
+    using namespace kop;
+    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    kop_status_t st = check_rows_cols(rows, cols);
+    if (st != KOP_OK) return st;
+    if (causal_period < 0 || causal_period > cols) return KOP_ERR_BAD_SHAPE;
+    if (rows == 0) return KOP_OK;
+    if (x == nullptr || y == nullptr) return KOP_ERR_NULL_POINTER;
+    if ((st = check_row_stride(x_row_stride, cols, rows)) != KOP_OK) return st;
+    if ((st = check_row_stride(y_row_stride, cols, rows)) != KOP_OK) return st;
+    const int esz = elem_size(dtype);
+    if (!aligned_to(x, esz) || !aligned_to(y, esz) || (bias != nullptr && !aligned_to(bias, 4)))
+        return KOP_ERR_MISALIGNED;
+    if (!alias_ok(x, x_row_stride, y, y_row_stride, rows, cols, esz, true)) return KOP_ERR_BAD_ALIAS;
+    if ((st = check_device()) != KOP_OK) return st;
+    cudaStream_t s = as_stream(stream);
+    const SmOpts opts{log_output != 0, causal_period, cols};
+    return dtype == KOP_F32
+               ? launch_softmax<float>(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale, s, true, opts)
+               : dtype == KOP_BF16 ? launch_softmax<__nv_bfloat16>(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale, s, true, opts)
+               : launch_softmax<__half>(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale, s, true, opts);
 }

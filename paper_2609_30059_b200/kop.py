@@ -52,6 +52,8 @@ def lib() -> C.CDLL:
     L.kop_status_string.restype = C.c_char_p
     L.kop_status_string.argtypes = [i32]
     L.kop_softmax_scale_bias.argtypes = [vp, vp, vp, i64, i64, i64, i64, f32, i32, vp]
+    L.kop_softmax_opts.argtypes = [vp, vp, vp, i64, i64, i64, i64, f32, i32, i64, i32, vp]
+    L.kop_softmax_opts.restype = i32
     L.kop_bias_gelu_residual_layernorm.argtypes = [vp] * 8 + [i64] * 5 + [f32, i32, vp]
     L.kop_bias_erfgelu_residual_layernorm.argtypes = [vp] * 8 + [i64] * 5 + [f32, i32, vp]
     L.kop_bias_erfgelu_residual_layernorm.restype = i32
@@ -152,6 +154,17 @@ def kop_softmax_scale_bias(x, bias, scale, out=None, stream=None):
     _check(lib().kop_softmax_scale_bias(x.data_ptr(), _param(bias, "bias", cols), out.data_ptr(), rows,
                                         cols, xs, ys, float(scale), _dtype_tag(x), _stream(stream)),
            "kop_softmax_scale_bias")
+    return out
+
+
+def kop_softmax_opts(x, bias, scale, log_output=False, causal_period=0, out=None, stream=None):
+    rows, cols, xs = _rows2d(x, "x")
+    out = torch.empty_like(x) if out is None else out
+    _, _, ys = _rows2d(out, "out")
+    assert out.shape == x.shape and out.dtype == x.dtype
+    _check(lib().kop_softmax_opts(x.data_ptr(), _param(bias, "bias", cols), out.data_ptr(), rows, cols, xs, ys,
+                                  float(scale), int(bool(log_output)), int(causal_period), _dtype_tag(x),
+                                  _stream(stream)), "kop_softmax_opts")
     return out
 
 

@@ -69,6 +69,17 @@ def test_softmax_validation(L):
     assert f(P, None, P, 0, 8, 8, 8, 1.0, 0, None) == OK
 
 
+def test_softmax_opts_validation(L):
+    f = L.kop_softmax_opts
+    assert f(P, None, Q, 0, 8, 8, 8, 1.0, 0, 0, 0, None) == OK
+    assert f(None, None, Q, 4, 8, 8, 8, 1.0, 0, 0, 0, None) == NULLP
+    assert f(P, None, Q, 4, 8, 8, 8, 1.0, 1, 9, 0, None) == SHAPE          # period beyond the row length
+    assert f(P, None, Q, 4, 8, 8, 8, 1.0, 1, -1, 0, None) == SHAPE
+    assert f(P, None, Q, 4, 8, 7, 8, 1.0, 0, 8, 0, None) == STRIDE
+    assert f(P, None, Q, 4, 8, 8, 8, 1.0, 0, 8, 5, None) == DTYPE
+    assert f(P, None, P + 16, 4, 8, 8, 8, 1.0, 0, 8, 0, None) == ALIAS
+
+
 def test_layernorm_validation(L):
     f = L.kop_bias_gelu_residual_layernorm
     good = [P, Q, R, R + 4096, R + 8192, 0x800000, None, None, 4, 64, 64, 64, 64, 1e-5, 1, None]

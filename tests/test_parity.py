@@ -354,6 +354,55 @@ def test_bn_full_config_seed0_and_options(kop):
     assert ye.shape == e.shape and pe.shape == (0, 256)
 
 
+# ------------------------------------------------------------------------------------------ softmax variants
+
+def assert_close_with_neg_inf(got, ref, tol, what):
+    g = to_f64(got)
+    assert np.array_equal(np.isneginf(g), np.isneginf(ref)), what + ": masked positions"
+    fin = ~np.isneginf(ref)
+    err = np.abs(g[fin] - ref[fin])
+    assert np.all(err <= tol * np.maximum(1.0, np.abs(ref[fin]))), f"{what}: max err {err.max():.3e}"
+
+
+@pytest.mark.parametrize("rows,cols,dtype", [(96, 512, F32), (1024, 128, BF16), (130, 1000, F32), (66, 1001, F32),
+                                             (20, 16384, BF16), (12, 20000, F32), (9, 1, F32)])
+@pytest.mark.parametrize("seed", SEEDS)
+def test_softmax_opts_parity(kop, rows, cols, dtype, seed):
+    x, bias = synth.softmax_inputs(rows, cols, dtype, seed, "cuda")
+    tol = tol_of(dtype)
+    period = cols if cols <= 512 else cols // 3
+    for log_output in (False, True):
+        for causal in (0, period):
+            for use_bias in (True, False):
+                y = Guarded((rows, cols), dtype)
+                kop.kop_softmax_opts(x, bias if use_bias else None, 0.125, log_output, causal, out=y.t)
+                ref = kopref.softmax_opts(host(x), host(bias) if use_bias else None, 0.125, log_output, causal, threads=None)
+                what = f"softmax_opts log={log_output} causal={causal} bias={use_bias}"
+                if log_output:
+                    assert_close_with_neg_inf(y.t, ref, tol, what)
+                else:
+                    assert_close(y.t, ref, tol, what)
+                y.check(what)
+    # no options: the same values as the plain entry point (another kernel path for short rows)
+    plain = kop.kop_softmax_scale_bias(x, bias, 0.125)
+    assert_close(kop.kop_softmax_opts(x, bias, 0.125), to_f64(plain), 1e-6 if dtype == F32 else tol, "softmax_opts without options")
+
+
+def test_softmax_opts_attention_shape_and_validation(kop):
+    # attention scores of 4 heads x 256 queries over 256 keys, square causal mask, in place
+    S = 256
+    x, _ = synth.softmax_inputs(4 * S, S, BF16, 3, "cuda")
+    ref = kopref.softmax_opts(host(x), None, 0.125, False, S, threads=None)
+    xi = x.clone()
+    kop.kop_softmax_opts(xi, None, 0.125, False, S, out=xi)
+    assert_close(xi, ref, 2e-2, "causal attention softmax in place")
+    assert bool((xi.view(4, S, S).triu(1) == 0).all())
+    assert bool(torch.allclose(xi.float().sum(dim=1), torch.ones(4 * S, device="cuda"), atol=2e-2))
+    with pytest.raises(kop.KopError) as ei:
+        kop.kop_softmax_opts(x, None, 1.0, False, S + 1)
+    assert ei.value.status == 2
+
+
 # ------------------------------------------------------------------------------------------ cross-entropy
 
 CE_SHAPES = [
