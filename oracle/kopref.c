@@ -757,3 +757,26 @@ int kopref_softmax_opts(const void* x, const float* bias, double* y, int64_t row
     }
     return 0;
 }
+
+/* ---- pointwise epilogue chain (the paper's L2-064 case: several pointwise operations after a vendor GEMM,
+ * fused into one pass; its exact operations are not given, this is the general form of the class) ---------
+ *   u = (x[i,j] + bias[j]) * scale + residual[i,j] * residual_scale     (bias / residual NULL: term absent)
+ *   u = min(max(u, lo), hi)                                              (NaN stays NaN; lo = -inf, hi = +inf: none)
+ *   y = act(u)                                                           (activations of kopref_bias_act) */
+int kopref_epilogue_chain(const void* x, const float* bias, const void* residual, double* y, int64_t rows,
+        int64_t cols, int64_t x_row_stride, int64_t res_row_stride, int64_t y_row_stride, double scale,
+        double residual_scale, double lo, double hi, int act, double alpha, int dtype, int threads)
+{
+    if (!x || !y || rows < 0 || cols <= 0 || act < 0 || act > 10 || bad_dtype(dtype) || !(lo <= hi)) return -1;
+    int nt = pick_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t i = 0; i < rows; ++i)
+        for (int64_t j = 0; j < cols; ++j) {
+            double u = (load_elem(x, i * x_row_stride + j, dtype) + (bias ? (double)bias[j] : 0.0)) * scale;
+            if (residual) u += load_elem(residual, i * res_row_stride + j, dtype) * residual_scale;
+            if (u == u) u = u < lo ? lo : (u > hi ? hi : u);
+            y[i * y_row_stride + j] = act_value(u, act, alpha);
+        }
+    return 0;
+}

@@ -56,6 +56,7 @@ def lib() -> C.CDLL:
         _lib.kopref_act_value.restype = dbl
         _lib.kopref_act_value.argtypes = [dbl, C.c_int, dbl]
         _lib.kopref_softmax_opts.argtypes = [vp, vp, vp, i64, i64, i64, i64, dbl, C.c_int, i64, C.c_int, C.c_int]
+        _lib.kopref_epilogue_chain.argtypes = [vp, vp, vp, vp] + [i64] * 5 + [dbl] * 4 + [C.c_int, dbl, C.c_int, C.c_int]
         _lib.kopref_cumsum_rows.argtypes = [vp, vp, vp] + [i64] * 5 + [C.c_int] * 4
         _lib.kopref_matvec_bias.argtypes = [vp, vp, dbl, vp, i64, i64, i64, C.c_int, C.c_int]
     return _lib
@@ -379,6 +380,23 @@ def bias_act(x, bias, act, alpha=0.01, threads=1) -> np.ndarray:
     y = np.empty((rows, cols), dtype=np.float64)
     _check(lib().kopref_bias_act(_p(xa), _p(b), _p(y), rows, cols, cols, cols, ACTS[act], float(alpha), dt, _nt(threads)),
            "bias_act")
+    return y
+
+
+def epilogue_chain(x, bias, residual, scale=1.0, residual_scale=1.0, lo=-np.inf, hi=np.inf, act="identity", alpha=0.01,
+                   threads=1) -> np.ndarray:
+    """y = act(clamp((x + bias) * scale + residual * residual_scale, lo, hi)); bias / residual may be None."""
+    xa, dt = as_data(x)
+    rows, cols = xa.shape
+    b = as_param(bias)
+    ra = None
+    if residual is not None:
+        ra, dt2 = as_data(residual)
+        assert dt2 == dt and ra.shape == xa.shape
+    y = np.empty((rows, cols), dtype=np.float64)
+    _check(lib().kopref_epilogue_chain(_p(xa), _p(b), _p(ra), _p(y), rows, cols, cols, cols, cols, float(scale),
+                                       float(residual_scale), float(lo), float(hi), ACTS[act], float(alpha), dt, _nt(threads)),
+           "epilogue_chain")
     return y
 
 

@@ -936,3 +936,30 @@ def test_softmax_opts_log_and_causal():
     for r in range(8):
         vis = 5 + (r % 4) + 1
         assert np.all(q[r, vis:] == 0) and q[r, :vis].sum() == pytest.approx(1.0, rel=1e-14) and np.all(q[r, :vis] > 0)
+
+
+# --------------------------------------------------------------------------- pointwise epilogue chain
+
+def test_epilogue_chain_composition_and_special_cases():
+    x = torch.from_numpy(f32(RNG.normal(0, 2, (5, 33))))
+    r = torch.from_numpy(f32(RNG.normal(0, 2, (5, 33))))
+    b = torch.from_numpy(f32(RNG.normal(0, 0.5, 33)))
+    u = (x.double() + b.double()) * 0.7 + r.double() * 1.5
+    # the composition written with library operations in float64
+    np.testing.assert_allclose(kopref.epilogue_chain(x, b, r, 0.7, 1.5, -1.0, 2.0, "gelu_tanh"),
+                               F.gelu(torch.clamp(u, -1.0, 2.0), approximate="tanh").numpy(), rtol=1e-13, atol=1e-14)
+    np.testing.assert_allclose(kopref.epilogue_chain(x, b, r, 0.7, 1.5, act="mish"), F.mish(u).numpy(), rtol=1e-13, atol=1e-14)
+    # special cases reduce to the other oracles: no residual, unit scale, no clamp = bias_act; x + r = residual_add
+    assert np.array_equal(kopref.epilogue_chain(x, b, None, act="silu"), kopref.bias_act(x, b, "silu"))
+    assert np.array_equal(kopref.epilogue_chain(x, None, r), kopref.residual_add(x, r))
+    # hardtanh is the clamp alone; relu6 is clamp(0, 6)
+    np.testing.assert_allclose(kopref.epilogue_chain(x, None, None, 3.0, lo=-1.0, hi=1.0), F.hardtanh(x.double() * 3.0).numpy(),
+                               rtol=0, atol=0)
+    np.testing.assert_allclose(kopref.epilogue_chain(x, None, None, 3.0, lo=0.0, hi=6.0), F.relu6(x.double() * 3.0).numpy(),
+                               rtol=0, atol=0)
+    # the order matters: the bias is added before the scale, the clamp comes before the activation
+    one = torch.tensor([[2.0]])
+    assert kopref.epilogue_chain(one, torch.tensor([1.0]), None, 10.0)[0, 0] == 30.0
+    assert kopref.epilogue_chain(one, None, None, 1.0, lo=-1.0, hi=1.0, act="sigmoid")[0, 0] == pytest.approx(1 / (1 + math.exp(-1.0)))
+    # NaN passes through the clamp
+    assert math.isnan(kopref.epilogue_chain(torch.tensor([[float("nan")]]), None, None, lo=0.0, hi=1.0)[0, 0])
