@@ -350,6 +350,21 @@ kop_status_t kop_bias_act(const void* x, const float* bias, void* y, int64_t row
                           kop_dtype_t dtype, kop_stream_t stream);
 
 /*
+ * Pointwise epilogue chain: the general form of the "several pointwise operations after a vendor GEMM" class
+ * (the paper's L2-064 case, whose operations are not listed; fusion agent: "pointwise + pointwise: load once,
+ * store once"), one pass:
+ *   u = (x[i,j] + bias[j]) * scale + residual[i,j] * residual_scale     (bias / residual NULL: term absent)
+ *   u = min(max(u, clamp_lo), clamp_hi)     (NaN stays NaN; -INFINITY / +INFINITY switch a side off)
+ *   y[i,j] = act(u)                          (act and alpha as in kop_bias_act)
+ * x, residual, y: [rows, cols] of `dtype`; bias: fp32 [cols]. clamp_lo <= clamp_hi, else KOP_ERR_BAD_SHAPE.
+ * y may alias x or residual exactly.
+ */
+kop_status_t kop_epilogue_chain(const void* x, const float* bias, const void* residual, void* y,
+                                int64_t rows, int64_t cols, int64_t x_row_stride, int64_t res_row_stride,
+                                int64_t y_row_stride, float scale, float residual_scale, float clamp_lo,
+                                float clamp_hi, int act, float alpha, kop_dtype_t dtype, kop_stream_t stream);
+
+/*
  * Row reductions (the "Reduction" rows of the paper's result tables and its planner's "single-pass
  * reductions" / "LogSumExp reductions"), one read-only pass:
  *   op 0 sum, 1 mean, 2 max, 3 min, 4 logsumexp = m + ln sum_j exp(x[i,j] - m), m = max_j x[i,j]

@@ -101,6 +101,131 @@ bias_act_scalar_kernel(const T* __restrict__ x, const float* __restrict__ bias, 
     }
 }
 
+// ---- the general chain: y = act(clamp((x + bias) * scale + residual * residual_scale, lo, hi)) ----------
+struct ChainArgs {
+    float scale, residual_scale, lo, hi, alpha;
+};
+
+__device__ __forceinline__ float chain_value(float x, float b, float r, const ChainArgs& a)
+{
+    float u = fmaf(r, a.residual_scale, (x + b) * a.scale);
+    float c;                                   // clamp with NaN-propagating min / max: a NaN stays a NaN
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(c) : "f"(u), "f"(a.lo));
+    asm("min.NaN.f32 %0, %1, %2;" : "=f"(u) : "f"(c), "f"(a.hi));
+    return u;
+}
+
+template <typename T, int ACT>
+__global__ void __launch_bounds__(256)
+chain_kernel(const T* __restrict__ x, const float* __restrict__ bias, const T* __restrict__ res, T* __restrict__ y,
+             int nvec, int tiles_per_row, int64_t x_stride, int64_t r_stride, int64_t y_stride, ChainArgs a)
+{
+    constexpr int E = Elem<T>::kPerVec, U = 2;
+    constexpr bool kFast = sizeof(T) == 2;
+    const int64_t row = blockIdx.x / tiles_per_row;
+    const int tile = (int)(blockIdx.x - row * tiles_per_row);
+    const T* xr = x + row * x_stride;
+    const T* rr = res != nullptr ? res + row * r_stride : nullptr;
+    T* yr = y + row * y_stride;
+    const int v0 = tile * (U * blockDim.x) + threadIdx.x;
+    Vec16 rx[U], rres[U];
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+        const int v = v0 + k * blockDim.x;
+        if (v < nvec) {
+            rx[k] = ld_stream(xr + (int64_t)v * E);
+            if (rr != nullptr) rres[k] = ld_stream(rr + (int64_t)v * E);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+        const int v = v0 + k * blockDim.x;
+        if (v < nvec) {
+            float f[E], g[E], b[E];
+            Elem<T>::unpack(rx[k], f);
+            if (rr != nullptr) Elem<T>::unpack(rres[k], g);
+#pragma unroll
+            for (int q = 0; q < E / 4; ++q) {
+                float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (bias != nullptr) t = ldg_f4(bias + (int64_t)v * E + 4 * q);
+                b[4 * q] = t.x;
+                b[4 * q + 1] = t.y;
+                b[4 * q + 2] = t.z;
+                b[4 * q + 3] = t.w;
+            }
+#pragma unroll
+            for (int e = 0; e < E; ++e)
+                f[e] = act_dev<ACT, kFast>(chain_value(f[e], b[e], rr != nullptr ? g[e] : 0.0f, a), a.alpha);
+            st_stream(yr + (int64_t)v * E, Elem<T>::pack(f));
+        }
+    }
+}
+
+template <typename T, int ACT>
+__global__ void __launch_bounds__(256)
+chain_scalar_kernel(const T* __restrict__ x, const float* __restrict__ bias, const T* __restrict__ res,
+                    T* __restrict__ y, int64_t rows, int64_t cols, int64_t x_stride, int64_t r_stride,
+                    int64_t y_stride, ChainArgs a)
+{
+    constexpr bool kFast = sizeof(T) == 2;
+    const int64_t total = rows * cols;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / cols, j = i - r * cols;
+        const float u = chain_value(Elem<T>::load1(x + r * x_stride + j), bias != nullptr ? __ldg(bias + j) : 0.0f,
+                                    res != nullptr ? Elem<T>::load1(res + r * r_stride + j) : 0.0f, a);
+        Elem<T>::store1(y + r * y_stride + j, act_dev<ACT, kFast>(u, a.alpha));
+    }
+}
+
+template <typename T, int ACT>
+kop_status_t launch_chain_a(const T* x, const float* bias, const T* res, T* y, int64_t rows, int64_t cols, int64_t xs,
+                            int64_t rs, int64_t ys, const ChainArgs& a, cudaStream_t stream)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    const bool vec = vec_ok(x, cols, xs, sizeof(T)) && vec_ok(y, cols, ys, sizeof(T)) && cols / E <= 0x3FFFFFFF &&
+                     (res == nullptr || vec_ok(res, cols, rs, sizeof(T))) && (bias == nullptr || aligned_to(bias, 16));
+    if (vec) {
+        const int nvec = (int)(cols / E);
+        int threads = ((nvec + 1) / 2 + 31) / 32 * 32;
+        if (threads > 256) threads = 256;
+        const int tiles = (nvec + 2 * threads - 1) / (2 * threads);
+        const int64_t grid = rows * tiles;
+        if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+        chain_kernel<T, ACT><<<(unsigned)grid, threads, 0, stream>>>(x, bias, res, y, nvec, tiles, xs, rs, ys, a);
+        return launch_status();
+    }
+    int64_t blocks = (rows * cols + 255) / 256;
+    const int64_t cap = 32LL * sm_count();
+    if (blocks > cap) blocks = cap;
+    chain_scalar_kernel<T, ACT><<<(unsigned)blocks, 256, 0, stream>>>(x, bias, res, y, rows, cols, xs, rs, ys, a);
+    return launch_status();
+}
+
+template <typename T>
+kop_status_t launch_chain(const void* xv, const float* bias, const void* rv, void* yv, int64_t rows, int64_t cols,
+                          int64_t xs, int64_t rs, int64_t ys, int act, const ChainArgs& a, cudaStream_t stream)
+{
+    const T* x = static_cast<const T*>(xv);
+    const T* r = static_cast<const T*>(rv);
+    T* y = static_cast<T*>(yv);
+#define KOP_CHAIN_CASE(A) \
+    case A: return launch_chain_a<T, A>(x, bias, r, y, rows, cols, xs, rs, ys, a, stream)
+    switch (act) {
+        KOP_CHAIN_CASE(kActRelu);
+        KOP_CHAIN_CASE(kActLeakyRelu);
+        KOP_CHAIN_CASE(kActGeluTanh);
+        KOP_CHAIN_CASE(kActGeluErf);
+        KOP_CHAIN_CASE(kActSilu);
+        KOP_CHAIN_CASE(kActSigmoid);
+        KOP_CHAIN_CASE(kActTanh);
+        KOP_CHAIN_CASE(kActMish);
+        KOP_CHAIN_CASE(kActHardswish);
+        KOP_CHAIN_CASE(kActElu);
+    default: return launch_chain_a<T, kActIdentity>(x, bias, r, y, rows, cols, xs, rs, ys, a, stream);
+    }
+#undef KOP_CHAIN_CASE
+}
+
 template <typename T, int ACT>
 kop_status_t launch_bias_act_a(const T* x, const float* bias, T* y, int64_t rows, int64_t cols, int64_t xs,
                                int64_t ys, float alpha, cudaStream_t stream)
@@ -180,4 +305,38 @@ extern "C" kop_status_t kop_bias_act(const void* x, const float* bias, void* y, 
            : dtype == KOP_BF16
                ? launch_bias_act<__nv_bfloat16>(x, bias, y, rows, cols, x_row_stride, y_row_stride, act, alpha, s)
                : launch_bias_act<__half>(x, bias, y, rows, cols, x_row_stride, y_row_stride, act, alpha, s);
+}
+
+extern "C" kop_status_t kop_epilogue_chain(const void* x, const float* bias, const void* residual, void* y,
+                                           int64_t rows, int64_t cols, int64_t x_row_stride, int64_t res_row_stride,
+                                           int64_t y_row_stride, float scale, float residual_scale, float clamp_lo,
+                                           float clamp_hi, int act, float alpha, kop_dtype_t dtype,
+                                           kop_stream_t stream)
+{
+    using namespace kop;
+    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    kop_status_t st = check_rows_cols(rows, cols);
+    if (st != KOP_OK) return st;
+    if (act < 0 || act >= kActCount || !(clamp_lo <= clamp_hi)) return KOP_ERR_BAD_SHAPE;
+    if ((st = check_row_stride(x_row_stride, cols, rows)) != KOP_OK) return st;
+    if (residual != nullptr && (st = check_row_stride(res_row_stride, cols, rows)) != KOP_OK) return st;
+    if ((st = check_row_stride(y_row_stride, cols, rows)) != KOP_OK) return st;
+    if (rows == 0) return KOP_OK;
+    if (!x || !y) return KOP_ERR_NULL_POINTER;
+    const int esz = elem_size(dtype);
+    if (!aligned_to(x, esz) || !aligned_to(y, esz) || (residual && !aligned_to(residual, esz)) ||
+        (bias && !aligned_to(bias, 4)))
+        return KOP_ERR_MISALIGNED;
+    if (!alias_ok(x, x_row_stride, y, y_row_stride, rows, cols, esz, true) ||
+        (residual && !alias_ok(residual, res_row_stride, y, y_row_stride, rows, cols, esz, true)))
+        return KOP_ERR_BAD_ALIAS;
+    if ((st = check_device()) != KOP_OK) return st;
+    cudaStream_t s = as_stream(stream);
+    const ChainArgs a{scale, residual_scale, clamp_lo, clamp_hi, alpha};
+    return dtype == KOP_F32 ? launch_chain<float>(x, bias, residual, y, rows, cols, x_row_stride, res_row_stride,
+                                                  y_row_stride, act, a, s)
+           : dtype == KOP_BF16 ? launch_chain<__nv_bfloat16>(x, bias, residual, y, rows, cols, x_row_stride,
+                                                             res_row_stride, y_row_stride, act, a, s)
+                               : launch_chain<__half>(x, bias, residual, y, rows, cols, x_row_stride, res_row_stride,
+                                                      y_row_stride, act, a, s);
 }

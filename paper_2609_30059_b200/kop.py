@@ -86,6 +86,8 @@ def lib() -> C.CDLL:
     L.kop_reduce_rows.restype = i32
     L.kop_bias_act.argtypes = [vp, vp, vp, i64, i64, i64, i64, i32, f32, i32, vp]
     L.kop_bias_act.restype = i32
+    L.kop_epilogue_chain.argtypes = [vp, vp, vp, vp] + [i64] * 5 + [f32] * 4 + [i32, f32, i32, vp]
+    L.kop_epilogue_chain.restype = i32
     L.kop_cumsum_rows.argtypes = [vp, vp, vp] + [i64] * 5 + [i32, i32, i32, vp]
     L.kop_cumsum_rows.restype = i32
     L.kop_groupnorm_wait_timeouts.argtypes = [C.POINTER(C.c_uint)]
@@ -401,6 +403,22 @@ def kop_bias_act(x, bias, act, alpha=0.01, out=None, stream=None):
     assert out.shape == x.shape and out.dtype == x.dtype
     _check(lib().kop_bias_act(x.data_ptr(), _param(bias, "bias", cols), out.data_ptr(), rows, cols, xs, ys, ACTS[act],
                               float(alpha), _dtype_tag(x), _stream(stream)), "kop_bias_act")
+    return out
+
+
+def kop_epilogue_chain(x, bias, residual, scale=1.0, residual_scale=1.0, lo=float("-inf"), hi=float("inf"),
+                       act="identity", alpha=0.01, out=None, stream=None):
+    rows, cols, xs = _rows2d(x, "x")
+    rs = cols
+    if residual is not None:
+        _, _, rs = _rows2d(residual, "residual")
+        assert residual.shape == x.shape and residual.dtype == x.dtype
+    out = torch.empty_like(x) if out is None else out
+    _, _, ys = _rows2d(out, "out")
+    assert out.shape == x.shape and out.dtype == x.dtype
+    _check(lib().kop_epilogue_chain(x.data_ptr(), _param(bias, "bias", cols), None if residual is None else residual.data_ptr(),
+                                    out.data_ptr(), rows, cols, xs, rs, ys, float(scale), float(residual_scale), float(lo),
+                                    float(hi), ACTS[act], float(alpha), _dtype_tag(x), _stream(stream)), "kop_epilogue_chain")
     return out
 
 

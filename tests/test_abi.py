@@ -264,6 +264,22 @@ def test_bias_act_validation(L):
     assert f(P, Q, P + 8, 4, 64, 64, 64, 1, 0.0, 0, None) == ALIAS
 
 
+def test_epilogue_chain_validation(L):
+    f = L.kop_epilogue_chain
+    inf = float("inf")
+    S = 0x600000
+    assert f(P, Q, S, R, 0, 64, 64, 64, 64, 1.0, 1.0, -inf, inf, 0, 0.0, 0, None) == OK
+    assert f(None, Q, S, R, 4, 64, 64, 64, 64, 1.0, 1.0, -inf, inf, 0, 0.0, 0, None) == NULLP
+    assert f(P, None, None, R, 4, 64, 64, 1, 64, 1.0, 1.0, -inf, inf, 0, 0.0, 0, None) not in (NULLP, STRIDE)   # both optional
+    assert f(P, Q, S, R, 4, 64, 64, 63, 64, 1.0, 1.0, -inf, inf, 0, 0.0, 0, None) == STRIDE
+    assert f(P, Q, S, R, 4, 64, 64, 64, 64, 1.0, 1.0, 2.0, 1.0, 0, 0.0, 0, None) == SHAPE          # lo > hi
+    assert f(P, Q, S, R, 4, 64, 64, 64, 64, 1.0, 1.0, float("nan"), 1.0, 0, 0.0, 0, None) == SHAPE
+    assert f(P, Q, S, R, 4, 64, 64, 64, 64, 1.0, 1.0, -inf, inf, 11, 0.0, 0, None) == SHAPE
+    assert f(P, Q, S, R, 4, 64, 64, 64, 64, 1.0, 1.0, -inf, inf, 0, 0.0, 9, None) == DTYPE
+    assert f(P, Q, S + 2, R, 4, 64, 64, 64, 64, 1.0, 1.0, -inf, inf, 0, 0.0, 0, None) == MISAL
+    assert f(P, Q, S, S + 8, 4, 64, 64, 64, 64, 1.0, 1.0, -inf, inf, 0, 0.0, 0, None) == ALIAS      # y overlaps residual
+
+
 def test_mlp_driver_validation(L):
     f = L.kop_rmsnorm_swiglu_residual
     wsb = L.kop_rmsnorm_swiglu_residual_workspace_bytes(16, 64, 128, 1)

@@ -77,3 +77,32 @@ def test_bias_act_options(kop):
     e = torch.empty((0, 8), dtype=F32, device="cuda")
     assert kop.kop_bias_act(e, None, "relu").shape == (0, 8)
     assert kop.lib().kop_bias_act(x.data_ptr(), None, x.data_ptr(), 4, 16, 16, 16, 11, 0.0, 0, None) == 2
+
+
+@pytest.mark.parametrize("rows,cols,dtype", [(256, 4096, BF16), (300, 4096, F32), (65, 1000, F16), (33, 1001, F32), (7, 1, BF16)])
+@pytest.mark.parametrize("seed", SEEDS)
+def test_epilogue_chain_parity(kop, rows, cols, dtype, seed):
+    """The general chain y = act(clamp((x + bias) * scale + residual * residual_scale, lo, hi))."""
+    x, bias = synth.softmax_inputs(rows, cols, dtype, seed, "cuda")
+    r, _ = synth.softmax_inputs(rows, cols, dtype, seed + 1, "cuda")
+    tol = tol_of(dtype)
+    inf = float("inf")
+    cases = [(bias, r, 0.7, 1.5, -1.0, 2.0, "gelu_tanh"), (bias, None, 2.0, 1.0, -inf, inf, "mish"),
+             (None, r, 1.0, 1.0, -inf, inf, "identity"), (bias, r, 3.0, -0.5, 0.0, 6.0, "identity"),
+             (None, None, 4.0, 1.0, -1.0, 1.0, "sigmoid"), (bias, r, 1.0, 1.0, -inf, 0.5, "elu")]
+    for b, res, scale, rscale, lo, hi, act in cases:
+        y = Guarded((rows, cols), dtype)
+        kop.kop_epilogue_chain(x, b, res, scale, rscale, lo, hi, act, alpha=0.3, out=y.t)
+        ref = kopref.epilogue_chain(host(x), host(b), host(res), scale, rscale, lo, hi, act, alpha=0.3, threads=None)
+        assert_close(y.t, ref, tol, f"chain {act} bias={b is not None} res={res is not None}")
+        y.check("chain")
+    # in place over the residual, and NaN through the clamp
+    ri = r.clone()
+    kop.kop_epilogue_chain(x, bias, ri, 0.7, 1.5, -1.0, 2.0, "gelu_tanh", out=ri)
+    assert_close(ri, kopref.epilogue_chain(host(x), host(bias), host(r), 0.7, 1.5, -1.0, 2.0, "gelu_tanh"), tol, "chain in place")
+    xn = x.clone()
+    xn[0, 0] = float("nan")
+    assert bool(torch.isnan(kop.kop_epilogue_chain(xn, None, None, lo=0.0, hi=1.0)[0, 0]))
+    with pytest.raises(kop.KopError) as ei:
+        kop.kop_epilogue_chain(x, None, None, lo=1.0, hi=0.0)
+    assert ei.value.status == 2
