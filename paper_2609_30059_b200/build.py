@@ -8,6 +8,7 @@ from __future__ import annotations
 
 import concurrent.futures
 import glob
+import hashlib
 import os
 import shutil
 import subprocess
@@ -39,20 +40,33 @@ def sources() -> list[str]:
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
 
 
-def _deps_mtime() -> float:
-    files = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(INCLUDE, "*.h"))
-    return max(os.path.getmtime(f) for f in files)
+def _fingerprint(flags: list[str]) -> str:
+    """Hash of every source, header and flag that goes into the library. File times are useless for this:
+    a copy of the tree (another machine, a fresh checkout) has new times on unchanged files."""
+    h = hashlib.sha256()
+    files = sources() + sorted(glob.glob(os.path.join(CSRC, "*.cuh"))) + sorted(glob.glob(os.path.join(INCLUDE, "*.h")))
+    for f in files:
+        h.update(os.path.basename(f).encode())
+        with open(f, "rb") as fh:
+            h.update(fh.read())
+    h.update(" ".join(x for x in flags if not x.startswith("-I")).encode())
+    return h.hexdigest()
 
 
 def build(force: bool = False, verbose: bool = False, extra_flags: list[str] | None = None,
           out: str | None = None) -> str:
     """Compile and link; returns the path of the shared library."""
     lib = out or LIB
-    if not force and os.path.exists(lib) and os.path.getmtime(lib) >= _deps_mtime():
-        return lib
+    stamp = lib + ".stamp"
+    base_flags = NVCC_FLAGS + (extra_flags or [])
+    want = _fingerprint(base_flags)
+    if not force and os.path.exists(lib) and os.path.exists(stamp):
+        with open(stamp) as fh:
+            if fh.read().strip() == want:
+                return lib
     nvcc = _nvcc()
     os.makedirs(OBJ, exist_ok=True)
-    flags = NVCC_FLAGS + (extra_flags or []) + (["-Xptxas", "-v"] if verbose else [])
+    flags = base_flags + (["-Xptxas", "-v"] if verbose else [])
 
     def compile_one(src: str) -> str:
         obj = os.path.join(OBJ, os.path.basename(src)[:-3] + (".o" if out is None else f".{os.getpid()}.o"))
@@ -70,6 +84,9 @@ def build(force: bool = False, verbose: bool = False, extra_flags: list[str] | N
     subprocess.run([nvcc, "-shared", *ARCH, "-o", tmp, *objs, "-L" + libdir, "-lcublas", "-lcublasLt",
                     "-Xlinker", "-rpath", "-Xlinker", libdir], check=True)
     os.replace(tmp, lib)
+    with open(stamp + f".tmp{os.getpid()}", "w") as fh:
+        fh.write(want + "\n")
+    os.replace(stamp + f".tmp{os.getpid()}", stamp)
     if out is not None:
         for o in objs:
             os.remove(o)
