@@ -220,6 +220,14 @@ def rmsnorm(x, weight, eps, threads=1) -> np.ndarray:
     return y
 
 
+def residual_rmsnorm(x, residual, weight, eps, threads=1):
+    """The residual stream step of a pre-norm transformer block: h = x + residual, y = rmsnorm(h; weight, eps),
+    both from the unrounded float64 sum. Returns (h, y). A composition of the two oracle functions above and
+    below (residual_add, rmsnorm): nothing new is computed here."""
+    h = residual_add(x, residual, threads)
+    return h, rmsnorm(h, weight, eps, threads)
+
+
 def silu_mul(gate_up, threads=1) -> np.ndarray:
     ga, dt = as_data(gate_up)
     rows, two_i = ga.shape

@@ -963,3 +963,23 @@ def test_epilogue_chain_composition_and_special_cases():
     assert kopref.epilogue_chain(one, None, None, 1.0, lo=-1.0, hi=1.0, act="sigmoid")[0, 0] == pytest.approx(1 / (1 + math.exp(-1.0)))
     # NaN passes through the clamp
     assert math.isnan(kopref.epilogue_chain(torch.tensor([[float("nan")]]), None, None, lo=0.0, hi=1.0)[0, 0])
+
+
+# --------------------------------------------------------------------------- residual + RMSNorm
+
+def test_residual_rmsnorm_composition_against_torch():
+    x = torch.from_numpy(f32(RNG.normal(0, 1, (6, 40))))
+    r = torch.from_numpy(f32(RNG.normal(0, 1, (6, 40))))
+    w = torch.from_numpy(f32(RNG.normal(1, 0.02, 40)))
+    h, y = kopref.residual_rmsnorm(x, r, w, 1e-6)
+    v = x.double() + r.double()
+    assert np.array_equal(h, v.numpy())
+    np.testing.assert_allclose(y, F.rms_norm(v, (40,), w.double(), 1e-6).numpy(), rtol=1e-14, atol=1e-15)
+    # the norm sees the unrounded sum: with bf16 inputs it differs from rounding h first
+    xb, rb = x.to(torch.bfloat16), r.to(torch.bfloat16)
+    hb, yb = kopref.residual_rmsnorm(xb, rb, w, 1e-6)
+    assert np.array_equal(hb, (xb.double() + rb.double()).numpy())
+    rounded_first = kopref.rmsnorm((xb.float() + rb.float()).to(torch.bfloat16), w, 1e-6)
+    assert np.abs(yb - rounded_first).max() > 1e-4
+    # zero residual: plain RMSNorm
+    assert np.array_equal(kopref.residual_rmsnorm(x, torch.zeros_like(x), w, 1e-6)[1], kopref.rmsnorm(x, w, 1e-6))
