@@ -104,6 +104,7 @@ def segment_bytes():
     out["reduce_max"] = dict(bytes=q["rows"] * q["cols"] * 2 + q["rows"] * 8, elems=q["rows"] * q["cols"])
     out["reduce_logsumexp"] = dict(bytes=q["rows"] * q["cols"] * 2 + q["rows"] * 4, elems=q["rows"] * q["cols"])
     out["bias_gelu"] = dict(bytes=2 * m["rows"] * m["inter"] * 2 + m["inter"] * 4, elems=m["rows"] * m["inter"])
+    out["residual_rmsnorm"] = dict(bytes=4 * m["rows"] * m["hidden"] * 2 + m["hidden"] * 4, elems=m["rows"] * m["hidden"])
     u = c["cumsum"]
     out["cumsum"] = dict(bytes=2 * u["rows"] * u["cols"] * 4, elems=u["rows"] * u["cols"])
     return out
@@ -249,7 +250,7 @@ class Workload:
 
     ORDER = ["softmax_small", "softmax_large", "layernorm", "bn_pool", "ce_loss", "rmsnorm", "silu_mul", "residual_add"]
     # Beyond the benchmark configs (not part of `value`): the two kernels the paper's case studies print.
-    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc", "pool2d", "reduce_max", "reduce_logsumexp", "bias_gelu"]
+    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc", "pool2d", "reduce_max", "reduce_logsumexp", "bias_gelu", "residual_rmsnorm"]
 
     def __init__(self, kop, device, seed, only=None, rows_div=1):
         """only: build just these segments (None = all, plus the MLP segment); rows_div cuts the row
@@ -335,7 +336,7 @@ class Workload:
         m = c["mlp"]
         self.eps = m["eps"]
         rows = cut(m["rows"])
-        if want & {"rmsnorm", "residual_add", "silu_mul", "mlp"}:
+        if want & {"rmsnorm", "residual_add", "silu_mul", "mlp", "residual_rmsnorm"}:
             g = torch.Generator(device=dev)
             g.manual_seed(seed)
             if "mlp" in want:
@@ -356,7 +357,7 @@ class Workload:
                 if "silu_mul" in want:
                     self.gu = synth.gate_up_inputs(rows, m["inter"], m["dtype"], seed, dev)
                     self.act = torch.empty((rows, m["inter"]), dtype=m["dtype"], device=dev)
-                if "residual_add" in want:
+                if want & {"residual_add", "residual_rmsnorm"}:
                     _, self.d = synth.pair_inputs(rows, m["hidden"], m["dtype"], seed, dev)
             self.res = torch.empty_like(self.h)
 
@@ -408,6 +409,8 @@ class Workload:
             k.kop_reduce_rows(self.rx, "logsumexp", out=self.rv)
         elif name == "bias_gelu":                # bias + tanh-GELU epilogue, bf16 [16384, 14336]
             k.kop_bias_act(self.ax, self.ab, "gelu_tanh", out=self.ay)
+        elif name == "residual_rmsnorm":         # residual add + RMSNorm of the MLP config in one pass
+            k.kop_residual_rmsnorm(self.h, self.d, self.rw, self.eps, h_out=self.res, out=self.n)
         elif name == "cumsum":                   # inclusive running sum along rows, fp32 [32768, 4096]
             k.kop_cumsum_rows(self.ux, out=self.uy)
         else:

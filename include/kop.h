@@ -249,6 +249,20 @@ kop_status_t kop_rmsnorm(const void* x, const float* weight, void* y,
                          float eps, kop_dtype_t dtype, kop_stream_t stream);
 
 /*
+ * Residual add and RMSNorm in one pass (fusion agent: "residual + norm: one kernel, one memory pass", for the
+ * RMSNorm sequences of pre-norm transformer blocks: the add that ends one sub-layer and the norm that opens
+ * the next):
+ *   v = x + residual;   h = v (rounded to `dtype`);   y = v / sqrt(mean_j v^2 + eps) * weight
+ * The normalisation uses the unrounded fp32 v. x, residual, h, y: [rows, hidden] of `dtype`; weight: fp32
+ * [hidden]. h and y may each be x or residual exactly; h and y must be different tensors. Against
+ * kop_residual_add followed by kop_rmsnorm this saves one write-then-read of h (4 instead of 5 tensor passes).
+ */
+kop_status_t kop_residual_rmsnorm(const void* x, const void* residual, const float* weight, void* h, void* y,
+                                  int64_t rows, int64_t hidden, int64_t x_row_stride, int64_t res_row_stride,
+                                  int64_t h_row_stride, int64_t y_row_stride, float eps, kop_dtype_t dtype,
+                                  kop_stream_t stream);
+
+/*
  * SwiGLU epilogue of a preserved GEMM (fusion agent: "activation fusion
  * (GELU/SiLU/ReLU)"; codegen agent: keep the matmul as a library call and fuse only
  * the epilogue):

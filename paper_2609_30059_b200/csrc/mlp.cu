@@ -13,10 +13,18 @@ namespace {
 // ---- RMSNorm: CTA per row, row in registers -----------------------------------------------------
 // kFull: the row is exactly blockDim.x * VPT vectors (no tail predicates). kWide: the eight fp32
 // weights of a bf16 vector come in one 256-bit load per lane (each 128-byte line touched once).
-template <typename T, int VPT, bool kFull, bool kWide>
+// kRes (kop_residual_rmsnorm): the row is v = x + residual, kept in fp32; its rounded copy goes to `h`
+// (the residual stream of the next layer) and the normalisation runs on the unrounded v.
+struct RmsRes {
+    const void* res;
+    void* h;
+    int64_t res_stride, h_stride;
+};
+
+template <typename T, int VPT, bool kFull, bool kWide, bool kRes>
 __global__ void __launch_bounds__(max_threads_for(VPT * Elem<T>::kPerVec))
 rmsnorm_block_kernel(const T* __restrict__ x, const float* __restrict__ w, T* __restrict__ y, int nvec,
-                     int64_t x_stride, int64_t y_stride, float eps, float inv_hidden)
+                     int64_t x_stride, int64_t y_stride, float eps, float inv_hidden, RmsRes rr)
 {
     constexpr int E = Elem<T>::kPerVec;
     constexpr int P = E / 2;
@@ -24,18 +32,33 @@ rmsnorm_block_kernel(const T* __restrict__ x, const float* __restrict__ w, T* __
     const int64_t row = blockIdx.x;
     const T* xr = x + row * x_stride;
     T* yr = y + row * y_stride;
-    Vec16 raw[VPT];
+    const T* resr = kRes ? static_cast<const T*>(rr.res) + row * rr.res_stride : nullptr;
+    T* hr = kRes ? static_cast<T*>(rr.h) + row * rr.h_stride : nullptr;
+    Vec16 raw[VPT], rraw[kRes ? VPT : 1];
 #pragma unroll
     for (int k = 0; k < VPT; ++k) {
         const int v = k * blockDim.x + threadIdx.x;
-        if (kFull || v < nvec) raw[k] = ld_stream(xr + (int64_t)v * E);
-        else raw[k] = Vec16{{0u, 0u, 0u, 0u}};
+        if (kFull || v < nvec) {
+            raw[k] = ld_stream(xr + (int64_t)v * E);
+            if (kRes) rraw[k] = ld_stream(resr + (int64_t)v * E);
+        } else {
+            raw[k] = Vec16{{0u, 0u, 0u, 0u}};
+            if (kRes) rraw[k] = Vec16{{0u, 0u, 0u, 0u}};
+        }
     }
     float2 val[VPT][P];
     float2 ss2 = make_float2(0.0f, 0.0f);
 #pragma unroll
     for (int k = 0; k < VPT; ++k) {
         Elem<T>::unpack2(raw[k], val[k]);
+        if (kRes) {
+            float2 rv[P];
+            Elem<T>::unpack2(rraw[k], rv);
+#pragma unroll
+            for (int q = 0; q < P; ++q) val[k][q] = __fadd2_rn(val[k][q], rv[q]);
+            const int v = k * blockDim.x + threadIdx.x;
+            if (kFull || v < nvec) st_stream(hr + (int64_t)v * E, Elem<T>::pack2(val[k]));
+        }
 #pragma unroll
         for (int q = 0; q < P; ++q) ss2 = __ffma2_rn(val[k][q], val[k][q], ss2);
     }
@@ -54,23 +77,29 @@ rmsnorm_block_kernel(const T* __restrict__ x, const float* __restrict__ w, T* __
     }
 }
 
-template <typename T>
+template <typename T, bool kRes>
 __global__ void __launch_bounds__(256)
 rmsnorm_generic_kernel(const T* __restrict__ x, const float* __restrict__ w, T* __restrict__ y,
-                       int64_t hidden, int64_t x_stride, int64_t y_stride, float eps, float inv_hidden)
+                       int64_t hidden, int64_t x_stride, int64_t y_stride, float eps, float inv_hidden, RmsRes rr)
 {
     __shared__ float red[32];
     const int64_t row = blockIdx.x;
     const T* xr = x + row * x_stride;
     T* yr = y + row * y_stride;
+    const T* resr = kRes ? static_cast<const T*>(rr.res) + row * rr.res_stride : nullptr;
+    T* hr = kRes ? static_cast<T*>(rr.h) + row * rr.h_stride : nullptr;
     float ss = 0.0f;
     for (int64_t j = threadIdx.x; j < hidden; j += blockDim.x) {
-        const float v = Elem<T>::load1(xr + j);
+        const float v = Elem<T>::load1(xr + j) + (kRes ? Elem<T>::load1(resr + j) : 0.0f);
         ss = fmaf(v, v, ss);
     }
     const float r = rsqrtf(block_sum(ss, red) * inv_hidden + eps);
-    for (int64_t j = threadIdx.x; j < hidden; j += blockDim.x)
-        Elem<T>::store1(yr + j, Elem<T>::load1(xr + j) * r * __ldg(w + j));
+    // v is formed again from the inputs, which the same thread overwrites only afterwards: h and y may alias them
+    for (int64_t j = threadIdx.x; j < hidden; j += blockDim.x) {
+        const float v = Elem<T>::load1(xr + j) + (kRes ? Elem<T>::load1(resr + j) : 0.0f);
+        if (kRes) Elem<T>::store1(hr + j, v);
+        Elem<T>::store1(yr + j, v * r * __ldg(w + j));
+    }
 }
 
 // ---- SiLU(gate) * up ------------------------------------------------------------------------------
@@ -255,14 +284,17 @@ residual_add_scalar_kernel(const T* __restrict__ a, const T* __restrict__ b, T* 
 // ---- launchers ------------------------------------------------------------------------------------
 template <typename T>
 kop_status_t launch_rmsnorm(const void* xv, const float* w, void* yv, int64_t rows, int64_t hidden,
-                            int64_t xs, int64_t ys, float eps, cudaStream_t stream)
+                            int64_t xs, int64_t ys, float eps, cudaStream_t stream, bool with_res = false,
+                            RmsRes rr = RmsRes{nullptr, nullptr, 0, 0})
 {
     const T* x = static_cast<const T*>(xv);
     T* y = static_cast<T*>(yv);
     constexpr int E = Elem<T>::kPerVec;
     if (rows > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
     const float inv_hidden = (float)(1.0 / (double)hidden);
-    const bool vec = vec_ok(x, hidden, xs, sizeof(T)) && vec_ok(y, hidden, ys, sizeof(T)) && aligned_to(w, 16);
+    const bool vec = vec_ok(x, hidden, xs, sizeof(T)) && vec_ok(y, hidden, ys, sizeof(T)) && aligned_to(w, 16) &&
+                     (!with_res || (vec_ok(rr.res, hidden, rr.res_stride, sizeof(T)) &&
+                                    vec_ok(rr.h, hidden, rr.h_stride, sizeof(T))));
     const int64_t nvec64 = hidden / E;
     if (vec && hidden <= kMaxRegisterRow) {
         const int nvec = (int)nvec64;
@@ -274,8 +306,11 @@ kop_status_t launch_rmsnorm(const void* xv, const float* w, void* yv, int64_t ro
         const int threads = ((nvec + vpt - 1) / vpt + 31) / 32 * 32;
         const bool full = (nvec % vpt) == 0 && (nvec / vpt) == threads;
         const bool wide = E == 8 && aligned_to(w, 32);
-#define KOP_RMS_LAUNCH(V, F, W) \
-    rmsnorm_block_kernel<T, V, F, W><<<(unsigned)rows, threads, 0, stream>>>(x, w, y, nvec, xs, ys, eps, inv_hidden)
+#define KOP_RMS_LAUNCH(V, F, W)                                                                                       \
+    do {                                                                                                              \
+        if (with_res) rmsnorm_block_kernel<T, V, F, W, true><<<(unsigned)rows, threads, 0, stream>>>(x, w, y, nvec, xs, ys, eps, inv_hidden, rr); \
+        else rmsnorm_block_kernel<T, V, F, W, false><<<(unsigned)rows, threads, 0, stream>>>(x, w, y, nvec, xs, ys, eps, inv_hidden, rr);         \
+    } while (0)
 #define KOP_RMS(V)                                             \
     do {                                                       \
         if (full && wide) KOP_RMS_LAUNCH(V, true, true);       \
@@ -293,7 +328,8 @@ kop_status_t launch_rmsnorm(const void* xv, const float* w, void* yv, int64_t ro
 #undef KOP_RMS
         return launch_status();
     }
-    rmsnorm_generic_kernel<T><<<(unsigned)rows, 256, 0, stream>>>(x, w, y, hidden, xs, ys, eps, inv_hidden);
+    if (with_res) rmsnorm_generic_kernel<T, true><<<(unsigned)rows, 256, 0, stream>>>(x, w, y, hidden, xs, ys, eps, inv_hidden, rr);
+    else rmsnorm_generic_kernel<T, false><<<(unsigned)rows, 256, 0, stream>>>(x, w, y, hidden, xs, ys, eps, inv_hidden, rr);
     return launch_status();
 }
 
@@ -518,6 +554,42 @@ extern "C" kop_status_t kop_rmsnorm(const void* x, const float* weight, void* y,
                ? launch_rmsnorm<float>(x, weight, y, rows, hidden, x_row_stride, y_row_stride, eps, s)
                : dtype == KOP_BF16 ? launch_rmsnorm<__nv_bfloat16>(x, weight, y, rows, hidden, x_row_stride, y_row_stride, eps, s)
                : launch_rmsnorm<__half>(x, weight, y, rows, hidden, x_row_stride, y_row_stride, eps, s);
+}
+
+extern "C" kop_status_t kop_residual_rmsnorm(const void* x, const void* residual, const float* weight, void* h,
+                                             void* y, int64_t rows, int64_t hidden, int64_t x_row_stride,
+                                             int64_t res_row_stride, int64_t h_row_stride, int64_t y_row_stride,
+                                             float eps, kop_dtype_t dtype, kop_stream_t stream)
+{
+    using namespace kop;
+    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    kop_status_t st = check_rows_cols(rows, hidden);
+    if (st != KOP_OK) return st;
+    if (rows == 0) return KOP_OK;
+    if (!x || !residual || !weight || !h || !y) return KOP_ERR_NULL_POINTER;
+    if ((st = check_row_stride(x_row_stride, hidden, rows)) != KOP_OK) return st;
+    if ((st = check_row_stride(res_row_stride, hidden, rows)) != KOP_OK) return st;
+    if ((st = check_row_stride(h_row_stride, hidden, rows)) != KOP_OK) return st;
+    if ((st = check_row_stride(y_row_stride, hidden, rows)) != KOP_OK) return st;
+    if (!(eps >= 0.0f)) return KOP_ERR_BAD_SHAPE;
+    const int esz = elem_size(dtype);
+    if (!aligned_to(x, esz) || !aligned_to(residual, esz) || !aligned_to(h, esz) || !aligned_to(y, esz) ||
+        !aligned_to(weight, 4))
+        return KOP_ERR_MISALIGNED;
+    // each output may be one of the inputs exactly, but the two outputs must be different tensors
+    if (!alias_ok(x, x_row_stride, h, h_row_stride, rows, hidden, esz, true) ||
+        !alias_ok(residual, res_row_stride, h, h_row_stride, rows, hidden, esz, true) ||
+        !alias_ok(x, x_row_stride, y, y_row_stride, rows, hidden, esz, true) ||
+        !alias_ok(residual, res_row_stride, y, y_row_stride, rows, hidden, esz, true) ||
+        !alias_ok(h, h_row_stride, y, y_row_stride, rows, hidden, esz, false))
+        return KOP_ERR_BAD_ALIAS;
+    if ((st = check_device()) != KOP_OK) return st;
+    cudaStream_t s = as_stream(stream);
+    const RmsRes rr{residual, h, res_row_stride, h_row_stride};
+    return dtype == KOP_F32 ? launch_rmsnorm<float>(x, weight, y, rows, hidden, x_row_stride, y_row_stride, eps, s, true, rr)
+           : dtype == KOP_BF16
+               ? launch_rmsnorm<__nv_bfloat16>(x, weight, y, rows, hidden, x_row_stride, y_row_stride, eps, s, true, rr)
+               : launch_rmsnorm<__half>(x, weight, y, rows, hidden, x_row_stride, y_row_stride, eps, s, true, rr);
 }
 
 extern "C" kop_status_t kop_silu_mul(const void* gate_up, void* out, int64_t rows, int64_t inter,

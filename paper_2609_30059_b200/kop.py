@@ -66,6 +66,8 @@ def lib() -> C.CDLL:
     L.kop_ce_loss_rowwise_static_max_rows.restype = i64
     L.kop_ce_loss_rowwise_static_max_rows.argtypes = []
     L.kop_rmsnorm.argtypes = [vp, vp, vp, i64, i64, i64, i64, f32, i32, vp]
+    L.kop_residual_rmsnorm.argtypes = [vp] * 5 + [i64] * 6 + [f32, i32, vp]
+    L.kop_residual_rmsnorm.restype = i32
     L.kop_silu_mul.argtypes = [vp, vp, i64, i64, i64, i64, i32, vp]
     L.kop_residual_add.argtypes = [vp, vp, vp, i64, i64, i64, i64, i64, i32, vp]
     L.kop_ce_loss_rowwise_opts.argtypes = [vp] * 6 + [i64] * 3 + [C.c_int32, f32, vp, sz, i32, vp]
@@ -257,6 +259,21 @@ def kop_rmsnorm(x, weight, eps, out=None, stream=None):
     _check(lib().kop_rmsnorm(x.data_ptr(), _param(weight, "weight", hidden), out.data_ptr(), rows, hidden,
                              xs, ys, float(eps), _dtype_tag(x), _stream(stream)), "kop_rmsnorm")
     return out
+
+
+def kop_residual_rmsnorm(x, residual, weight, eps, h_out=None, out=None, stream=None):
+    """Returns (h, y): h = x + residual, y = rmsnorm(h)."""
+    rows, hidden, xs = _rows2d(x, "x")
+    _, _, rs = _rows2d(residual, "residual")
+    assert residual.shape == x.shape and residual.dtype == x.dtype
+    h_out = torch.empty_like(x) if h_out is None else h_out
+    out = torch.empty_like(x) if out is None else out
+    _, _, hs = _rows2d(h_out, "h_out")
+    _, _, ys = _rows2d(out, "out")
+    _check(lib().kop_residual_rmsnorm(x.data_ptr(), residual.data_ptr(), _param(weight, "weight", hidden), h_out.data_ptr(),
+                                      out.data_ptr(), rows, hidden, xs, rs, hs, ys, float(eps), _dtype_tag(x),
+                                      _stream(stream)), "kop_residual_rmsnorm")
+    return h_out, out
 
 
 def kop_silu_mul(gate_up, out=None, stream=None):

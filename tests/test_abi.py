@@ -147,6 +147,13 @@ def test_mlp_pieces_validation(L):
     assert L.kop_rmsnorm(P, None, R, 4, 64, 64, 64, 1e-6, 1, None) == NULLP
     assert L.kop_rmsnorm(P, Q, R, 4, 64, 32, 64, 1e-6, 1, None) == STRIDE
     assert L.kop_rmsnorm(P, Q, P + 2, 4, 64, 64, 64, 1e-6, 1, None) == ALIAS
+    H2, Y2 = 0x600000, 0x700000
+    assert L.kop_residual_rmsnorm(P, Q, R, H2, Y2, 0, 64, 64, 64, 64, 64, 1e-6, 1, None) == OK
+    assert L.kop_residual_rmsnorm(P, None, R, H2, Y2, 4, 64, 64, 64, 64, 64, 1e-6, 1, None) == NULLP
+    assert L.kop_residual_rmsnorm(P, Q, R, H2, Y2, 4, 64, 64, 64, 32, 64, 1e-6, 1, None) == STRIDE
+    assert L.kop_residual_rmsnorm(P, Q, R, H2, H2, 4, 64, 64, 64, 64, 64, 1e-6, 1, None) == ALIAS      # h is y
+    assert L.kop_residual_rmsnorm(P, Q, R, P + 2, Y2, 4, 64, 64, 64, 64, 64, 1e-6, 1, None) == ALIAS   # h overlaps x
+    assert L.kop_residual_rmsnorm(P, Q, R, P, Q, 4, 64, 64, 64, 64, 64, 1e-6, 1, None) not in (ALIAS, NULLP)   # in place
     assert L.kop_silu_mul(P, R, 0, 64, 128, 64, 1, None) == OK
     assert L.kop_silu_mul(P, R, 4, 64, 127, 64, 1, None) == STRIDE      # input rows hold 2*inter
     assert L.kop_silu_mul(P, P, 4, 64, 128, 64, 1, None) == ALIAS       # no in-place for SwiGLU

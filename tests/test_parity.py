@@ -516,6 +516,32 @@ def test_rmsnorm_parity(kop, rows, hidden, dtype, seed):
     out.check("rmsnorm")
 
 
+@pytest.mark.parametrize("rows,hidden,dtype", [(2048, 4096, BF16), (300, 4096, F32), (65, 512, torch.float16), (17, 16384, BF16),
+                                               (9, 20480, BF16), (33, 1001, F32), (5, 1, F32)])
+@pytest.mark.parametrize("seed", SEEDS)
+def test_residual_rmsnorm_parity(kop, rows, hidden, dtype, seed):
+    h, w, _, _ = synth.mlp_inputs(rows, hidden, 1, dtype, seed, "cuda")
+    _, d = synth.pair_inputs(rows, hidden, dtype, seed + 1, "cuda")
+    hg, yg = Guarded((rows, hidden), dtype), Guarded((rows, hidden), dtype)
+    kop.kop_residual_rmsnorm(h, d, w, 1e-6, h_out=hg.t, out=yg.t)
+    rh, ry = kopref.residual_rmsnorm(host(h), host(d), host(w), 1e-6, threads=None)
+    tol = tol_of(dtype)
+    assert_close(hg.t, rh, tol, "residual_rmsnorm h")
+    assert_close(yg.t, ry, tol, "residual_rmsnorm y")
+    if dtype == BF16:
+        assert_bf16_tight(yg.t, ry, "residual_rmsnorm y")
+    hg.check("h")
+    yg.check("y")
+    # h equals the stand-alone residual add bit for bit; the residual stream updated in place
+    assert torch.equal(hg.t, kop.kop_residual_add(h, d))
+    hi = h.clone()
+    _, yi = kop.kop_residual_rmsnorm(hi, d, w, 1e-6, h_out=hi)
+    assert torch.equal(hi, hg.t) and torch.equal(yi, yg.t)
+    with pytest.raises(kop.KopError) as ei:
+        kop.kop_residual_rmsnorm(h, d, w, 1e-6, h_out=hg.t, out=hg.t)          # the two outputs must differ
+    assert ei.value.status == 6
+
+
 SILU_SHAPES = [(512, 14336, BF16), (100, 14336, F32), (33, 1000, BF16), (17, 1001, F32),
                (64, 8, BF16), (5, 1, F32)]
 
