@@ -53,6 +53,7 @@ def test_all_entry_points_in_one_graph(kop):
         "row_scale": torch.empty_like(bm), "matvec": torch.empty(rows, device=dev), "red": torch.empty(rows, device=dev),
         "red_i": torch.empty(rows, dtype=torch.int32, device=dev), "lse": torch.empty(rows, device=dev),
         "act": torch.empty_like(x), "chain": torch.empty_like(x), "mlp": torch.empty_like(h),
+        "rr_h": torch.empty_like(lx), "rr_y": torch.empty_like(lx),
     }
 
     def run():
@@ -79,6 +80,7 @@ def test_all_entry_points_in_one_graph(kop):
         kop.kop_reduce_rows(x, "logsumexp", out=o["lse"])
         kop.kop_bias_act(x, bias, "mish", out=o["act"])
         kop.kop_epilogue_chain(x, bias, lx, 0.5, 2.0, -1.0, 1.0, "gelu_erf", out=o["chain"])
+        kop.kop_residual_rmsnorm(lx, lr, lg, 1e-6, h_out=o["rr_h"], out=o["rr_y"])
         kop.kop_rmsnorm_swiglu_residual(handle, h, w, W1, W2, 1e-6, out=o["mlp"], workspace=ws_mlp)
 
     try:
