@@ -780,3 +780,33 @@ int kopref_epilogue_chain(const void* x, const float* bias, const void* residual
         }
     return 0;
 }
+
+/* ---- LSTM cell, pointwise part (the gate arithmetic that follows the two preserved GEMMs of an LSTM step; the
+ * paper's level-3 table lists LSTM / GRU models) -------------------------------------------------------------
+ * gates[b, 0:H] = i, [H:2H] = f, [2H:3H] = g, [3H:4H] = o (pre-activations; gates2 and bias, when given, are
+ * added first: a = gates + gates2 + bias):
+ *   c_out = sigmoid(f) * c_prev + sigmoid(i) * tanh(g);   h_out = sigmoid(o) * tanh(c_out)
+ * h_out uses the unrounded c_out. */
+int kopref_lstm_cell(const void* gates, const void* gates2, const float* bias, const void* c_prev, double* h_out,
+        double* c_out, int64_t rows, int64_t hidden, int dtype, int threads)
+{
+    if (!gates || !c_prev || !h_out || !c_out || rows < 0 || hidden <= 0 || bad_dtype(dtype)) return -1;
+    int nt = pick_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t b = 0; b < rows; ++b)
+        for (int64_t j = 0; j < hidden; ++j) {
+            double a[4];
+            for (int k = 0; k < 4; ++k) {
+                int64_t idx = b * 4 * hidden + k * hidden + j;
+                a[k] = load_elem(gates, idx, dtype) + (gates2 ? load_elem(gates2, idx, dtype) : 0.0)
+                     + (bias ? (double)bias[k * hidden + j] : 0.0);
+            }
+            double ig = 1.0 / (1.0 + exp(-a[0])), fg = 1.0 / (1.0 + exp(-a[1])), gg = tanh(a[2]),
+                   og = 1.0 / (1.0 + exp(-a[3]));
+            double c = fg * load_elem(c_prev, b * hidden + j, dtype) + ig * gg;
+            c_out[b * hidden + j] = c;
+            h_out[b * hidden + j] = og * tanh(c);
+        }
+    return 0;
+}

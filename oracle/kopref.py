@@ -57,6 +57,7 @@ def lib() -> C.CDLL:
         _lib.kopref_act_value.argtypes = [dbl, C.c_int, dbl]
         _lib.kopref_softmax_opts.argtypes = [vp, vp, vp, i64, i64, i64, i64, dbl, C.c_int, i64, C.c_int, C.c_int]
         _lib.kopref_epilogue_chain.argtypes = [vp, vp, vp, vp] + [i64] * 5 + [dbl] * 4 + [C.c_int, dbl, C.c_int, C.c_int]
+        _lib.kopref_lstm_cell.argtypes = [vp] * 6 + [i64, i64, C.c_int, C.c_int]
         _lib.kopref_cumsum_rows.argtypes = [vp, vp, vp] + [i64] * 5 + [C.c_int] * 4
         _lib.kopref_matvec_bias.argtypes = [vp, vp, dbl, vp, i64, i64, i64, C.c_int, C.c_int]
     return _lib
@@ -406,6 +407,25 @@ def epilogue_chain(x, bias, residual, scale=1.0, residual_scale=1.0, lo=-np.inf,
                                        float(residual_scale), float(lo), float(hi), ACTS[act], float(alpha), dt, _nt(threads)),
            "epilogue_chain")
     return y
+
+
+def lstm_cell(gates, c_prev, gates2=None, bias=None, threads=1):
+    """Pointwise part of an LSTM step. gates (+ gates2 + bias): [rows, 4 * hidden] in the order i, f, g, o;
+    c_prev: [rows, hidden]. Returns (h_out, c_out)."""
+    ga, dt = as_data(gates)
+    ca, dt2 = as_data(c_prev)
+    rows, four_h = ga.shape
+    hidden = four_h // 4
+    assert dt == dt2 and four_h == 4 * hidden and ca.shape == (rows, hidden)
+    g2 = None
+    if gates2 is not None:
+        g2, dt3 = as_data(gates2)
+        assert dt3 == dt and g2.shape == ga.shape
+    b = as_param(bias)
+    h = np.empty((rows, hidden), dtype=np.float64)
+    c = np.empty((rows, hidden), dtype=np.float64)
+    _check(lib().kopref_lstm_cell(_p(ga), _p(g2), _p(b), _p(ca), _p(h), _p(c), rows, hidden, dt, _nt(threads)), "lstm_cell")
+    return h, c
 
 
 def cumsum_rows(x, mask=None, exclusive=False, reverse=False, threads=1) -> np.ndarray:

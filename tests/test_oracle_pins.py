@@ -983,3 +983,39 @@ def test_residual_rmsnorm_composition_against_torch():
     assert np.abs(yb - rounded_first).max() > 1e-4
     # zero residual: plain RMSNorm
     assert np.array_equal(kopref.residual_rmsnorm(x, torch.zeros_like(x), w, 1e-6)[1], kopref.rmsnorm(x, w, 1e-6))
+
+
+# --------------------------------------------------------------------------- LSTM cell (pointwise part)
+
+def test_lstm_cell_against_torch_lstmcell_and_closed_forms():
+    B, I, H = 5, 7, 6
+    cell = torch.nn.LSTMCell(I, H).double()
+    xin = torch.from_numpy(RNG.normal(0, 1, (B, I)))
+    h0 = torch.from_numpy(RNG.normal(0, 1, (B, H)))
+    c0 = torch.from_numpy(RNG.normal(0, 1, (B, H)))
+    with torch.no_grad():
+        h1, c1 = cell(xin, (h0, c0))                                   # the library routine fixes the gate order i, f, g, o
+        ig = xin @ cell.weight_ih.t()                                  # the two preserved GEMMs
+        hg = h0 @ cell.weight_hh.t()
+        bias = (cell.bias_ih + cell.bias_hh).float()
+    h, c = kopref.lstm_cell(ig, c0, gates2=hg, bias=bias)
+    b64 = bias.double()
+    href, cref = kopref.lstm_cell(ig + hg + b64, c0)                   # the same with the sum formed outside
+    np.testing.assert_allclose(h, href, rtol=0, atol=1e-15)
+    tol = 1e-7                                                         # the bias went through fp32
+    np.testing.assert_allclose(h, h1.numpy(), rtol=0, atol=tol)
+    np.testing.assert_allclose(c, c1.numpy(), rtol=0, atol=tol)
+    hx, cx = kopref.lstm_cell(ig + hg + (cell.bias_ih + cell.bias_hh).detach(), c0)
+    np.testing.assert_allclose(hx, h1.numpy(), rtol=0, atol=1e-14)
+    np.testing.assert_allclose(cx, c1.numpy(), rtol=0, atol=1e-14)
+    # closed forms: all-zero gates halve the cell state; saturated gates pass or block it
+    z = np.zeros((1, 8))
+    h, c = kopref.lstm_cell(z, np.array([[2.0, -4.0]]))
+    assert np.array_equal(c, [[1.0, -2.0]]) and h[0, 0] == pytest.approx(0.5 * math.tanh(1.0), rel=1e-15)
+    big = np.array([[-40.0, -40.0, 40.0, 40.0, 0.3, -0.7, 40.0, 40.0]])   # i closed, f open, o open, H = 2
+    h, c = kopref.lstm_cell(big, np.array([[0.25, -1.5]]))
+    np.testing.assert_allclose(c, [[0.25, -1.5]], rtol=1e-15)
+    np.testing.assert_allclose(h, np.tanh([[0.25, -1.5]]), rtol=1e-15)
+    big = np.array([[40.0, 40.0, -40.0, -40.0, 0.3, -0.7, 40.0, 40.0]])   # i open, f closed: c = tanh(g)
+    h, c = kopref.lstm_cell(big, np.array([[9.0, 9.0]]))
+    np.testing.assert_allclose(c, np.tanh([[0.3, -0.7]]), rtol=1e-15)
