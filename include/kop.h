@@ -410,6 +410,23 @@ kop_status_t kop_cumsum_rows(const void* x, const unsigned char* mask, void* y, 
                              int exclusive, int reverse, kop_dtype_t dtype, kop_stream_t stream);
 
 /*
+ * The pointwise part of one LSTM step (the LSTM models of the paper's level-3 table, L3-035 to L3-038, for
+ * which its compiler emitted no kernels and the recurrent layer stayed with the vendor library; here the
+ * two gate GEMMs stay with the vendor library and everything after them is one pass). With H = hidden and
+ *   a[i, :] = gates[i, :] + gates2[i, :] + bias          (gates2 and bias optional)
+ * split into four blocks of H columns in the order input i, forget f, candidate g, output o:
+ *   c_out = sigmoid(a_f) * c_prev + sigmoid(a_i) * tanh(a_g)
+ *   h_out = sigmoid(a_o) * tanh(c_out)                    (from c_out before it is rounded to `dtype`)
+ * gates, gates2: [rows, 4H] of `dtype`, contiguous (the outputs of x W_ih^T and h W_hh^T; pass one and NULL
+ * when a single GEMM produced their sum); bias: fp32 [4H] or NULL (b_ih + b_hh); c_prev, h_out, c_out:
+ * [rows, H] of `dtype`, contiguous. Arithmetic is fp32. c_out may be c_prev exactly (the state updated in
+ * place); otherwise h_out and c_out overlap no input and not each other. hidden <= 2^31 - 1.
+ */
+kop_status_t kop_lstm_cell(const void* gates, const void* gates2, const float* bias, const void* c_prev,
+                           void* h_out, void* c_out, int64_t rows, int64_t hidden, kop_dtype_t dtype,
+                           kop_stream_t stream);
+
+/*
  * Diagnostic for kop_groupnorm_act (no counterpart in the paper): its staged kernel waits for its bulk
  * copies with a bounded number of polls; a CTA whose wait runs out writes nothing, and counts itself here.
  * host_count: HOST pointer, receives the count for the current device since the library was loaded (always

@@ -92,6 +92,8 @@ def lib() -> C.CDLL:
     L.kop_epilogue_chain.restype = i32
     L.kop_cumsum_rows.argtypes = [vp, vp, vp] + [i64] * 5 + [i32, i32, i32, vp]
     L.kop_cumsum_rows.restype = i32
+    L.kop_lstm_cell.argtypes = [vp] * 6 + [i64, i64, i32, vp]
+    L.kop_lstm_cell.restype = i32
     L.kop_groupnorm_wait_timeouts.argtypes = [C.POINTER(C.c_uint)]
     L.kop_groupnorm_wait_timeouts.restype = i32
     L.kop_rmsnorm_swiglu_residual.argtypes = [vp] * 6 + [i64] * 3 + [f32, vp, sz, i32, vp]
@@ -472,6 +474,28 @@ def kop_cumsum_rows(x, mask=None, exclusive=False, reverse=False, out=None, stre
     _check(lib().kop_cumsum_rows(x.data_ptr(), mp, out.data_ptr(), rows, cols, xs, ms, ys, int(bool(exclusive)),
                                  int(bool(reverse)), _dtype_tag(x), _stream(stream)), "kop_cumsum_rows")
     return out
+
+
+def kop_lstm_cell(gates, c_prev, gates2=None, bias=None, h_out=None, c_out=None, stream=None):
+    """gates (and gates2): contiguous [rows, 4H]; c_prev: contiguous [rows, H]; bias: fp32 [4H].
+    Returns (h_out, c_out); pass c_out=c_prev to update the state in place."""
+    if gates.dim() != 2 or c_prev.dim() != 2 or not gates.is_contiguous() or not c_prev.is_contiguous():
+        raise ValueError("gates / c_prev: expected contiguous 2-D tensors")
+    rows, hidden = c_prev.shape
+    if gates.shape != (rows, 4 * hidden) or gates.dtype != c_prev.dtype:
+        raise ValueError("gates: expected [rows, 4 * hidden] of c_prev's dtype")
+    if gates2 is not None and (gates2.shape != gates.shape or gates2.dtype != gates.dtype or not gates2.is_contiguous()):
+        raise ValueError("gates2: expected a contiguous tensor like gates")
+    if bias is not None and (bias.dtype != torch.float32 or bias.shape != (4 * hidden,) or not bias.is_contiguous()):
+        raise ValueError("bias: expected contiguous fp32 [4 * hidden]")
+    h_out = torch.empty_like(c_prev) if h_out is None else h_out
+    c_out = torch.empty_like(c_prev) if c_out is None else c_out
+    for t in (h_out, c_out):
+        assert t.shape == c_prev.shape and t.dtype == c_prev.dtype and t.is_contiguous()
+    _check(lib().kop_lstm_cell(gates.data_ptr(), None if gates2 is None else gates2.data_ptr(),
+                               None if bias is None else bias.data_ptr(), c_prev.data_ptr(), h_out.data_ptr(),
+                               c_out.data_ptr(), rows, hidden, _dtype_tag(gates), _stream(stream)), "kop_lstm_cell")
+    return h_out, c_out
 
 
 def kop_groupnorm_wait_timeouts() -> int:

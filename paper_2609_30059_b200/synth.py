@@ -29,6 +29,8 @@ CONFIGS = {
     # BatchNorm + ReLU + 3x3 / stride-2 max pool on a 112 x 112 map with 64 channels (a CNN stem)
     "pool2d": dict(N=64, C=64, H=112, W=112, kernel=(3, 3), stride=(2, 2), padding=(1, 1), mode="max",
                    dtype=torch.float32),
+    # pointwise part of one LSTM step: batch 16384, hidden 1024 (shape ours)
+    "lstm_cell": dict(rows=16384, hidden=1024, dtype=torch.bfloat16),
     # row reductions (shape ours)
     "reduce": dict(rows=32768, cols=8192, dtype=torch.bfloat16),
 }
@@ -144,3 +146,15 @@ def cumsum_inputs(rows, cols, dtype=torch.float32, seed=0, device="cpu", keep=0.
     x = _normal((rows, cols), 0.0, 1.0, g, device).to(dtype)
     mask = (torch.rand((rows, cols), generator=g, device=device, dtype=torch.float32) < keep).to(torch.uint8)
     return x, mask
+
+
+def lstm_inputs(rows, hidden, dtype=torch.float32, seed=0, device="cpu"):
+    """gates, gates2 ~ N(0,1) [rows, 4 * hidden]; c_prev ~ N(0,1) [rows, hidden]; bias fp32 ~ N(0,0.1) with
+    +1 on the forget block (the usual initialisation)."""
+    g = _gen(seed, device)
+    gates = _normal((rows, 4 * hidden), 0.0, 1.0, g, device).to(dtype)
+    gates2 = _normal((rows, 4 * hidden), 0.0, 1.0, g, device).to(dtype)
+    c_prev = _normal((rows, hidden), 0.0, 1.0, g, device).to(dtype)
+    bias = _normal((4 * hidden,), 0.0, 0.1, g, device)
+    bias[hidden:2 * hidden] += 1.0
+    return gates, gates2, bias, c_prev

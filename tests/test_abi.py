@@ -223,6 +223,28 @@ def test_cumsum_validation(L):
     assert f(P, Q + 16, Q, 4, 64, 64, 64, 64, 0, 0, 0, None) == ALIAS          # mask overlaps y
 
 
+def test_lstm_cell_validation(L):
+    f = L.kop_lstm_cell
+    G, G2, B, CP, H, CO = 0x100000, 0x200000, 0x300000, 0x400000, 0x500000, 0x600000
+    assert f(G, G2, B, CP, H, CO, 0, 64, 0, None) == OK
+    assert f(None, G2, B, CP, H, CO, 4, 64, 0, None) == NULLP
+    assert f(G, None, None, None, H, CO, 4, 64, 0, None) == NULLP
+    assert f(G, None, None, CP, None, CO, 4, 64, 0, None) == NULLP
+    assert f(G, None, None, CP, H, None, 4, 64, 0, None) == NULLP
+    assert f(G, None, None, CP, H, CO, 4, 0, 0, None) == SHAPE
+    assert f(G, None, None, CP, H, CO, -1, 64, 0, None) == SHAPE
+    assert f(G, None, None, CP, H, CO, 4, 2 ** 45, 0, None) == SHAPE           # 4 * hidden * rows overflows
+    assert f(G, None, None, CP, H, CO, 4, 64, 3, None) == DTYPE
+    assert f(G + 2, None, None, CP, H, CO, 4, 64, 0, None) == MISAL
+    assert f(G, G2 + 1, None, CP, H, CO, 4, 64, 1, None) == MISAL
+    assert f(G, None, B + 2, CP, H, CO, 4, 64, 1, None) == MISAL               # bias is fp32 whatever the data
+    assert f(G, None, None, CP, H, CP + 16, 4, 64, 0, None) == ALIAS           # c_out overlaps c_prev partly
+    assert f(G, None, None, CP, CP, CO, 4, 64, 0, None) == ALIAS               # h_out may not be c_prev
+    assert f(G, None, None, CP, H, H, 4, 64, 0, None) == ALIAS
+    assert f(G, None, None, CP, G + 4 * 4 * 64 * 3, CO, 4, 64, 0, None) == ALIAS   # h_out inside gates
+    assert f(G, G2, None, CP, H, G2, 4, 64, 0, None) == ALIAS
+
+
 def test_pool2d_validation(L):
     f = L.kop_affine_relu_pool2d
     S, T = 0x600000, 0x610000

@@ -134,6 +134,14 @@ def test_fuzz_row_kernels(kop):
         xa, ba = synth.softmax_inputs(rows, cols, dtype, seed, "cuda")
         assert_close(kop.kop_bias_act(strided(rng, xa), ba, act, alpha=0.3), kopref.bias_act(host(xa), host(ba), act, alpha=0.3),
                      tol, f"bias_act {act} " + what)
+        # LSTM gate arithmetic (cols = hidden units, any length: vector and element kernels)
+        hid = max(1, cols // 4)
+        tg, tg2, tb, tc = synth.lstm_inputs(rows, hid, dtype, seed, "cuda")
+        two, wb = bool(rng.integers(0, 2)), bool(rng.integers(0, 2))
+        gh, gc = kop.kop_lstm_cell(tg, tc, tg2 if two else None, tb if wb else None)
+        rh, rc = kopref.lstm_cell(host(tg), host(tc), host(tg2) if two else None, host(tb) if wb else None)
+        assert_close(gh, rh, tol, "lstm h " + what)
+        assert_close(gc, rc, tol, "lstm c " + what)
         # running sums
         xc, mask = synth.cumsum_inputs(rows, cols, dtype, seed, "cuda")
         ex, rv, um = bool(rng.integers(0, 2)), bool(rng.integers(0, 2)), bool(rng.integers(0, 2))
