@@ -810,3 +810,32 @@ int kopref_lstm_cell(const void* gates, const void* gates2, const float* bias, c
         }
     return 0;
 }
+
+/* ---- GRU cell, pointwise part (what follows the two preserved GEMMs gi = x W_ih^T and gh = h W_hh^T of a GRU
+ * step; the paper's level-3 table lists GRU models) ----------------------------------------------------------
+ * gi, gh: [rows, 3H], blocks r (reset), z (update), n (candidate); bias_i, bias_h: [3H] or NULL, added to gi
+ * and gh respectively (they cannot be merged: the candidate's hidden part is gated before the sum):
+ *   r = sigmoid(gi_r + gh_r);  z = sigmoid(gi_z + gh_z);  n = tanh(gi_n + r * gh_n);
+ *   h_out = (1 - z) * n + z * h_prev */
+int kopref_gru_cell(const void* gi, const void* gh, const float* bias_i, const float* bias_h, const void* h_prev,
+        double* h_out, int64_t rows, int64_t hidden, int dtype, int threads)
+{
+    if (!gi || !gh || !h_prev || !h_out || rows < 0 || hidden <= 0 || bad_dtype(dtype)) return -1;
+    int nt = pick_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t b = 0; b < rows; ++b)
+        for (int64_t j = 0; j < hidden; ++j) {
+            double xi[3], xh[3];
+            for (int k = 0; k < 3; ++k) {
+                int64_t idx = b * 3 * hidden + k * hidden + j;
+                xi[k] = load_elem(gi, idx, dtype) + (bias_i ? (double)bias_i[k * hidden + j] : 0.0);
+                xh[k] = load_elem(gh, idx, dtype) + (bias_h ? (double)bias_h[k * hidden + j] : 0.0);
+            }
+            double r = 1.0 / (1.0 + exp(-(xi[0] + xh[0])));
+            double z = 1.0 / (1.0 + exp(-(xi[1] + xh[1])));
+            double n = tanh(xi[2] + r * xh[2]);
+            h_out[b * hidden + j] = (1.0 - z) * n + z * load_elem(h_prev, b * hidden + j, dtype);
+        }
+    return 0;
+}

@@ -58,6 +58,7 @@ def lib() -> C.CDLL:
         _lib.kopref_softmax_opts.argtypes = [vp, vp, vp, i64, i64, i64, i64, dbl, C.c_int, i64, C.c_int, C.c_int]
         _lib.kopref_epilogue_chain.argtypes = [vp, vp, vp, vp] + [i64] * 5 + [dbl] * 4 + [C.c_int, dbl, C.c_int, C.c_int]
         _lib.kopref_lstm_cell.argtypes = [vp] * 6 + [i64, i64, C.c_int, C.c_int]
+        _lib.kopref_gru_cell.argtypes = [vp] * 6 + [i64, i64, C.c_int, C.c_int]
         _lib.kopref_cumsum_rows.argtypes = [vp, vp, vp] + [i64] * 5 + [C.c_int] * 4
         _lib.kopref_matvec_bias.argtypes = [vp, vp, dbl, vp, i64, i64, i64, C.c_int, C.c_int]
     return _lib
@@ -426,6 +427,21 @@ def lstm_cell(gates, c_prev, gates2=None, bias=None, threads=1):
     c = np.empty((rows, hidden), dtype=np.float64)
     _check(lib().kopref_lstm_cell(_p(ga), _p(g2), _p(b), _p(ca), _p(h), _p(c), rows, hidden, dt, _nt(threads)), "lstm_cell")
     return h, c
+
+
+def gru_cell(gi, gh, h_prev, bias_i=None, bias_h=None, threads=1) -> np.ndarray:
+    """Pointwise part of a GRU step. gi, gh: [rows, 3 * hidden] in the order r, z, n; h_prev: [rows, hidden];
+    bias_i / bias_h are added to gi / gh. Returns h_out."""
+    ia, dt = as_data(gi)
+    ha, dt2 = as_data(gh)
+    pa, dt3 = as_data(h_prev)
+    rows, three_h = ia.shape
+    hidden = three_h // 3
+    assert dt == dt2 == dt3 and three_h == 3 * hidden and ha.shape == ia.shape and pa.shape == (rows, hidden)
+    bi, bh = as_param(bias_i), as_param(bias_h)
+    out = np.empty((rows, hidden), dtype=np.float64)
+    _check(lib().kopref_gru_cell(_p(ia), _p(ha), _p(bi), _p(bh), _p(pa), _p(out), rows, hidden, dt, _nt(threads)), "gru_cell")
+    return out
 
 
 def cumsum_rows(x, mask=None, exclusive=False, reverse=False, threads=1) -> np.ndarray:

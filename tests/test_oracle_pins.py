@@ -1019,3 +1019,39 @@ def test_lstm_cell_against_torch_lstmcell_and_closed_forms():
     big = np.array([[40.0, 40.0, -40.0, -40.0, 0.3, -0.7, 40.0, 40.0]])   # i open, f closed: c = tanh(g)
     h, c = kopref.lstm_cell(big, np.array([[9.0, 9.0]]))
     np.testing.assert_allclose(c, np.tanh([[0.3, -0.7]]), rtol=1e-15)
+
+
+def test_gru_cell_against_torch_grucell_and_closed_forms():
+    B, I, H = 5, 7, 6
+    cell = torch.nn.GRUCell(I, H).double()
+    xin = torch.from_numpy(RNG.normal(0, 1, (B, I)))
+    h0 = torch.from_numpy(RNG.normal(0, 1, (B, H)))
+    with torch.no_grad():
+        h1 = cell(xin, h0)                         # the library routine fixes the block order r, z, n and the n-gate form
+        gi = xin @ cell.weight_ih.t()              # the two preserved GEMMs
+        gh = h0 @ cell.weight_hh.t()
+        bi, bh = cell.bias_ih.detach(), cell.bias_hh.detach()
+    got = kopref.gru_cell(gi + bi, gh + bh, h0)                        # biases added outside, in float64
+    np.testing.assert_allclose(got, h1.numpy(), rtol=0, atol=1e-14)
+    got32 = kopref.gru_cell(gi, gh, h0, bias_i=bi.float(), bias_h=bh.float())
+    np.testing.assert_allclose(got32, h1.numpy(), rtol=0, atol=1e-6)   # the biases went through fp32
+    same = kopref.gru_cell(gi + bi.float().double(), gh + bh.float().double(), h0)
+    np.testing.assert_allclose(got32, same, rtol=0, atol=1e-15)
+    # the hidden bias of the candidate sits inside the reset gate: moving it to the input side changes the result
+    moved = kopref.gru_cell(gi + bi + torch.cat([torch.zeros(2 * H, dtype=torch.float64), bh[2 * H:]]),
+                            gh + torch.cat([bh[:2 * H], torch.zeros(H, dtype=torch.float64)]), h0)
+    assert np.abs(moved - h1.numpy()).max() > 1e-3
+    # closed forms (H = 2): zero gates average tanh(0) = 0 and h; z saturated keeps h; z closed and r closed give tanh(gi_n)
+    z6 = np.zeros((1, 6))
+    assert np.array_equal(kopref.gru_cell(z6, z6, np.array([[2.0, -4.0]])), [[1.0, -2.0]])
+    keep = np.array([[0.0, 0.0, 40.0, 40.0, 0.3, -0.7]])
+    np.testing.assert_allclose(kopref.gru_cell(keep, z6, np.array([[0.25, -1.5]])), [[0.25, -1.5]], rtol=1e-15)
+    gi_c = np.array([[-40.0, -40.0, -40.0, -40.0, 0.3, -0.7]])         # r = 0, z = 0
+    gh_c = np.array([[0.0, 0.0, 0.0, 0.0, 5.0, 5.0]])                  # blocked by r
+    np.testing.assert_allclose(kopref.gru_cell(gi_c, gh_c, np.array([[9.0, 9.0]])), np.tanh([[0.3, -0.7]]), rtol=1e-12)
+    gi_o = np.array([[40.0, 40.0, -40.0, -40.0, 0.3, -0.7]])           # r = 1, z = 0: n = tanh(gi_n + gh_n)
+    np.testing.assert_allclose(kopref.gru_cell(gi_o, gh_c, np.array([[9.0, 9.0]])), np.tanh([[5.3, 4.3]]), rtol=1e-12)
+    # 16-bit inputs are widened exactly
+    g16 = torch.from_numpy(RNG.normal(0, 1, (3, 12))).to(torch.bfloat16)
+    h16 = torch.from_numpy(RNG.normal(0, 1, (3, 4))).to(torch.bfloat16)
+    np.testing.assert_array_equal(kopref.gru_cell(g16, g16, h16), kopref.gru_cell(g16.double(), g16.double(), h16.double()))
