@@ -107,6 +107,8 @@ def segment_bytes():
     out["residual_rmsnorm"] = dict(bytes=4 * m["rows"] * m["hidden"] * 2 + m["hidden"] * 4, elems=m["rows"] * m["hidden"])
     t = c["lstm_cell"]
     out["lstm_cell"] = dict(bytes=(2 * 4 + 3) * t["rows"] * t["hidden"] * 2 + 4 * t["hidden"] * 4, elems=t["rows"] * t["hidden"])
+    t = c["gru_cell"]
+    out["gru_cell"] = dict(bytes=(2 * 3 + 2) * t["rows"] * t["hidden"] * 2 + 6 * t["hidden"] * 4, elems=t["rows"] * t["hidden"])
     u = c["cumsum"]
     out["cumsum"] = dict(bytes=2 * u["rows"] * u["cols"] * 4, elems=u["rows"] * u["cols"])
     return out
@@ -252,7 +254,7 @@ class Workload:
 
     ORDER = ["softmax_small", "softmax_large", "layernorm", "bn_pool", "ce_loss", "rmsnorm", "silu_mul", "residual_add"]
     # Beyond the benchmark configs (not part of `value`): the two kernels the paper's case studies print.
-    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc", "pool2d", "reduce_max", "reduce_logsumexp", "bias_gelu", "residual_rmsnorm", "lstm_cell"]
+    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc", "pool2d", "reduce_max", "reduce_logsumexp", "bias_gelu", "residual_rmsnorm", "lstm_cell", "gru_cell"]
 
     def __init__(self, kop, device, seed, only=None, rows_div=1):
         """only: build just these segments (None = all, plus the MLP segment); rows_div cuts the row
@@ -336,6 +338,10 @@ class Workload:
             self.tg, self.tg2, self.tb, self.tc = synth.lstm_inputs(cut(t["rows"]), t["hidden"], t["dtype"], seed, dev)
             self.th = torch.empty_like(self.tc)
             self.tco = torch.empty_like(self.tc)
+        if "gru_cell" in want:
+            t = c["gru_cell"]
+            self.ui, self.uh, self.ubi, self.ubh, self.up = synth.gru_inputs(cut(t["rows"]), t["hidden"], t["dtype"], seed, dev)
+            self.uo = torch.empty_like(self.up)
         if "cumsum" in want:
             u = c["cumsum"]
             self.ux, _ = synth.cumsum_inputs(cut(u["rows"]), u["cols"], u["dtype"], seed, dev)
@@ -420,6 +426,8 @@ class Workload:
             k.kop_residual_rmsnorm(self.h, self.d, self.rw, self.eps, h_out=self.res, out=self.n)
         elif name == "lstm_cell":                # gate sums, activations and state update, bf16 [16384, 4 x 1024]
             k.kop_lstm_cell(self.tg, self.tc, self.tg2, self.tb, h_out=self.th, c_out=self.tco)
+        elif name == "gru_cell":                 # gate sums, activations and state update, bf16 [16384, 3 x 1024]
+            k.kop_gru_cell(self.ui, self.uh, self.up, self.ubi, self.ubh, h_out=self.uo)
         elif name == "cumsum":                   # inclusive running sum along rows, fp32 [32768, 4096]
             k.kop_cumsum_rows(self.ux, out=self.uy)
         else:

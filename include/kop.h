@@ -427,6 +427,22 @@ kop_status_t kop_lstm_cell(const void* gates, const void* gates2, const float* b
                            kop_stream_t stream);
 
 /*
+ * The pointwise part of one GRU step (the GRU models of the paper's level-3 table, L3-039 to L3-042, which
+ * its compiler also left to the vendor library's recurrent layer). With gi = x W_ih^T and gh = h W_hh^T
+ * from the two preserved GEMMs, each split into three blocks of H columns in the order reset r, update z,
+ * candidate n, and a = gi + bias_i, b = gh + bias_h:
+ *   r = sigmoid(a_r + b_r);  z = sigmoid(a_z + b_z);  n = tanh(a_n + r * b_n)
+ *   h_out = (1 - z) * n + z * h_prev
+ * gi, gh: [rows, 3H] of `dtype`, contiguous; bias_i, bias_h: fp32 [3H] or NULL, independently (they are
+ * separate because the candidate's hidden part is gated before the sum); h_prev, h_out: [rows, H] of
+ * `dtype`, contiguous. Arithmetic is fp32. h_out may be h_prev exactly (the state updated in place);
+ * otherwise it overlaps no input. hidden <= 2^31 - 1.
+ */
+kop_status_t kop_gru_cell(const void* gi, const void* gh, const float* bias_i, const float* bias_h,
+                          const void* h_prev, void* h_out, int64_t rows, int64_t hidden, kop_dtype_t dtype,
+                          kop_stream_t stream);
+
+/*
  * Diagnostic for kop_groupnorm_act (no counterpart in the paper): its staged kernel waits for its bulk
  * copies with a bounded number of polls; a CTA whose wait runs out writes nothing, and counts itself here.
  * host_count: HOST pointer, receives the count for the current device since the library was loaded (always

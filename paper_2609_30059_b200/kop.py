@@ -94,6 +94,8 @@ def lib() -> C.CDLL:
     L.kop_cumsum_rows.restype = i32
     L.kop_lstm_cell.argtypes = [vp] * 6 + [i64, i64, i32, vp]
     L.kop_lstm_cell.restype = i32
+    L.kop_gru_cell.argtypes = [vp] * 6 + [i64, i64, i32, vp]
+    L.kop_gru_cell.restype = i32
     L.kop_groupnorm_wait_timeouts.argtypes = [C.POINTER(C.c_uint)]
     L.kop_groupnorm_wait_timeouts.restype = i32
     L.kop_rmsnorm_swiglu_residual.argtypes = [vp] * 6 + [i64] * 3 + [f32, vp, sz, i32, vp]
@@ -496,6 +498,27 @@ def kop_lstm_cell(gates, c_prev, gates2=None, bias=None, h_out=None, c_out=None,
                                None if bias is None else bias.data_ptr(), c_prev.data_ptr(), h_out.data_ptr(),
                                c_out.data_ptr(), rows, hidden, _dtype_tag(gates), _stream(stream)), "kop_lstm_cell")
     return h_out, c_out
+
+
+def kop_gru_cell(gi, gh, h_prev, bias_i=None, bias_h=None, h_out=None, stream=None):
+    """gi, gh: contiguous [rows, 3H] (blocks r, z, n); h_prev: contiguous [rows, H]; biases fp32 [3H].
+    Returns h_out; pass h_out=h_prev to update the state in place."""
+    if gi.dim() != 2 or h_prev.dim() != 2 or not gi.is_contiguous() or not h_prev.is_contiguous():
+        raise ValueError("gi / h_prev: expected contiguous 2-D tensors")
+    rows, hidden = h_prev.shape
+    if gi.shape != (rows, 3 * hidden) or gi.dtype != h_prev.dtype:
+        raise ValueError("gi: expected [rows, 3 * hidden] of h_prev's dtype")
+    if gh.shape != gi.shape or gh.dtype != gi.dtype or not gh.is_contiguous():
+        raise ValueError("gh: expected a contiguous tensor like gi")
+    for b in (bias_i, bias_h):
+        if b is not None and (b.dtype != torch.float32 or b.shape != (3 * hidden,) or not b.is_contiguous()):
+            raise ValueError("bias: expected contiguous fp32 [3 * hidden]")
+    h_out = torch.empty_like(h_prev) if h_out is None else h_out
+    assert h_out.shape == h_prev.shape and h_out.dtype == h_prev.dtype and h_out.is_contiguous()
+    _check(lib().kop_gru_cell(gi.data_ptr(), gh.data_ptr(), None if bias_i is None else bias_i.data_ptr(),
+                              None if bias_h is None else bias_h.data_ptr(), h_prev.data_ptr(), h_out.data_ptr(),
+                              rows, hidden, _dtype_tag(gi), _stream(stream)), "kop_gru_cell")
+    return h_out
 
 
 def kop_groupnorm_wait_timeouts() -> int:

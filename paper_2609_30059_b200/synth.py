@@ -31,6 +31,7 @@ CONFIGS = {
                    dtype=torch.float32),
     # pointwise part of one LSTM step: batch 16384, hidden 1024 (shape ours)
     "lstm_cell": dict(rows=16384, hidden=1024, dtype=torch.bfloat16),
+    "gru_cell": dict(rows=16384, hidden=1024, dtype=torch.bfloat16),
     # row reductions (shape ours)
     "reduce": dict(rows=32768, cols=8192, dtype=torch.bfloat16),
 }
@@ -158,3 +159,15 @@ def lstm_inputs(rows, hidden, dtype=torch.float32, seed=0, device="cpu"):
     bias = _normal((4 * hidden,), 0.0, 0.1, g, device)
     bias[hidden:2 * hidden] += 1.0
     return gates, gates2, bias, c_prev
+
+
+def gru_inputs(rows, hidden, dtype=torch.float32, seed=0, device="cpu"):
+    """gi, gh ~ N(0,1) [rows, 3 * hidden]; h_prev ~ U(-1,1) [rows, hidden] (a hidden state is a convex mix of
+    tanh values); bias_i, bias_h fp32 ~ N(0,0.1)."""
+    g = _gen(seed, device)
+    gi = _normal((rows, 3 * hidden), 0.0, 1.0, g, device).to(dtype)
+    gh = _normal((rows, 3 * hidden), 0.0, 1.0, g, device).to(dtype)
+    h_prev = _uniform((rows, hidden), -1.0, 1.0, g, device).to(dtype)
+    bias_i = _normal((3 * hidden,), 0.0, 0.1, g, device)
+    bias_h = _normal((3 * hidden,), 0.0, 0.1, g, device)
+    return gi, gh, bias_i, bias_h, h_prev

@@ -245,6 +245,25 @@ def test_lstm_cell_validation(L):
     assert f(G, G2, None, CP, H, G2, 4, 64, 0, None) == ALIAS
 
 
+def test_gru_cell_validation(L):
+    f = L.kop_gru_cell
+    GI, GH, BI, BH, HP, HO = 0x100000, 0x200000, 0x300000, 0x310000, 0x400000, 0x500000
+    assert f(GI, GH, BI, BH, HP, HO, 0, 64, 0, None) == OK
+    assert f(None, GH, BI, BH, HP, HO, 4, 64, 0, None) == NULLP
+    assert f(GI, None, None, None, HP, HO, 4, 64, 0, None) == NULLP
+    assert f(GI, GH, None, None, None, HO, 4, 64, 0, None) == NULLP
+    assert f(GI, GH, None, None, HP, None, 4, 64, 0, None) == NULLP
+    assert f(GI, GH, None, None, HP, HO, 4, 0, 0, None) == SHAPE
+    assert f(GI, GH, None, None, HP, HO, -1, 64, 0, None) == SHAPE
+    assert f(GI, GH, None, None, HP, HO, 4, 2 ** 45, 0, None) == SHAPE
+    assert f(GI, GH, None, None, HP, HO, 4, 64, 3, None) == DTYPE
+    assert f(GI + 1, GH, None, None, HP, HO, 4, 64, 2, None) == MISAL
+    assert f(GI, GH, None, BH + 2, HP, HO, 4, 64, 1, None) == MISAL
+    assert f(GI, GH, None, None, HP, HP + 16, 4, 64, 0, None) == ALIAS         # h_out overlaps h_prev partly
+    assert f(GI, GH, None, None, HP, GH + 64, 4, 64, 0, None) == ALIAS         # h_out inside gh
+    assert f(GI, GH, None, None, HP, GI, 4, 64, 0, None) == ALIAS
+
+
 def test_pool2d_validation(L):
     f = L.kop_affine_relu_pool2d
     S, T = 0x600000, 0x610000

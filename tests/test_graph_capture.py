@@ -35,6 +35,7 @@ def test_all_entry_points_in_one_graph(kop):
     mx, mw, mb = synth.matvec_inputs(rows, cols, BF16, 9, dev)
     h, w, W1, W2 = synth.mlp_inputs(64, 256, 512, BF16, 10, dev)
     tg, tg2, tb, tc = synth.lstm_inputs(rows, 96, BF16, 11, dev)
+    ui, uh, ubi, ubh, up = synth.gru_inputs(rows, 96, BF16, 12, dev)
     handle = kop.MlpHandle()
     ws_ce = torch.empty(max(16, kop.kop_ce_loss_rowwise_workspace_bytes(rows, cols, kop.KOP_BF16)), dtype=torch.uint8, device=dev)
     ws_mlp = torch.empty(kop.kop_rmsnorm_swiglu_residual_workspace_bytes(64, 256, 512, kop.KOP_BF16), dtype=torch.uint8, device=dev)
@@ -55,6 +56,7 @@ def test_all_entry_points_in_one_graph(kop):
         "red_i": torch.empty(rows, dtype=torch.int32, device=dev), "lse": torch.empty(rows, device=dev),
         "act": torch.empty_like(x), "chain": torch.empty_like(x), "mlp": torch.empty_like(h),
         "rr_h": torch.empty_like(lx), "rr_y": torch.empty_like(lx), "lstm_h": torch.empty_like(tc), "lstm_c": torch.empty_like(tc),
+        "gru_h": torch.empty_like(up),
     }
 
     def run():
@@ -83,6 +85,7 @@ def test_all_entry_points_in_one_graph(kop):
         kop.kop_epilogue_chain(x, bias, lx, 0.5, 2.0, -1.0, 1.0, "gelu_erf", out=o["chain"])
         kop.kop_residual_rmsnorm(lx, lr, lg, 1e-6, h_out=o["rr_h"], out=o["rr_y"])
         kop.kop_lstm_cell(tg, tc, tg2, tb, h_out=o["lstm_h"], c_out=o["lstm_c"])
+        kop.kop_gru_cell(ui, uh, up, ubi, ubh, h_out=o["gru_h"])
         kop.kop_rmsnorm_swiglu_residual(handle, h, w, W1, W2, 1e-6, out=o["mlp"], workspace=ws_mlp)
 
     try:

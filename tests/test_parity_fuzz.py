@@ -142,6 +142,11 @@ def test_fuzz_row_kernels(kop):
         rh, rc = kopref.lstm_cell(host(tg), host(tc), host(tg2) if two else None, host(tb) if wb else None)
         assert_close(gh, rh, tol, "lstm h " + what)
         assert_close(gc, rc, tol, "lstm c " + what)
+        ui, uh, ubi, ubh, up = synth.gru_inputs(rows, hid, dtype, seed, "cuda")
+        wi, wh = bool(rng.integers(0, 2)), bool(rng.integers(0, 2))
+        assert_close(kop.kop_gru_cell(ui, uh, up, ubi if wi else None, ubh if wh else None),
+                     kopref.gru_cell(host(ui), host(uh), host(up), host(ubi) if wi else None, host(ubh) if wh else None),
+                     tol, "gru " + what)
         # running sums
         xc, mask = synth.cumsum_inputs(rows, cols, dtype, seed, "cuda")
         ex, rv, um = bool(rng.integers(0, 2)), bool(rng.integers(0, 2)), bool(rng.integers(0, 2))
