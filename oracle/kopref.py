@@ -100,13 +100,18 @@ def as_data(a):
 
 
 def as_param(a):
-    """fp32 parameter vector as a contiguous numpy array (None stays None)."""
+    """Parameter vector as a contiguous fp32 numpy array (None stays None). fp32 input is taken as is; a
+    bf16 / fp16 torch tensor (parameters stored in the data type) is widened to fp32, which is exact: every
+    value of either 16-bit format is an fp32 value."""
     if a is None:
         return None
     if hasattr(a, "detach"):
-        a = a.detach().cpu().numpy()
+        a = a.detach().cpu()
+        if str(a.dtype) in ("torch.bfloat16", "torch.float16"):
+            a = a.float()
+        a = a.numpy()
     a = np.ascontiguousarray(a)
-    assert a.dtype == np.float32, "parameter vectors are fp32"
+    assert a.dtype == np.float32, "parameter vectors are fp32, or 16-bit torch tensors"
     return a
 
 

@@ -1055,3 +1055,33 @@ def test_gru_cell_against_torch_grucell_and_closed_forms():
     g16 = torch.from_numpy(RNG.normal(0, 1, (3, 12))).to(torch.bfloat16)
     h16 = torch.from_numpy(RNG.normal(0, 1, (3, 4))).to(torch.bfloat16)
     np.testing.assert_array_equal(kopref.gru_cell(g16, g16, h16), kopref.gru_cell(g16.double(), g16.double(), h16.double()))
+
+
+def test_16_bit_parameters_widen_exactly_and_match_the_float64_library_norms():
+    """Parameters stored in bf16 / fp16: the oracle widens them to fp32 before use. Every one of the 65,536 bit
+    patterns of each format must come out as the value the format defines (checked against the oracle's own
+    bit-field decoder for data tensors, a separate implementation), and LayerNorm / RMSNorm with such
+    parameters must equal the float64 library routine given the same parameters widened by torch."""
+    bits = torch.arange(65536, dtype=torch.int32).to(torch.int16)
+    for tdt in (torch.bfloat16, torch.float16):
+        t = bits.view(tdt)
+        with np.errstate(invalid="ignore"):                       # signalling NaN patterns
+            via_param = kopref.as_param(t).astype(np.float64)
+        decoded = kopref.residual_add(t.reshape(1, -1), torch.zeros((1, 65536), dtype=tdt))[0]   # the C decoder, + 0
+        ref = t.double().numpy()
+        ok = ~np.isnan(ref)
+        assert np.array_equal(via_param[ok], ref[ok]) and np.array_equal(np.isnan(via_param), np.isnan(ref))
+        assert np.array_equal(via_param[ok], decoded[ok]) and np.array_equal(np.isnan(via_param), np.isnan(decoded))
+    H = 96
+    x = torch.from_numpy(RNG.normal(0, 1, (7, H))).to(torch.bfloat16)
+    g16 = torch.from_numpy(RNG.normal(1, 0.1, H)).to(torch.bfloat16)
+    b16 = torch.from_numpy(RNG.normal(0, 0.1, H)).to(torch.bfloat16)
+    y, _, _ = kopref.residual_layernorm(x, None, g16, b16, 1e-5)
+    ref = torch.nn.functional.layer_norm(x.double(), (H,), g16.double(), b16.double(), 1e-5).numpy()
+    np.testing.assert_allclose(y, ref, rtol=0, atol=1e-13)
+    yr = kopref.rmsnorm(x, g16, 1e-6)
+    refr = torch.nn.functional.rms_norm(x.double(), (H,), g16.double(), 1e-6).numpy()
+    np.testing.assert_allclose(yr, refr, rtol=0, atol=1e-13)
+    # rounding the parameters to bf16 is visible: the fp32 originals give a different result
+    g32 = torch.from_numpy(RNG.normal(1, 0.1, H)).float()
+    assert np.abs(kopref.rmsnorm(x, g32, 1e-6) - kopref.rmsnorm(x, g32.to(torch.bfloat16), 1e-6)).max() > 1e-4
