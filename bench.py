@@ -88,6 +88,8 @@ def segment_bytes():
     out["matvec_bias"] = dict(bytes=v["rows"] * v["k"] * 2 + v["k"] * 4 + v["rows"] * 4, elems=v["rows"] * v["k"])
     out["residual_layernorm"] = dict(bytes=3 * n["rows"] * n["hidden"] * 2 + 2 * n["hidden"] * 4 + 2 * n["rows"] * 4,
                                      elems=n["rows"] * n["hidden"])
+    out["layernorm_params16"] = dict(bytes=3 * n["rows"] * n["hidden"] * 2 + 3 * n["hidden"] * 2 + 2 * n["rows"] * 4,
+                                     elems=n["rows"] * n["hidden"])
     out["silu_mul_interleaved"] = dict(out["silu_mul"])
     kept = z["rows"] - (z["rows"] + 4) // 5            # every fifth row is ignored and never read
     out["ce_loss_opts"] = dict(bytes=kept * z["vocab"] * 2 + 2 * z["rows"] * 4 + 8, elems=kept * z["vocab"])
@@ -254,7 +256,7 @@ class Workload:
 
     ORDER = ["softmax_small", "softmax_large", "layernorm", "bn_pool", "ce_loss", "rmsnorm", "silu_mul", "residual_add"]
     # Beyond the benchmark configs (not part of `value`): the two kernels the paper's case studies print.
-    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc", "pool2d", "reduce_max", "reduce_logsumexp", "bias_gelu", "residual_rmsnorm", "lstm_cell", "gru_cell"]
+    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "layernorm_params16", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc", "pool2d", "reduce_max", "reduce_logsumexp", "bias_gelu", "residual_rmsnorm", "lstm_cell", "gru_cell"]
 
     def __init__(self, kop, device, seed, only=None, rows_div=1):
         """only: build just these segments (None = all, plus the MLP segment); rows_div cuts the row
@@ -274,12 +276,13 @@ class Workload:
             L = c["softmax_large"]
             self.lx, self.lb = synth.softmax_inputs(cut(L["rows"]), L["cols"], L["dtype"], seed, dev)
             self.ly = torch.empty_like(self.lx)
-        if "layernorm" in want:
+        if want & {"layernorm", "residual_layernorm", "layernorm_params16"}:
             n = c["layernorm"]
             self.nx, self.nr, self.nb, self.ng, self.nbe = synth.layernorm_inputs(cut(n["rows"]), n["hidden"], n["dtype"], seed, dev)
             self.ny = torch.empty_like(self.nx)
             self.nmean = torch.empty(self.nx.shape[0], dtype=torch.float32, device=dev)
             self.nrstd = torch.empty(self.nx.shape[0], dtype=torch.float32, device=dev)
+            self.np16 = [t.to(n["dtype"]) for t in (self.nb, self.ng, self.nbe)]
         if "bn_pool" in want:
             b = c["bn_pool"]
             self.bx, self.bscale, self.bshift = synth.bn_pool_inputs(cut(b["N"]), b["C"], b["H"], b["W"], b["dtype"], seed, dev)
@@ -401,6 +404,9 @@ class Workload:
         elif name == "residual_layernorm":       # same tensors and shape as the LayerNorm config, no bias / GELU
             k.kop_residual_layernorm(self.nx, self.nr, self.ng, self.nbe, c["layernorm"]["eps"], out=self.ny,
                                      mean=self.nmean, rstd=self.nrstd)
+        elif name == "layernorm_params16":       # the LayerNorm config with bias / gamma / beta stored in bf16
+            k.kop_layernorm_ex(self.nx, self.nr, *self.np16, c["layernorm"]["eps"], "bias_gelu_residual", out=self.ny,
+                               mean=self.nmean, rstd=self.nrstd)
         elif name == "silu_mul_interleaved":     # the SiLU*up config read as [g0, u0, g1, u1, ...]
             k.kop_silu_mul_interleaved(self.gu, out=self.act)
         elif name == "ce_loss_opts":             # the CE config with every fifth row ignored, smoothing 0.1

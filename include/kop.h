@@ -263,6 +263,32 @@ kop_status_t kop_residual_rmsnorm(const void* x, const void* residual, const flo
                                   kop_stream_t stream);
 
 /*
+ * The LayerNorm and RMSNorm entry points above with the parameter vectors in either fp32 or the data type
+ * (models held in bf16 / fp16 keep their norm weights in that type; 16-bit parameters also halve the
+ * parameter bytes every row re-reads from L1, which is what bounds the LayerNorm kernel). param_dtype is
+ * KOP_F32 or equal to `dtype`; anything else returns KOP_ERR_UNSUPPORTED_DTYPE. A 16-bit parameter is
+ * widened exactly to fp32 and the arithmetic is the same.
+ *
+ * kop_layernorm_ex: `prologue` selects what precedes the normalisation:
+ *   0  v = residual + gelu_tanh(x + bias)      (kop_bias_gelu_residual_layernorm)
+ *   1  v = x + residual                        (kop_residual_layernorm with a residual; bias ignored)
+ *   2  v = x                                   (kop_residual_layernorm without; residual and bias ignored)
+ *   3  v = residual + gelu_erf(x + bias)       (kop_bias_erfgelu_residual_layernorm)
+ * bias, gamma, beta: [hidden] of param_dtype. Everything else as in those entry points.
+ *
+ * kop_rmsnorm_ex: residual == NULL gives kop_rmsnorm (h and the two residual strides are ignored), otherwise
+ * kop_residual_rmsnorm. weight: [hidden] of param_dtype.
+ */
+kop_status_t kop_layernorm_ex(const void* x, const void* residual, const void* bias, const void* gamma,
+                              const void* beta, void* y, float* mean, float* rstd, int64_t rows, int64_t hidden,
+                              int64_t x_row_stride, int64_t res_row_stride, int64_t y_row_stride, float eps,
+                              int prologue, kop_dtype_t dtype, kop_dtype_t param_dtype, kop_stream_t stream);
+kop_status_t kop_rmsnorm_ex(const void* x, const void* residual, const void* weight, void* h, void* y, int64_t rows,
+                            int64_t hidden, int64_t x_row_stride, int64_t res_row_stride, int64_t h_row_stride,
+                            int64_t y_row_stride, float eps, kop_dtype_t dtype, kop_dtype_t param_dtype,
+                            kop_stream_t stream);
+
+/*
  * SwiGLU epilogue of a preserved GEMM (fusion agent: "activation fusion
  * (GELU/SiLU/ReLU)"; codegen agent: keep the matmul as a library call and fuse only
  * the epilogue):

@@ -364,4 +364,18 @@ __device__ __forceinline__ float block_max(float v, float* slots)
 
 #endif  // __CUDACC__
 
+// Parameter vectors stored in a 16-bit data type: the eight that go with one data vector are one 16-byte
+// load (half the bytes and L1 wavefronts of fp32 parameters). kWide has no meaning here.
+template <int E, bool kWide, typename PT>
+__device__ __forceinline__ void load_params(const PT* p, float2 (&out)[E / 2])
+{
+    static_assert(E == 8 && sizeof(PT) == 2, "16-bit parameters go with 16-bit data");
+    const uint4 t = __ldg(reinterpret_cast<const uint4*>(p));
+    Elem<PT>::unpack2(Vec16{{t.x, t.y, t.z, t.w}}, out);
+}
+// One parameter as fp32.
+__device__ __forceinline__ float param1(const float* p, int64_t j) { return __ldg(p + j); }
+__device__ __forceinline__ float param1(const __nv_bfloat16* p, int64_t j) { return Elem<__nv_bfloat16>::load1(p + j); }
+__device__ __forceinline__ float param1(const __half* p, int64_t j) { return Elem<__half>::load1(p + j); }
+
 }  // namespace kop

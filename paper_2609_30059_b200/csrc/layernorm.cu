@@ -69,10 +69,10 @@ __device__ __forceinline__ float prologue1(float x, float b, float r)
 // (no tail predicates). kWide: the eight fp32 parameters that go with a bf16 vector are fetched
 // with one 256-bit load per lane, so a warp touches each 128-byte line once (two 128-bit loads
 // per lane would walk every line twice and double the L1 wavefronts, which bound this kernel).
-template <typename T, int VPT, bool kFull, bool kWide, int PRO>
+template <typename T, typename PT, int VPT, bool kFull, bool kWide, int PRO>
 __global__ void __launch_bounds__(max_threads_for(VPT * Elem<T>::kPerVec))
-ln_block_kernel(const T* __restrict__ x, const T* __restrict__ res, const float* __restrict__ bias,
-                const float* __restrict__ gamma, const float* __restrict__ beta, T* __restrict__ y,
+ln_block_kernel(const T* __restrict__ x, const T* __restrict__ res, const PT* __restrict__ bias,
+                const PT* __restrict__ gamma, const PT* __restrict__ beta, T* __restrict__ y,
                 float* __restrict__ mean, float* __restrict__ rstd, int nvec, int64_t x_stride,
                 int64_t r_stride, int64_t y_stride, float eps, float inv_hidden)
 {
@@ -160,10 +160,10 @@ ln_block_kernel(const T* __restrict__ x, const T* __restrict__ res, const float*
 // fetches its bias / gamma / beta once and applies them to the same columns of two rows, which
 // halves that traffic; both rows' reductions share the two barriers. The row must be exactly
 // blockDim.x * VPT vectors; `rows` may be odd (the last CTA then skips its second row).
-template <typename T, int VPT, bool kWide, int kMaxThreads, int PRO>
+template <typename T, typename PT, int VPT, bool kWide, int kMaxThreads, int PRO>
 __global__ void __launch_bounds__(kMaxThreads, 768 / kMaxThreads)
-ln_pair_kernel(const T* __restrict__ x, const T* __restrict__ res, const float* __restrict__ bias,
-               const float* __restrict__ gamma, const float* __restrict__ beta, T* __restrict__ y,
+ln_pair_kernel(const T* __restrict__ x, const T* __restrict__ res, const PT* __restrict__ bias,
+               const PT* __restrict__ gamma, const PT* __restrict__ beta, T* __restrict__ y,
                float* __restrict__ mean, float* __restrict__ rstd, int64_t rows, int64_t x_stride,
                int64_t r_stride, int64_t y_stride, float eps, float inv_hidden)
 {
@@ -267,19 +267,19 @@ ln_pair_kernel(const T* __restrict__ x, const T* __restrict__ res, const float* 
 }
 
 // Any hidden size / alignment: scalar loads, v recomputed in each of three sweeps.
-template <typename T, int PRO, bool kFast>
-__device__ __forceinline__ float ln_value(const T* xr, const T* rr, const float* bias, int64_t j)
+template <typename T, typename PT, int PRO, bool kFast>
+__device__ __forceinline__ float ln_value(const T* xr, const T* rr, const PT* bias, int64_t j)
 {
     const float xv = Elem<T>::load1(xr + j);
     const float rv = pro_has_residual(PRO) ? Elem<T>::load1(rr + j) : 0.0f;
-    const float bv = pro_has_bias(PRO) ? __ldg(bias + j) : 0.0f;
+    const float bv = pro_has_bias(PRO) ? param1(bias, j) : 0.0f;
     return prologue1<PRO, kFast>(xv, bv, rv);
 }
 
-template <typename T, int PRO>
+template <typename T, typename PT, int PRO>
 __global__ void __launch_bounds__(256)
-ln_generic_kernel(const T* __restrict__ x, const T* __restrict__ res, const float* __restrict__ bias,
-                  const float* __restrict__ gamma, const float* __restrict__ beta, T* __restrict__ y,
+ln_generic_kernel(const T* __restrict__ x, const T* __restrict__ res, const PT* __restrict__ bias,
+                  const PT* __restrict__ gamma, const PT* __restrict__ beta, T* __restrict__ y,
                   float* __restrict__ mean, float* __restrict__ rstd, int64_t hidden, int64_t x_stride,
                   int64_t r_stride, int64_t y_stride, float eps, float inv_hidden)
 {
@@ -291,12 +291,12 @@ ln_generic_kernel(const T* __restrict__ x, const T* __restrict__ res, const floa
     T* yr = y + row * y_stride;
     float sum = 0.0f;
     for (int64_t j = threadIdx.x; j < hidden; j += blockDim.x)
-        sum += ln_value<T, PRO, kFast>(xr, rr, bias, j);
+        sum += ln_value<T, PT, PRO, kFast>(xr, rr, bias, j);
     const float mu = block_sum(sum, red_a) * inv_hidden;
     float ss = 0.0f;
     for (int64_t j = threadIdx.x; j < hidden; j += blockDim.x) {
         const float d =
-            ln_value<T, PRO, kFast>(xr, rr, bias, j) - mu;
+            ln_value<T, PT, PRO, kFast>(xr, rr, bias, j) - mu;
         ss = fmaf(d, d, ss);
     }
     const float rs = rsqrtf(block_sum(ss, red_b) * inv_hidden + eps);
@@ -306,20 +306,23 @@ ln_generic_kernel(const T* __restrict__ x, const T* __restrict__ res, const floa
     }
     for (int64_t j = threadIdx.x; j < hidden; j += blockDim.x) {
         const float d =
-            ln_value<T, PRO, kFast>(xr, rr, bias, j) - mu;
-        Elem<T>::store1(yr + j, fmaf(d * rs, __ldg(gamma + j), __ldg(beta + j)));
+            ln_value<T, PT, PRO, kFast>(xr, rr, bias, j) - mu;
+        Elem<T>::store1(yr + j, fmaf(d * rs, param1(gamma, j), param1(beta, j)));
     }
 }
 
-template <typename T, int PRO>
-kop_status_t launch_ln(const void* xv, const void* rv, const float* bias, const float* gamma,
-                       const float* beta, void* yv, float* mean, float* rstd, int64_t rows,
+template <typename T, typename PT, int PRO>
+kop_status_t launch_ln(const void* xv, const void* rv, const void* biasv, const void* gammav,
+                       const void* betav, void* yv, float* mean, float* rstd, int64_t rows,
                        int64_t hidden, int64_t xs, int64_t rs, int64_t ys, float eps,
                        cudaStream_t stream)
 {
     const T* x = static_cast<const T*>(xv);
     const T* r = static_cast<const T*>(rv);
     T* y = static_cast<T*>(yv);
+    const PT* bias = static_cast<const PT*>(biasv);
+    const PT* gamma = static_cast<const PT*>(gammav);
+    const PT* beta = static_cast<const PT*>(betav);
     constexpr int E = Elem<T>::kPerVec;
     const float inv_hidden = (float)(1.0 / (double)hidden);
     if (rows > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
@@ -331,18 +334,20 @@ kop_status_t launch_ln(const void* xv, const void* rv, const float* bias, const 
         const int nvec = (int)nvec64;
         // 32 values per thread (hidden 4096 -> 128-thread CTAs, eight 16-byte loads in flight per
         // thread and ~8 CTAs per SM); short rows use fewer, rows beyond 512 threads' worth use 64.
-        const bool wide = E == 8 && (!pro_has_bias(PRO) || aligned_to(bias, 32)) && aligned_to(gamma, 32) &&
+        const bool wide = sizeof(PT) == 4 && E == 8 && (!pro_has_bias(PRO) || aligned_to(bias, 32)) && aligned_to(gamma, 32) &&
                           aligned_to(beta, 32);
-        // Rows of 2048..8192 elements that split evenly into 16 values per thread go two per CTA
-        // (parameters fetched once per pair) once there are enough pairs to fill the GPU.
+        // Rows of 2048..5120 elements that split evenly into 16 values per thread go two per CTA
+        // (parameters fetched once per pair) once there are enough pairs to fill the GPU. Longer rows do
+        // better one per CTA with 32 values a thread (bf16 [8192, 8192]: 86 us against 106 us; 6144: 66
+        // against 90), where the pair kernel's 384- to 512-thread CTAs leave one CTA per SM.
         {
             const int vpt2 = 16 / E;
             const int threads2 = nvec / vpt2;
-            if (nvec % vpt2 == 0 && threads2 % 32 == 0 && threads2 >= 128 && threads2 <= 512 &&
+            if (nvec % vpt2 == 0 && threads2 % 32 == 0 && threads2 >= 128 && threads2 <= 320 &&
                 rows >= 8 * (int64_t)sm_count()) {
                 const unsigned grid = (unsigned)((rows + 1) / 2);
 #define KOP_LN_PAIR(W, MT)                                                                              \
-    ln_pair_kernel<T, 16 / E, W, MT, PRO><<<grid, threads2, 0, stream>>>(x, r, bias, gamma, beta, y, mean, rstd, \
+    ln_pair_kernel<T, PT, 16 / E, W, MT, PRO><<<grid, threads2, 0, stream>>>(x, r, bias, gamma, beta, y, mean, rstd, \
                                                                     rows, xs, rs, ys, eps, inv_hidden)
                 if (threads2 <= 256) { if (wide) KOP_LN_PAIR(true, 256); else KOP_LN_PAIR(false, 256); }
                 else { if (wide) KOP_LN_PAIR(true, 512); else KOP_LN_PAIR(false, 512); }
@@ -358,7 +363,7 @@ kop_status_t launch_ln(const void* xv, const void* rv, const float* bias, const 
         const int threads = ((nvec + vpt - 1) / vpt + 31) / 32 * 32;
         const bool full = (nvec % vpt) == 0 && (nvec / vpt) == threads;
 #define KOP_LN_LAUNCH(V, F, W)                                                                    \
-    ln_block_kernel<T, V, F, W, PRO><<<(unsigned)rows, threads, 0, stream>>>(x, r, bias, gamma, beta, y, mean, \
+    ln_block_kernel<T, PT, V, F, W, PRO><<<(unsigned)rows, threads, 0, stream>>>(x, r, bias, gamma, beta, y, mean, \
                                                                         rstd, nvec, xs, rs, ys, eps, inv_hidden)
 #define KOP_LN(V)                                             \
     do {                                                      \
@@ -377,7 +382,7 @@ kop_status_t launch_ln(const void* xv, const void* rv, const float* bias, const 
 #undef KOP_LN
         return launch_status();
     }
-    ln_generic_kernel<T, PRO><<<(unsigned)rows, 256, 0, stream>>>(x, r, bias, gamma, beta, y, mean, rstd,
+    ln_generic_kernel<T, PT, PRO><<<(unsigned)rows, 256, 0, stream>>>(x, r, bias, gamma, beta, y, mean, rstd,
                                                              hidden, xs, rs, ys, eps, inv_hidden);
     return launch_status();
 }
@@ -387,39 +392,62 @@ kop_status_t launch_ln(const void* xv, const void* rv, const float* bias, const 
 
 namespace kop {
 namespace {
-template <int PRO>
-kop_status_t bias_gelu_ln_entry(
-    const void* x, const void* residual, const float* bias, const float* gamma, const float* beta,
-    void* y, float* mean, float* rstd, int64_t rows, int64_t hidden, int64_t x_row_stride,
-    int64_t res_row_stride, int64_t y_row_stride, float eps, kop_dtype_t dtype, kop_stream_t stream)
+
+// One validated entry for every LayerNorm variant. `pro` is one of the kPro* values; pdtype is KOP_F32 or, for
+// 16-bit data, the data type itself (bias / gamma / beta then hold elements of that type).
+kop_status_t ln_entry(int pro, const void* x, const void* residual, const void* bias, const void* gamma,
+                      const void* beta, void* y, float* mean, float* rstd, int64_t rows, int64_t hidden,
+                      int64_t x_row_stride, int64_t res_row_stride, int64_t y_row_stride, float eps, kop_dtype_t dtype,
+                      kop_dtype_t pdtype, kop_stream_t stream)
 {
-    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    if (!dtype_ok(dtype) || !dtype_ok(pdtype) || (pdtype != KOP_F32 && pdtype != dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    if (pro < 0 || pro > 3) return KOP_ERR_BAD_SHAPE;
+    const bool has_res = pro_has_residual(pro), has_bias = pro_has_bias(pro);
     kop_status_t st = check_rows_cols(rows, hidden);
     if (st != KOP_OK) return st;
     if (rows == 0) return KOP_OK;
-    if (!x || !residual || !bias || !gamma || !beta || !y) return KOP_ERR_NULL_POINTER;
+    if (!x || (has_res && !residual) || (has_bias && !bias) || !gamma || !beta || !y) return KOP_ERR_NULL_POINTER;
     if ((st = check_row_stride(x_row_stride, hidden, rows)) != KOP_OK) return st;
-    if ((st = check_row_stride(res_row_stride, hidden, rows)) != KOP_OK) return st;
+    if (has_res && (st = check_row_stride(res_row_stride, hidden, rows)) != KOP_OK) return st;
     if ((st = check_row_stride(y_row_stride, hidden, rows)) != KOP_OK) return st;
     if (!(eps >= 0.0f)) return KOP_ERR_BAD_SHAPE;
-    const int esz = elem_size(dtype);
-    if (!aligned_to(x, esz) || !aligned_to(residual, esz) || !aligned_to(y, esz) ||
-        !aligned_to(bias, 4) || !aligned_to(gamma, 4) || !aligned_to(beta, 4) ||
+    const int esz = elem_size(dtype), psz = elem_size(pdtype);
+    if (!aligned_to(x, esz) || (has_res && !aligned_to(residual, esz)) || !aligned_to(y, esz) ||
+        (has_bias && !aligned_to(bias, psz)) || !aligned_to(gamma, psz) || !aligned_to(beta, psz) ||
         (mean && !aligned_to(mean, 4)) || (rstd && !aligned_to(rstd, 4)))
         return KOP_ERR_MISALIGNED;
     if (!alias_ok(x, x_row_stride, y, y_row_stride, rows, hidden, esz, true) ||
-        !alias_ok(residual, res_row_stride, y, y_row_stride, rows, hidden, esz, true))
+        (has_res && !alias_ok(residual, res_row_stride, y, y_row_stride, rows, hidden, esz, true)))
         return KOP_ERR_BAD_ALIAS;
     if ((st = check_device()) != KOP_OK) return st;
     cudaStream_t s = as_stream(stream);
-    return dtype == KOP_F32
-               ? launch_ln<float, PRO>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
-                                  x_row_stride, res_row_stride, y_row_stride, eps, s)
-               : dtype == KOP_BF16 ? launch_ln<__nv_bfloat16, PRO>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
-                                          x_row_stride, res_row_stride, y_row_stride, eps, s)
-               : launch_ln<__half, PRO>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
-                                          x_row_stride, res_row_stride, y_row_stride, eps, s);
+    if (!has_res) {                                          // never loaded; keep the pointer arithmetic valid
+        residual = x;
+        res_row_stride = x_row_stride;
+    }
+#define KOP_LN_GO(T, PT, PRO) \
+    return launch_ln<T, PT, PRO>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden, x_row_stride, \
+                                 res_row_stride, y_row_stride, eps, s)
+#define KOP_LN_TYPES(PRO)                                                         \
+    do {                                                                          \
+        if (dtype == KOP_F32) KOP_LN_GO(float, float, PRO);                       \
+        if (dtype == KOP_BF16) {                                                  \
+            if (pdtype == KOP_F32) KOP_LN_GO(__nv_bfloat16, float, PRO);          \
+            KOP_LN_GO(__nv_bfloat16, __nv_bfloat16, PRO);                         \
+        }                                                                         \
+        if (pdtype == KOP_F32) KOP_LN_GO(__half, float, PRO);                     \
+        KOP_LN_GO(__half, __half, PRO);                                           \
+    } while (0)
+    switch (pro) {
+    case kProBiasGeluResidual: KOP_LN_TYPES(kProBiasGeluResidual);
+    case kProResidual: KOP_LN_TYPES(kProResidual);
+    case kProNone: KOP_LN_TYPES(kProNone);
+    default: KOP_LN_TYPES(kProBiasErfGeluResidual);
+    }
+#undef KOP_LN_TYPES
+#undef KOP_LN_GO
 }
+
 }  // namespace
 }  // namespace kop
 
@@ -428,8 +456,8 @@ extern "C" kop_status_t kop_bias_gelu_residual_layernorm(
     void* y, float* mean, float* rstd, int64_t rows, int64_t hidden, int64_t x_row_stride,
     int64_t res_row_stride, int64_t y_row_stride, float eps, kop_dtype_t dtype, kop_stream_t stream)
 {
-    return kop::bias_gelu_ln_entry<kop::kProBiasGeluResidual>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
-                                                              x_row_stride, res_row_stride, y_row_stride, eps, dtype, stream);
+    return kop::ln_entry(kop::kProBiasGeluResidual, x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
+                         x_row_stride, res_row_stride, y_row_stride, eps, dtype, KOP_F32, stream);
 }
 
 extern "C" kop_status_t kop_bias_erfgelu_residual_layernorm(
@@ -437,8 +465,8 @@ extern "C" kop_status_t kop_bias_erfgelu_residual_layernorm(
     void* y, float* mean, float* rstd, int64_t rows, int64_t hidden, int64_t x_row_stride,
     int64_t res_row_stride, int64_t y_row_stride, float eps, kop_dtype_t dtype, kop_stream_t stream)
 {
-    return kop::bias_gelu_ln_entry<kop::kProBiasErfGeluResidual>(x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
-                                                                 x_row_stride, res_row_stride, y_row_stride, eps, dtype, stream);
+    return kop::ln_entry(kop::kProBiasErfGeluResidual, x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden,
+                         x_row_stride, res_row_stride, y_row_stride, eps, dtype, KOP_F32, stream);
 }
 
 extern "C" kop_status_t kop_residual_layernorm(const void* x, const void* residual, const float* gamma,
@@ -447,39 +475,16 @@ extern "C" kop_status_t kop_residual_layernorm(const void* x, const void* residu
                                                int64_t res_row_stride, int64_t y_row_stride, float eps,
                                                kop_dtype_t dtype, kop_stream_t stream)
 {
-    using namespace kop;
-    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
-    kop_status_t st = check_rows_cols(rows, hidden);
-    if (st != KOP_OK) return st;
-    if (rows == 0) return KOP_OK;
-    if (!x || !gamma || !beta || !y) return KOP_ERR_NULL_POINTER;
-    if ((st = check_row_stride(x_row_stride, hidden, rows)) != KOP_OK) return st;
-    if (residual && (st = check_row_stride(res_row_stride, hidden, rows)) != KOP_OK) return st;
-    if ((st = check_row_stride(y_row_stride, hidden, rows)) != KOP_OK) return st;
-    if (!(eps >= 0.0f)) return KOP_ERR_BAD_SHAPE;
-    const int esz = elem_size(dtype);
-    if (!aligned_to(x, esz) || (residual && !aligned_to(residual, esz)) || !aligned_to(y, esz) ||
-        !aligned_to(gamma, 4) || !aligned_to(beta, 4) || (mean && !aligned_to(mean, 4)) ||
-        (rstd && !aligned_to(rstd, 4)))
-        return KOP_ERR_MISALIGNED;
-    if (!alias_ok(x, x_row_stride, y, y_row_stride, rows, hidden, esz, true) ||
-        (residual && !alias_ok(residual, res_row_stride, y, y_row_stride, rows, hidden, esz, true)))
-        return KOP_ERR_BAD_ALIAS;
-    if ((st = check_device()) != KOP_OK) return st;
-    cudaStream_t s = as_stream(stream);
-    const int64_t rs = residual ? res_row_stride : x_row_stride;
-    if (residual != nullptr)
-        return dtype == KOP_F32
-                   ? launch_ln<float, kProResidual>(x, residual, nullptr, gamma, beta, y, mean, rstd, rows, hidden,
-                                                    x_row_stride, rs, y_row_stride, eps, s)
-                   : dtype == KOP_BF16 ? launch_ln<__nv_bfloat16, kProResidual>(x, residual, nullptr, gamma, beta, y, mean, rstd, rows,
-                                                            hidden, x_row_stride, rs, y_row_stride, eps, s)
-                   : launch_ln<__half, kProResidual>(x, residual, nullptr, gamma, beta, y, mean, rstd, rows,
-                                                            hidden, x_row_stride, rs, y_row_stride, eps, s);
-    return dtype == KOP_F32 ? launch_ln<float, kProNone>(x, x, nullptr, gamma, beta, y, mean, rstd, rows, hidden,
-                                                         x_row_stride, rs, y_row_stride, eps, s)
-                            : dtype == KOP_BF16 ? launch_ln<__nv_bfloat16, kProNone>(x, x, nullptr, gamma, beta, y, mean, rstd, rows,
-                                                                 hidden, x_row_stride, rs, y_row_stride, eps, s)
-                            : launch_ln<__half, kProNone>(x, x, nullptr, gamma, beta, y, mean, rstd, rows,
-                                                                 hidden, x_row_stride, rs, y_row_stride, eps, s);
+    return kop::ln_entry(residual ? kop::kProResidual : kop::kProNone, x, residual, nullptr, gamma, beta, y, mean, rstd,
+                         rows, hidden, x_row_stride, res_row_stride, y_row_stride, eps, dtype, KOP_F32, stream);
+}
+
+extern "C" kop_status_t kop_layernorm_ex(const void* x, const void* residual, const void* bias, const void* gamma,
+                                         const void* beta, void* y, float* mean, float* rstd, int64_t rows,
+                                         int64_t hidden, int64_t x_row_stride, int64_t res_row_stride,
+                                         int64_t y_row_stride, float eps, int prologue, kop_dtype_t dtype,
+                                         kop_dtype_t param_dtype, kop_stream_t stream)
+{
+    return kop::ln_entry(prologue, x, residual, bias, gamma, beta, y, mean, rstd, rows, hidden, x_row_stride,
+                         res_row_stride, y_row_stride, eps, dtype, param_dtype, stream);
 }

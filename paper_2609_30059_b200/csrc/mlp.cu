@@ -21,9 +21,9 @@ struct RmsRes {
     int64_t res_stride, h_stride;
 };
 
-template <typename T, int VPT, bool kFull, bool kWide, bool kRes>
+template <typename T, typename PT, int VPT, bool kFull, bool kWide, bool kRes>
 __global__ void __launch_bounds__(max_threads_for(VPT * Elem<T>::kPerVec))
-rmsnorm_block_kernel(const T* __restrict__ x, const float* __restrict__ w, T* __restrict__ y, int nvec,
+rmsnorm_block_kernel(const T* __restrict__ x, const PT* __restrict__ w, T* __restrict__ y, int nvec,
                      int64_t x_stride, int64_t y_stride, float eps, float inv_hidden, RmsRes rr)
 {
     constexpr int E = Elem<T>::kPerVec;
@@ -77,9 +77,9 @@ rmsnorm_block_kernel(const T* __restrict__ x, const float* __restrict__ w, T* __
     }
 }
 
-template <typename T, bool kRes>
+template <typename T, typename PT, bool kRes>
 __global__ void __launch_bounds__(256)
-rmsnorm_generic_kernel(const T* __restrict__ x, const float* __restrict__ w, T* __restrict__ y,
+rmsnorm_generic_kernel(const T* __restrict__ x, const PT* __restrict__ w, T* __restrict__ y,
                        int64_t hidden, int64_t x_stride, int64_t y_stride, float eps, float inv_hidden, RmsRes rr)
 {
     __shared__ float red[32];
@@ -98,7 +98,7 @@ rmsnorm_generic_kernel(const T* __restrict__ x, const float* __restrict__ w, T* 
     for (int64_t j = threadIdx.x; j < hidden; j += blockDim.x) {
         const float v = Elem<T>::load1(xr + j) + (kRes ? Elem<T>::load1(resr + j) : 0.0f);
         if (kRes) Elem<T>::store1(hr + j, v);
-        Elem<T>::store1(yr + j, v * r * __ldg(w + j));
+        Elem<T>::store1(yr + j, v * r * param1(w, j));
     }
 }
 
@@ -282,13 +282,14 @@ residual_add_scalar_kernel(const T* __restrict__ a, const T* __restrict__ b, T* 
 }
 
 // ---- launchers ------------------------------------------------------------------------------------
-template <typename T>
-kop_status_t launch_rmsnorm(const void* xv, const float* w, void* yv, int64_t rows, int64_t hidden,
+template <typename T, typename PT = float>
+kop_status_t launch_rmsnorm(const void* xv, const void* wv, void* yv, int64_t rows, int64_t hidden,
                             int64_t xs, int64_t ys, float eps, cudaStream_t stream, bool with_res = false,
                             RmsRes rr = RmsRes{nullptr, nullptr, 0, 0})
 {
     const T* x = static_cast<const T*>(xv);
     T* y = static_cast<T*>(yv);
+    const PT* w = static_cast<const PT*>(wv);
     constexpr int E = Elem<T>::kPerVec;
     if (rows > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
     const float inv_hidden = (float)(1.0 / (double)hidden);
@@ -305,11 +306,11 @@ kop_status_t launch_rmsnorm(const void* xv, const float* w, void* yv, int64_t ro
         const int vpt = vals / E;
         const int threads = ((nvec + vpt - 1) / vpt + 31) / 32 * 32;
         const bool full = (nvec % vpt) == 0 && (nvec / vpt) == threads;
-        const bool wide = E == 8 && aligned_to(w, 32);
+        const bool wide = sizeof(PT) == 4 && E == 8 && aligned_to(w, 32);
 #define KOP_RMS_LAUNCH(V, F, W)                                                                                       \
     do {                                                                                                              \
-        if (with_res) rmsnorm_block_kernel<T, V, F, W, true><<<(unsigned)rows, threads, 0, stream>>>(x, w, y, nvec, xs, ys, eps, inv_hidden, rr); \
-        else rmsnorm_block_kernel<T, V, F, W, false><<<(unsigned)rows, threads, 0, stream>>>(x, w, y, nvec, xs, ys, eps, inv_hidden, rr);         \
+        if (with_res) rmsnorm_block_kernel<T, PT, V, F, W, true><<<(unsigned)rows, threads, 0, stream>>>(x, w, y, nvec, xs, ys, eps, inv_hidden, rr); \
+        else rmsnorm_block_kernel<T, PT, V, F, W, false><<<(unsigned)rows, threads, 0, stream>>>(x, w, y, nvec, xs, ys, eps, inv_hidden, rr);         \
     } while (0)
 #define KOP_RMS(V)                                             \
     do {                                                       \
@@ -328,8 +329,8 @@ kop_status_t launch_rmsnorm(const void* xv, const float* w, void* yv, int64_t ro
 #undef KOP_RMS
         return launch_status();
     }
-    if (with_res) rmsnorm_generic_kernel<T, true><<<(unsigned)rows, 256, 0, stream>>>(x, w, y, hidden, xs, ys, eps, inv_hidden, rr);
-    else rmsnorm_generic_kernel<T, false><<<(unsigned)rows, 256, 0, stream>>>(x, w, y, hidden, xs, ys, eps, inv_hidden, rr);
+    if (with_res) rmsnorm_generic_kernel<T, PT, true><<<(unsigned)rows, 256, 0, stream>>>(x, w, y, hidden, xs, ys, eps, inv_hidden, rr);
+    else rmsnorm_generic_kernel<T, PT, false><<<(unsigned)rows, 256, 0, stream>>>(x, w, y, hidden, xs, ys, eps, inv_hidden, rr);
     return launch_status();
 }
 
@@ -532,28 +533,61 @@ kop_status_t gemm_nt_plus_residual(MlpHandle* mh, const void* A, const void* Wt,
 }  // namespace
 }  // namespace kop
 
+namespace kop {
+namespace {
+
+// One validated entry for RMSNorm with or without the residual add. residual == NULL: y = rmsnorm(x) and h is
+// ignored; else h = x + residual, y = rmsnorm(h). pdtype is KOP_F32 or, for 16-bit data, the data type itself.
+kop_status_t rms_entry(const void* x, const void* residual, const void* weight, void* h, void* y, int64_t rows,
+                       int64_t hidden, int64_t x_row_stride, int64_t res_row_stride, int64_t h_row_stride,
+                       int64_t y_row_stride, float eps, kop_dtype_t dtype, kop_dtype_t pdtype, kop_stream_t stream)
+{
+    if (!dtype_ok(dtype) || !dtype_ok(pdtype) || (pdtype != KOP_F32 && pdtype != dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    kop_status_t st = check_rows_cols(rows, hidden);
+    if (st != KOP_OK) return st;
+    if (rows == 0) return KOP_OK;
+    const bool with_res = residual != nullptr;
+    if (!x || !weight || !y || (with_res && !h)) return KOP_ERR_NULL_POINTER;
+    if ((st = check_row_stride(x_row_stride, hidden, rows)) != KOP_OK) return st;
+    if (with_res && (st = check_row_stride(res_row_stride, hidden, rows)) != KOP_OK) return st;
+    if (with_res && (st = check_row_stride(h_row_stride, hidden, rows)) != KOP_OK) return st;
+    if ((st = check_row_stride(y_row_stride, hidden, rows)) != KOP_OK) return st;
+    if (!(eps >= 0.0f)) return KOP_ERR_BAD_SHAPE;
+    const int esz = elem_size(dtype);
+    if (!aligned_to(x, esz) || !aligned_to(y, esz) || !aligned_to(weight, elem_size(pdtype)) ||
+        (with_res && (!aligned_to(residual, esz) || !aligned_to(h, esz))))
+        return KOP_ERR_MISALIGNED;
+    if (!alias_ok(x, x_row_stride, y, y_row_stride, rows, hidden, esz, true)) return KOP_ERR_BAD_ALIAS;
+    // each output may be one of the inputs exactly, but the two outputs must be different tensors
+    if (with_res && (!alias_ok(x, x_row_stride, h, h_row_stride, rows, hidden, esz, true) ||
+                     !alias_ok(residual, res_row_stride, h, h_row_stride, rows, hidden, esz, true) ||
+                     !alias_ok(residual, res_row_stride, y, y_row_stride, rows, hidden, esz, true) ||
+                     !alias_ok(h, h_row_stride, y, y_row_stride, rows, hidden, esz, false)))
+        return KOP_ERR_BAD_ALIAS;
+    if ((st = check_device()) != KOP_OK) return st;
+    cudaStream_t s = as_stream(stream);
+    const RmsRes rr{residual, h, res_row_stride, h_row_stride};
+#define KOP_RMS_GO(T, PT) \
+    return launch_rmsnorm<T, PT>(x, weight, y, rows, hidden, x_row_stride, y_row_stride, eps, s, with_res, rr)
+    if (dtype == KOP_F32) KOP_RMS_GO(float, float);
+    if (dtype == KOP_BF16) {
+        if (pdtype == KOP_F32) KOP_RMS_GO(__nv_bfloat16, float);
+        KOP_RMS_GO(__nv_bfloat16, __nv_bfloat16);
+    }
+    if (pdtype == KOP_F32) KOP_RMS_GO(__half, float);
+    KOP_RMS_GO(__half, __half);
+#undef KOP_RMS_GO
+}
+
+}  // namespace
+}  // namespace kop
+
 extern "C" kop_status_t kop_rmsnorm(const void* x, const float* weight, void* y, int64_t rows,
                                     int64_t hidden, int64_t x_row_stride, int64_t y_row_stride,
                                     float eps, kop_dtype_t dtype, kop_stream_t stream)
 {
-    using namespace kop;
-    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
-    kop_status_t st = check_rows_cols(rows, hidden);
-    if (st != KOP_OK) return st;
-    if (rows == 0) return KOP_OK;
-    if (!x || !weight || !y) return KOP_ERR_NULL_POINTER;
-    if ((st = check_row_stride(x_row_stride, hidden, rows)) != KOP_OK) return st;
-    if ((st = check_row_stride(y_row_stride, hidden, rows)) != KOP_OK) return st;
-    if (!(eps >= 0.0f)) return KOP_ERR_BAD_SHAPE;
-    const int esz = elem_size(dtype);
-    if (!aligned_to(x, esz) || !aligned_to(y, esz) || !aligned_to(weight, 4)) return KOP_ERR_MISALIGNED;
-    if (!alias_ok(x, x_row_stride, y, y_row_stride, rows, hidden, esz, true)) return KOP_ERR_BAD_ALIAS;
-    if ((st = check_device()) != KOP_OK) return st;
-    cudaStream_t s = as_stream(stream);
-    return dtype == KOP_F32
-               ? launch_rmsnorm<float>(x, weight, y, rows, hidden, x_row_stride, y_row_stride, eps, s)
-               : dtype == KOP_BF16 ? launch_rmsnorm<__nv_bfloat16>(x, weight, y, rows, hidden, x_row_stride, y_row_stride, eps, s)
-               : launch_rmsnorm<__half>(x, weight, y, rows, hidden, x_row_stride, y_row_stride, eps, s);
+    return kop::rms_entry(x, nullptr, weight, nullptr, y, rows, hidden, x_row_stride, 0, 0, y_row_stride, eps, dtype,
+                          KOP_F32, stream);
 }
 
 extern "C" kop_status_t kop_residual_rmsnorm(const void* x, const void* residual, const float* weight, void* h,
@@ -561,35 +595,18 @@ extern "C" kop_status_t kop_residual_rmsnorm(const void* x, const void* residual
                                              int64_t res_row_stride, int64_t h_row_stride, int64_t y_row_stride,
                                              float eps, kop_dtype_t dtype, kop_stream_t stream)
 {
-    using namespace kop;
-    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
-    kop_status_t st = check_rows_cols(rows, hidden);
-    if (st != KOP_OK) return st;
-    if (rows == 0) return KOP_OK;
-    if (!x || !residual || !weight || !h || !y) return KOP_ERR_NULL_POINTER;
-    if ((st = check_row_stride(x_row_stride, hidden, rows)) != KOP_OK) return st;
-    if ((st = check_row_stride(res_row_stride, hidden, rows)) != KOP_OK) return st;
-    if ((st = check_row_stride(h_row_stride, hidden, rows)) != KOP_OK) return st;
-    if ((st = check_row_stride(y_row_stride, hidden, rows)) != KOP_OK) return st;
-    if (!(eps >= 0.0f)) return KOP_ERR_BAD_SHAPE;
-    const int esz = elem_size(dtype);
-    if (!aligned_to(x, esz) || !aligned_to(residual, esz) || !aligned_to(h, esz) || !aligned_to(y, esz) ||
-        !aligned_to(weight, 4))
-        return KOP_ERR_MISALIGNED;
-    // each output may be one of the inputs exactly, but the two outputs must be different tensors
-    if (!alias_ok(x, x_row_stride, h, h_row_stride, rows, hidden, esz, true) ||
-        !alias_ok(residual, res_row_stride, h, h_row_stride, rows, hidden, esz, true) ||
-        !alias_ok(x, x_row_stride, y, y_row_stride, rows, hidden, esz, true) ||
-        !alias_ok(residual, res_row_stride, y, y_row_stride, rows, hidden, esz, true) ||
-        !alias_ok(h, h_row_stride, y, y_row_stride, rows, hidden, esz, false))
-        return KOP_ERR_BAD_ALIAS;
-    if ((st = check_device()) != KOP_OK) return st;
-    cudaStream_t s = as_stream(stream);
-    const RmsRes rr{residual, h, res_row_stride, h_row_stride};
-    return dtype == KOP_F32 ? launch_rmsnorm<float>(x, weight, y, rows, hidden, x_row_stride, y_row_stride, eps, s, true, rr)
-           : dtype == KOP_BF16
-               ? launch_rmsnorm<__nv_bfloat16>(x, weight, y, rows, hidden, x_row_stride, y_row_stride, eps, s, true, rr)
-               : launch_rmsnorm<__half>(x, weight, y, rows, hidden, x_row_stride, y_row_stride, eps, s, true, rr);
+    if (rows > 0 && hidden > 0 && kop::dtype_ok(dtype) && !residual) return KOP_ERR_NULL_POINTER;
+    return kop::rms_entry(x, residual, weight, h, y, rows, hidden, x_row_stride, res_row_stride, h_row_stride,
+                          y_row_stride, eps, dtype, KOP_F32, stream);
+}
+
+extern "C" kop_status_t kop_rmsnorm_ex(const void* x, const void* residual, const void* weight, void* h, void* y,
+                                       int64_t rows, int64_t hidden, int64_t x_row_stride, int64_t res_row_stride,
+                                       int64_t h_row_stride, int64_t y_row_stride, float eps, kop_dtype_t dtype,
+                                       kop_dtype_t param_dtype, kop_stream_t stream)
+{
+    return kop::rms_entry(x, residual, weight, h, y, rows, hidden, x_row_stride, res_row_stride, h_row_stride,
+                          y_row_stride, eps, dtype, param_dtype, stream);
 }
 
 extern "C" kop_status_t kop_silu_mul(const void* gate_up, void* out, int64_t rows, int64_t inter,

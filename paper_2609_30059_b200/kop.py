@@ -68,6 +68,10 @@ def lib() -> C.CDLL:
     L.kop_rmsnorm.argtypes = [vp, vp, vp, i64, i64, i64, i64, f32, i32, vp]
     L.kop_residual_rmsnorm.argtypes = [vp] * 5 + [i64] * 6 + [f32, i32, vp]
     L.kop_residual_rmsnorm.restype = i32
+    L.kop_layernorm_ex.argtypes = [vp] * 8 + [i64] * 5 + [f32, i32, i32, i32, vp]
+    L.kop_layernorm_ex.restype = i32
+    L.kop_rmsnorm_ex.argtypes = [vp] * 5 + [i64] * 6 + [f32, i32, i32, vp]
+    L.kop_rmsnorm_ex.restype = i32
     L.kop_silu_mul.argtypes = [vp, vp, i64, i64, i64, i64, i32, vp]
     L.kop_residual_add.argtypes = [vp, vp, vp, i64, i64, i64, i64, i64, i32, vp]
     L.kop_ce_loss_rowwise_opts.argtypes = [vp] * 6 + [i64] * 3 + [C.c_int32, f32, vp, sz, i32, vp]
@@ -278,6 +282,60 @@ def kop_residual_rmsnorm(x, residual, weight, eps, h_out=None, out=None, stream=
                                       out.data_ptr(), rows, hidden, xs, rs, hs, ys, float(eps), _dtype_tag(x),
                                       _stream(stream)), "kop_residual_rmsnorm")
     return h_out, out
+
+
+LN_PROLOGUES = ("bias_gelu_residual", "residual", "none", "bias_erfgelu_residual")
+
+
+def _param_any(t, name: str, n: int, data):
+    """Parameter vector in fp32 or in the data tensor's own type. Returns (pointer, dtype tag)."""
+    if t.dtype not in (torch.float32, data.dtype) or not t.is_cuda or not t.is_contiguous() or t.numel() != n:
+        raise ValueError(f"{name}: expected a contiguous CUDA vector of {n} fp32 or {data.dtype} elements")
+    return t.data_ptr(), (KOP_F32 if t.dtype == torch.float32 else _dtype_tag(data))
+
+
+def kop_layernorm_ex(x, residual, bias, gamma, beta, eps, prologue="bias_gelu_residual", out=None, mean=None,
+                     rstd=None, want_stats=True, stream=None):
+    """LayerNorm with a chosen prologue (LN_PROLOGUES) and parameters in fp32 or x.dtype (all the same type)."""
+    pro = LN_PROLOGUES.index(prologue)
+    rows, hidden, xs = _rows2d(x, "x")
+    rs = xs
+    if pro != 2:
+        _, _, rs = _rows2d(residual, "residual")
+        assert residual.shape == x.shape and residual.dtype == x.dtype
+    out = torch.empty_like(x) if out is None else out
+    _, _, ys = _rows2d(out, "out")
+    if want_stats:
+        mean = torch.empty(rows, dtype=torch.float32, device=x.device) if mean is None else mean
+        rstd = torch.empty(rows, dtype=torch.float32, device=x.device) if rstd is None else rstd
+    gp, ptag = _param_any(gamma, "gamma", hidden, x)
+    bp, btag = _param_any(beta, "beta", hidden, x)
+    ip, itag = _param_any(bias, "bias", hidden, x) if pro in (0, 3) else (None, ptag)
+    if not (ptag == btag == itag):
+        raise ValueError("bias, gamma and beta must share one dtype")
+    _check(lib().kop_layernorm_ex(x.data_ptr(), None if pro == 2 else residual.data_ptr(), ip, gp, bp, out.data_ptr(),
+                                  None if mean is None else mean.data_ptr(), None if rstd is None else rstd.data_ptr(),
+                                  rows, hidden, xs, rs, ys, float(eps), pro, _dtype_tag(x), ptag, _stream(stream)),
+           "kop_layernorm_ex")
+    return out, mean, rstd
+
+
+def kop_rmsnorm_ex(x, weight, eps, residual=None, h_out=None, out=None, stream=None):
+    """RMSNorm with the weight in fp32 or x.dtype. With a residual returns (h, y), h = x + residual; else y."""
+    rows, hidden, xs = _rows2d(x, "x")
+    out = torch.empty_like(x) if out is None else out
+    _, _, ys = _rows2d(out, "out")
+    wp, ptag = _param_any(weight, "weight", hidden, x)
+    rs = hs = 0
+    if residual is not None:
+        _, _, rs = _rows2d(residual, "residual")
+        assert residual.shape == x.shape and residual.dtype == x.dtype
+        h_out = torch.empty_like(x) if h_out is None else h_out
+        _, _, hs = _rows2d(h_out, "h_out")
+    _check(lib().kop_rmsnorm_ex(x.data_ptr(), None if residual is None else residual.data_ptr(), wp,
+                                None if residual is None else h_out.data_ptr(), out.data_ptr(), rows, hidden, xs, rs, hs,
+                                ys, float(eps), _dtype_tag(x), ptag, _stream(stream)), "kop_rmsnorm_ex")
+    return (h_out, out) if residual is not None else out
 
 
 def kop_silu_mul(gate_up, out=None, stream=None):

@@ -264,6 +264,40 @@ def test_gru_cell_validation(L):
     assert f(GI, GH, None, None, HP, GI, 4, 64, 0, None) == ALIAS
 
 
+def test_norm_ex_validation(L):
+    f = L.kop_layernorm_ex
+    B, G, E_ = 0x600000, 0x610000, 0x620000
+    ok = (P, Q, B, G, E_, R, None, None)
+    assert f(*ok, 0, 64, 64, 64, 64, 1e-5, 0, 1, 1, None) == OK
+    assert f(*ok, 4, 64, 64, 64, 64, 1e-5, 0, 1, 2, None) == DTYPE             # fp16 parameters with bf16 data
+    assert f(*ok, 4, 64, 64, 64, 64, 1e-5, 0, 0, 1, None) == DTYPE             # 16-bit parameters with fp32 data
+    assert f(*ok, 4, 64, 64, 64, 64, 1e-5, 0, 1, 3, None) == DTYPE
+    assert f(*ok, 4, 64, 64, 64, 64, 1e-5, 4, 1, 1, None) == SHAPE             # unknown prologue
+    assert f(*ok, 4, 64, 64, 64, 64, 1e-5, -1, 1, 1, None) == SHAPE
+    assert f(P, None, B, G, E_, R, None, None, 4, 64, 64, 64, 64, 1e-5, 0, 1, 1, None) == NULLP
+    assert f(P, None, B, G, E_, R, None, None, 4, 64, 64, 64, 64, 1e-5, 1, 1, 1, None) == NULLP
+    assert f(P, Q, None, G, E_, R, None, None, 4, 64, 64, 64, 64, 1e-5, 3, 1, 1, None) == NULLP
+    assert f(P, Q, B, None, E_, R, None, None, 4, 64, 64, 64, 64, 1e-5, 2, 1, 1, None) == NULLP
+    assert f(P, Q, B, G + 2, E_, R, None, None, 4, 64, 64, 64, 64, 1e-5, 0, 1, 0, None) == MISAL   # fp32 params: 4 bytes
+    assert f(P, Q, B, G + 1, E_, R, None, None, 4, 64, 64, 64, 64, 1e-5, 0, 1, 1, None) == MISAL
+    assert f(P, Q, B, G, E_, R, None, None, 4, 64, 63, 64, 64, 1e-5, 0, 1, 1, None) == STRIDE
+    assert f(P, Q, B, G, E_, R, None, None, 4, 64, 64, 1, 64, 1e-5, 0, 1, 1, None) == STRIDE
+    assert f(P, None, None, G, E_, R, None, None, 4, 64, 64, 1, 64, 1e-5, 2, 1, 1, None) != STRIDE  # ignored without residual
+    g = L.kop_rmsnorm_ex
+    assert g(P, None, G, None, R, 0, 64, 64, 0, 0, 64, 1e-6, 1, 1, None) == OK
+    assert g(P, None, G, None, R, 4, 64, 64, 0, 0, 64, 1e-6, 1, 2, None) == DTYPE
+    assert g(P, None, G, None, R, 4, 64, 64, 0, 0, 64, 1e-6, 0, 2, None) == DTYPE
+    assert g(P, None, None, None, R, 4, 64, 64, 0, 0, 64, 1e-6, 1, 1, None) == NULLP
+    assert g(P, Q, G, None, R, 4, 64, 64, 64, 64, 64, 1e-6, 1, 1, None) == NULLP                 # residual needs h
+    assert g(P, Q, G, B, R, 4, 64, 64, 64, 8, 64, 1e-6, 1, 1, None) == STRIDE
+    assert g(P, None, G + 1, None, R, 4, 64, 64, 0, 0, 64, 1e-6, 2, 2, None) == MISAL
+    assert g(P, Q, G, R, R, 4, 64, 64, 64, 64, 64, 1e-6, 1, 1, None) == ALIAS                    # h and y the same tensor
+    # the fixed-type entry points keep their behaviour
+    assert L.kop_residual_rmsnorm(P, None, G, B, R, 4, 64, 64, 64, 64, 64, 1e-6, 1, None) == NULLP
+    assert L.kop_residual_rmsnorm(P, None, G, B, R, 0, 64, 64, 64, 64, 64, 1e-6, 1, None) == OK
+    assert L.kop_residual_rmsnorm(P, None, G, B, R, 4, 0, 64, 64, 64, 64, 1e-6, 1, None) == SHAPE
+
+
 def test_pool2d_validation(L):
     f = L.kop_affine_relu_pool2d
     S, T = 0x600000, 0x610000
