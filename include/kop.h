@@ -17,8 +17,9 @@
  *   dtype      `dtype` is the element type of the data tensors (inputs and the main
  *              output): KOP_F32, KOP_BF16 or KOP_F16 (IEEE binary16; results beyond
  *              65504 in magnitude are stored as infinity). Parameter vectors (bias, gamma, beta,
- *              scale, shift, weight) and statistics outputs (mean, rstd, pooled,
- *              loss) are always fp32. All arithmetic is fp32; the only rounding to
+ *              scale, shift, weight) are fp32 (kop_layernorm_ex / kop_rmsnorm_ex also take
+ *              them in the data type); statistics outputs (mean, rstd, pooled, loss) are
+ *              always fp32. All arithmetic is fp32; the only rounding to
  *              bf16 / fp16 is the final store (round to nearest even), as the paper's
  *              numerics rule requires (accumulate in fp32, cast only at the store).
  *   strides    In elements. The innermost stride is 1 by contract; a row stride
@@ -32,6 +33,11 @@
  *   stream     Work is enqueued on `stream`; nothing synchronises, allocates or frees,
  *              and the library keeps no state between calls (kop_mlp_handle_* aside,
  *              which only wrap cuBLAS handle creation).
+ *   threads    Any entry point may be called from several host threads at once, on the
+ *              same or different streams, as long as concurrent calls do not share an
+ *              output, a workspace or a kop_mlp_handle (kop_ce_loss_rowwise_static's
+ *              built-in scratch counts as a shared workspace). Results do not depend on
+ *              what else runs.
  *   errors     Static validation (the paper's Gate 1: structural checks before any
  *              numerics) runs first and touches no CUDA API: a call that fails
  *              validation launches nothing. rows == 0 (or N == 0) returns KOP_OK
