@@ -235,6 +235,35 @@ __device__ __forceinline__ void add_vector(Acc<OP>& acc, const Vec16& raw, int j
     }
 }
 
+// logsumexp over a batch of U vectors: the batch maximum on the packed values, one rescale of the running sum
+// for the whole batch (U * E + 1 special-function operations instead of U * (E + 1)), two partial sums to
+// halve the chain of dependent adds. Vectors past the end of the row must hold -inf.
+template <typename T, int U>
+__device__ __forceinline__ void add_vectors_lse(Acc<kOpLse>& acc, const Vec16 (&raw)[U])
+{
+    constexpr int E = Elem<T>::kPerVec;
+    float bm = vec_ext_nan<T, true>(raw[0]);
+#pragma unroll
+    for (int k = 1; k < U; ++k) bm = ext_nan(bm, vec_ext_nan<T, true>(raw[k]), true);
+    if (bm != bm) acc.nan_idx = 0;
+    const float m2 = fmaxf(acc.a, bm);                            // fmaxf drops a NaN operand
+    const float off = m2 == -INFINITY ? 0.0f : m2;                // all -inf so far: avoid inf - inf
+    const float noff = -off * kLog2e;
+    float t0 = 0.0f, t1 = 0.0f;
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+        float f[E];
+        Elem<T>::unpack(raw[k], f);
+#pragma unroll
+        for (int e = 0; e < E; e += 2) {
+            t0 += ex2_approx(fmaf(f[e], kLog2e, noff));
+            t1 += ex2_approx(fmaf(f[e + 1], kLog2e, noff));
+        }
+    }
+    acc.s = fmaf(acc.s, ex2_approx(fmaf(acc.a, kLog2e, noff)), t0 + t1);
+    acc.a = m2;
+}
+
 template <typename T, int OP>
 __device__ __forceinline__ void write_result(const Acc<OP>& acc, float* out, int32_t* index, int64_t row, float inv_cols)
 {
@@ -261,12 +290,17 @@ reduce_row_block_kernel(const T* __restrict__ x, float* __restrict__ out, int32_
 #pragma unroll
             for (int k = 0; k < U; ++k) {
                 const int v = base + k * blockDim.x + threadIdx.x;
+                if (OP == kOpLse) raw[k] = Elem<T>::fill_neg_inf();
                 if (v < nvec) raw[k] = ld_stream(xr + (int64_t)v * E);
             }
+            if constexpr (OP == kOpLse) {
+                add_vectors_lse<T, U>(acc, raw);
+            } else {
 #pragma unroll
-            for (int k = 0; k < U; ++k) {
-                const int v = base + k * blockDim.x + threadIdx.x;
-                if (v < nvec) add_vector<T, OP>(acc, raw[k], v * E);
+                for (int k = 0; k < U; ++k) {
+                    const int v = base + k * blockDim.x + threadIdx.x;
+                    if (v < nvec) add_vector<T, OP>(acc, raw[k], v * E);
+                }
             }
         }
         if (OP == kOpMax || OP == kOpMin) acc.template resolve<T>();
