@@ -1,6 +1,7 @@
 // kop_reduce_rows: sum / mean / max (+ argmax) / min (+ argmin) / logsumexp of every row in one read-only
-// pass. Long rows get a CTA each (batches of four 16-byte vectors per thread in flight, one-barrier block
-// merge), short rows a warp each (eight rows per CTA), like the softmax kernels. Per-thread partial results
+// pass. Rows beyond 16 KB get a CTA each (batches of four 16-byte vectors per thread in flight, one-barrier
+// block merge); shorter rows get 4 to 32 lanes of a warp each, sixteen vectors a lane where the row has them,
+// so that the butterfly merge (the per-row cost) has two to five steps and no barrier. Per-thread partial results
 // are merged in a fixed order, so results do not depend on scheduling; max / min and their indices are exact
 // (first position on ties; a NaN outranks every number and the first NaN's position is reported).
 #include <climits>
@@ -139,11 +140,11 @@ struct Acc {
 
 // Lanes must merge in the same order on both sides of a butterfly to agree bit for bit (fp32 sums): the
 // lower lane's partial is always the left operand.
-template <int OP>
+template <int OP, int L = 32>
 __device__ __forceinline__ Acc<OP> warp_merge(Acc<OP> acc)
 {
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
+    for (int o = L / 2; o > 0; o >>= 1) {
         Acc<OP> other = acc.shuffled(o);
         if ((threadIdx.x & o) == 0) {
             acc.merge(other);
@@ -271,6 +272,32 @@ __device__ __forceinline__ void write_result(const Acc<OP>& acc, float* out, int
     if ((OP == kOpMax || OP == kOpMin) && index != nullptr) index[row] = acc.position();
 }
 
+// The vector sweep of one row by `nthreads` threads (a CTA or a warp), U loads in flight per thread.
+template <typename T, int OP, int U>
+__device__ __forceinline__ void sweep_vectors(Acc<OP>& acc, const T* xr, int nvec, int tid, int nthreads)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    for (int base = 0; base < nvec; base += U * nthreads) {
+        Vec16 raw[U];
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const int v = base + k * nthreads + tid;
+            if (OP == kOpLse) raw[k] = Elem<T>::fill_neg_inf();
+            if (v < nvec) raw[k] = ld_stream(xr + (int64_t)v * E);
+        }
+        if constexpr (OP == kOpLse) {
+            add_vectors_lse<T, U>(acc, raw);
+        } else {
+#pragma unroll
+            for (int k = 0; k < U; ++k) {
+                const int v = base + k * nthreads + tid;
+                if (v < nvec) add_vector<T, OP>(acc, raw[k], v * E);
+            }
+        }
+    }
+    if (OP == kOpMax || OP == kOpMin) acc.template resolve<T>();
+}
+
 // One CTA per row; vector path (rows are whole 16-byte vectors and aligned) or scalar path.
 template <typename T, int OP, bool kVec>
 __global__ void __launch_bounds__(256)
@@ -284,26 +311,7 @@ reduce_row_block_kernel(const T* __restrict__ x, float* __restrict__ out, int32_
     Acc<OP> acc;
     acc.init();
     if (kVec) {
-        const int nvec = cols / E;
-        for (int base = 0; base < nvec; base += U * blockDim.x) {
-            Vec16 raw[U];
-#pragma unroll
-            for (int k = 0; k < U; ++k) {
-                const int v = base + k * blockDim.x + threadIdx.x;
-                if (OP == kOpLse) raw[k] = Elem<T>::fill_neg_inf();
-                if (v < nvec) raw[k] = ld_stream(xr + (int64_t)v * E);
-            }
-            if constexpr (OP == kOpLse) {
-                add_vectors_lse<T, U>(acc, raw);
-            } else {
-#pragma unroll
-                for (int k = 0; k < U; ++k) {
-                    const int v = base + k * blockDim.x + threadIdx.x;
-                    if (v < nvec) add_vector<T, OP>(acc, raw[k], v * E);
-                }
-            }
-        }
-        if (OP == kOpMax || OP == kOpMin) acc.template resolve<T>();
+        sweep_vectors<T, OP, U>(acc, xr, cols / E, threadIdx.x, blockDim.x);
     } else {
         for (int j = threadIdx.x; j < cols; j += blockDim.x) {
             const float v = Elem<T>::load1(xr + j);
@@ -338,25 +346,27 @@ reduce_row_block_kernel(const T* __restrict__ x, float* __restrict__ out, int32_
     }
 }
 
-// One warp per row (short rows), eight rows per CTA.
-template <typename T, int OP, bool kVec>
+// L lanes per row (L = 4 .. 32, a power of two), 32 / L rows per warp, eight warps per CTA: a short row does
+// not pay for a full warp's five butterfly steps, and a lane still has up to four loads in flight. Lanes
+// whose row is past the end sweep nothing but take part in the shuffles.
+template <typename T, int OP, bool kVec, int L>
 __global__ void __launch_bounds__(256)
-reduce_row_warp_kernel(const T* __restrict__ x, float* __restrict__ out, int32_t* __restrict__ index, int64_t rows,
-                       int cols, int64_t stride, float inv_cols)
+reduce_row_group_kernel(const T* __restrict__ x, float* __restrict__ out, int32_t* __restrict__ index, int64_t rows,
+                        int cols, int64_t stride, float inv_cols)
 {
     constexpr int E = Elem<T>::kPerVec;
-    const int lane = threadIdx.x & 31;
-    const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (row >= rows) return;                                 // whole warps leave together
-    const T* xr = x + row * stride;
+    constexpr int kRowsPerWarp = 32 / L;
+    const int lane = threadIdx.x & 31, sub = lane & (L - 1);
+    const int64_t row = ((int64_t)blockIdx.x * 8 + (threadIdx.x >> 5)) * kRowsPerWarp + lane / L;
+    const bool live = row < rows;
+    const T* xr = x + (live ? row : 0) * stride;
+    const int n = live ? cols : 0;
     Acc<OP> acc;
     acc.init();
     if (kVec) {
-        const int nvec = cols / E;
-        for (int v = lane; v < nvec; v += 32) add_vector<T, OP>(acc, ld_stream(xr + (int64_t)v * E), v * E);
-        if (OP == kOpMax || OP == kOpMin) acc.template resolve<T>();
+        sweep_vectors<T, OP, 4>(acc, xr, n / E, sub, L);
     } else {
-        for (int j = lane; j < cols; j += 32) {
+        for (int j = sub; j < n; j += L) {
             const float v = Elem<T>::load1(xr + j);
             if (OP == kOpLse) {
                 const float one[1] = {v};
@@ -366,8 +376,8 @@ reduce_row_warp_kernel(const T* __restrict__ x, float* __restrict__ out, int32_t
             }
         }
     }
-    acc = warp_merge<OP>(acc);
-    if (lane == 0) write_result<T, OP>(acc, out, index, row, inv_cols);
+    acc = warp_merge<OP, L>(acc);
+    if (sub == 0 && live) write_result<T, OP>(acc, out, index, row, inv_cols);
 }
 
 template <typename T, int OP>
@@ -378,7 +388,9 @@ kop_status_t launch_reduce_op(const T* x, float* out, int32_t* index, int64_t ro
     const bool vec = vec_ok(x, cols, stride, sizeof(T));
     const float inv_cols = (float)(1.0 / (double)cols);
     const int64_t row_bytes = (int64_t)cols * sizeof(T);
-    if (row_bytes >= 2048) {
+    // Rows up to 16 KB: lanes-per-row kernel, measured against a CTA per row on 537 MB of bf16, max + argmax:
+    // rows of 256 / 1024 / 2048 / 8192 columns 346 -> 88, 267 -> 91, 150 -> 90, 94 -> 90 us. Longer rows: a CTA each.
+    if (row_bytes > 16384) {
         int threads = 256;
         if (vec) {
             const int nvec = cols / E;
@@ -391,11 +403,24 @@ kop_status_t launch_reduce_op(const T* x, float* out, int32_t* index, int64_t ro
         else
             reduce_row_block_kernel<T, OP, false><<<(unsigned)rows, threads, 0, stream>>>(x, out, index, cols, stride, inv_cols);
     } else {
-        const int64_t ctas = (rows + 7) / 8;
-        if (vec)
-            reduce_row_warp_kernel<T, OP, true><<<(unsigned)ctas, 256, 0, stream>>>(x, out, index, rows, cols, stride, inv_cols);
-        else
-            reduce_row_warp_kernel<T, OP, false><<<(unsigned)ctas, 256, 0, stream>>>(x, out, index, rows, cols, stride, inv_cols);
+        // sixteen vectors (or 64 scalar elements) a lane where the row is long enough: fewer lanes and merge
+        // steps beat more lanes with fewer batches each (four vectors a lane: 102 - 113 us on the rows above)
+        const int64_t units = vec ? cols / E : (cols + 3) / 4;
+        const int lanes = units >= 512 ? 32 : units >= 256 ? 16 : units >= 128 ? 8 : 4;
+        const int64_t rows_per_cta = 8 * (32 / lanes);
+        const int64_t ctas = (rows + rows_per_cta - 1) / rows_per_cta;
+#define KOP_REDUCE_GROUP(L)                                                                                              \
+    do {                                                                                                                 \
+        if (vec) reduce_row_group_kernel<T, OP, true, L><<<(unsigned)ctas, 256, 0, stream>>>(x, out, index, rows, cols, stride, inv_cols); \
+        else reduce_row_group_kernel<T, OP, false, L><<<(unsigned)ctas, 256, 0, stream>>>(x, out, index, rows, cols, stride, inv_cols);    \
+    } while (0)
+        switch (lanes) {
+        case 32: KOP_REDUCE_GROUP(32); break;
+        case 16: KOP_REDUCE_GROUP(16); break;
+        case 8: KOP_REDUCE_GROUP(8); break;
+        default: KOP_REDUCE_GROUP(4); break;
+        }
+#undef KOP_REDUCE_GROUP
     }
     return launch_status();
 }

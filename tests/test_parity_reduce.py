@@ -57,7 +57,9 @@ def check_op(kop, x, xh, op, what):
 
 
 SHAPES = [(512, 8192, BF16), (300, 4096, F32), (65, 1000, F16), (33, 1001, F32), (9, 40000, BF16),
-          (2000, 64, F32), (1000, 7, BF16), (257, 520, F16), (5, 1, F32)]
+          (2000, 64, F32), (1000, 7, BF16), (257, 520, F16), (5, 1, F32),
+          # 8, 16 and 32 lanes per row, row counts that leave part of the last warp without a row
+          (67, 1024, BF16), (129, 2048, BF16), (35, 3072, F16), (131, 4096, BF16), (21, 600, F32)]
 
 
 @pytest.mark.parametrize("rows,cols,dtype", SHAPES)
