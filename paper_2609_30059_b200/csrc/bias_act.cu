@@ -46,34 +46,49 @@ __device__ __forceinline__ float act_dev(float u, float alpha)
     }
 }
 
-template <typename T, int ACT>
+// kFlat: rows shorter than a tile; the CTA takes U * blockDim.x vectors in row-major order across rows
+// (nvec_total = rows * nvec). Otherwise a CTA is one tile of one row.
+template <typename T, int ACT, bool kFlat>
 __global__ void __launch_bounds__(256)
 bias_act_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* __restrict__ y, int nvec,
-                int tiles_per_row, int64_t x_stride, int64_t y_stride, float alpha)
+                int tiles_per_row, int64_t nvec_total, int64_t x_stride, int64_t y_stride, float alpha)
 {
     constexpr int E = Elem<T>::kPerVec, U = 4;
     constexpr bool kFast = sizeof(T) == 2;
-    const int64_t row = blockIdx.x / tiles_per_row;
-    const int tile = (int)(blockIdx.x - row * tiles_per_row);
-    const T* xr = x + row * x_stride;
-    T* yr = y + row * y_stride;
-    const int v0 = tile * (U * blockDim.x) + threadIdx.x;
+    int64_t row[U];
+    int v[U];
+    bool live[U];
+    if (kFlat) {
+        const int64_t g0 = (int64_t)blockIdx.x * (U * blockDim.x) + threadIdx.x;
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const int64_t g = g0 + k * blockDim.x;
+            live[k] = g < nvec_total;
+            flat_position(live[k] ? g : 0, nvec, &row[k], &v[k]);
+        }
+    } else {
+        const int64_t r = blockIdx.x / tiles_per_row;
+        const int tile = (int)(blockIdx.x - r * tiles_per_row);
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            row[k] = r;
+            v[k] = tile * (U * blockDim.x) + threadIdx.x + k * blockDim.x;
+            live[k] = v[k] < nvec;
+        }
+    }
     Vec16 raw[U];
 #pragma unroll
-    for (int k = 0; k < U; ++k) {
-        const int v = v0 + k * blockDim.x;
-        if (v < nvec) raw[k] = ld_stream(xr + (int64_t)v * E);
-    }
+    for (int k = 0; k < U; ++k)
+        if (live[k]) raw[k] = ld_stream(x + row[k] * x_stride + (int64_t)v[k] * E);
 #pragma unroll
     for (int k = 0; k < U; ++k) {
-        const int v = v0 + k * blockDim.x;
-        if (v < nvec) {
+        if (live[k]) {
             float f[E];
             Elem<T>::unpack(raw[k], f);
             if (bias != nullptr) {
 #pragma unroll
                 for (int q = 0; q < E / 4; ++q) {
-                    const float4 b = ldg_f4(bias + (int64_t)v * E + 4 * q);
+                    const float4 b = ldg_f4(bias + (int64_t)v[k] * E + 4 * q);
                     f[4 * q] += b.x;
                     f[4 * q + 1] += b.y;
                     f[4 * q + 2] += b.z;
@@ -82,7 +97,7 @@ bias_act_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* __re
             }
 #pragma unroll
             for (int e = 0; e < E; ++e) f[e] = act_dev<ACT, kFast>(f[e], alpha);
-            st_stream(yr + (int64_t)v * E, Elem<T>::pack(f));
+            st_stream(y + row[k] * y_stride + (int64_t)v[k] * E, Elem<T>::pack(f));
         }
     }
 }
@@ -115,39 +130,53 @@ __device__ __forceinline__ float chain_value(float x, float b, float r, const Ch
     return u;
 }
 
-template <typename T, int ACT>
+template <typename T, int ACT, bool kFlat>
 __global__ void __launch_bounds__(256)
 chain_kernel(const T* __restrict__ x, const float* __restrict__ bias, const T* __restrict__ res, T* __restrict__ y,
-             int nvec, int tiles_per_row, int64_t x_stride, int64_t r_stride, int64_t y_stride, ChainArgs a)
+             int nvec, int tiles_per_row, int64_t nvec_total, int64_t x_stride, int64_t r_stride, int64_t y_stride,
+             ChainArgs a)
 {
     constexpr int E = Elem<T>::kPerVec, U = 2;
     constexpr bool kFast = sizeof(T) == 2;
-    const int64_t row = blockIdx.x / tiles_per_row;
-    const int tile = (int)(blockIdx.x - row * tiles_per_row);
-    const T* xr = x + row * x_stride;
-    const T* rr = res != nullptr ? res + row * r_stride : nullptr;
-    T* yr = y + row * y_stride;
-    const int v0 = tile * (U * blockDim.x) + threadIdx.x;
+    int64_t row[U];
+    int v[U];
+    bool live[U];
+    if (kFlat) {
+        const int64_t g0 = (int64_t)blockIdx.x * (U * blockDim.x) + threadIdx.x;
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const int64_t g = g0 + k * blockDim.x;
+            live[k] = g < nvec_total;
+            flat_position(live[k] ? g : 0, nvec, &row[k], &v[k]);
+        }
+    } else {
+        const int64_t r = blockIdx.x / tiles_per_row;
+        const int tile = (int)(blockIdx.x - r * tiles_per_row);
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            row[k] = r;
+            v[k] = tile * (U * blockDim.x) + threadIdx.x + k * blockDim.x;
+            live[k] = v[k] < nvec;
+        }
+    }
     Vec16 rx[U], rres[U];
 #pragma unroll
     for (int k = 0; k < U; ++k) {
-        const int v = v0 + k * blockDim.x;
-        if (v < nvec) {
-            rx[k] = ld_stream(xr + (int64_t)v * E);
-            if (rr != nullptr) rres[k] = ld_stream(rr + (int64_t)v * E);
+        if (live[k]) {
+            rx[k] = ld_stream(x + row[k] * x_stride + (int64_t)v[k] * E);
+            if (res != nullptr) rres[k] = ld_stream(res + row[k] * r_stride + (int64_t)v[k] * E);
         }
     }
 #pragma unroll
     for (int k = 0; k < U; ++k) {
-        const int v = v0 + k * blockDim.x;
-        if (v < nvec) {
+        if (live[k]) {
             float f[E], g[E], b[E];
             Elem<T>::unpack(rx[k], f);
-            if (rr != nullptr) Elem<T>::unpack(rres[k], g);
+            if (res != nullptr) Elem<T>::unpack(rres[k], g);
 #pragma unroll
             for (int q = 0; q < E / 4; ++q) {
                 float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (bias != nullptr) t = ldg_f4(bias + (int64_t)v * E + 4 * q);
+                if (bias != nullptr) t = ldg_f4(bias + (int64_t)v[k] * E + 4 * q);
                 b[4 * q] = t.x;
                 b[4 * q + 1] = t.y;
                 b[4 * q + 2] = t.z;
@@ -155,8 +184,8 @@ chain_kernel(const T* __restrict__ x, const float* __restrict__ bias, const T* _
             }
 #pragma unroll
             for (int e = 0; e < E; ++e)
-                f[e] = act_dev<ACT, kFast>(chain_value(f[e], b[e], rr != nullptr ? g[e] : 0.0f, a), a.alpha);
-            st_stream(yr + (int64_t)v * E, Elem<T>::pack(f));
+                f[e] = act_dev<ACT, kFast>(chain_value(f[e], b[e], res != nullptr ? g[e] : 0.0f, a), a.alpha);
+            st_stream(y + row[k] * y_stride + (int64_t)v[k] * E, Elem<T>::pack(f));
         }
     }
 }
@@ -186,12 +215,20 @@ kop_status_t launch_chain_a(const T* x, const float* bias, const T* res, T* y, i
                      (res == nullptr || vec_ok(res, cols, rs, sizeof(T))) && (bias == nullptr || aligned_to(bias, 16));
     if (vec) {
         const int nvec = (int)(cols / E);
+        // a CTA is one tile of one row, sized to the row (32 to 256 threads); rows too short for that, or whose
+        // last tile would be mostly empty, take tiles that cross rows
         int threads = ((nvec + 1) / 2 + 31) / 32 * 32;
         if (threads > 256) threads = 256;
         const int tiles = (nvec + 2 * threads - 1) / (2 * threads);
+        if (nvec < 64 || ((int64_t)tiles * 2 * threads - nvec) * 8 > nvec) {
+            const int64_t total = rows * nvec, grid = (total + 511) / 512;
+            if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+            chain_kernel<T, ACT, true><<<(unsigned)grid, 256, 0, stream>>>(x, bias, res, y, nvec, 1, total, xs, rs, ys, a);
+            return launch_status();
+        }
         const int64_t grid = rows * tiles;
         if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
-        chain_kernel<T, ACT><<<(unsigned)grid, threads, 0, stream>>>(x, bias, res, y, nvec, tiles, xs, rs, ys, a);
+        chain_kernel<T, ACT, false><<<(unsigned)grid, threads, 0, stream>>>(x, bias, res, y, nvec, tiles, 0, xs, rs, ys, a);
         return launch_status();
     }
     int64_t blocks = (rows * cols + 255) / 256;
@@ -241,12 +278,20 @@ kop_status_t launch_bias_act_a(const T* x, const float* bias, T* y, int64_t rows
                      (bias == nullptr || aligned_to(bias, 16));
     if (vec) {
         const int nvec = (int)(cols / E);
+        // a CTA is one tile of one row, sized to the row (32 to 256 threads); rows too short for that, or whose
+        // last tile would be mostly empty, take tiles that cross rows
         int threads = ((nvec + 3) / 4 + 31) / 32 * 32;
         if (threads > 256) threads = 256;
         const int tiles = (nvec + 4 * threads - 1) / (4 * threads);
+        if (nvec < 128 || ((int64_t)tiles * 4 * threads - nvec) * 8 > nvec) {
+            const int64_t total = rows * nvec, grid = (total + 1023) / 1024;
+            if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+            bias_act_kernel<T, ACT, true><<<(unsigned)grid, 256, 0, stream>>>(x, bias, y, nvec, 1, total, xs, ys, alpha);
+            return launch_status();
+        }
         const int64_t grid = rows * tiles;
         if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
-        bias_act_kernel<T, ACT><<<(unsigned)grid, threads, 0, stream>>>(x, bias, y, nvec, tiles, xs, ys, alpha);
+        bias_act_kernel<T, ACT, false><<<(unsigned)grid, threads, 0, stream>>>(x, bias, y, nvec, tiles, 0, xs, ys, alpha);
         return launch_status();
     }
     int64_t blocks = (rows * cols + 255) / 256;

@@ -364,6 +364,21 @@ __device__ __forceinline__ float block_max(float v, float* slots)
 
 #endif  // __CUDACC__
 
+// Rows shorter than a CTA's tile: the vectors of a [rows, nvec] tensor are numbered row after row and a CTA
+// takes a run of them whatever rows they fall in. Position of vector g (g < rows * nvec).
+__device__ __forceinline__ void flat_position(int64_t g, int nvec, int64_t* row, int* v)
+{
+    if (g <= 0xFFFFFFFFLL) {                                 // one 32-bit division
+        const unsigned r = (unsigned)g / (unsigned)nvec;
+        *row = r;
+        *v = (int)((unsigned)g - r * (unsigned)nvec);
+    } else {
+        const int64_t r = g / nvec;
+        *row = r;
+        *v = (int)(g - r * nvec);
+    }
+}
+
 // Parameter vectors stored in a 16-bit data type: the eight that go with one data vector are one 16-byte
 // load (half the bytes and L1 wavefronts of fp32 parameters). kWide has no meaning here.
 template <int E, bool kWide, typename PT>

@@ -102,6 +102,69 @@ rmsnorm_generic_kernel(const T* __restrict__ x, const PT* __restrict__ w, T* __r
     }
 }
 
+// Short rows (at most L * 4 vectors): L lanes of a warp per row (L = 2 .. 32), 32 / L rows per warp, eight warps
+// per CTA, the row in registers; the sum of squares is a butterfly over the row's lanes. A CTA per row would
+// leave most of its one or two warps without data (per-head norms of 64 to 256 columns, small hidden sizes).
+template <typename T, typename PT, int L, bool kRes>
+__global__ void __launch_bounds__(256)
+rmsnorm_group_kernel(const T* __restrict__ x, const PT* __restrict__ w, T* __restrict__ y, int64_t rows, int nvec,
+                     int64_t x_stride, int64_t y_stride, float eps, float inv_hidden, RmsRes rr)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    constexpr int P = E / 2;
+    constexpr int VPL = 4;
+    const int lane = threadIdx.x & 31, sub = lane & (L - 1);
+    const int64_t row = ((int64_t)blockIdx.x * 8 + (threadIdx.x >> 5)) * (32 / L) + lane / L;
+    const bool live = row < rows;
+    const int64_t r = live ? row : 0;
+    const T* xr = x + r * x_stride;
+    const T* resr = kRes ? static_cast<const T*>(rr.res) + r * rr.res_stride : nullptr;
+    T* hr = kRes ? static_cast<T*>(rr.h) + r * rr.h_stride : nullptr;
+    Vec16 raw[VPL], rraw[kRes ? VPL : 1];
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) {
+        const int v = k * L + sub;
+        raw[k] = Vec16{{0u, 0u, 0u, 0u}};
+        if (kRes) rraw[k] = Vec16{{0u, 0u, 0u, 0u}};
+        if (live && v < nvec) {
+            raw[k] = ld_stream(xr + (int64_t)v * E);
+            if (kRes) rraw[k] = ld_stream(resr + (int64_t)v * E);
+        }
+    }
+    float2 val[VPL][P];
+    float2 ss2 = make_float2(0.0f, 0.0f);
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) {
+        Elem<T>::unpack2(raw[k], val[k]);
+        if (kRes) {
+            float2 rv[P];
+            Elem<T>::unpack2(rraw[k], rv);
+#pragma unroll
+            for (int q = 0; q < P; ++q) val[k][q] = __fadd2_rn(val[k][q], rv[q]);
+            const int v = k * L + sub;
+            if (live && v < nvec) st_stream(hr + (int64_t)v * E, Elem<T>::pack2(val[k]));
+        }
+#pragma unroll
+        for (int q = 0; q < P; ++q) ss2 = __ffma2_rn(val[k][q], val[k][q], ss2);
+    }
+    float ss = ss2.x + ss2.y;
+#pragma unroll
+    for (int o = L / 2; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
+    const float rs = rsqrtf(ss * inv_hidden + eps);
+    const float2 r2 = make_float2(rs, rs);
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) {
+        const int v = k * L + sub;
+        if (live && v < nvec) {
+            float2 g[P], o[P];
+            load_params<E, false>(w + (int64_t)v * E, g);
+#pragma unroll
+            for (int q = 0; q < P; ++q) o[q] = __fmul2_rn(__fmul2_rn(val[k][q], r2), g[q]);
+            st_stream(y + r * y_stride + (int64_t)v * E, Elem<T>::pack2(o));
+        }
+    }
+}
+
 // ---- SiLU(gate) * up ------------------------------------------------------------------------------
 // silu(g) = g / (1 + 2^(-g log2e)): one ex2 and one reciprocal. bf16 rows use the approximate
 // reciprocal (relative error ~2^-23, far below the bf16 store step); fp32 rows divide exactly.
@@ -192,6 +255,55 @@ silu_mul_interleaved_kernel(const T* __restrict__ gu, T* __restrict__ out, int n
 #pragma unroll
             for (int e = 0; e < E; ++e) res[e] = silu<kFast>(f[2 * e]) * f[2 * e + 1];
             st_stream(o + (int64_t)v * E, Elem<T>::pack(res));
+        }
+    }
+}
+
+// Rows shorter than a tile (or with a mostly empty last tile), both layouts: the CTA's U * blockDim.x output
+// vectors are taken in row-major order across rows, so no thread idles.
+template <typename T, int U, bool kInterleaved>
+__global__ void __launch_bounds__(128)
+silu_mul_flat_kernel(const T* __restrict__ gu, T* __restrict__ out, int nvec, int64_t nvec_total, int64_t inter,
+                     int64_t in_stride, int64_t out_stride)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    constexpr bool kFast = sizeof(T) == 2;
+    const int64_t g0 = (int64_t)blockIdx.x * (U * blockDim.x) + threadIdx.x;
+    int64_t row[U];
+    int v[U];
+    bool live[U];
+    Vec16 ra[U], rb[U];
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+        const int64_t g = g0 + k * blockDim.x;
+        live[k] = g < nvec_total;
+        flat_position(live[k] ? g : 0, nvec, &row[k], &v[k]);
+        if (live[k]) {
+            const T* p = gu + row[k] * in_stride;
+            ra[k] = ld_stream(kInterleaved ? p + (int64_t)(2 * v[k]) * E : p + (int64_t)v[k] * E);
+            rb[k] = ld_stream(kInterleaved ? p + (int64_t)(2 * v[k] + 1) * E : p + inter + (int64_t)v[k] * E);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+        if (live[k]) {
+            float a[E], b[E], res[E];
+            Elem<T>::unpack(ra[k], a);
+            Elem<T>::unpack(rb[k], b);
+            if (kInterleaved) {
+                float f[2 * E];
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    f[e] = a[e];
+                    f[E + e] = b[e];
+                }
+#pragma unroll
+                for (int e = 0; e < E; ++e) res[e] = silu<kFast>(f[2 * e]) * f[2 * e + 1];
+            } else {
+#pragma unroll
+                for (int e = 0; e < E; ++e) res[e] = silu<kFast>(a[e]) * b[e];
+            }
+            st_stream(out + row[k] * out_stride + (int64_t)v[k] * E, Elem<T>::pack(res));
         }
     }
 }
@@ -297,6 +409,28 @@ kop_status_t launch_rmsnorm(const void* xv, const void* wv, void* yv, int64_t ro
                      (!with_res || (vec_ok(rr.res, hidden, rr.res_stride, sizeof(T)) &&
                                     vec_ok(rr.h, hidden, rr.h_stride, sizeof(T))));
     const int64_t nvec64 = hidden / E;
+    // rows of at most 128 vectors: lanes-per-row kernel (bf16 rows of 64 / 256 / 512 columns ran at 0.5 / 1.9 /
+    // 3.8 TB/s with a CTA per row, 5 - 6 TB/s this way)
+    if (vec && nvec64 <= 128) {
+        const int nvec = (int)nvec64;
+        const int lanes = nvec > 64 ? 32 : nvec > 32 ? 16 : nvec > 16 ? 8 : nvec > 8 ? 4 : 2;
+        const int64_t rows_per_cta = 8 * (32 / lanes);
+        const unsigned grid = (unsigned)((rows + rows_per_cta - 1) / rows_per_cta);
+#define KOP_RMS_GROUP(L)                                                                                                  \
+    do {                                                                                                                  \
+        if (with_res) rmsnorm_group_kernel<T, PT, L, true><<<grid, 256, 0, stream>>>(x, w, y, rows, nvec, xs, ys, eps, inv_hidden, rr); \
+        else rmsnorm_group_kernel<T, PT, L, false><<<grid, 256, 0, stream>>>(x, w, y, rows, nvec, xs, ys, eps, inv_hidden, rr);         \
+    } while (0)
+        switch (lanes) {
+        case 32: KOP_RMS_GROUP(32); break;
+        case 16: KOP_RMS_GROUP(16); break;
+        case 8: KOP_RMS_GROUP(8); break;
+        case 4: KOP_RMS_GROUP(4); break;
+        default: KOP_RMS_GROUP(2); break;
+        }
+#undef KOP_RMS_GROUP
+        return launch_status();
+    }
     if (vec && hidden <= kMaxRegisterRow) {
         const int nvec = (int)nvec64;
         int vals = 32;
@@ -358,6 +492,12 @@ kop_status_t launch_silu_mul(const void* guv, void* outv, int64_t rows, int64_t 
         // (1792 vectors = 7 tiles of 256) exactly.
         constexpr int U = 2;
         const int tiles = (nvec + threads * U - 1) / (threads * U);
+        if (nvec < threads * U || ((int64_t)tiles * threads * U - nvec) * 8 > nvec) {
+            const int64_t total = rows * nvec, fgrid = (total + threads * U - 1) / (threads * U);
+            if (fgrid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+            silu_mul_flat_kernel<T, U, false><<<(unsigned)fgrid, threads, 0, stream>>>(gu, out, nvec, total, inter, is, os);
+            return launch_status();
+        }
         const int64_t grid = rows * tiles;
         if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
         if (nvec % (threads * U) == 0)
@@ -385,6 +525,12 @@ kop_status_t launch_silu_mul_interleaved(const void* guv, void* outv, int64_t ro
         const int threads = 128;
         constexpr int U = 2;
         const int tiles = (nvec + threads * U - 1) / (threads * U);
+        if (nvec < threads * U || ((int64_t)tiles * threads * U - nvec) * 8 > nvec) {
+            const int64_t total = rows * nvec, fgrid = (total + threads * U - 1) / (threads * U);
+            if (fgrid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+            silu_mul_flat_kernel<T, U, true><<<(unsigned)fgrid, threads, 0, stream>>>(gu, out, nvec, total, inter, is, os);
+            return launch_status();
+        }
         const int64_t grid = rows * tiles;
         if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
         if (nvec % (threads * U) == 0)

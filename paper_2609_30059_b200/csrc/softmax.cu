@@ -14,23 +14,29 @@ namespace {
 // (A grid-stride version with the bias held in registers across rows measured 8 % slower on
 // [131072, 512] fp32: many short-lived CTAs at different phases overlap loads, math and stores better
 // than a few resident warps that each serialise them.)
-// kFull: the row is exactly 32 * VPL vectors (no tail predicates); kBias: bias != NULL.
-template <typename T, int VPL, bool kFull, bool kBias>
+// kFull: the row is exactly L * VPL vectors (no tail predicates); kBias: bias != NULL. L: lanes per row (32, or
+// 2 .. 16 for rows of fewer than 32 vectors, 32 / L rows per warp: attention scores and class logits of 64 to
+// 256 columns would leave most of a warp idle otherwise).
+template <typename T, int VPL, bool kFull, bool kBias, int L = 32>
 __global__ void __launch_bounds__(256)
 softmax_warp_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* __restrict__ y,
                     int64_t rows, int nvec, int64_t x_stride, int64_t y_stride, float scale)
 {
     constexpr int E = Elem<T>::kPerVec;
-    const int lane = threadIdx.x & 31;
-    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (row >= rows) return;
+    const int lane = L == 32 ? (threadIdx.x & 31) : (threadIdx.x & (L - 1));
+    int64_t row = ((int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * (32 / L) + (threadIdx.x & 31) / L;
+    if (L == 32 && row >= rows) return;                      // whole warps leave together
+    // narrower groups: a group past the end reads the last row again and stores nothing, so that its lanes
+    // still take part in the shuffles
+    const bool live = row < rows;
+    if (!live) row = rows - 1;
     const float s2 = scale * kLog2e;
     const T* xr = x + row * x_stride;
     T* yr = y + row * y_stride;
     Vec16 raw[VPL];
 #pragma unroll
     for (int k = 0; k < VPL; ++k) {
-        const int v = k * 32 + lane;
+        const int v = k * L + lane;
         if (kFull || v < nvec) raw[k] = ld_stream(xr + (int64_t)v * E);
         else raw[k] = Vec16{{0u, 0u, 0u, 0u}};
     }
@@ -38,7 +44,7 @@ softmax_warp_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* 
     float m = -INFINITY;
 #pragma unroll
     for (int k = 0; k < VPL; ++k) {
-        const int v = k * 32 + lane;
+        const int v = k * L + lane;
         float f[E];
         Elem<T>::unpack(raw[k], f);
 #pragma unroll
@@ -54,7 +60,8 @@ softmax_warp_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* 
             }
         }
     }
-    m = warp_max(m);
+#pragma unroll
+    for (int o = L / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
     float s = 0.0f;
 #pragma unroll
     for (int k = 0; k < VPL; ++k)
@@ -63,15 +70,16 @@ softmax_warp_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* 
             t[k][e] = ex2_approx(t[k][e] - m);
             s += t[k][e];
         }
-    s = warp_sum(s);
+#pragma unroll
+    for (int o = L / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
     const float inv = 1.0f / s;
 #pragma unroll
     for (int k = 0; k < VPL; ++k) {
-        const int v = k * 32 + lane;
+        const int v = k * L + lane;
         float o[E];
 #pragma unroll
         for (int e = 0; e < E; ++e) o[e] = t[k][e] * inv;
-        if (kFull || v < nvec) st_stream(yr + (int64_t)v * E, Elem<T>::pack(o));
+        if (live && (kFull || v < nvec)) st_stream(yr + (int64_t)v * E, Elem<T>::pack(o));
     }
 }
 
@@ -199,6 +207,29 @@ kop_status_t launch_softmax(const void* xv, const float* bias, void* yv, int64_t
     const bool vec = vec_ok(x, cols, xs, sizeof(T)) && vec_ok(y, cols, ys, sizeof(T)) &&
                      (bias == nullptr || aligned_to(bias, 16));
     const int64_t nvec64 = cols / E;
+    if (vec && nvec64 < 32 && !with_opts) {                  // fewer than 32 vectors: 2 to 8 lanes per row, four vectors each
+        const int nvec = (int)nvec64;
+        const int lanes = nvec > 16 ? 8 : nvec > 8 ? 4 : 2;
+        const int64_t rows_per_cta = 8 * (32 / lanes);
+        const int64_t ctas = (rows + rows_per_cta - 1) / rows_per_cta;
+        if (ctas > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+        const unsigned grid = (unsigned)ctas;
+        const bool full = nvec == lanes * 4;
+#define KOP_SM_GROUP_L(F, B, L) softmax_warp_kernel<T, 4, F, B, L><<<grid, 256, 0, stream>>>(x, bias, y, rows, nvec, xs, ys, scale)
+#define KOP_SM_GROUP(L)                                                         \
+    do {                                                                        \
+        if (full && bias != nullptr) KOP_SM_GROUP_L(true, true, L);             \
+        else if (full) KOP_SM_GROUP_L(true, false, L);                          \
+        else if (bias != nullptr) KOP_SM_GROUP_L(false, true, L);               \
+        else KOP_SM_GROUP_L(false, false, L);                                   \
+    } while (0)
+        if (lanes == 8) KOP_SM_GROUP(8);
+        else if (lanes == 4) KOP_SM_GROUP(4);
+        else KOP_SM_GROUP(2);
+#undef KOP_SM_GROUP_L
+#undef KOP_SM_GROUP
+        return launch_status();
+    }
     if (vec && nvec64 <= 32 * 4 && !with_opts) {
         const int nvec = (int)nvec64;
         const int vpl = (nvec + 31) / 32;
