@@ -237,26 +237,6 @@ kop_status_t launch_bn(const void* xv, const float* scale, const float* shift, v
 // writes its column sums into the first CTA's shared memory (distributed shared memory), one cluster
 // barrier, and the first CTA adds them in rank order. No atomics, no workspace, and for a given call
 // shape a fixed summation order.
-__device__ __forceinline__ uint32_t cluster_rank()
-{
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-
-__device__ __forceinline__ void store_to_cluster_cta(float* local_slot, uint32_t cta, float v)
-{
-    const uint32_t la = (uint32_t)__cvta_generic_to_shared(local_slot);
-    uint32_t ra;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(la), "r"(cta));
-    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(ra), "f"(v) : "memory");
-}
-
-__device__ __forceinline__ void cluster_barrier()
-{
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-
 constexpr int kBnMaxSlabs = 8;      // portable cluster size
 
 template <typename T, int TV, int U, bool kCluster>

@@ -362,7 +362,6 @@ __device__ __forceinline__ float block_max(float v, float* slots)
     return warp_max(t);
 }
 
-#endif  // __CUDACC__
 
 // Rows shorter than a CTA's tile: the vectors of a [rows, nvec] tensor are numbered row after row and a CTA
 // takes a run of them whatever rows they fall in. Position of vector g (g < rows * nvec).
@@ -392,5 +391,28 @@ __device__ __forceinline__ void load_params(const PT* p, float2 (&out)[E / 2])
 __device__ __forceinline__ float param1(const float* p, int64_t j) { return __ldg(p + j); }
 __device__ __forceinline__ float param1(const __nv_bfloat16* p, int64_t j) { return Elem<__nv_bfloat16>::load1(p + j); }
 __device__ __forceinline__ float param1(const __half* p, int64_t j) { return Elem<__half>::load1(p + j); }
+
+// ---- thread-block clusters: distributed shared memory between the CTAs of a cluster ----------------------
+__device__ __forceinline__ uint32_t cluster_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+
+__device__ __forceinline__ void store_to_cluster_cta(float* local_slot, uint32_t cta, float v)
+{
+    const uint32_t la = (uint32_t)__cvta_generic_to_shared(local_slot);
+    uint32_t ra;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(la), "r"(cta));
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(ra), "f"(v) : "memory");
+}
+
+__device__ __forceinline__ void cluster_barrier()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+#endif  // __CUDACC__
 
 }  // namespace kop

@@ -40,7 +40,14 @@ SOFTMAX_SHAPES = [
     (333, 96, F32),        # partial last vector group in the warp
     (257, 2048, F32),      # CTA-per-row, row in registers
     (19, 16384, F32),      # longest register-resident row
-    (7, 20000, F32),       # beyond registers: generic
+    (7, 20000, F32),       # beyond one CTA's registers: two sweeps with vector loads
+    (5, 40000, BF16),
+    (3, 131072, BF16),
+    (2, 100000, F32),
+    (3, 128256, BF16),     # a vocabulary size
+    (2, 140008, BF16),
+    (9, 12288, F32),       # fp32 rows beyond 32 KB: two sweeps although the row would fit the registers
+    (3, 20001, BF16),      # odd length: the scalar three-sweep kernel
     (37, 513, F32),        # odd length: scalar
     (64, 1, F32),
     (515, 1000, BF16),
@@ -365,7 +372,7 @@ def assert_close_with_neg_inf(got, ref, tol, what):
 
 
 @pytest.mark.parametrize("rows,cols,dtype", [(96, 512, F32), (1024, 128, BF16), (130, 1000, F32), (66, 1001, F32),
-                                             (20, 16384, BF16), (12, 20000, F32), (9, 1, F32)])
+                                             (20, 16384, BF16), (12, 20000, F32), (9, 1, F32), (4, 50000, BF16)])
 @pytest.mark.parametrize("seed", SEEDS)
 def test_softmax_opts_parity(kop, rows, cols, dtype, seed):
     x, bias = synth.softmax_inputs(rows, cols, dtype, seed, "cuda")
