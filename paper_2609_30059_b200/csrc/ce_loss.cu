@@ -79,46 +79,16 @@ __device__ __forceinline__ int warp_sum_int(int v)
     return v;
 }
 
-// Merge the per-thread (M, S) pairs and finish the row; then the mean, without anybody waiting:
-// only warp 0 stays. Its lane 0 takes a ticket of the row's group (kGroupRows consecutive rows);
-// the warp that draws a group's last ticket sums that group's losses in a fixed lane-strided order
-// and takes a global ticket; the warp that draws the last global ticket sums the group partials,
-// again in a fixed order. Which CTA does the summing varies, the order of the additions does not,
-// so the mean is bit-identical run to run. (A whole-CTA wait on a single ticket held every CTA's
-// registers for an extra L2 round trip and cost 12 % on the benchmark shape.)
-template <typename T, bool kOpts, bool kSmooth>
-__device__ __forceinline__ void ce_finish(float M, float S, float Z, const T* zr, const int32_t* labels,
-                                          float* loss, float* mean_loss, int32_t* bad_label_count,
-                                          CeWorkspace ws, int64_t row, int64_t rows, int64_t vocab,
-                                          CeOpts opts)
+// What a whole warp does once its row's ticket `t` is known (the same value in all 32 lanes): nothing unless
+// it was the group's last ticket.
+template <bool kOpts>
+__device__ __forceinline__ void ce_after_ticket(unsigned t, int64_t row, int lane, const int32_t* labels, float* loss,
+                                                float* mean_loss, int32_t* bad_label_count, CeWorkspace ws,
+                                                int64_t rows, int64_t vocab, CeOpts opts)
 {
-    __shared__ float red_a[32], red_b[32], red_c[32];
-    const float Mb = block_max(M, red_a);
-    // A thread that saw nothing has M = -inf and S = 0; keep its term at 0 rather than 0 * 2^nan.
-    const float Sb = block_sum(M == -INFINITY ? 0.0f : S * ex2_approx(M - Mb), red_b);
-    float Zb = 0.0f;
-    if (kSmooth) Zb = block_sum(Z, red_c);          // sum of the row's logits, for label smoothing
-    if (threadIdx.x >= 32) return;
-    const int lane = threadIdx.x;
     const int64_t g = row / kGroupRows;
     const int64_t g0 = g * kGroupRows;
     const int gsize = (int)(rows - g0 < kGroupRows ? rows - g0 : kGroupRows);
-    unsigned t = 0;
-    if (lane == 0) {
-        const float lse = (Mb + log2f(Sb)) * kLn2;
-        const int32_t lab = labels[row];
-        float l;
-        if (kOpts && lab == opts.ignore_index) l = 0.0f;
-        else if (lab < 0 || (int64_t)lab >= vocab) l = __int_as_float(0x7FC00000);
-        else {
-            l = lse - Elem<T>::load1(zr + lab);
-            if (kSmooth) l = (1.0f - opts.smoothing) * l + opts.smoothing * (lse - Zb / (float)vocab);
-        }
-        loss[row] = l;
-        __threadfence();
-        t = atomicAdd(ws.group_ticket + g, 1u);
-    }
-    t = __shfl_sync(0xFFFFFFFFu, t, 0);
     if (t != (unsigned)(gsize - 1)) return;
     __threadfence();
     float acc = 0.0f;
@@ -167,6 +137,47 @@ __device__ __forceinline__ void ce_finish(float M, float S, float Z, const T* zr
         if (bad_label_count != nullptr)
             *bad_label_count = (int32_t)(nbad > 0x7FFFFFFF ? 0x7FFFFFFF : nbad);
     }
+}
+
+// Merge the per-thread (M, S) pairs and finish the row; then the mean, without anybody waiting:
+// only warp 0 stays. Its lane 0 takes a ticket of the row's group (kGroupRows consecutive rows);
+// the warp that draws a group's last ticket sums that group's losses in a fixed lane-strided order
+// and takes a global ticket; the warp that draws the last global ticket sums the group partials,
+// again in a fixed order. Which CTA does the summing varies, the order of the additions does not,
+// so the mean is bit-identical run to run. (A whole-CTA wait on a single ticket held every CTA's
+// registers for an extra L2 round trip and cost 12 % on the benchmark shape.)
+template <typename T, bool kOpts, bool kSmooth>
+__device__ __forceinline__ void ce_finish(float M, float S, float Z, const T* zr, const int32_t* labels,
+                                          float* loss, float* mean_loss, int32_t* bad_label_count,
+                                          CeWorkspace ws, int64_t row, int64_t rows, int64_t vocab,
+                                          CeOpts opts)
+{
+    __shared__ float red_a[32], red_b[32], red_c[32];
+    const float Mb = block_max(M, red_a);
+    // A thread that saw nothing has M = -inf and S = 0; keep its term at 0 rather than 0 * 2^nan.
+    const float Sb = block_sum(M == -INFINITY ? 0.0f : S * ex2_approx(M - Mb), red_b);
+    float Zb = 0.0f;
+    if (kSmooth) Zb = block_sum(Z, red_c);          // sum of the row's logits, for label smoothing
+    if (threadIdx.x >= 32) return;
+    const int lane = threadIdx.x;
+    const int64_t g = row / kGroupRows;
+    unsigned t = 0;
+    if (lane == 0) {
+        const float lse = (Mb + log2f(Sb)) * kLn2;
+        const int32_t lab = labels[row];
+        float l;
+        if (kOpts && lab == opts.ignore_index) l = 0.0f;
+        else if (lab < 0 || (int64_t)lab >= vocab) l = __int_as_float(0x7FC00000);
+        else {
+            l = lse - Elem<T>::load1(zr + lab);
+            if (kSmooth) l = (1.0f - opts.smoothing) * l + opts.smoothing * (lse - Zb / (float)vocab);
+        }
+        loss[row] = l;
+        __threadfence();
+        t = atomicAdd(ws.group_ticket + g, 1u);
+    }
+    t = __shfl_sync(0xFFFFFFFFu, t, 0);
+    ce_after_ticket<kOpts>(t, row, lane, labels, loss, mean_loss, bad_label_count, ws, rows, vocab, opts);
 }
 
 // One batch of VPT vectors per thread: loads first (all in flight), then the batch maximum on the
@@ -234,6 +245,93 @@ ce_row_kernel(const T* __restrict__ z, const int32_t* __restrict__ labels, float
     ce_finish<T, kOpts, kSmooth>(M, S, Z, zr, labels, loss, mean_loss, bad_label_count, ws, row, rows, vocab, opts);
 }
 
+// Rows of at most 16 KB (classification heads, small vocabularies): L lanes of a warp per row (L = 4 .. 32),
+// 32 / L rows per warp, eight warps per CTA. Each lane sweeps its share in batches of four vectors with the
+// same recurrence as above; the row's (maximum, sum) pair is a butterfly over its lanes; the row's first lane
+// writes the loss and draws the ticket, and the warp then walks its rows so that whichever drew a group's
+// last ticket has all 32 lanes for the group sum, exactly as in the CTA-per-row kernel.
+template <typename T, int L, bool kOpts, bool kSmooth>
+__global__ void __launch_bounds__(256)
+ce_group_kernel(const T* __restrict__ z, const int32_t* __restrict__ labels, float* __restrict__ loss,
+                float* __restrict__ mean_loss, int32_t* __restrict__ bad_label_count, CeWorkspace ws,
+                int64_t rows, int nvec, int64_t row_stride, int64_t vocab, CeOpts opts)
+{
+    constexpr int E = Elem<T>::kPerVec, U = 4;
+    constexpr int kRowsPerWarp = 32 / L;
+    const int lane = threadIdx.x & 31, sub = lane & (L - 1);
+    const int64_t warp_row0 = ((int64_t)blockIdx.x * 8 + (threadIdx.x >> 5)) * kRowsPerWarp;
+    const int64_t row = warp_row0 + lane / L;
+    const bool live = row < rows;
+    const T* zr = z + (live ? row : 0) * row_stride;
+    int n = live ? nvec : 0;
+    if (kOpts && live && __ldg(labels + row) == opts.ignore_index) n = 0;     // an ignored row is not read
+    float M = -INFINITY, S = 0.0f, Z = 0.0f;
+    for (int base = 0; base < n; base += U * L) {
+        Vec16 raw[U];
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const int v = base + k * L + sub;
+            raw[k] = Elem<T>::fill_neg_inf();
+            if (v < n) raw[k] = ld_stream(zr + (int64_t)v * E);
+        }
+        float cm = vec_max<T>(raw[0]);
+#pragma unroll
+        for (int k = 1; k < U; ++k) cm = fmaxf(cm, vec_max<T>(raw[k]));
+        const float cm2 = cm * kLog2e;
+        if (cm2 > -INFINITY) {
+            const float newM = fmaxf(M, cm2);
+            float s = S * ex2_approx(M - newM);
+            const float neg = -newM;
+#pragma unroll
+            for (int k = 0; k < U; ++k) {
+                float f[E];
+                Elem<T>::unpack(raw[k], f);
+#pragma unroll
+                for (int e = 0; e < E; ++e) s += ex2_approx(fmaf(f[e], kLog2e, neg));
+                if (kSmooth && base + k * L + sub < n) {
+#pragma unroll
+                    for (int e = 0; e < E; e += 2) Z += f[e] + f[e + 1];
+                }
+            }
+            S = s;
+            M = newM;
+        }
+    }
+    // the row's lanes: butterfly merge of (M, S) and of Z
+#pragma unroll
+    for (int o = L / 2; o > 0; o >>= 1) {
+        const float Mo = __shfl_xor_sync(0xFFFFFFFFu, M, o), So = __shfl_xor_sync(0xFFFFFFFFu, S, o);
+        const float M2 = fmaxf(M, Mo);
+        const float a = M == -INFINITY ? 0.0f : S * ex2_approx(M - M2);
+        const float b = Mo == -INFINITY ? 0.0f : So * ex2_approx(Mo - M2);
+        // the lower lane's term first on both sides, so that the two lanes agree bit for bit
+        S = (lane & o) ? b + a : a + b;
+        M = M2;
+        if (kSmooth) Z += __shfl_xor_sync(0xFFFFFFFFu, Z, o);
+    }
+    unsigned t = 0xFFFFFFFFu;
+    if (live && sub == 0) {
+        const float lse = (M + log2f(S)) * kLn2;
+        const int32_t lab = labels[row];
+        float l;
+        if (kOpts && lab == opts.ignore_index) l = 0.0f;
+        else if (lab < 0 || (int64_t)lab >= vocab) l = __int_as_float(0x7FC00000);
+        else {
+            l = lse - Elem<T>::load1(zr + lab);
+            if (kSmooth) l = (1.0f - opts.smoothing) * l + opts.smoothing * (lse - Z / (float)vocab);
+        }
+        loss[row] = l;
+        __threadfence();
+        t = atomicAdd(ws.group_ticket + row / kGroupRows, 1u);
+    }
+#pragma unroll
+    for (int r = 0; r < kRowsPerWarp; ++r) {
+        const unsigned tr = __shfl_sync(0xFFFFFFFFu, t, r * L);
+        if (warp_row0 + r < rows)                            // uniform over the warp
+            ce_after_ticket<kOpts>(tr, warp_row0 + r, lane, labels, loss, mean_loss, bad_label_count, ws, rows, vocab, opts);
+    }
+}
+
 // Any vocab / alignment: scalar loads, element-wise online recurrence.
 template <typename T, bool kOpts>
 __global__ void __launch_bounds__(256)
@@ -272,6 +370,27 @@ kop_status_t launch_ce(const void* zv, const int32_t* labels, float* loss, float
     if (cudaMemsetAsync(workspace, 0, ce_workspace_clear_bytes(rows), stream) != cudaSuccess) return KOP_ERR_CUDA;
     const bool vec = vec_ok(z, vocab, stride, sizeof(T));
     const int64_t nvec64 = vocab / E;
+    if (vec && vocab * (int64_t)sizeof(T) <= 16384) {
+        const int nvec = (int)nvec64;
+        const int lanes = nvec >= 512 ? 32 : nvec >= 256 ? 16 : nvec >= 128 ? 8 : 4;
+        const int64_t rows_per_cta = 8 * (32 / lanes);
+        const unsigned grid = (unsigned)((rows + rows_per_cta - 1) / rows_per_cta);
+#define KOP_CE_G(L, SM) ce_group_kernel<T, L, kOpts, SM><<<grid, 256, 0, stream>>>(z, labels, loss, mean_loss, bad, ws, rows, nvec, stride, vocab, opts)
+#define KOP_CE_GROUP(L)                                            \
+    do {                                                           \
+        if (kOpts && opts.smoothing > 0.0f) KOP_CE_G(L, true);     \
+        else KOP_CE_G(L, false);                                   \
+    } while (0)
+        switch (lanes) {
+        case 32: KOP_CE_GROUP(32); break;
+        case 16: KOP_CE_GROUP(16); break;
+        case 8: KOP_CE_GROUP(8); break;
+        default: KOP_CE_GROUP(4); break;
+        }
+#undef KOP_CE_G
+#undef KOP_CE_GROUP
+        return launch_status();
+    }
     if (vec && nvec64 <= 0x7FFFFFFF) {
         const int nvec = (int)nvec64;
         const int threads = 256;

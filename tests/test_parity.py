@@ -422,6 +422,16 @@ CE_SHAPES = [
     (21, 32001, BF16),     # odd vocab: scalar
     (9, 1, F32),
     (5, 8, BF16),
+    # small vocabularies (rows of at most 16 KB): 4, 8, 16 and 32 lanes of a warp per row; row counts that span
+    # several ticket groups and leave part of the last warp without a row
+    (3001, 16, BF16),
+    (1025, 1000, BF16),
+    (777, 1024, BF16),
+    (515, 2048, BF16),
+    (259, 4096, F32),
+    (70, 8192, BF16),
+    (1031, 100, F32),
+    (600, 1000, torch.float16),
 ]
 
 
@@ -721,7 +731,8 @@ def test_silu_mul_interleaved_parity(kop, rows, inter, dtype, seed):
     assert torch.equal(out.t, kop.kop_silu_mul(split))
 
 
-@pytest.mark.parametrize("rows,vocab,dtype", [(2048, 32000, BF16), (300, 4096, F32), (257, 50264, BF16), (21, 32001, BF16), (9, 8, F32)])
+@pytest.mark.parametrize("rows,vocab,dtype", [(2048, 32000, BF16), (300, 4096, F32), (257, 50264, BF16), (21, 32001, BF16), (9, 8, F32),
+                                              (1300, 1000, BF16), (523, 2048, BF16), (2051, 40, F32), (67, 8192, BF16)])
 @pytest.mark.parametrize("smoothing", [0.0, 0.1])
 @pytest.mark.parametrize("seed", SEEDS[:3])
 def test_ce_opts_parity(kop, rows, vocab, dtype, smoothing, seed):
