@@ -60,6 +60,10 @@ SCAN_SHAPES = [
     (37, 1001, F32),       # scalar kernel (1001 % 4 != 0)
     (21, 1003, BF16),      # scalar kernel bf16
     (7, 1, F32),           # single column
+    # short rows: 1, 2, 4, 8, 16 and 32 lanes of a warp per row; row counts that leave lanes without a row
+    (1031, 16, F32), (515, 32, F32), (259, 64, BF16), (131, 136, BF16), (67, 256, F32), (35, 512, BF16),
+    (19, 1024, BF16), (1025, 8, BF16), (77, 100, F32),
+    (41, 1032, BF16), (13, 8192, BF16), (11, 16384, torch.float16), (9, 16392, BF16),   # a warp per row with a carry; just beyond it
     (4, 3, BF16),
 ]
 
