@@ -220,7 +220,7 @@ kop_status_t launch_chain_a(const T* x, const float* bias, const T* res, T* y, i
         int threads = ((nvec + 1) / 2 + 31) / 32 * 32;
         if (threads > 256) threads = 256;
         const int tiles = (nvec + 2 * threads - 1) / (2 * threads);
-        if (nvec < 64 || ((int64_t)tiles * 2 * threads - nvec) * 8 > nvec) {
+        if (nvec < 64 || ((int64_t)tiles * 2 * threads - nvec) * 4 > nvec) {
             const int64_t total = rows * nvec, grid = (total + 511) / 512;
             if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
             chain_kernel<T, ACT, true><<<(unsigned)grid, 256, 0, stream>>>(x, bias, res, y, nvec, 1, total, xs, rs, ys, a);
@@ -283,7 +283,7 @@ kop_status_t launch_bias_act_a(const T* x, const float* bias, T* y, int64_t rows
         int threads = ((nvec + 3) / 4 + 31) / 32 * 32;
         if (threads > 256) threads = 256;
         const int tiles = (nvec + 4 * threads - 1) / (4 * threads);
-        if (nvec < 128 || ((int64_t)tiles * 4 * threads - nvec) * 8 > nvec) {
+        if (nvec < 128 || ((int64_t)tiles * 4 * threads - nvec) * 4 > nvec) {
             const int64_t total = rows * nvec, grid = (total + 1023) / 1024;
             if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
             bias_act_kernel<T, ACT, true><<<(unsigned)grid, 256, 0, stream>>>(x, bias, y, nvec, 1, total, xs, ys, alpha);
