@@ -358,6 +358,108 @@ ln_group_kernel(const T* __restrict__ x, const T* __restrict__ res, const PT* __
     }
 }
 
+// Rows beyond one CTA's registers, vector loads, three sweeps (sum; centred squares, walking backwards over
+// what the first sweep left in the L2; output, forwards again). v is recomputed from the inputs in each
+// sweep, and y is written only in the last one by the thread that read the same position, so exact aliasing
+// stays safe.
+template <typename T, typename PT, int PRO>
+__global__ void __launch_bounds__(512)
+ln_long_kernel(const T* __restrict__ x, const T* __restrict__ res, const PT* __restrict__ bias,
+               const PT* __restrict__ gamma, const PT* __restrict__ beta, T* __restrict__ y,
+               float* __restrict__ mean, float* __restrict__ rstd, int nvec, int64_t x_stride, int64_t r_stride,
+               int64_t y_stride, float eps, float inv_hidden)
+{
+    constexpr int E = Elem<T>::kPerVec, P = E / 2, U = 4;
+    constexpr bool kFast = sizeof(T) == 2;
+    __shared__ float red_a[32], red_b[32];
+    const int64_t row = blockIdx.x;
+    const T* xr = x + row * x_stride;
+    const T* rr = res + row * r_stride;
+    T* yr = y + row * y_stride;
+    const int step = U * blockDim.x;
+    const int nbatch = (nvec + step - 1) / step;
+
+    // the U vectors of batch b that belong to this thread, as v = prologue(x, bias, residual); false past the end
+    auto load_batch = [&](int b, float2 (&val)[U][P], bool (&in)[U]) {
+        Vec16 rx[U], rres[U];
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const int v = b * step + k * blockDim.x + threadIdx.x;
+            in[k] = v < nvec;
+            rx[k] = Vec16{{0u, 0u, 0u, 0u}};
+            rres[k] = Vec16{{0u, 0u, 0u, 0u}};
+            if (in[k]) {
+                rx[k] = ld_stream(xr + (int64_t)v * E);
+                if (pro_has_residual(PRO)) rres[k] = ld_stream(rr + (int64_t)v * E);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const int v = b * step + k * blockDim.x + threadIdx.x;
+            float2 bb[P], fx[P], fr[P];
+            if (pro_has_bias(PRO) && in[k]) load_params<E, false>(bias + (int64_t)v * E, bb);
+            else {
+#pragma unroll
+                for (int q = 0; q < P; ++q) bb[q] = make_float2(0.0f, 0.0f);
+            }
+            Elem<T>::unpack2(rx[k], fx);
+            Elem<T>::unpack2(rres[k], fr);
+#pragma unroll
+            for (int q = 0; q < P; ++q) val[k][q] = prologue2<PRO, kFast>(fx[q], bb[q], fr[q]);
+        }
+    };
+
+    float2 sum2 = make_float2(0.0f, 0.0f);
+    for (int b = 0; b < nbatch; ++b) {
+        float2 val[U][P];
+        bool in[U];
+        load_batch(b, val, in);
+#pragma unroll
+        for (int k = 0; k < U; ++k)
+#pragma unroll
+            for (int q = 0; q < P; ++q)
+                if (in[k]) sum2 = __fadd2_rn(sum2, val[k][q]);
+    }
+    const float mu = block_sum(sum2.x + sum2.y, red_a) * inv_hidden;
+    const float2 nmu = make_float2(-mu, -mu);
+    float2 ss2 = make_float2(0.0f, 0.0f);
+    for (int b = nbatch - 1; b >= 0; --b) {
+        float2 val[U][P];
+        bool in[U];
+        load_batch(b, val, in);
+#pragma unroll
+        for (int k = 0; k < U; ++k)
+#pragma unroll
+            for (int q = 0; q < P; ++q) {
+                const float2 d = __fadd2_rn(val[k][q], nmu);
+                if (in[k]) ss2 = __ffma2_rn(d, d, ss2);
+            }
+    }
+    const float rs = rsqrtf(block_sum(ss2.x + ss2.y, red_b) * inv_hidden + eps);
+    if (threadIdx.x == 0) {
+        if (mean != nullptr) mean[row] = mu;
+        if (rstd != nullptr) rstd[row] = rs;
+    }
+    const float2 rs2 = make_float2(rs, rs);
+    for (int b = 0; b < nbatch; ++b) {
+        float2 val[U][P];
+        bool in[U];
+        load_batch(b, val, in);
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const int v = b * step + k * blockDim.x + threadIdx.x;
+            if (in[k]) {
+                float2 g[P], be[P], o[P];
+                load_params<E, false>(gamma + (int64_t)v * E, g);
+                load_params<E, false>(beta + (int64_t)v * E, be);
+#pragma unroll
+                for (int q = 0; q < P; ++q) o[q] = __ffma2_rn(__fmul2_rn(__fadd2_rn(val[k][q], nmu), rs2), g[q], be[q]);
+                st_stream(yr + (int64_t)v * E, Elem<T>::pack2(o));
+            }
+        }
+    }
+}
+
 // Any hidden size / alignment: scalar loads, v recomputed in each of three sweeps.
 template <typename T, typename PT, int PRO, bool kFast>
 __device__ __forceinline__ float ln_value(const T* xr, const T* rr, const PT* bias, int64_t j)
@@ -492,6 +594,11 @@ kop_status_t launch_ln(const void* xv, const void* rv, const void* biasv, const 
         }
 #undef KOP_LN_LAUNCH
 #undef KOP_LN
+        return launch_status();
+    }
+    if (vec && nvec64 <= 0x7FFFFFFF) {
+        ln_long_kernel<T, PT, PRO><<<(unsigned)rows, 512, 0, stream>>>(x, r, bias, gamma, beta, y, mean, rstd, (int)nvec64,
+                                                                      xs, rs, ys, eps, inv_hidden);
         return launch_status();
     }
     ln_generic_kernel<T, PT, PRO><<<(unsigned)rows, 256, 0, stream>>>(x, r, bias, gamma, beta, y, mean, rstd,

@@ -165,6 +165,84 @@ rmsnorm_group_kernel(const T* __restrict__ x, const PT* __restrict__ w, T* __res
     }
 }
 
+// Rows beyond one CTA's registers, vector loads, two sweeps: the sum of squares forwards, then the output
+// backwards (what the first sweep left in the L2 is read first). With a residual the sum v = x + residual is
+// formed again in the second sweep from the inputs, which the same thread overwrites only afterwards.
+template <typename T, typename PT, bool kRes>
+__global__ void __launch_bounds__(512)
+rmsnorm_long_kernel(const T* __restrict__ x, const PT* __restrict__ w, T* __restrict__ y, int nvec, int64_t x_stride,
+                    int64_t y_stride, float eps, float inv_hidden, RmsRes rr)
+{
+    constexpr int E = Elem<T>::kPerVec, P = E / 2, U = 4;
+    __shared__ float red[32];
+    const int64_t row = blockIdx.x;
+    const T* xr = x + row * x_stride;
+    T* yr = y + row * y_stride;
+    const T* resr = kRes ? static_cast<const T*>(rr.res) + row * rr.res_stride : nullptr;
+    T* hr = kRes ? static_cast<T*>(rr.h) + row * rr.h_stride : nullptr;
+    const int step = U * blockDim.x;
+    const int nbatch = (nvec + step - 1) / step;
+    float2 ss2 = make_float2(0.0f, 0.0f);
+    for (int b = 0; b < nbatch; ++b) {
+        Vec16 raw[U], rraw[kRes ? U : 1];
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const int v = b * step + k * blockDim.x + threadIdx.x;
+            raw[k] = Vec16{{0u, 0u, 0u, 0u}};
+            if (kRes) rraw[k] = Vec16{{0u, 0u, 0u, 0u}};
+            if (v < nvec) {
+                raw[k] = ld_stream(xr + (int64_t)v * E);
+                if (kRes) rraw[k] = ld_stream(resr + (int64_t)v * E);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            float2 val[P];
+            Elem<T>::unpack2(raw[k], val);
+            if (kRes) {
+                float2 rv[P];
+                Elem<T>::unpack2(rraw[k], rv);
+#pragma unroll
+                for (int q = 0; q < P; ++q) val[q] = __fadd2_rn(val[q], rv[q]);
+            }
+#pragma unroll
+            for (int q = 0; q < P; ++q) ss2 = __ffma2_rn(val[q], val[q], ss2);
+        }
+    }
+    const float r = rsqrtf(block_sum(ss2.x + ss2.y, red) * inv_hidden + eps);
+    const float2 r2 = make_float2(r, r);
+    for (int b = nbatch - 1; b >= 0; --b) {
+        Vec16 raw[U], rraw[kRes ? U : 1];
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const int v = b * step + k * blockDim.x + threadIdx.x;
+            if (v < nvec) {
+                raw[k] = ld_stream(xr + (int64_t)v * E);
+                if (kRes) rraw[k] = ld_stream(resr + (int64_t)v * E);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const int v = b * step + k * blockDim.x + threadIdx.x;
+            if (v < nvec) {
+                float2 val[P], g[P], o[P];
+                Elem<T>::unpack2(raw[k], val);
+                if (kRes) {
+                    float2 rv[P];
+                    Elem<T>::unpack2(rraw[k], rv);
+#pragma unroll
+                    for (int q = 0; q < P; ++q) val[q] = __fadd2_rn(val[q], rv[q]);
+                    st_stream(hr + (int64_t)v * E, Elem<T>::pack2(val));
+                }
+                load_params<E, false>(w + (int64_t)v * E, g);
+#pragma unroll
+                for (int q = 0; q < P; ++q) o[q] = __fmul2_rn(__fmul2_rn(val[q], r2), g[q]);
+                st_stream(yr + (int64_t)v * E, Elem<T>::pack2(o));
+            }
+        }
+    }
+}
+
 // ---- SiLU(gate) * up ------------------------------------------------------------------------------
 // silu(g) = g / (1 + 2^(-g log2e)): one ex2 and one reciprocal. bf16 rows use the approximate
 // reciprocal (relative error ~2^-23, far below the bf16 store step); fp32 rows divide exactly.
@@ -461,6 +539,12 @@ kop_status_t launch_rmsnorm(const void* xv, const void* wv, void* yv, int64_t ro
         }
 #undef KOP_RMS_LAUNCH
 #undef KOP_RMS
+        return launch_status();
+    }
+    if (vec && nvec64 <= 0x7FFFFFFF) {
+        const int nvec = (int)nvec64;
+        if (with_res) rmsnorm_long_kernel<T, PT, true><<<(unsigned)rows, 512, 0, stream>>>(x, w, y, nvec, xs, ys, eps, inv_hidden, rr);
+        else rmsnorm_long_kernel<T, PT, false><<<(unsigned)rows, 512, 0, stream>>>(x, w, y, nvec, xs, ys, eps, inv_hidden, rr);
         return launch_status();
     }
     if (with_res) rmsnorm_generic_kernel<T, PT, true><<<(unsigned)rows, 256, 0, stream>>>(x, w, y, hidden, xs, ys, eps, inv_hidden, rr);

@@ -123,7 +123,9 @@ LN_SHAPES = [
     (65, 256, BF16),
     (33, 8192, BF16),
     (17, 16384, F32),      # longest register-resident row
-    (9, 20480, BF16),      # generic
+    (9, 20480, BF16),      # beyond one CTA's registers: three sweeps with vector loads
+    (5, 40004, F32),       # several batches, ragged last one
+    (3, 20481, BF16),      # odd length: the scalar three-sweep kernel
     (21, 513, F32),        # scalar
     (40, 1000, BF16),      # 125 vectors: ragged CTA
     (5, 1, F32),
@@ -517,7 +519,7 @@ def test_ce_options(kop):
 # ------------------------------------------------------------------------------------------ MLP pieces
 
 RMS_SHAPES = [(2048, 4096, BF16), (300, 4096, F32), (65, 512, BF16), (17, 16384, BF16),
-              (9, 20480, F32), (21, 1001, BF16), (7, 1, F32)]
+              (9, 20480, F32), (5, 40008, BF16), (3, 20481, BF16), (21, 1001, BF16), (7, 1, F32)]
 
 
 @pytest.mark.parametrize("rows,hidden,dtype", RMS_SHAPES)
@@ -690,7 +692,7 @@ def test_row_ops_options_and_full_configs(kop):
 
 # ------------------------------------------------------------------------------------------ coverage variants
 
-RLN_SHAPES = [(2048, 4096, BF16), (1185, 4096, BF16), (300, 4096, F32), (65, 256, BF16), (9, 20480, BF16),
+RLN_SHAPES = [(2048, 4096, BF16), (1185, 4096, BF16), (300, 4096, F32), (65, 256, BF16), (9, 20480, BF16), (4, 33000, F32),
               (21, 513, F32)]
 
 
