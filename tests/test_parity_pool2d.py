@@ -45,6 +45,15 @@ POOL_CASES = [
     (3, 4, 7, 7, (7, 7), (1, 1), (0, 0), F32),         # window = image (global pooling)
     (2, 2, 9, 8, (1, 1), (1, 1), (0, 0), BF16),        # identity window
     (1, 2, 6, 5000, (3, 3), (2, 2), (1, 1), F32),      # rows too wide for a tile: direct kernel
+    # small planes: runs of planes per CTA, vectors crossing plane boundaries, a last run that ends inside a vector
+    (5, 37, 7, 7, (3, 3), (2, 2), (1, 1), F32),
+    (3, 50, 14, 14, (3, 3), (2, 2), (1, 1), BF16),
+    (4, 9, 14, 14, (2, 2), (2, 2), (0, 0), torch.float16),
+    (7, 11, 4, 4, (3, 3), (1, 1), (1, 1), F32),
+    (2, 13, 28, 28, (3, 3), (2, 2), (1, 1), BF16),
+    (3, 5, 5, 9, (2, 3), (1, 2), (1, 1), F32),         # generic window on a small plane
+    (3, 3, 3, 3, (3, 3), (3, 3), (0, 0), BF16),        # 9-element planes
+    (70, 64, 7, 7, (3, 3), (1, 1), (1, 1), BF16),      # several runs
 ]
 
 
