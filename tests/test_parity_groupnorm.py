@@ -47,6 +47,15 @@ GN_SHAPES = [
     (1, 16, 4, 4, 2, BF16, 2),
     (10, 256, 56, 56, 32, F32, 0),     # 320 chunks of 100 KB: more CTAs than fit the GPU at once
     (80, 64, 56, 56, 8, BF16, 1),      # 640 chunks of 50 KB
+    # small chunks: runs of chunks per CTA, vectors that cross chunk, channel and group boundaries, a last run
+    # that ends inside a vector, runs that wrap around the group index
+    (9, 37, 7, 7, 37, F32, 2),         # InstanceNorm 7 x 7
+    (5, 48, 14, 14, 48, BF16, 2),      # InstanceNorm 14 x 14 bf16
+    (7, 30, 7, 7, 5, F32, 1),          # 6 channels of 49 a group
+    (3, 21, 5, 3, 7, torch.float16, 0),
+    (11, 64, 4, 4, 32, BF16, 2),       # 2 channels of 16 a group
+    (2, 2048, 7, 7, 32, F32, 2),       # 64 channels of 49: 3136 elements, beyond the small kernel (scalar)
+    (6, 40, 7, 7, 1, F32, 0),          # groups == 1, chunk of 1960
 ]
 
 
