@@ -51,13 +51,13 @@ FALLBACK_HBM_GBS = 6650.0
 # quarter / half of the rows (same row length, same kernel variant) and are scaled by the row count,
 # which their traffic is proportional to. Written-back bytes exclude dirty lines still in L2 at kernel end.
 NCU_DRAM_TRAFFIC_BYTES = {
-    "ce_loss": 4 * (524357120 + 3634944),
-    "silu_mul": 2 * (469768448 + 180619264),
-    "softmax_large": 268470528 + 210199296,
-    "layernorm": 134280960 + 11149568,
-    "bn_pool": 205530624 + 149531392,
-    "rmsnorm": 134240768 + 77395712,
-    "residual_add": 268443648 + 83034880,
+    "ce_loss": 4 * (524355584 + 3218944),
+    "silu_mul": 2 * (469769216 + 180785920),
+    "softmax_large": 268447232 + 210064896,
+    "layernorm": 134281728 + 10796544,
+    "bn_pool": 205531136 + 148790528,
+    "rmsnorm": 134242560 + 77360128,
+    "residual_add": 268443648 + 81811200,
 }
 
 
