@@ -159,9 +159,11 @@ ln_block_kernel(const T* __restrict__ x, const T* __restrict__ res, const PT* __
 // out the kernel runs at the speed of a plain two-reads-one-write stream). Each thread therefore
 // fetches its bias / gamma / beta once and applies them to the same columns of two rows, which
 // halves that traffic; both rows' reductions share the two barriers. The row must be exactly
-// blockDim.x * VPT vectors; `rows` may be odd (the last CTA then skips its second row).
+// blockDim.x * VPT vectors; `rows` may be odd (the last CTA then skips its second row). Capped at 64 registers
+// (four 256-thread CTAs per SM): at the 76 the compiler takes by itself three fit, and the benchmark shape ran
+// 5 % slower (rows of 5120: 12 %); a cap of 48 spills and loses 25 %.
 template <typename T, typename PT, int VPT, bool kWide, int kMaxThreads, int PRO>
-__global__ void __launch_bounds__(kMaxThreads, 768 / kMaxThreads)
+__global__ void __launch_bounds__(kMaxThreads, 1024 / kMaxThreads)
 ln_pair_kernel(const T* __restrict__ x, const T* __restrict__ res, const PT* __restrict__ bias,
                const PT* __restrict__ gamma, const PT* __restrict__ beta, T* __restrict__ y,
                float* __restrict__ mean, float* __restrict__ rstd, int64_t rows, int64_t x_stride,
