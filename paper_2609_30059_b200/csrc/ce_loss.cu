@@ -17,6 +17,7 @@ namespace {
 // kGroupRows rows: a ticket, a partial loss sum, a bad-label count, a counted-row count (the last
 // only used by the variant with ignore_index).
 constexpr int kGroupRows = 256;
+static_assert(kGroupRows % 8 == 0, "a warp of the lanes-per-row kernel (up to 8 rows) must stay inside one group");
 struct CeWorkspace {
     unsigned int* global_ticket;
     unsigned int* group_ticket;
@@ -248,8 +249,9 @@ ce_row_kernel(const T* __restrict__ z, const int32_t* __restrict__ labels, float
 // Rows of at most 16 KB (classification heads, small vocabularies): L lanes of a warp per row (L = 4 .. 32),
 // 32 / L rows per warp, eight warps per CTA. Each lane sweeps its share in batches of four vectors with the
 // same recurrence as above; the row's (maximum, sum) pair is a butterfly over its lanes; the row's first lane
-// writes the loss and draws the ticket, and the warp then walks its rows so that whichever drew a group's
-// last ticket has all 32 lanes for the group sum, exactly as in the CTA-per-row kernel.
+// writes the loss, and the warp draws one ticket for all of its rows (an atomic per row was the cost of rows
+// this short), so that whichever warp draws a group's last ticket has all 32 lanes for the group sum, exactly
+// as in the CTA-per-row kernel.
 template <typename T, int L, bool kOpts, bool kSmooth>
 __global__ void __launch_bounds__(256)
 ce_group_kernel(const T* __restrict__ z, const int32_t* __restrict__ labels, float* __restrict__ loss,
@@ -309,7 +311,6 @@ ce_group_kernel(const T* __restrict__ z, const int32_t* __restrict__ labels, flo
         M = M2;
         if (kSmooth) Z += __shfl_xor_sync(0xFFFFFFFFu, Z, o);
     }
-    unsigned t = 0xFFFFFFFFu;
     if (live && sub == 0) {
         const float lse = (M + log2f(S)) * kLn2;
         const int32_t lab = labels[row];
@@ -321,15 +322,21 @@ ce_group_kernel(const T* __restrict__ z, const int32_t* __restrict__ labels, flo
             if (kSmooth) l = (1.0f - opts.smoothing) * l + opts.smoothing * (lse - Z / (float)vocab);
         }
         loss[row] = l;
+    }
+    // One ticket draw per warp, worth all of its rows: a warp's rows are consecutive and kGroupRows is a multiple
+    // of every rows-per-warp count, so they share a group. The losses were written by other lanes: the warp
+    // barrier orders them before lane 0's fence, which orders them before its ticket.
+    if (warp_row0 >= rows) return;                           // the whole warp is past the end
+    __syncwarp();
+    const int64_t left = rows - warp_row0;
+    const unsigned mine = (unsigned)(left < kRowsPerWarp ? left : kRowsPerWarp);
+    unsigned t = 0;
+    if (lane == 0) {
         __threadfence();
-        t = atomicAdd(ws.group_ticket + row / kGroupRows, 1u);
+        t = atomicAdd(ws.group_ticket + warp_row0 / kGroupRows, mine) + mine - 1u;
     }
-#pragma unroll
-    for (int r = 0; r < kRowsPerWarp; ++r) {
-        const unsigned tr = __shfl_sync(0xFFFFFFFFu, t, r * L);
-        if (warp_row0 + r < rows)                            // uniform over the warp
-            ce_after_ticket<kOpts>(tr, warp_row0 + r, lane, labels, loss, mean_loss, bad_label_count, ws, rows, vocab, opts);
-    }
+    t = __shfl_sync(0xFFFFFFFFu, t, 0);
+    ce_after_ticket<kOpts>(t, warp_row0, lane, labels, loss, mean_loss, bad_label_count, ws, rows, vocab, opts);
 }
 
 // Any vocab / alignment: scalar loads, element-wise online recurrence.
