@@ -456,6 +456,41 @@ residual_add_kernel(const T* __restrict__ a, const T* __restrict__ b, T* __restr
     }
 }
 
+// Strided rows shorter than a tile (or with a mostly empty last tile): tiles that cross rows.
+template <typename T, int U>
+__global__ void __launch_bounds__(256)
+residual_add_flat_kernel(const T* __restrict__ a, const T* __restrict__ b, T* __restrict__ out, int nvec,
+                         int64_t nvec_total, int64_t a_stride, int64_t b_stride, int64_t o_stride)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    const int64_t g0 = (int64_t)blockIdx.x * (U * blockDim.x) + threadIdx.x;
+    int64_t row[U];
+    int v[U];
+    bool live[U];
+    Vec16 ra[U], rb[U];
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+        const int64_t g = g0 + k * blockDim.x;
+        live[k] = g < nvec_total;
+        flat_position(live[k] ? g : 0, nvec, &row[k], &v[k]);
+        if (live[k]) {
+            ra[k] = ld_stream(a + row[k] * a_stride + (int64_t)v[k] * E);
+            rb[k] = ld_stream(b + row[k] * b_stride + (int64_t)v[k] * E);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+        if (live[k]) {
+            float fa[E], fb[E];
+            Elem<T>::unpack(ra[k], fa);
+            Elem<T>::unpack(rb[k], fb);
+#pragma unroll
+            for (int e = 0; e < E; ++e) fa[e] += fb[e];
+            st_stream(out + row[k] * o_stride + (int64_t)v[k] * E, Elem<T>::pack(fa));
+        }
+    }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256)
 residual_add_scalar_kernel(const T* __restrict__ a, const T* __restrict__ b, T* __restrict__ out,
@@ -648,6 +683,12 @@ kop_status_t launch_residual_add(const void* av, const void* bv, void* ov, int64
         const int threads = 128;
         constexpr int U = 4;
         const int64_t tiles = (nvec + threads * U - 1) / (threads * U);
+        if (rows > 1 && nvec <= 0x7FFFFFFF && (nvec < threads * U || (tiles * threads * U - nvec) * 4 > nvec)) {
+            const int64_t total = rows * nvec, fgrid = (total + 256 * U - 1) / (256 * U);
+            if (fgrid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+            residual_add_flat_kernel<T, U><<<(unsigned)fgrid, 256, 0, stream>>>(a, b, out, (int)nvec, total, as, bs, os);
+            return launch_status();
+        }
         const int64_t grid = rows * tiles;
         if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
         if (nvec % (threads * U) == 0)

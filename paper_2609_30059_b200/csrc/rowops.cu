@@ -40,6 +40,42 @@ row_scale_kernel(const T* __restrict__ a, const T* __restrict__ b, T* __restrict
     }
 }
 
+// Rows shorter than a tile (or with a mostly empty last tile): the CTA's U * blockDim.x vectors are taken in
+// row-major order across rows; a[row] is then one load per vector (L1-resident: neighbours share it).
+template <typename T, int U>
+__global__ void __launch_bounds__(256)
+row_scale_flat_kernel(const T* __restrict__ a, const T* __restrict__ b, T* __restrict__ out, int nvec,
+                      int64_t nvec_total, int64_t b_stride, int64_t o_stride)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    const int64_t g0 = (int64_t)blockIdx.x * (U * blockDim.x) + threadIdx.x;
+    int64_t row[U];
+    int v[U];
+    bool live[U];
+    Vec16 raw[U];
+    float s[U];
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+        const int64_t g = g0 + k * blockDim.x;
+        live[k] = g < nvec_total;
+        flat_position(live[k] ? g : 0, nvec, &row[k], &v[k]);
+        if (live[k]) {
+            raw[k] = ld_stream(b + row[k] * b_stride + (int64_t)v[k] * E);
+            s[k] = Elem<T>::load1(a + row[k]);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+        if (live[k]) {
+            float f[E];
+            Elem<T>::unpack(raw[k], f);
+#pragma unroll
+            for (int e = 0; e < E; ++e) f[e] *= s[k];
+            st_stream(out + row[k] * o_stride + (int64_t)v[k] * E, Elem<T>::pack(f));
+        }
+    }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256)
 row_scale_scalar_kernel(const T* __restrict__ a, const T* __restrict__ b, T* __restrict__ out, int64_t rows,
@@ -115,6 +151,43 @@ matvec_rows_kernel(const T* __restrict__ x, const float* __restrict__ w, float b
     }
 }
 
+// Short rows (at most 4 L vectors): L lanes of a warp per row, 32 / L rows per warp, eight warps per CTA; the
+// dot product is a butterfly over the row's lanes.
+template <typename T, int L>
+__global__ void __launch_bounds__(256)
+matvec_group_kernel(const T* __restrict__ x, const float* __restrict__ w, float b_sum, float* __restrict__ out,
+                    int64_t rows, int nvec, int64_t x_stride)
+{
+    constexpr int E = Elem<T>::kPerVec, P = E / 2, VPL = 4;
+    const int lane = threadIdx.x & 31, sub = lane & (L - 1);
+    const int64_t row = ((int64_t)blockIdx.x * 8 + (threadIdx.x >> 5)) * (32 / L) + lane / L;
+    const bool live = row < rows;
+    const T* xr = x + (live ? row : 0) * x_stride;
+    Vec16 raw[VPL];
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) {
+        const int v = k * L + sub;
+        raw[k] = Vec16{{0u, 0u, 0u, 0u}};
+        if (live && v < nvec) raw[k] = ld_stream(xr + (int64_t)v * E);
+    }
+    float2 acc = make_float2(0.0f, 0.0f);
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) {
+        const int v = k * L + sub;
+        if (v < nvec) {
+            float2 wv[P], f[P];
+            load_params<E, false>(w + (int64_t)v * E, wv);
+            Elem<T>::unpack2(raw[k], f);
+#pragma unroll
+            for (int q = 0; q < P; ++q) acc = __ffma2_rn(f[q], wv[q], acc);
+        }
+    }
+    float s = acc.x + acc.y;
+#pragma unroll
+    for (int o = L / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+    if (live && sub == 0) out[row] = s + b_sum;
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256)
 matvec_scalar_kernel(const T* __restrict__ x, const float* __restrict__ w, float b_sum, float* __restrict__ out,
@@ -151,6 +224,12 @@ kop_status_t launch_row_scale(const void* av, const void* bv, void* ov, int64_t 
         const int threads = 128;
         constexpr int U = 4;
         const int tiles = (nvec + threads * U - 1) / (threads * U);
+        if (nvec < threads * U || ((int64_t)tiles * threads * U - nvec) * 4 > nvec) {
+            const int64_t total = rows * nvec, fgrid = (total + 256 * U - 1) / (256 * U);
+            if (fgrid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+            row_scale_flat_kernel<T, U><<<(unsigned)fgrid, 256, 0, stream>>>(a, b, out, nvec, total, bs, os);
+            return launch_status();
+        }
         const int64_t grid = rows * tiles;
         if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
         if (nvec % (threads * U) == 0)
@@ -173,14 +252,33 @@ kop_status_t launch_matvec(const void* xv, const float* w, float b_sum, float* o
     const int64_t nvec64 = K / E;
     if (vec && nvec64 <= 0x7FFFFFFF) {
         const int nvec = (int)nvec64;
+        if (nvec <= 128) {                                   // short rows: lanes of a warp per row
+            const int lanes = nvec > 64 ? 32 : nvec > 32 ? 16 : nvec > 16 ? 8 : nvec > 8 ? 4 : 2;
+            const int64_t rows_per_cta = 8 * (32 / lanes);
+            const int64_t ctas = (M + rows_per_cta - 1) / rows_per_cta;
+            if (ctas > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+#define KOP_MV_GROUP(L) matvec_group_kernel<T, L><<<(unsigned)ctas, 256, 0, stream>>>(x, w, b_sum, out, M, nvec, xs)
+            switch (lanes) {
+            case 32: KOP_MV_GROUP(32); break;
+            case 16: KOP_MV_GROUP(16); break;
+            case 8: KOP_MV_GROUP(8); break;
+            case 4: KOP_MV_GROUP(4); break;
+            default: KOP_MV_GROUP(2); break;
+            }
+#undef KOP_MV_GROUP
+            return launch_status();
+        }
         // Two rows per CTA, 64 threads, four vector columns per trip (eight matrix loads in flight per
         // thread). Measured on [32768, 4096] bf16: 43.5 us; eight rows per CTA 59 us, one row 47.7 us,
         // a warp-per-row variant without barriers 44.3 us.
         constexpr int R = 2;
         const int64_t grid = (M + R - 1) / R;
         if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+        // long rows get up to 256 threads (a 64-thread CTA would loop 64 times over a 65536-column fp32 row with too
+        // few CTAs to fill the GPU: 1.2 TB/s against 4.0; rows of 16384 columns 4.0 - 4.4 against 4.9 - 5.5)
+        const int cap = nvec > 1024 ? 256 : 64;
         int threads = 32;
-        while (threads < 64 && threads < nvec) threads *= 2;
+        while (threads < cap && threads * 4 < nvec) threads *= 2;
         if (E == 8 && aligned_to(w, 32))
             matvec_rows_kernel<T, R, 4, true><<<(unsigned)grid, threads, 0, stream>>>(x, w, b_sum, out, M, nvec, xs);
         else

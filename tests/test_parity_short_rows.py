@@ -106,3 +106,40 @@ def test_short_row_elementwise(kop, rows, cols, dtype):
         kop.kop_silu_mul_interleaved(x, out=o2.t)
         assert_close(o2.t, kopref.silu_mul_interleaved(host(x)), tol, "silu_mul_interleaved")
         o2.check("silu_mul_interleaved")
+
+
+@pytest.mark.parametrize("rows,cols,dtype", SHAPES)
+def test_short_row_scale_matvec_and_strided_add(kop, rows, cols, dtype):
+    seed = rows * 5 + cols
+    tol = tol_of(dtype)
+    a, b = synth.row_scale_inputs(rows, cols, dtype, seed, "cuda")
+    y = Guarded((rows, cols), dtype)
+    kop.kop_row_scale(a, b, out=y.t)
+    assert_close(y.t, kopref.row_scale(host(a), host(b)), tol, "row_scale")
+    y.check("row_scale")
+    xv, wv, bs = synth.matvec_inputs(rows, cols, dtype, seed, "cuda")
+    o = Guarded((rows,), F32)
+    kop.kop_matvec_bias(xv, wv, bs, out=o.t)
+    ref = kopref.matvec_bias(host(xv), host(wv), bs)
+    mag = (host(xv).double().abs() @ host(wv).double().abs()).numpy() + abs(bs)
+    assert np.all(np.abs(to_f64(o.t) - ref) <= 1e-5 * np.maximum(1.0, mag)), "matvec"
+    o.check("matvec")
+    p, q = synth.pair_inputs(rows, cols, dtype, seed, "cuda")
+    pad = 8 if dtype != F32 else 4
+    bp = torch.zeros((rows, cols + pad), dtype=dtype, device="cuda")          # strided rows: no collapse to one long row
+    bq = torch.zeros((rows, cols + 2 * pad), dtype=dtype, device="cuda")
+    bp[:, :cols] = p
+    bq[:, :cols] = q
+    outb = torch.full((rows, cols + pad), 7.0, dtype=dtype, device="cuda")
+    kop.kop_residual_add(bp[:, :cols], bq[:, :cols], out=outb[:, :cols])
+    assert_close(outb[:, :cols], kopref.residual_add(host(p), host(q)), tol, "strided residual_add")
+    assert bool((outb[:, cols:] == 7.0).all())
+
+
+def test_matvec_long_rows(kop):
+    for rows, cols, dtype in ((37, 16384, BF16), (9, 65536, F32), (5, 40008, BF16)):
+        xv, wv, bs = synth.matvec_inputs(rows, cols, dtype, 3, "cuda")
+        ref = kopref.matvec_bias(host(xv), host(wv), bs)
+        mag = (host(xv).double().abs() @ host(wv).double().abs()).numpy() + abs(bs)
+        got = to_f64(kop.kop_matvec_bias(xv, wv, bs))
+        assert np.all(np.abs(got - ref) <= 1e-5 * np.maximum(1.0, mag)), f"matvec [{rows},{cols}]"
