@@ -358,6 +358,245 @@ groupnorm_staged_kernel(const T* __restrict__ x, const float* __restrict__ gamma
     }
 }
 
+// Chunks just beyond one CTA's staging budget (200 KB to 512 KB: GroupNorm on 128 x 128 maps): a thread-block cluster
+// of up to 8 CTAs stages the chunk, a slice each, and the two sums are combined over the cluster through
+// distributed shared memory, so the chunk is still read from HBM once. The same structure as the staged kernel;
+// every CTA runs every cluster barrier whatever happens to its copies.
+constexpr int kGnClusterThreads = 512;
+
+template <typename T, int ACT>
+__global__ void __launch_bounds__(kGnClusterThreads)
+groupnorm_cluster_kernel(const T* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
+                         T* __restrict__ y, float* __restrict__ mean, float* __restrict__ rstd, int nvec,
+                         int slice_vecs, int csize, int vec_per_plane, int cpg, int groups, float eps, float inv_count)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    constexpr int P = E / 2;
+    constexpr int NT = kGnClusterThreads;
+    constexpr int kPartVecs = kGnUnroll * NT;
+    extern __shared__ __align__(128) unsigned char gn_smem[];
+    Vec16* stage = reinterpret_cast<Vec16*>(gn_smem);
+    __shared__ float slots_a[32], slots_b[32];
+    __shared__ float from_sum[8], from_sq[8], from_bad[8];
+    __shared__ __align__(8) uint64_t bars[kGnMaxParts];
+
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");   // "this CTA has started"; waited for below
+    const uint32_t rank = cluster_rank();
+    const int64_t chunk = blockIdx.x / (unsigned)csize;      // image * groups + group
+    const int g = (int)(chunk % groups);
+    const int v_lo = (int)rank * slice_vecs;                 // this CTA's slice of the chunk
+    const int n_here = max(0, min(slice_vecs, nvec - v_lo));
+    const T* xc = x + (chunk * (int64_t)nvec + v_lo) * E;
+    T* yc = y + (chunk * (int64_t)nvec + v_lo) * E;
+    const int nparts = (n_here + kGnCopyVecs - 1) / kGnCopyVecs;
+
+    if (threadIdx.x == 0) {
+        for (int p = 0; p < nparts; ++p) mbar_init(bars + p, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        for (int p = 0; p < nparts; ++p) {
+            const int v0 = p * kGnCopyVecs;
+            const uint32_t bytes = (uint32_t)min(kGnCopyVecs, n_here - v0) * 16u;
+            mbar_expect_tx(bars + p, bytes);
+            bulk_load(stage + v0, xc + (int64_t)v0 * E, bytes, bars + p);
+        }
+    }
+    __syncthreads();
+
+    float2 s2 = make_float2(0.0f, 0.0f);
+    bool ok = true;                                          // uniform over the CTA
+    for (int p = 0; p < nparts && ok; ++p) {
+        bool landed = true;
+        if (threadIdx.x == 0) landed = mbar_wait_bounded(bars + p, 0);
+        ok = __syncthreads_and(landed);
+        if (!ok) {
+            // give the copies one more bounded chance to drain; this CTA then contributes nothing and the whole
+            // cluster writes nothing (it still takes part in both cluster barriers below)
+            if (threadIdx.x == 0) {
+                for (int q = p; q < nparts; ++q) mbar_wait_bounded(bars + q, 0);
+                atomicAdd(&g_gn_wait_timeouts, 1u);
+            }
+            break;
+        }
+        const int end = min(n_here, (p + 1) * kGnCopyVecs);
+        for (int base = p * kGnCopyVecs; base < end; base += kPartVecs) {
+#pragma unroll
+            for (int k = 0; k < kGnUnroll; ++k) {
+                const int v = base + k * NT + threadIdx.x;
+                if (v < end) {
+                    float2 f[P];
+                    Elem<T>::unpack2(stage[v], f);
+#pragma unroll
+                    for (int e = 0; e < P; ++e) s2 = __fadd2_rn(s2, f[e]);
+                }
+            }
+        }
+    }
+    const float local_sum = block_sum(ok ? s2.x + s2.y : 0.0f, slots_a);
+    // every CTA of the cluster has started (arrival at kernel entry): their shared memory may be written now
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    // one exchange for the sum and the failure flag: both slots written, one cluster barrier, folded in rank order
+    if (threadIdx.x < (unsigned)csize) {
+        store_to_cluster_cta(&from_sum[rank], threadIdx.x, local_sum);
+        store_to_cluster_cta(&from_bad[rank], threadIdx.x, ok ? 0.0f : 1.0f);
+    }
+    cluster_barrier();
+    float tot = 0.0f, bad = 0.0f;
+    for (int i = 0; i < csize; ++i) {
+        tot += from_sum[i];
+        bad += from_bad[i];
+    }
+    const float mu = tot * inv_count;
+    const float2 nmu = make_float2(-mu, -mu);
+    float2 q2 = make_float2(0.0f, 0.0f);
+    if (ok) {
+        for (int base = 0; base < n_here; base += kPartVecs) {
+#pragma unroll
+            for (int k = 0; k < kGnUnroll; ++k) {
+                const int v = base + k * NT + threadIdx.x;
+                if (v < n_here) {
+                    float2 f[P];
+                    Elem<T>::unpack2(stage[v], f);
+#pragma unroll
+                    for (int e = 0; e < P; ++e) {
+                        const float2 d = __fadd2_rn(f[e], nmu);
+                        q2 = __ffma2_rn(d, d, q2);
+                    }
+                }
+            }
+        }
+    }
+    const float local_sq = block_sum(q2.x + q2.y, slots_b);
+    const float rs = rsqrtf(cluster_sum(local_sq, from_sq, rank, (uint32_t)csize) * inv_count + eps);   // last remote access
+    if (bad != 0.0f) return;                                 // some CTA of the cluster lost a copy: nothing is written
+    if (threadIdx.x == 0 && rank == 0) {
+        if (mean != nullptr) mean[chunk] = mu;
+        if (rstd != nullptr) rstd[chunk] = rs;
+    }
+    const float inv_vpp = 1.0f / (float)vec_per_plane;
+    for (int base = 0; base < n_here; base += kPartVecs) {
+#pragma unroll
+        for (int k = 0; k < kGnUnroll; ++k) {
+            const int v = base + k * NT + threadIdx.x;
+            if (v < n_here)
+                normalize_store<T, ACT>(stage[v], yc + (int64_t)v * E,
+                                        g * cpg + div_small(v_lo + v, vec_per_plane, inv_vpp), gamma, beta, mu, rs);
+        }
+    }
+}
+
+// Few, very large chunks (a batch of one or two images through an image generator's GroupNorm: 32 to 128 chunks of
+// megabytes): one CTA per chunk would leave most SMs idle. A cluster of up to 8 CTAs shares the chunk, a slice
+// each, in the two-sweep manner (moments in one sweep, output in a second, mostly from the L2); the slices'
+// (count, mean, M2) triples are exchanged through distributed shared memory and merged pairwise in rank order.
+template <typename T, int ACT>
+__global__ void __launch_bounds__(kGnThreads)
+groupnorm_twosweep_cluster_kernel(const T* __restrict__ x, const float* __restrict__ gamma,
+                                  const float* __restrict__ beta, T* __restrict__ y, float* __restrict__ mean,
+                                  float* __restrict__ rstd, int nvec, int slice_vecs, int csize, int vec_per_plane,
+                                  int cpg, int groups, float eps)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    __shared__ float red_n[32], red_mean[32], red_m2[32];
+    __shared__ float from_n[8], from_mean[8], from_m2[8];
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");   // "this CTA has started"; waited for below
+    const uint32_t rank = cluster_rank();
+    const int64_t chunk = blockIdx.x / (unsigned)csize;
+    const int g = (int)(chunk % groups);
+    const int v_lo = (int)rank * slice_vecs;
+    const int n_here = max(0, min(slice_vecs, nvec - v_lo));
+    const T* xc = x + (chunk * (int64_t)nvec + v_lo) * E;
+    T* yc = y + (chunk * (int64_t)nvec + v_lo) * E;
+
+    Moments acc{0.0f, 0.0f, 0.0f};
+    for (int base = 0; base < n_here; base += kGnUnroll * kGnThreads) {
+        Vec16 raw[kGnUnroll];
+        int cnt = 0;
+#pragma unroll
+        for (int k = 0; k < kGnUnroll; ++k) {
+            const int v = base + k * kGnThreads + threadIdx.x;
+            if (v < n_here) {
+                raw[k] = ld_stream(xc + (int64_t)v * E);
+                ++cnt;
+            } else {
+                raw[k] = Vec16{{0u, 0u, 0u, 0u}};
+            }
+        }
+        if (cnt > 0) {
+            float f[kGnUnroll][E];
+            float s = 0.0f;
+#pragma unroll
+            for (int k = 0; k < kGnUnroll; ++k) {
+                Elem<T>::unpack(raw[k], f[k]);
+#pragma unroll
+                for (int e = 0; e < E; ++e) s += f[k][e];
+            }
+            const float bn = (float)(cnt * E);
+            const float bmean = s / bn;
+            float m2 = 0.0f;
+#pragma unroll
+            for (int k = 0; k < kGnUnroll; ++k) {
+                if (k < cnt) {
+#pragma unroll
+                    for (int e = 0; e < E; ++e) {
+                        const float d = f[k][e] - bmean;
+                        m2 = fmaf(d, d, m2);
+                    }
+                }
+            }
+            acc = merge(acc, Moments{bn, bmean, m2});
+        }
+    }
+    acc = warp_merge(acc);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) {
+        red_n[warp] = acc.n;
+        red_mean[warp] = acc.mean;
+        red_m2[warp] = acc.m2;
+    }
+    __syncthreads();
+    // every warp merges the CTA's warp partials for itself (the same order everywhere, so the same triple)
+    constexpr int NW = kGnThreads / 32;
+    Moments t = lane < NW ? Moments{red_n[lane], red_mean[lane], red_m2[lane]} : Moments{0.0f, 0.0f, 0.0f};
+    t = warp_merge(t);
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");     // every CTA of the cluster has started
+    if (threadIdx.x < (unsigned)csize) {
+        store_to_cluster_cta(&from_n[rank], threadIdx.x, t.n);
+        store_to_cluster_cta(&from_mean[rank], threadIdx.x, t.mean);
+        store_to_cluster_cta(&from_m2[rank], threadIdx.x, t.m2);
+    }
+    cluster_barrier();                                       // the only exchange: last remote access before it
+    Moments all{0.0f, 0.0f, 0.0f};
+    for (int i = 0; i < csize; ++i) all = merge(all, Moments{from_n[i], from_mean[i], from_m2[i]});
+    const float mu = all.mean, rs = rsqrtf(all.m2 / all.n + eps);
+    if (threadIdx.x == 0 && rank == 0) {
+        if (mean != nullptr) mean[chunk] = mu;
+        if (rstd != nullptr) rstd[chunk] = rs;
+    }
+    for (int base = 0; base < n_here; base += kGnUnroll * kGnThreads) {
+        Vec16 raw[kGnUnroll];
+#pragma unroll
+        for (int k = 0; k < kGnUnroll; ++k) {
+            const int v = base + k * kGnThreads + threadIdx.x;
+            if (v < n_here) raw[k] = ld_stream(xc + (int64_t)v * E);
+        }
+#pragma unroll
+        for (int k = 0; k < kGnUnroll; ++k) {
+            const int v = base + k * kGnThreads + threadIdx.x;
+            if (v < n_here) {
+                const int c = g * cpg + (v_lo + v) / vec_per_plane;
+                const float ga = gamma != nullptr ? __ldg(gamma + c) : 1.0f;
+                const float be = beta != nullptr ? __ldg(beta + c) : 0.0f;
+                const float sc = rs * ga;
+                float f[E];
+                Elem<T>::unpack(raw[k], f);
+#pragma unroll
+                for (int e = 0; e < E; ++e) f[e] = activate<ACT>(fmaf(f[e] - mu, sc, be));
+                st_stream(yc + (int64_t)v * E, Elem<T>::pack(f));
+            }
+        }
+    }
+}
+
 // Small chunks (InstanceNorm on 7 x 7 .. 32 x 32 planes, GroupNorm with few channels a group on small maps): a CTA
 // per chunk would be mostly idle threads and fixed costs, and such chunks are often not a whole number of 16-byte
 // vectors. Consecutive chunks are contiguous, so a CTA takes a run of R chunks (R a multiple of the vector length:
@@ -564,6 +803,65 @@ kop_status_t launch_gn_act(const T* x, const float* gamma, const float* beta, T*
             else
                 groupnorm_staged_kernel<T, ACT, 512><<<(unsigned)chunks, 512, bytes, stream>>>(
                     x, gamma, beta, y, mean, rstd, nvec, vpp, cpg, groups, eps, inv_count);
+        } else if (bytes <= 512 * 1024 && chunks * 8 <= 0x7FFFFFFFLL) {
+            // a cluster per chunk, slices of at most 64 KB (three CTAs per SM). Measured against the two-sweep
+            // kernel on fp32 chunks of 256 KB: 3.7 against 3.0 TB/s; at 1 MB (six slices of 175 KB, one CTA per
+            // SM) it lost, 3.2 against 3.9, and at 98 KB against the single-CTA staged kernel too (4.1 against
+            // 5.3): a cluster barrier costs about what a CTA needs for 100 KB, so only this window uses it.
+            int csize = (int)((bytes + 64 * 1024 - 1) / (64 * 1024));
+            if (csize < 2) csize = 2;
+            const int slice_vecs = (nvec + csize - 1) / csize;
+            const size_t smem = (size_t)slice_vecs * 16;
+            static std::atomic<bool> configured_c[kMaxDevices];
+            int dev = 0;
+            if (cudaGetDevice(&dev) != cudaSuccess) return KOP_ERR_CUDA;
+            if (dev < 0 || dev >= kMaxDevices || !configured_c[dev].load(std::memory_order_acquire)) {
+                if (cudaFuncSetAttribute(groupnorm_cluster_kernel<T, ACT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)kGnStageLimit) != cudaSuccess)
+                    return KOP_ERR_CUDA;
+                if (dev >= 0 && dev < kMaxDevices) configured_c[dev].store(true, std::memory_order_release);
+            }
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3((unsigned)(chunks * csize), 1, 1);
+            cfg.blockDim = dim3(kGnClusterThreads, 1, 1);
+            cfg.dynamicSmemBytes = smem;
+            cfg.stream = stream;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = (unsigned)csize;
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            const float inv_count = (float)(1.0 / (double)chunk_elems);
+            if (cudaLaunchKernelEx(&cfg, groupnorm_cluster_kernel<T, ACT>, x, gamma, beta, y, mean, rstd, nvec, slice_vecs,
+                                   csize, vpp, cpg, groups, eps, inv_count) != cudaSuccess) {
+                (void)cudaGetLastError();
+                return KOP_ERR_CUDA;
+            }
+        } else if (chunks <= (int64_t)sm_count() && bytes >= 1024 * 1024) {
+            // too few chunks to fill the GPU: clusters share them, about two CTAs per SM in all
+            int csize = (int)((2 * (int64_t)sm_count() + chunks - 1) / chunks);
+            if (csize > 8) csize = 8;
+            if (csize < 2) csize = 2;
+            const int slice_vecs = (nvec + csize - 1) / csize;
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3((unsigned)(chunks * csize), 1, 1);
+            cfg.blockDim = dim3(kGnThreads, 1, 1);
+            cfg.dynamicSmemBytes = 0;
+            cfg.stream = stream;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = (unsigned)csize;
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            if (cudaLaunchKernelEx(&cfg, groupnorm_twosweep_cluster_kernel<T, ACT>, x, gamma, beta, y, mean, rstd, nvec,
+                                   slice_vecs, csize, vpp, cpg, groups, eps) != cudaSuccess) {
+                (void)cudaGetLastError();
+                return KOP_ERR_CUDA;
+            }
         } else {
             groupnorm_twosweep_kernel<T, ACT><<<(unsigned)chunks, kGnThreads, 0, stream>>>(
                 x, gamma, beta, y, mean, rstd, nvec, vpp, cpg, groups, eps);

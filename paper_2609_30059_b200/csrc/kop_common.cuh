@@ -413,6 +413,19 @@ __device__ __forceinline__ void cluster_barrier()
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
+// A block-reduced value (the same in every thread of the CTA) summed over the CTAs of a cluster: every CTA writes
+// its value into slot [rank] of every CTA's `slots`, one hardware cluster barrier, and each CTA adds the slots in
+// rank order (a fixed order: the same result in every CTA and from run to run). Every thread of every CTA of
+// the cluster must call it; `slots` holds at least csize floats and is used for one call only.
+__device__ __forceinline__ float cluster_sum(float v, float* slots, uint32_t rank, uint32_t csize)
+{
+    if (threadIdx.x < csize) store_to_cluster_cta(&slots[rank], threadIdx.x, v);
+    cluster_barrier();
+    float r = 0.0f;
+    for (uint32_t i = 0; i < csize; ++i) r += slots[i];
+    return r;
+}
+
 #endif  // __CUDACC__
 
 }  // namespace kop

@@ -38,8 +38,14 @@ GN_SHAPES = [
     (3, 64, 28, 28, 8, BF16, 2),       # staged bf16
     (2, 32, 56, 56, 32, F32, 0),       # InstanceNorm (groups == C)
     (2, 6, 40, 40, 1, F32, 1),         # groups == 1, chunk 38,400 B
-    (2, 64, 64, 64, 2, F32, 2),        # chunk 512 KB: beyond the staging budget, unstaged vector kernel
-    (2, 128, 64, 64, 2, BF16, 1),      # chunk 1 MB bf16, unstaged
+    (2, 64, 64, 64, 2, F32, 2),        # chunk 512 KB: beyond one CTA's staging budget, a cluster of 8 CTAs
+    (2, 128, 64, 64, 2, BF16, 1),      # chunk 1 MB bf16: beyond the cluster window, two sweeps
+    (3, 8, 160, 160, 2, F32, 2),       # 400 KB: cluster of 7
+    (2, 3, 290, 290, 1, BF16, 1),      # 493 KB, slices that do not divide evenly
+    (1, 2, 600, 600, 1, F32, 0),       # one chunk of 2.9 MB: a cluster of 8 shares it, two sweeps
+    (2, 12, 256, 256, 3, BF16, 2),     # six chunks of 512 KB bf16 (staged cluster); 1 MB fp32 below
+    (2, 12, 256, 256, 3, F32, 1),      # six chunks of 1 MB: shared by clusters of 8, uneven slices
+    (1, 6, 256, 256, 3, torch.float16, 2),   # 256 KB fp16: cluster of 4
     (3, 12, 7, 7, 4, F32, 2),          # plane 49: scalar kernel
     (3, 12, 5, 6, 3, BF16, 0),         # plane 30 bf16: scalar kernel (30 % 8 != 0)
     (2, 8, 2, 2, 4, F32, 1),           # plane of one vector, chunk shorter than a warp's worth
