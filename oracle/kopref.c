@@ -326,6 +326,32 @@ int kopref_rmsnorm(const void* x, const float* weight, double* y,
     return 0;
 }
 
+/* ---- Lp normalisation of rows (p = 1 or 2) ---------------------------------------
+ * n_i = sum_j |x_ij|  (p = 1)   or   sqrt(sum_j x_ij^2)  (p = 2);   y_ij = x_ij / max(n_i, eps).
+ * norm_out (may be NULL) receives n_i. ("Normalization fusion": a reduction and the pointwise pass that
+ * uses it, in one kernel.) */
+int kopref_lp_normalize_rows(const void* x, double* y, double* norm_out, int64_t rows, int64_t cols,
+        int64_t x_row_stride, int64_t y_row_stride, int p, double eps, int dtype, int threads)
+{
+    if (!x || !y || rows < 0 || cols <= 0 || (p != 1 && p != 2) || bad_dtype(dtype)) return -1;
+    int nt = pick_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t i = 0; i < rows; ++i) {
+        double acc = 0.0;
+        for (int64_t j = 0; j < cols; ++j) {
+            double v = load_elem(x, i * x_row_stride + j, dtype);
+            acc += p == 1 ? fabs(v) : v * v;
+        }
+        double n = p == 1 ? acc : sqrt(acc);
+        if (norm_out) norm_out[i] = n;
+        double d = n > eps ? n : eps;             /* a NaN norm fails the comparison: d = eps, y = x / eps ... */
+        if (n != n) d = n;                        /* ... so keep the NaN: every output of that row is NaN */
+        for (int64_t j = 0; j < cols; ++j) y[i * y_row_stride + j] = load_elem(x, i * x_row_stride + j, dtype) / d;
+    }
+    return 0;
+}
+
 /* ---- SiLU(gate) * up -------------------------------------------------------------
  * Row layout [gate(0..I) | up(I..2I)]; out_j = gate_j / (1 + exp(-gate_j)) * up_j.
  * ("activation fusion (GELU/SiLU/ReLU)"; only the epilogue is fused.) */

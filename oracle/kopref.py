@@ -59,6 +59,7 @@ def lib() -> C.CDLL:
         _lib.kopref_epilogue_chain.argtypes = [vp, vp, vp, vp] + [i64] * 5 + [dbl] * 4 + [C.c_int, dbl, C.c_int, C.c_int]
         _lib.kopref_lstm_cell.argtypes = [vp] * 6 + [i64, i64, C.c_int, C.c_int]
         _lib.kopref_gru_cell.argtypes = [vp] * 6 + [i64, i64, C.c_int, C.c_int]
+        _lib.kopref_lp_normalize_rows.argtypes = [vp, vp, vp, i64, i64, i64, i64, C.c_int, C.c_double, C.c_int, C.c_int]
         _lib.kopref_cumsum_rows.argtypes = [vp, vp, vp] + [i64] * 5 + [C.c_int] * 4
         _lib.kopref_matvec_bias.argtypes = [vp, vp, dbl, vp, i64, i64, i64, C.c_int, C.c_int]
     return _lib
@@ -233,6 +234,17 @@ def residual_rmsnorm(x, residual, weight, eps, threads=1):
     below (residual_add, rmsnorm): nothing new is computed here."""
     h = residual_add(x, residual, threads)
     return h, rmsnorm(h, weight, eps, threads)
+
+
+def lp_normalize_rows(x, p=2, eps=1e-12, threads=1):
+    """y = x / max(||x||_p, eps) per row, p in (1, 2). Returns (y, norms)."""
+    xa, dt = as_data(x)
+    rows, cols = xa.shape
+    y = np.empty((rows, cols), dtype=np.float64)
+    n = np.empty((rows,), dtype=np.float64)
+    _check(lib().kopref_lp_normalize_rows(_p(xa), _p(y), _p(n), rows, cols, cols, cols, int(p), float(eps), dt, _nt(threads)),
+           "lp_normalize_rows")
+    return y, n
 
 
 def silu_mul(gate_up, threads=1) -> np.ndarray:

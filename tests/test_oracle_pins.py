@@ -1085,3 +1085,35 @@ def test_16_bit_parameters_widen_exactly_and_match_the_float64_library_norms():
     # rounding the parameters to bf16 is visible: the fp32 originals give a different result
     g32 = torch.from_numpy(RNG.normal(1, 0.1, H)).float()
     assert np.abs(kopref.rmsnorm(x, g32, 1e-6) - kopref.rmsnorm(x, g32.to(torch.bfloat16), 1e-6)).max() > 1e-4
+
+
+def test_lp_normalize_rows_against_torch_and_closed_forms():
+    x = torch.from_numpy(RNG.normal(0, 2, (9, 37)))
+    for p in (1, 2):
+        y, n = kopref.lp_normalize_rows(x, p, 1e-12)
+        np.testing.assert_allclose(y, torch.nn.functional.normalize(x, p=float(p), dim=1, eps=1e-12).numpy(), rtol=1e-14, atol=0)
+        np.testing.assert_allclose(n, torch.linalg.vector_norm(x, ord=p, dim=1).numpy(), rtol=1e-14)
+        # the result has unit p-norm, and scaling the row by c only changes the sign
+        np.testing.assert_allclose(np.linalg.norm(y, ord=p, axis=1), 1.0, rtol=1e-13)
+        y3, n3 = kopref.lp_normalize_rows(x * -3.0, p, 1e-12)
+        np.testing.assert_allclose(y3, -y, rtol=1e-13, atol=0)
+        np.testing.assert_allclose(n3, 3.0 * n, rtol=1e-13)
+    # closed forms: the 3-4-5 triangle; p = 1 divides by the sum of magnitudes
+    y, n = kopref.lp_normalize_rows(np.array([[3.0, -4.0]]), 2)
+    assert n[0] == 5.0 and np.array_equal(y, [[0.6, -0.8]])
+    y, n = kopref.lp_normalize_rows(np.array([[1.0, -2.0, 5.0]]), 1)
+    assert n[0] == 8.0 and np.array_equal(y, [[0.125, -0.25, 0.625]])
+    # eps: a zero row stays zero (0 / eps), a tiny row is divided by eps, not by its norm
+    y, n = kopref.lp_normalize_rows(np.zeros((1, 4)), 2, 1e-6)
+    assert n[0] == 0.0 and np.array_equal(y, np.zeros((1, 4)))
+    y, _ = kopref.lp_normalize_rows(np.array([[1e-9, 0.0]]), 2, 1e-6)
+    np.testing.assert_allclose(y, [[1e-3, 0.0]], rtol=1e-15)
+    # p = 1 and p = 2 differ (a transposed switch would show here)
+    a, _ = kopref.lp_normalize_rows(np.array([[1.0, 1.0]]), 1)
+    b, _ = kopref.lp_normalize_rows(np.array([[1.0, 1.0]]), 2)
+    assert a[0, 0] == 0.5 and b[0, 0] == pytest.approx(2 ** -0.5, rel=1e-15)
+    # a NaN makes its whole row NaN; 16-bit data is widened exactly
+    y, n = kopref.lp_normalize_rows(np.array([[1.0, float("nan")], [3.0, 4.0]]), 2)
+    assert np.isnan(y[0]).all() and np.isnan(n[0]) and np.array_equal(y[1], [0.6, 0.8])
+    h = torch.from_numpy(RNG.normal(0, 1, (3, 16))).to(torch.bfloat16)
+    np.testing.assert_array_equal(kopref.lp_normalize_rows(h, 2)[0], kopref.lp_normalize_rows(h.double(), 2)[0])
