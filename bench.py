@@ -109,6 +109,7 @@ def segment_bytes():
     out["residual_rmsnorm"] = dict(bytes=4 * m["rows"] * m["hidden"] * 2 + m["hidden"] * 4, elems=m["rows"] * m["hidden"])
     t = c["lstm_cell"]
     out["lstm_cell"] = dict(bytes=(2 * 4 + 3) * t["rows"] * t["hidden"] * 2 + 4 * t["hidden"] * 4, elems=t["rows"] * t["hidden"])
+    out["l2_normalize"] = dict(bytes=2 * m["rows"] * m["hidden"] * 2 + m["rows"] * 4, elems=m["rows"] * m["hidden"])
     t = c["gru_cell"]
     out["gru_cell"] = dict(bytes=(2 * 3 + 2) * t["rows"] * t["hidden"] * 2 + 6 * t["hidden"] * 4, elems=t["rows"] * t["hidden"])
     u = c["cumsum"]
@@ -256,7 +257,7 @@ class Workload:
 
     ORDER = ["softmax_small", "softmax_large", "layernorm", "bn_pool", "ce_loss", "rmsnorm", "silu_mul", "residual_add"]
     # Beyond the benchmark configs (not part of `value`): the two kernels the paper's case studies print.
-    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "layernorm_params16", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc", "pool2d", "reduce_max", "reduce_logsumexp", "bias_gelu", "residual_rmsnorm", "lstm_cell", "gru_cell"]
+    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "layernorm_params16", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc", "pool2d", "reduce_max", "reduce_logsumexp", "bias_gelu", "residual_rmsnorm", "l2_normalize", "lstm_cell", "gru_cell"]
 
     def __init__(self, kop, device, seed, only=None, rows_div=1):
         """only: build just these segments (None = all, plus the MLP segment); rows_div cuts the row
@@ -352,7 +353,7 @@ class Workload:
         m = c["mlp"]
         self.eps = m["eps"]
         rows = cut(m["rows"])
-        if want & {"rmsnorm", "residual_add", "silu_mul", "silu_mul_interleaved", "mlp", "residual_rmsnorm"}:
+        if want & {"rmsnorm", "residual_add", "silu_mul", "silu_mul_interleaved", "mlp", "residual_rmsnorm", "l2_normalize"}:
             g = torch.Generator(device=dev)
             g.manual_seed(seed)
             if "mlp" in want:
@@ -432,6 +433,10 @@ class Workload:
             k.kop_residual_rmsnorm(self.h, self.d, self.rw, self.eps, h_out=self.res, out=self.n)
         elif name == "lstm_cell":                # gate sums, activations and state update, bf16 [16384, 4 x 1024]
             k.kop_lstm_cell(self.tg, self.tc, self.tg2, self.tb, h_out=self.th, c_out=self.tco)
+        elif name == "l2_normalize":             # x / max(||x||_2, eps) per row with the norms, bf16 [16384, 4096]
+            if not hasattr(self, "l2n"):
+                self.l2n = torch.empty(self.h.shape[0], dtype=torch.float32, device=self.h.device)
+            k.kop_lp_normalize_rows(self.h, 2, 1e-12, out=self.n, norms=self.l2n)
         elif name == "gru_cell":                 # gate sums, activations and state update, bf16 [16384, 3 x 1024]
             k.kop_gru_cell(self.ui, self.uh, self.up, self.ubi, self.ubh, h_out=self.uo)
         elif name == "cumsum":                   # inclusive running sum along rows, fp32 [32768, 4096]

@@ -442,6 +442,19 @@ kop_status_t kop_cumsum_rows(const void* x, const unsigned char* mask, void* y, 
                              int exclusive, int reverse, kop_dtype_t dtype, kop_stream_t stream);
 
 /*
+ * Lp normalisation of rows (fusion agent: "normalization fusion", a reduction and the pointwise pass that uses it
+ * in one kernel; the vector-norm rows of the paper's level-1 table):
+ *   n_i = sum_j |x[i,j]|  (p = 1)   or   sqrt(sum_j x[i,j]^2)  (p = 2);     y[i,j] = x[i,j] / max(n_i, eps)
+ * x, y: [rows, cols] of `dtype`; norm_out: fp32 [rows] or NULL, receives n_i (the L1 / L2 norm of every row; a
+ * tensor passed as one row gives its Frobenius norm). Sums are fp32 in a fixed order. eps >= 0. A NaN in a row
+ * makes its norm and every output of that row NaN; an infinite element gives norm inf and outputs 0 (NaN at the
+ * infinite positions). y may alias x exactly; norm_out overlaps neither. rows <= 2^31 - 1.
+ */
+kop_status_t kop_lp_normalize_rows(const void* x, void* y, float* norm_out, int64_t rows, int64_t cols,
+                                   int64_t x_row_stride, int64_t y_row_stride, int p, float eps, kop_dtype_t dtype,
+                                   kop_stream_t stream);
+
+/*
  * The pointwise part of one LSTM step (the LSTM models of the paper's level-3 table, L3-035 to L3-038, for
  * which its compiler emitted no kernels and the recurrent layer stayed with the vendor library; here the
  * two gate GEMMs stay with the vendor library and everything after them is one pass). With H = hidden and

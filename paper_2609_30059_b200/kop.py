@@ -96,6 +96,8 @@ def lib() -> C.CDLL:
     L.kop_epilogue_chain.restype = i32
     L.kop_cumsum_rows.argtypes = [vp, vp, vp] + [i64] * 5 + [i32, i32, i32, vp]
     L.kop_cumsum_rows.restype = i32
+    L.kop_lp_normalize_rows.argtypes = [vp, vp, vp, i64, i64, i64, i64, i32, f32, i32, vp]
+    L.kop_lp_normalize_rows.restype = i32
     L.kop_lstm_cell.argtypes = [vp] * 6 + [i64, i64, i32, vp]
     L.kop_lstm_cell.restype = i32
     L.kop_gru_cell.argtypes = [vp] * 6 + [i64, i64, i32, vp]
@@ -534,6 +536,18 @@ def kop_cumsum_rows(x, mask=None, exclusive=False, reverse=False, out=None, stre
     _check(lib().kop_cumsum_rows(x.data_ptr(), mp, out.data_ptr(), rows, cols, xs, ms, ys, int(bool(exclusive)),
                                  int(bool(reverse)), _dtype_tag(x), _stream(stream)), "kop_cumsum_rows")
     return out
+
+
+def kop_lp_normalize_rows(x, p=2, eps=1e-12, out=None, norms=None, want_norms=True, stream=None):
+    """y = x / max(||x||_p, eps) per row (p = 1 or 2). Returns (y, norms[rows] or None)."""
+    rows, cols, xs = _rows2d(x, "x")
+    out = torch.empty_like(x) if out is None else out
+    _, _, ys = _rows2d(out, "out")
+    if want_norms and norms is None:
+        norms = torch.empty(rows, dtype=torch.float32, device=x.device)
+    _check(lib().kop_lp_normalize_rows(x.data_ptr(), out.data_ptr(), None if norms is None else norms.data_ptr(), rows, cols,
+                                       xs, ys, int(p), float(eps), _dtype_tag(x), _stream(stream)), "kop_lp_normalize_rows")
+    return out, norms
 
 
 def kop_lstm_cell(gates, c_prev, gates2=None, bias=None, h_out=None, c_out=None, stream=None):

@@ -298,6 +298,27 @@ def test_norm_ex_validation(L):
     assert L.kop_residual_rmsnorm(P, None, G, B, R, 4, 0, 64, 64, 64, 64, 1e-6, 1, None) == SHAPE
 
 
+def test_lp_normalize_validation(L):
+    f = L.kop_lp_normalize_rows
+    N = 0x600000
+    assert f(P, Q, N, 0, 64, 64, 64, 2, 1e-12, 0, None) == OK
+    assert f(None, Q, N, 4, 64, 64, 64, 2, 1e-12, 0, None) == NULLP
+    assert f(P, None, None, 4, 64, 64, 64, 2, 1e-12, 0, None) == NULLP
+    assert f(P, Q, None, 4, 0, 64, 64, 2, 1e-12, 0, None) == SHAPE
+    assert f(P, Q, None, 4, 64, 64, 64, 3, 1e-12, 0, None) == SHAPE            # p is 1 or 2
+    assert f(P, Q, None, 4, 64, 64, 64, 0, 1e-12, 0, None) == SHAPE
+    assert f(P, Q, None, 4, 64, 64, 64, 2, -1.0, 0, None) == SHAPE
+    assert f(P, Q, None, 4, 64, 64, 64, 2, float("nan"), 0, None) == SHAPE
+    assert f(P, Q, None, 4, 64, 63, 64, 2, 1e-12, 0, None) == STRIDE
+    assert f(P, Q, None, 4, 64, 64, 8, 2, 1e-12, 0, None) == STRIDE
+    assert f(P, Q, None, 4, 64, 64, 64, 2, 1e-12, 3, None) == DTYPE
+    assert f(P + 2, Q, None, 4, 64, 64, 64, 2, 1e-12, 0, None) == MISAL
+    assert f(P, Q, N + 2, 4, 64, 64, 64, 2, 1e-12, 1, None) == MISAL
+    assert f(P, P + 8, None, 4, 64, 64, 64, 2, 1e-12, 0, None) == ALIAS
+    assert f(P, Q, Q + 16, 4, 64, 64, 64, 2, 1e-12, 0, None) == ALIAS           # norms inside y
+    assert f(P, Q, P, 4, 64, 64, 64, 2, 1e-12, 0, None) == ALIAS
+
+
 def test_pool2d_validation(L):
     f = L.kop_affine_relu_pool2d
     S, T = 0x600000, 0x610000

@@ -56,7 +56,7 @@ def test_all_entry_points_in_one_graph(kop):
         "red_i": torch.empty(rows, dtype=torch.int32, device=dev), "lse": torch.empty(rows, device=dev),
         "act": torch.empty_like(x), "chain": torch.empty_like(x), "mlp": torch.empty_like(h),
         "rr_h": torch.empty_like(lx), "rr_y": torch.empty_like(lx), "lstm_h": torch.empty_like(tc), "lstm_c": torch.empty_like(tc),
-        "gru_h": torch.empty_like(up),
+        "gru_h": torch.empty_like(up), "lpn": torch.empty_like(lx), "lpn_n": torch.empty(rows, device=dev),
     }
 
     def run():
@@ -86,6 +86,7 @@ def test_all_entry_points_in_one_graph(kop):
         kop.kop_residual_rmsnorm(lx, lr, lg, 1e-6, h_out=o["rr_h"], out=o["rr_y"])
         kop.kop_lstm_cell(tg, tc, tg2, tb, h_out=o["lstm_h"], c_out=o["lstm_c"])
         kop.kop_gru_cell(ui, uh, up, ubi, ubh, h_out=o["gru_h"])
+        kop.kop_lp_normalize_rows(lx, 2, 1e-12, out=o["lpn"], norms=o["lpn_n"])
         kop.kop_rmsnorm_swiglu_residual(handle, h, w, W1, W2, 1e-6, out=o["mlp"], workspace=ws_mlp)
 
     try:
