@@ -110,6 +110,10 @@ def segment_bytes():
     t = c["lstm_cell"]
     out["lstm_cell"] = dict(bytes=(2 * 4 + 3) * t["rows"] * t["hidden"] * 2 + 4 * t["hidden"] * 4, elems=t["rows"] * t["hidden"])
     out["l2_normalize"] = dict(bytes=2 * m["rows"] * m["hidden"] * 2 + m["rows"] * 4, elems=m["rows"] * m["hidden"])
+    q = c["rmsnorm_head128"]
+    out["rmsnorm_head128"] = dict(bytes=2 * q["rows"] * q["hidden"] * 2 + q["hidden"] * 4, elems=q["rows"] * q["hidden"])
+    q = c["softmax_vocab"]
+    out["softmax_vocab"] = dict(bytes=2 * q["rows"] * q["cols"] * 2, elems=q["rows"] * q["cols"])
     t = c["gru_cell"]
     out["gru_cell"] = dict(bytes=(2 * 3 + 2) * t["rows"] * t["hidden"] * 2 + 6 * t["hidden"] * 4, elems=t["rows"] * t["hidden"])
     u = c["cumsum"]
@@ -257,7 +261,7 @@ class Workload:
 
     ORDER = ["softmax_small", "softmax_large", "layernorm", "bn_pool", "ce_loss", "rmsnorm", "silu_mul", "residual_add"]
     # Beyond the benchmark configs (not part of `value`): the two kernels the paper's case studies print.
-    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "layernorm_params16", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc", "pool2d", "reduce_max", "reduce_logsumexp", "bias_gelu", "residual_rmsnorm", "l2_normalize", "lstm_cell", "gru_cell"]
+    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "layernorm_params16", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc", "pool2d", "reduce_max", "reduce_logsumexp", "bias_gelu", "residual_rmsnorm", "l2_normalize", "lstm_cell", "gru_cell", "rmsnorm_head128", "softmax_vocab"]
 
     def __init__(self, kop, device, seed, only=None, rows_div=1):
         """only: build just these segments (None = all, plus the MLP segment); rows_div cuts the row
@@ -346,6 +350,15 @@ class Workload:
             t = c["gru_cell"]
             self.ui, self.uh, self.ubi, self.ubh, self.up = synth.gru_inputs(cut(t["rows"]), t["hidden"], t["dtype"], seed, dev)
             self.uo = torch.empty_like(self.up)
+        if "rmsnorm_head128" in want:
+            q = c["rmsnorm_head128"]
+            self.qkx, _ = synth.softmax_inputs(cut(q["rows"]), q["hidden"], q["dtype"], seed, dev)
+            self.qkw = torch.ones(q["hidden"], dtype=torch.float32, device=dev)
+            self.qky = torch.empty_like(self.qkx)
+        if "softmax_vocab" in want:
+            q = c["softmax_vocab"]
+            self.vx2, _ = synth.softmax_inputs(cut(q["rows"]), q["cols"], q["dtype"], seed, dev)
+            self.vy2 = torch.empty_like(self.vx2)
         if "cumsum" in want:
             u = c["cumsum"]
             self.ux, _ = synth.cumsum_inputs(cut(u["rows"]), u["cols"], u["dtype"], seed, dev)
@@ -437,6 +450,10 @@ class Workload:
             if not hasattr(self, "l2n"):
                 self.l2n = torch.empty(self.h.shape[0], dtype=torch.float32, device=self.h.device)
             k.kop_lp_normalize_rows(self.h, 2, 1e-12, out=self.n, norms=self.l2n)
+        elif name == "rmsnorm_head128":          # per-head RMSNorm: bf16 [1048576, 128], lanes-per-row kernel
+            k.kop_rmsnorm(self.qkx, self.qkw, c["rmsnorm_head128"]["eps"], out=self.qky)
+        elif name == "softmax_vocab":            # softmax over a vocabulary: bf16 [2048, 128256], two-sweep kernel
+            k.kop_softmax_scale_bias(self.vx2, None, 1.0, out=self.vy2)
         elif name == "gru_cell":                 # gate sums, activations and state update, bf16 [16384, 3 x 1024]
             k.kop_gru_cell(self.ui, self.uh, self.up, self.ubi, self.ubh, h_out=self.uo)
         elif name == "cumsum":                   # inclusive running sum along rows, fp32 [32768, 4096]

@@ -117,6 +117,36 @@ __device__ __forceinline__ void st_stream(void* p, const Vec16& v)
                  : "memory");
 }
 
+// L2 eviction policies for the kernels that read a row twice: the first sweep asks the L2 to keep what it reads
+// (evict_last), the second sweep and the output stores mark their lines as the first to go (evict_first), so that
+// the rows in flight, not the finished ones, occupy the L2.
+__device__ __forceinline__ uint64_t l2_policy_keep()
+{
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_drop()
+{
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ Vec16 ld_stream_hint(const void* p, uint64_t policy)
+{
+    Vec16 v;
+    asm volatile("ld.global.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=r"(v.w[0]), "=r"(v.w[1]), "=r"(v.w[2]), "=r"(v.w[3])
+                 : "l"(p), "l"(policy));
+    return v;
+}
+__device__ __forceinline__ void st_stream_hint(void* p, const Vec16& v, uint64_t policy)
+{
+    asm volatile("st.global.L2::cache_hint.v4.u32 [%0], {%1,%2,%3,%4}, %5;"
+                 :: "l"(p), "r"(v.w[0]), "r"(v.w[1]), "r"(v.w[2]), "r"(v.w[3]), "l"(policy)
+                 : "memory");
+}
+
 __device__ __forceinline__ float4 ldg_f4(const float* p)
 {
     return __ldg(reinterpret_cast<const float4*>(p));

@@ -382,7 +382,8 @@ ln_long_kernel(const T* __restrict__ x, const T* __restrict__ res, const PT* __r
     const int nbatch = (nvec + step - 1) / step;
 
     // the U vectors of batch b that belong to this thread, as v = prologue(x, bias, residual); false past the end
-    auto load_batch = [&](int b, float2 (&val)[U][P], bool (&in)[U]) {
+    const uint64_t keep = l2_policy_keep(), drop = l2_policy_drop();
+    auto load_batch = [&](int b, float2 (&val)[U][P], bool (&in)[U], uint64_t policy) {
         Vec16 rx[U], rres[U];
 #pragma unroll
         for (int k = 0; k < U; ++k) {
@@ -391,8 +392,8 @@ ln_long_kernel(const T* __restrict__ x, const T* __restrict__ res, const PT* __r
             rx[k] = Vec16{{0u, 0u, 0u, 0u}};
             rres[k] = Vec16{{0u, 0u, 0u, 0u}};
             if (in[k]) {
-                rx[k] = ld_stream(xr + (int64_t)v * E);
-                if (pro_has_residual(PRO)) rres[k] = ld_stream(rr + (int64_t)v * E);
+                rx[k] = ld_stream_hint(xr + (int64_t)v * E, policy);
+                if (pro_has_residual(PRO)) rres[k] = ld_stream_hint(rr + (int64_t)v * E, policy);
             }
         }
 #pragma unroll
@@ -415,7 +416,7 @@ ln_long_kernel(const T* __restrict__ x, const T* __restrict__ res, const PT* __r
     for (int b = 0; b < nbatch; ++b) {
         float2 val[U][P];
         bool in[U];
-        load_batch(b, val, in);
+        load_batch(b, val, in, keep);
 #pragma unroll
         for (int k = 0; k < U; ++k)
 #pragma unroll
@@ -428,7 +429,7 @@ ln_long_kernel(const T* __restrict__ x, const T* __restrict__ res, const PT* __r
     for (int b = nbatch - 1; b >= 0; --b) {
         float2 val[U][P];
         bool in[U];
-        load_batch(b, val, in);
+        load_batch(b, val, in, keep);
 #pragma unroll
         for (int k = 0; k < U; ++k)
 #pragma unroll
@@ -446,7 +447,7 @@ ln_long_kernel(const T* __restrict__ x, const T* __restrict__ res, const PT* __r
     for (int b = 0; b < nbatch; ++b) {
         float2 val[U][P];
         bool in[U];
-        load_batch(b, val, in);
+        load_batch(b, val, in, drop);
 #pragma unroll
         for (int k = 0; k < U; ++k) {
             const int v = b * step + k * blockDim.x + threadIdx.x;
@@ -456,7 +457,7 @@ ln_long_kernel(const T* __restrict__ x, const T* __restrict__ res, const PT* __r
                 load_params<E, false>(beta + (int64_t)v * E, be);
 #pragma unroll
                 for (int q = 0; q < P; ++q) o[q] = __ffma2_rn(__fmul2_rn(__fadd2_rn(val[k][q], nmu), rs2), g[q], be[q]);
-                st_stream(yr + (int64_t)v * E, Elem<T>::pack2(o));
+                st_stream_hint(yr + (int64_t)v * E, Elem<T>::pack2(o), drop);
             }
         }
     }

@@ -121,6 +121,7 @@ lpnorm_long_kernel(const T* __restrict__ x, T* __restrict__ y, float* __restrict
     T* yr = y + row * y_stride;
     const int step = U * blockDim.x;
     const int nbatch = (nvec + step - 1) / step;
+    const uint64_t keep = l2_policy_keep(), drop = l2_policy_drop();
     float2 acc = make_float2(0.0f, 0.0f);
     for (int b = 0; b < nbatch; ++b) {
         Vec16 raw[U];
@@ -128,7 +129,7 @@ lpnorm_long_kernel(const T* __restrict__ x, T* __restrict__ y, float* __restrict
         for (int k = 0; k < U; ++k) {
             const int v = b * step + k * blockDim.x + threadIdx.x;
             raw[k] = Vec16{{0u, 0u, 0u, 0u}};
-            if (v < nvec) raw[k] = ld_stream(xr + (int64_t)v * E);
+            if (v < nvec) raw[k] = ld_stream_hint(xr + (int64_t)v * E, keep);
         }
 #pragma unroll
         for (int k = 0; k < U; ++k) {
@@ -149,7 +150,7 @@ lpnorm_long_kernel(const T* __restrict__ x, T* __restrict__ y, float* __restrict
 #pragma unroll
         for (int k = 0; k < U; ++k) {
             const int v = b * step + k * blockDim.x + threadIdx.x;
-            if (v < nvec) raw[k] = ld_stream(xr + (int64_t)v * E);
+            if (v < nvec) raw[k] = ld_stream_hint(xr + (int64_t)v * E, drop);
         }
 #pragma unroll
         for (int k = 0; k < U; ++k) {
@@ -159,7 +160,7 @@ lpnorm_long_kernel(const T* __restrict__ x, T* __restrict__ y, float* __restrict
                 Elem<T>::unpack2(raw[k], val);
 #pragma unroll
                 for (int q = 0; q < Q; ++q) val[q] = __fmul2_rn(val[q], inv2);
-                st_stream(yr + (int64_t)v * E, Elem<T>::pack2(val));
+                st_stream_hint(yr + (int64_t)v * E, Elem<T>::pack2(val), drop);
             }
         }
     }

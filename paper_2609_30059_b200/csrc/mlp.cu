@@ -182,6 +182,7 @@ rmsnorm_long_kernel(const T* __restrict__ x, const PT* __restrict__ w, T* __rest
     T* hr = kRes ? static_cast<T*>(rr.h) + row * rr.h_stride : nullptr;
     const int step = U * blockDim.x;
     const int nbatch = (nvec + step - 1) / step;
+    const uint64_t keep = l2_policy_keep(), drop = l2_policy_drop();
     float2 ss2 = make_float2(0.0f, 0.0f);
     for (int b = 0; b < nbatch; ++b) {
         Vec16 raw[U], rraw[kRes ? U : 1];
@@ -191,8 +192,8 @@ rmsnorm_long_kernel(const T* __restrict__ x, const PT* __restrict__ w, T* __rest
             raw[k] = Vec16{{0u, 0u, 0u, 0u}};
             if (kRes) rraw[k] = Vec16{{0u, 0u, 0u, 0u}};
             if (v < nvec) {
-                raw[k] = ld_stream(xr + (int64_t)v * E);
-                if (kRes) rraw[k] = ld_stream(resr + (int64_t)v * E);
+                raw[k] = ld_stream_hint(xr + (int64_t)v * E, keep);
+                if (kRes) rraw[k] = ld_stream_hint(resr + (int64_t)v * E, keep);
             }
         }
 #pragma unroll
@@ -217,8 +218,8 @@ rmsnorm_long_kernel(const T* __restrict__ x, const PT* __restrict__ w, T* __rest
         for (int k = 0; k < U; ++k) {
             const int v = b * step + k * blockDim.x + threadIdx.x;
             if (v < nvec) {
-                raw[k] = ld_stream(xr + (int64_t)v * E);
-                if (kRes) rraw[k] = ld_stream(resr + (int64_t)v * E);
+                raw[k] = ld_stream_hint(xr + (int64_t)v * E, drop);
+                if (kRes) rraw[k] = ld_stream_hint(resr + (int64_t)v * E, drop);
             }
         }
 #pragma unroll
@@ -232,12 +233,12 @@ rmsnorm_long_kernel(const T* __restrict__ x, const PT* __restrict__ w, T* __rest
                     Elem<T>::unpack2(rraw[k], rv);
 #pragma unroll
                     for (int q = 0; q < P; ++q) val[q] = __fadd2_rn(val[q], rv[q]);
-                    st_stream(hr + (int64_t)v * E, Elem<T>::pack2(val));
+                    st_stream_hint(hr + (int64_t)v * E, Elem<T>::pack2(val), drop);
                 }
                 load_params<E, false>(w + (int64_t)v * E, g);
 #pragma unroll
                 for (int q = 0; q < P; ++q) o[q] = __fmul2_rn(__fmul2_rn(val[q], r2), g[q]);
-                st_stream(yr + (int64_t)v * E, Elem<T>::pack2(o));
+                st_stream_hint(yr + (int64_t)v * E, Elem<T>::pack2(o), drop);
             }
         }
     }

@@ -203,6 +203,7 @@ softmax_twosweep_kernel(const T* __restrict__ x, const float* __restrict__ bias,
         }
     };
 
+    const uint64_t keep = l2_policy_keep(), drop = l2_policy_drop();
     float m = -INFINITY, s = 0.0f;
     for (int b = 0; b < nbatch; ++b) {
         Vec16 raw[U];
@@ -210,7 +211,7 @@ softmax_twosweep_kernel(const T* __restrict__ x, const float* __restrict__ bias,
 #pragma unroll
         for (int k = 0; k < U; ++k) {
             const int v = b * step + k * blockDim.x + threadIdx.x;
-            if (v < nvec) raw[k] = ld_stream(xr + (int64_t)v * E);
+            if (v < nvec) raw[k] = ld_stream_hint(xr + (int64_t)v * E, keep);
         }
         float bm = -INFINITY;
 #pragma unroll
@@ -245,7 +246,7 @@ softmax_twosweep_kernel(const T* __restrict__ x, const float* __restrict__ bias,
 #pragma unroll
         for (int k = 0; k < U; ++k) {
             const int v = b * step + k * blockDim.x + threadIdx.x;
-            if (v < nvec) raw[k] = ld_stream(xr + (int64_t)v * E);
+            if (v < nvec) raw[k] = ld_stream_hint(xr + (int64_t)v * E, drop);
         }
 #pragma unroll
         for (int k = 0; k < U; ++k) {
@@ -258,7 +259,7 @@ softmax_twosweep_kernel(const T* __restrict__ x, const float* __restrict__ bias,
                     const float d = t[e] - M;
                     o[e] = log_out ? (d - lg) * kLn2 : ex2_approx(d) * inv;
                 }
-                st_stream(yr + (int64_t)v * E, Elem<T>::pack(o));
+                st_stream_hint(yr + (int64_t)v * E, Elem<T>::pack(o), drop);
             }
         }
     }
@@ -358,9 +359,10 @@ kop_status_t launch_softmax(const void* xv, const float* bias, void* yv, int64_t
         return launch_status();
     }
     if (rows > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
-    // rows up to 32 KB stay in one CTA's registers; longer ones take the two-sweep kernel (fp32 rows of 12288 /
-    // 16384 columns: 3.3 / 3.6 TB/s in registers with 64 values a thread, 4.0 / 4.3 TB/s in two sweeps)
-    if (vec && cols <= kMaxRegisterRow && cols * (int64_t)sizeof(T) <= 32768) {
+    // 16-bit rows up to 32 KB and fp32 rows up to 16 KB stay in one CTA's registers; longer ones take the two-sweep
+    // kernel (fp32 rows of 8192 / 16384 columns: 4.3 / 3.6 TB/s in registers, 4.8 / 5.5 TB/s in two sweeps with the L2
+    // eviction hints; bf16 rows of 16384 columns: 4.6 in registers against 4.0)
+    if (vec && cols <= kMaxRegisterRow && cols * (int64_t)sizeof(T) <= (sizeof(T) == 4 ? 16384 : 32768)) {
         const int nvec = (int)nvec64;
         // Per-thread vector count: 16 values per thread while the CTA stays within 1024 threads
         // keeps many CTAs resident; longer rows double the count (and halve the CTA limit).

@@ -32,6 +32,10 @@ CONFIGS = {
     # pointwise part of one LSTM step: batch 16384, hidden 1024 (shape ours)
     "lstm_cell": dict(rows=16384, hidden=1024, dtype=torch.bfloat16),
     "gru_cell": dict(rows=16384, hidden=1024, dtype=torch.bfloat16),
+    # shapes away from the benchmark's row lengths (ours): per-head RMSNorm of 16384 tokens x 64 heads of 128, and a
+    # softmax over a 128256-entry vocabulary
+    "rmsnorm_head128": dict(rows=1048576, hidden=128, eps=1e-6, dtype=torch.bfloat16),
+    "softmax_vocab": dict(rows=2048, cols=128256, scale=1.0, dtype=torch.bfloat16),
     # row reductions (shape ours)
     "reduce": dict(rows=32768, cols=8192, dtype=torch.bfloat16),
 }
