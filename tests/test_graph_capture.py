@@ -36,6 +36,7 @@ def test_all_entry_points_in_one_graph(kop):
     h, w, W1, W2 = synth.mlp_inputs(64, 256, 512, BF16, 10, dev)
     tg, tg2, tb, tc = synth.lstm_inputs(rows, 96, BF16, 11, dev)
     ui, uh, ubi, ubh, up = synth.gru_inputs(rows, 96, BF16, 12, dev)
+    lb16, lg16, lbe16 = lb.to(lx.dtype), lg.to(lx.dtype), lbe.to(lx.dtype)
     handle = kop.MlpHandle()
     ws_ce = torch.empty(max(16, kop.kop_ce_loss_rowwise_workspace_bytes(rows, cols, kop.KOP_BF16)), dtype=torch.uint8, device=dev)
     ws_mlp = torch.empty(kop.kop_rmsnorm_swiglu_residual_workspace_bytes(64, 256, 512, kop.KOP_BF16), dtype=torch.uint8, device=dev)
@@ -57,6 +58,7 @@ def test_all_entry_points_in_one_graph(kop):
         "act": torch.empty_like(x), "chain": torch.empty_like(x), "mlp": torch.empty_like(h),
         "rr_h": torch.empty_like(lx), "rr_y": torch.empty_like(lx), "lstm_h": torch.empty_like(tc), "lstm_c": torch.empty_like(tc),
         "gru_h": torch.empty_like(up), "lpn": torch.empty_like(lx), "lpn_n": torch.empty(rows, device=dev),
+        "ln_ex": torch.empty_like(lx), "rms_ex_h": torch.empty_like(lx), "rms_ex_y": torch.empty_like(lx),
     }
 
     def run():
@@ -87,6 +89,8 @@ def test_all_entry_points_in_one_graph(kop):
         kop.kop_lstm_cell(tg, tc, tg2, tb, h_out=o["lstm_h"], c_out=o["lstm_c"])
         kop.kop_gru_cell(ui, uh, up, ubi, ubh, h_out=o["gru_h"])
         kop.kop_lp_normalize_rows(lx, 2, 1e-12, out=o["lpn"], norms=o["lpn_n"])
+        kop.kop_layernorm_ex(lx, lr, lb16, lg16, lbe16, 1e-5, "bias_erfgelu_residual", out=o["ln_ex"], want_stats=False)
+        kop.kop_rmsnorm_ex(lx, lg16, 1e-6, residual=lr, h_out=o["rms_ex_h"], out=o["rms_ex_y"])
         kop.kop_rmsnorm_swiglu_residual(handle, h, w, W1, W2, 1e-6, out=o["mlp"], workspace=ws_mlp)
 
     try:
