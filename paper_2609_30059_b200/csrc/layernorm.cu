@@ -70,7 +70,7 @@ __device__ __forceinline__ float prologue1(float x, float b, float r)
 // with one 256-bit load per lane, so a warp touches each 128-byte line once (two 128-bit loads
 // per lane would walk every line twice and double the L1 wavefronts, which bound this kernel).
 template <typename T, typename PT, int VPT, bool kFull, bool kWide, int PRO>
-__global__ void __launch_bounds__(max_threads_for(VPT * Elem<T>::kPerVec))
+__global__ void __launch_bounds__(max_threads_for(VPT * Elem<T>::kPerVec), VPT * Elem<T>::kPerVec >= 32 ? 2 : 1)
 ln_block_kernel(const T* __restrict__ x, const T* __restrict__ res, const PT* __restrict__ bias,
                 const PT* __restrict__ gamma, const PT* __restrict__ beta, T* __restrict__ y,
                 float* __restrict__ mean, float* __restrict__ rstd, int nvec, int64_t x_stride,

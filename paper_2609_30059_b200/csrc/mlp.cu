@@ -22,7 +22,7 @@ struct RmsRes {
 };
 
 template <typename T, typename PT, int VPT, bool kFull, bool kWide, bool kRes>
-__global__ void __launch_bounds__(max_threads_for(VPT * Elem<T>::kPerVec))
+__global__ void __launch_bounds__(max_threads_for(VPT * Elem<T>::kPerVec), VPT * Elem<T>::kPerVec >= 32 ? 2 : 1)
 rmsnorm_block_kernel(const T* __restrict__ x, const PT* __restrict__ w, T* __restrict__ y, int nvec,
                      int64_t x_stride, int64_t y_stride, float eps, float inv_hidden, RmsRes rr)
 {
