@@ -53,11 +53,11 @@ FALLBACK_HBM_GBS = 6650.0
 NCU_DRAM_TRAFFIC_BYTES = {
     "ce_loss": 4 * (524355584 + 3218944),
     "silu_mul": 2 * (469769216 + 180785920),
-    "softmax_large": 268447232 + 210064896,
-    "layernorm": 134281728 + 10796544,
-    "bn_pool": 205531136 + 148790528,
-    "rmsnorm": 134242560 + 77360128,
-    "residual_add": 268443648 + 81811200,
+    "softmax_large": 268446720 + 209117184,
+    "layernorm": 134281984 + 11015680,
+    "bn_pool": 205530368 + 148711424,
+    "rmsnorm": 134260736 + 77681152,
+    "residual_add": 268452352 + 81950464,
 }
 
 
