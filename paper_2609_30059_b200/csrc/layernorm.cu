@@ -529,7 +529,13 @@ kop_status_t launch_ln(const void* xv, const void* rv, const void* biasv, const 
     const int64_t nvec64 = hidden / E;
     // rows of at most 128 vectors: lanes-per-row kernel (bf16 rows of 64 / 256 / 512 columns ran at 0.5 / 1.9 /
     // 3.8 TB/s with a CTA per row, 5 - 6 TB/s this way)
-    if (vec && nvec64 <= 128) {
+    // (16-bit rows of 512 columns and up that can go two to a CTA do better there: the row-pair kernel fetches
+    // the fp32 parameters once for two rows, and those loads, not HBM, bound the lanes-per-row kernel on 16-bit
+    // data: 4.9 - 5.0 TB/s against 6.2)
+    const bool pair_ok = vec && (nvec64 % (16 / E)) == 0 && ((nvec64 / (16 / E)) % 32) == 0 &&
+                         nvec64 / (16 / E) >= (sizeof(T) == 2 ? 32 : 128) && nvec64 / (16 / E) <= 320 &&
+                         rows >= 8 * (int64_t)sm_count();
+    if (vec && nvec64 <= 128 && !pair_ok) {
         const int nvec = (int)nvec64;
         const int lanes = nvec > 64 ? 32 : nvec > 32 ? 16 : nvec > 16 ? 8 : nvec > 8 ? 4 : 2;
         const int64_t rows_per_cta = 8 * (32 / lanes);
@@ -553,15 +559,15 @@ kop_status_t launch_ln(const void* xv, const void* rv, const void* biasv, const 
         // thread and ~8 CTAs per SM); short rows use fewer, rows beyond 512 threads' worth use 64.
         const bool wide = sizeof(PT) == 4 && E == 8 && (!pro_has_bias(PRO) || aligned_to(bias, 32)) && aligned_to(gamma, 32) &&
                           aligned_to(beta, 32);
-        // Rows of 2048..5120 elements that split evenly into 16 values per thread go two per CTA
+        // Rows of up to 5120 elements that split evenly into 16 values per thread (from 512 elements for 16-bit data,
+        // 2048 for fp32) go two per CTA
         // (parameters fetched once per pair) once there are enough pairs to fill the GPU. Longer rows do
         // better one per CTA with 32 values a thread (bf16 [8192, 8192]: 86 us against 106 us; 6144: 66
         // against 90), where the pair kernel's 384- to 512-thread CTAs leave one CTA per SM.
         {
             const int vpt2 = 16 / E;
             const int threads2 = nvec / vpt2;
-            if (nvec % vpt2 == 0 && threads2 % 32 == 0 && threads2 >= 128 && threads2 <= 320 &&
-                rows >= 8 * (int64_t)sm_count()) {
+            if (pair_ok) {
                 const unsigned grid = (unsigned)((rows + 1) / 2);
 #define KOP_LN_PAIR(W, MT)                                                                              \
     ln_pair_kernel<T, PT, 16 / E, W, MT, PRO><<<grid, threads2, 0, stream>>>(x, r, bias, gamma, beta, y, mean, rstd, \
