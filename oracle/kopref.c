@@ -547,6 +547,23 @@ int kopref_ce_loss_opts(const void* logits, const int32_t* labels, double* loss,
     return 0;
 }
 
+/* Cross-entropy with reduction "sum": the per-row losses of kopref_ce_loss_opts (same options) added up over
+ * the rows that count, i.e. mean * counted_rows without the division. No counted row gives 0 (an empty sum). */
+int kopref_ce_loss_sum(const void* logits, const int32_t* labels, double* loss, double* sum_loss,
+        int64_t rows, int64_t vocab, int64_t row_stride, int32_t ignore_index, double smoothing, int dtype,
+        int threads)
+{
+    if (!sum_loss) return -1;
+    int rc = kopref_ce_loss_opts(logits, labels, loss, NULL, NULL, NULL, rows, vocab, row_stride, ignore_index,
+                                 smoothing, dtype, threads);
+    if (rc != 0) return rc;
+    double total = 0.0;
+    for (int64_t i = 0; i < rows; ++i)
+        if (labels[i] != ignore_index) total += loss[i];
+    *sum_loss = total;
+    return 0;
+}
+
 /* ---- GroupNorm (InstanceNorm when groups == C) + activation, NCHW -------------------------------------------
  * For every image n and group g (C/groups consecutive channels): mu, var (biased) over the group's
  * (C/groups) * H * W elements; y = (x - mu) / sqrt(var + eps) * gamma[c] + beta[c] (gamma / beta may be NULL:

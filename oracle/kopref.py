@@ -48,6 +48,7 @@ def lib() -> C.CDLL:
         _lib.kopref_residual_layernorm.argtypes = [vp] * 7 + [i64] * 5 + [dbl, C.c_int, C.c_int]
         _lib.kopref_silu_mul_interleaved.argtypes = [vp] * 2 + [i64] * 4 + [C.c_int, C.c_int]
         _lib.kopref_ce_loss_opts.argtypes = [vp] * 6 + [i64] * 3 + [C.c_int32, dbl, C.c_int, C.c_int]
+        _lib.kopref_ce_loss_sum.argtypes = [vp] * 4 + [i64] * 3 + [C.c_int32, dbl, C.c_int, C.c_int]
         _lib.kopref_groupnorm_act.argtypes = [vp] * 6 + [i64] * 5 + [dbl, C.c_int, C.c_int, C.c_int]
         _lib.kopref_row_scale.argtypes = [vp, vp, vp, i64, i64, i64, i64, C.c_int, C.c_int]
         _lib.kopref_affine_relu_pool2d.argtypes = [vp] * 4 + [i64] * 4 + [C.c_int] * 10
@@ -324,6 +325,20 @@ def ce_loss_opts(logits, labels, ignore_index=-100, smoothing=0.0, threads=1):
                                      C.addressof(cnt), rows, vocab, vocab, int(ignore_index), float(smoothing),
                                      dt, _nt(threads)), "ce_loss_opts")
     return loss, mean.value, bad.value, cnt.value
+
+
+def ce_loss_sum(logits, labels, ignore_index=-100, smoothing=0.0, threads=1) -> float:
+    """Cross-entropy with reduction "sum": the per-row losses added over the rows whose label is not ignore_index."""
+    za, dt = as_data(logits)
+    rows, vocab = za.shape
+    if hasattr(labels, "detach"):
+        labels = labels.detach().cpu().numpy()
+    lab = np.ascontiguousarray(labels, dtype=np.int32)
+    loss = np.empty(rows, dtype=np.float64)
+    total = C.c_double(0.0)
+    _check(lib().kopref_ce_loss_sum(_p(za), _p(lab), _p(loss), C.addressof(total), rows, vocab, vocab,
+                                    int(ignore_index), float(smoothing), dt, _nt(threads)), "ce_loss_sum")
+    return total.value
 
 
 def groupnorm_act(x, gamma, beta, groups, eps, act=0, threads=1):

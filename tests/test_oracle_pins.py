@@ -544,6 +544,58 @@ def test_ce_options_against_library_and_base_oracle():
     assert b3 == 1 and c3 == 2 and math.isnan(l3[0]) and math.isnan(m3)
 
 
+def test_ce_sum_reduction_against_library_and_closed_forms():
+    M, V = 17, 53
+    z = f32(RNG.standard_normal((M, V)) * 2)
+    lab = RNG.integers(0, V, M).astype(np.int32)
+    lab[[0, 9]] = -100
+    tz, tl = torch.from_numpy(z.astype(np.float64)), torch.from_numpy(lab.astype(np.int64))
+    for s in (0.0, 0.2):
+        total = kopref.ce_loss_sum(z, lab, ignore_index=-100, smoothing=s)
+        ref = float(F.cross_entropy(tz, tl, reduction="sum", ignore_index=-100, label_smoothing=s))
+        assert total == pytest.approx(ref, rel=1e-13)
+        # sum = mean * counted rows, and = the sum of the per-row output
+        loss, mean, _, cnt = kopref.ce_loss_opts(z, lab, ignore_index=-100, smoothing=s)
+        assert total == pytest.approx(mean * cnt, rel=1e-13)
+        assert total == pytest.approx(math.fsum(loss), rel=1e-13)
+    # another ignore_index: label 5 no longer counts, -100 becomes a bad label (NaN sum)
+    lab5 = RNG.integers(0, V, M).astype(np.int32)
+    lab5[3] = 5
+    t5 = kopref.ce_loss_sum(z, lab5, ignore_index=5)
+    keep = lab5 != 5
+    ref5 = float(F.cross_entropy(tz[keep], torch.from_numpy(lab5[keep].astype(np.int64)), reduction="sum"))
+    assert t5 == pytest.approx(ref5, rel=1e-13)
+    assert math.isnan(kopref.ce_loss_sum(z, lab, ignore_index=5))
+    # closed forms: n uniform rows sum to n ln V whatever the smoothing; nothing counted sums to 0, not NaN
+    zu = f32(np.full((6, V), -0.25))
+    assert kopref.ce_loss_sum(zu, np.arange(6, dtype=np.int32), smoothing=0.4) == pytest.approx(6 * math.log(V), rel=1e-14)
+    assert kopref.ce_loss_sum(zu, np.full(6, -100, dtype=np.int32)) == 0.0
+    # two-class rows: loss = log1p(exp(-(z_label - z_other)))
+    z2 = f32(np.array([[1.5, -0.5], [0.25, 2.0]]))
+    want = math.log1p(math.exp(-2.0)) + math.log1p(math.exp(1.75))
+    assert kopref.ce_loss_sum(z2, np.array([0, 0], dtype=np.int32)) == pytest.approx(want, rel=1e-14)
+
+
+def test_ce_non_finite_logits_follow_the_shifted_definition():
+    # A NaN anywhere in a row, or a +inf logit (inf - inf in the max-shifted form), makes that row's loss NaN and
+    # leaves the other rows alone; -inf logits are ordinary (exp gives 0). torch's cross_entropy in float64 agrees.
+    V = 40
+    z = f32(RNG.standard_normal((6, V)))
+    z[1, 7] = np.nan
+    z[2, :] = np.nan
+    z[3, 0] = np.inf
+    z[4, 5] = -np.inf
+    lab = np.array([1, 2, 3, 4, 6, 39], dtype=np.int32)
+    loss, mean, bad = kopref.ce_loss_rowwise(z, lab)
+    ref = F.cross_entropy(torch.from_numpy(z.astype(np.float64)), torch.from_numpy(lab.astype(np.int64)),
+                          reduction="none").numpy()
+    assert np.array_equal(np.isnan(loss), [False, True, True, True, False, False])
+    assert np.array_equal(np.isnan(loss), np.isnan(ref))
+    ok = ~np.isnan(ref)
+    assert np.max(np.abs(loss[ok] - ref[ok])) <= 1e-13
+    assert math.isnan(mean) and bad == 0
+
+
 # --------------------------------------------------------------------------- GroupNorm / InstanceNorm + activation
 
 def test_groupnorm_library_invariants_and_instance_norm():

@@ -441,7 +441,10 @@ CE_SHAPES = [
 @pytest.mark.parametrize("seed", SEEDS)
 def test_ce_parity(kop, rows, vocab, dtype, seed):
     if rows * vocab > 40_000_000 and seed not in (0, 42):
-        pytest.skip("large shape: two seeds keep the CPU oracle time bounded")
+        # every seed runs at this row length; the other three use fewer rows (rows are independent, so the
+        # kernel variant is the same) to keep the CPU oracle's time bounded. 640 rows still span three ticket
+        # groups with a ragged last one.
+        rows = 640
     z, lab = synth.ce_inputs(rows, vocab, dtype, seed, "cuda")
     loss = Guarded((rows,), F32)
     mean = Guarded((1,), F32)

@@ -56,18 +56,23 @@ def strided(rng, t):
     return t
 
 
+LN_ILL_CONDITIONED = 32.0      # rstd * max|gamma| above which a row's bound gets the conditioning term
+
+
 def assert_close_ln(got, ref, rmean, rrstd, gamma, beta, tol, what):
     """LayerNorm outputs with the conditioning of the row taken into account. In fp32 the deviation v - mean carries
-    an absolute error of a few ulps of max|v|, which the normalisation multiplies by rstd * |gamma|; for ordinary
-    rows (rstd around 1) that is far below `tol`, but a random two- or three-column row can have a spread of 1e-3
-    (rstd 300) and then no fp32 evaluation order reaches 1e-5. The extra term is 8 ulp(fp32) * max|v| * rstd *
-    max|gamma| per row, with max|v| bounded from the oracle's own outputs."""
+    an absolute error of about one ulp of max|v| (2^-24 * max|v|), which the normalisation multiplies by
+    k = rstd * max|gamma|. With max|v| at most about 5 for these inputs the product stays below 1e-5 as long as
+    k <= 32, so every such row is held to the plain rule. Only rows beyond that (a random two- or three-column row
+    whose values differ by 1e-3 has rstd 300, and then no fp32 evaluation order reaches 1e-5) get the extra term
+    8 ulp(fp32) * max|v| * k, with max|v| bounded from the oracle's own outputs."""
     g = to_f64(got)
     ga = gamma.detach().cpu().double().numpy()
     be = beta.detach().cpu().double().numpy()
     dev = np.abs((ref - be) / (rrstd[:, None] * np.where(ga == 0.0, 1.0, ga)))            # |v - mean| per element
     vmax = np.abs(rmean) + dev.max(axis=1)
-    extra = 8.0 * 2.0 ** -24 * vmax * rrstd * np.abs(ga).max()
+    k = rrstd * np.abs(ga).max()
+    extra = np.where(k > LN_ILL_CONDITIONED, 8.0 * 2.0 ** -24 * vmax * k, 0.0)
     err = np.abs(g - ref)
     bound = tol * np.maximum(1.0, np.abs(ref)) + extra[:, None]
     assert np.all(err <= bound), f"{what}: max err {err.max():.3e} (worst bound excess {np.max(err - bound):.3e})"
