@@ -46,19 +46,17 @@ UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch at the benchmark shape, from the ncu captures
-# summarised under profiles/ (one file per kernel). The cross-entropy and SiLU*up captures ran on a
-# quarter / half of the rows (same row length, same kernel variant) and are scaled by the row count,
-# which their traffic is proportional to. Written-back bytes exclude dirty lines still in L2 at kernel end.
-NCU_DRAM_TRAFFIC_BYTES = {
-    "ce_loss": 4 * (524355584 + 3218944),
-    "silu_mul": 2 * (469769216 + 180785920),
-    "softmax_large": 268446720 + 209117184,
-    "layernorm": 134281984 + 11015680,
-    "bn_pool": 205530368 + 148711424,
-    "rmsnorm": 134260736 + 77681152,
-    "residual_add": 268452352 + 81950464,
-}
+
+
+def ncu_traffic(segment):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one launch at the benchmark shape, from the ncu captures
+    summarised under profiles/ (profiles/ncu_dram_traffic.json, written by paper_2609_30059_b200.ncu_summary
+    together with each summary, so the two cannot drift; a test compares them). Captures of the cross-entropy and
+    SiLU*up kernels ran on a quarter / half of the rows (same row length, same kernel variant) and are scaled by
+    the row count, which their traffic is proportional to. Written bytes exclude dirty lines still in L2 at
+    kernel end. None when no capture of that segment's kernel has been committed."""
+    from paper_2609_30059_b200 import ncu_summary
+    return ncu_summary.traffic_per_full_launch(segment)
 
 
 # ----------------------------------------------------------------------------- workload description
@@ -479,6 +477,49 @@ class Workload:
         self.graph = g
 
 
+def small_config_latency(wl, per_event_ms, reps=100, replays=20):
+    """The small softmax config ([128,512] fp32, 0.5 MB) is latency-bound, so it is reported three ways: the
+    CUDA-event time around one launch inside the fused step (includes the launch gap and event overhead), the mean
+    per launch over a CUDA graph of `reps` back-to-back launches (kernel + the GPU's own launch-to-launch gap, no
+    host in the way: what a C caller or a captured model sees), and the ncu duration of the kernel alone from the
+    committed capture. The Python binding's per-call cost is the fourth figure, for contrast."""
+    from paper_2609_30059_b200 import ncu_summary
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        wl.launch("softmax_small")
+        side.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            for _ in range(reps):
+                wl.launch("softmax_small")
+    torch.cuda.current_stream().wait_stream(side)
+    g.replay()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(replays):
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record()
+        g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        ts.append(e0.elapsed_time(e1) / reps * 1e3)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(1000):
+        wl.launch("softmax_small")
+    torch.cuda.synchronize()
+    binding_us = (time.perf_counter() - t0) / 1000 * 1e6
+    e = ncu_summary.load_traffic().get("softmax_small")
+    return {"event_us_per_launch_in_step": round(statistics.mean(per_event_ms) * 1e3, 2),
+            "graph_us_per_launch": round(statistics.median(ts), 3), "graph_us_per_launch_min": round(min(ts), 3),
+            "graph": f"{reps} back-to-back launches captured once, replayed {replays} times",
+            "ncu_duration_us": None if e is None else e["ncu_duration_us"],
+            "python_binding_us_per_call": round(binding_us, 2),
+            "what": "softmax fp32 [128,512]: 526,336 algorithmic bytes, 0.08 us at the HBM peak - latency-bound"}
+
+
 def run_ours(args, rank, world, local_rank):
     from paper_2609_30059_b200 import build as kbuild
     if rank == 0:
@@ -648,11 +689,23 @@ def run_ours(args, rank, world, local_rank):
     dom = max(names, key=lambda nm: statistics.mean(per[nm]))
     dom_ms = statistics.mean(per[dom])
     achieved = segs[dom]["bytes"] / (dom_ms * 1e-3) / 1e9
-    traffic = NCU_DRAM_TRAFFIC_BYTES.get(dom)
+    # every benchmark kernel's own roofline line (the top-level keys describe the dominant one): algorithmic bytes
+    # of one launch / its mean CUDA-event time over the timed steps, against the same measured peak
+    per_kernel = []
+    for nm in names:
+        ms = statistics.mean(per[nm])
+        gbs = segs[nm]["bytes"] / (ms * 1e-3) / 1e9
+        per_kernel.append(dict(kernel=nm, algorithmic_bytes=segs[nm]["bytes"], avg_launch_us=round(ms * 1e3, 2),
+                               achieved=round(gbs, 1), frac=round(gbs / peak, 4), traffic=ncu_traffic(nm)))
+    large = [k for k in per_kernel if k["kernel"] != "softmax_small"]       # 0.5 MB: latency-, not HBM-bound
+    worst = min(large, key=lambda k: k["frac"])
     roofline = dict(bound="hbm", kernel=dom, achieved=round(achieved, 1), peak=peak, unit="GB/s",
-                    frac=round(achieved / peak, 4), traffic=traffic, peak_source=peak_src,
-                    algorithmic_bytes=segs[dom]["bytes"], avg_launch_us=round(dom_ms * 1e3, 2))
+                    frac=round(achieved / peak, 4), traffic=ncu_traffic(dom), peak_source=peak_src,
+                    algorithmic_bytes=segs[dom]["bytes"], avg_launch_us=round(dom_ms * 1e3, 2),
+                    per_kernel=per_kernel, worst=dict(kernel=worst["kernel"], frac=worst["frac"],
+                                                      among="the large configs (softmax_small excluded)"))
 
+    small = small_config_latency(wl, per["softmax_small"]) if rank == 0 else None
     gate = perf_gate(wl, names, inductor=args.inductor) if (rank == 0 and not args.no_perf_gate) else None
     e2e = run_e2e(args, wl, kop, dev, segs, names, world)
     cpu = None
@@ -676,6 +729,7 @@ def run_ours(args, rank, world, local_rank):
             "gpu_launches": args.steps * len(names),
             "segments": seg_report,
             "roofline": roofline,
+            "softmax_small_latency": small,
             "frac_of_nominal_8TBs": round(value / world / NOMINAL_HBM_GBS, 4),
             "clocks": clocks,
             "mlp_segment_graph": {

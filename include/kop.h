@@ -171,6 +171,9 @@ kop_status_t kop_bn_relu_avgpool(const void* x, const float* scale, const float*
  * A label outside [0, vocab) gives loss NaN for that row and is counted in
  * *bad_label_count (then *mean_loss is NaN). The mean is summed in a fixed order:
  * results are bit-identical run to run.
+ * Non-finite logits follow the max-shifted definition lse = m + ln sum_j exp(z_j - m): -inf entries
+ * are ordinary (they add 0); a NaN anywhere in a row, or a +inf logit (exp(inf - inf)), makes that
+ * row's loss NaN (and with it the mean); a row of nothing but -inf is NaN too. Other rows are unaffected.
  * workspace: device scratch of at least kop_ce_loss_rowwise_workspace_bytes() bytes,
  * 16-byte aligned, contents irrelevant on entry (the call clears what it needs on
  * `stream`); calls sharing one workspace must not overlap on the GPU.
@@ -200,6 +203,7 @@ size_t kop_ce_loss_rowwise_workspace_bytes(int64_t rows, int64_t vocab, kop_dtyp
  * workspace pair, with these additions:
  *   limit     rows <= kop_ce_loss_rowwise_static_max_rows() (1,048,576). More rows return
  *             KOP_ERR_WORKSPACE_TOO_SMALL before anything is launched; use the workspace variant.
+ *             Like every entry point it checks all of its arguments before its first CUDA call.
  *   set-up    The first call on each device looks up the device address of the built-in array
  *             (once per device, with that device current). Make that first call outside any
  *             stream capture. The call itself never calls cudaMalloc, cudaFree or any allocating
@@ -218,15 +222,19 @@ kop_status_t kop_ce_loss_rowwise_static(const void* logits, const int32_t* label
 int64_t kop_ce_loss_rowwise_static_max_rows(void);
 
 /*
- * kop_ce_loss_rowwise with ignore_index and label smoothing (coverage variant of the same segment):
+ * kop_ce_loss_rowwise with ignore_index, label smoothing and all three reductions (coverage variant of the
+ * same segment; the reductions are the "none" / "mean" / "sum" forms of the loss):
  *   loss[i] = (1 - s) (lse_i - z[i, label_i]) + s (lse_i - (1/vocab) sum_j z[i,j]),  s = label_smoothing in [0, 1)
  * Rows whose label equals ignore_index get loss 0, are not read, and do not count;
- * *mean_loss = sum of counted losses / *counted_rows (NaN when no row counts); a label outside [0, vocab)
- * that is not ignore_index is a bad label as above. counted_rows: int32 [1] or NULL. Workspace as for
+ * *sum_loss = sum of the counted losses (0 when no row counts); *mean_loss = *sum_loss / *counted_rows (NaN
+ * when no row counts); both come from one fixed-order sum, so they are bit-identical run to run. A label
+ * outside [0, vocab) that is not ignore_index is a bad label as above (sum and mean NaN). loss: fp32 [rows]
+ * ("none"); mean_loss, sum_loss: fp32 [1] or NULL; counted_rows: int32 [1] or NULL. Workspace as for
  * kop_ce_loss_rowwise (same size function).
  */
 kop_status_t kop_ce_loss_rowwise_opts(const void* logits, const int32_t* labels,
-                                      float* loss, float* mean_loss, int32_t* bad_label_count,
+                                      float* loss, float* mean_loss, float* sum_loss,
+                                      int32_t* bad_label_count,
                                       int32_t* counted_rows, int64_t rows, int64_t vocab, int64_t row_stride,
                                       int32_t ignore_index, float label_smoothing,
                                       void* workspace, size_t workspace_bytes,
@@ -530,6 +538,18 @@ size_t kop_rmsnorm_swiglu_residual_workspace_bytes(int64_t rows, int64_t hidden,
  */
 kop_status_t kop_mlp_handle_create(void** handle);
 kop_status_t kop_mlp_handle_destroy(void* handle);
+
+/*
+ * The same handle around a cuBLAS handle the CALLER owns (problem formulation: the extern library calls and
+ * their set-up stay exactly as the surrounding program has them): cublas_handle is a cublasHandle_t created by
+ * the caller, on the current device, with the cuBLAS that this library is linked against (a handle from another
+ * copy of cuBLAS in the process is undefined). Nothing is created on the device: the call only allocates a
+ * few host bytes for the segment's settings. Every kop_rmsnorm_swiglu_residual call sets the handle's stream
+ * to its `stream` (and leaves it so), lends it the call's workspace and hands the handle back with cuBLAS's
+ * default workspace; its other settings (math mode; pointer mode must be host) are left alone.
+ * kop_mlp_handle_destroy frees the wrapper and leaves the caller's cuBLAS handle alive.
+ */
+kop_status_t kop_mlp_handle_wrap(void* cublas_handle, void** handle);
 
 /*
  * Vendor-library configuration of the segment (the paper's stated future work: besides rewriting the fused

@@ -40,12 +40,15 @@ def sources() -> list[str]:
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
 
 
-def _fingerprint(flags: list[str]) -> str:
-    """Hash of every source, header and flag that goes into the library. File times are useless for this:
+def _headers() -> list[str]:
+    return sorted(glob.glob(os.path.join(CSRC, "*.cuh"))) + sorted(glob.glob(os.path.join(INCLUDE, "*.h")))
+
+
+def _fingerprint(flags: list[str], srcs: list[str] | None = None) -> str:
+    """Hash of the given sources (default: all), every header and the flags. File times are useless for this:
     a copy of the tree (another machine, a fresh checkout) has new times on unchanged files."""
     h = hashlib.sha256()
-    files = sources() + sorted(glob.glob(os.path.join(CSRC, "*.cuh"))) + sorted(glob.glob(os.path.join(INCLUDE, "*.h")))
-    for f in files:
+    for f in (sources() if srcs is None else srcs) + _headers():
         h.update(os.path.basename(f).encode())
         with open(f, "rb") as fh:
             h.update(fh.read())
@@ -70,11 +73,21 @@ def build(force: bool = False, verbose: bool = False, extra_flags: list[str] | N
 
     def compile_one(src: str) -> str:
         obj = os.path.join(OBJ, os.path.basename(src)[:-3] + (".o" if out is None else f".{os.getpid()}.o"))
+        # an object whose source, headers and flags are unchanged is kept (not when forced or verbose)
+        ostamp = obj + ".stamp"
+        owant = _fingerprint(base_flags, [src])
+        if out is None and not force and not verbose and os.path.exists(obj) and os.path.exists(ostamp):
+            with open(ostamp) as fh:
+                if fh.read().strip() == owant:
+                    return obj
         res = subprocess.run([nvcc, *flags, "-c", src, "-o", obj], capture_output=True, text=True)
         if verbose or res.returncode != 0:
             sys.stderr.write(res.stdout + res.stderr)
         if res.returncode != 0:
             raise RuntimeError(f"nvcc failed on {src}")
+        if out is None:
+            with open(ostamp, "w") as fh:
+                fh.write(owant + "\n")
         return obj
 
     with concurrent.futures.ThreadPoolExecutor(max_workers=min(8, len(sources()))) as pool:
@@ -94,4 +107,4 @@ def build(force: bool = False, verbose: bool = False, extra_flags: list[str] | N
 
 
 if __name__ == "__main__":
-    print(build(force=True, verbose="-v" in sys.argv))
+    print(build(force="--incremental" not in sys.argv, verbose="-v" in sys.argv))

@@ -234,8 +234,8 @@ kop_status_t launch_bn(const void* xv, const float* scale, const float* shift, v
 // column t % TV and walks rows t / TV, t / TV + R, ... of the slab (R = 256 / TV rows per sweep, U of them
 // in flight) with its scale / shift values and running column sums in registers. When an image has too
 // few (tile) CTAs to fill the GPU its rows are split over a thread-block cluster of up to 8 CTAs: each
-// writes its column sums into the first CTA's shared memory (distributed shared memory), one cluster
-// barrier, and the first CTA adds them in rank order. No atomics, no workspace, and for a given call
+// writes its column sums into the first CTA's shared memory (distributed shared memory) once all CTAs of
+// the cluster are known to run, one cluster barrier, and the first CTA adds them in rank order. No atomics, no workspace, and for a given call
 // shape a fixed summation order.
 constexpr int kBnMaxSlabs = 8;      // portable cluster size
 
@@ -249,6 +249,10 @@ bn_nhwc_kernel(const T* __restrict__ x, const float* __restrict__ scale, const f
     constexpr int NT = 256, R = NT / TV;
     __shared__ float part[R][TV * E];
     __shared__ float from_ranks[kCluster ? kBnMaxSlabs : 1][TV * E];
+    // "This CTA has started": distributed shared memory may only be touched once every CTA of the cluster is
+    // running, so each arrives here and waits (below) just before the first remote store. The row sweep in
+    // between hides the wait.
+    if (kCluster) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     const int col = threadIdx.x % TV, phase = threadIdx.x / TV;
     const int slab = kCluster ? (int)cluster_rank() : 0;     // consecutive CTAs form a cluster
     const int64_t unit = blockIdx.x / slabs;                 // (image, channel tile)
@@ -302,8 +306,9 @@ bn_nhwc_kernel(const T* __restrict__ x, const float* __restrict__ scale, const f
         for (int r = 0; r < R; ++r) s += part[r][threadIdx.x];
     }
     if (kCluster) {
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");    // every CTA of the cluster has started
         if (threadIdx.x < TV * E) store_to_cluster_cta(&from_ranks[slab][threadIdx.x], 0u, s);
-        cluster_barrier();                                   // hardware barrier over the cluster's CTAs
+        cluster_barrier();                                   // the stores have landed in the first CTA
         if (slab != 0) return;
         if (threadIdx.x < TV * E) {
             s = 0.0f;

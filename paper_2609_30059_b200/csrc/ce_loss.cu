@@ -8,6 +8,8 @@
 // per-thread (M, S) pairs are merged across the CTA, lse = (M + log2 S) * ln 2, and thread 0
 // subtracts the label logit. The last CTA to finish (a ticket counter in the workspace; nobody
 // waits on it) sums loss[] in a fixed order, so the mean is bit-identical run to run.
+#include <atomic>
+
 #include "kop_common.cuh"
 
 namespace kop {
@@ -30,6 +32,7 @@ struct CeOpts {
     int32_t ignore_index;
     float smoothing;
     int32_t* counted_rows;
+    float* sum_loss;
 };
 __host__ __device__ inline int64_t ce_groups(int64_t rows) { return (rows + kGroupRows - 1) / kGroupRows; }
 __host__ __device__ inline CeWorkspace ce_workspace(void* base, int64_t rows)
@@ -134,6 +137,8 @@ __device__ __forceinline__ void ce_after_ticket(unsigned t, int64_t row, int lan
             // mean over the rows that count; no counted row gives 0 / 0 = NaN, as the definition does
             if (mean_loss != nullptr) *mean_loss = tot / (float)ncnt;
             if (opts.counted_rows != nullptr) *opts.counted_rows = (int32_t)ncnt;
+            // reduction "sum": the same fixed-order total before the division (ignored rows added 0)
+            if (opts.sum_loss != nullptr) *opts.sum_loss = tot;
         } else if (mean_loss != nullptr) *mean_loss = tot / (float)rows;
         if (bad_label_count != nullptr)
             *bad_label_count = (int32_t)(nbad > 0x7FFFFFFF ? 0x7FFFFFFF : nbad);
@@ -155,8 +160,9 @@ __device__ __forceinline__ void ce_finish(float M, float S, float Z, const T* zr
 {
     __shared__ float red_a[32], red_b[32], red_c[32];
     const float Mb = block_max(M, red_a);
-    // A thread that saw nothing has M = -inf and S = 0; keep its term at 0 rather than 0 * 2^nan.
-    const float Sb = block_sum(M == -INFINITY ? 0.0f : S * ex2_approx(M - Mb), red_b);
+    // A thread that saw nothing has M = -inf and S = 0; keep its term at 0 rather than 0 * 2^nan. A thread that
+    // saw only NaNs also has M = -inf, but S = NaN: S * 0 keeps that NaN in the row's sum.
+    const float Sb = block_sum(M == -INFINITY ? S * 0.0f : S * ex2_approx(M - Mb), red_b);
     float Zb = 0.0f;
     if (kSmooth) Zb = block_sum(Z, red_c);          // sum of the row's logits, for label smoothing
     if (threadIdx.x >= 32) return;
@@ -202,7 +208,9 @@ __device__ __forceinline__ void ce_batch(const T* zr, int base, int nvec, float&
 #pragma unroll
     for (int k = 1; k < VPT; ++k) cm = fmaxf(cm, vec_max<T>(raw[k]));
     const float cm2 = cm * kLog2e;
-    if (cm2 > -INFINITY) {
+    // != rather than >: a batch of nothing but NaNs has a NaN maximum (the packed max drops a NaN only against a
+    // number) and must enter, so that its ex2(NaN) terms reach S.
+    if (cm2 != -INFINITY) {
         const float newM = fmaxf(M, cm2);
         float s = S * ex2_approx(M - newM);          // M = -inf on the first batch: S * 0
         const float neg = -newM;
@@ -280,7 +288,7 @@ ce_group_kernel(const T* __restrict__ z, const int32_t* __restrict__ labels, flo
 #pragma unroll
         for (int k = 1; k < U; ++k) cm = fmaxf(cm, vec_max<T>(raw[k]));
         const float cm2 = cm * kLog2e;
-        if (cm2 > -INFINITY) {
+        if (cm2 != -INFINITY) {                              // a NaN maximum enters (see ce_batch)
             const float newM = fmaxf(M, cm2);
             float s = S * ex2_approx(M - newM);
             const float neg = -newM;
@@ -304,8 +312,8 @@ ce_group_kernel(const T* __restrict__ z, const int32_t* __restrict__ labels, flo
     for (int o = L / 2; o > 0; o >>= 1) {
         const float Mo = __shfl_xor_sync(0xFFFFFFFFu, M, o), So = __shfl_xor_sync(0xFFFFFFFFu, S, o);
         const float M2 = fmaxf(M, Mo);
-        const float a = M == -INFINITY ? 0.0f : S * ex2_approx(M - M2);
-        const float b = Mo == -INFINITY ? 0.0f : So * ex2_approx(Mo - M2);
+        const float a = M == -INFINITY ? S * 0.0f : S * ex2_approx(M - M2);       // S * 0 keeps a NaN sum
+        const float b = Mo == -INFINITY ? So * 0.0f : So * ex2_approx(Mo - M2);
         // the lower lane's term first on both sides, so that the two lanes agree bit for bit
         S = (lane & o) ? b + a : a + b;
         M = M2;
@@ -357,7 +365,9 @@ ce_row_scalar_kernel(const T* __restrict__ z, const int32_t* __restrict__ labels
         const float x2 = xj * kLog2e;
         if (x2 == -INFINITY) continue;
         if (x2 > M) {
-            S = S * ex2_approx(M - x2) + 1.0f;
+            // + 1 for this element; (x2 - x2) is 0 for a number and NaN for +inf, where the max-shifted
+            // definition has exp(inf - inf): the row becomes NaN as in the vector kernels
+            S = S * ex2_approx(M - x2) + (1.0f + (x2 - x2));
             M = x2;
         } else {
             S += ex2_approx(x2 - M);
@@ -431,6 +441,61 @@ extern "C" size_t kop_ce_loss_rowwise_workspace_bytes(int64_t rows, int64_t voca
     return kop::ce_workspace_bytes(rows);
 }
 
+namespace kop {
+namespace {
+
+// Static validation shared by the three cross-entropy entry points (no CUDA call). `done` is set when the call
+// has nothing to do (rows == 0). kOwnScratch: the scratch is the library's built-in array, so there is no
+// caller workspace to check, but the problem must fit the array.
+struct CeArgs {
+    const void* logits;
+    const int32_t* labels;
+    float* loss;
+    float* mean_loss;
+    int32_t* bad_label_count;
+    int32_t* counted_rows;
+    float* sum_loss;
+    int64_t rows, vocab, row_stride;
+    kop_dtype_t dtype;
+};
+kop_status_t ce_validate(const CeArgs& a, bool own_scratch, int64_t own_scratch_max_rows, const void* workspace,
+                         size_t workspace_bytes, bool* done)
+{
+    *done = false;
+    if (!dtype_ok(a.dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    kop_status_t st = check_rows_cols(a.rows, a.vocab);
+    if (st != KOP_OK) return st;
+    if (a.rows == 0) {
+        *done = true;
+        return KOP_OK;
+    }
+    if (own_scratch && a.rows > own_scratch_max_rows) return KOP_ERR_WORKSPACE_TOO_SMALL;
+    if (!a.logits || !a.labels || !a.loss || (!own_scratch && !workspace)) return KOP_ERR_NULL_POINTER;
+    if (a.vocab > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;            // labels are int32
+    if (a.rows > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;             // one CTA per row
+    if ((st = check_row_stride(a.row_stride, a.vocab, a.rows)) != KOP_OK) return st;
+    const int esz = elem_size(a.dtype);
+    if (!aligned_to(a.logits, esz) || !aligned_to(a.labels, 4) || !aligned_to(a.loss, 4) ||
+        (a.mean_loss && !aligned_to(a.mean_loss, 4)) || (a.bad_label_count && !aligned_to(a.bad_label_count, 4)) ||
+        (a.counted_rows && !aligned_to(a.counted_rows, 4)) || (a.sum_loss && !aligned_to(a.sum_loss, 4)) ||
+        (!own_scratch && !aligned_to(workspace, 16)))
+        return KOP_ERR_MISALIGNED;
+    if (!own_scratch && workspace_bytes < ce_workspace_bytes(a.rows)) return KOP_ERR_WORKSPACE_TOO_SMALL;
+    return KOP_OK;
+}
+
+template <bool kOpts>
+kop_status_t ce_dispatch(const CeArgs& a, void* workspace, cudaStream_t s, CeOpts opts)
+{
+    return a.dtype == KOP_F32
+               ? launch_ce<float, kOpts>(a.logits, a.labels, a.loss, a.mean_loss, a.bad_label_count, a.rows, a.vocab, a.row_stride, workspace, s, opts)
+               : a.dtype == KOP_BF16 ? launch_ce<__nv_bfloat16, kOpts>(a.logits, a.labels, a.loss, a.mean_loss, a.bad_label_count, a.rows, a.vocab, a.row_stride, workspace, s, opts)
+               : launch_ce<__half, kOpts>(a.logits, a.labels, a.loss, a.mean_loss, a.bad_label_count, a.rows, a.vocab, a.row_stride, workspace, s, opts);
+}
+
+}  // namespace
+}  // namespace kop
+
 extern "C" kop_status_t kop_ce_loss_rowwise(const void* logits, const int32_t* labels, float* loss,
                                             float* mean_loss, int32_t* bad_label_count, int64_t rows,
                                             int64_t vocab, int64_t row_stride, void* workspace,
@@ -438,31 +503,16 @@ extern "C" kop_status_t kop_ce_loss_rowwise(const void* logits, const int32_t* l
                                             kop_stream_t stream)
 {
     using namespace kop;
-    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
-    kop_status_t st = check_rows_cols(rows, vocab);
-    if (st != KOP_OK) return st;
-    if (rows == 0) return KOP_OK;
-    if (!logits || !labels || !loss || !workspace) return KOP_ERR_NULL_POINTER;
-    if (vocab > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;            // labels are int32
-    if (rows > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;             // one CTA per row
-    if ((st = check_row_stride(row_stride, vocab, rows)) != KOP_OK) return st;
-    const int esz = elem_size(dtype);
-    if (!aligned_to(logits, esz) || !aligned_to(labels, 4) || !aligned_to(loss, 4) ||
-        (mean_loss && !aligned_to(mean_loss, 4)) || (bad_label_count && !aligned_to(bad_label_count, 4)) ||
-        !aligned_to(workspace, 16))
-        return KOP_ERR_MISALIGNED;
-    if (workspace_bytes < kop_ce_loss_rowwise_workspace_bytes(rows, vocab, dtype))
-        return KOP_ERR_WORKSPACE_TOO_SMALL;
+    const CeArgs a{logits, labels, loss, mean_loss, bad_label_count, nullptr, nullptr, rows, vocab, row_stride, dtype};
+    bool done = false;
+    kop_status_t st = ce_validate(a, false, 0, workspace, workspace_bytes, &done);
+    if (st != KOP_OK || done) return st;
     if ((st = check_device()) != KOP_OK) return st;
-    cudaStream_t s = as_stream(stream);
-    return dtype == KOP_F32
-               ? launch_ce<float, false>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s, CeOpts{0, 0.0f, nullptr})
-               : dtype == KOP_BF16 ? launch_ce<__nv_bfloat16, false>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s, CeOpts{0, 0.0f, nullptr})
-               : launch_ce<__half, false>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s, CeOpts{0, 0.0f, nullptr});
+    return ce_dispatch<false>(a, workspace, as_stream(stream), CeOpts{0, 0.0f, nullptr, nullptr});
 }
 
 extern "C" kop_status_t kop_ce_loss_rowwise_opts(const void* logits, const int32_t* labels, float* loss,
-                                                 float* mean_loss, int32_t* bad_label_count,
+                                                 float* mean_loss, float* sum_loss, int32_t* bad_label_count,
                                                  int32_t* counted_rows, int64_t rows, int64_t vocab,
                                                  int64_t row_stride, int32_t ignore_index,
                                                  float label_smoothing, void* workspace,
@@ -470,28 +520,15 @@ extern "C" kop_status_t kop_ce_loss_rowwise_opts(const void* logits, const int32
                                                  kop_stream_t stream)
 {
     using namespace kop;
-    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
-    kop_status_t st = check_rows_cols(rows, vocab);
-    if (st != KOP_OK) return st;
-    if (!(label_smoothing >= 0.0f && label_smoothing < 1.0f)) return KOP_ERR_BAD_SHAPE;
-    if (rows == 0) return KOP_OK;
-    if (!logits || !labels || !loss || !workspace) return KOP_ERR_NULL_POINTER;
-    if (vocab > 0x7FFFFFFFLL || rows > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
-    if ((st = check_row_stride(row_stride, vocab, rows)) != KOP_OK) return st;
-    const int esz = elem_size(dtype);
-    if (!aligned_to(logits, esz) || !aligned_to(labels, 4) || !aligned_to(loss, 4) ||
-        (mean_loss && !aligned_to(mean_loss, 4)) || (bad_label_count && !aligned_to(bad_label_count, 4)) ||
-        (counted_rows && !aligned_to(counted_rows, 4)) || !aligned_to(workspace, 16))
-        return KOP_ERR_MISALIGNED;
-    if (workspace_bytes < kop_ce_loss_rowwise_workspace_bytes(rows, vocab, dtype))
-        return KOP_ERR_WORKSPACE_TOO_SMALL;
+    const CeArgs a{logits, labels, loss, mean_loss, bad_label_count, counted_rows, sum_loss, rows, vocab, row_stride, dtype};
+    if (dtype_ok(dtype) && check_rows_cols(rows, vocab) == KOP_OK &&
+        !(label_smoothing >= 0.0f && label_smoothing < 1.0f))
+        return KOP_ERR_BAD_SHAPE;
+    bool done = false;
+    kop_status_t st = ce_validate(a, false, 0, workspace, workspace_bytes, &done);
+    if (st != KOP_OK || done) return st;
     if ((st = check_device()) != KOP_OK) return st;
-    cudaStream_t s = as_stream(stream);
-    const CeOpts opts{ignore_index, label_smoothing, counted_rows};
-    return dtype == KOP_F32
-               ? launch_ce<float, true>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s, opts)
-               : dtype == KOP_BF16 ? launch_ce<__nv_bfloat16, true>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s, opts)
-               : launch_ce<__half, true>(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride, workspace, s, opts);
+    return ce_dispatch<true>(a, workspace, as_stream(stream), CeOpts{ignore_index, label_smoothing, counted_rows, sum_loss});
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -514,7 +551,9 @@ static __device__ __align__(256) unsigned int g_ce_static_scratch[kStaticScratch
 // In host code the array's name is only a stand-in for the symbol, not a device address: the address
 // the kernel needs comes from cudaGetSymbolAddress, asked once per device with that device current.
 constexpr int kStaticMaxDevices = 64;
-void* g_ce_static_ptr[kStaticMaxDevices];      // benign race: every writer stores the same value
+// Several host threads may make a device's first call together: each looks the address up and stores the same
+// value, so relaxed atomics are all the ordering this needs.
+std::atomic<void*> g_ce_static_ptr[kStaticMaxDevices];
 
 kop_status_t ce_static_scratch(void** out)
 {
@@ -524,15 +563,15 @@ kop_status_t ce_static_scratch(void** out)
         return KOP_ERR_CUDA;
     }
     if (dev < 0 || dev >= kStaticMaxDevices) return KOP_ERR_UNSUPPORTED_DEVICE;
-    if (g_ce_static_ptr[dev] == nullptr) {
-        void* p = nullptr;
+    void* p = g_ce_static_ptr[dev].load(std::memory_order_relaxed);
+    if (p == nullptr) {
         if (cudaGetSymbolAddress(&p, g_ce_static_scratch) != cudaSuccess || p == nullptr) {
             (void)cudaGetLastError();
             return KOP_ERR_CUDA;
         }
-        g_ce_static_ptr[dev] = p;
+        g_ce_static_ptr[dev].store(p, std::memory_order_relaxed);
     }
-    *out = g_ce_static_ptr[dev];
+    *out = p;
     return KOP_OK;
 }
 
@@ -548,17 +587,16 @@ extern "C" kop_status_t kop_ce_loss_rowwise_static(const void* logits, const int
                                                    kop_stream_t stream)
 {
     using namespace kop;
-    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
-    kop_status_t st = check_rows_cols(rows, vocab);
-    if (st != KOP_OK) return st;
-    if (rows == 0) return KOP_OK;
-    // Beyond the built-in scratch: refuse, loudly, before touching the device.
-    if (rows > kStaticMaxRows) return KOP_ERR_WORKSPACE_TOO_SMALL;
+    // All argument checks first, without touching the device: more rows than the built-in scratch holds, NULL or
+    // misaligned pointers and bad strides are refused before any CUDA call, as for every other entry point.
+    const CeArgs a{logits, labels, loss, mean_loss, bad_label_count, nullptr, nullptr, rows, vocab, row_stride, dtype};
+    bool done = false;
+    kop_status_t st = ce_validate(a, true, kStaticMaxRows, nullptr, 0, &done);
+    if (st != KOP_OK || done) return st;
     if ((st = check_device()) != KOP_OK) return st;
     void* scratch = nullptr;
     if ((st = ce_static_scratch(&scratch)) != KOP_OK) return st;
-    // Same validation, same clearing of the tickets on `stream`, same kernels as the caller-workspace
-    // entry point; only the scratch pointer differs.
-    return kop_ce_loss_rowwise(logits, labels, loss, mean_loss, bad_label_count, rows, vocab, row_stride,
-                               scratch, (size_t)kStaticScratchWords * sizeof(unsigned int), dtype, stream);
+    // Same clearing of the tickets on `stream`, same kernels as the caller-workspace entry point; only the
+    // scratch pointer differs.
+    return ce_dispatch<false>(a, scratch, as_stream(stream), CeOpts{0, 0.0f, nullptr, nullptr});
 }

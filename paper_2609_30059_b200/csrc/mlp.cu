@@ -737,6 +737,7 @@ kop_status_t gemm_nt(cublasHandle_t h, const void* A, const void* Wt, void* Cout
 // What kop_mlp_handle_create hands out: the vendor handle plus the segment's vendor-library configuration.
 struct MlpHandle {
     cublasHandle_t cb = nullptr;
+    bool owns_cb = true;           // false: the caller's own cuBLAS handle (kop_mlp_handle_wrap), never destroyed here
     bool residual_in_gemm = false;
     // single-entry cache of the cublasLt plan for the down projection with the residual epilogue
     bool plan_valid = false;
@@ -989,6 +990,17 @@ extern "C" kop_status_t kop_mlp_handle_create(void** handle)
     return KOP_OK;
 }
 
+extern "C" kop_status_t kop_mlp_handle_wrap(void* cublas_handle, void** handle)
+{
+    if (cublas_handle == nullptr || handle == nullptr) return KOP_ERR_NULL_POINTER;
+    kop::MlpHandle* mh = new (std::nothrow) kop::MlpHandle();
+    if (mh == nullptr) return KOP_ERR_CUBLAS;
+    mh->cb = static_cast<cublasHandle_t>(cublas_handle);
+    mh->owns_cb = false;
+    *handle = mh;
+    return KOP_OK;
+}
+
 extern "C" kop_status_t kop_mlp_handle_set_residual_in_gemm(void* handle, int enable)
 {
     if (handle == nullptr) return KOP_ERR_NULL_POINTER;
@@ -1001,7 +1013,7 @@ extern "C" kop_status_t kop_mlp_handle_destroy(void* handle)
     if (handle == nullptr) return KOP_ERR_NULL_POINTER;
     kop::MlpHandle* mh = static_cast<kop::MlpHandle*>(handle);
     kop::drop_plan(mh);
-    const cublasStatus_t st = cublasDestroy(mh->cb);
+    const cublasStatus_t st = mh->owns_cb ? cublasDestroy(mh->cb) : CUBLAS_STATUS_SUCCESS;
     delete mh;
     return st == CUBLAS_STATUS_SUCCESS ? KOP_OK : KOP_ERR_CUBLAS;
 }
@@ -1040,6 +1052,13 @@ extern "C" kop_status_t kop_rmsnorm_swiglu_residual(void* handle, const void* h,
     if (cublasSetStream(cb, as_stream(stream)) != CUBLAS_STATUS_SUCCESS) return KOP_ERR_CUBLAS;
     if (cublasSetWorkspace(cb, ws + L.cublas_off, kCublasWorkspace) != CUBLAS_STATUS_SUCCESS)
         return KOP_ERR_CUBLAS;
+
+    // A caller-owned vendor handle goes back with its own default workspace: ours is only valid for this call's
+    // enqueued work (already bound to the GEMM launches above by the time this runs).
+    struct WorkspaceGuard {
+        MlpHandle* mh;
+        ~WorkspaceGuard() { if (!mh->owns_cb) (void)cublasSetWorkspace(mh->cb, nullptr, 0); }
+    } guard{mh};
 
     if ((st = kop_rmsnorm(h, rms_weight, n, rows, hidden, hidden, hidden, eps, dtype, stream)) != KOP_OK) return st;
     if ((st = gemm_nt(cb, n, w_gate_up, gu, rows, 2 * inter, hidden, dtype)) != KOP_OK) return st;

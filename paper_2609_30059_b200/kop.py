@@ -74,7 +74,7 @@ def lib() -> C.CDLL:
     L.kop_rmsnorm_ex.restype = i32
     L.kop_silu_mul.argtypes = [vp, vp, i64, i64, i64, i64, i32, vp]
     L.kop_residual_add.argtypes = [vp, vp, vp, i64, i64, i64, i64, i64, i32, vp]
-    L.kop_ce_loss_rowwise_opts.argtypes = [vp] * 6 + [i64] * 3 + [C.c_int32, f32, vp, sz, i32, vp]
+    L.kop_ce_loss_rowwise_opts.argtypes = [vp] * 7 + [i64] * 3 + [C.c_int32, f32, vp, sz, i32, vp]
     L.kop_ce_loss_rowwise_opts.restype = i32
     L.kop_residual_layernorm.argtypes = [vp] * 7 + [i64] * 5 + [f32, i32, vp]
     L.kop_residual_layernorm.restype = i32
@@ -109,6 +109,8 @@ def lib() -> C.CDLL:
     L.kop_rmsnorm_swiglu_residual_workspace_bytes.argtypes = [i64, i64, i64, i32]
     L.kop_mlp_handle_create.argtypes = [C.POINTER(vp)]
     L.kop_mlp_handle_destroy.argtypes = [vp]
+    L.kop_mlp_handle_wrap.argtypes = [vp, C.POINTER(vp)]
+    L.kop_mlp_handle_wrap.restype = i32
     L.kop_mlp_handle_set_residual_in_gemm.argtypes = [vp, i32]
     L.kop_mlp_handle_set_residual_in_gemm.restype = i32
     for name in ("kop_softmax_scale_bias", "kop_bias_gelu_residual_layernorm", "kop_bn_relu_avgpool",
@@ -142,6 +144,14 @@ def _param(t, name: str, n: int):
         return None
     if t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous() or t.numel() != n:
         raise ValueError(f"{name}: expected a contiguous fp32 CUDA vector of {n} elements")
+    return t.data_ptr()
+
+
+def _out1(t, name: str, dtype, device, n: int = 1):
+    """A caller-owned output vector: contiguous, of `dtype`, on `device`, with at least n elements. Returns its pointer."""
+    if (not isinstance(t, torch.Tensor) or t.dtype != dtype or not t.is_cuda or t.device != device
+            or not t.is_contiguous() or t.numel() < n):
+        raise ValueError(f"{name}: expected a contiguous {dtype} tensor of at least {n} element(s) on {device}")
     return t.data_ptr()
 
 
@@ -254,10 +264,15 @@ def kop_ce_loss_rowwise_static(logits, labels, loss, mean_loss, bad_label_count,
     rows, vocab, zs = _rows2d(logits, "logits")
     if labels.dtype != torch.int32 or not labels.is_cuda or not labels.is_contiguous() or labels.numel() != rows:
         raise ValueError("labels: expected a contiguous int32 CUDA vector of `rows` elements")
+    # The caller owns every output here, so a short or wrongly typed one would be written out of bounds on the
+    # device: refuse it on the host.
+    dev = logits.device
+    if loss is None or not isinstance(loss, torch.Tensor) or loss.numel() != rows:
+        raise ValueError("loss: expected a contiguous float32 CUDA vector of `rows` elements")
     _check(lib().kop_ce_loss_rowwise_static(
-        logits.data_ptr(), labels.data_ptr(), loss.data_ptr(),
-        None if mean_loss is None else mean_loss.data_ptr(),
-        None if bad_label_count is None else bad_label_count.data_ptr(),
+        logits.data_ptr(), labels.data_ptr(), _out1(loss, "loss", torch.float32, dev, rows),
+        None if mean_loss is None else _out1(mean_loss, "mean_loss", torch.float32, dev),
+        None if bad_label_count is None else _out1(bad_label_count, "bad_label_count", torch.int32, dev),
         rows, vocab, zs, _dtype_tag(logits), _stream(stream)), "kop_ce_loss_rowwise_static")
     return loss, mean_loss, bad_label_count
 
@@ -364,8 +379,9 @@ def kop_residual_add(a, b, out=None, stream=None):
 
 
 def kop_ce_loss_rowwise_opts(logits, labels, ignore_index=-100, label_smoothing=0.0, loss=None, mean_loss=None,
-                             bad_label_count=None, counted_rows=None, workspace=None, stream=None):
-    """Returns (loss[rows], mean_loss[1], bad_label_count[1], counted_rows[1]) as device tensors."""
+                             bad_label_count=None, counted_rows=None, workspace=None, stream=None, sum_loss=None):
+    """Returns (loss[rows], mean_loss[1], bad_label_count[1], counted_rows[1]) as device tensors; the "sum"
+    reduction is written to `sum_loss` (fp32 [1]) when the caller passes one."""
     rows, vocab, zs = _rows2d(logits, "logits")
     if labels.dtype != torch.int32 or not labels.is_cuda or not labels.is_contiguous() or labels.numel() != rows:
         raise ValueError("labels: expected a contiguous int32 CUDA vector of `rows` elements")
@@ -378,7 +394,9 @@ def kop_ce_loss_rowwise_opts(logits, labels, ignore_index=-100, label_smoothing=
     if workspace is None:
         workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
     _check(lib().kop_ce_loss_rowwise_opts(logits.data_ptr(), labels.data_ptr(), loss.data_ptr(),
-                                          mean_loss.data_ptr(), bad_label_count.data_ptr(),
+                                          mean_loss.data_ptr(),
+                                          None if sum_loss is None else _out1(sum_loss, "sum_loss", torch.float32, dev),
+                                          bad_label_count.data_ptr(),
                                           counted_rows.data_ptr(), rows, vocab, zs, int(ignore_index),
                                           float(label_smoothing), workspace.data_ptr(),
                                           workspace.numel() * workspace.element_size(), _dtype_tag(logits),

@@ -31,7 +31,7 @@ def assert_close(got: torch.Tensor, ref: np.ndarray, tol: float, what: str):
         i = np.unravel_index(np.argmax(np.where(bad, err, 0)), err.shape)
         raise AssertionError(f"{what}: {bad.sum()} of {bad.size} outside tol={tol:g}; worst at {i}: "
                              f"got {g[i]!r} ref {ref[i]!r} err {err[i]:.3e}")
-    return float(np.nanmax(err)) if err.size else 0.0
+    return float(np.nanmax(err)) if err.size and not np.isnan(err).all() else 0.0
 
 
 def assert_bf16_tight(got: torch.Tensor, ref: np.ndarray, what: str, rel=2.0 ** -7, floor=4e-3):

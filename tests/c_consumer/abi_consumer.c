@@ -3,8 +3,12 @@
  *   softmax of a constant row is uniform and every row sums to 1;
  *   cross-entropy of constant logits is ln(V) for every row, and so is the mean;
  *   the running sum of ones is 1, 2, ..., n (exact in fp32), the reverse exclusive one n-1, ..., 0;
- *   GroupNorm output has zero mean and unit variance per group.
+ *   GroupNorm output has zero mean and unit variance per group;
+ *   the MLP segment (vendor GEMMs kept) on constant rows and constant weights collapses to
+ *   out = c + 2 s silu(s), s = c / sqrt(c^2 + eps), with a handle the library creates and with a cuBLAS handle
+ *   this program owns.
  * Exit code 0 and "abi consumer ok" on success. */
+#include <cublas_v2.h>
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stdint.h>
@@ -138,6 +142,58 @@ int main(void)
         EXPECT(timeouts == 0, "no bulk-copy wait ran out");
         cudaFree(dmu);
         cudaFree(drs);
+    }
+
+    /* MLP segment: rows of constant c_i, RMSNorm weight 1, gate rows of W1 = 1/H, up rows = 2/H, W2 = 1/I */
+    {
+        const int64_t M = 6, H = 16, I = 24;
+        const float eps = 1e-6f;
+        float *dh, *dw, *dW1, *dW2, *dout;
+        void* mws;
+        const size_t need = kop_rmsnorm_swiglu_residual_workspace_bytes(M, H, I, KOP_F32);
+        EXPECT(need > 0, "MLP workspace size");
+        CHECK_CUDA(cudaMalloc((void**)&dh, M * H * sizeof(float)));
+        CHECK_CUDA(cudaMalloc((void**)&dout, M * H * sizeof(float)));
+        CHECK_CUDA(cudaMalloc((void**)&dw, H * sizeof(float)));
+        CHECK_CUDA(cudaMalloc((void**)&dW1, 2 * I * H * sizeof(float)));
+        CHECK_CUDA(cudaMalloc((void**)&dW2, H * I * sizeof(float)));
+        CHECK_CUDA(cudaMalloc(&mws, need));
+        for (int64_t i = 0; i < M; ++i)
+            for (int64_t j = 0; j < H; ++j) h[i * H + j] = (float)(i - 2) * 0.75f + 0.25f;
+        CHECK_CUDA(cudaMemcpy(dh, h, M * H * sizeof(float), cudaMemcpyHostToDevice));
+        for (int64_t j = 0; j < H; ++j) out[j] = 1.0f;
+        CHECK_CUDA(cudaMemcpy(dw, out, H * sizeof(float), cudaMemcpyHostToDevice));
+        for (int64_t r = 0; r < 2 * I; ++r)
+            for (int64_t j = 0; j < H; ++j) out[r * H + j] = (r < I ? 1.0f : 2.0f) / (float)H;
+        CHECK_CUDA(cudaMemcpy(dW1, out, 2 * I * H * sizeof(float), cudaMemcpyHostToDevice));
+        for (int64_t k = 0; k < H * I; ++k) out[k] = 1.0f / (float)I;
+        CHECK_CUDA(cudaMemcpy(dW2, out, H * I * sizeof(float), cudaMemcpyHostToDevice));
+        cublasHandle_t mine;
+        EXPECT(cublasCreate(&mine) == CUBLAS_STATUS_SUCCESS, "cublasCreate");
+        for (int pass = 0; pass < 2; ++pass) {
+            void* mh = NULL;
+            if (pass == 0) CHECK_KOP(kop_mlp_handle_create(&mh));
+            else CHECK_KOP(kop_mlp_handle_wrap((void*)mine, &mh));      /* the caller-owned vendor handle */
+            CHECK_CUDA(cudaMemsetAsync(dout, 0, M * H * sizeof(float), stream));
+            CHECK_KOP(kop_rmsnorm_swiglu_residual(mh, dh, dw, dW1, dW2, dout, M, H, I, eps, mws, need, KOP_F32,
+                                                  (kop_stream_t)stream));
+            CHECK_CUDA(cudaMemcpyAsync(out, dout, M * H * sizeof(float), cudaMemcpyDeviceToHost, stream));
+            CHECK_CUDA(cudaStreamSynchronize(stream));
+            for (int64_t i = 0; i < M; ++i) {
+                const double c = (double)h[i * H];
+                const double sgn = c / sqrt(c * c + (double)eps);
+                const double want = c + 2.0 * sgn * (sgn / (1.0 + exp(-sgn)));
+                for (int64_t j = 0; j < H; ++j)
+                    EXPECT(fabs((double)out[i * H + j] - want) <= 1e-5 * fmax(1.0, fabs(want)), "MLP segment closed form");
+            }
+            CHECK_KOP(kop_mlp_handle_destroy(mh));
+        }
+        /* the wrapper's destruction left this program's handle alive */
+        int ver = 0;
+        EXPECT(cublasGetVersion(mine, &ver) == CUBLAS_STATUS_SUCCESS && ver > 0, "caller's cuBLAS handle still valid");
+        EXPECT(cublasDestroy(mine) == CUBLAS_STATUS_SUCCESS, "cublasDestroy");
+        EXPECT(kop_mlp_handle_wrap(NULL, NULL) == KOP_ERR_NULL_POINTER, "NULL handle is rejected");
+        cudaFree(dh); cudaFree(dout); cudaFree(dw); cudaFree(dW1); cudaFree(dW2); cudaFree(mws);
     }
 
     /* validation happens before any launch */

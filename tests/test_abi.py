@@ -420,3 +420,26 @@ def test_product_package_never_imports_the_oracle():
                 assert "kopref" not in text, fn
                 assert not re.search(r"^\s*(from|import)\s+\.*oracle\b", text, flags=re.M), fn
                 assert not re.search(r'#include\s+"[^"]*oracle', text), fn
+
+
+def test_ncu_traffic_table_agrees_with_the_committed_summaries():
+    """bench.py reports measured DRAM traffic from profiles/ncu_dram_traffic.json; every entry must be the
+    figures printed in the ncu summary it names."""
+    import json
+    import re
+    prof = os.path.join(ROOT, "profiles")
+    table = json.load(open(os.path.join(prof, "ncu_dram_traffic.json")))
+    assert {"ce_loss", "layernorm", "softmax_large", "bn_pool", "rmsnorm", "silu_mul", "residual_add"} <= set(table)
+    unit = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}
+    for seg, e in table.items():
+        text = open(os.path.join(prof, e["summary"])).read()
+        assert e["kernel"] in text.splitlines()[0], seg
+        for key, field in (("dram__bytes_read.sum", "dram_read_bytes"), ("dram__bytes_write.sum", "dram_write_bytes")):
+            m = re.search(r"`" + re.escape(key) + r"`\) \| ([\d.,]+) (\w+)", text)
+            assert m, (seg, key)
+            assert abs(float(m.group(1).replace(",", "")) * unit[m.group(2)] - e[field]) <= 1.0, (seg, key)
+        assert e["rows_div"] >= 1
+    from paper_2609_30059_b200 import ncu_summary
+    e = table["ce_loss"]
+    assert ncu_summary.traffic_per_full_launch("ce_loss") == (e["dram_read_bytes"] + e["dram_write_bytes"]) * e["rows_div"]
+    assert ncu_summary.traffic_per_full_launch("no such segment") is None

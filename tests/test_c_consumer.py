@@ -24,7 +24,7 @@ def build_consumer():
     cuda = cuda_home()
     cmd = ["gcc", "-std=c11", "-O1", "-Wall", "-Werror", SRC, "-o", EXE, "-I" + os.path.join(ROOT, "include"),
            "-I" + os.path.join(cuda, "include"), "-L" + libdir, "-lkop", "-L" + os.path.join(cuda, "lib64"),
-           "-lcudart", "-lm", "-Wl,-rpath," + libdir, "-Wl,-rpath," + os.path.join(cuda, "lib64")]
+           "-lcudart", "-lcublas", "-lm", "-Wl,-rpath," + libdir, "-Wl,-rpath," + os.path.join(cuda, "lib64")]
     res = subprocess.run(cmd, capture_output=True, text=True)
     assert res.returncode == 0, res.stderr
     return EXE

@@ -748,14 +748,20 @@ def test_ce_opts_parity(kop, rows, vocab, dtype, smoothing, seed):
     mean = Guarded((1,), F32)
     bad = Guarded((1,), torch.int32)
     cnt = Guarded((1,), torch.int32)
+    total = Guarded((1,), F32)
     kop.kop_ce_loss_rowwise_opts(z, lab, -100, smoothing, loss=loss.t, mean_loss=mean.t, bad_label_count=bad.t,
-                                 counted_rows=cnt.t)
+                                 counted_rows=cnt.t, sum_loss=total.t)
     rl, rmean, rbad, rcnt = kopref.ce_loss_opts(host(z), host(lab), -100, smoothing, threads=None)
     assert_close(loss.t, rl, 2e-5, "ce opts loss")
     assert_close(mean.t, np.array([rmean]), 2e-5, "ce opts mean")
+    # reduction "sum" against its own oracle function, to the same relative accuracy
+    rsum = kopref.ce_loss_sum(host(z), host(lab), -100, smoothing, threads=None)
+    assert_close(total.t, np.array([rsum]), 2e-5, "ce opts sum")
+    # sum and mean come from one fixed-order total: mean is exactly that total divided by the count
+    assert float(mean.t.item()) == float((total.t / cnt.t.float()).item())
     assert int(bad.t.item()) == rbad == 0 and int(cnt.t.item()) == rcnt
     assert bool((loss.t[::5] == 0).all())
-    for gd in (loss, mean, bad, cnt):
+    for gd in (loss, mean, bad, cnt, total):
         gd.check("ce opts")
 
 
@@ -778,3 +784,50 @@ def test_ce_opts_edge_cases(kop):
     with pytest.raises(kop.KopError) as ei:
         kop.kop_ce_loss_rowwise_opts(z, lab, -100, 1.0)
     assert ei.value.status == 2
+    # reduction "sum": nothing counted sums to 0 (the mean is NaN), a bad label makes it NaN, and it is
+    # bit-identical run to run
+    tot = torch.full((1,), -7.0, dtype=F32, device="cuda")
+    kop.kop_ce_loss_rowwise_opts(z, allig, 7, 0.2, sum_loss=tot)
+    assert float(tot.item()) == 0.0
+    kop.kop_ce_loss_rowwise_opts(z, lab2, -100, 0.0, sum_loss=tot)
+    assert bool(torch.isnan(tot[0]))
+    t1, t2 = torch.empty_like(tot), torch.empty_like(tot)
+    zz, ll = synth.ce_inputs(3000, 1000, BF16, 4, "cuda")
+    kop.kop_ce_loss_rowwise_opts(zz, ll, -100, 0.1, sum_loss=t1)
+    kop.kop_ce_loss_rowwise_opts(zz, ll, -100, 0.1, sum_loss=t2)
+    assert torch.equal(t1, t2)
+    assert_close(t1, np.array([kopref.ce_loss_sum(host(zz), host(ll), -100, 0.1, threads=None)]), 2e-5, "ce sum 3000 rows")
+
+
+@pytest.mark.parametrize("vocab,dtype", [(32000, BF16),     # CTA per row, batches of four vectors
+                                         (4096, BF16),      # 32 lanes per row
+                                         (1024, F32),       # lanes-per-row kernel, 8-vector rows
+                                         (64, BF16),        # four lanes per row
+                                         (1001, F32),       # odd length: scalar kernel
+                                         (40000, F32)])
+def test_ce_non_finite_logits(kop, vocab, dtype):
+    """NaN and +inf logits make exactly their own row NaN, whichever kernel the shape selects and wherever in the
+    row they sit (one element, a whole thread's batch, the whole row); -inf logits are ordinary. The oracle's
+    max-shifted definition says the same (pinned against torch float64 on the CPU)."""
+    rows = 12
+    z, lab = synth.ce_inputs(rows, vocab, dtype, 8, "cuda")
+    z = z.clone()
+    z[1, vocab // 3] = float("nan")                     # one NaN
+    z[2, : min(vocab, 64)] = float("nan")               # a run of NaNs: whole vectors / a thread's whole batch
+    z[3, :] = float("nan")                              # nothing but NaNs
+    z[4, vocab - 1] = float("inf")                      # +inf in the last column
+    z[5, 0] = float("inf")
+    z[5, vocab // 2] = float("inf")                     # two +inf
+    z[6, 1::2] = float("-inf")                          # half the row masked: still a number
+    z[7, :] = float("-inf")                             # empty row: NaN
+    z[8, 0] = float("nan")
+    z[8, 1:] = float("-inf")                            # a NaN among nothing
+    lab = lab.clone()
+    lab[6] = 0
+    loss, mean, bad = kop.kop_ce_loss_rowwise(z, lab)
+    rl, rmean, rbad = kopref.ce_loss_rowwise(host(z), host(lab))
+    want_nan = np.array([False, True, True, True, True, True, False, True, True, False, False, False])
+    assert np.array_equal(np.isnan(rl), want_nan)
+    assert np.array_equal(torch.isnan(loss).cpu().numpy(), want_nan), loss
+    assert_close(loss, rl, 2e-5, "ce with non-finite logits")
+    assert bool(torch.isnan(mean[0])) and np.isnan(rmean) and int(bad.item()) == 0
