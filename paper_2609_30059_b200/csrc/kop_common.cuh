@@ -244,6 +244,7 @@ struct Elem<float> {
         v.w[3] = __float_as_uint(f[1].y);
         return v;
     }
+    static constexpr bool kMixedAdd = false;
     __device__ __forceinline__ static float load1(const float* p) { return *p; }
     __device__ __forceinline__ static void store1(float* p, float f) { *p = f; }
     __device__ __forceinline__ static Vec16 fill_neg_inf()
@@ -294,6 +295,17 @@ struct Elem<__nv_bfloat16> {
         }
         return v;
     }
+    // widen(w) + c for both halves of a packed word with the mixed-precision add of this target (the 16-bit
+    // operand is widened exactly inside the instruction, one rounding: bit-identical to unpacking first). It
+    // replaces the two mask / shift instructions plus a packed add by two adds.
+    static constexpr bool kMixedAdd = true;
+    __device__ __forceinline__ static float2 add_widen2(uint32_t w, float2 c)
+    {
+        float2 r;
+        asm("{ .reg .b16 lo, hi; mov.b32 {lo, hi}, %2; add.rn.f32.bf16 %0, lo, %3; add.rn.f32.bf16 %1, hi, %4; }"
+            : "=f"(r.x), "=f"(r.y) : "r"(w), "f"(c.x), "f"(c.y));
+        return r;
+    }
     __device__ __forceinline__ static float load1(const __nv_bfloat16* p) { return __bfloat162float(*p); }
     __device__ __forceinline__ static void store1(__nv_bfloat16* p, float f) { *p = __float2bfloat16_rn(f); }
     __device__ __forceinline__ static Vec16 fill_neg_inf()
@@ -342,6 +354,14 @@ struct Elem<__half> {
             v.w[i] = *reinterpret_cast<uint32_t*>(&h);
         }
         return v;
+    }
+    static constexpr bool kMixedAdd = true;
+    __device__ __forceinline__ static float2 add_widen2(uint32_t w, float2 c)
+    {
+        float2 r;
+        asm("{ .reg .b16 lo, hi; mov.b32 {lo, hi}, %2; add.rn.f32.f16 %0, lo, %3; add.rn.f32.f16 %1, hi, %4; }"
+            : "=f"(r.x), "=f"(r.y) : "r"(w), "f"(c.x), "f"(c.y));
+        return r;
     }
     __device__ __forceinline__ static float load1(const __half* p) { return __half2float(*p); }
     __device__ __forceinline__ static void store1(__half* p, float f) { *p = __float2half_rn(f); }
