@@ -17,8 +17,8 @@
  *   dtype      `dtype` is the element type of the data tensors (inputs and the main
  *              output): KOP_F32, KOP_BF16 or KOP_F16 (IEEE binary16; results beyond
  *              65504 in magnitude are stored as infinity). Parameter vectors (bias, gamma, beta,
- *              scale, shift, weight) are fp32 (kop_layernorm_ex / kop_rmsnorm_ex also take
- *              them in the data type); statistics outputs (mean, rstd, pooled, loss) are
+ *              scale, shift, weight) are fp32; the *_ex entry points also take them in the
+ *              data type; statistics outputs (mean, rstd, pooled, loss) are
  *              always fp32. All arithmetic is fp32; the only rounding to
  *              bf16 / fp16 is the final store (round to nearest even), as the paper's
  *              numerics rule requires (accumulate in fp32, cast only at the store).
@@ -448,6 +448,37 @@ kop_status_t kop_reduce_rows(const void* x, float* out, int32_t* index, int64_t 
 kop_status_t kop_cumsum_rows(const void* x, const unsigned char* mask, void* y, int64_t rows, int64_t cols,
                              int64_t x_row_stride, int64_t mask_row_stride, int64_t y_row_stride,
                              int exclusive, int reverse, kop_dtype_t dtype, kop_stream_t stream);
+
+/*
+ * The entry points above with their parameter vectors in fp32 OR in the data type (a model held in bf16 / fp16
+ * keeps its biases, folded BatchNorm coefficients and norm weights in that type; the coverage variant "16-bit
+ * parameters" of the same segments). param_dtype is KOP_F32 or equal to `dtype`, anything else returns
+ * KOP_ERR_UNSUPPORTED_DTYPE; all parameter vectors of one call share it. A 16-bit parameter is widened exactly to
+ * fp32 and the arithmetic, the results for fp32 parameters and every other rule are those of the base entry point:
+ *   kop_softmax_ex           kop_softmax_scale_bias (log_output == 0 and causal_period == 0) / kop_softmax_opts
+ *   kop_bn_relu_avgpool_ex   kop_bn_relu_avgpool      (scale, shift)
+ *   kop_groupnorm_act_ex     kop_groupnorm_act        (gamma, beta; each may be NULL)
+ *   kop_bias_act_ex          kop_bias_act             (bias; may be NULL)
+ *   kop_epilogue_chain_ex    kop_epilogue_chain       (bias; may be NULL)
+ * Parameter pointers must be aligned to their element size; 16-byte alignment takes the vector kernels.
+ */
+kop_status_t kop_softmax_ex(const void* x, const void* bias, void* y, int64_t rows, int64_t cols,
+                            int64_t x_row_stride, int64_t y_row_stride, float scale, int log_output,
+                            int64_t causal_period, kop_dtype_t dtype, kop_dtype_t param_dtype, kop_stream_t stream);
+kop_status_t kop_bn_relu_avgpool_ex(const void* x, const void* scale, const void* shift, void* y, float* pooled,
+                                    int64_t N, int64_t C, int64_t H, int64_t W, const int64_t x_strides[4],
+                                    const int64_t y_strides[4], kop_dtype_t dtype, kop_dtype_t param_dtype,
+                                    kop_stream_t stream);
+kop_status_t kop_groupnorm_act_ex(const void* x, const void* gamma, const void* beta, void* y, float* mean,
+                                  float* rstd, int64_t N, int64_t C, int64_t H, int64_t W, int64_t groups, float eps,
+                                  int act, kop_dtype_t dtype, kop_dtype_t param_dtype, kop_stream_t stream);
+kop_status_t kop_bias_act_ex(const void* x, const void* bias, void* y, int64_t rows, int64_t cols,
+                             int64_t x_row_stride, int64_t y_row_stride, int act, float alpha, kop_dtype_t dtype,
+                             kop_dtype_t param_dtype, kop_stream_t stream);
+kop_status_t kop_epilogue_chain_ex(const void* x, const void* bias, const void* residual, void* y, int64_t rows,
+                                   int64_t cols, int64_t x_row_stride, int64_t res_row_stride, int64_t y_row_stride,
+                                   float scale, float residual_scale, float clamp_lo, float clamp_hi, int act,
+                                   float alpha, kop_dtype_t dtype, kop_dtype_t param_dtype, kop_stream_t stream);
 
 /*
  * Lp normalisation of rows (fusion agent: "normalization fusion", a reduction and the pointwise pass that uses it

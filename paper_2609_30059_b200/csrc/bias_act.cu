@@ -48,9 +48,9 @@ __device__ __forceinline__ float act_dev(float u, float alpha)
 
 // kFlat: rows shorter than a tile; the CTA takes U * blockDim.x vectors in row-major order across rows
 // (nvec_total = rows * nvec). Otherwise a CTA is one tile of one row.
-template <typename T, int ACT, bool kFlat>
+template <typename T, typename PT, int ACT, bool kFlat>
 __global__ void __launch_bounds__(256)
-bias_act_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* __restrict__ y, int nvec,
+bias_act_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __restrict__ y, int nvec,
                 int tiles_per_row, int64_t nvec_total, int64_t x_stride, int64_t y_stride, float alpha)
 {
     constexpr int E = Elem<T>::kPerVec, U = 4;
@@ -88,7 +88,7 @@ bias_act_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* __re
             if (bias != nullptr) {
 #pragma unroll
                 for (int q = 0; q < E / 4; ++q) {
-                    const float4 b = ldg_f4(bias + (int64_t)v[k] * E + 4 * q);
+                    const float4 b = ldg_p4(bias + (int64_t)v[k] * E + 4 * q);
                     f[4 * q] += b.x;
                     f[4 * q + 1] += b.y;
                     f[4 * q + 2] += b.z;
@@ -102,16 +102,16 @@ bias_act_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* __re
     }
 }
 
-template <typename T, int ACT>
+template <typename T, typename PT, int ACT>
 __global__ void __launch_bounds__(256)
-bias_act_scalar_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* __restrict__ y, int64_t rows,
+bias_act_scalar_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __restrict__ y, int64_t rows,
                        int64_t cols, int64_t x_stride, int64_t y_stride, float alpha)
 {
     constexpr bool kFast = sizeof(T) == 2;
     const int64_t total = rows * cols;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
         const int64_t r = i / cols, j = i - r * cols;
-        const float u = Elem<T>::load1(x + r * x_stride + j) + (bias != nullptr ? __ldg(bias + j) : 0.0f);
+        const float u = Elem<T>::load1(x + r * x_stride + j) + (bias != nullptr ? param1(bias, j) : 0.0f);
         Elem<T>::store1(y + r * y_stride + j, act_dev<ACT, kFast>(u, alpha));
     }
 }
@@ -130,9 +130,9 @@ __device__ __forceinline__ float chain_value(float x, float b, float r, const Ch
     return u;
 }
 
-template <typename T, int ACT, bool kFlat>
+template <typename T, typename PT, int ACT, bool kFlat>
 __global__ void __launch_bounds__(256)
-chain_kernel(const T* __restrict__ x, const float* __restrict__ bias, const T* __restrict__ res, T* __restrict__ y,
+chain_kernel(const T* __restrict__ x, const PT* __restrict__ bias, const T* __restrict__ res, T* __restrict__ y,
              int nvec, int tiles_per_row, int64_t nvec_total, int64_t x_stride, int64_t r_stride, int64_t y_stride,
              ChainArgs a)
 {
@@ -176,7 +176,7 @@ chain_kernel(const T* __restrict__ x, const float* __restrict__ bias, const T* _
 #pragma unroll
             for (int q = 0; q < E / 4; ++q) {
                 float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (bias != nullptr) t = ldg_f4(bias + (int64_t)v[k] * E + 4 * q);
+                if (bias != nullptr) t = ldg_p4(bias + (int64_t)v[k] * E + 4 * q);
                 b[4 * q] = t.x;
                 b[4 * q + 1] = t.y;
                 b[4 * q + 2] = t.z;
@@ -190,9 +190,9 @@ chain_kernel(const T* __restrict__ x, const float* __restrict__ bias, const T* _
     }
 }
 
-template <typename T, int ACT>
+template <typename T, typename PT, int ACT>
 __global__ void __launch_bounds__(256)
-chain_scalar_kernel(const T* __restrict__ x, const float* __restrict__ bias, const T* __restrict__ res,
+chain_scalar_kernel(const T* __restrict__ x, const PT* __restrict__ bias, const T* __restrict__ res,
                     T* __restrict__ y, int64_t rows, int64_t cols, int64_t x_stride, int64_t r_stride,
                     int64_t y_stride, ChainArgs a)
 {
@@ -200,14 +200,14 @@ chain_scalar_kernel(const T* __restrict__ x, const float* __restrict__ bias, con
     const int64_t total = rows * cols;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
         const int64_t r = i / cols, j = i - r * cols;
-        const float u = chain_value(Elem<T>::load1(x + r * x_stride + j), bias != nullptr ? __ldg(bias + j) : 0.0f,
+        const float u = chain_value(Elem<T>::load1(x + r * x_stride + j), bias != nullptr ? param1(bias, j) : 0.0f,
                                     res != nullptr ? Elem<T>::load1(res + r * r_stride + j) : 0.0f, a);
         Elem<T>::store1(y + r * y_stride + j, act_dev<ACT, kFast>(u, a.alpha));
     }
 }
 
-template <typename T, int ACT>
-kop_status_t launch_chain_a(const T* x, const float* bias, const T* res, T* y, int64_t rows, int64_t cols, int64_t xs,
+template <typename T, typename PT, int ACT>
+kop_status_t launch_chain_a(const T* x, const PT* bias, const T* res, T* y, int64_t rows, int64_t cols, int64_t xs,
                             int64_t rs, int64_t ys, const ChainArgs& a, cudaStream_t stream)
 {
     constexpr int E = Elem<T>::kPerVec;
@@ -223,30 +223,31 @@ kop_status_t launch_chain_a(const T* x, const float* bias, const T* res, T* y, i
         if (nvec < 64 || ((int64_t)tiles * 2 * threads - nvec) * 4 > nvec) {
             const int64_t total = rows * nvec, grid = (total + 511) / 512;
             if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
-            chain_kernel<T, ACT, true><<<(unsigned)grid, 256, 0, stream>>>(x, bias, res, y, nvec, 1, total, xs, rs, ys, a);
+            chain_kernel<T, PT, ACT, true><<<(unsigned)grid, 256, 0, stream>>>(x, bias, res, y, nvec, 1, total, xs, rs, ys, a);
             return launch_status();
         }
         const int64_t grid = rows * tiles;
         if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
-        chain_kernel<T, ACT, false><<<(unsigned)grid, threads, 0, stream>>>(x, bias, res, y, nvec, tiles, 0, xs, rs, ys, a);
+        chain_kernel<T, PT, ACT, false><<<(unsigned)grid, threads, 0, stream>>>(x, bias, res, y, nvec, tiles, 0, xs, rs, ys, a);
         return launch_status();
     }
     int64_t blocks = (rows * cols + 255) / 256;
     const int64_t cap = 32LL * sm_count();
     if (blocks > cap) blocks = cap;
-    chain_scalar_kernel<T, ACT><<<(unsigned)blocks, 256, 0, stream>>>(x, bias, res, y, rows, cols, xs, rs, ys, a);
+    chain_scalar_kernel<T, PT, ACT><<<(unsigned)blocks, 256, 0, stream>>>(x, bias, res, y, rows, cols, xs, rs, ys, a);
     return launch_status();
 }
 
-template <typename T>
-kop_status_t launch_chain(const void* xv, const float* bias, const void* rv, void* yv, int64_t rows, int64_t cols,
+template <typename T, typename PT>
+kop_status_t launch_chain(const void* xv, const void* biasv, const void* rv, void* yv, int64_t rows, int64_t cols,
                           int64_t xs, int64_t rs, int64_t ys, int act, const ChainArgs& a, cudaStream_t stream)
 {
     const T* x = static_cast<const T*>(xv);
+    const PT* bias = static_cast<const PT*>(biasv);
     const T* r = static_cast<const T*>(rv);
     T* y = static_cast<T*>(yv);
 #define KOP_CHAIN_CASE(A) \
-    case A: return launch_chain_a<T, A>(x, bias, r, y, rows, cols, xs, rs, ys, a, stream)
+    case A: return launch_chain_a<T, PT, A>(x, bias, r, y, rows, cols, xs, rs, ys, a, stream)
     switch (act) {
         KOP_CHAIN_CASE(kActRelu);
         KOP_CHAIN_CASE(kActLeakyRelu);
@@ -258,13 +259,13 @@ kop_status_t launch_chain(const void* xv, const float* bias, const void* rv, voi
         KOP_CHAIN_CASE(kActMish);
         KOP_CHAIN_CASE(kActHardswish);
         KOP_CHAIN_CASE(kActElu);
-    default: return launch_chain_a<T, kActIdentity>(x, bias, r, y, rows, cols, xs, rs, ys, a, stream);
+    default: return launch_chain_a<T, PT, kActIdentity>(x, bias, r, y, rows, cols, xs, rs, ys, a, stream);
     }
 #undef KOP_CHAIN_CASE
 }
 
-template <typename T, int ACT>
-kop_status_t launch_bias_act_a(const T* x, const float* bias, T* y, int64_t rows, int64_t cols, int64_t xs,
+template <typename T, typename PT, int ACT>
+kop_status_t launch_bias_act_a(const T* x, const PT* bias, T* y, int64_t rows, int64_t cols, int64_t xs,
                                int64_t ys, float alpha, cudaStream_t stream)
 {
     constexpr int E = Elem<T>::kPerVec;
@@ -286,29 +287,30 @@ kop_status_t launch_bias_act_a(const T* x, const float* bias, T* y, int64_t rows
         if (nvec < 128 || ((int64_t)tiles * 4 * threads - nvec) * 4 > nvec) {
             const int64_t total = rows * nvec, grid = (total + 1023) / 1024;
             if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
-            bias_act_kernel<T, ACT, true><<<(unsigned)grid, 256, 0, stream>>>(x, bias, y, nvec, 1, total, xs, ys, alpha);
+            bias_act_kernel<T, PT, ACT, true><<<(unsigned)grid, 256, 0, stream>>>(x, bias, y, nvec, 1, total, xs, ys, alpha);
             return launch_status();
         }
         const int64_t grid = rows * tiles;
         if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
-        bias_act_kernel<T, ACT, false><<<(unsigned)grid, threads, 0, stream>>>(x, bias, y, nvec, tiles, 0, xs, ys, alpha);
+        bias_act_kernel<T, PT, ACT, false><<<(unsigned)grid, threads, 0, stream>>>(x, bias, y, nvec, tiles, 0, xs, ys, alpha);
         return launch_status();
     }
     int64_t blocks = (rows * cols + 255) / 256;
     const int64_t cap = 32LL * sm_count();
     if (blocks > cap) blocks = cap;
-    bias_act_scalar_kernel<T, ACT><<<(unsigned)blocks, 256, 0, stream>>>(x, bias, y, rows, cols, xs, ys, alpha);
+    bias_act_scalar_kernel<T, PT, ACT><<<(unsigned)blocks, 256, 0, stream>>>(x, bias, y, rows, cols, xs, ys, alpha);
     return launch_status();
 }
 
-template <typename T>
-kop_status_t launch_bias_act(const void* xv, const float* bias, void* yv, int64_t rows, int64_t cols, int64_t xs,
+template <typename T, typename PT>
+kop_status_t launch_bias_act(const void* xv, const void* biasv, void* yv, int64_t rows, int64_t cols, int64_t xs,
                              int64_t ys, int act, float alpha, cudaStream_t stream)
 {
     const T* x = static_cast<const T*>(xv);
+    const PT* bias = static_cast<const PT*>(biasv);
     T* y = static_cast<T*>(yv);
 #define KOP_ACT_CASE(A) \
-    case A: return launch_bias_act_a<T, A>(x, bias, y, rows, cols, xs, ys, alpha, stream)
+    case A: return launch_bias_act_a<T, PT, A>(x, bias, y, rows, cols, xs, ys, alpha, stream)
     switch (act) {
         KOP_ACT_CASE(kActRelu);
         KOP_ACT_CASE(kActLeakyRelu);
@@ -320,7 +322,7 @@ kop_status_t launch_bias_act(const void* xv, const float* bias, void* yv, int64_
         KOP_ACT_CASE(kActMish);
         KOP_ACT_CASE(kActHardswish);
         KOP_ACT_CASE(kActElu);
-    default: return launch_bias_act_a<T, kActIdentity>(x, bias, y, rows, cols, xs, ys, alpha, stream);
+    default: return launch_bias_act_a<T, PT, kActIdentity>(x, bias, y, rows, cols, xs, ys, alpha, stream);
     }
 #undef KOP_ACT_CASE
 }
@@ -328,12 +330,14 @@ kop_status_t launch_bias_act(const void* xv, const float* bias, void* yv, int64_
 }  // namespace
 }  // namespace kop
 
-extern "C" kop_status_t kop_bias_act(const void* x, const float* bias, void* y, int64_t rows, int64_t cols,
-                                     int64_t x_row_stride, int64_t y_row_stride, int act, float alpha,
-                                     kop_dtype_t dtype, kop_stream_t stream)
+namespace kop {
+namespace {
+
+kop_status_t bias_act_entry(const void* x, const void* bias, void* y, int64_t rows, int64_t cols, int64_t x_row_stride,
+                            int64_t y_row_stride, int act, float alpha, kop_dtype_t dtype, kop_dtype_t pdtype,
+                            kop_stream_t stream)
 {
-    using namespace kop;
-    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    if (!param_dtype_ok(dtype, pdtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
     kop_status_t st = check_rows_cols(rows, cols);
     if (st != KOP_OK) return st;
     if (act < 0 || act >= kActCount) return KOP_ERR_BAD_SHAPE;
@@ -342,24 +346,21 @@ extern "C" kop_status_t kop_bias_act(const void* x, const float* bias, void* y, 
     if (rows == 0) return KOP_OK;
     if (!x || !y) return KOP_ERR_NULL_POINTER;
     const int esz = elem_size(dtype);
-    if (!aligned_to(x, esz) || !aligned_to(y, esz) || (bias && !aligned_to(bias, 4))) return KOP_ERR_MISALIGNED;
+    if (!aligned_to(x, esz) || !aligned_to(y, esz) || (bias && !aligned_to(bias, elem_size(pdtype)))) return KOP_ERR_MISALIGNED;
     if (!alias_ok(x, x_row_stride, y, y_row_stride, rows, cols, esz, true)) return KOP_ERR_BAD_ALIAS;
     if ((st = check_device()) != KOP_OK) return st;
     cudaStream_t s = as_stream(stream);
-    return dtype == KOP_F32 ? launch_bias_act<float>(x, bias, y, rows, cols, x_row_stride, y_row_stride, act, alpha, s)
-           : dtype == KOP_BF16
-               ? launch_bias_act<__nv_bfloat16>(x, bias, y, rows, cols, x_row_stride, y_row_stride, act, alpha, s)
-               : launch_bias_act<__half>(x, bias, y, rows, cols, x_row_stride, y_row_stride, act, alpha, s);
+#define KOP_BA_GO(T, PT) launch_bias_act<T, PT>(x, bias, y, rows, cols, x_row_stride, y_row_stride, act, alpha, s)
+    return KOP_DISPATCH_TYPES(dtype, pdtype, KOP_BA_GO);
+#undef KOP_BA_GO
 }
 
-extern "C" kop_status_t kop_epilogue_chain(const void* x, const float* bias, const void* residual, void* y,
-                                           int64_t rows, int64_t cols, int64_t x_row_stride, int64_t res_row_stride,
-                                           int64_t y_row_stride, float scale, float residual_scale, float clamp_lo,
-                                           float clamp_hi, int act, float alpha, kop_dtype_t dtype,
-                                           kop_stream_t stream)
+kop_status_t chain_entry(const void* x, const void* bias, const void* residual, void* y, int64_t rows, int64_t cols,
+                         int64_t x_row_stride, int64_t res_row_stride, int64_t y_row_stride, float scale,
+                         float residual_scale, float clamp_lo, float clamp_hi, int act, float alpha, kop_dtype_t dtype,
+                         kop_dtype_t pdtype, kop_stream_t stream)
 {
-    using namespace kop;
-    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    if (!param_dtype_ok(dtype, pdtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
     kop_status_t st = check_rows_cols(rows, cols);
     if (st != KOP_OK) return st;
     if (act < 0 || act >= kActCount || !(clamp_lo <= clamp_hi)) return KOP_ERR_BAD_SHAPE;
@@ -370,7 +371,7 @@ extern "C" kop_status_t kop_epilogue_chain(const void* x, const float* bias, con
     if (!x || !y) return KOP_ERR_NULL_POINTER;
     const int esz = elem_size(dtype);
     if (!aligned_to(x, esz) || !aligned_to(y, esz) || (residual && !aligned_to(residual, esz)) ||
-        (bias && !aligned_to(bias, 4)))
+        (bias && !aligned_to(bias, elem_size(pdtype))))
         return KOP_ERR_MISALIGNED;
     if (!alias_ok(x, x_row_stride, y, y_row_stride, rows, cols, esz, true) ||
         (residual && !alias_ok(residual, res_row_stride, y, y_row_stride, rows, cols, esz, true)))
@@ -378,10 +379,44 @@ extern "C" kop_status_t kop_epilogue_chain(const void* x, const float* bias, con
     if ((st = check_device()) != KOP_OK) return st;
     cudaStream_t s = as_stream(stream);
     const ChainArgs a{scale, residual_scale, clamp_lo, clamp_hi, alpha};
-    return dtype == KOP_F32 ? launch_chain<float>(x, bias, residual, y, rows, cols, x_row_stride, res_row_stride,
-                                                  y_row_stride, act, a, s)
-           : dtype == KOP_BF16 ? launch_chain<__nv_bfloat16>(x, bias, residual, y, rows, cols, x_row_stride,
-                                                             res_row_stride, y_row_stride, act, a, s)
-                               : launch_chain<__half>(x, bias, residual, y, rows, cols, x_row_stride, res_row_stride,
-                                                      y_row_stride, act, a, s);
+#define KOP_CH_GO(T, PT) launch_chain<T, PT>(x, bias, residual, y, rows, cols, x_row_stride, res_row_stride, y_row_stride, act, a, s)
+    return KOP_DISPATCH_TYPES(dtype, pdtype, KOP_CH_GO);
+#undef KOP_CH_GO
+}
+
+}  // namespace
+}  // namespace kop
+
+extern "C" kop_status_t kop_bias_act(const void* x, const float* bias, void* y, int64_t rows, int64_t cols,
+                                     int64_t x_row_stride, int64_t y_row_stride, int act, float alpha,
+                                     kop_dtype_t dtype, kop_stream_t stream)
+{
+    return kop::bias_act_entry(x, bias, y, rows, cols, x_row_stride, y_row_stride, act, alpha, dtype, KOP_F32, stream);
+}
+
+extern "C" kop_status_t kop_bias_act_ex(const void* x, const void* bias, void* y, int64_t rows, int64_t cols,
+                                        int64_t x_row_stride, int64_t y_row_stride, int act, float alpha,
+                                        kop_dtype_t dtype, kop_dtype_t param_dtype, kop_stream_t stream)
+{
+    return kop::bias_act_entry(x, bias, y, rows, cols, x_row_stride, y_row_stride, act, alpha, dtype, param_dtype, stream);
+}
+
+extern "C" kop_status_t kop_epilogue_chain(const void* x, const float* bias, const void* residual, void* y,
+                                           int64_t rows, int64_t cols, int64_t x_row_stride, int64_t res_row_stride,
+                                           int64_t y_row_stride, float scale, float residual_scale, float clamp_lo,
+                                           float clamp_hi, int act, float alpha, kop_dtype_t dtype,
+                                           kop_stream_t stream)
+{
+    return kop::chain_entry(x, bias, residual, y, rows, cols, x_row_stride, res_row_stride, y_row_stride, scale,
+                            residual_scale, clamp_lo, clamp_hi, act, alpha, dtype, KOP_F32, stream);
+}
+
+extern "C" kop_status_t kop_epilogue_chain_ex(const void* x, const void* bias, const void* residual, void* y,
+                                              int64_t rows, int64_t cols, int64_t x_row_stride, int64_t res_row_stride,
+                                              int64_t y_row_stride, float scale, float residual_scale, float clamp_lo,
+                                              float clamp_hi, int act, float alpha, kop_dtype_t dtype,
+                                              kop_dtype_t param_dtype, kop_stream_t stream)
+{
+    return kop::chain_entry(x, bias, residual, y, rows, cols, x_row_stride, res_row_stride, y_row_stride, scale,
+                            residual_scale, clamp_lo, clamp_hi, act, alpha, dtype, param_dtype, stream);
 }

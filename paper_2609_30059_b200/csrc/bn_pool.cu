@@ -11,17 +11,17 @@ namespace {
 __device__ __forceinline__ float relu_keep_nan(float v) { return v > 0.0f ? v : (v <= 0.0f ? 0.0f : v); }
 
 // One CTA per plane; every thread issues up to UNROLL independent 16-byte loads per trip.
-template <typename T, int UNROLL>
+template <typename T, typename PT, int UNROLL>
 __global__ void __launch_bounds__(1024)
-bn_plane_block_kernel(const T* __restrict__ x, const float* __restrict__ scale,
-                      const float* __restrict__ shift, T* __restrict__ y, float* __restrict__ pooled,
+bn_plane_block_kernel(const T* __restrict__ x, const PT* __restrict__ scale,
+                      const PT* __restrict__ shift, T* __restrict__ y, float* __restrict__ pooled,
                       int nvec, int64_t plane_elems, int C, float inv_plane)
 {
     constexpr int E = Elem<T>::kPerVec;
     __shared__ float red[32];
     const int64_t p = blockIdx.x;
     const int c = (int)(p % C);
-    const float sc = __ldg(scale + c), sh = __ldg(shift + c);
+    const float sc = param1(scale, c), sh = param1(shift, c);
     const T* xp = x + p * plane_elems;
     T* yp = y + p * plane_elems;
     float sum = 0.0f;
@@ -52,10 +52,10 @@ bn_plane_block_kernel(const T* __restrict__ x, const float* __restrict__ scale,
 }
 
 // One warp per plane (small planes), scalar or vector by template flag.
-template <typename T, bool kVec>
+template <typename T, typename PT, bool kVec>
 __global__ void __launch_bounds__(256)
-bn_plane_warp_kernel(const T* __restrict__ x, const float* __restrict__ scale,
-                     const float* __restrict__ shift, T* __restrict__ y, float* __restrict__ pooled,
+bn_plane_warp_kernel(const T* __restrict__ x, const PT* __restrict__ scale,
+                     const PT* __restrict__ shift, T* __restrict__ y, float* __restrict__ pooled,
                      int64_t planes, int64_t plane_elems, int C, float inv_plane)
 {
     constexpr int E = Elem<T>::kPerVec;
@@ -63,7 +63,7 @@ bn_plane_warp_kernel(const T* __restrict__ x, const float* __restrict__ scale,
     const int64_t p = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (p < planes) {
         const int c = (int)(p % C);
-        const float sc = __ldg(scale + c), sh = __ldg(shift + c);
+        const float sc = param1(scale, c), sh = param1(shift, c);
         const T* xp = x + p * plane_elems;
         T* yp = y + p * plane_elems;
         float sum = 0.0f;
@@ -101,9 +101,9 @@ bn_plane_warp_kernel(const T* __restrict__ x, const float* __restrict__ scale,
 constexpr int kFlatThreads = 256;
 constexpr int kFlatMaxElems = 4096;                       // activations parked per CTA (16 KB)
 
-template <typename T>
+template <typename T, typename PT>
 __global__ void __launch_bounds__(kFlatThreads)
-bn_flat_kernel(const T* __restrict__ x, const float* __restrict__ scale, const float* __restrict__ shift,
+bn_flat_kernel(const T* __restrict__ x, const PT* __restrict__ scale, const PT* __restrict__ shift,
                T* __restrict__ y, float* __restrict__ pooled, int64_t planes, int plane, int G, int C,
                float inv_plane)
 {
@@ -117,8 +117,8 @@ bn_flat_kernel(const T* __restrict__ x, const float* __restrict__ scale, const f
     T* yc = y + p0 * plane;
     for (int g = threadIdx.x; g < g_here; g += kFlatThreads) {
         const int c = (int)((p0 + g) % C);
-        sc_s[g] = __ldg(scale + c);
-        sh_s[g] = __ldg(shift + c);
+        sc_s[g] = param1(scale, c);
+        sh_s[g] = param1(shift, c);
     }
     __syncthreads();
     const float inv = 1.0f / (float)plane;
@@ -157,16 +157,16 @@ bn_flat_kernel(const T* __restrict__ x, const float* __restrict__ scale, const f
 }
 
 // Large planes that cannot be vectorised: one CTA per plane, scalar loads.
-template <typename T>
+template <typename T, typename PT>
 __global__ void __launch_bounds__(256)
-bn_plane_scalar_kernel(const T* __restrict__ x, const float* __restrict__ scale,
-                       const float* __restrict__ shift, T* __restrict__ y, float* __restrict__ pooled,
+bn_plane_scalar_kernel(const T* __restrict__ x, const PT* __restrict__ scale,
+                       const PT* __restrict__ shift, T* __restrict__ y, float* __restrict__ pooled,
                        int64_t plane_elems, int C, float inv_plane)
 {
     __shared__ float red[32];
     const int64_t p = blockIdx.x;
     const int c = (int)(p % C);
-    const float sc = __ldg(scale + c), sh = __ldg(shift + c);
+    const float sc = param1(scale, c), sh = param1(shift, c);
     const T* xp = x + p * plane_elems;
     T* yp = y + p * plane_elems;
     float sum = 0.0f;
@@ -179,11 +179,13 @@ bn_plane_scalar_kernel(const T* __restrict__ x, const float* __restrict__ scale,
     if (threadIdx.x == 0) pooled[p] = sum * inv_plane;
 }
 
-template <typename T>
-kop_status_t launch_bn(const void* xv, const float* scale, const float* shift, void* yv, float* pooled,
+template <typename T, typename PT>
+kop_status_t launch_bn(const void* xv, const void* scalev, const void* shiftv, void* yv, float* pooled,
                        int64_t N, int64_t C, int64_t H, int64_t W, cudaStream_t stream)
 {
     const T* x = static_cast<const T*>(xv);
+    const PT* scale = static_cast<const PT*>(scalev);
+    const PT* shift = static_cast<const PT*>(shiftv);
     T* y = static_cast<T*>(yv);
     constexpr int E = Elem<T>::kPerVec;
     const int64_t plane = H * W, planes = N * C;
@@ -200,7 +202,7 @@ kop_status_t launch_bn(const void* xv, const float* scale, const float* shift, v
         if (G * plane <= kFlatMaxElems) {
             const int64_t ctas = (planes + G - 1) / G;
             if (ctas > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
-            bn_flat_kernel<T><<<(unsigned)ctas, kFlatThreads, 0, stream>>>(x, scale, shift, y, pooled, planes,
+            bn_flat_kernel<T, PT><<<(unsigned)ctas, kFlatThreads, 0, stream>>>(x, scale, shift, y, pooled, planes,
                                                                           (int)plane, (int)G, (int)C, inv_plane);
             return launch_status();
         }
@@ -210,9 +212,9 @@ kop_status_t launch_bn(const void* xv, const float* scale, const float* shift, v
         if (ctas > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
         const unsigned grid = (unsigned)ctas;
         if (vec)
-            bn_plane_warp_kernel<T, true><<<grid, 256, 0, stream>>>(x, scale, shift, y, pooled, planes, plane, (int)C, inv_plane);
+            bn_plane_warp_kernel<T, PT, true><<<grid, 256, 0, stream>>>(x, scale, shift, y, pooled, planes, plane, (int)C, inv_plane);
         else
-            bn_plane_warp_kernel<T, false><<<grid, 256, 0, stream>>>(x, scale, shift, y, pooled, planes, plane, (int)C, inv_plane);
+            bn_plane_warp_kernel<T, PT, false><<<grid, 256, 0, stream>>>(x, scale, shift, y, pooled, planes, plane, (int)C, inv_plane);
         return launch_status();
     }
     if (vec && nvec64 <= 0x7FFFFFFF) {
@@ -221,10 +223,10 @@ kop_status_t launch_bn(const void* xv, const float* scale, const float* shift, v
         // and a single trip (196 threads would cover it exactly; 224 is the next warp multiple).
         int threads = ((nvec + 3) / 4 + 31) / 32 * 32;
         if (threads > 512) threads = 512;
-        bn_plane_block_kernel<T, 4><<<(unsigned)planes, threads, 0, stream>>>(x, scale, shift, y, pooled, nvec, plane, (int)C, inv_plane);
+        bn_plane_block_kernel<T, PT, 4><<<(unsigned)planes, threads, 0, stream>>>(x, scale, shift, y, pooled, nvec, plane, (int)C, inv_plane);
         return launch_status();
     }
-    bn_plane_scalar_kernel<T><<<(unsigned)planes, 256, 0, stream>>>(x, scale, shift, y, pooled, plane, (int)C, inv_plane);
+    bn_plane_scalar_kernel<T, PT><<<(unsigned)planes, 256, 0, stream>>>(x, scale, shift, y, pooled, plane, (int)C, inv_plane);
     return launch_status();
 }
 
@@ -239,9 +241,9 @@ kop_status_t launch_bn(const void* xv, const float* scale, const float* shift, v
 // shape a fixed summation order.
 constexpr int kBnMaxSlabs = 8;      // portable cluster size
 
-template <typename T, int TV, int U, bool kCluster>
+template <typename T, typename PT, int TV, int U, bool kCluster>
 __global__ void __launch_bounds__(256)
-bn_nhwc_kernel(const T* __restrict__ x, const float* __restrict__ scale, const float* __restrict__ shift,
+bn_nhwc_kernel(const T* __restrict__ x, const PT* __restrict__ scale, const PT* __restrict__ shift,
                T* __restrict__ y, float* __restrict__ pooled, int64_t hw, int cvec, int tiles, int slabs,
                float inv_hw)
 {
@@ -267,8 +269,8 @@ bn_nhwc_kernel(const T* __restrict__ x, const float* __restrict__ scale, const f
     float sc[E], sh[E], acc[E];
 #pragma unroll
     for (int e = 0; e < E; ++e) {
-        sc[e] = live ? __ldg(scale + (int64_t)cv * E + e) : 0.0f;
-        sh[e] = live ? __ldg(shift + (int64_t)cv * E + e) : 0.0f;
+        sc[e] = live ? param1(scale, (int64_t)cv * E + e) : 0.0f;
+        sh[e] = live ? param1(shift, (int64_t)cv * E + e) : 0.0f;
         acc[e] = 0.0f;
     }
     const T* xn = x + n * hw * C + (int64_t)cv * E;
@@ -322,9 +324,9 @@ bn_nhwc_kernel(const T* __restrict__ x, const float* __restrict__ scale, const f
 }
 
 // Any channel count / alignment: lanes along channels with scalar loads, warps along rows.
-template <typename T>
+template <typename T, typename PT>
 __global__ void __launch_bounds__(256)
-bn_nhwc_scalar_kernel(const T* __restrict__ x, const float* __restrict__ scale, const float* __restrict__ shift,
+bn_nhwc_scalar_kernel(const T* __restrict__ x, const PT* __restrict__ scale, const PT* __restrict__ shift,
                       T* __restrict__ y, float* __restrict__ pooled, int64_t hw, int64_t C, int tiles,
                       float inv_hw)
 {
@@ -334,7 +336,7 @@ bn_nhwc_scalar_kernel(const T* __restrict__ x, const float* __restrict__ scale, 
     const int64_t c = (blockIdx.x - n * tiles) * 32 + lane;
     float acc = 0.0f;
     if (c < C) {
-        const float sc = __ldg(scale + c), sh = __ldg(shift + c);
+        const float sc = param1(scale, c), sh = param1(shift, c);
         const T* xn = x + n * hw * C + c;
         T* yn = y + n * hw * C + c;
         for (int64_t r = warp; r < hw; r += 8) {
@@ -353,11 +355,13 @@ bn_nhwc_scalar_kernel(const T* __restrict__ x, const float* __restrict__ scale, 
     }
 }
 
-template <typename T>
-kop_status_t launch_bn_nhwc(const void* xv, const float* scale, const float* shift, void* yv, float* pooled,
+template <typename T, typename PT>
+kop_status_t launch_bn_nhwc(const void* xv, const void* scalev, const void* shiftv, void* yv, float* pooled,
                             int64_t N, int64_t C, int64_t H, int64_t W, cudaStream_t stream)
 {
     const T* x = static_cast<const T*>(xv);
+    const PT* scale = static_cast<const PT*>(scalev);
+    const PT* shift = static_cast<const PT*>(shiftv);
     T* y = static_cast<T*>(yv);
     constexpr int E = Elem<T>::kPerVec;
     const int64_t hw = H * W;
@@ -390,9 +394,9 @@ kop_status_t launch_bn_nhwc(const void* xv, const float* scale, const float* shi
         cfg.numAttrs = slabs > 1 ? 1 : 0;
         cudaError_t err;
 #define KOP_BN_NHWC(TVV)                                                                                         \
-    err = slabs > 1 ? cudaLaunchKernelEx(&cfg, bn_nhwc_kernel<T, TVV, 4, true>, x, scale, shift, y, pooled, hw,   \
+    err = slabs > 1 ? cudaLaunchKernelEx(&cfg, bn_nhwc_kernel<T, PT, TVV, 4, true>, x, scale, shift, y, pooled, hw,   \
                                          cvec, tiles, slabs, inv_hw)                                              \
-                    : cudaLaunchKernelEx(&cfg, bn_nhwc_kernel<T, TVV, 4, false>, x, scale, shift, y, pooled, hw,  \
+                    : cudaLaunchKernelEx(&cfg, bn_nhwc_kernel<T, PT, TVV, 4, false>, x, scale, shift, y, pooled, hw,  \
                                          cvec, tiles, slabs, inv_hw)
         switch (tv) {
         case 16: KOP_BN_NHWC(16); break;
@@ -410,21 +414,21 @@ kop_status_t launch_bn_nhwc(const void* xv, const float* scale, const float* shi
     }
     const int64_t tiles = (C + 31) / 32;
     if (N * tiles > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
-    bn_nhwc_scalar_kernel<T><<<(unsigned)(N * tiles), 256, 0, stream>>>(x, scale, shift, y, pooled, hw, C, (int)tiles, inv_hw);
+    bn_nhwc_scalar_kernel<T, PT><<<(unsigned)(N * tiles), 256, 0, stream>>>(x, scale, shift, y, pooled, hw, C, (int)tiles, inv_hw);
     return launch_status();
 }
 
 }  // namespace
 }  // namespace kop
 
-extern "C" kop_status_t kop_bn_relu_avgpool(const void* x, const float* scale, const float* shift,
-                                            void* y, float* pooled, int64_t N, int64_t C, int64_t H,
-                                            int64_t W, const int64_t x_strides[4],
-                                            const int64_t y_strides[4], kop_dtype_t dtype,
-                                            kop_stream_t stream)
+namespace kop {
+namespace {
+
+kop_status_t bn_entry(const void* x, const void* scale, const void* shift, void* y, float* pooled, int64_t N, int64_t C,
+                      int64_t H, int64_t W, const int64_t x_strides[4], const int64_t y_strides[4], kop_dtype_t dtype,
+                      kop_dtype_t pdtype, kop_stream_t stream)
 {
-    using namespace kop;
-    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    if (!param_dtype_ok(dtype, pdtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
     if (N < 0 || C <= 0 || H <= 0 || W <= 0) return KOP_ERR_BAD_SHAPE;
     if (N == 0) return KOP_OK;
     if (!x || !scale || !shift || !y || !pooled || !x_strides || !y_strides) return KOP_ERR_NULL_POINTER;
@@ -446,18 +450,38 @@ extern "C" kop_status_t kop_bn_relu_avgpool(const void* x, const float* scale, c
     }
     if (!is_nchw && !is_nhwc) return KOP_ERR_BAD_STRIDE;
     const int esz = elem_size(dtype);
-    if (!aligned_to(x, esz) || !aligned_to(y, esz) || !aligned_to(scale, 4) || !aligned_to(shift, 4) ||
+    if (!aligned_to(x, esz) || !aligned_to(y, esz) || !aligned_to(scale, elem_size(pdtype)) ||
+        !aligned_to(shift, elem_size(pdtype)) ||
         !aligned_to(pooled, 4))
         return KOP_ERR_MISALIGNED;
     if (!alias_ok(x, C * plane, y, C * plane, N, C * plane, esz, true)) return KOP_ERR_BAD_ALIAS;
     kop_status_t st = check_device();
     if (st != KOP_OK) return st;
     cudaStream_t s = as_stream(stream);
-    if (!is_nchw)
-        return dtype == KOP_F32 ? launch_bn_nhwc<float>(x, scale, shift, y, pooled, N, C, H, W, s)
-                                : dtype == KOP_BF16 ? launch_bn_nhwc<__nv_bfloat16>(x, scale, shift, y, pooled, N, C, H, W, s)
-                                : launch_bn_nhwc<__half>(x, scale, shift, y, pooled, N, C, H, W, s);
-    return dtype == KOP_F32 ? launch_bn<float>(x, scale, shift, y, pooled, N, C, H, W, s)
-                            : dtype == KOP_BF16 ? launch_bn<__nv_bfloat16>(x, scale, shift, y, pooled, N, C, H, W, s)
-                            : launch_bn<__half>(x, scale, shift, y, pooled, N, C, H, W, s);
+#define KOP_BN_NHWC_GO(T, PT) launch_bn_nhwc<T, PT>(x, scale, shift, y, pooled, N, C, H, W, s)
+#define KOP_BN_GO(T, PT) launch_bn<T, PT>(x, scale, shift, y, pooled, N, C, H, W, s)
+    if (!is_nchw) return KOP_DISPATCH_TYPES(dtype, pdtype, KOP_BN_NHWC_GO);
+    return KOP_DISPATCH_TYPES(dtype, pdtype, KOP_BN_GO);
+#undef KOP_BN_NHWC_GO
+#undef KOP_BN_GO
+}
+
+}  // namespace
+}  // namespace kop
+
+extern "C" kop_status_t kop_bn_relu_avgpool(const void* x, const float* scale, const float* shift,
+                                            void* y, float* pooled, int64_t N, int64_t C, int64_t H,
+                                            int64_t W, const int64_t x_strides[4],
+                                            const int64_t y_strides[4], kop_dtype_t dtype,
+                                            kop_stream_t stream)
+{
+    return kop::bn_entry(x, scale, shift, y, pooled, N, C, H, W, x_strides, y_strides, dtype, KOP_F32, stream);
+}
+
+extern "C" kop_status_t kop_bn_relu_avgpool_ex(const void* x, const void* scale, const void* shift, void* y,
+                                               float* pooled, int64_t N, int64_t C, int64_t H, int64_t W,
+                                               const int64_t x_strides[4], const int64_t y_strides[4],
+                                               kop_dtype_t dtype, kop_dtype_t param_dtype, kop_stream_t stream)
+{
+    return kop::bn_entry(x, scale, shift, y, pooled, N, C, H, W, x_strides, y_strides, dtype, param_dtype, stream);
 }

@@ -77,13 +77,13 @@ constexpr int kGnMaxParts = 7;                           // covers the 200 KB st
 
 // y = act((x - mu) * rstd * gamma[c] + beta[c]) for one vector; a vector never straddles two channels.
 // (x - mu) first: folding mu into a shift would cost |mu| * rstd ulps when the spread is small.
-template <typename T, int ACT>
-__device__ __forceinline__ void normalize_store(const Vec16& raw, T* dst, int c, const float* gamma,
-                                                const float* beta, float mu, float rs)
+template <typename T, int ACT, typename PT>
+__device__ __forceinline__ void normalize_store(const Vec16& raw, T* dst, int c, const PT* gamma,
+                                                const PT* beta, float mu, float rs)
 {
     constexpr int P = Elem<T>::kPerVec / 2;
-    const float sc = rs * (gamma != nullptr ? __ldg(gamma + c) : 1.0f);
-    const float be = beta != nullptr ? __ldg(beta + c) : 0.0f;
+    const float sc = rs * (gamma != nullptr ? param1(gamma, c) : 1.0f);
+    const float be = beta != nullptr ? param1(beta, c) : 0.0f;
     const float2 nmu = make_float2(-mu, -mu), sc2 = make_float2(sc, sc), be2 = make_float2(be, be);
     float2 f[P];
     Elem<T>::unpack2(raw, f);
@@ -109,9 +109,9 @@ __device__ __forceinline__ void normalize_store(const Vec16& raw, T* dst, int c,
 
 // Chunks beyond the staging budget: two sweeps over global memory (the second mostly served by L2).
 // Self-contained on purpose (it shares only merge / warp_merge / activate with the staged kernel).
-template <typename T, int ACT>
+template <typename T, typename PT, int ACT>
 __global__ void __launch_bounds__(kGnThreads)
-groupnorm_twosweep_kernel(const T* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
+groupnorm_twosweep_kernel(const T* __restrict__ x, const PT* __restrict__ gamma, const PT* __restrict__ beta,
                           T* __restrict__ y, float* __restrict__ mean, float* __restrict__ rstd, int nvec,
                           int vec_per_plane, int cpg, int groups, float eps)
 {
@@ -200,8 +200,8 @@ groupnorm_twosweep_kernel(const T* __restrict__ x, const float* __restrict__ gam
             const int v = base + k * kGnThreads + threadIdx.x;
             if (v < nvec) {
                 const int c = g * cpg + v / vec_per_plane;           // a vector never straddles two channels
-                const float ga = gamma != nullptr ? __ldg(gamma + c) : 1.0f;
-                const float be = beta != nullptr ? __ldg(beta + c) : 0.0f;
+                const float ga = gamma != nullptr ? param1(gamma, c) : 1.0f;
+                const float be = beta != nullptr ? param1(beta, c) : 0.0f;
                 const float sc = rs * ga;
                 float f[E];
                 Elem<T>::unpack(raw[k], f);
@@ -267,9 +267,9 @@ __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src, uint3
 // warps). With the chunk in shared memory the statistics are the textbook two-pass ones: the sum is
 // accumulated part by part as the copies land, the squared deviations from the exact mean in a second
 // sweep over shared memory; both CTA reductions are plain sums (one barrier each, fixed order).
-template <typename T, int ACT, int NT>
+template <typename T, typename PT, int ACT, int NT>
 __global__ void __launch_bounds__(NT)
-groupnorm_staged_kernel(const T* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
+groupnorm_staged_kernel(const T* __restrict__ x, const PT* __restrict__ gamma, const PT* __restrict__ beta,
                         T* __restrict__ y, float* __restrict__ mean, float* __restrict__ rstd, int nvec,
                         int vec_per_plane, int cpg, int groups, float eps, float inv_count)
 {
@@ -369,9 +369,9 @@ groupnorm_staged_kernel(const T* __restrict__ x, const float* __restrict__ gamma
 // every CTA runs every cluster barrier whatever happens to its copies.
 constexpr int kGnClusterThreads = 512;
 
-template <typename T, int ACT>
+template <typename T, typename PT, int ACT>
 __global__ void __launch_bounds__(kGnClusterThreads)
-groupnorm_cluster_kernel(const T* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
+groupnorm_cluster_kernel(const T* __restrict__ x, const PT* __restrict__ gamma, const PT* __restrict__ beta,
                          T* __restrict__ y, float* __restrict__ mean, float* __restrict__ rstd, int nvec,
                          int slice_vecs, int csize, int vec_per_plane, int cpg, int groups, float eps, float inv_count)
 {
@@ -493,10 +493,10 @@ groupnorm_cluster_kernel(const T* __restrict__ x, const float* __restrict__ gamm
 // megabytes): one CTA per chunk would leave most SMs idle. A cluster of up to 8 CTAs shares the chunk, a slice
 // each, in the two-sweep manner (moments in one sweep, output in a second, mostly from the L2); the slices'
 // (count, mean, M2) triples are exchanged through distributed shared memory and merged pairwise in rank order.
-template <typename T, int ACT>
+template <typename T, typename PT, int ACT>
 __global__ void __launch_bounds__(kGnThreads)
-groupnorm_twosweep_cluster_kernel(const T* __restrict__ x, const float* __restrict__ gamma,
-                                  const float* __restrict__ beta, T* __restrict__ y, float* __restrict__ mean,
+groupnorm_twosweep_cluster_kernel(const T* __restrict__ x, const PT* __restrict__ gamma,
+                                  const PT* __restrict__ beta, T* __restrict__ y, float* __restrict__ mean,
                                   float* __restrict__ rstd, int nvec, int slice_vecs, int csize, int vec_per_plane,
                                   int cpg, int groups, float eps)
 {
@@ -589,8 +589,8 @@ groupnorm_twosweep_cluster_kernel(const T* __restrict__ x, const float* __restri
             const int v = base + k * kGnThreads + threadIdx.x;
             if (v < n_here) {
                 const int c = g * cpg + (v_lo + v) / vec_per_plane;
-                const float ga = gamma != nullptr ? __ldg(gamma + c) : 1.0f;
-                const float be = beta != nullptr ? __ldg(beta + c) : 0.0f;
+                const float ga = gamma != nullptr ? param1(gamma, c) : 1.0f;
+                const float be = beta != nullptr ? param1(beta, c) : 0.0f;
                 const float sc = rs * ga;
                 float f[E];
                 Elem<T>::unpack(raw[k], f);
@@ -612,9 +612,9 @@ constexpr int kGnSmallThreads = 256;
 constexpr int kGnSmallMaxChunk = 2048;           // elements
 constexpr int kGnSmallRunElems = 6144;           // about 24 KB of activations per CTA
 
-template <typename T, int ACT>
+template <typename T, typename PT, int ACT>
 __global__ void __launch_bounds__(kGnSmallThreads)
-groupnorm_small_kernel(const T* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
+groupnorm_small_kernel(const T* __restrict__ x, const PT* __restrict__ gamma, const PT* __restrict__ beta,
                        T* __restrict__ y, float* __restrict__ mean, float* __restrict__ rstd, int64_t chunks, int R,
                        int chunk_elems, int plane, int cpg, int groups, float eps)
 {
@@ -676,8 +676,8 @@ groupnorm_small_kernel(const T* __restrict__ x, const float* __restrict__ gamma,
     const int g0 = (int)(p0 % groups);                       // group of the run's first chunk
     // the normalised value of element i of the run: chunk r, channel ch of the tensor
     auto out_value = [&](int i, int r, int ch) {
-        const float sc = rs_s[r] * (gamma != nullptr ? __ldg(gamma + ch) : 1.0f);
-        const float be = beta != nullptr ? __ldg(beta + ch) : 0.0f;
+        const float sc = rs_s[r] * (gamma != nullptr ? param1(gamma, ch) : 1.0f);
+        const float be = beta != nullptr ? param1(beta, ch) : 0.0f;
         return activate<ACT>(fmaf(val[i] - mu_s[r], sc, be));
     };
     for (int v = threadIdx.x; v < nvec; v += kGnSmallThreads) {
@@ -711,9 +711,9 @@ groupnorm_small_kernel(const T* __restrict__ x, const float* __restrict__ gamma,
 }
 
 // Any plane size / alignment: scalar loads, two sweeps over global memory, same moment arithmetic.
-template <typename T, int ACT>
+template <typename T, typename PT, int ACT>
 __global__ void __launch_bounds__(256)
-groupnorm_scalar_kernel(const T* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
+groupnorm_scalar_kernel(const T* __restrict__ x, const PT* __restrict__ gamma, const PT* __restrict__ beta,
                         T* __restrict__ y, float* __restrict__ mean, float* __restrict__ rstd,
                         int64_t chunk_elems, int64_t plane, int cpg, int groups, float eps)
 {
@@ -749,8 +749,8 @@ groupnorm_scalar_kernel(const T* __restrict__ x, const float* __restrict__ gamma
     const float mu = bc_mean, rs = bc_rstd;
     for (int64_t j = threadIdx.x; j < chunk_elems; j += blockDim.x) {
         const int c = g * cpg + (int)(j / plane);
-        const float sc = rs * (gamma != nullptr ? __ldg(gamma + c) : 1.0f);
-        const float be = beta != nullptr ? __ldg(beta + c) : 0.0f;
+        const float sc = rs * (gamma != nullptr ? param1(gamma, c) : 1.0f);
+        const float be = beta != nullptr ? param1(beta, c) : 0.0f;
         Elem<T>::store1(yc + j, activate<ACT>(fmaf(Elem<T>::load1(xc + j) - mu, sc, be)));
     }
 }
@@ -759,8 +759,8 @@ constexpr size_t kGnStageLimit = 200 * 1024;     // leaves room for the static r
 static_assert(kGnStageLimit <= (size_t)kGnMaxParts * kGnCopyVecs * 16, "one barrier per 32 KB part");
 constexpr int kMaxDevices = 64;
 
-template <typename T, int ACT>
-kop_status_t launch_gn_act(const T* x, const float* gamma, const float* beta, T* y, float* mean, float* rstd,
+template <typename T, typename PT, int ACT>
+kop_status_t launch_gn_act(const T* x, const PT* gamma, const PT* beta, T* y, float* mean, float* rstd,
                            int64_t chunks, int64_t chunk_elems, int64_t plane, int cpg, int groups, float eps,
                            cudaStream_t stream)
 {
@@ -775,7 +775,7 @@ kop_status_t launch_gn_act(const T* x, const float* gamma, const float* beta, T*
         const int64_t ctas = (chunks + R - 1) / R;
         const size_t smem = ((size_t)R * chunk_elems + 2 * (size_t)R) * sizeof(float);
         if (ctas <= 0x7FFFFFFFLL && smem <= 47 * 1024) {
-            groupnorm_small_kernel<T, ACT><<<(unsigned)ctas, kGnSmallThreads, smem, stream>>>(
+            groupnorm_small_kernel<T, PT, ACT><<<(unsigned)ctas, kGnSmallThreads, smem, stream>>>(
                 x, gamma, beta, y, mean, rstd, chunks, R, (int)chunk_elems, (int)plane, cpg, groups, eps);
             return launch_status();
         }
@@ -792,7 +792,7 @@ kop_status_t launch_gn_act(const T* x, const float* gamma, const float* beta, T*
             if (cudaGetDevice(&dev) != cudaSuccess) return KOP_ERR_CUDA;
             if (dev < 0 || dev >= kMaxDevices || !configured[dev].load(std::memory_order_acquire)) {
                 // only the 512-thread instance ever needs more than the default 48 KB (chunks beyond 32 KB)
-                if (cudaFuncSetAttribute(groupnorm_staged_kernel<T, ACT, 512>,
+                if (cudaFuncSetAttribute(groupnorm_staged_kernel<T, PT, ACT, 512>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)kGnStageLimit) != cudaSuccess)
                     return KOP_ERR_CUDA;
@@ -800,13 +800,13 @@ kop_status_t launch_gn_act(const T* x, const float* gamma, const float* beta, T*
             }
             const float inv_count = (float)(1.0 / (double)chunk_elems);
             if (nvec <= 512)
-                groupnorm_staged_kernel<T, ACT, 128><<<(unsigned)chunks, 128, bytes, stream>>>(
+                groupnorm_staged_kernel<T, PT, ACT, 128><<<(unsigned)chunks, 128, bytes, stream>>>(
                     x, gamma, beta, y, mean, rstd, nvec, vpp, cpg, groups, eps, inv_count);
             else if (nvec <= 2048)
-                groupnorm_staged_kernel<T, ACT, 256><<<(unsigned)chunks, 256, bytes, stream>>>(
+                groupnorm_staged_kernel<T, PT, ACT, 256><<<(unsigned)chunks, 256, bytes, stream>>>(
                     x, gamma, beta, y, mean, rstd, nvec, vpp, cpg, groups, eps, inv_count);
             else
-                groupnorm_staged_kernel<T, ACT, 512><<<(unsigned)chunks, 512, bytes, stream>>>(
+                groupnorm_staged_kernel<T, PT, ACT, 512><<<(unsigned)chunks, 512, bytes, stream>>>(
                     x, gamma, beta, y, mean, rstd, nvec, vpp, cpg, groups, eps, inv_count);
         } else if (bytes <= 512 * 1024 && chunks * 8 <= 0x7FFFFFFFLL) {
             // a cluster per chunk, slices of at most 64 KB (three CTAs per SM). Measured against the two-sweep
@@ -821,7 +821,7 @@ kop_status_t launch_gn_act(const T* x, const float* gamma, const float* beta, T*
             int dev = 0;
             if (cudaGetDevice(&dev) != cudaSuccess) return KOP_ERR_CUDA;
             if (dev < 0 || dev >= kMaxDevices || !configured_c[dev].load(std::memory_order_acquire)) {
-                if (cudaFuncSetAttribute(groupnorm_cluster_kernel<T, ACT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                if (cudaFuncSetAttribute(groupnorm_cluster_kernel<T, PT, ACT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)kGnStageLimit) != cudaSuccess)
                     return KOP_ERR_CUDA;
                 if (dev >= 0 && dev < kMaxDevices) configured_c[dev].store(true, std::memory_order_release);
@@ -839,7 +839,7 @@ kop_status_t launch_gn_act(const T* x, const float* gamma, const float* beta, T*
             cfg.attrs = attr;
             cfg.numAttrs = 1;
             const float inv_count = (float)(1.0 / (double)chunk_elems);
-            if (cudaLaunchKernelEx(&cfg, groupnorm_cluster_kernel<T, ACT>, x, gamma, beta, y, mean, rstd, nvec, slice_vecs,
+            if (cudaLaunchKernelEx(&cfg, groupnorm_cluster_kernel<T, PT, ACT>, x, gamma, beta, y, mean, rstd, nvec, slice_vecs,
                                    csize, vpp, cpg, groups, eps, inv_count) != cudaSuccess) {
                 (void)cudaGetLastError();
                 return KOP_ERR_CUDA;
@@ -862,46 +862,49 @@ kop_status_t launch_gn_act(const T* x, const float* gamma, const float* beta, T*
             attr[0].val.clusterDim.z = 1;
             cfg.attrs = attr;
             cfg.numAttrs = 1;
-            if (cudaLaunchKernelEx(&cfg, groupnorm_twosweep_cluster_kernel<T, ACT>, x, gamma, beta, y, mean, rstd, nvec,
+            if (cudaLaunchKernelEx(&cfg, groupnorm_twosweep_cluster_kernel<T, PT, ACT>, x, gamma, beta, y, mean, rstd, nvec,
                                    slice_vecs, csize, vpp, cpg, groups, eps) != cudaSuccess) {
                 (void)cudaGetLastError();
                 return KOP_ERR_CUDA;
             }
         } else {
-            groupnorm_twosweep_kernel<T, ACT><<<(unsigned)chunks, kGnThreads, 0, stream>>>(
+            groupnorm_twosweep_kernel<T, PT, ACT><<<(unsigned)chunks, kGnThreads, 0, stream>>>(
                 x, gamma, beta, y, mean, rstd, nvec, vpp, cpg, groups, eps);
         }
         return launch_status();
     }
-    groupnorm_scalar_kernel<T, ACT><<<(unsigned)chunks, 256, 0, stream>>>(x, gamma, beta, y, mean, rstd, chunk_elems,
+    groupnorm_scalar_kernel<T, PT, ACT><<<(unsigned)chunks, 256, 0, stream>>>(x, gamma, beta, y, mean, rstd, chunk_elems,
                                                                           plane, cpg, groups, eps);
     return launch_status();
 }
 
-template <typename T>
-kop_status_t launch_gn(const void* x, const float* gamma, const float* beta, void* y, float* mean, float* rstd,
+template <typename T, typename PT>
+kop_status_t launch_gn(const void* x, const void* gammav, const void* betav, void* y, float* mean, float* rstd,
                        int64_t chunks, int64_t chunk_elems, int64_t plane, int cpg, int groups, float eps, int act,
                        cudaStream_t stream)
 {
     const T* xt = static_cast<const T*>(x);
+    const PT* gamma = static_cast<const PT*>(gammav);
+    const PT* beta = static_cast<const PT*>(betav);
     T* yt = static_cast<T*>(y);
     switch (act) {
-    case kActRelu: return launch_gn_act<T, kActRelu>(xt, gamma, beta, yt, mean, rstd, chunks, chunk_elems, plane, cpg, groups, eps, stream);
-    case kActSilu: return launch_gn_act<T, kActSilu>(xt, gamma, beta, yt, mean, rstd, chunks, chunk_elems, plane, cpg, groups, eps, stream);
-    default: return launch_gn_act<T, kActNone>(xt, gamma, beta, yt, mean, rstd, chunks, chunk_elems, plane, cpg, groups, eps, stream);
+    case kActRelu: return launch_gn_act<T, PT, kActRelu>(xt, gamma, beta, yt, mean, rstd, chunks, chunk_elems, plane, cpg, groups, eps, stream);
+    case kActSilu: return launch_gn_act<T, PT, kActSilu>(xt, gamma, beta, yt, mean, rstd, chunks, chunk_elems, plane, cpg, groups, eps, stream);
+    default: return launch_gn_act<T, PT, kActNone>(xt, gamma, beta, yt, mean, rstd, chunks, chunk_elems, plane, cpg, groups, eps, stream);
     }
 }
 
 }  // namespace
 }  // namespace kop
 
-extern "C" kop_status_t kop_groupnorm_act(const void* x, const float* gamma, const float* beta, void* y,
-                                          float* mean, float* rstd, int64_t N, int64_t C, int64_t H, int64_t W,
-                                          int64_t groups, float eps, int act, kop_dtype_t dtype,
-                                          kop_stream_t stream)
+namespace kop {
+namespace {
+
+kop_status_t gn_entry(const void* x, const void* gamma, const void* beta, void* y, float* mean, float* rstd, int64_t N,
+                      int64_t C, int64_t H, int64_t W, int64_t groups, float eps, int act, kop_dtype_t dtype,
+                      kop_dtype_t pdtype, kop_stream_t stream)
 {
-    using namespace kop;
-    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    if (!param_dtype_ok(dtype, pdtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
     if (N < 0 || C <= 0 || H <= 0 || W <= 0 || groups <= 0 || groups > C || C % groups != 0) return KOP_ERR_BAD_SHAPE;
     if (act < 0 || act > 2 || !(eps >= 0.0f)) return KOP_ERR_BAD_SHAPE;
     if (C > 0x7FFFFFFF || H > kMaxElems || W > kMaxElems || N > kMaxElems || H > kMaxElems / W) return KOP_ERR_BAD_SHAPE;
@@ -912,8 +915,8 @@ extern "C" kop_status_t kop_groupnorm_act(const void* x, const float* gamma, con
     if (N * groups > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;           // one CTA per (image, group)
     if (!x || !y) return KOP_ERR_NULL_POINTER;
     const int esz = elem_size(dtype);
-    if (!aligned_to(x, esz) || !aligned_to(y, esz) || (gamma && !aligned_to(gamma, 4)) ||
-        (beta && !aligned_to(beta, 4)) || (mean && !aligned_to(mean, 4)) || (rstd && !aligned_to(rstd, 4)))
+    if (!aligned_to(x, esz) || !aligned_to(y, esz) || (gamma && !aligned_to(gamma, elem_size(pdtype))) ||
+        (beta && !aligned_to(beta, elem_size(pdtype))) || (mean && !aligned_to(mean, 4)) || (rstd && !aligned_to(rstd, 4)))
         return KOP_ERR_MISALIGNED;
     if (!alias_ok(x, C * plane, y, C * plane, N, C * plane, esz, true)) return KOP_ERR_BAD_ALIAS;
     kop_status_t st = check_device();
@@ -921,10 +924,28 @@ extern "C" kop_status_t kop_groupnorm_act(const void* x, const float* gamma, con
     const int cpg = (int)(C / groups);
     const int64_t chunk_elems = (int64_t)cpg * plane;
     cudaStream_t s = as_stream(stream);
-    return dtype == KOP_F32
-               ? launch_gn<float>(x, gamma, beta, y, mean, rstd, N * groups, chunk_elems, plane, cpg, (int)groups, eps, act, s)
-               : dtype == KOP_BF16 ? launch_gn<__nv_bfloat16>(x, gamma, beta, y, mean, rstd, N * groups, chunk_elems, plane, cpg, (int)groups, eps, act, s)
-               : launch_gn<__half>(x, gamma, beta, y, mean, rstd, N * groups, chunk_elems, plane, cpg, (int)groups, eps, act, s);
+#define KOP_GN_GO(T, PT) launch_gn<T, PT>(x, gamma, beta, y, mean, rstd, N * groups, chunk_elems, plane, cpg, (int)groups, eps, act, s)
+    return KOP_DISPATCH_TYPES(dtype, pdtype, KOP_GN_GO);
+#undef KOP_GN_GO
+}
+
+}  // namespace
+}  // namespace kop
+
+extern "C" kop_status_t kop_groupnorm_act(const void* x, const float* gamma, const float* beta, void* y,
+                                          float* mean, float* rstd, int64_t N, int64_t C, int64_t H, int64_t W,
+                                          int64_t groups, float eps, int act, kop_dtype_t dtype,
+                                          kop_stream_t stream)
+{
+    return kop::gn_entry(x, gamma, beta, y, mean, rstd, N, C, H, W, groups, eps, act, dtype, KOP_F32, stream);
+}
+
+extern "C" kop_status_t kop_groupnorm_act_ex(const void* x, const void* gamma, const void* beta, void* y, float* mean,
+                                             float* rstd, int64_t N, int64_t C, int64_t H, int64_t W, int64_t groups,
+                                             float eps, int act, kop_dtype_t dtype, kop_dtype_t param_dtype,
+                                             kop_stream_t stream)
+{
+    return kop::gn_entry(x, gamma, beta, y, mean, rstd, N, C, H, W, groups, eps, act, dtype, param_dtype, stream);
 }
 
 extern "C" kop_status_t kop_groupnorm_wait_timeouts(unsigned int* host_count)

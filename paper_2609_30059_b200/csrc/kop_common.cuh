@@ -17,6 +17,18 @@ namespace kop {
 inline bool dtype_ok(kop_dtype_t d) { return d == KOP_F32 || d == KOP_BF16 || d == KOP_F16; }
 inline int elem_size(kop_dtype_t d) { return d == KOP_F32 ? 4 : 2; }
 inline bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+// Parameter vectors are fp32 or stored in the data type (a 16-bit model keeps its biases and norm weights in that type).
+inline bool param_dtype_ok(kop_dtype_t dtype, kop_dtype_t pdtype)
+{
+    return dtype_ok(dtype) && dtype_ok(pdtype) && (pdtype == KOP_F32 || pdtype == dtype);
+}
+
+// CALL(T, PT) for the C++ types behind (dtype, pdtype); the caller has checked param_dtype_ok. CALL is a
+// function-like macro that expands to an expression of type kop_status_t.
+#define KOP_DISPATCH_TYPES(dtype, pdtype, CALL)                                                              \
+    ((dtype) == KOP_F32    ? CALL(float, float)                                                              \
+     : (dtype) == KOP_BF16 ? ((pdtype) == KOP_F32 ? CALL(__nv_bfloat16, float) : CALL(__nv_bfloat16, __nv_bfloat16)) \
+                           : ((pdtype) == KOP_F32 ? CALL(__half, float) : CALL(__half, __half)))
 
 // Largest product / offset we accept: keeps every byte offset inside int64.
 constexpr int64_t kMaxElems = (int64_t)1 << 46;
@@ -436,6 +448,21 @@ __device__ __forceinline__ void load_params(const PT* p, float2 (&out)[E / 2])
     static_assert(E == 8 && sizeof(PT) == 2, "16-bit parameters go with 16-bit data");
     const uint4 t = __ldg(reinterpret_cast<const uint4*>(p));
     Elem<PT>::unpack2(Vec16{{t.x, t.y, t.z, t.w}}, out);
+}
+// Four consecutive parameters as fp32 (16-byte aligned for fp32, 8-byte for 16-bit parameters).
+__device__ __forceinline__ float4 ldg_p4(const float* p) { return ldg_f4(p); }
+__device__ __forceinline__ float4 ldg_p4(const __nv_bfloat16* p)
+{
+    const uint2 t = __ldg(reinterpret_cast<const uint2*>(p));
+    return make_float4(__uint_as_float(t.x << 16), __uint_as_float(t.x & 0xFFFF0000u), __uint_as_float(t.y << 16),
+                       __uint_as_float(t.y & 0xFFFF0000u));
+}
+__device__ __forceinline__ float4 ldg_p4(const __half* p)
+{
+    const uint2 t = __ldg(reinterpret_cast<const uint2*>(p));
+    const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&t.x));
+    const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&t.y));
+    return make_float4(a.x, a.y, b.x, b.y);
 }
 // One parameter as fp32.
 __device__ __forceinline__ float param1(const float* p, int64_t j) { return __ldg(p + j); }

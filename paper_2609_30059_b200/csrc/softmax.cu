@@ -21,9 +21,9 @@ namespace {
 // kFull: the row is exactly L * VPL vectors (no tail predicates); kBias: bias != NULL. L: lanes per row (32, or
 // 2 .. 16 for rows of fewer than 32 vectors, 32 / L rows per warp: attention scores and class logits of 64 to
 // 256 columns would leave most of a warp idle otherwise).
-template <typename T, int VPL, bool kFull, bool kBias, int L = 32>
+template <typename T, typename PT, int VPL, bool kFull, bool kBias, int L = 32>
 __global__ void __launch_bounds__(256)
-softmax_warp_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* __restrict__ y,
+softmax_warp_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __restrict__ y,
                     int64_t rows, int nvec, int64_t x_stride, int64_t y_stride, float scale)
 {
     constexpr int E = Elem<T>::kPerVec;
@@ -54,7 +54,7 @@ softmax_warp_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* 
 #pragma unroll
         for (int q = 0; q < E / 4; ++q) {
             float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (kBias && (kFull || v < nvec)) b = ldg_f4(bias + (int64_t)v * E + 4 * q);
+            if (kBias && (kFull || v < nvec)) b = ldg_p4(bias + (int64_t)v * E + 4 * q);
             const float bb[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -100,9 +100,9 @@ __device__ __forceinline__ int64_t last_visible(const SmOpts& o, int64_t row)
     return o.period > 0 ? (row % o.period) + (o.cols - o.period) : o.cols - 1;
 }
 
-template <typename T, int VPT, bool kOpts>
+template <typename T, typename PT, int VPT, bool kOpts>
 __global__ void __launch_bounds__(max_threads_for(VPT * Elem<T>::kPerVec))
-softmax_block_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* __restrict__ y,
+softmax_block_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __restrict__ y,
                      int nvec, int64_t x_stride, int64_t y_stride, float scale, SmOpts opts)
 {
     constexpr int E = Elem<T>::kPerVec;
@@ -129,7 +129,7 @@ softmax_block_kernel(const T* __restrict__ x, const float* __restrict__ bias, T*
 #pragma unroll
         for (int q = 0; q < E / 4; ++q) {
             float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (bias != nullptr && v < nvec) b = ldg_f4(bias + (int64_t)v * E + 4 * q);
+            if (bias != nullptr && v < nvec) b = ldg_p4(bias + (int64_t)v * E + 4 * q);
             const float bb[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -169,9 +169,9 @@ softmax_block_kernel(const T* __restrict__ x, const float* __restrict__ bias, T*
 // Sweep 1 reads the row once and keeps a running (maximum, sum) per thread, rescaled once per batch of U
 // vectors; sweep 2 walks the row backwards (the end of the row is what the first sweep left in L2) and writes
 // the result. HBM sees the row about once each way while the rows in flight fit the L2.
-template <typename T, bool kOpts, bool kBias>
+template <typename T, typename PT, bool kOpts, bool kBias>
 __global__ void __launch_bounds__(512)
-softmax_twosweep_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* __restrict__ y, int nvec,
+softmax_twosweep_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __restrict__ y, int nvec,
                         int64_t x_stride, int64_t y_stride, float scale, SmOpts opts)
 {
     constexpr int E = Elem<T>::kPerVec, U = 4;
@@ -192,7 +192,7 @@ softmax_twosweep_kernel(const T* __restrict__ x, const float* __restrict__ bias,
 #pragma unroll
         for (int q = 0; q < E / 4; ++q) {
             float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (kBias) b = ldg_f4(bias + (int64_t)v * E + 4 * q);
+            if (kBias) b = ldg_p4(bias + (int64_t)v * E + 4 * q);
             const float bb[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -266,9 +266,9 @@ softmax_twosweep_kernel(const T* __restrict__ x, const float* __restrict__ bias,
 }
 
 // ---- any length, any alignment: scalar loads, three sweeps over the row ----------------------------
-template <typename T, bool kOpts>
+template <typename T, typename PT, bool kOpts>
 __global__ void __launch_bounds__(256)
-softmax_generic_kernel(const T* __restrict__ x, const float* __restrict__ bias, T* __restrict__ y,
+softmax_generic_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __restrict__ y,
                        int64_t cols, int64_t x_stride, int64_t y_stride, float scale, SmOpts opts)
 {
     __shared__ float red_a[32], red_b[32];
@@ -280,13 +280,13 @@ softmax_generic_kernel(const T* __restrict__ x, const float* __restrict__ bias, 
     const float s2 = scale * kLog2e;
     float m = -INFINITY;
     for (int64_t j = threadIdx.x; j < cols; j += blockDim.x) {
-        const float b = bias != nullptr ? __ldg(bias + j) * kLog2e : 0.0f;
+        const float b = bias != nullptr ? param1(bias, j) * kLog2e : 0.0f;
         if (j <= last) m = fmaxf(m, fmaf(Elem<T>::load1(xr + j), s2, b));
     }
     m = block_max(m, red_a);
     float s = 0.0f;
     for (int64_t j = threadIdx.x; j < cols; j += blockDim.x) {
-        const float b = bias != nullptr ? __ldg(bias + j) * kLog2e : 0.0f;
+        const float b = bias != nullptr ? param1(bias, j) * kLog2e : 0.0f;
         if (j <= last) s += ex2_approx(fmaf(Elem<T>::load1(xr + j), s2, b) - m);
     }
     s = block_sum(s, red_b);
@@ -294,18 +294,19 @@ softmax_generic_kernel(const T* __restrict__ x, const float* __restrict__ bias, 
     const float lg = lg2_approx(s);
     // The last sweep reads x[j] and writes y[j] in the same thread, so exact aliasing stays safe.
     for (int64_t j = threadIdx.x; j < cols; j += blockDim.x) {
-        const float b = bias != nullptr ? __ldg(bias + j) * kLog2e : 0.0f;
+        const float b = bias != nullptr ? param1(bias, j) * kLog2e : 0.0f;
         const float d = j <= last ? fmaf(Elem<T>::load1(xr + j), s2, b) - m : -INFINITY;
         Elem<T>::store1(yr + j, log_out ? (d - lg) * kLn2 : ex2_approx(d) * inv);
     }
 }
 
-template <typename T>
-kop_status_t launch_softmax(const void* xv, const float* bias, void* yv, int64_t rows, int64_t cols,
+template <typename T, typename PT>
+kop_status_t launch_softmax(const void* xv, const void* biasv, void* yv, int64_t rows, int64_t cols,
                             int64_t xs, int64_t ys, float scale, cudaStream_t stream, bool with_opts = false,
                             SmOpts opts = SmOpts{0, 0, 0})
 {
     const T* x = static_cast<const T*>(xv);
+    const PT* bias = static_cast<const PT*>(biasv);
     T* y = static_cast<T*>(yv);
     constexpr int E = Elem<T>::kPerVec;
     const bool vec = vec_ok(x, cols, xs, sizeof(T)) && vec_ok(y, cols, ys, sizeof(T)) &&
@@ -319,7 +320,7 @@ kop_status_t launch_softmax(const void* xv, const float* bias, void* yv, int64_t
         if (ctas > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
         const unsigned grid = (unsigned)ctas;
         const bool full = nvec == lanes * 4;
-#define KOP_SM_GROUP_L(F, B, L) softmax_warp_kernel<T, 4, F, B, L><<<grid, 256, 0, stream>>>(x, bias, y, rows, nvec, xs, ys, scale)
+#define KOP_SM_GROUP_L(F, B, L) softmax_warp_kernel<T, PT, 4, F, B, L><<<grid, 256, 0, stream>>>(x, bias, y, rows, nvec, xs, ys, scale)
 #define KOP_SM_GROUP(L)                                                         \
     do {                                                                        \
         if (full && bias != nullptr) KOP_SM_GROUP_L(true, true, L);             \
@@ -343,7 +344,7 @@ kop_status_t launch_softmax(const void* xv, const float* bias, void* yv, int64_t
         const unsigned grid = (unsigned)ctas;
         const int vp = vpl <= 1 ? 1 : (vpl <= 2 ? 2 : 4);
         const bool full = nvec == 32 * vp;
-#define KOP_SM_WARP_L(V, F, B) softmax_warp_kernel<T, V, F, B><<<grid, threads, 0, stream>>>(x, bias, y, rows, nvec, xs, ys, scale)
+#define KOP_SM_WARP_L(V, F, B) softmax_warp_kernel<T, PT, V, F, B><<<grid, threads, 0, stream>>>(x, bias, y, rows, nvec, xs, ys, scale)
 #define KOP_SM_WARP(V)                                                         \
     do {                                                                       \
         if (full && bias != nullptr) KOP_SM_WARP_L(V, true, true);             \
@@ -371,8 +372,8 @@ kop_status_t launch_softmax(const void* xv, const float* bias, void* yv, int64_t
         const int threads = ((nvec + vpt - 1) / vpt + 31) / 32 * 32;
 #define KOP_SM_BLOCK(V)                                                                                              \
     do {                                                                                                             \
-        if (with_opts) softmax_block_kernel<T, V, true><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, nvec, xs, ys, scale, opts); \
-        else softmax_block_kernel<T, V, false><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, nvec, xs, ys, scale, opts);          \
+        if (with_opts) softmax_block_kernel<T, PT, V, true><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, nvec, xs, ys, scale, opts); \
+        else softmax_block_kernel<T, PT, V, false><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, nvec, xs, ys, scale, opts);          \
     } while (0)
         switch (vpt * E) {
         case 16: KOP_SM_BLOCK(16 / E); break;
@@ -385,15 +386,47 @@ kop_status_t launch_softmax(const void* xv, const float* bias, void* yv, int64_t
     if (vec && nvec64 <= 0x7FFFFFFF) {
         const int nvec = (int)nvec64;
         const int threads = 512;
-#define KOP_SM_TWO(O, B) softmax_twosweep_kernel<T, O, B><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, nvec, xs, ys, scale, opts)
+#define KOP_SM_TWO(O, B) softmax_twosweep_kernel<T, PT, O, B><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, nvec, xs, ys, scale, opts)
         if (with_opts) { if (bias != nullptr) KOP_SM_TWO(true, true); else KOP_SM_TWO(true, false); }
         else { if (bias != nullptr) KOP_SM_TWO(false, true); else KOP_SM_TWO(false, false); }
 #undef KOP_SM_TWO
         return launch_status();
     }
-    if (with_opts) softmax_generic_kernel<T, true><<<(unsigned)rows, 256, 0, stream>>>(x, bias, y, cols, xs, ys, scale, opts);
-    else softmax_generic_kernel<T, false><<<(unsigned)rows, 256, 0, stream>>>(x, bias, y, cols, xs, ys, scale, opts);
+    if (with_opts) softmax_generic_kernel<T, PT, true><<<(unsigned)rows, 256, 0, stream>>>(x, bias, y, cols, xs, ys, scale, opts);
+    else softmax_generic_kernel<T, PT, false><<<(unsigned)rows, 256, 0, stream>>>(x, bias, y, cols, xs, ys, scale, opts);
     return launch_status();
+}
+
+}  // namespace
+}  // namespace kop
+
+namespace kop {
+namespace {
+
+// One validation and dispatch routine for the three softmax entry points. with_opts selects the kernels that carry
+// the log-output / causal options (kop_softmax_scale_bias never pays for them).
+kop_status_t softmax_entry(const void* x, const void* bias, void* y, int64_t rows, int64_t cols, int64_t x_row_stride,
+                           int64_t y_row_stride, float scale, bool with_opts, int log_output, int64_t causal_period,
+                           kop_dtype_t dtype, kop_dtype_t pdtype, kop_stream_t stream)
+{
+    if (!param_dtype_ok(dtype, pdtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    kop_status_t st = check_rows_cols(rows, cols);
+    if (st != KOP_OK) return st;
+    if (with_opts && (causal_period < 0 || causal_period > cols)) return KOP_ERR_BAD_SHAPE;
+    if (rows == 0) return KOP_OK;                       // empty: nothing to validate further or launch
+    if (x == nullptr || y == nullptr) return KOP_ERR_NULL_POINTER;
+    if ((st = check_row_stride(x_row_stride, cols, rows)) != KOP_OK) return st;
+    if ((st = check_row_stride(y_row_stride, cols, rows)) != KOP_OK) return st;
+    const int esz = elem_size(dtype);
+    if (!aligned_to(x, esz) || !aligned_to(y, esz) || (bias != nullptr && !aligned_to(bias, elem_size(pdtype))))
+        return KOP_ERR_MISALIGNED;
+    if (!alias_ok(x, x_row_stride, y, y_row_stride, rows, cols, esz, true)) return KOP_ERR_BAD_ALIAS;
+    if ((st = check_device()) != KOP_OK) return st;
+    cudaStream_t s = as_stream(stream);
+    const SmOpts opts{log_output != 0, causal_period, cols};
+#define KOP_SM_GO(T, PT) launch_softmax<T, PT>(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale, s, with_opts, opts)
+    return KOP_DISPATCH_TYPES(dtype, pdtype, KOP_SM_GO);
+#undef KOP_SM_GO
 }
 
 }  // namespace
@@ -404,48 +437,23 @@ extern "C" kop_status_t kop_softmax_scale_bias(const void* x, const float* bias,
                                                int64_t y_row_stride, float scale,
                                                kop_dtype_t dtype, kop_stream_t stream)
 {
-    using namespace kop;
-    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
-    kop_status_t st = check_rows_cols(rows, cols);
-    if (st != KOP_OK) return st;
-    if (rows == 0) return KOP_OK;                       // empty: nothing to validate further or launch
-    if (x == nullptr || y == nullptr) return KOP_ERR_NULL_POINTER;
-    if ((st = check_row_stride(x_row_stride, cols, rows)) != KOP_OK) return st;
-    if ((st = check_row_stride(y_row_stride, cols, rows)) != KOP_OK) return st;
-    const int esz = elem_size(dtype);
-    if (!aligned_to(x, esz) || !aligned_to(y, esz) || (bias != nullptr && !aligned_to(bias, 4)))
-        return KOP_ERR_MISALIGNED;
-    if (!alias_ok(x, x_row_stride, y, y_row_stride, rows, cols, esz, true)) return KOP_ERR_BAD_ALIAS;
-    if ((st = check_device()) != KOP_OK) return st;
-    cudaStream_t s = as_stream(stream);
-    return dtype == KOP_F32
-               ? launch_softmax<float>(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale, s)
-               : dtype == KOP_BF16 ? launch_softmax<__nv_bfloat16>(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale, s)
-               : launch_softmax<__half>(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale, s);
+    return kop::softmax_entry(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale, false, 0, 0, dtype, KOP_F32, stream);
 }
 
 extern "C" kop_status_t kop_softmax_opts(const void* x, const float* bias, void* y, int64_t rows, int64_t cols,
                                          int64_t x_row_stride, int64_t y_row_stride, float scale, int log_output,
                                          int64_t causal_period, kop_dtype_t dtype, kop_stream_t stream)
 {
-    using namespace kop;
-    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
-    kop_status_t st = check_rows_cols(rows, cols);
-    if (st != KOP_OK) return st;
-    if (causal_period < 0 || causal_period > cols) return KOP_ERR_BAD_SHAPE;
-    if (rows == 0) return KOP_OK;
-    if (x == nullptr || y == nullptr) return KOP_ERR_NULL_POINTER;
-    if ((st = check_row_stride(x_row_stride, cols, rows)) != KOP_OK) return st;
-    if ((st = check_row_stride(y_row_stride, cols, rows)) != KOP_OK) return st;
-    const int esz = elem_size(dtype);
-    if (!aligned_to(x, esz) || !aligned_to(y, esz) || (bias != nullptr && !aligned_to(bias, 4)))
-        return KOP_ERR_MISALIGNED;
-    if (!alias_ok(x, x_row_stride, y, y_row_stride, rows, cols, esz, true)) return KOP_ERR_BAD_ALIAS;
-    if ((st = check_device()) != KOP_OK) return st;
-    cudaStream_t s = as_stream(stream);
-    const SmOpts opts{log_output != 0, causal_period, cols};
-    return dtype == KOP_F32
-               ? launch_softmax<float>(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale, s, true, opts)
-               : dtype == KOP_BF16 ? launch_softmax<__nv_bfloat16>(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale, s, true, opts)
-               : launch_softmax<__half>(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale, s, true, opts);
+    return kop::softmax_entry(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale, true, log_output, causal_period,
+                              dtype, KOP_F32, stream);
+}
+
+extern "C" kop_status_t kop_softmax_ex(const void* x, const void* bias, void* y, int64_t rows, int64_t cols,
+                                       int64_t x_row_stride, int64_t y_row_stride, float scale, int log_output,
+                                       int64_t causal_period, kop_dtype_t dtype, kop_dtype_t param_dtype,
+                                       kop_stream_t stream)
+{
+    // no options asked for: the kernels of kop_softmax_scale_bias
+    return kop::softmax_entry(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale,
+                              log_output != 0 || causal_period != 0, log_output, causal_period, dtype, param_dtype, stream);
 }

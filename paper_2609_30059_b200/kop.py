@@ -109,6 +109,16 @@ def lib() -> C.CDLL:
     L.kop_rmsnorm_swiglu_residual_workspace_bytes.argtypes = [i64, i64, i64, i32]
     L.kop_mlp_handle_create.argtypes = [C.POINTER(vp)]
     L.kop_mlp_handle_destroy.argtypes = [vp]
+    L.kop_softmax_ex.argtypes = [vp, vp, vp, i64, i64, i64, i64, f32, i32, i64, i32, i32, vp]
+    L.kop_softmax_ex.restype = i32
+    L.kop_bn_relu_avgpool_ex.argtypes = [vp] * 5 + [i64] * 4 + [C.POINTER(i64), C.POINTER(i64), i32, i32, vp]
+    L.kop_bn_relu_avgpool_ex.restype = i32
+    L.kop_groupnorm_act_ex.argtypes = [vp] * 6 + [i64] * 5 + [f32, i32, i32, i32, vp]
+    L.kop_groupnorm_act_ex.restype = i32
+    L.kop_bias_act_ex.argtypes = [vp, vp, vp, i64, i64, i64, i64, i32, f32, i32, i32, vp]
+    L.kop_bias_act_ex.restype = i32
+    L.kop_epilogue_chain_ex.argtypes = [vp, vp, vp, vp] + [i64] * 5 + [f32] * 4 + [i32, f32, i32, i32, vp]
+    L.kop_epilogue_chain_ex.restype = i32
     L.kop_mlp_handle_wrap.argtypes = [vp, C.POINTER(vp)]
     L.kop_mlp_handle_wrap.restype = i32
     L.kop_mlp_handle_set_residual_in_gemm.argtypes = [vp, i32]
@@ -309,6 +319,99 @@ def _param_any(t, name: str, n: int, data):
     if t.dtype not in (torch.float32, data.dtype) or not t.is_cuda or not t.is_contiguous() or t.numel() != n:
         raise ValueError(f"{name}: expected a contiguous CUDA vector of {n} fp32 or {data.dtype} elements")
     return t.data_ptr(), (KOP_F32 if t.dtype == torch.float32 else _dtype_tag(data))
+
+
+def _params_any(data, n, **named):
+    """Optional parameter vectors that must share one type (fp32 or the data type). Returns (pointers, dtype tag)."""
+    tag, ptrs = None, []
+    for name, t in named.items():
+        if t is None:
+            ptrs.append(None)
+            continue
+        ptr, tg = _param_any(t, name, n, data)
+        if tag is not None and tg != tag:
+            raise ValueError("parameter vectors must share one dtype: " + ", ".join(named))
+        tag = tg
+        ptrs.append(ptr)
+    return ptrs, (KOP_F32 if tag is None else tag)
+
+
+def kop_softmax_ex(x, bias, scale, log_output=False, causal_period=0, out=None, stream=None):
+    """kop_softmax_scale_bias / kop_softmax_opts with the bias in fp32 or in x.dtype."""
+    rows, cols, xs = _rows2d(x, "x")
+    out = torch.empty_like(x) if out is None else out
+    _, _, ys = _rows2d(out, "out")
+    assert out.shape == x.shape and out.dtype == x.dtype
+    (bp,), ptag = _params_any(x, cols, bias=bias)
+    _check(lib().kop_softmax_ex(x.data_ptr(), bp, out.data_ptr(), rows, cols, xs, ys, float(scale),
+                                int(bool(log_output)), int(causal_period), _dtype_tag(x), ptag, _stream(stream)),
+           "kop_softmax_ex")
+    return out
+
+
+def kop_bn_relu_avgpool_ex(x, scale, shift, out=None, pooled=None, stream=None):
+    """kop_bn_relu_avgpool with scale / shift in fp32 or in x.dtype (both the same)."""
+    if x.dim() != 4 or not x.is_cuda:
+        raise ValueError("x: expected a 4-D NCHW CUDA tensor")
+    N, Cc, H, W = x.shape
+    out = torch.empty_like(x) if out is None else out
+    pooled = torch.empty((N, Cc), dtype=torch.float32, device=x.device) if pooled is None else pooled
+    xs = (C.c_int64 * 4)(*x.stride())
+    ys = (C.c_int64 * 4)(*out.stride())
+    (sp, hp), ptag = _params_any(x, Cc, scale=scale, shift=shift)
+    _check(lib().kop_bn_relu_avgpool_ex(x.data_ptr(), sp, hp, out.data_ptr(), pooled.data_ptr(), N, Cc, H, W, xs, ys,
+                                        _dtype_tag(x), ptag, _stream(stream)), "kop_bn_relu_avgpool_ex")
+    return out, pooled
+
+
+def kop_groupnorm_act_ex(x, gamma, beta, groups, eps, act=0, out=None, mean=None, rstd=None, want_stats=True,
+                         stream=None):
+    """kop_groupnorm_act with gamma / beta in fp32 or in x.dtype (both the same; each may be None)."""
+    if x.dim() != 4 or not x.is_cuda or not x.is_contiguous():
+        raise ValueError("x: expected a contiguous 4-D NCHW CUDA tensor")
+    N, Cc, H, W = x.shape
+    out = torch.empty_like(x) if out is None else out
+    if out.shape != x.shape or out.dtype != x.dtype or not out.is_contiguous():
+        raise ValueError("out: expected a contiguous tensor of x's shape and dtype")
+    if want_stats:
+        mean = torch.empty((N, groups), dtype=torch.float32, device=x.device) if mean is None else mean
+        rstd = torch.empty((N, groups), dtype=torch.float32, device=x.device) if rstd is None else rstd
+    (gp, bp), ptag = _params_any(x, Cc, gamma=gamma, beta=beta)
+    _check(lib().kop_groupnorm_act_ex(x.data_ptr(), gp, bp, out.data_ptr(), None if mean is None else mean.data_ptr(),
+                                      None if rstd is None else rstd.data_ptr(), N, Cc, H, W, int(groups), float(eps),
+                                      int(act), _dtype_tag(x), ptag, _stream(stream)), "kop_groupnorm_act_ex")
+    return out, mean, rstd
+
+
+def kop_bias_act_ex(x, bias, act, alpha=0.01, out=None, stream=None):
+    """kop_bias_act with the bias in fp32 or in x.dtype."""
+    rows, cols, xs = _rows2d(x, "x")
+    out = torch.empty_like(x) if out is None else out
+    _, _, ys = _rows2d(out, "out")
+    assert out.shape == x.shape and out.dtype == x.dtype
+    (bp,), ptag = _params_any(x, cols, bias=bias)
+    _check(lib().kop_bias_act_ex(x.data_ptr(), bp, out.data_ptr(), rows, cols, xs, ys, ACTS[act], float(alpha),
+                                 _dtype_tag(x), ptag, _stream(stream)), "kop_bias_act_ex")
+    return out
+
+
+def kop_epilogue_chain_ex(x, bias, residual, scale=1.0, residual_scale=1.0, lo=float("-inf"), hi=float("inf"),
+                          act="identity", alpha=0.01, out=None, stream=None):
+    """kop_epilogue_chain with the bias in fp32 or in x.dtype."""
+    rows, cols, xs = _rows2d(x, "x")
+    rs = cols
+    if residual is not None:
+        _, _, rs = _rows2d(residual, "residual")
+        assert residual.shape == x.shape and residual.dtype == x.dtype
+    out = torch.empty_like(x) if out is None else out
+    _, _, ys = _rows2d(out, "out")
+    assert out.shape == x.shape and out.dtype == x.dtype
+    (bp,), ptag = _params_any(x, cols, bias=bias)
+    _check(lib().kop_epilogue_chain_ex(x.data_ptr(), bp, None if residual is None else residual.data_ptr(),
+                                       out.data_ptr(), rows, cols, xs, rs, ys, float(scale), float(residual_scale),
+                                       float(lo), float(hi), ACTS[act], float(alpha), _dtype_tag(x), ptag,
+                                       _stream(stream)), "kop_epilogue_chain_ex")
+    return out
 
 
 def kop_layernorm_ex(x, residual, bias, gamma, beta, eps, prologue="bias_gelu_residual", out=None, mean=None,

@@ -114,3 +114,115 @@ def test_layernorm_ex_benchmark_shape_sampled_rows(kop):
     idx = torch.tensor(sorted({0, 1, rows - 2, rows - 1} | set(np.random.default_rng(1).integers(0, rows, 60).tolist()))).cuda()
     ref, _, _ = ln_oracle("bias_gelu_residual", x[idx], r[idx], *p, cfg["eps"])
     assert_close(y[idx], ref, tol_of(dtype), "full-size sampled rows, 16-bit parameters")
+
+
+# ------------------------------------------------------------------ the other entry points with 16-bit parameters
+
+# vector kernels (lanes per row, warp per row, CTA per row, two sweeps), ragged and odd lengths (scalar kernel)
+@pytest.mark.parametrize("rows,cols,dtype", [(700, 64, BF16), (333, 512, F16), (129, 4096, BF16), (5, 40000, BF16),
+                                             (33, 777, F16), (9, 1000, BF16)])
+@pytest.mark.parametrize("seed", SEEDS)
+def test_softmax_ex_16_bit_bias(kop, rows, cols, dtype, seed):
+    x, bias = synth.softmax_inputs(rows, cols, dtype, seed, "cuda")
+    b16 = bias.to(dtype)
+    tol = tol_of(dtype)
+    y = Guarded((rows, cols), dtype)
+    kop.kop_softmax_ex(x, b16, 0.125, out=y.t)
+    assert_close(y.t, kopref.softmax_scale_bias(host(x), host(b16), 0.125, threads=None), tol, "softmax_ex")
+    y.check("softmax_ex")
+    for log_out, period in ((True, 0), (False, cols), (True, max(1, cols // 2))):
+        got = kop.kop_softmax_ex(x, b16, 0.5, log_out, period).cpu().double().numpy()
+        ref = kopref.softmax_opts(host(x), host(b16), 0.5, log_out, period, threads=None)
+        fin = np.isfinite(ref)
+        assert np.array_equal(np.isneginf(got), np.isneginf(ref))
+        assert np.all(np.abs(got[fin] - ref[fin]) <= tol * np.maximum(1.0, np.abs(ref[fin]))), (log_out, period)
+    # fp32 bias through the same entry point: bit for bit what the fixed-type entry points give; no bias at all
+    assert torch.equal(kop.kop_softmax_ex(x, bias, 0.125), kop.kop_softmax_scale_bias(x, bias, 0.125))
+    assert torch.equal(kop.kop_softmax_ex(x, bias, 0.125, True, cols), kop.kop_softmax_opts(x, bias, 0.125, True, cols))
+    assert torch.equal(kop.kop_softmax_ex(x, None, 0.125), kop.kop_softmax_scale_bias(x, None, 0.125))
+
+
+@pytest.mark.parametrize("shape,dtype", [((3, 40, 56, 56), BF16), ((2, 24, 7, 7), F16), ((5, 16, 14, 14), BF16),
+                                         ((2, 9, 5, 3), F16), ((2, 64, 28, 28), BF16)])
+@pytest.mark.parametrize("seed", SEEDS)
+def test_bn_relu_avgpool_ex_16_bit_scale_shift(kop, shape, dtype, seed):
+    x, sc, sh = synth.bn_pool_inputs(*shape, dtype, seed, "cuda")
+    sc16, sh16 = sc.to(dtype), sh.to(dtype)
+    tol = tol_of(dtype)
+    ry, rp = kopref.bn_relu_avgpool(host(x), host(sc16), host(sh16), threads=None)
+    y, p = kop.kop_bn_relu_avgpool_ex(x, sc16, sh16)
+    assert_close(y, ry, tol, "bn_ex y")
+    assert_close(p, rp, 1e-5, "bn_ex pooled")
+    xl = x.contiguous(memory_format=torch.channels_last)
+    yl, pl = kop.kop_bn_relu_avgpool_ex(xl, sc16, sh16)
+    assert_close(yl, ry, tol, "bn_ex channels-last y")
+    assert_close(pl, rp, 1e-5, "bn_ex channels-last pooled")
+    a = kop.kop_bn_relu_avgpool_ex(x, sc, sh)
+    b = kop.kop_bn_relu_avgpool(x, sc, sh)
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+
+
+@pytest.mark.parametrize("shape,groups,dtype", [((3, 32, 28, 28), 8, BF16), ((2, 16, 56, 56), 16, F16), ((4, 12, 7, 7), 4, BF16),
+                                                ((2, 6, 5, 3), 2, F16), ((1, 8, 112, 112), 1, BF16)])
+@pytest.mark.parametrize("seed", SEEDS)
+def test_groupnorm_act_ex_16_bit_gamma_beta(kop, shape, groups, dtype, seed):
+    x, g, b = synth.groupnorm_inputs(*shape, dtype, seed, "cuda")
+    g16, b16 = g.to(dtype), b.to(dtype)
+    tol = tol_of(dtype)
+    for act in (0, 1, 2):
+        y, mu, rs = kop.kop_groupnorm_act_ex(x, g16, b16, groups, 1e-5, act)
+        ry, rm, rr = kopref.groupnorm_act(host(x), host(g16), host(b16), groups, 1e-5, act, threads=None)
+        assert_close(y, ry, tol, f"groupnorm_ex act={act}")
+        assert_close(mu, rm, 1e-3, "groupnorm_ex mean")
+        assert_close(rs, rr, 1e-3, "groupnorm_ex rstd")
+    y, _, _ = kop.kop_groupnorm_act_ex(x, g16, None, groups, 1e-5, 0)        # gamma only
+    assert_close(y, kopref.groupnorm_act(host(x), host(g16), None, groups, 1e-5, 0, threads=None)[0], tol, "gamma only")
+    a = kop.kop_groupnorm_act_ex(x, g, b, groups, 1e-5, 2)
+    c = kop.kop_groupnorm_act(x, g, b, groups, 1e-5, 2)
+    assert torch.equal(a[0], c[0]) and torch.equal(a[1], c[1]) and torch.equal(a[2], c[2])
+    assert kop.kop_groupnorm_wait_timeouts() == 0
+
+
+@pytest.mark.parametrize("rows,cols,dtype", [(300, 4096, BF16), (2000, 64, F16), (65, 1000, BF16), (17, 1001, F16)])
+@pytest.mark.parametrize("seed", SEEDS)
+def test_bias_act_and_chain_ex_16_bit_bias(kop, rows, cols, dtype, seed):
+    x, bias = synth.softmax_inputs(rows, cols, dtype, seed, "cuda")
+    r, _ = synth.softmax_inputs(rows, cols, dtype, seed + 7, "cuda")
+    b16 = bias.to(dtype)
+    tol = tol_of(dtype)
+    for act in ("gelu_tanh", "silu", "relu", "mish"):
+        y = Guarded((rows, cols), dtype)
+        kop.kop_bias_act_ex(x, b16, act, out=y.t)
+        assert_close(y.t, kopref.bias_act(host(x), host(b16), act, threads=None), tol, f"bias_act_ex {act}")
+        y.check("bias_act_ex")
+    y = kop.kop_epilogue_chain_ex(x, b16, r, 0.5, 2.0, -1.0, 1.5, "silu")
+    assert_close(y, kopref.epilogue_chain(host(x), host(b16), host(r), 0.5, 2.0, -1.0, 1.5, "silu", threads=None), tol, "chain_ex")
+    y = kop.kop_epilogue_chain_ex(x, b16, None, 1.25, 1.0, act="gelu_erf")
+    assert_close(y, kopref.epilogue_chain(host(x), host(b16), None, 1.25, 1.0, act="gelu_erf", threads=None), tol, "chain_ex no residual")
+    assert torch.equal(kop.kop_bias_act_ex(x, bias, "gelu_tanh"), kop.kop_bias_act(x, bias, "gelu_tanh"))
+    assert torch.equal(kop.kop_epilogue_chain_ex(x, bias, r, 0.5, 2.0, -1.0, 1.5, "silu"),
+                       kop.kop_epilogue_chain(x, bias, r, 0.5, 2.0, -1.0, 1.5, "silu"))
+    assert torch.equal(kop.kop_bias_act_ex(x, None, "relu"), kop.kop_bias_act(x, None, "relu"))
+
+
+def test_ex_entry_points_misaligned_parameters_and_type_rules(kop):
+    rows, cols = 40, 2048
+    x, bias = synth.softmax_inputs(rows, cols, BF16, 2, "cuda")
+    b16 = bias.to(BF16)
+    buf = torch.zeros(cols + 1, dtype=BF16, device="cuda")
+    buf[1:] = b16                                             # 2-byte aligned only: the scalar-load kernels
+    ref = kopref.softmax_scale_bias(host(x), host(b16), 1.0)
+    assert_close(kop.kop_softmax_ex(x, buf[1:], 1.0), ref, 2e-2, "misaligned 16-bit softmax bias")
+    assert_close(kop.kop_bias_act_ex(x, buf[1:], "silu"), kopref.bias_act(host(x), host(b16), "silu"), 2e-2, "misaligned bias")
+    # 16-bit parameters go with 16-bit data of the same type only
+    xf = x.float()
+    for call in (lambda: kop.kop_softmax_ex(xf, b16, 1.0), lambda: kop.kop_bias_act_ex(x, bias.half(), "relu")):
+        with pytest.raises(Exception):
+            call()
+    L = kop.lib()
+    P, Q, R = 0x10000, 0x20000, 0x30000
+    assert L.kop_softmax_ex(P, Q, R, 4, 8, 8, 8, 1.0, 0, 0, 0, 1, None) == 4          # fp32 data, bf16 params
+    assert L.kop_softmax_ex(P, Q, R, 4, 8, 8, 8, 1.0, 0, 0, 1, 2, None) == 4          # bf16 data, fp16 params
+    assert L.kop_bias_act_ex(P, Q, R, 4, 8, 8, 8, 1, 0.0, 2, 1, None) == 4
+    assert L.kop_epilogue_chain_ex(P, Q, None, R, 4, 8, 8, 8, 8, 1.0, 1.0, -1.0, 1.0, 0, 0.0, 1, 7, None) == 4
+    assert L.kop_softmax_ex(P, Q + 1, R, 4, 8, 8, 8, 1.0, 0, 0, 1, 1, None) == 5      # bias not on a 2-byte boundary
