@@ -206,23 +206,47 @@ __device__ __forceinline__ void load8(const __half* p, float (&f)[8])
     Elem<__half>::unpack(ld_stream(p), f);
 }
 
+// The raw values of one row for one thread: its eight columns and, for the first / last lane of a warp, the halo
+// element that no neighbour lane holds. All loads are issued here, before anything is computed.
+template <typename T>
+struct StripRowRaw {
+    float f[8];
+    float edge;
+};
+template <typename T>
+__device__ __forceinline__ void strip_load_s1(const T* __restrict__ row, int seg, int segs, int lane, StripRowRaw<T>& r)
+{
+    load8(row, r.f);
+    r.edge = 0.0f;
+    if (lane == 0 && seg > 0) r.edge = Elem<T>::load1(row - 1);
+    if (lane == 31 && seg < segs - 1) r.edge = Elem<T>::load1(row + 8);
+}
+
+// The stride-2 kernel's loads: only a left halo exists there.
+template <typename T, int KS>
+__device__ __forceinline__ void strip_load_s2(const T* __restrict__ row, int seg, int lane, StripRowRaw<T>& r)
+{
+    load8(row, r.f);
+    r.edge = 0.0f;
+    if (KS == 3 && lane == 0 && seg > 0) r.edge = Elem<T>::load1(row - 1);
+}
+
 // Horizontal reductions of one input row for this thread's four outputs. KS == 3: windows of columns
 // (2j-1, 2j, 2j+1) relative to the thread's first column, v[0] being the halo, which is the left
 // neighbour lane's last column (a shuffle; lane 0 of a warp loads it); KS == 2: (2j, 2j+1). Rows outside
 // the image are loaded from a clamped row and overridden with padding, so the warp stays converged for
 // the shuffle. Called by all 32 lanes.
 template <typename T, int MODE, int KS>
-__device__ __forceinline__ void strip_row(const T* __restrict__ row, bool row_ok, int seg, int lane, float sc,
+__device__ __forceinline__ void strip_row(const StripRowRaw<T>& raw, bool row_ok, int seg, int lane, float sc,
                                           float sf, float relu, float (&h)[4])
 {
     const float pad = MODE == 0 ? -INFINITY : 0.0f;
-    float v[9], f[8];
-    load8(row, f);
+    float v[9];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) v[1 + e] = row_ok ? act_of(f[e], sc, sf, relu) : pad;
+    for (int e = 0; e < 8; ++e) v[1 + e] = row_ok ? act_of(raw.f[e], sc, sf, relu) : pad;
     if (KS == 3) {
         float left = __shfl_up_sync(0xFFFFFFFFu, v[8], 1);
-        if (lane == 0 && seg > 0) left = row_ok ? act_of(Elem<T>::load1(row - 1), sc, sf, relu) : pad;
+        if (lane == 0) left = row_ok ? act_of(raw.edge, sc, sf, relu) : pad;
         v[0] = seg > 0 ? left : pad;
 #pragma unroll
         for (int j = 0; j < 4; ++j) h[j] = pool_op<T, MODE>(pool_op<T, MODE>(v[2 * j], v[2 * j + 1]), v[2 * j + 2]);
@@ -259,7 +283,9 @@ __device__ __forceinline__ void store4<__half>(__half* dst, const float (&o)[4])
     *reinterpret_cast<uint2*>(dst) = w;
 }
 
-template <typename T, int MODE, int KS>
+// R: output rows per trip, all 2 R row loads issued before the first is used (R = 2 measured slower for every data
+// type: bf16 3x3 4.4 to 3.6 TB/s, 2x2 5.5 to 5.0).
+template <typename T, int MODE, int KS, int R>
 __global__ void __launch_bounds__(256)
 pool2d_strip_kernel(const T* __restrict__ x, const float* __restrict__ scale, const float* __restrict__ shift,
                     T* __restrict__ y, int64_t strips, int C, int H, int W, int OH, int OW, int segs, int bands,
@@ -285,25 +311,128 @@ pool2d_strip_kernel(const T* __restrict__ x, const float* __restrict__ scale, co
     float carry[4];
     if (KS == 3) {
         const int i = 2 * oh0 - P;
-        strip_row<T, MODE, KS>(col + (int64_t)max(i, 0) * W, i >= 0, seg, lane, sc, sf, relu, carry);
+        StripRowRaw<T> r0;
+        strip_load_s2<T, KS>(col + (int64_t)max(i, 0) * W, seg, lane, r0);
+        strip_row<T, MODE, KS>(r0, i >= 0, seg, lane, sc, sf, relu, carry);
     }
     // every lane runs band_rows trips so that the shuffles stay warp-wide; trips past a short last band are idle
-    for (int t = 0; t < band_rows; ++t, out += OW) {
-        const int oi = min(oh0 + t, OH - 1);
-        float a[4], b[4], o[4];
-        const int i1 = 2 * oi - P + (KS == 3 ? 1 : 0), i2 = i1 + 1;   // the two rows first needed by this output row
-        strip_row<T, MODE, KS>(col + (int64_t)i1 * W, true, seg, lane, sc, sf, relu, a);
-        strip_row<T, MODE, KS>(col + (int64_t)min(i2, H - 1) * W, i2 < H, seg, lane, sc, sf, relu, b);
+    for (int t = 0; t < band_rows; t += R, out += (int64_t)R * OW) {
+        StripRowRaw<T> ra[R], rb[R];                                  // all rows' loads first, then the arithmetic
+        int i2s[R];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            float r = pool_op<T, MODE>(a[j], b[j]);
-            if (KS == 3) {
-                r = pool_op<T, MODE>(carry[j], r);
-                carry[j] = b[j];
-            }
-            o[j] = MODE == 1 ? r * inv_area : r;
+        for (int k = 0; k < R; ++k) {
+            const int oi = min(oh0 + t + k, OH - 1);
+            const int i1 = 2 * oi - P + (KS == 3 ? 1 : 0);            // the two rows first needed by this output row
+            i2s[k] = i1 + 1;
+            strip_load_s2<T, KS>(col + (int64_t)i1 * W, seg, lane, ra[k]);
+            strip_load_s2<T, KS>(col + (int64_t)min(i1 + 1, H - 1) * W, seg, lane, rb[k]);
         }
-        if (live && oh0 + t < oh1) store4<T>(out, o);
+#pragma unroll
+        for (int k = 0; k < R; ++k) {
+            float a[4], b[4], o[4];
+            strip_row<T, MODE, KS>(ra[k], true, seg, lane, sc, sf, relu, a);
+            strip_row<T, MODE, KS>(rb[k], i2s[k] < H, seg, lane, sc, sf, relu, b);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                float r = pool_op<T, MODE>(a[j], b[j]);
+                if (KS == 3) {
+                    r = pool_op<T, MODE>(carry[j], r);
+                    carry[j] = b[j];
+                }
+                o[j] = MODE == 1 ? r * inv_area : r;
+            }
+            if (live && oh0 + t + k < oh1) store4<T>(out + (int64_t)k * OW, o);
+        }
+    }
+}
+
+// ---- the same strip walk for 3x3 windows at stride 1 (pad 1): eight outputs per thread and row ----------------
+// A thread owns eight columns and produces the eight outputs above them: per input row one vector load, the left
+// and right halo values from the neighbour lanes by shuffle (the first / last lane of a warp loads its own; at the
+// image edge it is padding), eight horizontal window reductions; the horizontal results of the two rows above are
+// carried in registers, so every input row is loaded once per band. No shared memory, no barrier, loads of the
+// next rows in flight while the current ones are combined.
+template <typename T, int MODE>
+__device__ __forceinline__ void strip_row_s1(const StripRowRaw<T>& raw, bool row_ok, int seg, int segs, int lane,
+                                             float sc, float sf, float relu, float (&h)[8])
+{
+    const float pad = MODE == 0 ? -INFINITY : 0.0f;
+    float v[10];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[1 + e] = row_ok ? act_of(raw.f[e], sc, sf, relu) : pad;
+    const float edge = row_ok ? act_of(raw.edge, sc, sf, relu) : pad;
+    float left = __shfl_up_sync(0xFFFFFFFFu, v[8], 1);
+    float right = __shfl_down_sync(0xFFFFFFFFu, v[1], 1);
+    if (lane == 0) left = edge;
+    if (lane == 31) right = edge;
+    v[0] = seg > 0 ? left : pad;
+    v[9] = seg < segs - 1 ? right : pad;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) h[j] = pool_op<T, MODE>(pool_op<T, MODE>(v[j], v[j + 1]), v[j + 2]);
+}
+
+template <typename T>
+__device__ __forceinline__ void store8(T* dst, const float (&o)[8])
+{
+    if constexpr (sizeof(T) == 4) {
+        const float a[4] = {o[0], o[1], o[2], o[3]}, b[4] = {o[4], o[5], o[6], o[7]};
+        st_stream(dst, Elem<float>::pack(a));
+        st_stream(dst + 4, Elem<float>::pack(b));
+    } else {
+        st_stream(dst, Elem<T>::pack(o));
+    }
+}
+
+// R: input rows loaded per trip (all R loads are issued before the first is used).
+template <typename T, int MODE, int R>
+__global__ void __launch_bounds__(256)
+pool2d_strip_s1_kernel(const T* __restrict__ x, const float* __restrict__ scale, const float* __restrict__ shift,
+                       T* __restrict__ y, int64_t strips, int C, int H, int W, int segs, int bands, int band_rows,
+                       int relu_flag, float inv_area)
+{
+    const int64_t g_raw = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const bool live = g_raw < strips;                       // surplus threads of the last CTA shadow the last strip
+    const int64_t g = live ? g_raw : strips - 1;
+    const int lane = threadIdx.x & 31;
+    const int seg = (int)(g % segs);
+    const int64_t rest = g / segs;
+    const int band = (int)(rest % bands);
+    const int64_t plane = rest / bands;
+    const int c = (int)(plane % C);
+    const float sc = scale != nullptr ? __ldg(scale + c) : 1.0f;
+    const float sf = shift != nullptr ? __ldg(shift + c) : 0.0f;
+    const float relu = relu_flag ? 0.0f : -INFINITY;
+    const int oh0 = band * band_rows, oh1 = min(H, oh0 + band_rows);      // OH == H, OW == W
+    const T* col = x + plane * H * (int64_t)W + seg * 8;
+    T* out = y + (plane * H + oh0) * (int64_t)W + seg * 8;
+
+    float up[8], mid[8];
+    {
+        StripRowRaw<T> a, b;
+        strip_load_s1<T>(col + (int64_t)max(oh0 - 1, 0) * W, seg, segs, lane, a);
+        strip_load_s1<T>(col + (int64_t)oh0 * W, seg, segs, lane, b);
+        strip_row_s1<T, MODE>(a, oh0 >= 1, seg, segs, lane, sc, sf, relu, up);
+        strip_row_s1<T, MODE>(b, true, seg, segs, lane, sc, sf, relu, mid);
+    }
+    // every lane runs the same number of trips so that the shuffles stay warp-wide; rows past the band are idle
+    for (int t = 0; t < band_rows; t += R, out += (int64_t)R * W) {
+        StripRowRaw<T> raw[R];
+#pragma unroll
+        for (int k = 0; k < R; ++k) strip_load_s1<T>(col + (int64_t)min(oh0 + t + k + 1, H - 1) * W, seg, segs, lane, raw[k]);
+#pragma unroll
+        for (int k = 0; k < R; ++k) {
+            const int i2 = oh0 + t + k + 1;
+            float low[8], o[8];
+            strip_row_s1<T, MODE>(raw[k], i2 < H, seg, segs, lane, sc, sf, relu, low);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float r = pool_op<T, MODE>(pool_op<T, MODE>(up[j], mid[j]), low[j]);
+                o[j] = MODE == 1 ? r * inv_area : r;
+                up[j] = mid[j];
+                mid[j] = low[j];
+            }
+            if (live && oh0 + t + k < oh1) store8<T>(out + (int64_t)k * W, o);
+        }
     }
 }
 
@@ -414,6 +543,225 @@ pool2d_planes_kernel(const T* __restrict__ x, const float* __restrict__ scale, c
     }
 }
 
+// ---- walk kernel: 2x2 / 3x3 windows at stride 1 or 2, any width, any alignment --------------------------------
+// What the strip kernel above does in registers for its two aligned stride-2 cases, done out of a shared-memory tile
+// for everything else with these windows: stride 1, widths that are not whole vectors, rows that do not start on a
+// 16-byte boundary, small planes. A CTA takes either a band of output rows of one plane or a run of whole small
+// planes (always a contiguous piece of memory): flat 16-byte loads (scalar head / tail where the piece does not
+// start or end on a vector), fp32 activations parked in a tile that already holds the padding, every plane's row
+// 16-byte aligned. Then each thread owns four adjacent outputs of a row and walks down the output rows: per input
+// row one or two 128-bit shared-memory loads (plus the single left-halo float when the window is padded), the
+// KS - ST rows shared by consecutive windows kept in registers, vertical combination first (one operation per
+// column), then the four horizontal windows. No index division inside the walk, about five arithmetic
+// instructions and well under one shared-memory load per output.
+template <int KS, int ST>
+struct WalkGeom {
+    static constexpr int kCols = 3 * ST + KS;          // input columns under four adjacent windows
+};
+
+// Tile geometry (host and device): image column 0 at tile column `lead`; a tile row is long enough for the
+// last group's reads (groups of four outputs, the last one possibly ragged) plus a vector of slack.
+__host__ __device__ __forceinline__ int walk_row_floats(int W, int OW, int pw, int KS, int ST)
+{
+    const int lead = pool_lead(pw), OG = (OW + 3) / 4;
+    const int need_data = lead + W + pw, need_read = lead - pw + 4 * OG * ST - ST + KS + 3;
+    return ((need_data > need_read ? need_data : need_read) + 3) / 4 * 4;
+}
+
+template <typename T, int MODE, int KS, int ST, bool kPadW>
+__global__ void __launch_bounds__(kPoolThreads)
+pool2d_walk_kernel(const T* __restrict__ x, const float* __restrict__ scale, const float* __restrict__ shift,
+                   T* __restrict__ y, int64_t planes, int np, int C, int H, int W, int OH, int OW, int ph,
+                   int band_rows, int bands, int chunks, int relu_flag, float inv_area)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    constexpr int NV = WalkGeom<KS, ST>::kCols;
+    constexpr int pw = kPadW ? 1 : 0;
+    extern __shared__ __align__(16) float tile[];
+    const float relu = relu_flag ? 0.0f : -INFINITY;
+    const float pad = MODE == 0 ? -INFINITY : 0.0f;
+    const int lead = pool_lead(pw), Ws = walk_row_floats(W, OW, pw, KS, ST);
+
+    // what this CTA owns: planes [p0, p0 + nq), output rows [oh0, oh1) of each
+    int64_t p0;
+    int nq, oh0, oh1;
+    if (np > 1) {
+        p0 = (int64_t)blockIdx.x * np;
+        nq = (int)(planes - p0 < np ? planes - p0 : np);
+        oh0 = 0;
+        oh1 = OH;
+    } else {
+        p0 = blockIdx.x / bands;
+        const int band = (int)(blockIdx.x - p0 * bands);
+        nq = 1;
+        oh0 = band * band_rows;
+        oh1 = min(OH, oh0 + band_rows);
+    }
+    const int t0 = oh0 * ST - ph;                            // first tile row in image coordinates (may be < 0)
+    const int trows = (oh1 - 1 - oh0) * ST + KS;
+    const int i0 = max(t0, 0), i1 = min(t0 + trows, H);      // image rows present
+    const int top = i0 - t0, nrows = i1 - i0;
+    const int PS = ((np > 1 ? (OH - 1) * ST + KS : (band_rows - 1) * ST + KS)) * Ws;      // floats per plane in the tile
+    float* sc_s = tile + np * PS;                            // per-plane scale / shift behind the tiles
+    float* sf_s = sc_s + np;
+    for (int q = threadIdx.x; q < nq; q += kPoolThreads) {
+        const int c = (int)((p0 + q) % C);
+        sc_s[q] = scale != nullptr ? __ldg(scale + c) : 1.0f;
+        sf_s[q] = shift != nullptr ? __ldg(shift + c) : 0.0f;
+    }
+    // 1. padding cells: rows above / below the image, then the pw cells left and right of the image rows
+    {
+        const int bottom = trows - top - nrows;
+        const int per_plane = (top + bottom) * Ws;
+        for (int k = threadIdx.x; k < nq * per_plane; k += kPoolThreads) {
+            const int q = k / per_plane, m = k - q * per_plane;
+            tile[q * PS + (m < top * Ws ? m : m + nrows * Ws)] = pad;
+        }
+        if (kPadW) {
+            for (int k = threadIdx.x; k < nq * nrows * 2; k += kPoolThreads) {
+                const int q = k / (nrows * 2), m = k - q * nrows * 2;
+                const int r = m >> 1;
+                tile[q * PS + (top + r) * Ws + ((m & 1) ? lead + W : lead - 1)] = pad;
+            }
+        }
+    }
+    __syncthreads();                                         // scale / shift visible
+    // 2. the input: one contiguous piece of nq * nrows * W elements (nq > 1 only with whole planes: nrows == H)
+    {
+        const T* xp = x + (p0 * H + i0) * (int64_t)W;
+        const int n_in = nq * nrows * W;
+        const int plane_in = nrows * W;
+        const float inv_w = 1.0f / (float)W, inv_plane = 1.0f / (float)plane_in;
+        const int head_raw = (int)(((16 - (reinterpret_cast<uintptr_t>(xp) & 15)) & 15) / sizeof(T));
+        const int head = head_raw < n_in ? head_raw : n_in;
+        const int nvec = (n_in - head) / E;
+        auto put = [&](int idx, float v) {                   // one element by flat index (head, tail)
+            const int q = nq > 1 ? div_small(idx, plane_in, inv_plane) : 0;
+            const int rem = idx - q * plane_in;
+            const int r = div_small(rem, W, inv_w);
+            tile[q * PS + (top + r) * Ws + lead + (rem - r * W)] = act_of(v, sc_s[q], sf_s[q], relu);
+        };
+        for (int i = threadIdx.x; i < head; i += kPoolThreads) put(i, Elem<T>::load1(xp + i));
+        for (int i = head + nvec * E + threadIdx.x; i < n_in; i += kPoolThreads) put(i, Elem<T>::load1(xp + i));
+        constexpr int U = 4;
+        for (int base = 0; base < nvec; base += U * kPoolThreads) {
+            Vec16 raw[U];
+#pragma unroll
+            for (int k = 0; k < U; ++k) {
+                const int v = base + k * kPoolThreads + threadIdx.x;
+                if (v < nvec) raw[k] = ld_stream(xp + head + (int64_t)v * E);
+            }
+#pragma unroll
+            for (int k = 0; k < U; ++k) {
+                const int v = base + k * kPoolThreads + threadIdx.x;
+                if (v < nvec) {
+                    float f[E];
+                    Elem<T>::unpack(raw[k], f);
+                    const int idx = head + v * E;
+                    int q = nq > 1 ? div_small(idx, plane_in, inv_plane) : 0;
+                    const int rem = idx - q * plane_in;
+                    int r = div_small(rem, W, inv_w);
+                    int cc = rem - r * W;
+                    if (((W | head) & 3) == 0) {
+                        // rows are whole groups of four and the piece starts on one: a group never leaves its row
+#pragma unroll
+                        for (int h = 0; h < E / 4; ++h) {
+                            const float sc = sc_s[q], sf = sf_s[q];
+                            *reinterpret_cast<float4*>(tile + q * PS + (top + r) * Ws + lead + cc) =
+                                make_float4(act_of(f[4 * h], sc, sf, relu), act_of(f[4 * h + 1], sc, sf, relu),
+                                            act_of(f[4 * h + 2], sc, sf, relu), act_of(f[4 * h + 3], sc, sf, relu));
+                            cc += 4;
+                            if (cc == W) {
+                                cc = 0;
+                                if (++r == nrows) {
+                                    r = 0;
+                                    ++q;
+                                }
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < E; ++e) {
+                            tile[q * PS + (top + r) * Ws + lead + cc] = act_of(f[e], sc_s[q], sf_s[q], relu);
+                            if (++cc == W) {
+                                cc = 0;
+                                if (++r == nrows) {
+                                    r = 0;
+                                    ++q;
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+    __syncthreads();
+    // 3. walks: unit u = (chunk of output rows, plane, group of four outputs); consecutive threads take
+    // consecutive groups, so shared-memory reads and global stores of a warp run along rows
+    const int OG = (OW + 3) / 4;
+    const int walkers = nq * OG;
+    const int orows = oh1 - oh0;
+    const int rpc = (orows + chunks - 1) / chunks;           // output rows per chunk
+    const float inv_walkers = 1.0f / (float)walkers, inv_og = 1.0f / (float)OG;
+    const bool vec_out = (OW & 3) == 0 && (reinterpret_cast<uintptr_t>(y) & (4 * sizeof(T) - 1)) == 0;
+    for (int u = threadIdx.x; u < walkers * chunks; u += kPoolThreads) {
+        const int chunk = div_small(u, walkers, inv_walkers);
+        const int w = u - chunk * walkers;
+        const int q = div_small(w, OG, inv_og), g = w - q * OG;
+        const int r_lo = chunk * rpc, r_hi = min(orows, r_lo + rpc);
+        if (r_lo >= r_hi) continue;
+        const float* src = tile + q * PS + r_lo * ST * Ws + (lead - pw) + 4 * g * ST;
+        T* dst = y + ((p0 + q) * OH + oh0 + r_lo) * (int64_t)OW + 4 * g;
+        float rows[KS][NV];
+        auto load_row = [&](const float* p, float (&v)[NV]) {
+            // p is one float short of a 16-byte boundary when the window is padded, on one otherwise
+            constexpr int first = kPadW ? 1 : 0;
+            if (kPadW) v[0] = p[0];
+#pragma unroll
+            for (int b = first; b < NV; b += 4) {
+                const float4 t = *reinterpret_cast<const float4*>(p + b);
+                v[b] = t.x;
+                if (b + 1 < NV) v[b + 1] = t.y;
+                if (b + 2 < NV) v[b + 2] = t.z;
+                if (b + 3 < NV) v[b + 3] = t.w;
+            }
+        };
+#pragma unroll
+        for (int i = 0; i < KS - ST; ++i) load_row(src + i * Ws, rows[i]);
+        src += (KS - ST) * Ws;
+        for (int r = r_lo; r < r_hi; ++r, src += ST * Ws, dst += OW) {
+#pragma unroll
+            for (int i = 0; i < ST; ++i) load_row(src + i * Ws, rows[KS - ST + i]);
+            float colv[NV], o[4];
+#pragma unroll
+            for (int cidx = 0; cidx < NV; ++cidx) {
+                float a = rows[0][cidx];
+#pragma unroll
+                for (int i = 1; i < KS; ++i) a = pool_op<T, MODE>(a, rows[i][cidx]);
+                colv[cidx] = a;
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                float a = colv[j * ST];
+#pragma unroll
+                for (int d = 1; d < KS; ++d) a = pool_op<T, MODE>(a, colv[j * ST + d]);
+                o[j] = MODE == 1 ? a * inv_area : a;
+            }
+            if (vec_out) store4<T>(dst, o);
+            else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (4 * g + j < OW) Elem<T>::store1(dst + j, o[j]);
+            }
+#pragma unroll
+            for (int i = 0; i < KS - ST; ++i)
+#pragma unroll
+                for (int cidx = 0; cidx < NV; ++cidx) rows[i][cidx] = rows[i + ST][cidx];
+        }
+    }
+}
+
 // Any geometry (rows too wide for the tile): one thread per output, window read from global memory.
 template <typename T>
 __global__ void __launch_bounds__(256)
@@ -482,8 +830,8 @@ kop_status_t launch_pool(const void* xv, const float* scale, const float* shift,
         const int64_t blocks = (strips + 255) / 256;
         if (blocks <= 0x7FFFFFFFLL) {
 #define KOP_STRIP(MODE, KS)                                                                                       \
-    pool2d_strip_kernel<T, MODE, KS><<<(unsigned)blocks, 256, 0, stream>>>(x, scale, shift, y, strips, (int)C, H, W, \
-                                                                            OH, OW, segs, bands, band_rows, relu, inv_area)
+    pool2d_strip_kernel<T, MODE, KS, 1><<<(unsigned)blocks, 256, 0, stream>>>(               \
+        x, scale, shift, y, strips, (int)C, H, W, OH, OW, segs, bands, band_rows, relu, inv_area)
             if (mode == 0) {
                 if (k3) KOP_STRIP(0, 3);
                 else KOP_STRIP(0, 2);
@@ -492,6 +840,84 @@ kop_status_t launch_pool(const void* xv, const float* scale, const float* shift,
                 else KOP_STRIP(1, 2);
             }
 #undef KOP_STRIP
+            return launch_status();
+        }
+    }
+    // 3x3 / stride 1 / pad 1 over rows of whole, aligned 8-column segments: the stride-1 strip kernel
+    if (k3 && sh == 1 && sw == 1 && W % 8 == 0 && aligned_to(x, 32) && aligned_to(y, 32)) {
+        const int segs = W / 8;
+        // bands of at least 16 output rows (each band reads two rows of its neighbours again)
+        int band_rows = H;
+        const int64_t want = 64LL * 32 * sm_count();
+        while (band_rows > 16 && planes * segs * ((H + band_rows - 1) / band_rows) < want) band_rows = (band_rows + 1) / 2;
+        const int bands = (H + band_rows - 1) / band_rows;
+        const int64_t strips = planes * segs * bands;
+        const int64_t blocks = (strips + 255) / 256;
+        if (blocks <= 0x7FFFFFFFLL) {
+            // two input rows per trip (one: fp32 4.4 - 4.7 TB/s, bf16 2.9 - 3.4; two: 4.6 - 5.2 and 3.7 - 4.0; four: slower again)
+            if (mode == 0)
+                pool2d_strip_s1_kernel<T, 0, 2><<<(unsigned)blocks, 256, 0, stream>>>(x, scale, shift, y, strips, (int)C, H, W, segs, bands, band_rows, relu, inv_area);
+            else
+                pool2d_strip_s1_kernel<T, 1, 2><<<(unsigned)blocks, 256, 0, stream>>>(x, scale, shift, y, strips, (int)C, H, W, segs, bands, band_rows, relu, inv_area);
+            return launch_status();
+        }
+    }
+    // 2x2 / 3x3 windows at stride 1 or 2 that the strip kernel does not take (stride 1, any width or alignment,
+    // small planes): the walk kernel, on runs of whole small planes or on bands of output rows of a large one
+    // (planes of at most 1024 elements stay with the runs-of-planes kernel below, which copies them flat without
+    // padding, unless the stride is 1 and the plane has 512 elements or more: 28 x 28 fp32 3 x 3 / 1 2.4 against 3.7 TB/s
+    // here, but 14 x 14 2.4 against 2.2 and the stride-2 windows 3.1 - 3.4 against 2.7 - 3.1)
+    const bool small_plane = (int64_t)H * W <= 1024;
+    if (kh == kw && sh == sw && (kh == 2 || kh == 3) && (sh == 1 || sh == 2) && pw <= 1 &&
+        (!small_plane || (sh == 1 && (int64_t)H * W >= 512))) {
+        const int Ws = walk_row_floats(W, OW, pw, kh, sh);
+        const int64_t plane_tile = ((int64_t)(OH - 1) * sh + kh) * Ws * 4;        // bytes of one whole padded plane
+        const bool all_rows_used = (OH - 1) * sh + kh - ph >= H;                  // else a plane's rows are not one run
+        int np = 1, br = OH, bands = 1;
+        bool ok = true;
+        if (plane_tile <= 12 * 1024 && all_rows_used && planes > 1) {
+            np = (int)(32 * 1024 / plane_tile);
+            if (np > planes) np = (int)planes;
+        } else {
+            const int64_t row_bytes = (int64_t)Ws * 4;
+            // about 24 KB of tile per band (12 KB and 8 KB tiles were 25 - 45 % slower: more halo rows, shorter walks)
+            int64_t b = ((int64_t)kPoolTileBytes / row_bytes - kh) / sh + 1;
+            if (b < 1) b = 1;
+            if (b > OH) b = OH;
+            ok = ((b - 1) * sh + kh) * row_bytes + 8 <= kPoolTileMax;
+            bands = (int)((OH + b - 1) / b);
+            br = (int)((OH + bands - 1) / bands);                                 // even bands
+            bands = (OH + br - 1) / br;
+        }
+        const int64_t grid = np > 1 ? (planes + np - 1) / np : planes * bands;
+        const size_t smem = (size_t)np * (((size_t)(br - 1) * sh + kh) * Ws * 4 + 8);
+        if (ok && grid <= 0x7FFFFFFFLL && smem <= (size_t)kPoolTileMax) {
+            // one pass of the CTA's threads over (row chunks x planes x groups of four outputs), at least two output
+            // rows per chunk where the band has them (the rows shared by consecutive windows stay in registers)
+            const int walkers = np * ((OW + 3) / 4);
+            int chunks = kPoolThreads / walkers;
+            if (chunks > (br + 1) / 2) chunks = (br + 1) / 2;
+            if (chunks < 1) chunks = 1;
+#define KOP_WALK(M, K, S, P)                                                                                     \
+    pool2d_walk_kernel<T, M, K, S, P><<<(unsigned)grid, kPoolThreads, smem, stream>>>(                             \
+        x, scale, shift, y, planes, np, (int)C, H, W, OH, OW, ph, br, bands, chunks, relu, inv_area)
+#define KOP_WALK_P(M, K, S)            \
+    do {                               \
+        if (pw) KOP_WALK(M, K, S, true); \
+        else KOP_WALK(M, K, S, false);   \
+    } while (0)
+#define KOP_WALK_KS(M)                                   \
+    do {                                                 \
+        if (kh == 3 && sh == 1) KOP_WALK_P(M, 3, 1);     \
+        else if (kh == 3) KOP_WALK_P(M, 3, 2);           \
+        else if (sh == 1) KOP_WALK_P(M, 2, 1);           \
+        else KOP_WALK_P(M, 2, 2);                        \
+    } while (0)
+            if (mode == 0) KOP_WALK_KS(0);
+            else KOP_WALK_KS(1);
+#undef KOP_WALK_KS
+#undef KOP_WALK_P
+#undef KOP_WALK
             return launch_status();
         }
     }

@@ -54,6 +54,22 @@ POOL_CASES = [
     (3, 5, 5, 9, (2, 3), (1, 2), (1, 1), F32),         # generic window on a small plane
     (3, 3, 3, 3, (3, 3), (3, 3), (0, 0), BF16),        # 9-element planes
     (70, 64, 7, 7, (3, 3), (1, 1), (1, 1), BF16),      # several runs
+    # stride-1 3x3 over whole 8-column segments: the register strip kernel (four bands; odd height, ragged last band)
+    (2, 3, 56, 56, (3, 3), (1, 1), (1, 1), F32),
+    (1, 2, 57, 64, (3, 3), (1, 1), (1, 1), BF16),
+    (1, 1, 19, 8, (3, 3), (1, 1), (1, 1), torch.float16),          # one segment per row: both halos are padding
+    # 2x2 / 3x3 at stride 1 / 2 out of a shared-memory tile: widths that are not whole segments or vectors, padding
+    # in one direction only, a padded 2x2 window, one large plane in several bands, rows that start off a vector
+    (2, 3, 60, 60, (3, 3), (2, 2), (1, 1), F32),
+    (2, 3, 57, 57, (3, 3), (1, 1), (1, 1), BF16),
+    (2, 3, 40, 44, (2, 2), (1, 1), (0, 0), F32),
+    (2, 2, 33, 36, (3, 3), (1, 1), (1, 0), F32),
+    (2, 2, 36, 33, (3, 3), (2, 2), (0, 1), BF16),
+    (2, 2, 30, 30, (2, 2), (2, 2), (1, 1), torch.float16),
+    (1, 1, 200, 204, (3, 3), (1, 1), (1, 1), F32),
+    (1, 1, 301, 97, (3, 3), (2, 2), (1, 1), BF16),
+    (3, 7, 28, 28, (3, 3), (1, 1), (1, 1), F32),                   # runs of whole small planes through the same kernel
+    (5, 3, 23, 31, (2, 2), (1, 1), (0, 0), BF16),
 ]
 
 
