@@ -100,6 +100,12 @@ def segment_bytes():
     e_out = q["N"] * q["C"] * ((q["H"] + 2 * q["padding"][0] - q["kernel"][0]) // q["stride"][0] + 1) * \
         ((q["W"] + 2 * q["padding"][1] - q["kernel"][1]) // q["stride"][1] + 1)
     out["pool2d"] = dict(bytes=(e_in + e_out) * 4 + 2 * q["C"] * 4, elems=e_in)
+    for nm in ("pool2d_s1", "pool2d_14"):
+        q = c[nm]
+        e_in = q["N"] * q["C"] * q["H"] * q["W"]
+        e_out = q["N"] * q["C"] * ((q["H"] + 2 * q["padding"][0] - q["kernel"][0]) // q["stride"][0] + 1) * \
+            ((q["W"] + 2 * q["padding"][1] - q["kernel"][1]) // q["stride"][1] + 1)
+        out[nm] = dict(bytes=(e_in + e_out) * 4 + 2 * q["C"] * 4, elems=e_in)
     q = c["reduce"]
     out["reduce_max"] = dict(bytes=q["rows"] * q["cols"] * 2 + q["rows"] * 8, elems=q["rows"] * q["cols"])
     out["reduce_logsumexp"] = dict(bytes=q["rows"] * q["cols"] * 2 + q["rows"] * 4, elems=q["rows"] * q["cols"])
@@ -259,7 +265,7 @@ class Workload:
 
     ORDER = ["softmax_small", "softmax_large", "layernorm", "bn_pool", "ce_loss", "rmsnorm", "silu_mul", "residual_add"]
     # Beyond the benchmark configs (not part of `value`): the two kernels the paper's case studies print.
-    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "layernorm_params16", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc", "pool2d", "reduce_max", "reduce_logsumexp", "bias_gelu", "residual_rmsnorm", "l2_normalize", "lstm_cell", "gru_cell", "rmsnorm_head128", "softmax_vocab"]
+    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "layernorm_params16", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc", "pool2d", "pool2d_s1", "pool2d_14", "reduce_max", "reduce_logsumexp", "bias_gelu", "residual_rmsnorm", "l2_normalize", "lstm_cell", "gru_cell", "rmsnorm_head128", "softmax_vocab"]
 
     def __init__(self, kop, device, seed, only=None, rows_div=1):
         """only: build just these segments (None = all, plus the MLP segment); rows_div cuts the row
@@ -329,6 +335,13 @@ class Workload:
             oh = (q["H"] + 2 * q["padding"][0] - q["kernel"][0]) // q["stride"][0] + 1
             ow = (q["W"] + 2 * q["padding"][1] - q["kernel"][1]) // q["stride"][1] + 1
             self.py = torch.empty((self.px.shape[0], q["C"], oh, ow), dtype=q["dtype"], device=dev)
+        for nm in ("pool2d_s1", "pool2d_14"):
+            if nm in want:
+                q = c[nm]
+                px, ps, pf = synth.bn_pool_inputs(cut(q["N"]), q["C"], q["H"], q["W"], q["dtype"], seed, dev)
+                oh = (q["H"] + 2 * q["padding"][0] - q["kernel"][0]) // q["stride"][0] + 1
+                ow = (q["W"] + 2 * q["padding"][1] - q["kernel"][1]) // q["stride"][1] + 1
+                setattr(self, nm, (px, ps, pf, torch.empty((px.shape[0], q["C"], oh, ow), dtype=q["dtype"], device=dev)))
         if want & {"reduce_max", "reduce_logsumexp"}:
             q = c["reduce"]
             self.rx, _ = synth.softmax_inputs(cut(q["rows"]), q["cols"], q["dtype"], seed, dev)
@@ -436,6 +449,10 @@ class Workload:
             q = c["pool2d"]
             k.kop_affine_relu_pool2d(self.px, self.pscale, self.pshift, q["kernel"], q["stride"], q["padding"],
                                      q["mode"], True, out=self.py)
+        elif name in ("pool2d_s1", "pool2d_14"):  # 3x3 / stride-1 average on 112 x 112 maps; 3x3 / stride-2 max on 14 x 14 maps
+            q = c[name]
+            px, ps, pf, py = getattr(self, name)
+            k.kop_affine_relu_pool2d(px, ps, pf, q["kernel"], q["stride"], q["padding"], q["mode"], True, out=py)
         elif name == "reduce_max":               # row max + argmax, bf16 [32768, 8192]
             k.kop_reduce_rows(self.rx, "max", out=self.rv, index=self.ri)
         elif name == "reduce_logsumexp":

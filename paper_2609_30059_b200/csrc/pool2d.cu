@@ -680,14 +680,23 @@ pool2d_walk_kernel(const T* __restrict__ x, const float* __restrict__ scale, con
                             }
                         }
                     } else {
+                        // element by element with a running destination: rows and planes wrap rarely
+                        float* d = tile + q * PS + (top + r) * Ws + lead + cc;
+                        float sc = sc_s[q], sf = sf_s[q];
 #pragma unroll
                         for (int e = 0; e < E; ++e) {
-                            tile[q * PS + (top + r) * Ws + lead + cc] = act_of(f[e], sc_s[q], sf_s[q], relu);
+                            *d++ = act_of(f[e], sc, sf, relu);
                             if (++cc == W) {
                                 cc = 0;
+                                d += Ws - W;
                                 if (++r == nrows) {
                                     r = 0;
                                     ++q;
+                                    d += PS - nrows * Ws;
+                                    if (e + 1 < E) {
+                                        sc = sc_s[q];
+                                        sf = sf_s[q];
+                                    }
                                 }
                             }
                         }

@@ -29,6 +29,12 @@ CONFIGS = {
     # BatchNorm + ReLU + 3x3 / stride-2 max pool on a 112 x 112 map with 64 channels (a CNN stem)
     "pool2d": dict(N=64, C=64, H=112, W=112, kernel=(3, 3), stride=(2, 2), padding=(1, 1), mode="max",
                    dtype=torch.float32),
+    # the same epilogue with a stride-1 3x3 window (an inception-style pooling branch) and on the 14 x 14 maps of a
+    # CNN's later stages (shapes ours)
+    "pool2d_s1": dict(N=64, C=64, H=112, W=112, kernel=(3, 3), stride=(1, 1), padding=(1, 1), mode="avg",
+                      dtype=torch.float32),
+    "pool2d_14": dict(N=256, C=512, H=14, W=14, kernel=(3, 3), stride=(2, 2), padding=(1, 1), mode="max",
+                      dtype=torch.float32),
     # pointwise part of one LSTM step: batch 16384, hidden 1024 (shape ours)
     "lstm_cell": dict(rows=16384, hidden=1024, dtype=torch.bfloat16),
     "gru_cell": dict(rows=16384, hidden=1024, dtype=torch.bfloat16),

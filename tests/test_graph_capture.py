@@ -37,6 +37,8 @@ def test_all_entry_points_in_one_graph(kop):
     tg, tg2, tb, tc = synth.lstm_inputs(rows, 96, BF16, 11, dev)
     ui, uh, ubi, ubh, up = synth.gru_inputs(rows, 96, BF16, 12, dev)
     lb16, lg16, lbe16 = lb.to(lx.dtype), lg.to(lx.dtype), lbe.to(lx.dtype)
+    bias16 = bias.to(x.dtype)
+    img16, sc16, sh16 = img.to(BF16), sc.to(BF16), sh.to(BF16)
     handle = kop.MlpHandle()
     ws_ce = torch.empty(max(16, kop.kop_ce_loss_rowwise_workspace_bytes(rows, cols, kop.KOP_BF16)), dtype=torch.uint8, device=dev)
     ws_mlp = torch.empty(kop.kop_rmsnorm_swiglu_residual_workspace_bytes(64, 256, 512, kop.KOP_BF16), dtype=torch.uint8, device=dev)
@@ -59,6 +61,10 @@ def test_all_entry_points_in_one_graph(kop):
         "rr_h": torch.empty_like(lx), "rr_y": torch.empty_like(lx), "lstm_h": torch.empty_like(tc), "lstm_c": torch.empty_like(tc),
         "gru_h": torch.empty_like(up), "lpn": torch.empty_like(lx), "lpn_n": torch.empty(rows, device=dev),
         "ln_ex": torch.empty_like(lx), "rms_ex_h": torch.empty_like(lx), "rms_ex_y": torch.empty_like(lx),
+        "ceo_sum": torch.empty(1, device=dev), "softmax_ex": torch.empty_like(x), "act_ex": torch.empty_like(x),
+        "chain_ex": torch.empty_like(x), "bn_ex": torch.empty_like(img16), "bn_ex_p": torch.empty((3, 16), device=dev),
+        "gn_ex": torch.empty_like(img16), "pool_s1": torch.empty((3, 16, 28, 28), device=dev),
+        "pool_walk": torch.empty((3, 16, 27, 27), device=dev),
     }
 
     def run():
@@ -69,7 +75,8 @@ def test_all_entry_points_in_one_graph(kop):
         kop.kop_residual_layernorm(lx, lr, lg, lbe, 1e-5, out=o["rln"], want_stats=False)
         kop.kop_ce_loss_rowwise(z, lab, loss=o["ce_loss"], mean_loss=o["ce_mean"], bad_label_count=o["ce_bad"], workspace=ws_ce)
         kop.kop_ce_loss_rowwise_opts(z, lab_ig, -100, 0.1, loss=o["ceo_loss"], mean_loss=o["ceo_mean"],
-                                     bad_label_count=o["ceo_bad"], counted_rows=o["ceo_cnt"], workspace=ws_ce)
+                                     bad_label_count=o["ceo_bad"], counted_rows=o["ceo_cnt"], workspace=ws_ce,
+                                     sum_loss=o["ceo_sum"])
         kop.kop_bn_relu_avgpool(img, sc, sh, out=o["bn"], pooled=o["bn_p"])
         kop.kop_bn_relu_avgpool(img_cl, sc, sh, out=o["bn_cl"], pooled=o["bn_cl_p"])
         kop.kop_groupnorm_act(gx, gg, gb, 4, 1e-5, 2, out=o["gn"], mean=o["gn_mean"], rstd=o["gn_rstd"])
@@ -91,6 +98,13 @@ def test_all_entry_points_in_one_graph(kop):
         kop.kop_lp_normalize_rows(lx, 2, 1e-12, out=o["lpn"], norms=o["lpn_n"])
         kop.kop_layernorm_ex(lx, lr, lb16, lg16, lbe16, 1e-5, "bias_erfgelu_residual", out=o["ln_ex"], want_stats=False)
         kop.kop_rmsnorm_ex(lx, lg16, 1e-6, residual=lr, h_out=o["rms_ex_h"], out=o["rms_ex_y"])
+        kop.kop_softmax_ex(x, bias16, 0.125, True, cols, out=o["softmax_ex"])
+        kop.kop_bias_act_ex(x, bias16, "silu", out=o["act_ex"])
+        kop.kop_epilogue_chain_ex(x, bias16, lx, 0.5, 2.0, -1.0, 1.0, "relu", out=o["chain_ex"])
+        kop.kop_bn_relu_avgpool_ex(img16, sc16, sh16, out=o["bn_ex"], pooled=o["bn_ex_p"])
+        kop.kop_groupnorm_act_ex(img16, sc16, sh16, 4, 1e-5, 1, out=o["gn_ex"], want_stats=False)
+        kop.kop_affine_relu_pool2d(img, sc, sh, (3, 3), (1, 1), (1, 1), "avg", True, out=o["pool_s1"])
+        kop.kop_affine_relu_pool2d(img, sc, sh, (2, 2), (1, 1), (0, 0), "max", False, out=o["pool_walk"])
         kop.kop_rmsnorm_swiglu_residual(handle, h, w, W1, W2, 1e-6, out=o["mlp"], workspace=ws_mlp)
 
     try:
