@@ -156,6 +156,16 @@ def test_fuzz_row_kernels(kop):
         xa, ba = synth.softmax_inputs(rows, cols, dtype, seed, "cuda")
         assert_close(kop.kop_bias_act(strided(rng, xa), ba, act, alpha=0.3), kopref.bias_act(host(xa), host(ba), act, alpha=0.3),
                      tol, f"bias_act {act} " + what)
+        # the same epilogue, the chain and the softmax with the bias stored in the data type (16-bit data only)
+        if dtype != F32:
+            b16 = ba.to(dtype)
+            assert_close(kop.kop_bias_act_ex(strided(rng, xa), b16, act, alpha=0.3),
+                         kopref.bias_act(host(xa), host(b16), act, alpha=0.3), tol, f"bias_act_ex {act} " + what)
+            assert_close(kop.kop_epilogue_chain_ex(strided(rng, xa), b16, strided(rng, x), 0.75, 1.5, -2.0, 2.5, act, alpha=0.3),
+                         kopref.epilogue_chain(host(xa), host(b16), host(x), 0.75, 1.5, -2.0, 2.5, act, alpha=0.3), tol,
+                         f"epilogue_chain_ex {act} " + what)
+            assert_close(kop.kop_softmax_ex(strided(rng, xa), b16, scale),
+                         kopref.softmax_scale_bias(host(xa), host(b16), scale), tol, "softmax_ex " + what)
         # LSTM gate arithmetic (cols = hidden units, any length: vector and element kernels)
         hid = max(1, cols // 4)
         tg, tg2, tb, tc = synth.lstm_inputs(rows, hid, dtype, seed, "cuda")
@@ -222,4 +232,26 @@ def test_fuzz_image_kernels(kop):
         ref = kopref.affine_relu_pool2d(host(x), host(scale) if aff else None, host(shift) if aff else None, (kh, kw),
                                         (sh, sw), (ph, pw), mode, relu)
         assert_close(y, ref, tol, f"pool2d k=({kh},{kw}) s=({sh},{sw}) p=({ph},{pw}) {mode} " + what)
+        # the windows CNNs use (2 x 2 / 3 x 3, stride 1 / 2, pad 0 / 1) on larger planes: the strip and walk kernels,
+        # widths that are and are not whole 8-column segments
+        Hb = int(rng.choice([16, 24, 33, 40, 57, 64]))
+        Wb = int(rng.choice([16, 24, 30, 33, 40, 56, 60, 63, 64, 72]))
+        k = int(rng.integers(2, 4))
+        st = int(rng.integers(1, 3))
+        pd = (int(rng.integers(0, 2)), int(rng.integers(0, 2)))
+        xb, scb, shb = synth.bn_pool_inputs(int(rng.integers(1, 3)), int(rng.integers(1, 5)), Hb, Wb, dtype, seed, "cuda")
+        y = kop.kop_affine_relu_pool2d(xb, scb if aff else None, shb if aff else None, (k, k), (st, st), pd, mode, relu)
+        ref = kopref.affine_relu_pool2d(host(xb), host(scb) if aff else None, host(shb) if aff else None, (k, k), (st, st),
+                                        pd, mode, relu)
+        assert_close(y, ref, tol, f"pool2d {Hb}x{Wb} k={k} s={st} p={pd} {mode} " + what)
+        # 16-bit data: folded BatchNorm coefficients and GroupNorm weights stored in the data type
+        if dtype != F32:
+            s16, h16 = scale.to(dtype), shift.to(dtype)
+            y, p = kop.kop_bn_relu_avgpool_ex(xl if rng.integers(0, 2) else x, s16, h16)
+            ry, rp = kopref.bn_relu_avgpool(host(x), host(s16), host(h16))
+            assert_close(y, ry, tol, "bn_ex y " + what)
+            assert_close(p, rp, 1e-5, "bn_ex pooled " + what)
+            g16, be16 = gamma.to(dtype), beta.to(dtype)
+            y, _, _ = kop.kop_groupnorm_act_ex(xg, g16, be16, groups, 1e-5, act)
+            assert_close(y, kopref.groupnorm_act(host(xg), host(g16), host(be16), groups, 1e-5, act)[0], tol, "groupnorm_ex y " + what)
     assert kop.kop_groupnorm_wait_timeouts() == 0
