@@ -641,7 +641,7 @@ def run_ours(args, rank, world, local_rank):
             extra_per[nm].append(evs[nm][0].elapsed_time(evs[nm][1]))
 
     # ---- every kernel in a train of its own launches, alternating between two independent sets of tensors
-    # (different seeds) so that no launch finds its inputs in the L2: one event pair around 2 x 10 launches. In
+    # (different seeds) so that no launch finds its inputs in the L2: one event pair spanning 2 x 10 launches. In
     # steady state each launch inherits exactly the dirty output lines its twin left and leaves as many behind, so
     # nobody else's write-backs are charged to it and none of its own escape the clock - the figure that a kernel
     # timed alone after a memset (it pays for ~100 MB of the memset's dirty lines) or in the mixed step (it pays
