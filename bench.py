@@ -554,11 +554,29 @@ def run_ours(args, rank, world, local_rank):
     segs = segment_bytes()
     names = Workload.ORDER
 
-    def step(events, with_graph=False):
-        for i, nm in enumerate(names):
+    # The order of the eight launches inside a step cycles through the rows of a row-complete Latin square
+    # (Williams design: row r is r + (0, 1, n-1, 2, n-2, ...) mod n), so that over n consecutive steps every kernel
+    # follows every other kernel exactly once. A per-launch event time contains the write-back of the dirty L2 lines
+    # the predecessor left (up to ~100 MB) minus those the kernel itself leaves behind; with one fixed order each
+    # kernel would be charged (or spared) one particular neighbour's lines in every step. The sum over a step, and
+    # with it `value`, does not depend on the order.
+    n_k = len(names)
+    base = [0] + [((j + 1) // 2 if j % 2 else n_k - j // 2) % n_k for j in range(1, n_k)]
+    orders = [[(r + b) % n_k for b in base] for r in range(n_k)]
+    step_no = [0]
+    followed = []                 # per step: {kernel index: predecessor's name}, for the timed steps
+
+    def step(events, with_graph=False, log=None):
+        order = orders[step_no[0] % n_k]
+        step_no[0] += 1
+        prev = "mlp_graph" if with_graph else (names[orders[(step_no[0] - 2) % n_k][-1]] if step_no[0] > 1 else None)
+        for i in order:
+            if log is not None:
+                log[i] = prev
             events[i][0].record()
-            wl.launch(nm)
+            wl.launch(names[i])
             events[i][1].record()
+            prev = names[i]
         if with_graph:
             events[len(names)][0].record()
             wl.graph.replay()
@@ -576,14 +594,18 @@ def run_ours(args, rank, world, local_rank):
         if world > 1:
             torch.distributed.barrier()
         t0.record()
-        for ev in all_events:
-            step(ev, with_graph)
+        logs = [dict() for _ in all_events]
+        for ev, lg in zip(all_events, logs):
+            step(ev, with_graph, lg)
         t1.record()
         torch.cuda.synchronize()
         if world > 1:
             torch.distributed.barrier()
         per = {nm: [ev[i][0].elapsed_time(ev[i][1]) for ev in all_events] for i, nm in enumerate(names)}
         g = [ev[len(names)][0].elapsed_time(ev[len(names)][1]) for ev in all_events] if with_graph else []
+        if not with_graph:
+            followed.clear()
+            followed.extend(logs)
         return t0.elapsed_time(t1), per, g
 
     sampler = ClockSampler(local_rank, args.clock_sample_ms * 1e-3)
@@ -597,10 +619,10 @@ def run_ours(args, rank, world, local_rank):
     # LayerNorm launch replaced by a 2-reads-1-write add over the same three tensors (same bytes bar the parameter
     # vectors and statistics, same predecessor, same cache state). Per-launch event times in a sequence include the
     # write-back of the dirty L2 lines the predecessor left behind, so this, not bytes / peak, is what the slot allows.
-    ceil_seq = [("layernorm_stream_ceiling" if nm == "layernorm" else nm) for nm in names]
     ceil_ts = []
-    for it in range(3 + max(10, min(args.steps, 100))):
-        for nm in ceil_seq:
+    for it in range(3 + max(16, min(args.steps, 104))):
+        for i in orders[it % n_k]:                           # the same cycle of orders as the timed steps
+            nm = "layernorm_stream_ceiling" if names[i] == "layernorm" else names[i]
             if nm == "layernorm_stream_ceiling":
                 e0 = torch.cuda.Event(enable_timing=True)
                 e1 = torch.cuda.Event(enable_timing=True)
@@ -767,8 +789,15 @@ def run_ours(args, rank, world, local_rank):
         ms = statistics.mean(per[nm])
         gbs = segs[nm]["bytes"] / (ms * 1e-3) / 1e9
         own = segs[nm]["bytes"] / (self_seq[nm] * 1e-3) / 1e9
+        # the same launches split by the kernel that ran just before (each predecessor once in eight steps)
+        by_pred = {}
+        idx = names.index(nm)
+        for k, lg in enumerate(followed):
+            if lg.get(idx) is not None:
+                by_pred.setdefault(lg[idx], []).append(per[nm][k])
         per_kernel.append(dict(kernel=nm, algorithmic_bytes=segs[nm]["bytes"], avg_launch_us=round(ms * 1e3, 2),
                                achieved=round(gbs, 1), frac=round(gbs / peak, 4), traffic=ncu_traffic(nm),
+                               us_after_predecessor={p: round(statistics.mean(v) * 1e3, 2) for p, v in by_pred.items()},
                                train_of_own_launches_us=round(self_seq[nm] * 1e3, 2),
                                frac_train_of_own_launches=round(own / peak, 4)))
     for k in per_kernel:
@@ -776,7 +805,8 @@ def run_ours(args, rank, world, local_rank):
             k["stream_in_same_slot_us"] = round(ln_ceiling_us, 2)
             k["frac_of_stream_in_same_slot"] = round(ln_ceiling_us / k["avg_launch_us"], 4)
             k["stream_in_same_slot"] = ("kop_residual_add over the same x / residual / y tensors (2 reads, 1 write, "
-                                        "201,326,592 bytes) launched in this kernel's place in the step")
+                                        "201,326,592 bytes) launched in this kernel's place in the steps (same cycle "
+                                        "of orders)")
     large = [k for k in per_kernel if k["kernel"] != "softmax_small"]       # 0.5 MB: latency-, not HBM-bound
     worst = min(large, key=lambda k: k["frac"])
     roofline = dict(bound="hbm", kernel=dom, achieved=round(achieved, 1), peak=peak, unit="GB/s",
@@ -804,6 +834,8 @@ def run_ours(args, rank, world, local_rank):
                                    "fp32 [64,256,56,56]; cross-entropy bf16 [32768,32000]; RMSNorm bf16 "
                                    "[16384,4096]; SiLU*up bf16 [16384,2x14336]; residual add bf16 [16384,4096]",
                        "l2": "inputs larger than L2: each step streams > 5 GB through a 126 MB L2",
+                       "order": "the eight launches of a step cycle through the rows of a row-complete Latin square: "
+                                "every kernel follows every other kernel once in eight steps",
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "fused_ms_per_step": round(fused_ms_step_max, 4),
             "gpu_launches": args.steps * len(names),
