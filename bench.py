@@ -8,9 +8,12 @@ One STEP is one pass of the whole fused hot path over one batch of seeded synthe
   chain) and bracketed by CUDA events.
 
 value (GB/s) = algorithmic bytes of the fused kernels (every input read once, every output written
-once) / the time those kernels took inside the K timed steps. Every kernel's working set is far
-larger than L2 except the small softmax, and consecutive kernels evict each other, so all launches
-run cold. After the timed region the whole transformer-MLP segment (RMSNorm -> cuBLAS -> SiLU*up ->
+once) in K steps / the device time of the K timed steps (launch gaps included). One event is recorded
+between consecutive launches, so a kernel's time runs from the end of its predecessor to its own end
+and the per-kernel times of a step add up to the step; the order of the launches cycles through a
+row-complete Latin square, so every kernel follows every other one equally often. Every kernel's
+working set is far larger than L2 except the small softmax, and consecutive kernels evict each other,
+so all launches run cold. After the timed region the whole transformer-MLP segment (RMSNorm -> cuBLAS -> SiLU*up ->
 cuBLAS -> residual) is replayed as one CUDA graph and reported under "mlp_segment_graph", together
 with the fused kernels' numbers when they alternate with that graph: the preserved vendor GEMMs
 drive the GPU into its power cap, so those show the same kernels at the lower SM clock they see
@@ -566,25 +569,27 @@ def run_ours(args, rank, world, local_rank):
     step_no = [0]
     followed = []                 # per step: {kernel index: predecessor's name}, for the timed steps
 
+    # One event between consecutive launches: launch number p of a step is timed from the event recorded after
+    # its predecessor to the event recorded after itself, so its time contains its own launch gap and the step's
+    # intervals add up to the step exactly (two events per launch left the time between one launch's end event and
+    # the next one's start event in nobody's account, and put two stream operations into every gap).
     def step(events, with_graph=False, log=None):
         order = orders[step_no[0] % n_k]
         step_no[0] += 1
         prev = "mlp_graph" if with_graph else (names[orders[(step_no[0] - 2) % n_k][-1]] if step_no[0] > 1 else None)
-        for i in order:
+        events[0].record()
+        for pos, i in enumerate(order):
             if log is not None:
-                log[i] = prev
-            events[i][0].record()
+                log[i] = (prev, pos)
             wl.launch(names[i])
-            events[i][1].record()
+            events[pos + 1].record()
             prev = names[i]
         if with_graph:
-            events[len(names)][0].record()
             wl.graph.replay()
-            events[len(names)][1].record()
+            events[n_k + 1].record()
 
     def new_events():
-        return [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-                for _ in range(len(names) + 1)]
+        return [torch.cuda.Event(enable_timing=True) for _ in range(n_k + 2)]
 
     def timed(n_steps, with_graph):
         all_events = [new_events() for _ in range(n_steps)]
@@ -601,8 +606,9 @@ def run_ours(args, rank, world, local_rank):
         torch.cuda.synchronize()
         if world > 1:
             torch.distributed.barrier()
-        per = {nm: [ev[i][0].elapsed_time(ev[i][1]) for ev in all_events] for i, nm in enumerate(names)}
-        g = [ev[len(names)][0].elapsed_time(ev[len(names)][1]) for ev in all_events] if with_graph else []
+        per = {nm: [ev[lg[i][1]].elapsed_time(ev[lg[i][1] + 1]) for ev, lg in zip(all_events, logs)]
+               for i, nm in enumerate(names)}
+        g = [ev[n_k].elapsed_time(ev[n_k + 1]) for ev in all_events] if with_graph else []
         if not with_graph:
             followed.clear()
             followed.extend(logs)
@@ -620,19 +626,17 @@ def run_ours(args, rank, world, local_rank):
     # vectors and statistics, same predecessor, same cache state). Per-launch event times in a sequence include the
     # write-back of the dirty L2 lines the predecessor left behind, so this, not bytes / peak, is what the slot allows.
     ceil_ts = []
+    last = torch.cuda.Event(enable_timing=True)
+    last.record()
     for it in range(3 + max(16, min(args.steps, 104))):
-        for i in orders[it % n_k]:                           # the same cycle of orders as the timed steps
+        for i in orders[it % n_k]:                           # the same cycle of orders and the same event scheme
             nm = "layernorm_stream_ceiling" if names[i] == "layernorm" else names[i]
-            if nm == "layernorm_stream_ceiling":
-                e0 = torch.cuda.Event(enable_timing=True)
-                e1 = torch.cuda.Event(enable_timing=True)
-                e0.record()
-                wl.launch(nm)
-                e1.record()
-                if it >= 3:
-                    ceil_ts.append((e0, e1))
-            else:
-                wl.launch(nm)
+            wl.launch(nm)
+            e1 = torch.cuda.Event(enable_timing=True)
+            e1.record()
+            if nm == "layernorm_stream_ceiling" and it >= 3:
+                ceil_ts.append((last, e1))
+            last = e1
     torch.cuda.synchronize()
     ln_ceiling_us = statistics.mean(e0.elapsed_time(e1) for e0, e1 in ceil_ts) * 1e3
 
@@ -748,11 +752,13 @@ def run_ours(args, rank, world, local_rank):
                               "the intermediate d drop out of the graph"}
         del lt_graph
 
-    fused_ms_step = sum(statistics.mean(per[nm]) for nm in names)
-    fused_bytes = sum(segs[nm]["bytes"] for nm in names)
-    # max over ranks of the timed quantities
-    (total_ms,) = max_over_ranks([total_ms], world, dev)
-    value, fused_ms_step_max = aggregate_throughput(fused_bytes, fused_ms_step, world, dev)
+    fused_ms_step = sum(statistics.mean(per[nm]) for nm in names)      # the step's intervals: total_ms / steps bar the
+    fused_bytes = sum(segs[nm]["bytes"] for nm in names)               # event records between two steps
+    # `value` is the whole timed region: bytes of K steps over the time between the two synchronised ends of the
+    # region, max over ranks (ms_per_step is the same time per step)
+    value, step_ms_max = aggregate_throughput(fused_bytes, total_ms / args.steps, world, dev)
+    total_ms = step_ms_max * args.steps
+    (fused_ms_step_max,) = max_over_ranks([fused_ms_step], world, dev)
 
     peak, peak_src = measured_peak()
 
@@ -793,8 +799,8 @@ def run_ours(args, rank, world, local_rank):
         by_pred = {}
         idx = names.index(nm)
         for k, lg in enumerate(followed):
-            if lg.get(idx) is not None:
-                by_pred.setdefault(lg[idx], []).append(per[nm][k])
+            if lg.get(idx) is not None and lg[idx][0] is not None:
+                by_pred.setdefault(lg[idx][0], []).append(per[nm][k])
         per_kernel.append(dict(kernel=nm, algorithmic_bytes=segs[nm]["bytes"], avg_launch_us=round(ms * 1e3, 2),
                                achieved=round(gbs, 1), frac=round(gbs / peak, 4), traffic=ncu_traffic(nm),
                                us_after_predecessor={p: round(statistics.mean(v) * 1e3, 2) for p, v in by_pred.items()},
