@@ -460,6 +460,7 @@ kop_status_t kop_cumsum_rows(const void* x, const unsigned char* mask, void* y, 
  *   kop_groupnorm_act_ex     kop_groupnorm_act        (gamma, beta; each may be NULL)
  *   kop_bias_act_ex          kop_bias_act             (bias; may be NULL)
  *   kop_epilogue_chain_ex    kop_epilogue_chain       (bias; may be NULL)
+ *   kop_affine_relu_pool2d_ex  kop_affine_relu_pool2d  (scale, shift; both or neither NULL)
  * Parameter pointers must be aligned to their element size; 16-byte alignment takes the vector kernels.
  */
 kop_status_t kop_softmax_ex(const void* x, const void* bias, void* y, int64_t rows, int64_t cols,
@@ -479,6 +480,10 @@ kop_status_t kop_epilogue_chain_ex(const void* x, const void* bias, const void* 
                                    int64_t cols, int64_t x_row_stride, int64_t res_row_stride, int64_t y_row_stride,
                                    float scale, float residual_scale, float clamp_lo, float clamp_hi, int act,
                                    float alpha, kop_dtype_t dtype, kop_dtype_t param_dtype, kop_stream_t stream);
+kop_status_t kop_affine_relu_pool2d_ex(const void* x, const void* scale, const void* shift, void* y, int64_t N,
+                                       int64_t C, int64_t H, int64_t W, int kh, int kw, int sh, int sw, int ph,
+                                       int pw, int mode, int relu, kop_dtype_t dtype, kop_dtype_t param_dtype,
+                                       kop_stream_t stream);
 
 /*
  * Lp normalisation of rows (fusion agent: "normalization fusion", a reduction and the pointwise pass that uses it

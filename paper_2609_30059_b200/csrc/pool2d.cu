@@ -12,6 +12,19 @@
 namespace kop {
 namespace {
 
+// A per-channel parameter vector in fp32 or in a 16-bit type, read once per plane: the type is a runtime tag (no
+// second set of kernel instances for the parameter type; the load is outside every inner loop).
+struct ParamVec {
+    const void* p;
+    int tag;                                                 // kop_dtype_t of the vector
+    __device__ __forceinline__ float at(int64_t j) const
+    {
+        if (tag == KOP_F32) return __ldg(static_cast<const float*>(p) + j);
+        if (tag == KOP_BF16) return Elem<__nv_bfloat16>::load1(static_cast<const __nv_bfloat16*>(p) + j);
+        return Elem<__half>::load1(static_cast<const __half*>(p) + j);
+    }
+};
+
 constexpr int kPoolThreads = 256;
 constexpr int kPoolTileBytes = 24 * 1024;       // preferred tile size
 constexpr int kPoolTileMax = 46 * 1024;         // static + dynamic shared memory stays under the 48 KB default
@@ -77,7 +90,7 @@ __device__ __forceinline__ float window_value(const float* win, int Ws, int kh, 
 // long enough to keep most lanes busy. Otherwise threads walk the band's flat index range.
 template <typename T, int MODE, int KS, int ST, bool kVecIn, bool kRowMap>
 __global__ void __launch_bounds__(kPoolThreads)
-pool2d_tile_kernel(const T* __restrict__ x, const float* __restrict__ scale, const float* __restrict__ shift,
+pool2d_tile_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift,
                    T* __restrict__ y, int C, int H, int W, int OH, int OW, int kh_, int kw_, int sh_, int sw_,
                    int ph, int pw, int band_rows, int bands, int relu_flag, float inv_area)
 {
@@ -88,8 +101,8 @@ pool2d_tile_kernel(const T* __restrict__ x, const float* __restrict__ scale, con
     const int64_t plane = blockIdx.x / bands;
     const int band = (int)(blockIdx.x - plane * bands);
     const int c = (int)(plane % C);
-    const float sc = scale != nullptr ? __ldg(scale + c) : 1.0f;
-    const float sf = shift != nullptr ? __ldg(shift + c) : 0.0f;
+    const float sc = scale.p != nullptr ? scale.at(c) : 1.0f;
+    const float sf = shift.p != nullptr ? shift.at(c) : 0.0f;
     const float pad = MODE == 0 ? -INFINITY : 0.0f;
 
     const int oh0 = band * band_rows;
@@ -287,7 +300,7 @@ __device__ __forceinline__ void store4<__half>(__half* dst, const float (&o)[4])
 // type: bf16 3x3 4.4 to 3.6 TB/s, 2x2 5.5 to 5.0).
 template <typename T, int MODE, int KS, int R>
 __global__ void __launch_bounds__(256)
-pool2d_strip_kernel(const T* __restrict__ x, const float* __restrict__ scale, const float* __restrict__ shift,
+pool2d_strip_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift,
                     T* __restrict__ y, int64_t strips, int C, int H, int W, int OH, int OW, int segs, int bands,
                     int band_rows, int relu_flag, float inv_area)
 {
@@ -300,8 +313,8 @@ pool2d_strip_kernel(const T* __restrict__ x, const float* __restrict__ scale, co
     const int band = (int)(rest % bands);
     const int64_t plane = rest / bands;
     const int c = (int)(plane % C);
-    const float sc = scale != nullptr ? __ldg(scale + c) : 1.0f;
-    const float sf = shift != nullptr ? __ldg(shift + c) : 0.0f;
+    const float sc = scale.p != nullptr ? scale.at(c) : 1.0f;
+    const float sf = shift.p != nullptr ? shift.at(c) : 0.0f;
     const float relu = relu_flag ? 0.0f : -INFINITY;
     constexpr int P = KS == 3 ? 1 : 0;
     const int oh0 = band * band_rows, oh1 = min(OH, oh0 + band_rows);
@@ -386,7 +399,7 @@ __device__ __forceinline__ void store8(T* dst, const float (&o)[8])
 // R: input rows loaded per trip (all R loads are issued before the first is used).
 template <typename T, int MODE, int R>
 __global__ void __launch_bounds__(256)
-pool2d_strip_s1_kernel(const T* __restrict__ x, const float* __restrict__ scale, const float* __restrict__ shift,
+pool2d_strip_s1_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift,
                        T* __restrict__ y, int64_t strips, int C, int H, int W, int segs, int bands, int band_rows,
                        int relu_flag, float inv_area)
 {
@@ -399,8 +412,8 @@ pool2d_strip_s1_kernel(const T* __restrict__ x, const float* __restrict__ scale,
     const int band = (int)(rest % bands);
     const int64_t plane = rest / bands;
     const int c = (int)(plane % C);
-    const float sc = scale != nullptr ? __ldg(scale + c) : 1.0f;
-    const float sf = shift != nullptr ? __ldg(shift + c) : 0.0f;
+    const float sc = scale.p != nullptr ? scale.at(c) : 1.0f;
+    const float sf = shift.p != nullptr ? shift.at(c) : 0.0f;
     const float relu = relu_flag ? 0.0f : -INFINITY;
     const int oh0 = band * band_rows, oh1 = min(H, oh0 + band_rows);      // OH == H, OW == W
     const T* col = x + plane * H * (int64_t)W + seg * 8;
@@ -445,7 +458,7 @@ pool2d_strip_s1_kernel(const T* __restrict__ x, const float* __restrict__ scale,
 // KS: 3 or 2 for square windows of that size (taps unrolled), 0 for any window.
 template <typename T, int MODE, int KS>
 __global__ void __launch_bounds__(kPoolThreads)
-pool2d_planes_kernel(const T* __restrict__ x, const float* __restrict__ scale, const float* __restrict__ shift,
+pool2d_planes_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift,
                      T* __restrict__ y, int64_t planes, int G, int C, int H, int W, int OH, int OW, int kh, int kw,
                      int sh, int sw, int ph, int pw, float relu_floor, float inv_area)
 {
@@ -461,8 +474,8 @@ pool2d_planes_kernel(const T* __restrict__ x, const float* __restrict__ scale, c
     const T* xc = x + p0 * plane;
     for (int g = threadIdx.x; g < g_here; g += kPoolThreads) {
         const int c = (int)((p0 + g) % C);
-        sc_s[g] = scale != nullptr ? __ldg(scale + c) : 1.0f;
-        sf_s[g] = shift != nullptr ? __ldg(shift + c) : 0.0f;
+        sc_s[g] = scale.p != nullptr ? scale.at(c) : 1.0f;
+        sf_s[g] = shift.p != nullptr ? shift.at(c) : 0.0f;
     }
     __syncthreads();
     const float inv_plane = 1.0f / (float)plane;
@@ -570,7 +583,7 @@ __host__ __device__ __forceinline__ int walk_row_floats(int W, int OW, int pw, i
 
 template <typename T, int MODE, int KS, int ST, bool kPadW>
 __global__ void __launch_bounds__(kPoolThreads)
-pool2d_walk_kernel(const T* __restrict__ x, const float* __restrict__ scale, const float* __restrict__ shift,
+pool2d_walk_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift,
                    T* __restrict__ y, int64_t planes, int np, int C, int H, int W, int OH, int OW, int ph,
                    int band_rows, int bands, int chunks, int relu_flag, float inv_area)
 {
@@ -606,8 +619,8 @@ pool2d_walk_kernel(const T* __restrict__ x, const float* __restrict__ scale, con
     float* sf_s = sc_s + np;
     for (int q = threadIdx.x; q < nq; q += kPoolThreads) {
         const int c = (int)((p0 + q) % C);
-        sc_s[q] = scale != nullptr ? __ldg(scale + c) : 1.0f;
-        sf_s[q] = shift != nullptr ? __ldg(shift + c) : 0.0f;
+        sc_s[q] = scale.p != nullptr ? scale.at(c) : 1.0f;
+        sf_s[q] = shift.p != nullptr ? shift.at(c) : 0.0f;
     }
     // 1. padding cells: rows above / below the image, then the pw cells left and right of the image rows
     {
@@ -774,7 +787,7 @@ pool2d_walk_kernel(const T* __restrict__ x, const float* __restrict__ scale, con
 // Any geometry (rows too wide for the tile): one thread per output, window read from global memory.
 template <typename T>
 __global__ void __launch_bounds__(256)
-pool2d_direct_kernel(const T* __restrict__ x, const float* __restrict__ scale, const float* __restrict__ shift,
+pool2d_direct_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift,
                      T* __restrict__ y, int64_t total, int C, int H, int W, int OH, int OW, int kh, int kw, int sh,
                      int sw, int ph, int pw, int mode, int relu, float inv_area)
 {
@@ -783,8 +796,8 @@ pool2d_direct_kernel(const T* __restrict__ x, const float* __restrict__ scale, c
         const int oi = (int)((o / OW) % OH);
         const int64_t plane = o / ((int64_t)OW * OH);
         const int c = (int)(plane % C);
-        const float sc = scale != nullptr ? __ldg(scale + c) : 1.0f;
-        const float sf = shift != nullptr ? __ldg(shift + c) : 0.0f;
+        const float sc = scale.p != nullptr ? scale.at(c) : 1.0f;
+        const float sf = shift.p != nullptr ? shift.at(c) : 0.0f;
         const T* xp = x + plane * H * (int64_t)W;
         float res = mode == 0 ? -INFINITY : 0.0f;
         for (int di = 0; di < kh; ++di) {
@@ -803,7 +816,7 @@ pool2d_direct_kernel(const T* __restrict__ x, const float* __restrict__ scale, c
 
 template <typename T, int MODE, int KS, int ST>
 void launch_tile(bool vin, bool rowmap, unsigned grid, size_t smem, cudaStream_t stream, const T* x,
-                 const float* scale, const float* shift, T* y, int C, int H, int W, int OH, int OW, int kh, int kw,
+                 ParamVec scale, ParamVec shift, T* y, int C, int H, int W, int OH, int OW, int kh, int kw,
                  int sh, int sw, int ph, int pw, int band_rows, int bands, int relu, float inv_area)
 {
 #define KOP_POOL_GO(VI, RM)                                                                                         \
@@ -817,7 +830,7 @@ void launch_tile(bool vin, bool rowmap, unsigned grid, size_t smem, cudaStream_t
 }
 
 template <typename T>
-kop_status_t launch_pool(const void* xv, const float* scale, const float* shift, void* yv, int64_t N, int64_t C,
+kop_status_t launch_pool(const void* xv, ParamVec scale, ParamVec shift, void* yv, int64_t N, int64_t C,
                          int H, int W, int OH, int OW, int kh, int kw, int sh, int sw, int ph, int pw, int mode,
                          int relu, cudaStream_t stream)
 {
@@ -1018,13 +1031,14 @@ kop_status_t launch_pool(const void* xv, const float* scale, const float* shift,
 }  // namespace
 }  // namespace kop
 
-extern "C" kop_status_t kop_affine_relu_pool2d(const void* x, const float* scale, const float* shift, void* y,
-                                               int64_t N, int64_t C, int64_t H, int64_t W, int kh, int kw, int sh,
-                                               int sw, int ph, int pw, int mode, int relu, kop_dtype_t dtype,
-                                               kop_stream_t stream)
+namespace kop {
+namespace {
+
+kop_status_t pool_entry(const void* x, const void* scale, const void* shift, void* y, int64_t N, int64_t C, int64_t H,
+                        int64_t W, int kh, int kw, int sh, int sw, int ph, int pw, int mode, int relu, kop_dtype_t dtype,
+                        kop_dtype_t pdtype, kop_stream_t stream)
 {
-    using namespace kop;
-    if (!dtype_ok(dtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
+    if (!param_dtype_ok(dtype, pdtype)) return KOP_ERR_UNSUPPORTED_DTYPE;
     if (N < 0 || C <= 0 || H <= 0 || W <= 0) return KOP_ERR_BAD_SHAPE;
     if (kh <= 0 || kw <= 0 || sh <= 0 || sw <= 0 || ph < 0 || pw < 0 || ph > kh / 2 || pw > kw / 2)
         return KOP_ERR_BAD_SHAPE;
@@ -1037,7 +1051,8 @@ extern "C" kop_status_t kop_affine_relu_pool2d(const void* x, const float* scale
     if (!x || !y) return KOP_ERR_NULL_POINTER;
     if ((scale == nullptr) != (shift == nullptr)) return KOP_ERR_NULL_POINTER;      // both or neither
     const int esz = elem_size(dtype);
-    if (!aligned_to(x, esz) || !aligned_to(y, esz) || (scale && !aligned_to(scale, 4)) || (shift && !aligned_to(shift, 4)))
+    if (!aligned_to(x, esz) || !aligned_to(y, esz) || (scale && !aligned_to(scale, elem_size(pdtype))) ||
+        (shift && !aligned_to(shift, elem_size(pdtype))))
         return KOP_ERR_MISALIGNED;
     const int64_t OH = (H + 2 * (int64_t)ph - kh) / sh + 1, OW = (W + 2 * (int64_t)pw - kw) / sw + 1;
     {
@@ -1049,10 +1064,31 @@ extern "C" kop_status_t kop_affine_relu_pool2d(const void* x, const float* scale
     kop_status_t st = check_device();
     if (st != KOP_OK) return st;
     cudaStream_t s = as_stream(stream);
-    return dtype == KOP_F32 ? launch_pool<float>(x, scale, shift, y, N, C, (int)H, (int)W, (int)OH, (int)OW, kh, kw, sh,
-                                                 sw, ph, pw, mode, relu != 0, s)
-                            : dtype == KOP_BF16 ? launch_pool<__nv_bfloat16>(x, scale, shift, y, N, C, (int)H, (int)W, (int)OH, (int)OW, kh,
-                                                         kw, sh, sw, ph, pw, mode, relu != 0, s)
-                            : launch_pool<__half>(x, scale, shift, y, N, C, (int)H, (int)W, (int)OH, (int)OW, kh,
-                                                         kw, sh, sw, ph, pw, mode, relu != 0, s);
+    const ParamVec sc{scale, (int)pdtype}, sf{shift, (int)pdtype};
+    return dtype == KOP_F32 ? launch_pool<float>(x, sc, sf, y, N, C, (int)H, (int)W, (int)OH, (int)OW, kh, kw, sh, sw, ph, pw,
+                                                 mode, relu != 0, s)
+           : dtype == KOP_BF16
+               ? launch_pool<__nv_bfloat16>(x, sc, sf, y, N, C, (int)H, (int)W, (int)OH, (int)OW, kh, kw, sh, sw, ph, pw, mode,
+                                            relu != 0, s)
+               : launch_pool<__half>(x, sc, sf, y, N, C, (int)H, (int)W, (int)OH, (int)OW, kh, kw, sh, sw, ph, pw, mode,
+                                     relu != 0, s);
+}
+
+}  // namespace
+}  // namespace kop
+
+extern "C" kop_status_t kop_affine_relu_pool2d(const void* x, const float* scale, const float* shift, void* y,
+                                               int64_t N, int64_t C, int64_t H, int64_t W, int kh, int kw, int sh,
+                                               int sw, int ph, int pw, int mode, int relu, kop_dtype_t dtype,
+                                               kop_stream_t stream)
+{
+    return kop::pool_entry(x, scale, shift, y, N, C, H, W, kh, kw, sh, sw, ph, pw, mode, relu, dtype, KOP_F32, stream);
+}
+
+extern "C" kop_status_t kop_affine_relu_pool2d_ex(const void* x, const void* scale, const void* shift, void* y,
+                                                  int64_t N, int64_t C, int64_t H, int64_t W, int kh, int kw, int sh,
+                                                  int sw, int ph, int pw, int mode, int relu, kop_dtype_t dtype,
+                                                  kop_dtype_t param_dtype, kop_stream_t stream)
+{
+    return kop::pool_entry(x, scale, shift, y, N, C, H, W, kh, kw, sh, sw, ph, pw, mode, relu, dtype, param_dtype, stream);
 }

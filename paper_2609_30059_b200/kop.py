@@ -88,6 +88,8 @@ def lib() -> C.CDLL:
     L.kop_groupnorm_act.restype = i32
     L.kop_affine_relu_pool2d.argtypes = [vp] * 4 + [i64] * 4 + [i32] * 9 + [vp]
     L.kop_affine_relu_pool2d.restype = i32
+    L.kop_affine_relu_pool2d_ex.argtypes = [vp] * 4 + [i64] * 4 + [i32] * 10 + [vp]
+    L.kop_affine_relu_pool2d_ex.restype = i32
     L.kop_reduce_rows.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, vp]
     L.kop_reduce_rows.restype = i32
     L.kop_bias_act.argtypes = [vp, vp, vp, i64, i64, i64, i64, i32, f32, i32, vp]
@@ -591,6 +593,23 @@ def kop_affine_relu_pool2d(x, scale, shift, kernel, stride, padding, mode="max",
                                         out.data_ptr(), N, Cc, H, W, kh, kw, sh, sw, ph, pw,
                                         {"max": 0, "avg": 1}[mode], int(bool(relu)), _dtype_tag(x), _stream(stream)),
            "kop_affine_relu_pool2d")
+    return out
+
+
+def kop_affine_relu_pool2d_ex(x, scale, shift, kernel, stride, padding, mode="max", relu=True, out=None, stream=None):
+    """kop_affine_relu_pool2d with scale / shift in fp32 or in x.dtype."""
+    if x.dim() != 4 or not x.is_cuda or not x.is_contiguous():
+        raise ValueError("x: expected a contiguous 4-D NCHW CUDA tensor")
+    N, Cc, H, W = x.shape
+    (kh, kw), (sh, sw), (ph, pw) = kernel, stride, padding
+    OH, OW = (H + 2 * ph - kh) // sh + 1, (W + 2 * pw - kw) // sw + 1
+    out = torch.empty((N, Cc, max(OH, 0), max(OW, 0)), dtype=x.dtype, device=x.device) if out is None else out
+    if out.dtype != x.dtype or not out.is_contiguous():
+        raise ValueError("out: expected a contiguous tensor of x's dtype")
+    (sp, hp), ptag = _params_any(x, Cc, scale=scale, shift=shift)
+    _check(lib().kop_affine_relu_pool2d_ex(x.data_ptr(), sp, hp, out.data_ptr(), N, Cc, H, W, kh, kw, sh, sw, ph, pw,
+                                           {"max": 0, "avg": 1}[mode], int(bool(relu)), _dtype_tag(x), ptag,
+                                           _stream(stream)), "kop_affine_relu_pool2d_ex")
     return out
 
 

@@ -64,7 +64,7 @@ def test_all_entry_points_in_one_graph(kop):
         "ceo_sum": torch.empty(1, device=dev), "softmax_ex": torch.empty_like(x), "act_ex": torch.empty_like(x),
         "chain_ex": torch.empty_like(x), "bn_ex": torch.empty_like(img16), "bn_ex_p": torch.empty((3, 16), device=dev),
         "gn_ex": torch.empty_like(img16), "pool_s1": torch.empty((3, 16, 28, 28), device=dev),
-        "pool_walk": torch.empty((3, 16, 27, 27), device=dev),
+        "pool_walk": torch.empty((3, 16, 27, 27), device=dev), "pool_ex": torch.empty((3, 16, 14, 14), dtype=BF16, device=dev),
     }
 
     def run():
@@ -105,6 +105,7 @@ def test_all_entry_points_in_one_graph(kop):
         kop.kop_groupnorm_act_ex(img16, sc16, sh16, 4, 1e-5, 1, out=o["gn_ex"], want_stats=False)
         kop.kop_affine_relu_pool2d(img, sc, sh, (3, 3), (1, 1), (1, 1), "avg", True, out=o["pool_s1"])
         kop.kop_affine_relu_pool2d(img, sc, sh, (2, 2), (1, 1), (0, 0), "max", False, out=o["pool_walk"])
+        kop.kop_affine_relu_pool2d_ex(img16, sc16, sh16, (3, 3), (2, 2), (1, 1), "max", True, out=o["pool_ex"])
         kop.kop_rmsnorm_swiglu_residual(handle, h, w, W1, W2, 1e-6, out=o["mlp"], workspace=ws_mlp)
 
     try:

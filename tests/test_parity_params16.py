@@ -205,6 +205,41 @@ def test_bias_act_and_chain_ex_16_bit_bias(kop, rows, cols, dtype, seed):
     assert torch.equal(kop.kop_bias_act_ex(x, None, "relu"), kop.kop_bias_act(x, None, "relu"))
 
 
+# one geometry per pooling kernel: stride-2 strip, stride-1 strip, shared-memory walk, runs of small planes, generic
+# tile, direct (rows too wide for a tile)
+POOL_EX_CASES = [
+    (2, 8, 112, 112, (3, 3), (2, 2), (1, 1), BF16),
+    (1, 3, 57, 64, (3, 3), (1, 1), (1, 1), F16),
+    (2, 3, 57, 57, (3, 3), (1, 1), (1, 1), BF16),
+    (5, 37, 7, 7, (3, 3), (2, 2), (1, 1), F16),
+    (3, 50, 14, 14, (3, 3), (2, 2), (1, 1), BF16),
+    (2, 3, 30, 44, (5, 3), (2, 1), (2, 1), F16),
+    (1, 2, 6, 5000, (3, 3), (2, 2), (1, 1), BF16),
+]
+
+
+@pytest.mark.parametrize("N,C,H,W,kernel,stride,padding,dtype", POOL_EX_CASES)
+@pytest.mark.parametrize("seed", SEEDS)
+def test_affine_relu_pool2d_ex_16_bit_scale_shift(kop, N, C, H, W, kernel, stride, padding, dtype, seed):
+    x, sc, sh = synth.bn_pool_inputs(N, C, H, W, dtype, seed, "cuda")
+    sc16, sh16 = sc.to(dtype), sh.to(dtype)
+    tol = tol_of(dtype)
+    OH = (H + 2 * padding[0] - kernel[0]) // stride[0] + 1
+    OW = (W + 2 * padding[1] - kernel[1]) // stride[1] + 1
+    for mode in ("max", "avg"):
+        for relu in (True, False):
+            y = Guarded((N, C, OH, OW), dtype)
+            kop.kop_affine_relu_pool2d_ex(x, sc16, sh16, kernel, stride, padding, mode, relu, out=y.t)
+            ref = kopref.affine_relu_pool2d(host(x), host(sc16), host(sh16), kernel, stride, padding, mode, relu, threads=None)
+            assert_close(y.t, ref, tol, f"pool2d_ex {mode} relu={relu}")
+            y.check("pool2d_ex")
+        # fp32 parameters and no parameters through the new entry point: bit-equal to the base entry point
+        assert torch.equal(kop.kop_affine_relu_pool2d_ex(x, sc, sh, kernel, stride, padding, mode, True),
+                           kop.kop_affine_relu_pool2d(x, sc, sh, kernel, stride, padding, mode, True))
+        assert torch.equal(kop.kop_affine_relu_pool2d_ex(x, None, None, kernel, stride, padding, mode, False),
+                           kop.kop_affine_relu_pool2d(x, None, None, kernel, stride, padding, mode, False))
+
+
 def test_ex_entry_points_misaligned_parameters_and_type_rules(kop):
     rows, cols = 40, 2048
     x, bias = synth.softmax_inputs(rows, cols, BF16, 2, "cuda")
@@ -226,3 +261,9 @@ def test_ex_entry_points_misaligned_parameters_and_type_rules(kop):
     assert L.kop_bias_act_ex(P, Q, R, 4, 8, 8, 8, 1, 0.0, 2, 1, None) == 4
     assert L.kop_epilogue_chain_ex(P, Q, None, R, 4, 8, 8, 8, 8, 1.0, 1.0, -1.0, 1.0, 0, 0.0, 1, 7, None) == 4
     assert L.kop_softmax_ex(P, Q + 1, R, 4, 8, 8, 8, 1.0, 0, 0, 1, 1, None) == 5      # bias not on a 2-byte boundary
+    pool = (1, 2, 8, 8, 3, 3, 2, 2, 1, 1, 0, 1)
+    assert L.kop_affine_relu_pool2d_ex(P, Q, Q, R, *pool, 0, 1, None) == 4            # fp32 data, bf16 params
+    assert L.kop_affine_relu_pool2d_ex(P, Q, Q, R, *pool, 2, 1, None) == 4            # fp16 data, bf16 params
+    assert L.kop_affine_relu_pool2d_ex(P, Q, Q + 1, R, *pool, 1, 1, None) == 5        # shift not on a 2-byte boundary
+    assert L.kop_affine_relu_pool2d_ex(P, Q, Q + 2, R, *pool, 1, 0, None) == 5        # fp32 shift on a 2-byte boundary
+    assert L.kop_affine_relu_pool2d_ex(P, Q, None, R, *pool, 1, 1, None) == 1         # scale without shift
