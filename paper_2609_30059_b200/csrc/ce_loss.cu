@@ -12,6 +12,10 @@
 
 #include "kop_common.cuh"
 
+#ifndef KOP_CE_PACKED
+#define KOP_CE_PACKED 1
+#endif
+
 namespace kop {
 namespace {
 
@@ -214,6 +218,26 @@ __device__ __forceinline__ void ce_batch(const T* zr, int base, int nvec, float&
         const float newM = fmaxf(M, cm2);
         float s = S * ex2_approx(M - newM);          // M = -inf on the first batch: S * 0
         const float neg = -newM;
+#if KOP_CE_PACKED
+        float2 s2 = make_float2(s, 0.0f), z2 = make_float2(Z, 0.0f);
+        const float2 l2 = make_float2(kLog2e, kLog2e), n2 = make_float2(neg, neg);
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            float2 f[E / 2];
+            Elem<T>::unpack2(raw[k], f);
+#pragma unroll
+            for (int e = 0; e < E / 2; ++e) {
+                const float2 t = __ffma2_rn(f[e], l2, n2);
+                s2 = __fadd2_rn(s2, make_float2(ex2_approx(t.x), ex2_approx(t.y)));
+            }
+            if (kSum && (!kTail || base + k * (int)blockDim.x + (int)threadIdx.x < nvec)) {
+#pragma unroll
+                for (int e = 0; e < E / 2; ++e) z2 = __fadd2_rn(z2, f[e]);
+            }
+        }
+        s = s2.x + s2.y;
+        if (kSum) Z = z2.x + z2.y;
+#else
 #pragma unroll
         for (int k = 0; k < VPT; ++k) {
             float f[E];
@@ -226,6 +250,7 @@ __device__ __forceinline__ void ce_batch(const T* zr, int base, int nvec, float&
                 for (int e = 0; e < E; e += 2) Z += f[e] + f[e + 1];
             }
         }
+#endif
         S = s;
         M = newM;
     }

@@ -456,14 +456,17 @@ pool2d_strip_s1_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift,
 // plane's scale / shift, then one thread per output over the whole run, windows read from shared memory with
 // bounds checks, outputs (contiguous for the run) stored by consecutive threads.
 // KS: 3 or 2 for square windows of that size (taps unrolled), 0 for any window.
-template <typename T, int MODE, int KS>
-__global__ void __launch_bounds__(kPoolThreads)
+// kFixed (stride-1 windows, where outputs are as many as inputs and their index arithmetic was most of the kernel):
+// thread t keeps one output position of the plane for the whole run (see the output loop).
+template <typename T, int MODE, int KS, bool kFixed>
+__global__ void __launch_bounds__(kPoolThreads, kFixed ? 6 : 0)
 pool2d_planes_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift,
-                     T* __restrict__ y, int64_t planes, int G, int C, int H, int W, int OH, int OW, int kh, int kw,
+                     T* __restrict__ y, int64_t planes, int G, int Gp, int C, int H, int W, int OH, int OW, int kh, int kw,
                      int sh, int sw, int ph, int pw, float relu_floor, float inv_area)
 {
     constexpr int E = Elem<T>::kPerVec;
     extern __shared__ __align__(16) float planes_smem[];
+    const int nthreads = kFixed ? (int)blockDim.x : kPoolThreads;    // the fixed-position CTA is trimmed to whole passes
     const int plane = H * W, oplane = OH * OW;
     float* act = planes_smem;
     float* sc_s = act + G * plane;
@@ -472,7 +475,7 @@ pool2d_planes_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift,
     const int g_here = (int)(planes - p0 < G ? planes - p0 : G);
     const int elems = g_here * plane;
     const T* xc = x + p0 * plane;
-    for (int g = threadIdx.x; g < g_here; g += kPoolThreads) {
+    for (int g = threadIdx.x; g < g_here; g += nthreads) {
         const int c = (int)((p0 + g) % C);
         sc_s[g] = scale.p != nullptr ? scale.at(c) : 1.0f;
         sf_s[g] = shift.p != nullptr ? shift.at(c) : 0.0f;
@@ -481,16 +484,16 @@ pool2d_planes_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift,
     const float inv_plane = 1.0f / (float)plane;
     const int nvec = elems / E;
     constexpr int U = 4;                                     // loads in flight per thread
-    for (int base = 0; base < nvec; base += U * kPoolThreads) {
+    for (int base = 0; base < nvec; base += U * nthreads) {
         Vec16 raw[U];
 #pragma unroll
         for (int k = 0; k < U; ++k) {
-            const int v = base + k * kPoolThreads + threadIdx.x;
+            const int v = base + k * nthreads + threadIdx.x;
             if (v < nvec) raw[k] = ld_stream(xc + (int64_t)v * E);
         }
 #pragma unroll
         for (int k = 0; k < U; ++k) {
-            const int v = base + k * kPoolThreads + threadIdx.x;
+            const int v = base + k * nthreads + threadIdx.x;
             if (v < nvec) {
                 float f[E];
                 Elem<T>::unpack(raw[k], f);
@@ -511,7 +514,7 @@ pool2d_planes_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift,
             }
         }
     }
-    for (int i = nvec * E + threadIdx.x; i < elems; i += kPoolThreads) {     // the tensor's last run may end inside a vector
+    for (int i = nvec * E + threadIdx.x; i < elems; i += nthreads) {     // the tensor's last run may end inside a vector
         const int pl = i / plane;
         act[i] = act_of(Elem<T>::load1(xc + i), sc_s[pl], sf_s[pl], relu_floor);
     }
@@ -519,7 +522,56 @@ pool2d_planes_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift,
     const float inv_oplane = 1.0f / (float)oplane, inv_ow = 1.0f / (float)OW;
     T* yc = y + p0 * oplane;
     const int n_out = g_here * oplane;
-    for (int o = threadIdx.x; o < n_out; o += kPoolThreads) {
+    if (kFixed) {
+        // Plane slot t / oplane of each pass of Gp planes, position t % oplane. The window geometry is worked out
+        // once: clamped tap offsets (a clamped tap repeats an element of the same window, which leaves a maximum
+        // unchanged and is masked out of a sum), so a pass costs the taps and a store, with no index division and no
+        // bounds predicate per output. The CTA is trimmed to the warps that have a position.
+        const int slot = (int)threadIdx.x / oplane;
+        const int r = (int)threadIdx.x - slot * oplane;
+        if (slot >= Gp) return;
+        const int oi = r / OW, oj = r - oi * OW;
+        const int i_lo = oi * sh - ph, j_lo = oj * sw - pw;
+        int off[KS ? KS : 1][KS ? KS : 1];
+        unsigned rm[KS ? KS : 1], cm[KS ? KS : 1];
+#pragma unroll
+        for (int d = 0; d < KS; ++d) {
+            rm[d] = (unsigned)(i_lo + d) < (unsigned)H ? 0xFFFFFFFFu : 0u;
+            cm[d] = (unsigned)(j_lo + d) < (unsigned)W ? 0xFFFFFFFFu : 0u;
+        }
+#pragma unroll
+        for (int di = 0; di < KS; ++di)
+#pragma unroll
+            for (int dj = 0; dj < KS; ++dj)
+                off[di][dj] = min(max(i_lo + di, 0), H - 1) * W + min(max(j_lo + dj, 0), W - 1);
+        const float* a = act + slot * plane;
+        T* yo = yc + threadIdx.x;
+        const int a_step = Gp * plane, o_step = Gp * oplane;
+        for (int g = slot; g < g_here; g += Gp, a += a_step, yo += o_step) {
+            float res;
+            if (MODE == 0) {
+                res = a[off[0][0]];
+#pragma unroll
+                for (int di = 0; di < KS; ++di)
+#pragma unroll
+                    for (int dj = 0; dj < KS; ++dj)
+                        if (di + dj > 0) res = max_keep_nan(res, a[off[di][dj]]);
+            } else {
+                res = 0.0f;
+#pragma unroll
+                for (int di = 0; di < KS; ++di) {
+                    float rs = __uint_as_float(__float_as_uint(a[off[di][0]]) & cm[0]);
+#pragma unroll
+                    for (int dj = 1; dj < KS; ++dj) rs += __uint_as_float(__float_as_uint(a[off[di][dj]]) & cm[dj]);
+                    res += __uint_as_float(__float_as_uint(rs) & rm[di]);
+                }
+                res *= inv_area;
+            }
+            Elem<T>::store1(yo, res);
+        }
+        return;
+    }
+    for (int o = threadIdx.x; o < n_out; o += nthreads) {
         const int g = div_small(o, oplane, inv_oplane);
         const int r = o - g * oplane;
         const int oi = div_small(r, OW, inv_ow), oj = r - oi * OW;
@@ -953,18 +1005,32 @@ kop_status_t launch_pool(const void* xv, ParamVec scale, ParamVec shift, void* y
         const size_t smem = ((size_t)G * plane + 2 * (size_t)G) * sizeof(float);
         if (ctas <= 0x7FFFFFFFLL && smem <= (size_t)kPoolTileMax && (int64_t)G * plane < (1 << 22)) {
             const float floor_v = relu ? 0.0f : -INFINITY;
-#define KOP_POOL_PLANES(M, K) \
-    pool2d_planes_kernel<T, M, K><<<(unsigned)ctas, kPoolThreads, smem, stream>>>(x, scale, shift, y, planes, G, (int)C, H, W, OH, OW, kh, kw, sh, sw, ph, pw, floor_v, inv_area)
             const int ks = (kh == kw && (kh == 2 || kh == 3)) ? kh : 0;
+            // stride-1 2 x 2 / 3 x 3 windows with at most a CTA's worth of outputs per plane: one fixed output
+            // position per thread, Gp planes per pass (14 x 14 fp32 3 x 3 / 1 max: 2.4 -> 3.5 TB/s, 7 x 7: 2.4 -> 3.1,
+            // 4 x 4: 1.9 -> 2.9; at stride 2 the outputs are a quarter of the inputs and the extra registers of the
+            // fixed geometry cost more occupancy than the loop saves: 2.9 -> 2.7, so those keep the plain loop)
+            const int oplane = OH * OW;
+            const bool fixed = ks != 0 && sh == 1 && sw == 1 && oplane <= kPoolThreads;
+            const int Gp = fixed ? kPoolThreads / oplane : 0;
+            const int threads = fixed ? (Gp * oplane + 31) / 32 * 32 : kPoolThreads;
+#define KOP_POOL_PLANES(M, K, F) \
+    pool2d_planes_kernel<T, M, K, F><<<(unsigned)ctas, threads, smem, stream>>>(x, scale, shift, y, planes, G, Gp, (int)C, H, W, OH, OW, kh, kw, sh, sw, ph, pw, floor_v, inv_area)
+#define KOP_POOL_PLANES_F(M, K)             \
+    do {                                    \
+        if (fixed) KOP_POOL_PLANES(M, K, true); \
+        else KOP_POOL_PLANES(M, K, false);  \
+    } while (0)
             if (mode == 0) {
-                if (ks == 3) KOP_POOL_PLANES(0, 3);
-                else if (ks == 2) KOP_POOL_PLANES(0, 2);
-                else KOP_POOL_PLANES(0, 0);
+                if (ks == 3) KOP_POOL_PLANES_F(0, 3);
+                else if (ks == 2) KOP_POOL_PLANES_F(0, 2);
+                else KOP_POOL_PLANES(0, 0, false);
             } else {
-                if (ks == 3) KOP_POOL_PLANES(1, 3);
-                else if (ks == 2) KOP_POOL_PLANES(1, 2);
-                else KOP_POOL_PLANES(1, 0);
+                if (ks == 3) KOP_POOL_PLANES_F(1, 3);
+                else if (ks == 2) KOP_POOL_PLANES_F(1, 2);
+                else KOP_POOL_PLANES(1, 0, false);
             }
+#undef KOP_POOL_PLANES_F
 #undef KOP_POOL_PLANES
             return launch_status();
         }
