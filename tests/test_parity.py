@@ -522,7 +522,8 @@ def test_ce_options(kop):
 # ------------------------------------------------------------------------------------------ MLP pieces
 
 RMS_SHAPES = [(2048, 4096, BF16), (300, 4096, F32), (65, 512, BF16), (17, 16384, BF16),
-              (9, 20480, F32), (5, 40008, BF16), (3, 20481, BF16), (21, 1001, BF16), (7, 1, F32)]
+              (9, 20480, F32), (5, 40008, BF16), (3, 20481, BF16), (21, 1001, BF16), (7, 1, F32),
+              (19, 12288, BF16), (7, 10000, BF16)]       # packed rows with fp32 weights: 384 threads, and a ragged 320
 
 
 @pytest.mark.parametrize("rows,hidden,dtype", RMS_SHAPES)

@@ -61,7 +61,9 @@ def test_layernorm_ex_16_bit_parameters(kop, rows, hidden, dtype, seed):
 
 
 @pytest.mark.parametrize("rows,hidden,dtype", [(600, 4096, BF16), (40, 4096, F16), (33, 1000, BF16), (17, 1001, F16),
-                                               (5, 24576, F16)])
+                                               (5, 24576, F16),
+                                               # rows kept packed in registers: exact (384 / 512 threads) and ragged
+                                               (19, 12288, BF16), (11, 16384, F16), (7, 10000, BF16)])
 @pytest.mark.parametrize("seed", SEEDS)
 def test_rmsnorm_ex_16_bit_parameters(kop, rows, hidden, dtype, seed):
     x, r, _, g, _ = synth.layernorm_inputs(rows, hidden, dtype, seed, "cuda")
