@@ -89,6 +89,8 @@ def segment_bytes():
     out["matvec_bias"] = dict(bytes=v["rows"] * v["k"] * 2 + v["k"] * 4 + v["rows"] * 4, elems=v["rows"] * v["k"])
     out["residual_layernorm"] = dict(bytes=3 * n["rows"] * n["hidden"] * 2 + 2 * n["hidden"] * 4 + 2 * n["rows"] * 4,
                                      elems=n["rows"] * n["hidden"])
+    out["layernorm_plain"] = dict(bytes=2 * n["rows"] * n["hidden"] * 2 + 2 * n["hidden"] * 4 + 2 * n["rows"] * 4,
+                                  elems=n["rows"] * n["hidden"])
     out["layernorm_params16"] = dict(bytes=3 * n["rows"] * n["hidden"] * 2 + 3 * n["hidden"] * 2 + 2 * n["rows"] * 4,
                                      elems=n["rows"] * n["hidden"])
     out["silu_mul_interleaved"] = dict(out["silu_mul"])
@@ -268,7 +270,7 @@ class Workload:
 
     ORDER = ["softmax_small", "softmax_large", "layernorm", "bn_pool", "ce_loss", "rmsnorm", "silu_mul", "residual_add"]
     # Beyond the benchmark configs (not part of `value`): the two kernels the paper's case studies print.
-    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "layernorm_params16", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc", "pool2d", "pool2d_s1", "pool2d_14", "reduce_max", "reduce_logsumexp", "bias_gelu", "residual_rmsnorm", "l2_normalize", "lstm_cell", "gru_cell", "rmsnorm_head128", "softmax_vocab"]
+    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "layernorm_plain", "layernorm_params16", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc", "pool2d", "pool2d_s1", "pool2d_14", "reduce_max", "reduce_logsumexp", "bias_gelu", "residual_rmsnorm", "l2_normalize", "lstm_cell", "gru_cell", "rmsnorm_head128", "softmax_vocab"]
 
     def __init__(self, kop, device, seed, only=None, rows_div=1):
         """only: build just these segments (None = all, plus the MLP segment); rows_div cuts the row
@@ -288,7 +290,7 @@ class Workload:
             L = c["softmax_large"]
             self.lx, self.lb = synth.softmax_inputs(cut(L["rows"]), L["cols"], L["dtype"], seed, dev)
             self.ly = torch.empty_like(self.lx)
-        if want & {"layernorm", "residual_layernorm", "layernorm_params16"}:
+        if want & {"layernorm", "residual_layernorm", "layernorm_plain", "layernorm_params16"}:
             n = c["layernorm"]
             self.nx, self.nr, self.nb, self.ng, self.nbe = synth.layernorm_inputs(cut(n["rows"]), n["hidden"], n["dtype"], seed, dev)
             self.ny = torch.empty_like(self.nx)
@@ -433,6 +435,9 @@ class Workload:
             k.kop_matvec_bias(self.vx, self.vw, self.vb, out=self.vo)
         elif name == "residual_layernorm":       # same tensors and shape as the LayerNorm config, no bias / GELU
             k.kop_residual_layernorm(self.nx, self.nr, self.ng, self.nbe, c["layernorm"]["eps"], out=self.ny,
+                                     mean=self.nmean, rstd=self.nrstd)
+        elif name == "layernorm_plain":          # LayerNorm(x) alone on the same shape: one input stream, fp32 gamma / beta
+            k.kop_residual_layernorm(self.nx, None, self.ng, self.nbe, c["layernorm"]["eps"], out=self.ny,
                                      mean=self.nmean, rstd=self.nrstd)
         elif name == "layernorm_params16":       # the LayerNorm config with bias / gamma / beta stored in bf16
             k.kop_layernorm_ex(self.nx, self.nr, *self.np16, c["layernorm"]["eps"], "bias_gelu_residual", out=self.ny,
