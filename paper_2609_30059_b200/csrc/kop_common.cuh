@@ -318,6 +318,10 @@ struct Elem<__nv_bfloat16> {
             : "=f"(r.x), "=f"(r.y) : "r"(w), "f"(c.x), "f"(c.y));
         return r;
     }
+    __device__ __forceinline__ static void unpack_pair(uint32_t w, float2& f)
+    {
+        f = make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u));
+    }
     __device__ __forceinline__ static float load1(const __nv_bfloat16* p) { return __bfloat162float(*p); }
     __device__ __forceinline__ static void store1(__nv_bfloat16* p, float f) { *p = __float2bfloat16_rn(f); }
     __device__ __forceinline__ static Vec16 fill_neg_inf()
@@ -374,6 +378,10 @@ struct Elem<__half> {
         asm("{ .reg .b16 lo, hi; mov.b32 {lo, hi}, %2; add.rn.f32.f16 %0, lo, %3; add.rn.f32.f16 %1, hi, %4; }"
             : "=f"(r.x), "=f"(r.y) : "r"(w), "f"(c.x), "f"(c.y));
         return r;
+    }
+    __device__ __forceinline__ static void unpack_pair(uint32_t w, float2& f)
+    {
+        f = __half22float2(*reinterpret_cast<const __half2*>(&w));
     }
     __device__ __forceinline__ static float load1(const __half* p) { return __half2float(*p); }
     __device__ __forceinline__ static void store1(__half* p, float f) { *p = __float2half_rn(f); }

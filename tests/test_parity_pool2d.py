@@ -70,6 +70,16 @@ POOL_CASES = [
     (1, 1, 301, 97, (3, 3), (2, 2), (1, 1), BF16),
     (3, 7, 28, 28, (3, 3), (1, 1), (1, 1), F32),                   # runs of whole small planes through the same kernel
     (5, 3, 23, 31, (2, 2), (1, 1), (0, 0), BF16),
+    # 2x2 / stride 2 without padding, a thread per output: pair loads (even width), scalar loads (odd width), an odd
+    # height (the last row is never read), one-output planes, a CTA's worth of outputs that ends inside a plane
+    (5, 37, 14, 14, (2, 2), (2, 2), (0, 0), F32),
+    (3, 50, 28, 28, (2, 2), (2, 2), (0, 0), BF16),
+    (6, 11, 7, 7, (2, 2), (2, 2), (0, 0), F32),
+    (2, 3, 57, 57, (2, 2), (2, 2), (0, 0), BF16),
+    (3, 5, 15, 14, (2, 2), (2, 2), (0, 0), torch.float16),
+    (9, 13, 2, 2, (2, 2), (2, 2), (0, 0), F32),
+    (2, 3, 3, 2, (2, 2), (2, 2), (0, 0), BF16),
+    (1, 2, 60, 60, (2, 2), (2, 2), (0, 0), F32),
 ]
 
 
@@ -108,6 +118,23 @@ def test_pool2d_full_config_seed0(kop):
     g = kop.kop_affine_relu_pool2d(xs, scale, shift, (14, 14), (1, 1), (0, 0), "avg", True)
     _, pooled = kop.kop_bn_relu_avgpool(xs, scale, shift)
     assert float((g[:, :, 0, 0] - pooled).abs().max()) < 1e-5
+
+
+def test_pool2d_k2s2_unaligned_base(kop):
+    """2x2 / stride 2 on a tensor that starts one element into its buffer: the pair loads are not aligned, the scalar
+    loads take over; same results."""
+    for dtype in (F32, BF16):
+        x, scale, shift = synth.bn_pool_inputs(3, 5, 14, 14, dtype, 11, "cuda")
+        buf = torch.empty(x.numel() + 1, dtype=dtype, device="cuda")
+        xs = buf[1:].view(x.shape)
+        xs.copy_(x)
+        for mode in ("max", "avg"):
+            a = kop.kop_affine_relu_pool2d(x, scale, shift, (2, 2), (2, 2), (0, 0), mode, True)
+            b = kop.kop_affine_relu_pool2d(xs, scale, shift, (2, 2), (2, 2), (0, 0), mode, True)
+            ref = kopref.affine_relu_pool2d(host(x), host(scale), host(shift), (2, 2), (2, 2), (0, 0), mode, True)
+            assert_close(a, ref, tol_of(dtype), f"k2s2 aligned {mode}")
+            assert_close(b, ref, tol_of(dtype), f"k2s2 unaligned {mode}")
+            assert torch.equal(a, b)
 
 
 def test_pool2d_options(kop):
