@@ -362,10 +362,10 @@ kop_status_t launch_softmax(const void* xv, const void* biasv, void* yv, int64_t
         return launch_status();
     }
     if (rows > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
-    // 16-bit rows up to 32 KB and fp32 rows up to 16 KB stay in one CTA's registers; longer ones take the two-sweep
-    // kernel (fp32 rows of 8192 / 16384 columns: 4.3 / 3.6 TB/s in registers, 4.8 / 5.5 TB/s in two sweeps with the L2
-    // eviction hints; bf16 rows of 16384 columns: 4.6 in registers against 4.0)
-    if (vec && cols <= kMaxRegisterRow && cols * (int64_t)sizeof(T) <= (sizeof(T) == 4 ? 16384 : 32768)) {
+    // rows up to 32 KB stay in one CTA's registers; longer ones take the two-sweep kernel (fp32 rows of 8192 columns:
+    // 5.1 TB/s in two sweeps, 6.5 in registers with 32 values a thread; of 16384 columns 5.7 either way; bf16 rows of
+    // 16384 columns: 4.7 in registers against 4.0)
+    if (vec && cols <= kMaxRegisterRow && cols * (int64_t)sizeof(T) <= 32768) {
         const int nvec = (int)nvec64;
         // Per-thread vector count: 16 values per thread while the CTA stays within 1024 threads
         // keeps many CTAs resident; longer rows double the count (and halve the CTA limit).
