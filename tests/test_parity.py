@@ -69,6 +69,21 @@ def test_softmax_parity(kop, rows, cols, dtype, seed):
     assert np.all(np.abs(sums - 1.0) <= (1e-5 if dtype == F32 else 2e-2))
 
 
+@pytest.mark.parametrize("rows,cols,dtype", [(257, 2048, F32), (129, 4096, BF16), (19, 8192, F32), (33, 16384, BF16),
+                                             (65, 3072, torch.float16), (40, 2056, BF16), (1500, 1032, F32)])
+@pytest.mark.parametrize("seed", SEEDS[:3])
+def test_softmax_no_bias_block_rows(kop, rows, cols, dtype, seed):
+    """Rows in one CTA's registers without a bias: exact rows take the predicate-free variant (32 values a thread from
+    2048 columns, fp32 rows up to 32 KB), ragged ones the general form."""
+    x, _ = synth.softmax_inputs(rows, cols, dtype, seed, "cuda")
+    out = Guarded((rows, cols), dtype)
+    kop.kop_softmax_scale_bias(x, None, 0.5, out=out.t)
+    ref = kopref.softmax_scale_bias(host(x), None, 0.5, threads=None)
+    assert_close(out.t, ref, tol_of(dtype), "softmax no bias")
+    out.check("softmax no bias")
+    assert torch.equal(out.t, kop.kop_softmax_scale_bias(x, None, 0.5))
+
+
 def test_softmax_large_config_seed0(kop):
     c = synth.CONFIGS["softmax_large"]
     x, bias = synth.softmax_inputs(c["rows"], c["cols"], c["dtype"], 0, "cuda")
