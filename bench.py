@@ -123,6 +123,8 @@ def segment_bytes():
     out["rmsnorm_head128"] = dict(bytes=2 * q["rows"] * q["hidden"] * 2 + q["hidden"] * 4, elems=q["rows"] * q["hidden"])
     q = c["softmax_vocab"]
     out["softmax_vocab"] = dict(bytes=2 * q["rows"] * q["cols"] * 2, elems=q["rows"] * q["cols"])
+    q = c["softmax_4096"]
+    out["softmax_4096"] = dict(bytes=2 * q["rows"] * q["cols"] * 2, elems=q["rows"] * q["cols"])
     t = c["gru_cell"]
     out["gru_cell"] = dict(bytes=(2 * 3 + 2) * t["rows"] * t["hidden"] * 2 + 6 * t["hidden"] * 4, elems=t["rows"] * t["hidden"])
     u = c["cumsum"]
@@ -270,7 +272,7 @@ class Workload:
 
     ORDER = ["softmax_small", "softmax_large", "layernorm", "bn_pool", "ce_loss", "rmsnorm", "silu_mul", "residual_add"]
     # Beyond the benchmark configs (not part of `value`): the two kernels the paper's case studies print.
-    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "layernorm_plain", "layernorm_params16", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc", "pool2d", "pool2d_s1", "pool2d_14", "reduce_max", "reduce_logsumexp", "bias_gelu", "residual_rmsnorm", "l2_normalize", "lstm_cell", "gru_cell", "rmsnorm_head128", "softmax_vocab"]
+    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "layernorm_plain", "layernorm_params16", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc", "pool2d", "pool2d_s1", "pool2d_14", "reduce_max", "reduce_logsumexp", "bias_gelu", "residual_rmsnorm", "l2_normalize", "lstm_cell", "gru_cell", "rmsnorm_head128", "softmax_vocab", "softmax_4096"]
 
     def __init__(self, kop, device, seed, only=None, rows_div=1):
         """only: build just these segments (None = all, plus the MLP segment); rows_div cuts the row
@@ -375,6 +377,10 @@ class Workload:
             q = c["softmax_vocab"]
             self.vx2, _ = synth.softmax_inputs(cut(q["rows"]), q["cols"], q["dtype"], seed, dev)
             self.vy2 = torch.empty_like(self.vx2)
+        if "softmax_4096" in want:
+            q = c["softmax_4096"]
+            self.vx3, _ = synth.softmax_inputs(cut(q["rows"]), q["cols"], q["dtype"], seed, dev)
+            self.vy3 = torch.empty_like(self.vx3)
         if "cumsum" in want:
             u = c["cumsum"]
             self.ux, _ = synth.cumsum_inputs(cut(u["rows"]), u["cols"], u["dtype"], seed, dev)
@@ -479,6 +485,8 @@ class Workload:
             k.kop_rmsnorm(self.qkx, self.qkw, c["rmsnorm_head128"]["eps"], out=self.qky)
         elif name == "softmax_vocab":            # softmax over a vocabulary: bf16 [2048, 128256], two-sweep kernel
             k.kop_softmax_scale_bias(self.vx2, None, 1.0, out=self.vy2)
+        elif name == "softmax_4096":             # rows of 4096 bf16 columns: one CTA per row, 32 values a thread in registers
+            k.kop_softmax_scale_bias(self.vx3, None, 1.0, out=self.vy3)
         elif name == "gru_cell":                 # gate sums, activations and state update, bf16 [16384, 3 x 1024]
             k.kop_gru_cell(self.ui, self.uh, self.up, self.ubi, self.ubh, h_out=self.uo)
         elif name == "cumsum":                   # inclusive running sum along rows, fp32 [32768, 4096]

@@ -42,6 +42,7 @@ CONFIGS = {
     # softmax over a 128256-entry vocabulary
     "rmsnorm_head128": dict(rows=1048576, hidden=128, eps=1e-6, dtype=torch.bfloat16),
     "softmax_vocab": dict(rows=2048, cols=128256, scale=1.0, dtype=torch.bfloat16),
+    "softmax_4096": dict(rows=32768, cols=4096, scale=1.0, dtype=torch.bfloat16),        # rows in one CTA's registers
     # row reductions (shape ours)
     "reduce": dict(rows=32768, cols=8192, dtype=torch.bfloat16),
 }
