@@ -398,7 +398,10 @@ kop_status_t launch_softmax(const void* xv, const void* biasv, void* yv, int64_t
     }
     if (vec && nvec64 <= 0x7FFFFFFF) {
         const int nvec = (int)nvec64;
-        const int threads = 512;
+        // 256-thread CTAs up to about 100 KB a row, 512 beyond (bf16 rows of 32000 / 50264 columns 4.9 / 4.7 TB/s with 512
+        // threads, 5.6 / 5.1 with 256; fp32 12288 columns 5.1 / 6.2; but bf16 128256 columns 5.2 / 4.6 and fp32 32000 / 65536
+        // columns 6.0 / 5.4 with 512 against 5.6 / 4.6)
+        const int threads = cols * (int64_t)sizeof(T) <= 112 * 1024 ? 256 : 512;
 #define KOP_SM_TWO(O, B) softmax_twosweep_kernel<T, PT, O, B><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, nvec, xs, ys, scale, opts)
         if (with_opts) { if (bias != nullptr) KOP_SM_TWO(true, true); else KOP_SM_TWO(true, false); }
         else { if (bias != nullptr) KOP_SM_TWO(false, true); else KOP_SM_TWO(false, false); }
