@@ -201,9 +201,10 @@ ln_block_kernel(const T* __restrict__ x, const T* __restrict__ res, const PT* __
 // blockDim.x * VPT vectors; `rows` may be odd (the last CTA then skips its second row). Capped at 64 registers
 // (four 256-thread CTAs per SM): at the 76 the compiler takes by itself three fit, and the benchmark shape ran
 // 5 % slower (rows of 5120: 12 %); a cap of 48 spills and loses 25 %. With 32 values a thread and row (plain LayerNorm,
-// CTAs of at most 160 threads) the cap is four CTAs' worth of a 160-thread CTA, 102 registers.
+// CTAs of at most 160 threads) the cap is four CTAs' worth of a 160-thread CTA, 102 registers; for its 192- to 256-thread
+// CTAs three per SM, 85 registers.
 template <typename T, typename PT, int VPT, bool kWide, int kMaxThreads, int PRO>
-__global__ void __launch_bounds__(kMaxThreads, VPT * Elem<T>::kPerVec == 32 ? 4 : 1024 / kMaxThreads)
+__global__ void __launch_bounds__(kMaxThreads, VPT * Elem<T>::kPerVec == 32 ? (kMaxThreads <= 160 ? 4 : 3) : 1024 / kMaxThreads)
 ln_pair_kernel(const T* __restrict__ x, const T* __restrict__ res, const PT* __restrict__ bias,
                const PT* __restrict__ gamma, const PT* __restrict__ beta, T* __restrict__ y,
                float* __restrict__ mean, float* __restrict__ rstd, int64_t rows, int64_t x_stride,
@@ -599,7 +600,18 @@ kop_status_t launch_ln(const void* xv, const void* rv, const void* biasv, const 
             // 160 threads at up to 102 registers, four to an SM. With one input stream the 256-thread pairs of 16
             // values left too few bytes in flight (bf16 rows of 2048 / 3072 / 4096 / 5120 columns, fp32 parameters:
             // 5.9 / 5.5 / 5.4 / 5.1 TB/s; this way 6.1 / 5.9 / 5.9 / 5.8, with 16-bit parameters 6.0 / 5.9 / 6.0 / 5.9).
-            // The same shape with 192 or 256 threads (6144, 8192 columns; two CTAs per SM) loses to one row per CTA.
+            // The same shape with 192 to 256 threads (6144 to 8192 columns) at three CTAs per SM (85 registers, a few
+            // spilled words): 6144 / 8192 columns 5.2 / 5.1 with one row per CTA, 5.8 / 5.4 this way (at two CTAs per SM
+            // and 128 registers it loses: 4.5 / 5.0).
+            if (nvec % 4 == 0 && (nvec / 4) % 32 == 0 && nvec / 4 > 160 && nvec / 4 <= 256 && rows >= 8 * (int64_t)sm_count()) {
+                const int threads4 = nvec / 4;
+                const unsigned grid = (unsigned)((rows + 1) / 2);
+                if (wide)
+                    ln_pair_kernel<T, PT, 32 / E, true, 256, PRO><<<grid, threads4, 0, stream>>>(x, r, bias, gamma, beta, y, mean, rstd, rows, xs, rs, ys, eps, inv_hidden);
+                else
+                    ln_pair_kernel<T, PT, 32 / E, false, 256, PRO><<<grid, threads4, 0, stream>>>(x, r, bias, gamma, beta, y, mean, rstd, rows, xs, rs, ys, eps, inv_hidden);
+                return launch_status();
+            }
             if (nvec % 4 == 0 && (nvec / 4) % 32 == 0 && nvec / 4 >= 64 && nvec / 4 <= 160 && rows >= 8 * (int64_t)sm_count()) {
                 const int threads4 = nvec / 4;
                 const unsigned grid = (unsigned)((rows + 1) / 2);

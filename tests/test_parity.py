@@ -714,7 +714,7 @@ def test_row_ops_options_and_full_configs(kop):
 RLN_SHAPES = [(2048, 4096, BF16), (1185, 4096, BF16), (300, 4096, F32), (65, 256, BF16), (9, 20480, BF16), (4, 33000, F32),
               (21, 513, F32),
               # plain LayerNorm of 16-bit rows: row pairs with 32 values a thread (64- and 160-thread CTAs, an odd row count)
-              (1301, 2048, torch.float16), (1187, 5120, BF16)]
+              (1301, 2048, torch.float16), (1187, 5120, BF16), (1185, 6144, BF16), (1186, 8192, torch.float16)]
 
 
 @pytest.mark.parametrize("rows,hidden,dtype", RLN_SHAPES)
