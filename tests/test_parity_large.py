@@ -113,3 +113,31 @@ def test_more_than_2_to_31_elements_images(kop):
         assert_close(z[n:n + 1, c0:c0 + cpg], rz, 2e-2, f"large groupnorm {n},{grp}")
         assert_close(mu[n:n + 1, grp:grp + 1], rm, 1e-5, "large groupnorm mean")
         assert_close(rs[n:n + 1, grp:grp + 1], rr, 1e-5, "large groupnorm rstd")
+
+
+def test_pool2d_k2s2_index_limits(kop):
+    """The thread-per-output 2x2 / stride 2 kernel at the edge of what its multiply-shift divisions cover: just under
+    2^24 planes of 4 x 4 (the largest quotient, 67 M outputs), sampled planes from both ends and the middle, and the
+    same geometry with one plane too many, which must take another kernel and give the same values."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 6 << 30:
+        pytest.skip("needs about 4 GB of free device memory")
+    for N, C in ((256, 65535), (257, 65536)):                      # 16,776,960 planes (inside), 16,842,752 (outside)
+        g = torch.Generator(device="cuda")
+        g.manual_seed(5)
+        x = torch.randn((N, C, 4, 4), generator=g, device="cuda", dtype=torch.float32)
+        scale = torch.rand(C, generator=g, device="cuda") + 0.5
+        shift = torch.randn(C, generator=g, device="cuda") * 0.1
+        for mode in ("max", "avg"):
+            y = kop.kop_affine_relu_pool2d(x, scale, shift, (2, 2), (2, 2), (0, 0), mode, True)
+            for n, c in [(0, 0), (0, C - 1), (N // 2, 12345), (N - 1, 0), (N - 1, C - 1)]:
+                ref = kopref.affine_relu_pool2d(x[n:n + 1, c:c + 1].cpu(), scale[c:c + 1].cpu(), shift[c:c + 1].cpu(), (2, 2),
+                                                (2, 2), (0, 0), mode, True, threads=None)
+                assert_close(y[n:n + 1, c:c + 1], ref, 1e-5, f"k2s2 limits {N}x{C} {mode} {n},{c}")
+            # a whole contiguous block of planes at the far end against the oracle
+            ref = kopref.affine_relu_pool2d(x[N - 1:, C - 4096:].cpu(), scale[C - 4096:].cpu(), shift[C - 4096:].cpu(), (2, 2),
+                                            (2, 2), (0, 0), mode, True, threads=None)
+            assert_close(y[N - 1:, C - 4096:], ref, 1e-5, f"k2s2 limits {N}x{C} {mode} last planes")
+            del y
+        del x
+        torch.cuda.empty_cache()
