@@ -80,6 +80,11 @@ POOL_CASES = [
     (9, 13, 2, 2, (2, 2), (2, 2), (0, 0), F32),
     (2, 3, 3, 2, (2, 2), (2, 2), (0, 0), BF16),
     (1, 2, 60, 60, (2, 2), (2, 2), (0, 0), F32),
+    # widths that are a multiple of four: two adjacent outputs a thread (4 x 4 planes: one pair per output row)
+    (3, 50, 28, 28, (2, 2), (2, 2), (0, 0), F32),
+    (5, 7, 12, 20, (2, 2), (2, 2), (0, 0), torch.float16),
+    (33, 17, 4, 4, (2, 2), (2, 2), (0, 0), BF16),
+    (2, 3, 61, 60, (2, 2), (2, 2), (0, 0), BF16),
 ]
 
 
