@@ -217,6 +217,10 @@ POOL_EX_CASES = [
     (3, 50, 14, 14, (3, 3), (2, 2), (1, 1), BF16),
     (2, 3, 30, 44, (5, 3), (2, 1), (2, 1), F16),
     (1, 2, 6, 5000, (3, 3), (2, 2), (1, 1), BF16),
+    # 2x2 / stride 2: a thread per output (pairs), two outputs a thread (width divisible by four), scalar loads (odd width)
+    (5, 37, 14, 14, (2, 2), (2, 2), (0, 0), F16),
+    (3, 50, 28, 28, (2, 2), (2, 2), (0, 0), BF16),
+    (6, 11, 7, 7, (2, 2), (2, 2), (0, 0), BF16),
 ]
 
 
