@@ -389,7 +389,8 @@ def assert_close_with_neg_inf(got, ref, tol, what):
 
 
 @pytest.mark.parametrize("rows,cols,dtype", [(96, 512, F32), (1024, 128, BF16), (130, 1000, F32), (66, 1001, F32),
-                                             (20, 16384, BF16), (12, 20000, F32), (9, 1, F32), (4, 50000, BF16)])
+                                             (20, 16384, BF16), (12, 20000, F32), (9, 1, F32), (4, 50000, BF16),
+                                             (65, 4096, BF16), (33, 2048, F32)])
 @pytest.mark.parametrize("seed", SEEDS)
 def test_softmax_opts_parity(kop, rows, cols, dtype, seed):
     x, bias = synth.softmax_inputs(rows, cols, dtype, seed, "cuda")
