@@ -21,10 +21,19 @@ namespace {
 // kFull: the row is exactly L * VPL vectors (no tail predicates); kBias: bias != NULL. L: lanes per row (32, or
 // 2 .. 16 for rows of fewer than 32 vectors, 32 / L rows per warp: attention scores and class logits of 64 to
 // 256 columns would leave most of a warp idle otherwise).
-template <typename T, typename PT, int VPL, bool kFull, bool kBias, int L = 32>
+// kLog: the log form of the output. kCausal: row r sees columns 0 .. (r mod period) + cols - period only (`causal`
+// carries the period, cols - period and ceil(2^64 / period) for the remainder); later columns count as -inf, and a
+// row's vectors beyond its last visible column are not read.
+struct SmCausal {
+    int period, base;
+    unsigned long long magic;
+};
+
+template <typename T, typename PT, int VPL, bool kFull, bool kBias, int L = 32, bool kLog = false, bool kCausal = false>
 __global__ void __launch_bounds__(256)
 softmax_warp_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __restrict__ y,
-                    int64_t rows, int nvec, int64_t x_stride, int64_t y_stride, float scale)
+                    int64_t rows, int nvec, int64_t x_stride, int64_t y_stride, float scale,
+                    SmCausal causal = SmCausal{0, 0, 0ull})
 {
     constexpr int E = Elem<T>::kPerVec;
     const int lane = L == 32 ? (threadIdx.x & 31) : (threadIdx.x & (L - 1));
@@ -37,11 +46,17 @@ softmax_warp_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __r
     const float s2 = scale * kLog2e;
     const T* xr = x + row * x_stride;
     T* yr = y + row * y_stride;
+    int last = 0;
+    if (kCausal) {
+        // row / period by multiply-shift (exact for row < 2^64 / period; a period of 1 has no 64-bit reciprocal)
+        const unsigned long long q = causal.period == 1 ? (unsigned long long)row : __umul64hi((unsigned long long)row, causal.magic);
+        last = (int)((unsigned long long)row - q * (unsigned)causal.period) + causal.base;
+    }
     Vec16 raw[VPL];
 #pragma unroll
     for (int k = 0; k < VPL; ++k) {
         const int v = k * L + lane;
-        if (kFull || v < nvec) raw[k] = ld_stream(xr + (int64_t)v * E);
+        if ((kFull || v < nvec) && (!kCausal || v * E <= last)) raw[k] = ld_stream(xr + (int64_t)v * E);
         else raw[k] = Vec16{{0u, 0u, 0u, 0u}};
     }
     float t[VPL][E];
@@ -51,6 +66,7 @@ softmax_warp_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __r
         const int v = k * L + lane;
         float f[E];
         Elem<T>::unpack(raw[k], f);
+        const int vis = kCausal ? last - v * E : 0;          // elements 0 .. vis of this vector are visible
 #pragma unroll
         for (int q = 0; q < E / 4; ++q) {
             float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -59,7 +75,7 @@ softmax_warp_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __r
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 const int e = 4 * q + c;
-                t[k][e] = (kFull || v < nvec) ? fmaf(f[e], s2, bb[c] * kLog2e) : -INFINITY;
+                t[k][e] = ((kFull || v < nvec) && (!kCausal || e <= vis)) ? fmaf(f[e], s2, bb[c] * kLog2e) : -INFINITY;
                 m = fmaxf(m, t[k][e]);
             }
         }
@@ -71,18 +87,21 @@ softmax_warp_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __r
     for (int k = 0; k < VPL; ++k)
 #pragma unroll
         for (int e = 0; e < E; ++e) {
-            t[k][e] = ex2_approx(t[k][e] - m);
-            s += t[k][e];
+            const float d = t[k][e] - m;
+            const float p = ex2_approx(d);
+            s += p;
+            t[k][e] = kLog ? d : p;                          // the log form keeps the base-2 exponent
         }
 #pragma unroll
     for (int o = L / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
     const float inv = 1.0f / s;
+    const float lg = lg2_approx(s);
 #pragma unroll
     for (int k = 0; k < VPL; ++k) {
         const int v = k * L + lane;
         float o[E];
 #pragma unroll
-        for (int e = 0; e < E; ++e) o[e] = t[k][e] * inv;
+        for (int e = 0; e < E; ++e) o[e] = kLog ? (t[k][e] - lg) * kLn2 : t[k][e] * inv;
         if (live && (kFull || v < nvec)) st_stream(yr + (int64_t)v * E, Elem<T>::pack(o));
     }
 }
@@ -320,7 +339,16 @@ kop_status_t launch_softmax(const void* xv, const void* biasv, void* yv, int64_t
     // log-softmax without a causal mask: the plain kernels with the log form of the output (no per-element test of the
     // visible range; bf16 rows of 1024 - 8192 columns 4.3 - 4.6 TB/s through the general form)
     const bool log_only = with_opts && opts.period == 0 && opts.log_out != 0;
-    if (vec && nvec64 < 32 && !with_opts) {                  // fewer than 32 vectors: 2 to 8 lanes per row, four vectors each
+    // causal rows without the log form on short rows: the lanes-per-row / warp-per-row kernels with the visible range
+    // worked out per row (attention scores of 256 / 512 keys ran at 2.0 / 3.8 TB/s through the CTA-per-row form)
+    const bool causal_short = with_opts && opts.period != 0 && opts.log_out == 0 && rows < (1LL << 53);
+    SmCausal cz{0, 0, 0ull};
+    if (causal_short) {
+        cz.period = (int)opts.period;
+        cz.base = (int)(opts.cols - opts.period);
+        cz.magic = opts.period > 1 ? (~0ull) / (unsigned long long)opts.period + 1ull : 0ull;
+    }
+    if (vec && nvec64 < 32 && (!with_opts || log_only || causal_short)) {                  // fewer than 32 vectors: 2 to 8 lanes per row, four vectors each
         const int nvec = (int)nvec64;
         const int lanes = nvec > 16 ? 8 : nvec > 8 ? 4 : 2;
         const int64_t rows_per_cta = 8 * (32 / lanes);
@@ -328,7 +356,12 @@ kop_status_t launch_softmax(const void* xv, const void* biasv, void* yv, int64_t
         if (ctas > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
         const unsigned grid = (unsigned)ctas;
         const bool full = nvec == lanes * 4;
-#define KOP_SM_GROUP_L(F, B, L) softmax_warp_kernel<T, PT, 4, F, B, L><<<grid, 256, 0, stream>>>(x, bias, y, rows, nvec, xs, ys, scale)
+#define KOP_SM_GROUP_L(F, B, L)                                                                                                  \
+    do {                                                                                                                         \
+        if (causal_short) softmax_warp_kernel<T, PT, 4, false, B, L, false, true><<<grid, 256, 0, stream>>>(x, bias, y, rows, nvec, xs, ys, scale, cz); \
+        else if (log_only) softmax_warp_kernel<T, PT, 4, F, B, L, true><<<grid, 256, 0, stream>>>(x, bias, y, rows, nvec, xs, ys, scale); \
+        else softmax_warp_kernel<T, PT, 4, F, B, L><<<grid, 256, 0, stream>>>(x, bias, y, rows, nvec, xs, ys, scale);           \
+    } while (0)
 #define KOP_SM_GROUP(L)                                                         \
     do {                                                                        \
         if (full && bias != nullptr) KOP_SM_GROUP_L(true, true, L);             \
@@ -343,7 +376,7 @@ kop_status_t launch_softmax(const void* xv, const void* biasv, void* yv, int64_t
 #undef KOP_SM_GROUP
         return launch_status();
     }
-    if (vec && nvec64 <= 32 * 4 && !with_opts) {
+    if (vec && nvec64 <= 32 * 4 && (!with_opts || log_only || causal_short)) {
         const int nvec = (int)nvec64;
         const int vpl = (nvec + 31) / 32;
         const int threads = 256;
@@ -352,7 +385,12 @@ kop_status_t launch_softmax(const void* xv, const void* biasv, void* yv, int64_t
         const unsigned grid = (unsigned)ctas;
         const int vp = vpl <= 1 ? 1 : (vpl <= 2 ? 2 : 4);
         const bool full = nvec == 32 * vp;
-#define KOP_SM_WARP_L(V, F, B) softmax_warp_kernel<T, PT, V, F, B><<<grid, threads, 0, stream>>>(x, bias, y, rows, nvec, xs, ys, scale)
+#define KOP_SM_WARP_L(V, F, B)                                                                                                   \
+    do {                                                                                                                         \
+        if (causal_short) softmax_warp_kernel<T, PT, V, false, B, 32, false, true><<<grid, threads, 0, stream>>>(x, bias, y, rows, nvec, xs, ys, scale, cz); \
+        else if (log_only) softmax_warp_kernel<T, PT, V, F, B, 32, true><<<grid, threads, 0, stream>>>(x, bias, y, rows, nvec, xs, ys, scale); \
+        else softmax_warp_kernel<T, PT, V, F, B><<<grid, threads, 0, stream>>>(x, bias, y, rows, nvec, xs, ys, scale);          \
+    } while (0)
 #define KOP_SM_WARP(V)                                                         \
     do {                                                                       \
         if (full && bias != nullptr) KOP_SM_WARP_L(V, true, true);             \

@@ -413,6 +413,24 @@ def test_softmax_opts_parity(kop, rows, cols, dtype, seed):
     assert_close(kop.kop_softmax_opts(x, bias, 0.125), to_f64(plain), 1e-6 if dtype == F32 else tol, "softmax_opts without options")
 
 
+@pytest.mark.parametrize("rows,cols,period,dtype", [(300, 256, 64, BF16), (77, 768, 256, F32), (1000, 64, 64, torch.float16),
+                                                    (515, 1024, 1, BF16), (131, 1000, 500, F32), (64, 32, 7, F32)])
+@pytest.mark.parametrize("seed", SEEDS[:3])
+def test_softmax_causal_short_rows(kop, rows, cols, period, dtype, seed):
+    """Causal rows of up to 128 vectors (the lanes-per-row and warp-per-row kernels): periods that wrap within the
+    rows, a visible range that starts inside the row (cols - period > 0), a period of one, with and without a bias."""
+    x, bias = synth.softmax_inputs(rows, cols, dtype, seed, "cuda")
+    for use_bias in (False, True):
+        y = Guarded((rows, cols), dtype)
+        kop.kop_softmax_opts(x, bias if use_bias else None, 0.25, False, period, out=y.t)
+        ref = kopref.softmax_opts(host(x), host(bias) if use_bias else None, 0.25, False, period, threads=None)
+        assert_close(y.t, ref, tol_of(dtype), f"causal short rows bias={use_bias}")
+        y.check("causal short rows")
+        # masked columns are exact zeros
+        g = to_f64(y.t)
+        assert np.array_equal(g == 0.0, ref == 0.0) or np.all(g[ref == 0.0] == 0.0)
+
+
 def test_softmax_opts_attention_shape_and_validation(kop):
     # attention scores of 4 heads x 256 queries over 256 keys, square causal mask, in place
     S = 256
