@@ -524,7 +524,7 @@ pool2d_planes_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift,
     const float inv_oplane = 1.0f / (float)oplane, inv_ow = 1.0f / (float)OW;
     T* yc = y + p0 * oplane;
     const int n_out = g_here * oplane;
-    if (kFixed) {
+    if constexpr (kFixed) {
         // Plane slot t / oplane of each pass of Gp planes, position t % oplane. The window geometry is worked out
         // once: clamped tap offsets (a clamped tap repeats an element of the same window, which leaves a maximum
         // unchanged and is masked out of a sum), so a pass costs the taps and a store, with no index division and no
@@ -571,8 +571,7 @@ pool2d_planes_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift,
             }
             Elem<T>::store1(yo, res);
         }
-        return;
-    }
+    } else {
     for (int o = threadIdx.x; o < n_out; o += nthreads) {
         const int g = div_small(o, oplane, inv_oplane);
         const int r = o - g * oplane;
@@ -607,6 +606,7 @@ pool2d_planes_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift,
             }
         }
         Elem<T>::store1(yc + o, MODE == 0 ? res : res * inv_area);
+    }
     }
 }
 
@@ -749,6 +749,109 @@ pool2d_k2s2_quad_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift,
             }
         }
     }
+}
+
+// ---- the window is the whole plane (global average / max pooling): a reduction per plane --------------------------
+// L lanes per plane (L = 2 .. 32, a power of two chosen from the plane's size), 32 / L planes per warp, eight warps per
+// CTA; a lane sweeps its share of the plane in batches of four 16-byte vectors (scalars when planes are not whole
+// aligned vectors), activates and accumulates in fp32, and a butterfly over the plane's lanes finishes it. The sum is
+// a fixed order (lane-sequential, then the butterfly): bit-identical from run to run.
+// VB: bytes per load (16, 8, 4 or one element: the widest that divides a plane's bytes and the tensor's alignment).
+// A load lands as raw words and is widened when it is used, so that a batch in flight costs its bytes in registers.
+template <int VB>
+struct RawUnit {
+    uint32_t w[VB >= 4 ? VB / 4 : 1];
+};
+
+template <typename T, int VB>
+__device__ __forceinline__ RawUnit<VB> load_raw(const T* p)
+{
+    RawUnit<VB> r;
+    if constexpr (VB == 16) {
+        const Vec16 v = ld_stream(p);
+        r.w[0] = v.w[0], r.w[1] = v.w[1], r.w[2] = v.w[2], r.w[3] = v.w[3];
+    } else if constexpr (VB == 8) {
+        const uint2 t = __ldg(reinterpret_cast<const uint2*>(p));
+        r.w[0] = t.x, r.w[1] = t.y;
+    } else if constexpr (VB == 4) {
+        r.w[0] = __ldg(reinterpret_cast<const uint32_t*>(p));
+    } else {
+        r.w[0] = __ldg(reinterpret_cast<const unsigned short*>(p));
+    }
+    return r;
+}
+
+template <typename T, int VB>
+__device__ __forceinline__ void widen_raw(const RawUnit<VB>& r, float (&f)[VB / (int)sizeof(T)])
+{
+    if constexpr (VB == 16) {
+        Elem<T>::unpack(Vec16{{r.w[0], r.w[1], r.w[2], r.w[3]}}, f);
+    } else if constexpr (sizeof(T) == 4) {
+#pragma unroll
+        for (int i = 0; i < VB / 4; ++i) f[i] = __uint_as_float(r.w[i]);
+    } else if constexpr (VB >= 4) {
+#pragma unroll
+        for (int i = 0; i < VB / 4; ++i) {
+            float2 a;
+            Elem<T>::unpack_pair(r.w[i], a);
+            f[2 * i] = a.x, f[2 * i + 1] = a.y;
+        }
+    } else {
+        float2 a;
+        Elem<T>::unpack_pair(r.w[0], a);                     // the value sits in the low half
+        f[0] = a.x;
+    }
+}
+
+template <typename T, int MODE, int VB, int L>
+__global__ void __launch_bounds__(256)
+pool2d_global_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift, T* __restrict__ y, int planes, int plane,
+                     MagicDiv by_c, float relu_floor, float inv_area)
+{
+    constexpr int EV = VB / (int)sizeof(T);                  // elements per load
+    constexpr int U = VB >= 16 ? 4 : (VB == 8 ? 8 : 16);     // loads in flight per lane: 64 bytes (32 for 2-byte loads)
+    constexpr int kPerWarp = 32 / L;
+    const int lane = threadIdx.x & 31, sub = lane & (L - 1);
+    const int p = ((int)blockIdx.x * 8 + ((int)threadIdx.x >> 5)) * kPerWarp + lane / L;
+    const bool live = p < planes;
+    const bool identity = scale.p == nullptr && relu_floor == -INFINITY;
+    float sc = 1.0f, sf = 0.0f;
+    if (live && !identity) {
+        const int c = p - by_c.div(p) * by_c.d;
+        sc = scale.p != nullptr ? scale.at(c) : 1.0f;
+        sf = shift.p != nullptr ? shift.at(c) : 0.0f;
+    }
+    const T* xp = x + (int64_t)(live ? p : 0) * plane;
+    float acc = MODE == 0 ? -INFINITY : 0.0f;
+    const int n = live ? plane / EV : 0;                     // loads this plane's lanes share
+    for (int base = 0; base < n; base += U * L) {
+        RawUnit<VB> raw[U];
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const int v = base + k * L + sub;
+            if (v < n) raw[k] = load_raw<T, VB>(xp + (int64_t)v * EV);
+        }
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const int v = base + k * L + sub;
+            if (v < n) {
+                float f[EV];
+                widen_raw<T, VB>(raw[k], f);
+#pragma unroll
+                for (int e = 0; e < EV; ++e) {
+                    const float a = identity ? f[e] : act_of(f[e], sc, sf, relu_floor);
+                    acc = MODE == 0 ? max_keep_nan(acc, a) : acc + a;
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int o = L / 2; o > 0; o >>= 1) {
+        const float other = __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+        // the lower lane's term first on both sides, so that the two lanes agree bit for bit
+        acc = MODE == 0 ? max_keep_nan(acc, other) : ((lane & o) ? other + acc : acc + other);
+    }
+    if (live && sub == 0) Elem<T>::store1(y + p, MODE == 0 ? acc : acc * inv_area);
 }
 
 // ---- walk kernel: 2x2 / 3x3 windows at stride 1 or 2, any width, any alignment --------------------------------
@@ -1034,6 +1137,47 @@ kop_status_t launch_pool(const void* xv, ParamVec scale, ParamVec shift, void* y
     T* y = static_cast<T*>(yv);
     const float inv_area = (float)(1.0 / ((double)kh * kw));
     const int64_t planes = N * C;
+    // the window is the plane: a reduction per plane (as windows 7 x 7 / 14 x 14 / 28 x 28 / 56 x 56 fp32 planes ran at 2.4 /
+    // 2.4 / 1.1 / 0.7 TB/s, a thread looping over the plane per output; this way 4.5 / 6.6 / 6.3 / 6.0, bf16 2.7 / 5.4 / 5.9 / 5.5)
+    if (kh == H && kw == W && ph == 0 && pw == 0 && planes < (1LL << 31) - 256 && (int64_t)H * W < (1 << 30) &&
+        planes * C < (1LL << 40) && planes < (1LL << 24) * C) {
+        const int plane = H * W;
+        const int pbytes = plane * (int)sizeof(T);
+        const int vb = (pbytes % 16 == 0 && aligned_to(x, 16)) ? 16
+                       : (pbytes % 8 == 0 && aligned_to(x, 8)) ? 8
+                       : (pbytes % 4 == 0 && aligned_to(x, 4)) ? 4 : (int)sizeof(T);
+        const int units = pbytes / vb, per_lane = vb >= 16 ? 4 : (vb == 8 ? 8 : 16);
+        int L = 2;
+        while (L < 32 && L * per_lane < units) L *= 2;
+        const MagicDiv by_c{((1ULL << 40) + (uint64_t)C - 1) / (uint64_t)C, (int)C};
+        const int per_cta = 8 * (32 / L);
+        const unsigned blocks = (unsigned)((planes + per_cta - 1) / per_cta);
+        const float floor_v = relu ? 0.0f : -INFINITY;
+        const float inv_plane = (float)(1.0 / ((double)H * W));
+#define KOP_GLOBAL_L(M, V, LL) \
+    pool2d_global_kernel<T, M, V, LL><<<blocks, 256, 0, stream>>>(x, scale, shift, y, (int)planes, plane, by_c, floor_v, inv_plane)
+#define KOP_GLOBAL_V(M, V)                        \
+    do {                                          \
+        if (L == 2) KOP_GLOBAL_L(M, V, 2);        \
+        else if (L == 4) KOP_GLOBAL_L(M, V, 4);   \
+        else if (L == 8) KOP_GLOBAL_L(M, V, 8);   \
+        else if (L == 16) KOP_GLOBAL_L(M, V, 16); \
+        else KOP_GLOBAL_L(M, V, 32);              \
+    } while (0)
+#define KOP_GLOBAL(M)                                            \
+    do {                                                         \
+        if (vb == 16) KOP_GLOBAL_V(M, 16);                       \
+        else if (vb == 8) KOP_GLOBAL_V(M, 8);                    \
+        else if (vb == 4) KOP_GLOBAL_V(M, 4);                    \
+        else KOP_GLOBAL_V(M, (int)sizeof(T));                    \
+    } while (0)
+        if (mode == 0) KOP_GLOBAL(0);
+        else KOP_GLOBAL(1);
+#undef KOP_GLOBAL_V
+#undef KOP_GLOBAL
+#undef KOP_GLOBAL_L
+        return launch_status();
+    }
     // the strip kernel: stride-2 3x3 (pad 1) or 2x2 (pad 0) windows over rows of whole 8-column segments
     const bool k3 = kh == 3 && kw == 3 && ph == 1 && pw == 1, k2 = kh == 2 && kw == 2 && ph == 0 && pw == 0;
     if ((k3 || k2) && sh == 2 && sw == 2 && W % 8 == 0 && H % 2 == 0 && aligned_to(x, 32) && aligned_to(y, 16)) {

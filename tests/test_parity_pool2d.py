@@ -85,6 +85,16 @@ POOL_CASES = [
     (5, 7, 12, 20, (2, 2), (2, 2), (0, 0), torch.float16),
     (33, 17, 4, 4, (2, 2), (2, 2), (0, 0), BF16),
     (2, 3, 61, 60, (2, 2), (2, 2), (0, 0), BF16),
+    # the window is the plane (global pooling): 16-, 8-, 4-byte and single-element loads, few and many lanes per plane
+    (5, 37, 7, 7, (7, 7), (1, 1), (0, 0), F32),
+    (5, 37, 7, 7, (7, 7), (7, 7), (0, 0), BF16),
+    (3, 50, 14, 14, (14, 14), (1, 1), (0, 0), BF16),
+    (2, 13, 28, 28, (28, 28), (1, 1), (0, 0), F32),
+    (4, 9, 8, 8, (8, 8), (3, 3), (0, 0), torch.float16),
+    (3, 5, 5, 9, (5, 9), (1, 1), (0, 0), BF16),
+    (1, 2, 224, 224, (224, 224), (1, 1), (0, 0), F32),
+    (70, 3, 2, 2, (2, 2), (1, 1), (0, 0), F32),
+    (33, 7, 1, 1, (1, 1), (1, 1), (0, 0), BF16),
 ]
 
 
@@ -140,6 +150,29 @@ def test_pool2d_k2s2_unaligned_base(kop):
             assert_close(a, ref, tol_of(dtype), f"k2s2 aligned {mode}")
             assert_close(b, ref, tol_of(dtype), f"k2s2 unaligned {mode}")
             assert torch.equal(a, b)
+
+
+def test_pool2d_global_unaligned_and_nan(kop):
+    """Global pooling on a tensor that starts one element into its buffer (narrower loads), and a NaN in one plane."""
+    for dtype in (F32, BF16):
+        x, scale, shift = synth.bn_pool_inputs(3, 5, 14, 14, dtype, 13, "cuda")
+        buf = torch.empty(x.numel() + 1, dtype=dtype, device="cuda")
+        xs = buf[1:].view(x.shape)
+        xs.copy_(x)
+        for mode in ("max", "avg"):
+            a = kop.kop_affine_relu_pool2d(x, scale, shift, (14, 14), (1, 1), (0, 0), mode, True)
+            b = kop.kop_affine_relu_pool2d(xs, scale, shift, (14, 14), (1, 1), (0, 0), mode, True)
+            ref = kopref.affine_relu_pool2d(host(x), host(scale), host(shift), (14, 14), (1, 1), (0, 0), mode, True)
+            assert_close(a, ref, tol_of(dtype), f"global aligned {mode}")
+            assert_close(b, ref, tol_of(dtype), f"global unaligned {mode}")
+            if mode == "max":
+                assert torch.equal(a, b)                       # a maximum does not depend on the order
+    xn, scale, shift = synth.bn_pool_inputs(2, 4, 7, 7, F32, 3, "cuda")
+    xn[1, 2, 3, 4] = float("nan")
+    for mode in ("max", "avg"):
+        y = kop.kop_affine_relu_pool2d(xn, scale, shift, (7, 7), (1, 1), (0, 0), mode, True)
+        ref = kopref.affine_relu_pool2d(host(xn), host(scale), host(shift), (7, 7), (1, 1), (0, 0), mode, True)
+        assert np.array_equal(np.isnan(y.cpu().numpy()), np.isnan(ref)) and np.isnan(ref).sum() == 1
 
 
 def test_pool2d_options(kop):
