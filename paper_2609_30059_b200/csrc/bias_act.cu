@@ -30,7 +30,7 @@ __device__ __forceinline__ float act_dev(float u, float alpha)
         const float hu = 0.5f * u;
         return fmaf(hu, t, hu);
     }
-    case kActGeluErf: return 0.5f * u * (1.0f + erff(u * 0.7071067811865476f));
+    case kActGeluErf: return 0.5f * u * (1.0f + erf_fast(u * 0.7071067811865476f));
     case kActSilu: return u * rcp_approx(1.0f + ex2_approx(-u * kLog2e));      // ~3e-7 relative
     case kActSigmoid: return rcp_approx(1.0f + ex2_approx(-u * kLog2e));
     case kActTanh: return kFast ? tanh_approx(u) : tanhf(u);
