@@ -596,7 +596,7 @@ kop_status_t kop_mlp_handle_wrap(void* cublas_handle, void** handle);
  * intermediate d is used. enable == 0 restores the default five-operation form. The setting belongs to
  * the handle and applies to later kop_rmsnorm_swiglu_residual calls; results differ from the default
  * form by at most one rounding of `dtype`. Calls with out == h keep the default form (the vendor
- * kernel is not used in place). Judge it with the perf gate on whole-segment time.
+ * kernel is not used in place). Assess it with the perf gate on whole-segment time.
  */
 kop_status_t kop_mlp_handle_set_residual_in_gemm(void* handle, int enable);
 
