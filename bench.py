@@ -763,7 +763,7 @@ def run_ours(args, rank, world, local_rank):
     clocks_situ = sampler2.stop()
 
     # ---- vendor-library configuration of the segment (the paper's future-work item): the residual add
-    # folded into the down projection's cuBLASLt epilogue, judged by the perf gate on whole-segment
+    # folded into the down projection's cuBLASLt epilogue, assessed by the perf gate on whole-segment
     # graph time. The two graphs are replayed alternately so that clock drift hits both alike.
     vendor_cfg = None
     if rank == 0:
