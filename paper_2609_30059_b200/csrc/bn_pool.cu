@@ -91,69 +91,111 @@ bn_plane_warp_kernel(const T* __restrict__ x, const PT* __restrict__ scale,
     }
 }
 
-// Small planes (7x7, 14x14, ...: the usual input of a global average pool) are shorter than a warp's
-// worth of vectors and often not a whole number of them, but consecutive planes are contiguous. A CTA
-// therefore takes a run of G planes (G a multiple of the vector length, so every run starts on a 16-byte
-// boundary) as one flat array: 16-byte loads and stores across plane boundaries, the plane of each
-// element found by one small division per vector and carried along it, per-plane scale / shift staged in
-// shared memory, the activations parked in shared memory, and the plane sums taken from there by one
-// warp per plane in a fixed order.
-constexpr int kFlatThreads = 256;
-constexpr int kFlatMaxElems = 4096;                       // activations parked per CTA (16 KB)
+// Planes of at most 1024 elements: L lanes per plane (2 .. 32, a power of two chosen from the plane's size), 32 / L
+// planes per warp, eight warps per CTA. A lane sweeps its share of the plane in batches that keep 64 bytes of loads in
+// flight, with the widest load that divides a plane's bytes and both tensors' alignment (VB = 16, 8, 4 bytes or one
+// element); every value is activated, stored back at the same width and added to the lane's sum, and a butterfly
+// over the plane's lanes finishes the mean. No shared memory, no barrier; a fixed summation order.
+template <int VB>
+struct BnRaw {
+    uint32_t w[VB >= 4 ? VB / 4 : 1];
+};
 
-template <typename T, typename PT>
-__global__ void __launch_bounds__(kFlatThreads)
-bn_flat_kernel(const T* __restrict__ x, const PT* __restrict__ scale, const PT* __restrict__ shift,
-               T* __restrict__ y, float* __restrict__ pooled, int64_t planes, int plane, int G, int C,
-               float inv_plane)
+template <typename T, typename PT, int VB, int L>
+__global__ void __launch_bounds__(256)
+bn_plane_group_kernel(const T* __restrict__ x, const PT* __restrict__ scale, const PT* __restrict__ shift,
+                      T* __restrict__ y, float* __restrict__ pooled, int64_t planes, int plane, int C, float inv_plane)
 {
-    constexpr int E = Elem<T>::kPerVec;
-    __shared__ __align__(16) float act[kFlatMaxElems];
-    __shared__ float sc_s[kFlatMaxElems / 4], sh_s[kFlatMaxElems / 4];      // G <= chunk / plane, plane >= 1 ...
-    const int64_t p0 = (int64_t)blockIdx.x * G;
-    const int g_here = (int)(planes - p0 < G ? planes - p0 : G);
-    const int elems = g_here * plane;
-    const T* xc = x + p0 * plane;
-    T* yc = y + p0 * plane;
-    for (int g = threadIdx.x; g < g_here; g += kFlatThreads) {
-        const int c = (int)((p0 + g) % C);
-        sc_s[g] = param1(scale, c);
-        sh_s[g] = param1(shift, c);
+    constexpr int EV = VB / (int)sizeof(T);
+    constexpr int U = VB >= 16 ? 4 : (VB == 8 ? 8 : 16);
+    constexpr int kPerWarp = 32 / L;
+    const int lane = threadIdx.x & 31, sub = lane & (L - 1);
+    const int64_t p = ((int64_t)blockIdx.x * 8 + (threadIdx.x >> 5)) * kPerWarp + lane / L;
+    const bool live = p < planes;
+    float sc = 1.0f, sh = 0.0f;
+    if (live) {
+        const int c = (int)(p % C);
+        sc = param1(scale, c);
+        sh = param1(shift, c);
     }
-    __syncthreads();
-    const float inv = 1.0f / (float)plane;
-    const int nvec = elems / E;
-    for (int v = threadIdx.x; v < nvec; v += kFlatThreads) {
-        float f[E];
-        Elem<T>::unpack(ld_stream(xc + (int64_t)v * E), f);
-        const int i0 = v * E;
-        int pl = (int)((float)i0 * inv);                 // i0 / plane: float estimate, one-step fix-up
-        int rem = i0 - pl * plane;
-        if (rem >= plane) { rem -= plane; ++pl; }
-        if (rem < 0) { rem += plane; --pl; }
+    const T* xp = x + (live ? p : 0) * plane;
+    T* yp = y + (live ? p : 0) * plane;
+    const int n = live ? plane / EV : 0;
+    float sum = 0.0f;
+    for (int base = 0; base < n; base += U * L) {
+        BnRaw<VB> raw[U];
 #pragma unroll
-        for (int e = 0; e < E; ++e) {
-            f[e] = relu_keep_nan(fmaf(f[e], sc_s[pl], sh_s[pl]));
-            act[i0 + e] = f[e];
-            if (++rem == plane) { rem = 0; ++pl; }
+        for (int k = 0; k < U; ++k) {
+            const int v = base + k * L + sub;
+            if (v < n) {
+                const T* q = xp + (int64_t)v * EV;
+                if constexpr (VB == 16) {
+                    const Vec16 t = ld_stream(q);
+                    raw[k].w[0] = t.w[0], raw[k].w[1] = t.w[1], raw[k].w[2] = t.w[2], raw[k].w[3] = t.w[3];
+                } else if constexpr (VB == 8) {
+                    const uint2 t = __ldg(reinterpret_cast<const uint2*>(q));
+                    raw[k].w[0] = t.x, raw[k].w[1] = t.y;
+                } else if constexpr (VB == 4) {
+                    raw[k].w[0] = __ldg(reinterpret_cast<const uint32_t*>(q));
+                } else {
+                    raw[k].w[0] = __ldg(reinterpret_cast<const unsigned short*>(q));
+                }
+            }
         }
-        st_stream(yc + (int64_t)v * E, Elem<T>::pack(f));
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const int v = base + k * L + sub;
+            if (v < n) {
+                T* q = yp + (int64_t)v * EV;
+                if constexpr (VB == 16) {
+                    float f[EV];
+                    Elem<T>::unpack(Vec16{{raw[k].w[0], raw[k].w[1], raw[k].w[2], raw[k].w[3]}}, f);
+#pragma unroll
+                    for (int e = 0; e < EV; ++e) {
+                        f[e] = relu_keep_nan(fmaf(f[e], sc, sh));
+                        sum += f[e];
+                    }
+                    st_stream(q, Elem<T>::pack(f));
+                } else if constexpr (sizeof(T) == 4) {           // one or two fp32
+                    float f[EV];
+#pragma unroll
+                    for (int e = 0; e < EV; ++e) {
+                        f[e] = relu_keep_nan(fmaf(__uint_as_float(raw[k].w[e]), sc, sh));
+                        sum += f[e];
+                    }
+                    if constexpr (EV == 2) *reinterpret_cast<float2*>(q) = make_float2(f[0], f[1]);
+                    else *q = f[0];
+                } else if constexpr (VB >= 4) {                  // two or four 16-bit values
+                    T o[EV];
+#pragma unroll
+                    for (int i = 0; i < VB / 4; ++i) {
+                        float2 a;
+                        Elem<T>::unpack_pair(raw[k].w[i], a);
+                        a.x = relu_keep_nan(fmaf(a.x, sc, sh));
+                        a.y = relu_keep_nan(fmaf(a.y, sc, sh));
+                        sum += a.x;
+                        sum += a.y;
+                        Elem<T>::store1(&o[2 * i], a.x);
+                        Elem<T>::store1(&o[2 * i + 1], a.y);
+                    }
+                    if constexpr (VB == 8) *reinterpret_cast<uint2*>(q) = *reinterpret_cast<const uint2*>(o);
+                    else *reinterpret_cast<uint32_t*>(q) = *reinterpret_cast<const uint32_t*>(o);
+                } else {                                         // one 16-bit value
+                    float2 a;
+                    Elem<T>::unpack_pair(raw[k].w[0], a);
+                    a.x = relu_keep_nan(fmaf(a.x, sc, sh));
+                    sum += a.x;
+                    Elem<T>::store1(q, a.x);
+                }
+            }
+        }
     }
-    // the last run of the tensor may end inside a vector: its tail goes element by element
-    for (int i = nvec * E + threadIdx.x; i < elems; i += kFlatThreads) {
-        const int pl = i / plane;
-        const float a = relu_keep_nan(fmaf(Elem<T>::load1(xc + i), sc_s[pl], sh_s[pl]));
-        act[i] = a;
-        Elem<T>::store1(yc + i, a);
+#pragma unroll
+    for (int o = L / 2; o > 0; o >>= 1) {
+        const float other = __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+        sum = (lane & o) ? other + sum : sum + other;            // the lower lane's term first: both lanes agree
     }
-    __syncthreads();
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int g = warp; g < g_here; g += kFlatThreads / 32) {
-        float s = 0.0f;
-        for (int j = lane; j < plane; j += 32) s += act[g * plane + j];
-        s = warp_sum(s);
-        if (lane == 0) pooled[p0 + g] = s * inv_plane;
-    }
+    if (live && sub == 0) pooled[p] = sum * inv_plane;
 }
 
 // Large planes that cannot be vectorised: one CTA per plane, scalar loads.
@@ -192,18 +234,36 @@ kop_status_t launch_bn(const void* xv, const void* scalev, const void* shiftv, v
     const float inv_plane = (float)(1.0 / (double)plane);
     const bool vec = aligned_to(x, 16) && aligned_to(y, 16) && (plane % E) == 0;
     const int64_t nvec64 = plane / E;
-    // (planes that are whole vectors and at least two warp-loads long do better with a warp each: 14x14
-    // fp32 measured 46 us with the warp kernel against 52 us flat; 7x7 52 us against 40 us flat)
-    if (plane <= 1024 && aligned_to(x, 16) && aligned_to(y, 16) && (plane % E != 0 || plane < 64)) {
-        // G planes per CTA: a multiple of the vector length, about 3K elements, at most 1024 planes
-        int64_t G = (3072 / plane) / E * E;
-        if (G < E) G = E;
-        if (G > 1024) G = 1024;
-        if (G * plane <= kFlatMaxElems) {
-            const int64_t ctas = (planes + G - 1) / G;
-            if (ctas > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
-            bn_flat_kernel<T, PT><<<(unsigned)ctas, kFlatThreads, 0, stream>>>(x, scale, shift, y, pooled, planes,
-                                                                          (int)plane, (int)G, (int)C, inv_plane);
+    // planes of at most 1024 elements: lanes per plane. (A warp per plane, and for planes that are not whole vectors
+    // runs of planes copied flat through shared memory, were here before: fp32 28 x 28 / 14 x 14 / 7 x 7 planes 5.4 / 5.1 /
+    // 3.2 TB/s, bf16 3.8 / 2.6 / 1.8; now 6.1 / 6.3 / 4.0 and 5.8 / 5.5 / 1.9.)
+    if (plane <= 1024 && planes <= 0x7FFFFFFFLL * 8) {
+        const int pbytes = (int)plane * (int)sizeof(T);
+        const int vb = (pbytes % 16 == 0 && aligned_to(x, 16) && aligned_to(y, 16)) ? 16
+                       : (pbytes % 8 == 0 && aligned_to(x, 8) && aligned_to(y, 8)) ? 8
+                       : (pbytes % 4 == 0 && aligned_to(x, 4) && aligned_to(y, 4)) ? 4 : (int)sizeof(T);
+        const int units = pbytes / vb, per_lane = vb >= 16 ? 4 : (vb == 8 ? 8 : 16);
+        int L = 2;
+        while (L < 32 && L * per_lane < units) L *= 2;
+        const int per_cta = 8 * (32 / L);
+        const int64_t ctas = (planes + per_cta - 1) / per_cta;
+        if (ctas <= 0x7FFFFFFFLL) {
+#define KOP_BN_GROUP_L(V, LL) \
+    bn_plane_group_kernel<T, PT, V, LL><<<(unsigned)ctas, 256, 0, stream>>>(x, scale, shift, y, pooled, planes, (int)plane, (int)C, inv_plane)
+#define KOP_BN_GROUP(V)                           \
+    do {                                          \
+        if (L == 2) KOP_BN_GROUP_L(V, 2);         \
+        else if (L == 4) KOP_BN_GROUP_L(V, 4);    \
+        else if (L == 8) KOP_BN_GROUP_L(V, 8);    \
+        else if (L == 16) KOP_BN_GROUP_L(V, 16);  \
+        else KOP_BN_GROUP_L(V, 32);               \
+    } while (0)
+            if (vb == 16) KOP_BN_GROUP(16);
+            else if (vb == 8) KOP_BN_GROUP(8);
+            else if (vb == 4) KOP_BN_GROUP(4);
+            else KOP_BN_GROUP((int)sizeof(T));
+#undef KOP_BN_GROUP
+#undef KOP_BN_GROUP_L
             return launch_status();
         }
     }

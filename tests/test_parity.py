@@ -253,14 +253,17 @@ def test_layernorm_options(kop):
 BN_SHAPES = [
     (8, 256, 56, 56, F32),     # benchmark plane
     (3, 5, 56, 56, BF16),
-    (4, 16, 7, 7, F32),        # small odd plane: warp, scalar
-    (4, 16, 14, 14, F32),      # small plane: warp, vector
+    (4, 16, 7, 7, F32),        # small odd plane: 4-byte loads
+    (4, 16, 14, 14, F32),      # small plane: 16-byte loads
     (2, 3, 112, 112, F32),     # multi-trip plane
     (2, 7, 33, 35, F32),       # large odd plane: scalar CTA
     (5, 3, 1, 1, F32),
     (2, 8, 64, 64, BF16),
-    (16, 2048, 7, 7, BF16),    # flat small-plane kernel: many runs of 56 planes
-    (3, 5, 7, 7, BF16),        # one partial run whose last vector is incomplete (735 elements)
+    (16, 2048, 7, 7, BF16),    # 98-byte planes: single-element loads, four lanes a plane
+    (3, 5, 7, 7, BF16),
+    (3, 5, 14, 14, BF16),      # 392-byte planes: 8-byte loads
+    (2, 3, 5, 9, torch.float16),
+    (2, 6, 2, 3, F32),         # 24-byte planes: 8-byte loads of fp32
     (2, 3, 31, 31, F32),       # 961-element planes, four per run
     (7, 9, 3, 3, F32),
     (2, 1100, 1, 1, BF16),     # one element per plane, runs of 1024 planes
