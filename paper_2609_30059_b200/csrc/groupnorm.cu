@@ -1,11 +1,12 @@
 // kop_groupnorm_act: GroupNorm (InstanceNorm when groups == C) with optional per-channel affine and an
 // activation, NCHW, in one HBM pass.
 //
-// A CTA owns one (image, group) chunk: (C / groups) * H * W contiguous elements. The chunk is far too
-// long for registers (100 KB for 8 channels of 56x56 fp32) but fits the 227 KB of shared memory a
-// Blackwell CTA can have, so the chunk is fetched into shared memory once (bulk asynchronous copies
-// requested up front), the statistics are accumulated as the parts land, and the normalising sweep
-// re-reads the chunk from shared memory instead of HBM.
+// One (image, group) chunk is (C / groups) * H * W contiguous elements. Chunks up to 40 KB stay in the
+// registers of a team of threads (8 lanes to 10 warps), whatever the plane size. A longer chunk (100 KB
+// for 8 channels of 56x56 fp32) gets a CTA and fits the 227 KB of shared memory a Blackwell CTA can
+// have: it is fetched into shared memory once (bulk asynchronous copies requested up front), the
+// statistics are accumulated as the parts land, and the normalising sweep re-reads the chunk from
+// shared memory instead of HBM.
 // With the chunk on chip the statistics are the exact two-pass ones (mean, then squared deviations from
 // it). Chunks beyond the shared-memory budget take two sweeps over global memory (the second mostly from
 // L2); there, and in the scalar kernel, mean and variance come from one sweep without the
@@ -602,112 +603,272 @@ groupnorm_twosweep_cluster_kernel(const T* __restrict__ x, const PT* __restrict_
     }
 }
 
-// Small chunks (InstanceNorm on 7 x 7 .. 32 x 32 planes, GroupNorm with few channels a group on small maps): a CTA
-// per chunk would be mostly idle threads and fixed costs, and such chunks are often not a whole number of 16-byte
-// vectors. Consecutive chunks are contiguous, so a CTA takes a run of R chunks (R a multiple of the vector length:
-// every run starts on a 16-byte boundary) as one flat array: 16-byte loads across chunk boundaries into shared
-// memory as fp32, one warp per chunk for the exact two-pass statistics out of shared memory, then flat 16-byte
-// stores with each element's chunk and channel carried along the vector.
-constexpr int kGnSmallThreads = 256;
-constexpr int kGnSmallMaxChunk = 2048;           // elements
-constexpr int kGnSmallRunElems = 6144;           // about 24 KB of activations per CTA
+// Chunks up to 40 KB held in registers. A team of threads owns a chunk: 8 lanes of a warp for chunks of at most 64
+// load units, else one to sixteen warps, every thread holding up to eight units. A unit is the widest access
+// (16, 8, 4 bytes or one element) that divides the chunk's bytes and the alignment of both tensors, so a chunk of
+// 16 channels of 14 x 14 bf16 values moves in 16-byte accesses although no plane is a whole vector; a unit then
+// straddles at most two channels (the dispatcher keeps a unit no longer than a plane) and picks gamma / beta per
+// element between the two. Exact two-pass statistics out of the registers; the raw words are kept and widened at
+// each use, which for 16-bit data halves the registers that a widened copy would take.
+template <int VB>
+struct GnUnit {
+    uint32_t w[VB >= 4 ? VB / 4 : 1];
+};
 
-template <typename T, typename PT, int ACT>
-__global__ void __launch_bounds__(kGnSmallThreads)
-groupnorm_small_kernel(const T* __restrict__ x, const PT* __restrict__ gamma, const PT* __restrict__ beta,
-                       T* __restrict__ y, float* __restrict__ mean, float* __restrict__ rstd, int64_t chunks, int R,
-                       int chunk_elems, int plane, int cpg, int groups, float eps)
+template <typename T, int VB>
+__device__ __forceinline__ GnUnit<VB> gn_load(const T* q)
 {
-    constexpr int E = Elem<T>::kPerVec, U = 4;
-    extern __shared__ __align__(16) float gn_small_smem[];
-    float* val = gn_small_smem;                              // R * chunk_elems activations
-    float* mu_s = val + R * chunk_elems;
-    float* rs_s = mu_s + R;
-    const int64_t p0 = (int64_t)blockIdx.x * R;
-    const int r_here = (int)(chunks - p0 < R ? chunks - p0 : R);
-    const int elems = r_here * chunk_elems;
-    const T* xc = x + p0 * chunk_elems;
-    T* yc = y + p0 * chunk_elems;
-    const int nvec = elems / E;
-    for (int base = 0; base < nvec; base += U * kGnSmallThreads) {
-        Vec16 raw[U];
+    GnUnit<VB> r;
+    if constexpr (VB == 16) {
+        const Vec16 t = ld_stream(q);
+        r.w[0] = t.w[0], r.w[1] = t.w[1], r.w[2] = t.w[2], r.w[3] = t.w[3];
+    } else if constexpr (VB == 8) {
+        const uint2 t = __ldg(reinterpret_cast<const uint2*>(q));
+        r.w[0] = t.x, r.w[1] = t.y;
+    } else if constexpr (VB == 4) {
+        r.w[0] = __ldg(reinterpret_cast<const uint32_t*>(q));
+    } else {
+        r.w[0] = __ldg(reinterpret_cast<const unsigned short*>(q));
+    }
+    return r;
+}
+
+template <typename T, int VB>
+__device__ __forceinline__ void gn_widen(const GnUnit<VB>& r, float (&f)[VB / (int)sizeof(T)])
+{
+    if constexpr (sizeof(T) == 4) {
 #pragma unroll
-        for (int k = 0; k < U; ++k) {
-            const int v = base + k * kGnSmallThreads + threadIdx.x;
-            if (v < nvec) raw[k] = ld_stream(xc + (int64_t)v * E);
+        for (int e = 0; e < VB / 4; ++e) f[e] = __uint_as_float(r.w[e]);
+    } else if constexpr (VB >= 4) {
+#pragma unroll
+        for (int i = 0; i < VB / 4; ++i) {
+            float2 a;
+            Elem<T>::unpack_pair(r.w[i], a);
+            f[2 * i] = a.x;
+            f[2 * i + 1] = a.y;
         }
+    } else {
+        float2 a;
+        Elem<T>::unpack_pair(r.w[0], a);
+        f[0] = a.x;
+    }
+}
+
+template <typename T, int VB>
+__device__ __forceinline__ void gn_store(T* q, const float (&f)[VB / (int)sizeof(T)])
+{
+    if constexpr (VB == 16) {
+        st_stream(q, Elem<T>::pack(f));
+    } else if constexpr (sizeof(T) == 4) {
+        if constexpr (VB == 8) *reinterpret_cast<float2*>(q) = make_float2(f[0], f[1]);
+        else *q = f[0];
+    } else if constexpr (VB >= 4) {
+        T o[VB / 2];
 #pragma unroll
-        for (int k = 0; k < U; ++k) {
-            const int v = base + k * kGnSmallThreads + threadIdx.x;
-            if (v < nvec) {
-                float f[E];
-                Elem<T>::unpack(raw[k], f);
-                float4* dst = reinterpret_cast<float4*>(val + v * E);
+        for (int e = 0; e < VB / 2; ++e) Elem<T>::store1(&o[e], f[e]);
+        if constexpr (VB == 8) *reinterpret_cast<uint2*>(q) = *reinterpret_cast<const uint2*>(o);
+        else *reinterpret_cast<uint32_t*>(q) = *reinterpret_cast<const uint32_t*>(o);
+    } else {
+        Elem<T>::store1(q, f[0]);
+    }
+}
+
+// The activation as the other kernels of this file compute it (16-bit SiLU through one hardware tanh).
+template <typename T, int ACT>
+__device__ __forceinline__ float gn_activate(float v)
+{
+    if (ACT == kActSilu && sizeof(T) == 2) {
+        const float h = 0.5f * v;
+        return fmaf(h, tanh_approx(h), h);
+    }
+    return activate<ACT>(v);
+}
+
+constexpr int kGnRegUnits = 8;                   // units a thread holds at most
+constexpr int kGnRegMaxWarps = 16;               // warps of the largest team
+constexpr int kGnRegLanes = 8;                   // lanes of a team inside a warp
+
+// Element pair j of a unit plus c; for 16-bit data the add widens its operand itself (exact, one rounding).
+template <typename T, int VB>
+__device__ __forceinline__ float2 gn_pair_plus(const GnUnit<VB>& r, int j, float2 c)
+{
+    if constexpr (sizeof(T) == 4)
+        return __fadd2_rn(make_float2(__uint_as_float(r.w[2 * j]), __uint_as_float(r.w[2 * j + 1])), c);
+    else
+        return Elem<T>::add_widen2(r.w[j], c);
+}
+
+template <typename T, int ACT>
+__device__ __forceinline__ float2 gn_activate2(float2 u)
+{
+    if (ACT == kActSilu && sizeof(T) == 2) {
+        const float2 h = __fmul2_rn(u, make_float2(0.5f, 0.5f));
+        return __ffma2_rn(h, make_float2(tanh_approx(h.x), tanh_approx(h.y)), h);
+    }
+    if (ACT == kActSilu) {
+        const float2 a = __fmul2_rn(u, make_float2(-kLog2e, -kLog2e));
+        const float2 d = __fadd2_rn(make_float2(ex2_approx(a.x), ex2_approx(a.y)), make_float2(1.0f, 1.0f));
+        return __fmul2_rn(u, make_float2(rcp_approx(d.x), rcp_approx(d.y)));
+    }
+    return make_float2(activate<ACT>(u.x), activate<ACT>(u.y));
+}
+
+// kStraddle: a unit may end in the next channel (planes that are not a whole number of units).
+template <typename T, typename PT, int VB, int NV, int ACT, bool kStraddle>
+__device__ __forceinline__ void gn_reg_normalize(const GnUnit<VB> (&raw)[NV], T* yc, int n, int ts, int tl, int plane,
+                                                 float inv_plane, int c_first, const PT* gamma, const PT* beta,
+                                                 float mu, float rs)
+{
+    constexpr int EU = VB / (int)sizeof(T);
+    const float2 nmu = make_float2(-mu, -mu);
 #pragma unroll
-                for (int q = 0; q < E / 4; ++q) dst[q] = make_float4(f[4 * q], f[4 * q + 1], f[4 * q + 2], f[4 * q + 3]);
+    for (int k = 0; k < NV; ++k) {
+        const int u = k * ts + tl;
+        if (u < n) {
+            const int i0 = u * EU;
+            const int cin = div_small(i0, plane, inv_plane);
+            const int c = c_first + cin;
+            const float sc0 = rs * (gamma != nullptr ? param1(gamma, c) : 1.0f);
+            const float be0 = beta != nullptr ? param1(beta, c) : 0.0f;
+            float sc1 = sc0, be1 = be0;
+            int left = EU;                                   // elements of this unit that belong to channel cin
+            if constexpr (kStraddle && EU > 1) {
+                left = plane - (i0 - cin * plane);
+                if (left < EU) {
+                    sc1 = rs * (gamma != nullptr ? param1(gamma, c + 1) : 1.0f);
+                    be1 = beta != nullptr ? param1(beta, c + 1) : 0.0f;
+                }
             }
-        }
-    }
-    for (int i = nvec * E + threadIdx.x; i < elems; i += kGnSmallThreads)    // the tensor's last run may end inside a vector
-        val[i] = Elem<T>::load1(xc + i);
-    __syncthreads();
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const float inv_count = 1.0f / (float)chunk_elems;
-    for (int r = warp; r < r_here; r += kGnSmallThreads / 32) {
-        const float* cv = val + r * chunk_elems;
-        float s = 0.0f;
-        for (int j = lane; j < chunk_elems; j += 32) s += cv[j];
-        const float mu = warp_sum(s) * inv_count;
-        float q = 0.0f;
-        for (int j = lane; j < chunk_elems; j += 32) {
-            const float d = cv[j] - mu;
-            q = fmaf(d, d, q);
-        }
-        const float rs = rsqrtf(warp_sum(q) * inv_count + eps);
-        if (lane == 0) {
-            mu_s[r] = mu;
-            rs_s[r] = rs;
-            if (mean != nullptr) mean[p0 + r] = mu;
-            if (rstd != nullptr) rstd[p0 + r] = rs;
-        }
-    }
-    __syncthreads();
-    const float inv_chunk = 1.0f / (float)chunk_elems, inv_plane = 1.0f / (float)plane;
-    const int g0 = (int)(p0 % groups);                       // group of the run's first chunk
-    // the normalised value of element i of the run: chunk r, channel ch of the tensor
-    auto out_value = [&](int i, int r, int ch) {
-        const float sc = rs_s[r] * (gamma != nullptr ? param1(gamma, ch) : 1.0f);
-        const float be = beta != nullptr ? param1(beta, ch) : 0.0f;
-        return activate<ACT>(fmaf(val[i] - mu_s[r], sc, be));
-    };
-    for (int v = threadIdx.x; v < nvec; v += kGnSmallThreads) {
-        const int i0 = v * E;
-        int r = div_small(i0, chunk_elems, inv_chunk);
-        int rem = i0 - r * chunk_elems;                      // position inside the chunk
-        int cin = div_small(rem, plane, inv_plane);          // channel inside the group
-        int pos = rem - cin * plane;                         // position inside the plane
-        int grp = g0 + r;
-        grp -= grp >= groups ? (grp / groups) * groups : 0;
-        float f[E];
+            float f[EU];
+            if constexpr (EU >= 2) {
 #pragma unroll
-        for (int e = 0; e < E; ++e) {
-            f[e] = out_value(i0 + e, r, grp * cpg + cin);
-            if (++pos == plane) {
-                pos = 0;
-                if (++cin == cpg) {
-                    cin = 0;
-                    ++r;
-                    if (++grp == groups) grp = 0;
+                for (int j = 0; j < EU / 2; ++j) {
+                    const float2 d = gn_pair_plus<T, VB>(raw[k], j, nmu);
+                    float2 sc = make_float2(sc0, sc0), be = make_float2(be0, be0);
+                    if constexpr (kStraddle) {
+                        if (2 * j >= left) sc.x = sc1, be.x = be1;
+                        if (2 * j + 1 >= left) sc.y = sc1, be.y = be1;
+                    }
+                    const float2 o = gn_activate2<T, ACT>(__ffma2_rn(d, sc, be));
+                    f[2 * j] = o.x;
+                    f[2 * j + 1] = o.y;
+                }
+            } else {
+                gn_widen<T, VB>(raw[k], f);
+                f[0] = gn_activate<T, ACT>(fmaf(f[0] - mu, sc0, be0));
+            }
+            gn_store<T, VB>(yc + i0, f);
+        }
+    }
+}
+
+template <typename T, typename PT, int VB, int NV, int L, bool kStraddle>
+__global__ void __launch_bounds__(kGnRegMaxWarps * 32)
+groupnorm_reg_kernel(const T* __restrict__ x, const PT* __restrict__ gamma, const PT* __restrict__ beta,
+                     T* __restrict__ y, float* __restrict__ mean, float* __restrict__ rstd, int64_t chunks, int units,
+                     int chunk_elems, int plane, int cpg, int groups, float eps, float inv_count, float inv_plane,
+                     int act, int tw)
+{
+    constexpr int EU = VB / (int)sizeof(T);
+    __shared__ float slot_a[kGnRegMaxWarps], slot_b[kGnRegMaxWarps];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int team, tl, ts, per_cta;
+    if constexpr (L < 32) {
+        team = threadIdx.x / L;
+        tl = threadIdx.x & (L - 1);
+        ts = L;
+        per_cta = blockDim.x / L;
+    } else {
+        team = warp / tw;
+        tl = threadIdx.x - team * tw * 32;
+        ts = tw * 32;
+        per_cta = (blockDim.x >> 5) / tw;
+    }
+    const int64_t chunk = (int64_t)blockIdx.x * per_cta + team;
+    const bool live = chunk < chunks;
+    const int n = live ? units : 0;
+    const T* xc = x + (live ? chunk : 0) * chunk_elems;
+    T* yc = y + (live ? chunk : 0) * chunk_elems;
+    GnUnit<VB> raw[NV];
+#pragma unroll
+    for (int k = 0; k < NV; ++k) {
+        const int u = k * ts + tl;
+        if (u < n) {
+            raw[k] = gn_load<T, VB>(xc + u * EU);
+        } else {
+#pragma unroll
+            for (int i = 0; i < (VB >= 4 ? VB / 4 : 1); ++i) raw[k].w[i] = 0u;
+        }
+    }
+    // a team's sum, the same value in all its threads
+    auto team_sum = [&](float v, float* slots) {
+        if constexpr (L < 32) {
+#pragma unroll
+            for (int o = L / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+            return v;
+        } else {
+            v = warp_sum(v);
+            if (tw == 1) return v;
+            if (lane == 0) slots[warp] = v;
+            __syncthreads();
+            return warp_sum(lane < tw ? slots[team * tw + lane] : 0.0f);
+        }
+    };
+    float s = 0.0f;
+    if constexpr (EU >= 2) {
+        float2 s2 = make_float2(0.0f, 0.0f);
+#pragma unroll
+        for (int k = 0; k < NV; ++k)
+#pragma unroll
+            for (int j = 0; j < EU / 2; ++j) s2 = gn_pair_plus<T, VB>(raw[k], j, s2);    // units past the chunk hold zeros
+        s = s2.x + s2.y;
+    } else {
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            float f[EU];
+            gn_widen<T, VB>(raw[k], f);
+            s += f[0];
+        }
+    }
+    const float mu = team_sum(s, slot_a) * inv_count;
+    float q = 0.0f;
+    if constexpr (EU >= 2) {
+        const float2 nmu = make_float2(-mu, -mu);
+        float2 q2 = make_float2(0.0f, 0.0f);
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            if (k * ts + tl < n) {
+#pragma unroll
+                for (int j = 0; j < EU / 2; ++j) {
+                    const float2 d = gn_pair_plus<T, VB>(raw[k], j, nmu);
+                    q2 = __ffma2_rn(d, d, q2);
                 }
             }
         }
-        st_stream(yc + (int64_t)i0, Elem<T>::pack(f));
+        q = q2.x + q2.y;
+    } else {
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            if (k * ts + tl < n) {
+                float f[EU];
+                gn_widen<T, VB>(raw[k], f);
+                const float d = f[0] - mu;
+                q = fmaf(d, d, q);
+            }
+        }
     }
-    for (int i = nvec * E + threadIdx.x; i < elems; i += kGnSmallThreads) {
-        const int r = i / chunk_elems, rem = i - r * chunk_elems;
-        const int grp = (int)((p0 + r) % groups);
-        Elem<T>::store1(yc + i, out_value(i, r, grp * cpg + rem / plane));
+    const float rs = rsqrtf(team_sum(q, slot_b) * inv_count + eps);
+    if (live && tl == 0) {
+        if (mean != nullptr) mean[chunk] = mu;
+        if (rstd != nullptr) rstd[chunk] = rs;
     }
+    const int c_first = (int)(chunk % groups) * cpg;
+    if (act == kActSilu)
+        gn_reg_normalize<T, PT, VB, NV, kActSilu, kStraddle>(raw, yc, n, ts, tl, plane, inv_plane, c_first, gamma, beta, mu, rs);
+    else if (act == kActRelu)
+        gn_reg_normalize<T, PT, VB, NV, kActRelu, kStraddle>(raw, yc, n, ts, tl, plane, inv_plane, c_first, gamma, beta, mu, rs);
+    else
+        gn_reg_normalize<T, PT, VB, NV, kActNone, kStraddle>(raw, yc, n, ts, tl, plane, inv_plane, c_first, gamma, beta, mu, rs);
 }
 
 // Any plane size / alignment: scalar loads, two sweeps over global memory, same moment arithmetic.
@@ -759,27 +920,79 @@ constexpr size_t kGnStageLimit = 200 * 1024;     // leaves room for the static r
 static_assert(kGnStageLimit <= (size_t)kGnMaxParts * kGnCopyVecs * 16, "one barrier per 32 KB part");
 constexpr int kMaxDevices = 64;
 
+// beyond 40 KB (more than ten warps a team) the staged kernel is ahead: bf16 chunks of 49 KB 4.7 against 4.1 TB/s
+constexpr int64_t kGnRegMaxBytes = 40 * 1024;
+
+// Launches the register kernel when the chunk fits a team; false when it does not.
+template <typename T, typename PT, int VB, bool kStraddle>
+bool launch_gn_reg_vb(const T* x, const PT* gamma, const PT* beta, T* y, float* mean, float* rstd, int64_t chunks,
+                      int64_t chunk_elems, int64_t plane, int cpg, int groups, float eps, int act, cudaStream_t stream)
+{
+    const int64_t units = chunk_elems * (int64_t)sizeof(T) / VB;
+    const float inv_count = (float)(1.0 / (double)chunk_elems), inv_plane = (float)(1.0 / (double)plane);
+#define KOP_GN_REG_GO(NV, L, CTAS, THREADS, TW)                                                                       \
+    groupnorm_reg_kernel<T, PT, VB, NV, L, kStraddle><<<(unsigned)(CTAS), (unsigned)(THREADS), 0, stream>>>(         \
+        x, gamma, beta, y, mean, rstd, chunks, (int)units, (int)chunk_elems, (int)plane, cpg, groups, eps, inv_count, \
+        inv_plane, act, (int)(TW))
+    if (units <= kGnRegLanes * kGnRegUnits) {
+        constexpr int kThreads = 128, kTeams = kThreads / kGnRegLanes;
+        const int64_t ctas = (chunks + kTeams - 1) / kTeams;
+        if (ctas > 0x7FFFFFFFLL) return false;
+        if (units <= kGnRegLanes * 2) KOP_GN_REG_GO(2, kGnRegLanes, ctas, kThreads, 1);
+        else KOP_GN_REG_GO(kGnRegUnits, kGnRegLanes, ctas, kThreads, 1);
+        return true;
+    }
+    // eight units a thread keep the most bytes in flight, four fill the team's last sweep better when the chunk
+    // is a small number of warp sweeps (98 units: 38 % of the slots of one warp at eight, 77 % at four)
+    const int64_t tw8 = (units + 32 * kGnRegUnits - 1) / (32 * kGnRegUnits);
+    const int64_t tw4 = (units + 16 * kGnRegUnits - 1) / (16 * kGnRegUnits);
+    bool eight = (double)units / (double)(tw8 * 32 * kGnRegUnits) >= 0.85 * (double)units / (double)(tw4 * 16 * kGnRegUnits);
+    if (!eight && tw4 > kGnRegMaxWarps) eight = true;
+    const int64_t tw = eight ? tw8 : tw4;
+    if (tw > kGnRegMaxWarps) return false;
+    const int teams = tw >= 4 ? 1 : 4 / (int)tw;
+    const int64_t ctas = (chunks + teams - 1) / teams;
+    if (ctas > 0x7FFFFFFFLL) return false;
+    if (eight) KOP_GN_REG_GO(kGnRegUnits, 32, ctas, teams * tw * 32, tw);
+    else KOP_GN_REG_GO(kGnRegUnits / 2, 32, ctas, teams * tw * 32, tw);
+#undef KOP_GN_REG_GO
+    return true;
+}
+
+template <typename T, typename PT>
+bool launch_gn_reg(const T* x, const PT* gamma, const PT* beta, T* y, float* mean, float* rstd, int64_t chunks,
+                   int64_t chunk_elems, int64_t plane, int cpg, int groups, float eps, int act, cudaStream_t stream)
+{
+    constexpr int esz = (int)sizeof(T);
+    const int64_t bytes = chunk_elems * esz;
+    if (bytes > kGnRegMaxBytes) return false;
+    int vb = 16;
+    while (vb > esz && (bytes % vb != 0 || !aligned_to(x, vb) || !aligned_to(y, vb) || vb / esz > plane)) vb >>= 1;
+#define KOP_GN_REG(VB)                                                                                                \
+    ((VB) > esz && plane % ((VB) / esz) != 0                                                                          \
+         ? launch_gn_reg_vb<T, PT, VB, (VB > esz)>(x, gamma, beta, y, mean, rstd, chunks, chunk_elems, plane, cpg,    \
+                                                   groups, eps, act, stream)                                          \
+         : launch_gn_reg_vb<T, PT, VB, false>(x, gamma, beta, y, mean, rstd, chunks, chunk_elems, plane, cpg, groups, \
+                                              eps, act, stream))
+    switch (vb) {
+    case 16: return KOP_GN_REG(16);
+    case 8: return KOP_GN_REG(8);
+    case 4: return KOP_GN_REG(4);
+    default:
+        if constexpr (esz == 2) return KOP_GN_REG(2);
+        else return false;
+    }
+#undef KOP_GN_REG
+}
+
 template <typename T, typename PT, int ACT>
 kop_status_t launch_gn_act(const T* x, const PT* gamma, const PT* beta, T* y, float* mean, float* rstd,
                            int64_t chunks, int64_t chunk_elems, int64_t plane, int cpg, int groups, float eps,
                            cudaStream_t stream)
 {
     constexpr int E = Elem<T>::kPerVec;
-    // up to 512 elements always (14 x 14 InstanceNorm: 1.2 TB/s staged, 2.8 TB/s this way; at 1024 elements the
-    // staged kernel is ahead again, 4.1 against 3.7); up to 2048 when the planes are not whole vectors and the
-    // alternative is the scalar kernel
-    if ((chunk_elems <= 512 || (chunk_elems <= kGnSmallMaxChunk && plane % E != 0)) && aligned_to(x, 16) &&
-        aligned_to(y, 16)) {
-        int R = (int)((kGnSmallRunElems / chunk_elems) / E * E);
-        if (R < E) R = E;
-        const int64_t ctas = (chunks + R - 1) / R;
-        const size_t smem = ((size_t)R * chunk_elems + 2 * (size_t)R) * sizeof(float);
-        if (ctas <= 0x7FFFFFFFLL && smem <= 47 * 1024) {
-            groupnorm_small_kernel<T, PT, ACT><<<(unsigned)ctas, kGnSmallThreads, smem, stream>>>(
-                x, gamma, beta, y, mean, rstd, chunks, R, (int)chunk_elems, (int)plane, cpg, groups, eps);
-            return launch_status();
-        }
-    }
+    if (launch_gn_reg<T, PT>(x, gamma, beta, y, mean, rstd, chunks, chunk_elems, plane, cpg, groups, eps, ACT, stream))
+        return launch_status();
     const bool vec = aligned_to(x, 16) && aligned_to(y, 16) && (plane % E) == 0 && chunk_elems / E <= 0x7FFFFFFF;
     if (vec) {
         const int nvec = (int)(chunk_elems / E);

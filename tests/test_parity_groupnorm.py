@@ -1,8 +1,10 @@
 """GPU parity of kop_groupnorm_act (GroupNorm / InstanceNorm with optional affine and activation)
-against the float64 CPU oracle: five seeds over shapes that hit the shared-memory-staged kernel
-(one and several parts, ragged last part, several waves of CTAs), the two-sweep kernel (chunks beyond the staging budget)
-and the scalar kernel (planes that do not split into 16-byte vectors, misaligned bases), all three
-activations, missing affine parameters, in-place use, guard bands and run-to-run bit equality.
+against the float64 CPU oracle: five seeds over shapes that hit the register kernel (chunks up to 40 KB: teams of
+8 lanes, of one warp and of several, every load width, units that straddle two channels), the
+shared-memory-staged kernel (one and several parts, ragged last part, several waves of CTAs), the cluster and
+two-sweep kernels (chunks beyond the staging budget) and the scalar kernel (long chunks that do not split into
+16-byte vectors), all three activations, missing affine parameters, in-place use, misaligned bases, guard bands
+and run-to-run bit equality.
 
 Tolerance: |got - ref| <= tol * max(1, |ref|), tol = 1e-5 for fp32 data and 2e-2 for bf16 data;
 the fp32 statistics are held to 1e-5 for both data types."""
@@ -46,21 +48,28 @@ GN_SHAPES = [
     (2, 12, 256, 256, 3, BF16, 2),     # six chunks of 512 KB bf16 (staged cluster); 1 MB fp32 below
     (2, 12, 256, 256, 3, F32, 1),      # six chunks of 1 MB: shared by clusters of 8, uneven slices
     (1, 6, 256, 256, 3, torch.float16, 2),   # 256 KB fp16: cluster of 4
-    (3, 12, 7, 7, 4, F32, 2),          # plane 49: scalar kernel
-    (3, 12, 5, 6, 3, BF16, 0),         # plane 30 bf16: scalar kernel (30 % 8 != 0)
-    (2, 8, 2, 2, 4, F32, 1),           # plane of one vector, chunk shorter than a warp's worth
+    (3, 12, 7, 7, 4, F32, 2),          # plane 49, chunk of 147: 4-byte units
+    (3, 12, 5, 6, 3, BF16, 0),         # plane 30 bf16: 16-byte units that straddle channels (30 % 8 != 0)
+    (2, 8, 2, 2, 4, F32, 1),           # plane of one vector, chunk of two
     (5, 3, 1, 1, 3, F32, 0),           # one element per group: variance 0, y = beta
     (1, 16, 4, 4, 2, BF16, 2),
     (10, 256, 56, 56, 32, F32, 0),     # 320 chunks of 100 KB: more CTAs than fit the GPU at once
     (80, 64, 56, 56, 8, BF16, 1),      # 640 chunks of 50 KB
-    # small chunks: runs of chunks per CTA, vectors that cross chunk, channel and group boundaries, a last run
-    # that ends inside a vector, runs that wrap around the group index
-    (9, 37, 7, 7, 37, F32, 2),         # InstanceNorm 7 x 7
-    (5, 48, 14, 14, 48, BF16, 2),      # InstanceNorm 14 x 14 bf16
-    (7, 30, 7, 7, 5, F32, 1),          # 6 channels of 49 a group
-    (3, 21, 5, 3, 7, torch.float16, 0),
-    (11, 64, 4, 4, 32, BF16, 2),       # 2 channels of 16 a group
-    (2, 2048, 7, 7, 32, F32, 2),       # 64 channels of 49: 3136 elements, beyond the small kernel (scalar)
+    # chunks held in registers: every team size and load width, the last CTA's idle teams
+    (9, 37, 7, 7, 37, F32, 2),         # InstanceNorm 7 x 7: 49 units of 4 bytes, 8 lanes a chunk
+    (5, 48, 14, 14, 48, BF16, 2),      # InstanceNorm 14 x 14 bf16: 49 units of 8 bytes
+    (7, 30, 7, 7, 5, F32, 1),          # 6 channels of 49 a group: 8-byte units that straddle channels
+    (3, 21, 5, 3, 7, torch.float16, 0),   # 45 elements: 2-byte units
+    (11, 64, 4, 4, 32, BF16, 2),       # 2 channels of 16 a group: 4 units, two a lane
+    (3, 16, 2, 2, 4, BF16, 2),         # plane of 4 bf16: the unit shrinks to 8 bytes to stay inside two channels
+    (4, 6, 6, 6, 6, torch.float16, 1),    # 72 bytes a chunk: 8-byte units
+    (2, 2048, 7, 7, 32, F32, 2),       # 64 channels of 49: 784 units of 16 bytes that straddle, four warps a chunk
+    (3, 64, 14, 14, 4, BF16, 2),       # 16 channels of 14 x 14 bf16: 392 straddling units, two warps a chunk
+    (5, 52, 14, 14, 13, F32, 1),       # 196 units: a warp a chunk, four chunks a CTA, 65 chunks (one idle team)
+    (3, 40, 8, 8, 2, F32, 2),          # 320 units: three warps of four units a thread
+    (7, 24, 10, 10, 12, BF16, 0),      # 25 units of 16 bytes: 8 lanes, four units a lane at most
+    (3, 20, 32, 32, 2, F32, 2),        # 40 KB: ten warps a chunk, the longest register chunk
+    (2, 22, 32, 32, 2, F32, 0),        # 44 KB: the first staged chunk
     (6, 40, 7, 7, 1, F32, 0),          # groups == 1, chunk of 1960
 ]
 
@@ -124,13 +133,23 @@ def test_groupnorm_options(kop):
     rb = kopref.groupnorm_act(host(xb), host(gb), host(bb), 2, 1e-5, 2, threads=None)[0]
     kop.kop_groupnorm_act(xb, gb, bb, 2, 1e-5, 2, out=xb)
     assert_close(xb, rb, 2e-2, "groupnorm in place unstaged")
-    # a base that is 4-byte but not 16-byte aligned takes the scalar kernel
+    # a base that is 4-byte but not 16-byte aligned: 4-byte units
     buf = torch.zeros(N * C * H * W + 1, dtype=F32, device="cuda")
     xo = buf[1:].view(N, C, H, W)
     xo.copy_(x)
     yo = torch.zeros(N * C * H * W + 1, dtype=F32, device="cuda")[1:].view(N, C, H, W)
     kop.kop_groupnorm_act(xo, gamma, beta, G, 1e-5, 2, out=yo)
     assert_close(yo, ry, 1e-5, "groupnorm misaligned base")
+    # a bf16 base that is only 2-byte aligned (one-element units), short and long chunks
+    for shp, grp in (((3, 8, 6, 6), 4), ((1, 4, 96, 96), 2)):
+        xh, gh, bh = synth.groupnorm_inputs(*shp, BF16, 5, "cuda")
+        n = xh.numel()
+        xo = torch.zeros(n + 1, dtype=BF16, device="cuda")[1:].view(*shp)
+        xo.copy_(xh)
+        yo = torch.zeros(n + 1, dtype=BF16, device="cuda")[1:].view(*shp)
+        kop.kop_groupnorm_act(xo, gh, bh, grp, 1e-5, 2, out=yo)
+        assert_close(yo, kopref.groupnorm_act(host(xh), host(gh), host(bh), grp, 1e-5, 2, threads=None)[0], 2e-2,
+                     "groupnorm bf16 misaligned base")
     # large offset, small spread: the one-sweep statistics must not lose the variance to cancellation
     xs = (x * 1e-2 + 100.0).contiguous()
     y, m, r = kop.kop_groupnorm_act(xs, gamma, beta, G, 1e-5, 0)
