@@ -191,6 +191,47 @@ __device__ __forceinline__ void ce_finish(float M, float S, float Z, const T* zr
     ce_after_ticket<kOpts>(t, row, lane, labels, loss, mean_loss, bad_label_count, ws, rows, vocab, opts);
 }
 
+// A row of any length and alignment as head elements (up to the first 16-byte boundary), whole 16-byte vectors
+// and tail elements: at most 2 (E - 1) elements outside the vectors, taken one per thread before the vector sweep.
+template <typename T>
+struct CeRowSplit {
+    const T* mid;        // first 16-byte boundary at or after the row's start
+    int head, nvec, tail;
+};
+
+template <typename T>
+__device__ __forceinline__ CeRowSplit<T> ce_split(const T* zr, int64_t vocab)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    CeRowSplit<T> r;
+    int head = (int)(((16u - (unsigned)(reinterpret_cast<uintptr_t>(zr) & 15u)) & 15u) / (unsigned)sizeof(T));
+    if ((int64_t)head > vocab) head = (int)vocab;
+    r.head = head;
+    r.mid = zr + head;
+    r.nvec = (int)((vocab - head) / E);
+    r.tail = (int)(vocab - head) - r.nvec * E;
+    return r;
+}
+
+// Edge element i (0 .. head + tail - 1) of a split row enters a thread's still empty (M, S, Z).
+template <typename T, bool kSum>
+__device__ __forceinline__ void ce_edge(const T* zr, const CeRowSplit<T>& sp, int i, float& M, float& S, float& Z)
+{
+    const int j = i < sp.head ? i : sp.head + sp.nvec * Elem<T>::kPerVec + (i - sp.head);
+    const float xj = Elem<T>::load1(zr + j);
+    if (kSum) Z += xj;
+    const float x2 = xj * kLog2e;
+    if (x2 == -INFINITY) return;
+    if (x2 > M) {
+        // + 1 for this element; (x2 - x2) is 0 for a number and NaN for +inf, where the max-shifted
+        // definition has exp(inf - inf): the row becomes NaN as in the vector sweep
+        S = S * ex2_approx(M - x2) + (1.0f + (x2 - x2));
+        M = x2;
+    } else {
+        S += ex2_approx(x2 - M);                             // a NaN element: S becomes NaN, M stays
+    }
+}
+
 // One batch of VPT vectors per thread: loads first (all in flight), then the batch maximum on the
 // packed values, then one ex2 per element against the updated running offset.
 template <typename T, int VPT, bool kTail, bool kSum>
@@ -265,18 +306,22 @@ template <typename T, int VPT, bool kOpts, bool kSmooth>
 __global__ void __launch_bounds__(256, 8)
 ce_row_kernel(const T* __restrict__ z, const int32_t* __restrict__ labels, float* __restrict__ loss,
               float* __restrict__ mean_loss, int32_t* __restrict__ bad_label_count,
-              CeWorkspace ws, int64_t rows, int nvec, int64_t row_stride, int64_t vocab, CeOpts opts)
+              CeWorkspace ws, int64_t rows, int64_t row_stride, int64_t vocab, CeOpts opts)
 {
     const int64_t row = blockIdx.x;
     const T* zr = z + row * row_stride;
     float M = -INFINITY, S = 0.0f, Z = 0.0f;
+    CeRowSplit<T> sp = ce_split<T>(zr, vocab);
     // An ignored row is not read at all: it only takes its tickets.
-    if (kOpts && __ldg(labels + row) == opts.ignore_index) nvec = 0;
+    if (kOpts && __ldg(labels + row) == opts.ignore_index) sp.head = sp.nvec = sp.tail = 0;
+    if ((int)threadIdx.x < sp.head + sp.tail) ce_edge<T, kSmooth>(zr, sp, threadIdx.x, M, S, Z);
     // One loop body with bounds predicates on every batch (out-of-range vectors read as -inf). A
     // predicate-free main loop plus a separate tail batch doubled the inlined body, pushed the kernel
     // from 32 to 40 registers (six CTAs per SM instead of eight) and measured 3-6 % slower.
     const int step = VPT * blockDim.x;
-    for (int base = 0; base < nvec; base += step) ce_batch<T, VPT, true, kSmooth>(zr, base, nvec, M, S, Z);
+    const int nvec = sp.nvec;
+    const T* zm = sp.mid;
+    for (int base = 0; base < nvec; base += step) ce_batch<T, VPT, true, kSmooth>(zm, base, nvec, M, S, Z);
     ce_finish<T, kOpts, kSmooth>(M, S, Z, zr, labels, loss, mean_loss, bad_label_count, ws, row, rows, vocab, opts);
 }
 
@@ -290,7 +335,7 @@ template <typename T, int L, bool kOpts, bool kSmooth>
 __global__ void __launch_bounds__(256)
 ce_group_kernel(const T* __restrict__ z, const int32_t* __restrict__ labels, float* __restrict__ loss,
                 float* __restrict__ mean_loss, int32_t* __restrict__ bad_label_count, CeWorkspace ws,
-                int64_t rows, int nvec, int64_t row_stride, int64_t vocab, CeOpts opts)
+                int64_t rows, int64_t row_stride, int64_t vocab, CeOpts opts)
 {
     constexpr int E = Elem<T>::kPerVec, U = 4;
     constexpr int kRowsPerWarp = 32 / L;
@@ -299,16 +344,20 @@ ce_group_kernel(const T* __restrict__ z, const int32_t* __restrict__ labels, flo
     const int64_t row = warp_row0 + lane / L;
     const bool live = row < rows;
     const T* zr = z + (live ? row : 0) * row_stride;
-    int n = live ? nvec : 0;
-    if (kOpts && live && __ldg(labels + row) == opts.ignore_index) n = 0;     // an ignored row is not read
+    CeRowSplit<T> sp = ce_split<T>(zr, vocab);
+    // a row past the end and an ignored row are not read
+    if (!live || (kOpts && __ldg(labels + row) == opts.ignore_index)) sp.head = sp.nvec = sp.tail = 0;
+    const int n = sp.nvec;
+    const T* zm = sp.mid;
     float M = -INFINITY, S = 0.0f, Z = 0.0f;
+    for (int i = sub; i < sp.head + sp.tail; i += L) ce_edge<T, kSmooth>(zr, sp, i, M, S, Z);
     for (int base = 0; base < n; base += U * L) {
         Vec16 raw[U];
 #pragma unroll
         for (int k = 0; k < U; ++k) {
             const int v = base + k * L + sub;
             raw[k] = Elem<T>::fill_neg_inf();
-            if (v < n) raw[k] = ld_stream(zr + (int64_t)v * E);
+            if (v < n) raw[k] = ld_stream(zm + (int64_t)v * E);
         }
         float cm = vec_max<T>(raw[0]);
 #pragma unroll
@@ -373,35 +422,6 @@ ce_group_kernel(const T* __restrict__ z, const int32_t* __restrict__ labels, flo
     ce_after_ticket<kOpts>(t, warp_row0, lane, labels, loss, mean_loss, bad_label_count, ws, rows, vocab, opts);
 }
 
-// Any vocab / alignment: scalar loads, element-wise online recurrence.
-template <typename T, bool kOpts>
-__global__ void __launch_bounds__(256)
-ce_row_scalar_kernel(const T* __restrict__ z, const int32_t* __restrict__ labels,
-                     float* __restrict__ loss, float* __restrict__ mean_loss,
-                     int32_t* __restrict__ bad_label_count, CeWorkspace ws,
-                     int64_t rows, int64_t row_stride, int64_t vocab, CeOpts opts)
-{
-    const int64_t row = blockIdx.x;
-    const T* zr = z + row * row_stride;
-    float M = -INFINITY, S = 0.0f, Z = 0.0f;
-    const int64_t n = (kOpts && __ldg(labels + row) == opts.ignore_index) ? 0 : vocab;
-    for (int64_t j = threadIdx.x; j < n; j += blockDim.x) {
-        const float xj = Elem<T>::load1(zr + j);
-        if (kOpts) Z += xj;
-        const float x2 = xj * kLog2e;
-        if (x2 == -INFINITY) continue;
-        if (x2 > M) {
-            // + 1 for this element; (x2 - x2) is 0 for a number and NaN for +inf, where the max-shifted
-            // definition has exp(inf - inf): the row becomes NaN as in the vector kernels
-            S = S * ex2_approx(M - x2) + (1.0f + (x2 - x2));
-            M = x2;
-        } else {
-            S += ex2_approx(x2 - M);
-        }
-    }
-    ce_finish<T, kOpts, kOpts>(M, S, Z, zr, labels, loss, mean_loss, bad_label_count, ws, row, rows, vocab, opts);
-}
-
 template <typename T, bool kOpts>
 kop_status_t launch_ce(const void* zv, const int32_t* labels, float* loss, float* mean_loss,
                        int32_t* bad, int64_t rows, int64_t vocab, int64_t stride, void* workspace,
@@ -411,14 +431,15 @@ kop_status_t launch_ce(const void* zv, const int32_t* labels, float* loss, float
     constexpr int E = Elem<T>::kPerVec;
     const CeWorkspace ws = ce_workspace(workspace, rows);
     if (cudaMemsetAsync(workspace, 0, ce_workspace_clear_bytes(rows), stream) != cudaSuccess) return KOP_ERR_CUDA;
-    const bool vec = vec_ok(z, vocab, stride, sizeof(T));
+    // every row is split in the kernel into head elements, whole 16-byte vectors and tail elements, so any vocabulary
+    // size, row stride and base alignment takes the vector kernels
     const int64_t nvec64 = vocab / E;
-    if (vec && vocab * (int64_t)sizeof(T) <= 16384) {
+    if (vocab * (int64_t)sizeof(T) <= 16384) {
         const int nvec = (int)nvec64;
         const int lanes = nvec >= 512 ? 32 : nvec >= 256 ? 16 : nvec >= 128 ? 8 : 4;
         const int64_t rows_per_cta = 8 * (32 / lanes);
         const unsigned grid = (unsigned)((rows + rows_per_cta - 1) / rows_per_cta);
-#define KOP_CE_G(L, SM) ce_group_kernel<T, L, kOpts, SM><<<grid, 256, 0, stream>>>(z, labels, loss, mean_loss, bad, ws, rows, nvec, stride, vocab, opts)
+#define KOP_CE_G(L, SM) ce_group_kernel<T, L, kOpts, SM><<<grid, 256, 0, stream>>>(z, labels, loss, mean_loss, bad, ws, rows, stride, vocab, opts)
 #define KOP_CE_GROUP(L)                                            \
     do {                                                           \
         if (kOpts && opts.smoothing > 0.0f) KOP_CE_G(L, true);     \
@@ -434,27 +455,22 @@ kop_status_t launch_ce(const void* zv, const int32_t* labels, float* loss, float
 #undef KOP_CE_GROUP
         return launch_status();
     }
-    if (vec && nvec64 <= 0x7FFFFFFF) {
-        const int nvec = (int)nvec64;
-        const int threads = 256;
-        const int per = (nvec + threads - 1) / threads;
-        // Batches of at most four vectors per thread: ~50 registers, so five 256-thread CTAs stay
-        // resident per SM and their load and exp phases interleave. Larger batches (more bytes in
-        // flight per thread, fewer resident warps) measured 5-30 % slower on a 32000-wide bf16 row.
-#define KOP_CE_L(V, SM) ce_row_kernel<T, V, kOpts, SM><<<(unsigned)rows, threads, 0, stream>>>(z, labels, loss, mean_loss, bad, ws, rows, nvec, stride, vocab, opts)
+    const int threads = 256;
+    const int64_t per = (nvec64 + threads - 1) / threads;
+    // Batches of at most four vectors per thread: ~50 registers, so five 256-thread CTAs stay
+    // resident per SM and their load and exp phases interleave. Larger batches (more bytes in
+    // flight per thread, fewer resident warps) measured 5-30 % slower on a 32000-wide bf16 row.
+#define KOP_CE_L(V, SM) ce_row_kernel<T, V, kOpts, SM><<<(unsigned)rows, threads, 0, stream>>>(z, labels, loss, mean_loss, bad, ws, rows, stride, vocab, opts)
 #define KOP_CE(V)                                                  \
     do {                                                           \
         if (kOpts && opts.smoothing > 0.0f) KOP_CE_L(V, true);     \
         else KOP_CE_L(V, false);                                   \
     } while (0)
-        if (per <= 1) KOP_CE(1);
-        else if (per <= 2) KOP_CE(2);
-        else KOP_CE(4);
+    if (per <= 1) KOP_CE(1);
+    else if (per <= 2) KOP_CE(2);
+    else KOP_CE(4);
 #undef KOP_CE
 #undef KOP_CE_L
-        return launch_status();
-    }
-    ce_row_scalar_kernel<T, kOpts><<<(unsigned)rows, 256, 0, stream>>>(z, labels, loss, mean_loss, bad, ws, rows, stride, vocab, opts);
     return launch_status();
 }
 

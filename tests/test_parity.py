@@ -458,7 +458,14 @@ CE_SHAPES = [
     (100, 50264, BF16),    # multi-batch rows (more than 16 vectors per thread)
     (64, 131072, BF16),
     (33, 1000, F32),
-    (21, 32001, BF16),     # odd vocab: scalar
+    (21, 32001, BF16),     # odd vocab: every row starts at another offset from a 16-byte boundary
+    (37, 50257, BF16),     # head and tail elements around the aligned vectors, several batches a thread
+    (19, 50257, F32),
+    (300, 1001, BF16),     # odd and short: lanes per row with edge elements
+    (523, 197, F32),
+    (1000, 77, torch.float16),
+    (200, 7, BF16),        # shorter than one vector: edge elements only
+    (64, 4102, F32),       # every second row starts 8 bytes off a boundary
     (9, 1, F32),
     (5, 8, BF16),
     # small vocabularies (rows of at most 16 KB): 4, 8, 16 and 32 lanes of a warp per row; row counts that span
@@ -777,7 +784,8 @@ def test_silu_mul_interleaved_parity(kop, rows, inter, dtype, seed):
 
 
 @pytest.mark.parametrize("rows,vocab,dtype", [(2048, 32000, BF16), (300, 4096, F32), (257, 50264, BF16), (21, 32001, BF16), (9, 8, F32),
-                                              (1300, 1000, BF16), (523, 2048, BF16), (2051, 40, F32), (67, 8192, BF16)])
+                                              (1300, 1000, BF16), (523, 2048, BF16), (2051, 40, F32), (67, 8192, BF16),
+                                              (37, 50257, BF16), (300, 197, F32), (129, 1001, torch.float16)])
 @pytest.mark.parametrize("smoothing", [0.0, 0.1])
 @pytest.mark.parametrize("seed", SEEDS[:3])
 def test_ce_opts_parity(kop, rows, vocab, dtype, smoothing, seed):
@@ -843,7 +851,9 @@ def test_ce_opts_edge_cases(kop):
                                          (4096, BF16),      # 32 lanes per row
                                          (1024, F32),       # lanes-per-row kernel, 8-vector rows
                                          (64, BF16),        # four lanes per row
-                                         (1001, F32),       # odd length: scalar kernel
+                                         (1001, F32),       # odd length: lanes per row with edge elements
+                                         (197, BF16),
+                                         (50257, BF16),     # odd and long: edge elements around the vector sweep
                                          (40000, F32)])
 def test_ce_non_finite_logits(kop, vocab, dtype):
     """NaN and +inf logits make exactly their own row NaN, whichever kernel the shape selects and wherever in the
