@@ -26,8 +26,9 @@
  *              must be >= the row length.
  *   alignment  16-byte-aligned bases, row strides and row lengths take the 128-bit
  *              vector kernels; anything else runs a GPU kernel of the same arithmetic
- *              with narrower accesses (kop_ce_loss_rowwise and kop_groupnorm_act keep
- *              128-bit accesses for any length and alignment). There is no CPU path.
+ *              with narrower accesses (the cross-entropy, softmax and GroupNorm entry
+ *              points keep 128-bit accesses for any length and alignment). There is no
+ *              CPU path.
  *   aliasing   Where stated, the output may be exactly the input (same pointer and
  *              stride). Any other overlap returns KOP_ERR_BAD_ALIAS when detectable
  *              and is undefined otherwise.

@@ -191,33 +191,13 @@ __device__ __forceinline__ void ce_finish(float M, float S, float Z, const T* zr
     ce_after_ticket<kOpts>(t, row, lane, labels, loss, mean_loss, bad_label_count, ws, rows, vocab, opts);
 }
 
-// A row of any length and alignment as head elements (up to the first 16-byte boundary), whole 16-byte vectors
-// and tail elements: at most 2 (E - 1) elements outside the vectors, taken one per thread before the vector sweep.
-template <typename T>
-struct CeRowSplit {
-    const T* mid;        // first 16-byte boundary at or after the row's start
-    int head, nvec, tail;
-};
-
-template <typename T>
-__device__ __forceinline__ CeRowSplit<T> ce_split(const T* zr, int64_t vocab)
-{
-    constexpr int E = Elem<T>::kPerVec;
-    CeRowSplit<T> r;
-    int head = (int)(((16u - (unsigned)(reinterpret_cast<uintptr_t>(zr) & 15u)) & 15u) / (unsigned)sizeof(T));
-    if ((int64_t)head > vocab) head = (int)vocab;
-    r.head = head;
-    r.mid = zr + head;
-    r.nvec = (int)((vocab - head) / E);
-    r.tail = (int)(vocab - head) - r.nvec * E;
-    return r;
-}
-
+// Rows of any length and alignment are split (row_split) into head elements, whole 16-byte vectors and tail
+// elements; the edge elements are taken one per thread before the vector sweep.
 // Edge element i (0 .. head + tail - 1) of a split row enters a thread's still empty (M, S, Z).
 template <typename T, bool kSum>
-__device__ __forceinline__ void ce_edge(const T* zr, const CeRowSplit<T>& sp, int i, float& M, float& S, float& Z)
+__device__ __forceinline__ void ce_edge(const T* zr, const RowSplit<T>& sp, int i, float& M, float& S, float& Z)
 {
-    const int j = i < sp.head ? i : sp.head + sp.nvec * Elem<T>::kPerVec + (i - sp.head);
+    const int j = sp.edge_col(i);
     const float xj = Elem<T>::load1(zr + j);
     if (kSum) Z += xj;
     const float x2 = xj * kLog2e;
@@ -311,7 +291,7 @@ ce_row_kernel(const T* __restrict__ z, const int32_t* __restrict__ labels, float
     const int64_t row = blockIdx.x;
     const T* zr = z + row * row_stride;
     float M = -INFINITY, S = 0.0f, Z = 0.0f;
-    CeRowSplit<T> sp = ce_split<T>(zr, vocab);
+    RowSplit<T> sp = row_split<T>(zr, vocab);
     // An ignored row is not read at all: it only takes its tickets.
     if (kOpts && __ldg(labels + row) == opts.ignore_index) sp.head = sp.nvec = sp.tail = 0;
     if ((int)threadIdx.x < sp.head + sp.tail) ce_edge<T, kSmooth>(zr, sp, threadIdx.x, M, S, Z);
@@ -320,7 +300,7 @@ ce_row_kernel(const T* __restrict__ z, const int32_t* __restrict__ labels, float
     // from 32 to 40 registers (six CTAs per SM instead of eight) and measured 3-6 % slower.
     const int step = VPT * blockDim.x;
     const int nvec = sp.nvec;
-    const T* zm = sp.mid;
+    const T* zm = zr + sp.head;
     for (int base = 0; base < nvec; base += step) ce_batch<T, VPT, true, kSmooth>(zm, base, nvec, M, S, Z);
     ce_finish<T, kOpts, kSmooth>(M, S, Z, zr, labels, loss, mean_loss, bad_label_count, ws, row, rows, vocab, opts);
 }
@@ -344,11 +324,11 @@ ce_group_kernel(const T* __restrict__ z, const int32_t* __restrict__ labels, flo
     const int64_t row = warp_row0 + lane / L;
     const bool live = row < rows;
     const T* zr = z + (live ? row : 0) * row_stride;
-    CeRowSplit<T> sp = ce_split<T>(zr, vocab);
+    RowSplit<T> sp = row_split<T>(zr, vocab);
     // a row past the end and an ignored row are not read
     if (!live || (kOpts && __ldg(labels + row) == opts.ignore_index)) sp.head = sp.nvec = sp.tail = 0;
     const int n = sp.nvec;
-    const T* zm = sp.mid;
+    const T* zm = zr + sp.head;
     float M = -INFINITY, S = 0.0f, Z = 0.0f;
     for (int i = sub; i < sp.head + sp.tail; i += L) ce_edge<T, kSmooth>(zr, sp, i, M, S, Z);
     for (int base = 0; base < n; base += U * L) {

@@ -407,6 +407,32 @@ __device__ __forceinline__ float warp_max(float v)
     return v;
 }
 
+// A row of any length and alignment as head elements (up to the first 16-byte boundary), whole 16-byte vectors
+// and tail elements: at most 2 (E - 1) edge elements outside the vectors.
+template <typename T>
+struct RowSplit {
+    int head, nvec, tail;
+    __device__ __forceinline__ int edges() const { return head + tail; }
+    // column of edge element i (0 .. head + tail - 1)
+    __device__ __forceinline__ int edge_col(int i) const
+    {
+        return i < head ? i : head + nvec * Elem<T>::kPerVec + (i - head);
+    }
+};
+
+template <typename T>
+__device__ __forceinline__ RowSplit<T> row_split(const T* row, int64_t cols)
+{
+    constexpr int E = Elem<T>::kPerVec;
+    RowSplit<T> r;
+    int head = (int)(((16u - (unsigned)(reinterpret_cast<uintptr_t>(row) & 15u)) & 15u) / (unsigned)sizeof(T));
+    if ((int64_t)head > cols) head = (int)cols;
+    r.head = head;
+    r.nvec = (int)((cols - head) / E);
+    r.tail = (int)(cols - head) - r.nvec * E;
+    return r;
+}
+
 // Block-wide sum / max with ONE barrier: every warp publishes its partial in `slots` (>= 32
 // floats of shared memory, a different array for each back-to-back reduction so no second
 // barrier is needed), then every thread folds the published partials in slot order. The

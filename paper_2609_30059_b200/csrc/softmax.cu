@@ -7,8 +7,10 @@
 // a warp each; rows beyond 32 KB (vocabulary-sized) are read twice, the second time backwards out of the
 // L2 (a cluster of up to 8 CTAs holding such a row in registers, with the maximum and the sum combined
 // through distributed shared memory, was measured too: 2.4 - 3.7 TB/s against 3.9 - 4.2 TB/s, the cluster
-// barriers serialise what short-lived CTAs overlap). Rows that cannot be read with 16-byte vectors go to
-// a scalar three-sweep kernel with the same arithmetic.
+// barriers serialise what short-lived CTAs overlap). Rows that are not whole aligned vectors (197 or 77
+// attention keys, a 50257-wide vocabulary) are split into head elements up to the first 16-byte boundary,
+// aligned vectors and tail elements inside the same three kernels; only a causal mask on such rows, or x and
+// y rows at different offsets from a boundary, go to a scalar three-sweep kernel with the same arithmetic.
 #include "kop_common.cuh"
 
 namespace kop {
@@ -29,12 +31,18 @@ struct SmCausal {
     unsigned long long magic;
 };
 
-template <typename T, typename PT, int VPL, bool kFull, bool kBias, int L = 32, bool kLog = false, bool kCausal = false>
+// kRagged: rows that are not whole aligned vectors (`nvec` then carries the row length in elements): a row is split
+// into head elements up to the first 16-byte boundary, whole vectors and tail elements; every lane holds at most one
+// of the edge elements (L >= 16 covers the 14 that 16-bit data can have) next to its vectors, the bias is read per
+// element, the edge results are stored one by one. x and y rows must sit at the same offset from a 16-byte boundary.
+template <typename T, typename PT, int VPL, bool kFull, bool kBias, int L = 32, bool kLog = false, bool kCausal = false,
+          bool kRagged = false>
 __global__ void __launch_bounds__(256)
 softmax_warp_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __restrict__ y,
                     int64_t rows, int nvec, int64_t x_stride, int64_t y_stride, float scale,
                     SmCausal causal = SmCausal{0, 0, 0ull})
 {
+    static_assert(!kRagged || (!kFull && !kCausal && L >= 16), "ragged rows: predicated vectors, no causal mask");
     constexpr int E = Elem<T>::kPerVec;
     const int lane = L == 32 ? (threadIdx.x & 31) : (threadIdx.x & (L - 1));
     int64_t row = ((int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * (32 / L) + (threadIdx.x & 31) / L;
@@ -46,6 +54,15 @@ softmax_warp_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __r
     const float s2 = scale * kLog2e;
     const T* xr = x + row * x_stride;
     T* yr = y + row * y_stride;
+    int head = 0, edge_col = -1;                             // ragged rows: first vector's column, this lane's edge column
+    if constexpr (kRagged) {
+        const RowSplit<T> sp = row_split<T>(xr, nvec);
+        head = sp.head;
+        if (lane < sp.edges()) edge_col = sp.edge_col(lane);
+        nvec = sp.nvec;
+        xr += head;
+        yr += head;
+    }
     int last = 0;
     if (kCausal) {
         // row / period by multiply-shift (exact for row < 2^64 / period; a period of 1 has no 64-bit reciprocal)
@@ -70,7 +87,14 @@ softmax_warp_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __r
 #pragma unroll
         for (int q = 0; q < E / 4; ++q) {
             float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (kBias && (kFull || v < nvec)) b = ldg_p4(bias + (int64_t)v * E + 4 * q);
+            if constexpr (kRagged) {
+                if (bias != nullptr && v < nvec) {
+                    const int j = head + v * E + 4 * q;
+                    b = make_float4(param1(bias, j), param1(bias, j + 1), param1(bias, j + 2), param1(bias, j + 3));
+                }
+            } else {
+                if (kBias && (kFull || v < nvec)) b = ldg_p4(bias + (int64_t)v * E + 4 * q);
+            }
             const float bb[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -80,9 +104,23 @@ softmax_warp_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __r
             }
         }
     }
+    float te = -INFINITY;                                    // this lane's edge element
+    if constexpr (kRagged) {
+        if (edge_col >= 0) {
+            const float b = bias != nullptr ? param1(bias, edge_col) * kLog2e : 0.0f;
+            te = fmaf(Elem<T>::load1(xr - head + edge_col), s2, b);
+        }
+        m = fmaxf(m, te);
+    }
 #pragma unroll
     for (int o = L / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
     float s = 0.0f;
+    if constexpr (kRagged) {
+        const float d = te - m;
+        const float p = ex2_approx(d);
+        s = p;
+        te = kLog ? d : p;
+    }
 #pragma unroll
     for (int k = 0; k < VPL; ++k)
 #pragma unroll
@@ -104,6 +142,9 @@ softmax_warp_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __r
         for (int e = 0; e < E; ++e) o[e] = kLog ? (t[k][e] - lg) * kLn2 : t[k][e] * inv;
         if (live && (kFull || v < nvec)) st_stream(yr + (int64_t)v * E, Elem<T>::pack(o));
     }
+    if constexpr (kRagged) {
+        if (live && edge_col >= 0) Elem<T>::store1(yr - head + edge_col, kLog ? (te - lg) * kLn2 : te * inv);
+    }
 }
 
 // ---- CTA per row, row in registers ---------------------------------------------------------------
@@ -121,11 +162,14 @@ __device__ __forceinline__ int64_t last_visible(const SmOpts& o, int64_t row)
 
 // kPlain: the row is exactly blockDim.x * VPT vectors and there is no bias (no tail predicates, no bias code); the
 // general form tests both at run time.
-template <typename T, typename PT, int VPT, bool kOpts, bool kPlain, bool kLog = false>
+// kRagged: rows that are not whole aligned vectors, split as in the warp kernel (opts.cols carries the row length),
+// one edge element to a thread.
+template <typename T, typename PT, int VPT, bool kOpts, bool kPlain, bool kLog = false, bool kRagged = false>
 __global__ void __launch_bounds__(max_threads_for(VPT * Elem<T>::kPerVec))
 softmax_block_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __restrict__ y,
                      int nvec, int64_t x_stride, int64_t y_stride, float scale, SmOpts opts)
 {
+    static_assert(!kRagged || (!kOpts && !kPlain), "ragged rows: predicated vectors, no causal mask");
     constexpr int E = Elem<T>::kPerVec;
     __shared__ float red_a[32], red_b[32];
     const int64_t row = blockIdx.x;
@@ -133,6 +177,15 @@ softmax_block_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __
     const T* xr = x + row * x_stride;
     T* yr = y + row * y_stride;
     const float s2 = scale * kLog2e;
+    int head = 0, edge_col = -1;
+    if constexpr (kRagged) {
+        const RowSplit<T> sp = row_split<T>(xr, opts.cols);
+        head = sp.head;
+        nvec = sp.nvec;
+        if ((int)threadIdx.x < sp.edges()) edge_col = sp.edge_col(threadIdx.x);
+        xr += head;
+        yr += head;
+    }
 
     Vec16 raw[VPT];
 #pragma unroll
@@ -153,7 +206,14 @@ softmax_block_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __
 #pragma unroll
         for (int q = 0; q < E / 4; ++q) {
             float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (!kPlain && bias != nullptr && v < nvec) b = ldg_p4(bias + (int64_t)v * E + 4 * q);
+            if constexpr (kRagged) {
+                if (bias != nullptr && v < nvec) {
+                    const int j = head + v * E + 4 * q;
+                    b = make_float4(param1(bias, j), param1(bias, j + 1), param1(bias, j + 2), param1(bias, j + 3));
+                }
+            } else {
+                if (!kPlain && bias != nullptr && v < nvec) b = ldg_p4(bias + (int64_t)v * E + 4 * q);
+            }
             const float bb[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -164,9 +224,23 @@ softmax_block_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __
             }
         }
     }
+    float te = -INFINITY;                                    // this thread's edge element
+    if constexpr (kRagged) {
+        if (edge_col >= 0) {
+            const float b = bias != nullptr ? param1(bias, edge_col) * kLog2e : 0.0f;
+            te = fmaf(Elem<T>::load1(xr - head + edge_col), s2, b);
+        }
+        m = fmaxf(m, te);
+    }
     m = block_max(m, red_a);
     float s = 0.0f;
     const bool log_out = kLog || (kOpts && opts.log_out != 0);
+    if constexpr (kRagged) {
+        const float d = te - m;
+        const float p = ex2_approx(d);
+        s = p;
+        te = log_out ? d : p;
+    }
 #pragma unroll
     for (int k = 0; k < VPT; ++k)
 #pragma unroll
@@ -187,17 +261,24 @@ softmax_block_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __
         for (int e = 0; e < E; ++e) o[e] = log_out ? (t[k][e] - lg) * kLn2 : t[k][e] * inv;
         if (kPlain || v < nvec) st_stream(yr + (int64_t)v * E, Elem<T>::pack(o));
     }
+    if constexpr (kRagged) {
+        if (edge_col >= 0) Elem<T>::store1(yr - head + edge_col, log_out ? (te - lg) * kLn2 : te * inv);
+    }
 }
 
 // ---- long rows, vector loads, two sweeps ------------------------------------------------------------
 // Sweep 1 reads the row once and keeps a running (maximum, sum) per thread, rescaled once per batch of U
 // vectors; sweep 2 walks the row backwards (the end of the row is what the first sweep left in L2) and writes
 // the result. HBM sees the row about once each way while the rows in flight fit the L2.
-template <typename T, typename PT, bool kOpts, bool kBias, bool kLog = false>
+// kRagged: rows that are not whole aligned vectors, split as in the warp kernel (opts.cols carries the row length);
+// the edge elements go one to a thread, enter its running (maximum, sum) before the first sweep and are stored after
+// the second.
+template <typename T, typename PT, bool kOpts, bool kBias, bool kLog = false, bool kRagged = false>
 __global__ void __launch_bounds__(512)
 softmax_twosweep_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __restrict__ y, int nvec,
                         int64_t x_stride, int64_t y_stride, float scale, SmOpts opts)
 {
+    static_assert(!kRagged || !kOpts, "ragged rows: no causal mask");
     constexpr int E = Elem<T>::kPerVec, U = 4;
     __shared__ float red_a[32], red_b[32];
     const int64_t row = blockIdx.x;
@@ -206,6 +287,15 @@ softmax_twosweep_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T*
     const T* xr = x + row * x_stride;
     T* yr = y + row * y_stride;
     const float s2 = scale * kLog2e;
+    int head = 0, edge_col = -1;
+    if constexpr (kRagged) {
+        const RowSplit<T> sp = row_split<T>(xr, opts.cols);
+        head = sp.head;
+        nvec = sp.nvec;
+        if ((int)threadIdx.x < sp.edges()) edge_col = sp.edge_col(threadIdx.x);
+        xr += head;
+        yr += head;
+    }
     const int step = U * blockDim.x;
     const int nbatch = (nvec + step - 1) / step;
 
@@ -216,7 +306,14 @@ softmax_twosweep_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T*
 #pragma unroll
         for (int q = 0; q < E / 4; ++q) {
             float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (kBias) b = ldg_p4(bias + (int64_t)v * E + 4 * q);
+            if constexpr (kRagged) {
+                if (kBias) {
+                    const int64_t j = head + (int64_t)v * E + 4 * q;
+                    b = make_float4(param1(bias, j), param1(bias, j + 1), param1(bias, j + 2), param1(bias, j + 3));
+                }
+            } else {
+                if (kBias) b = ldg_p4(bias + (int64_t)v * E + 4 * q);
+            }
             const float bb[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -229,6 +326,17 @@ softmax_twosweep_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T*
 
     const uint64_t keep = l2_policy_keep(), drop = l2_policy_drop();
     float m = -INFINITY, s = 0.0f;
+    float te = -INFINITY;                                    // this thread's edge element
+    if constexpr (kRagged) {
+        if (edge_col >= 0) {
+            const float b = kBias ? param1(bias, edge_col) * kLog2e : 0.0f;
+            te = fmaf(Elem<T>::load1(xr - head + edge_col), s2, b);
+            if (te != -INFINITY) {                           // a NaN enters too and reaches the sum through ex2
+                m = te;
+                s = 1.0f;
+            }
+        }
+    }
     for (int b = 0; b < nbatch; ++b) {
         Vec16 raw[U];
         float t[U][E];
@@ -285,6 +393,12 @@ softmax_twosweep_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T*
                 }
                 st_stream_hint(yr + (int64_t)v * E, Elem<T>::pack(o), drop);
             }
+        }
+    }
+    if constexpr (kRagged) {
+        if (edge_col >= 0) {
+            const float d = te - M;
+            Elem<T>::store1(yr - head + edge_col, log_out ? (d - lg) * kLn2 : ex2_approx(d) * inv);
         }
     }
 }
@@ -455,6 +569,57 @@ kop_status_t launch_softmax(const void* xv, const void* biasv, void* yv, int64_t
         } else if (with_opts) { if (bias != nullptr) KOP_SM_TWO(true, true); else KOP_SM_TWO(true, false); }
         else { if (bias != nullptr) KOP_SM_TWO(false, true); else KOP_SM_TWO(false, false); }
 #undef KOP_SM_TWO
+        return launch_status();
+    }
+    // rows that are not whole aligned vectors, x and y rows at the same offset from a 16-byte boundary, no causal mask:
+    // head elements, aligned vectors, tail elements (attention scores of 197 or 77 keys, a 50257-wide vocabulary)
+    const bool ragged = !vec && (!with_opts || log_only) &&
+                        (reinterpret_cast<uintptr_t>(x) - reinterpret_cast<uintptr_t>(y)) % 16 == 0 &&
+                        ((xs - ys) * (int64_t)sizeof(T)) % 16 == 0 && cols <= 0x7FFFFFFFLL;
+    if (ragged && nvec64 <= 32 * 4) {
+        // 16 lanes a row up to 32 vectors, a warp beyond; one, two or four vectors a lane
+        const int lanes = nvec64 <= 32 ? 16 : 32;
+        const int vp = nvec64 <= 16 ? 1 : (nvec64 <= 64 ? 2 : 4);
+        const int64_t rows_per_cta = 8 * (32 / lanes);
+        const int64_t ctas = (rows + rows_per_cta - 1) / rows_per_cta;
+        if (ctas > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+        const unsigned grid = (unsigned)ctas;
+#define KOP_SM_RAG(V, L)                                                                                               \
+    do {                                                                                                               \
+        if (log_only) softmax_warp_kernel<T, PT, V, false, false, L, true, false, true><<<grid, 256, 0, stream>>>(x, bias, y, rows, (int)cols, xs, ys, scale); \
+        else softmax_warp_kernel<T, PT, V, false, false, L, false, false, true><<<grid, 256, 0, stream>>>(x, bias, y, rows, (int)cols, xs, ys, scale); \
+    } while (0)
+        if (lanes == 16 && vp == 1) KOP_SM_RAG(1, 16);
+        else if (lanes == 16) KOP_SM_RAG(2, 16);
+        else if (vp == 2) KOP_SM_RAG(2, 32);
+        else KOP_SM_RAG(4, 32);
+#undef KOP_SM_RAG
+        return launch_status();
+    }
+    if (ragged && cols <= kMaxRegisterRow && cols * (int64_t)sizeof(T) <= 32768) {
+        const int nvec = (int)nvec64;                        // a row has this many whole vectors, or one fewer
+        int vpt = (cols >= 2048 ? 32 : 16) / E;
+        while (vpt * E < 64 && (nvec + vpt - 1) / vpt > max_threads_for(vpt * E)) vpt *= 2;
+        const int threads = ((nvec + vpt - 1) / vpt + 31) / 32 * 32;
+#define KOP_SM_BLOCK_RAG(V)                                                                                                       \
+    do {                                                                                                                          \
+        if (log_only) softmax_block_kernel<T, PT, V, false, false, true, true><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, 0, xs, ys, scale, opts); \
+        else softmax_block_kernel<T, PT, V, false, false, false, true><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, 0, xs, ys, scale, opts); \
+    } while (0)
+        switch (vpt * E) {
+        case 16: KOP_SM_BLOCK_RAG(16 / E); break;
+        case 32: KOP_SM_BLOCK_RAG(32 / E); break;
+        default: KOP_SM_BLOCK_RAG(64 / E); break;
+        }
+#undef KOP_SM_BLOCK_RAG
+        return launch_status();
+    }
+    if (ragged) {
+        const int threads = cols * (int64_t)sizeof(T) <= 112 * 1024 ? 256 : 512;
+#define KOP_SM_TWO_RAG(B, G) softmax_twosweep_kernel<T, PT, false, B, G, true><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, 0, xs, ys, scale, opts)
+        if (log_only) { if (bias != nullptr) KOP_SM_TWO_RAG(true, true); else KOP_SM_TWO_RAG(false, true); }
+        else { if (bias != nullptr) KOP_SM_TWO_RAG(true, false); else KOP_SM_TWO_RAG(false, false); }
+#undef KOP_SM_TWO_RAG
         return launch_status();
     }
     if (with_opts) softmax_generic_kernel<T, PT, true><<<(unsigned)rows, 256, 0, stream>>>(x, bias, y, cols, xs, ys, scale, opts);

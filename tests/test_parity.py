@@ -47,8 +47,8 @@ SOFTMAX_SHAPES = [
     (3, 128256, BF16),     # a vocabulary size
     (2, 140008, BF16),
     (9, 12288, F32),       # fp32 rows beyond 32 KB: two sweeps although the row would fit the registers
-    (3, 20001, BF16),      # odd length: the scalar three-sweep kernel
-    (37, 513, F32),        # odd length: scalar
+    (3, 20001, BF16),      # odd length: edge elements around two sweeps of aligned vectors
+    (37, 513, F32),        # odd length: edge elements, the row in a warp's registers
     (64, 1, F32),
     (515, 1000, BF16),
     (129, 4096, BF16),
@@ -84,6 +84,66 @@ def test_softmax_no_bias_block_rows(kop, rows, cols, dtype, seed):
     assert torch.equal(out.t, kop.kop_softmax_scale_bias(x, None, 0.5))
 
 
+@pytest.mark.parametrize("rows,cols,dtype", [(2364, 197, BF16), (1000, 77, F32), (900, 49, torch.float16), (333, 257, BF16),
+                                             (100, 577, F32), (40, 1025, BF16), (64, 1001, F32), (7, 50257, BF16),
+                                             (5, 50257, F32), (130, 7, BF16), (50, 3, F32), (21, 2051, torch.float16),
+                                             (3, 70001, F32)])
+@pytest.mark.parametrize("seed", SEEDS[:3])
+def test_softmax_ragged_rows(kop, rows, cols, dtype, seed):
+    """Rows that are not a whole number of aligned 16-byte vectors (attention scores of 197 or 77 keys, a 50257-wide
+    vocabulary): head elements, aligned vectors and tail elements, with the row in a half warp's or a warp's registers
+    up to 128 vectors and in two sweeps beyond; with and without a bias, plain and log form, in place, from a base that
+    is off a boundary, and (x and y at different offsets) through the element-wise kernel."""
+    x, bias = synth.softmax_inputs(rows, cols, dtype, seed, "cuda")
+    tol = tol_of(dtype)
+    for use_bias in (False, True):
+        b = bias if use_bias else None
+        hb = host(b) if use_bias else None
+        ref = kopref.softmax_scale_bias(host(x), hb, 0.25, threads=None)
+        out = Guarded((rows, cols), dtype)
+        kop.kop_softmax_scale_bias(x, b, 0.25, out=out.t)
+        assert_close(out.t, ref, tol, f"ragged softmax bias={use_bias}")
+        out.check("ragged softmax")
+        lref = kopref.softmax_opts(host(x), hb, 0.25, True, 0, threads=None)
+        lout = Guarded((rows, cols), dtype)
+        kop.kop_softmax_opts(x, b, 0.25, True, 0, out=lout.t)
+        assert_close(lout.t, lref, tol, f"ragged log-softmax bias={use_bias}")
+        lout.check("ragged log-softmax")
+    ref = kopref.softmax_scale_bias(host(x), None, 0.25, threads=None)
+    xi = x.clone()
+    kop.kop_softmax_scale_bias(xi, None, 0.25, out=xi)
+    assert_close(xi, ref, tol, "ragged softmax in place")
+    # one element off the allocation's boundary, x and y alike; then y alone (different offsets)
+    n = rows * cols
+    xo = torch.zeros(n + 9, dtype=dtype, device="cuda")
+    yo = torch.full((n + 9,), 3.0, dtype=dtype, device="cuda")
+    xo[1:n + 1] = x.reshape(-1)
+    kop.kop_softmax_scale_bias(xo[1:n + 1].view(rows, cols), None, 0.25, out=yo[1:n + 1].view(rows, cols))
+    assert_close(yo[1:n + 1].view(rows, cols), ref, tol, "ragged softmax off the boundary")
+    assert float(yo[0]) == 3.0 and bool((yo[n + 1:] == 3.0).all())
+    yo.fill_(3.0)
+    kop.kop_softmax_scale_bias(xo[1:n + 1].view(rows, cols), None, 0.25, out=yo[2:n + 2].view(rows, cols))
+    assert_close(yo[2:n + 2].view(rows, cols), ref, tol, "softmax, x and y at different offsets")
+    assert bool((yo[:2] == 3.0).all()) and bool((yo[n + 2:] == 3.0).all())
+    # masked first and last column (-inf bias): exact zeros there; a NaN in an edge element poisons its row only
+    b2 = bias.clone()
+    b2[0] = float("-inf")
+    b2[cols - 1] = float("-inf")
+    if cols > 2:
+        y = kop.kop_softmax_scale_bias(x, b2, 0.25)
+        assert_close(y, kopref.softmax_scale_bias(host(x), host(b2), 0.25, threads=None), tol, "ragged softmax masked")
+        assert bool((y[:, 0] == 0).all()) and bool((y[:, cols - 1] == 0).all())
+    xn = x.clone()
+    xn[rows // 2, 0] = float("nan")
+    xn[rows - 1, cols - 1] = float("nan")
+    y = kop.kop_softmax_scale_bias(xn, None, 0.25)
+    bad = torch.isnan(y).any(dim=1)
+    want = torch.zeros(rows, dtype=torch.bool, device="cuda")
+    want[rows // 2] = True
+    want[rows - 1] = True
+    assert torch.equal(bad, want) and bool(torch.isnan(y[rows // 2]).all()) and bool(torch.isnan(y[rows - 1]).all())
+
+
 def test_softmax_large_config_seed0(kop):
     c = synth.CONFIGS["softmax_large"]
     x, bias = synth.softmax_inputs(c["rows"], c["cols"], c["dtype"], 0, "cuda")
@@ -116,7 +176,7 @@ def test_softmax_options(kop):
     assert_close(ow[:, 64:576], ref, 1e-5, "strided")
     assert bool((ow[:, :64] == 7.0).all()) and bool((ow[:, 576:] == 7.0).all())
     wide[:, 257:769] = x
-    y = kop.kop_softmax_scale_bias(wide[:, 257:769], bias, 0.125)         # misaligned base: scalar path
+    y = kop.kop_softmax_scale_bias(wide[:, 257:769], bias, 0.125)         # misaligned base, y aligned: element-wise kernel
     assert_close(y, ref, 1e-5, "misaligned")
     # empty
     e = torch.empty((0, 512), dtype=F32, device="cuda")
