@@ -206,6 +206,82 @@ chain_scalar_kernel(const T* __restrict__ x, const PT* __restrict__ bias, const 
     }
 }
 
+// ---- contiguous tensors whose rows are not whole aligned vectors ------------------------------------------
+// The tensor as one span: head elements up to the first 16-byte boundary, aligned vectors that run across the row
+// boundaries, tail elements. A vector's first column comes from its flat index by a multiply-shift remainder
+// (magic = ceil(2^64 / cols), exact below 2^64 / cols); the following columns wrap at most once (cols >= the vector
+// length); the bias is read per element. x, y and the residual sit at the same offset from a boundary.
+template <typename T, typename PT, int ACT, bool kChain>
+__global__ void __launch_bounds__(256)
+span_kernel(const T* __restrict__ x, const PT* __restrict__ bias, const T* __restrict__ res, T* __restrict__ y,
+            int64_t total, int cols, unsigned long long magic, ChainArgs a)
+{
+    constexpr int E = Elem<T>::kPerVec, U = kChain ? 2 : 4;
+    constexpr bool kFast = sizeof(T) == 2;
+    int64_t head = (int64_t)(((16u - (unsigned)(reinterpret_cast<uintptr_t>(x) & 15u)) & 15u) / (unsigned)sizeof(T));
+    if (head > total) head = total;
+    const int64_t nv = (total - head) / E;
+    const int tail = (int)(total - head - nv * E);
+    auto value = [&](float xv, float rv, int c) {
+        const float b = bias != nullptr ? param1(bias, c) : 0.0f;
+        if constexpr (kChain) return act_dev<ACT, kFast>(chain_value(xv, b, rv, a), a.alpha);
+        else return act_dev<ACT, kFast>(xv + b, a.alpha);
+    };
+    if (blockIdx.x == 0 && (int)threadIdx.x < (int)head + tail) {
+        const int64_t j = (int64_t)threadIdx.x < head ? (int64_t)threadIdx.x : head + nv * E + ((int64_t)threadIdx.x - head);
+        const float rv = kChain && res != nullptr ? Elem<T>::load1(res + j) : 0.0f;
+        Elem<T>::store1(y + j, value(Elem<T>::load1(x + j), rv, (int)(j % cols)));
+    }
+    const T* xm = x + head;
+    const T* rm = res != nullptr ? res + head : nullptr;
+    T* ym = y + head;
+    const int64_t g0 = (int64_t)blockIdx.x * (U * blockDim.x) + threadIdx.x;
+    Vec16 rx[U], rres[U];
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+        const int64_t g = g0 + k * blockDim.x;
+        if (g < nv) {
+            rx[k] = ld_stream(xm + g * E);
+            if (kChain && res != nullptr) rres[k] = ld_stream(rm + g * E);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+        const int64_t g = g0 + k * blockDim.x;
+        if (g < nv) {
+            const unsigned long long i0 = (unsigned long long)(head + g * E);
+            int c = (int)(i0 - __umul64hi(i0, magic) * (unsigned)cols);
+            float f[E], r[E];
+            Elem<T>::unpack(rx[k], f);
+            if (kChain && res != nullptr) Elem<T>::unpack(rres[k], r);
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                f[e] = value(f[e], kChain && res != nullptr ? r[e] : 0.0f, c);
+                c = c + 1 == cols ? 0 : c + 1;
+            }
+            st_stream(ym + g * E, Elem<T>::pack(f));
+        }
+    }
+}
+
+// Launches span_kernel when the tensors qualify; false when they do not.
+template <typename T, typename PT, int ACT, bool kChain>
+bool launch_span(const T* x, const PT* bias, const T* res, T* y, int64_t rows, int64_t cols, int64_t xs, int64_t rs,
+                 int64_t ys, const ChainArgs& a, cudaStream_t stream)
+{
+    constexpr int E = Elem<T>::kPerVec, U = kChain ? 2 : 4;
+    if (xs != cols || ys != cols || (res != nullptr && rs != cols) || cols < E || cols > 0x7FFFFFFFLL) return false;
+    const uintptr_t off = reinterpret_cast<uintptr_t>(x) & 15u;
+    if ((reinterpret_cast<uintptr_t>(y) & 15u) != off || (res != nullptr && (reinterpret_cast<uintptr_t>(res) & 15u) != off))
+        return false;
+    const int64_t total = rows * cols;
+    const int64_t grid = (total / E + U * 256 - 1) / (U * 256) + 1;
+    if (grid > 0x7FFFFFFFLL) return false;
+    const unsigned long long magic = (~0ull) / (unsigned long long)cols + 1ull;
+    span_kernel<T, PT, ACT, kChain><<<(unsigned)grid, 256, 0, stream>>>(x, bias, res, y, total, (int)cols, magic, a);
+    return true;
+}
+
 template <typename T, typename PT, int ACT>
 kop_status_t launch_chain_a(const T* x, const PT* bias, const T* res, T* y, int64_t rows, int64_t cols, int64_t xs,
                             int64_t rs, int64_t ys, const ChainArgs& a, cudaStream_t stream)
@@ -231,6 +307,7 @@ kop_status_t launch_chain_a(const T* x, const PT* bias, const T* res, T* y, int6
         chain_kernel<T, PT, ACT, false><<<(unsigned)grid, threads, 0, stream>>>(x, bias, res, y, nvec, tiles, 0, xs, rs, ys, a);
         return launch_status();
     }
+    if (launch_span<T, PT, ACT, true>(x, bias, res, y, rows, cols, xs, rs, ys, a, stream)) return launch_status();
     int64_t blocks = (rows * cols + 255) / 256;
     const int64_t cap = 32LL * sm_count();
     if (blocks > cap) blocks = cap;
@@ -295,6 +372,9 @@ kop_status_t launch_bias_act_a(const T* x, const PT* bias, T* y, int64_t rows, i
         bias_act_kernel<T, PT, ACT, false><<<(unsigned)grid, threads, 0, stream>>>(x, bias, y, nvec, tiles, 0, xs, ys, alpha);
         return launch_status();
     }
+    if (launch_span<T, PT, ACT, false>(x, bias, static_cast<const T*>(nullptr), y, rows, cols, xs, 0, ys,
+                                       ChainArgs{1.0f, 0.0f, 0.0f, 0.0f, alpha}, stream))
+        return launch_status();
     int64_t blocks = (rows * cols + 255) / 256;
     const int64_t cap = 32LL * sm_count();
     if (blocks > cap) blocks = cap;

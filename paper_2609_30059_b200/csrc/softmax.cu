@@ -42,7 +42,8 @@ softmax_warp_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __r
                     int64_t rows, int nvec, int64_t x_stride, int64_t y_stride, float scale,
                     SmCausal causal = SmCausal{0, 0, 0ull})
 {
-    static_assert(!kRagged || (!kFull && !kCausal && L >= 16), "ragged rows: predicated vectors, no causal mask");
+    static_assert(!kRagged || (!kFull && !kCausal && L >= 8), "ragged rows: predicated vectors, no causal mask");
+    constexpr int KE = kRagged ? (2 * (Elem<T>::kPerVec - 1) + L - 1) / L : 1;      // edge elements a lane holds at most
     constexpr int E = Elem<T>::kPerVec;
     const int lane = L == 32 ? (threadIdx.x & 31) : (threadIdx.x & (L - 1));
     int64_t row = ((int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * (32 / L) + (threadIdx.x & 31) / L;
@@ -54,11 +55,15 @@ softmax_warp_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __r
     const float s2 = scale * kLog2e;
     const T* xr = x + row * x_stride;
     T* yr = y + row * y_stride;
-    int head = 0, edge_col = -1;                             // ragged rows: first vector's column, this lane's edge column
+    int head = 0, edge_col[KE];                              // ragged rows: first vector's column, this lane's edge columns
+#pragma unroll
+    for (int q = 0; q < KE; ++q) edge_col[q] = -1;
     if constexpr (kRagged) {
         const RowSplit<T> sp = row_split<T>(xr, nvec);
         head = sp.head;
-        if (lane < sp.edges()) edge_col = sp.edge_col(lane);
+#pragma unroll
+        for (int q = 0; q < KE; ++q)
+            if (lane + q * L < sp.edges()) edge_col[q] = sp.edge_col(lane + q * L);
         nvec = sp.nvec;
         xr += head;
         yr += head;
@@ -104,22 +109,30 @@ softmax_warp_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __r
             }
         }
     }
-    float te = -INFINITY;                                    // this lane's edge element
+    float te[KE];                                            // this lane's edge elements
+#pragma unroll
+    for (int q = 0; q < KE; ++q) te[q] = -INFINITY;
     if constexpr (kRagged) {
-        if (edge_col >= 0) {
-            const float b = bias != nullptr ? param1(bias, edge_col) * kLog2e : 0.0f;
-            te = fmaf(Elem<T>::load1(xr - head + edge_col), s2, b);
+#pragma unroll
+        for (int q = 0; q < KE; ++q) {
+            if (edge_col[q] >= 0) {
+                const float b = bias != nullptr ? param1(bias, edge_col[q]) * kLog2e : 0.0f;
+                te[q] = fmaf(Elem<T>::load1(xr - head + edge_col[q]), s2, b);
+            }
+            m = fmaxf(m, te[q]);
         }
-        m = fmaxf(m, te);
     }
 #pragma unroll
     for (int o = L / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
     float s = 0.0f;
     if constexpr (kRagged) {
-        const float d = te - m;
-        const float p = ex2_approx(d);
-        s = p;
-        te = kLog ? d : p;
+#pragma unroll
+        for (int q = 0; q < KE; ++q) {
+            const float d = te[q] - m;
+            const float p = ex2_approx(d);
+            s += p;
+            te[q] = kLog ? d : p;
+        }
     }
 #pragma unroll
     for (int k = 0; k < VPL; ++k)
@@ -143,7 +156,9 @@ softmax_warp_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __r
         if (live && (kFull || v < nvec)) st_stream(yr + (int64_t)v * E, Elem<T>::pack(o));
     }
     if constexpr (kRagged) {
-        if (live && edge_col >= 0) Elem<T>::store1(yr - head + edge_col, kLog ? (te - lg) * kLn2 : te * inv);
+#pragma unroll
+        for (int q = 0; q < KE; ++q)
+            if (live && edge_col[q] >= 0) Elem<T>::store1(yr - head + edge_col[q], kLog ? (te[q] - lg) * kLn2 : te[q] * inv);
     }
 }
 
@@ -577,9 +592,10 @@ kop_status_t launch_softmax(const void* xv, const void* biasv, void* yv, int64_t
                         (reinterpret_cast<uintptr_t>(x) - reinterpret_cast<uintptr_t>(y)) % 16 == 0 &&
                         ((xs - ys) * (int64_t)sizeof(T)) % 16 == 0 && cols <= 0x7FFFFFFFLL;
     if (ragged && nvec64 <= 32 * 4) {
-        // 16 lanes a row up to 32 vectors, a warp beyond; one, two or four vectors a lane
-        const int lanes = nvec64 <= 32 ? 16 : 32;
-        const int vp = nvec64 <= 16 ? 1 : (nvec64 <= 64 ? 2 : 4);
+        // 8 lanes a row up to 32 vectors, a warp beyond; two or four vectors a lane (fp32 rows of 197 columns: 54 us a
+        // warp a row, 58 with 16 lanes; bf16 rows of 77: 29 us with 8 lanes, 33 with 16)
+        const int lanes = nvec64 <= 32 ? 8 : 32;
+        const int vp = (nvec64 <= 16 || (nvec64 > 32 && nvec64 <= 64)) ? 2 : 4;
         const int64_t rows_per_cta = 8 * (32 / lanes);
         const int64_t ctas = (rows + rows_per_cta - 1) / rows_per_cta;
         if (ctas > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
@@ -589,8 +605,8 @@ kop_status_t launch_softmax(const void* xv, const void* biasv, void* yv, int64_t
         if (log_only) softmax_warp_kernel<T, PT, V, false, false, L, true, false, true><<<grid, 256, 0, stream>>>(x, bias, y, rows, (int)cols, xs, ys, scale); \
         else softmax_warp_kernel<T, PT, V, false, false, L, false, false, true><<<grid, 256, 0, stream>>>(x, bias, y, rows, (int)cols, xs, ys, scale); \
     } while (0)
-        if (lanes == 16 && vp == 1) KOP_SM_RAG(1, 16);
-        else if (lanes == 16) KOP_SM_RAG(2, 16);
+        if (lanes == 8 && vp == 2) KOP_SM_RAG(2, 8);
+        else if (lanes == 8) KOP_SM_RAG(4, 8);
         else if (vp == 2) KOP_SM_RAG(2, 32);
         else KOP_SM_RAG(4, 32);
 #undef KOP_SM_RAG

@@ -28,7 +28,8 @@ def host(t):
 
 
 @pytest.mark.parametrize("rows,cols,dtype", [(512, 4096, BF16), (300, 4096, F32), (65, 1000, F16), (33, 1001, F32),
-                                             (9, 20480, BF16), (7, 1, F32)])
+                                             (9, 20480, BF16), (7, 1, F32), (700, 197, BF16), (41, 5003, BF16),
+                                             (300, 9, F16), (50, 3, F32)])
 @pytest.mark.parametrize("seed", SEEDS)
 def test_bias_act_parity(kop, rows, cols, dtype, seed):
     x, bias = synth.softmax_inputs(rows, cols, dtype, seed, "cuda")
@@ -61,9 +62,30 @@ def test_bias_act_options(kop):
         kop.kop_bias_act(big[:, :cols], bias, act, alpha=1.0, out=outb[:, :cols])
         assert_close(outb[:, :cols], ref, 1e-5, act + " strided")
         assert bool((outb[:, cols:] == 5.0).all())
-        flat = torch.zeros(rows * cols + 1, dtype=F32, device="cuda")             # misaligned base: scalar kernel
+        flat = torch.zeros(rows * cols + 1, dtype=F32, device="cuda")             # misaligned base, y aligned: element-wise kernel
         flat[1:] = x.reshape(-1)
         assert_close(kop.kop_bias_act(flat[1:].view(rows, cols), bias, act, alpha=1.0), ref, 1e-5, act + " misaligned")
+    # rows that are not whole vectors, x and y one element off a 16-byte boundary alike (the span kernel's head and tail
+    # elements) and at different offsets (element-wise kernel); nothing written outside y
+    for dt, (r2, c2) in ((BF16, (300, 197)), (F32, (64, 1001)), (F16, (5, 7))):
+        xs_, bs_ = synth.softmax_inputs(r2, c2, dt, 3, "cuda")
+        n = r2 * c2
+        ref = kopref.bias_act(host(xs_), host(bs_), "silu", threads=None)
+        xo = torch.zeros(n + 16, dtype=dt, device="cuda")
+        xo[1:n + 1] = xs_.reshape(-1)
+        for yoff in (1, 2):
+            yo = torch.full((n + 16,), 9.0, dtype=dt, device="cuda")
+            kop.kop_bias_act(xo[1:n + 1].view(r2, c2), bs_, "silu", out=yo[yoff:n + yoff].view(r2, c2))
+            assert_close(yo[yoff:n + yoff].view(r2, c2), ref, tol_of(dt), f"bias_act off the boundary, y offset {yoff}")
+            assert bool((yo[:yoff] == 9.0).all()) and bool((yo[n + yoff:] == 9.0).all())
+        ro = torch.zeros(n + 16, dtype=dt, device="cuda")
+        ro[1:n + 1] = (xs_ * 0.5).reshape(-1)
+        yo = torch.full((n + 16,), 9.0, dtype=dt, device="cuda")
+        kop.kop_epilogue_chain(xo[1:n + 1].view(r2, c2), bs_, ro[1:n + 1].view(r2, c2), 0.7, 1.5, -1.0, 2.0, "gelu_tanh",
+                               out=yo[1:n + 1].view(r2, c2))
+        cref = kopref.epilogue_chain(host(xs_), host(bs_), host(xs_ * 0.5), 0.7, 1.5, -1.0, 2.0, "gelu_tanh", threads=None)
+        assert_close(yo[1:n + 1].view(r2, c2), cref, tol_of(dt), "chain off the boundary")
+        assert float(yo[0]) == 9.0 and bool((yo[n + 1:] == 9.0).all())
     # special values
     sp = torch.tensor([[float("nan"), float("inf"), float("-inf"), 0.0, -0.0, 100.0, -100.0, 1e-30]], device="cuda")
     for act in ACTS:
@@ -79,7 +101,8 @@ def test_bias_act_options(kop):
     assert kop.lib().kop_bias_act(x.data_ptr(), None, x.data_ptr(), 4, 16, 16, 16, 11, 0.0, 0, None) == 2
 
 
-@pytest.mark.parametrize("rows,cols,dtype", [(256, 4096, BF16), (300, 4096, F32), (65, 1000, F16), (33, 1001, F32), (7, 1, BF16)])
+@pytest.mark.parametrize("rows,cols,dtype", [(256, 4096, BF16), (300, 4096, F32), (65, 1000, F16), (33, 1001, F32), (7, 1, BF16),
+                                             (700, 197, BF16), (21, 5003, F32), (300, 9, F16)])
 @pytest.mark.parametrize("seed", SEEDS)
 def test_epilogue_chain_parity(kop, rows, cols, dtype, seed):
     """The general chain y = act(clamp((x + bias) * scale + residual * residual_scale, lo, hi))."""
