@@ -298,31 +298,48 @@ __device__ __forceinline__ void sweep_vectors(Acc<OP>& acc, const T* xr, int nve
     if (OP == kOpMax || OP == kOpMin) acc.template resolve<T>();
 }
 
-// One CTA per row; vector path (rows are whole 16-byte vectors and aligned) or scalar path.
-template <typename T, int OP, bool kVec>
+// A row of any length and alignment by `nthreads` threads: the aligned 16-byte vectors between the first boundary
+// and the last (positions counted from the row's start), then the at most 2 (E - 1) edge elements before and after
+// them, one to a thread at a time, merged in as a partial result of their own.
+template <typename T, int OP, int U>
+__device__ __forceinline__ void sweep_row(Acc<OP>& acc, const T* xr, int cols, int tid, int nthreads)
+{
+    const RowSplit<T> sp = row_split<T>(xr, cols);
+    sweep_vectors<T, OP, U>(acc, xr + sp.head, sp.nvec, tid, nthreads);
+    if (OP == kOpMax || OP == kOpMin) {
+        if (acc.idx != INT_MAX) acc.idx += sp.head;
+        if (acc.nan_idx != INT_MAX) acc.nan_idx += sp.head;
+    }
+    if (tid < sp.edges()) {
+        Acc<OP> edge;
+        edge.init();
+        for (int i = tid; i < sp.edges(); i += nthreads) {
+            const int j = sp.edge_col(i);
+            const float v = Elem<T>::load1(xr + j);
+            if constexpr (OP == kOpLse) {
+                const float one[1] = {v};
+                edge.template add_batch_lse<1>(one, 1);
+            } else {
+                edge.add(v, j);
+            }
+        }
+        acc.merge(edge);
+    }
+}
+
+// One CTA per row.
+template <typename T, int OP>
 __global__ void __launch_bounds__(256)
 reduce_row_block_kernel(const T* __restrict__ x, float* __restrict__ out, int32_t* __restrict__ index, int cols,
                         int64_t stride, float inv_cols)
 {
-    constexpr int E = Elem<T>::kPerVec, U = 4;
+    constexpr int U = 4;
     __shared__ float sa[8], ss[8];
     __shared__ int si[8], sn[8];
     const T* xr = x + (int64_t)blockIdx.x * stride;
     Acc<OP> acc;
     acc.init();
-    if (kVec) {
-        sweep_vectors<T, OP, U>(acc, xr, cols / E, threadIdx.x, blockDim.x);
-    } else {
-        for (int j = threadIdx.x; j < cols; j += blockDim.x) {
-            const float v = Elem<T>::load1(xr + j);
-            if (OP == kOpLse) {
-                const float one[1] = {v};
-                acc.template add_batch_lse<1>(one, 1);
-            } else {
-                acc.add(v, j);
-            }
-        }
-    }
+    sweep_row<T, OP, U>(acc, xr, cols, threadIdx.x, blockDim.x);
     acc = warp_merge<OP>(acc);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
     if (lane == 0) {
@@ -349,12 +366,11 @@ reduce_row_block_kernel(const T* __restrict__ x, float* __restrict__ out, int32_
 // L lanes per row (L = 4 .. 32, a power of two), 32 / L rows per warp, eight warps per CTA: a short row does
 // not pay for a full warp's five butterfly steps, and a lane still has up to four loads in flight. Lanes
 // whose row is past the end sweep nothing but take part in the shuffles.
-template <typename T, int OP, bool kVec, int L>
+template <typename T, int OP, int L>
 __global__ void __launch_bounds__(256)
 reduce_row_group_kernel(const T* __restrict__ x, float* __restrict__ out, int32_t* __restrict__ index, int64_t rows,
                         int cols, int64_t stride, float inv_cols)
 {
-    constexpr int E = Elem<T>::kPerVec;
     constexpr int kRowsPerWarp = 32 / L;
     const int lane = threadIdx.x & 31, sub = lane & (L - 1);
     const int64_t row = ((int64_t)blockIdx.x * 8 + (threadIdx.x >> 5)) * kRowsPerWarp + lane / L;
@@ -363,19 +379,7 @@ reduce_row_group_kernel(const T* __restrict__ x, float* __restrict__ out, int32_
     const int n = live ? cols : 0;
     Acc<OP> acc;
     acc.init();
-    if (kVec) {
-        sweep_vectors<T, OP, 4>(acc, xr, n / E, sub, L);
-    } else {
-        for (int j = sub; j < n; j += L) {
-            const float v = Elem<T>::load1(xr + j);
-            if (OP == kOpLse) {
-                const float one[1] = {v};
-                acc.template add_batch_lse<1>(one, 1);
-            } else {
-                acc.add(v, j);
-            }
-        }
-    }
+    sweep_row<T, OP, 4>(acc, xr, n, sub, L);
     acc = warp_merge<OP, L>(acc);
     if (sub == 0 && live) write_result<T, OP>(acc, out, index, row, inv_cols);
 }
@@ -385,35 +389,25 @@ kop_status_t launch_reduce_op(const T* x, float* out, int32_t* index, int64_t ro
                               cudaStream_t stream)
 {
     constexpr int E = Elem<T>::kPerVec;
-    const bool vec = vec_ok(x, cols, stride, sizeof(T));
     const float inv_cols = (float)(1.0 / (double)cols);
     const int64_t row_bytes = (int64_t)cols * sizeof(T);
     // Rows up to 16 KB: lanes-per-row kernel, measured against a CTA per row on 537 MB of bf16, max + argmax:
     // rows of 256 / 1024 / 2048 / 8192 columns 346 -> 88, 267 -> 91, 150 -> 90, 94 -> 90 us. Longer rows: a CTA each.
     if (row_bytes > 16384) {
-        int threads = 256;
-        if (vec) {
-            const int nvec = cols / E;
-            threads = ((nvec + 15) / 16 + 31) / 32 * 32;     // four batches of four vectors per thread if they fit
-            if (threads > 256) threads = 256;
-            if (threads < 64) threads = 64;
-        }
-        if (vec)
-            reduce_row_block_kernel<T, OP, true><<<(unsigned)rows, threads, 0, stream>>>(x, out, index, cols, stride, inv_cols);
-        else
-            reduce_row_block_kernel<T, OP, false><<<(unsigned)rows, threads, 0, stream>>>(x, out, index, cols, stride, inv_cols);
+        const int nvec = cols / E;
+        int threads = ((nvec + 15) / 16 + 31) / 32 * 32;     // four batches of four vectors per thread if they fit
+        if (threads > 256) threads = 256;
+        if (threads < 64) threads = 64;
+        reduce_row_block_kernel<T, OP><<<(unsigned)rows, threads, 0, stream>>>(x, out, index, cols, stride, inv_cols);
     } else {
-        // sixteen vectors (or 64 scalar elements) a lane where the row is long enough: fewer lanes and merge
-        // steps beat more lanes with fewer batches each (four vectors a lane: 102 - 113 us on the rows above)
-        const int64_t units = vec ? cols / E : (cols + 3) / 4;
+        // sixteen vectors a lane where the row is long enough: fewer lanes and merge steps beat more lanes with
+        // fewer batches each (four vectors a lane: 102 - 113 us on the rows above)
+        const int64_t units = cols / E;
         const int lanes = units >= 512 ? 32 : units >= 256 ? 16 : units >= 128 ? 8 : 4;
         const int64_t rows_per_cta = 8 * (32 / lanes);
         const int64_t ctas = (rows + rows_per_cta - 1) / rows_per_cta;
-#define KOP_REDUCE_GROUP(L)                                                                                              \
-    do {                                                                                                                 \
-        if (vec) reduce_row_group_kernel<T, OP, true, L><<<(unsigned)ctas, 256, 0, stream>>>(x, out, index, rows, cols, stride, inv_cols); \
-        else reduce_row_group_kernel<T, OP, false, L><<<(unsigned)ctas, 256, 0, stream>>>(x, out, index, rows, cols, stride, inv_cols);    \
-    } while (0)
+#define KOP_REDUCE_GROUP(L) \
+    reduce_row_group_kernel<T, OP, L><<<(unsigned)ctas, 256, 0, stream>>>(x, out, index, rows, cols, stride, inv_cols)
         switch (lanes) {
         case 32: KOP_REDUCE_GROUP(32); break;
         case 16: KOP_REDUCE_GROUP(16); break;

@@ -59,7 +59,11 @@ def check_op(kop, x, xh, op, what):
 SHAPES = [(512, 8192, BF16), (300, 4096, F32), (65, 1000, F16), (33, 1001, F32), (9, 40000, BF16),
           (2000, 64, F32), (1000, 7, BF16), (257, 520, F16), (5, 1, F32),
           # 8, 16 and 32 lanes per row, row counts that leave part of the last warp without a row
-          (67, 1024, BF16), (129, 2048, BF16), (35, 3072, F16), (131, 4096, BF16), (21, 600, F32)]
+          (67, 1024, BF16), (129, 2048, BF16), (35, 3072, F16), (131, 4096, BF16), (21, 600, F32),
+          # rows that are not whole aligned vectors: edge elements before and after the aligned vectors, every lane count
+          # and the CTA-per-row kernel
+          (700, 197, BF16), (300, 77, F32), (41, 4097, BF16), (130, 2051, F16), (9, 50257, BF16), (7, 50257, F32),
+          (50, 3, F16), (33, 8193, F32)]
 
 
 @pytest.mark.parametrize("rows,cols,dtype", SHAPES)
@@ -109,7 +113,23 @@ def test_reduce_ties_specials_and_layouts(kop):
     v, i = kop.kop_reduce_rows(xi, "max")
     assert float(v[2]) == float("-inf") and int(i[2]) == 0 and float(v[3]) == float("inf") and int(i[3]) == 100
     assert float(kop.kop_reduce_rows(xi, "logsumexp")[0][2]) == float("-inf")
-    # strided rows and a misaligned base (scalar kernels)
+    # ties and NaNs that sit in the edge elements of rows that are not whole vectors: first position, whichever part holds it
+    for rows, cols, dt in ((37, 197, BF16), (9, 20011, BF16), (21, 1001, F32)):
+        xt = torch.randint(-2, 3, (rows, cols), device="cuda").to(dt)
+        check_op(kop, xt, host(xt), "max", "edge ties")
+        check_op(kop, xt, host(xt), "min", "edge ties")
+        xe = xt.clone()
+        xe[1, cols - 1] = float("nan")
+        xe[2, 0] = float("nan")
+        xe[2, cols // 2] = float("nan")
+        xe[3, cols - 1] = 7.0                              # the maximum in the last element
+        xe[4, 0] = -7.0                                    # the minimum in the first
+        for op in OPS:
+            v, i = check_op(kop, xe, host(xe), op, "edge specials")
+            if op in ("max", "min"):
+                assert int(i[1]) == cols - 1 and int(i[2]) == 0
+        assert int(kop.kop_reduce_rows(xe, "max")[1][3]) == cols - 1 and int(kop.kop_reduce_rows(xe, "min")[1][4]) == 0
+    # strided rows and a misaligned base (edge elements around the aligned vectors)
     big = torch.zeros((40, 2048 + 24), dtype=F32, device="cuda")
     big[:, :2048] = x
     for op in OPS:
