@@ -125,6 +125,11 @@ def segment_bytes():
     out["softmax_vocab"] = dict(bytes=2 * q["rows"] * q["cols"] * 2, elems=q["rows"] * q["cols"])
     q = c["softmax_4096"]
     out["softmax_4096"] = dict(bytes=2 * q["rows"] * q["cols"] * 2, elems=q["rows"] * q["cols"])
+    q = c["softmax_197"]
+    out["softmax_197"] = dict(bytes=2 * q["rows"] * q["cols"] * 2, elems=q["rows"] * q["cols"])
+    q = c["groupnorm_14"]
+    e = q["N"] * q["C"] * q["H"] * q["W"]
+    out["groupnorm_14"] = dict(bytes=2 * e * 2 + 2 * q["C"] * 4 + 2 * q["N"] * q["groups"] * 4, elems=e)
     t = c["gru_cell"]
     out["gru_cell"] = dict(bytes=(2 * 3 + 2) * t["rows"] * t["hidden"] * 2 + 6 * t["hidden"] * 4, elems=t["rows"] * t["hidden"])
     u = c["cumsum"]
@@ -272,7 +277,7 @@ class Workload:
 
     ORDER = ["softmax_small", "softmax_large", "layernorm", "bn_pool", "ce_loss", "rmsnorm", "silu_mul", "residual_add"]
     # Beyond the benchmark configs (not part of `value`): the two kernels the paper's case studies print.
-    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "layernorm_plain", "layernorm_params16", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc", "pool2d", "pool2d_s1", "pool2d_14", "reduce_max", "reduce_logsumexp", "bias_gelu", "residual_rmsnorm", "l2_normalize", "lstm_cell", "gru_cell", "rmsnorm_head128", "softmax_vocab", "softmax_4096"]
+    EXTRA = ["row_scale", "matvec_bias", "residual_layernorm", "layernorm_plain", "layernorm_params16", "silu_mul_interleaved", "ce_loss_opts", "groupnorm", "cumsum", "bn_pool_nhwc", "pool2d", "pool2d_s1", "pool2d_14", "reduce_max", "reduce_logsumexp", "bias_gelu", "residual_rmsnorm", "l2_normalize", "lstm_cell", "gru_cell", "rmsnorm_head128", "softmax_vocab", "softmax_4096", "softmax_197", "groupnorm_14"]
 
     def __init__(self, kop, device, seed, only=None, rows_div=1):
         """only: build just these segments (None = all, plus the MLP segment); rows_div cuts the row
@@ -381,6 +386,16 @@ class Workload:
             q = c["softmax_4096"]
             self.vx3, _ = synth.softmax_inputs(cut(q["rows"]), q["cols"], q["dtype"], seed, dev)
             self.vy3 = torch.empty_like(self.vx3)
+        if "softmax_197" in want:
+            q = c["softmax_197"]
+            self.vx4, _ = synth.softmax_inputs(cut(q["rows"]), q["cols"], q["dtype"], seed, dev)
+            self.vy4 = torch.empty_like(self.vx4)
+        if "groupnorm_14" in want:
+            q = c["groupnorm_14"]
+            self.q14x, self.q14g, self.q14b = synth.groupnorm_inputs(cut(q["N"]), q["C"], q["H"], q["W"], q["dtype"], seed, dev)
+            self.q14y = torch.empty_like(self.q14x)
+            self.q14mean = torch.empty((self.q14x.shape[0], q["groups"]), dtype=torch.float32, device=dev)
+            self.q14rstd = torch.empty_like(self.q14mean)
         if "cumsum" in want:
             u = c["cumsum"]
             self.ux, _ = synth.cumsum_inputs(cut(u["rows"]), u["cols"], u["dtype"], seed, dev)
@@ -487,6 +502,12 @@ class Workload:
             k.kop_softmax_scale_bias(self.vx2, None, 1.0, out=self.vy2)
         elif name == "softmax_4096":             # rows of 4096 bf16 columns: one CTA per row, 32 values a thread in registers
             k.kop_softmax_scale_bias(self.vx3, None, 1.0, out=self.vy3)
+        elif name == "softmax_197":              # 197 keys a row, bf16: edge elements around the aligned vectors, 8 lanes a row
+            k.kop_softmax_scale_bias(self.vx4, None, 1.0, out=self.vy4)
+        elif name == "groupnorm_14":             # GroupNorm(32) + SiLU over bf16 [512, 512, 14, 14]: chunks in registers
+            q = c["groupnorm_14"]
+            k.kop_groupnorm_act(self.q14x, self.q14g, self.q14b, q["groups"], q["eps"], q["act"], out=self.q14y,
+                                mean=self.q14mean, rstd=self.q14rstd)
         elif name == "gru_cell":                 # gate sums, activations and state update, bf16 [16384, 3 x 1024]
             k.kop_gru_cell(self.ui, self.uh, self.up, self.ubi, self.ubh, h_out=self.uo)
         elif name == "cumsum":                   # inclusive running sum along rows, fp32 [32768, 4096]

@@ -43,6 +43,11 @@ CONFIGS = {
     "rmsnorm_head128": dict(rows=1048576, hidden=128, eps=1e-6, dtype=torch.bfloat16),
     "softmax_vocab": dict(rows=2048, cols=128256, scale=1.0, dtype=torch.bfloat16),
     "softmax_4096": dict(rows=32768, cols=4096, scale=1.0, dtype=torch.bfloat16),        # rows in one CTA's registers
+    # attention scores of a ViT with a class token (12 heads x 197 queries x 128 images, 197 keys): rows that are not
+    # whole 16-byte vectors
+    "softmax_197": dict(rows=12 * 197 * 128, cols=197, scale=1.0, dtype=torch.bfloat16),
+    # GroupNorm(32) + SiLU on a late-stage feature map: 16 channels of 14 x 14 bf16 a group, chunks held in registers
+    "groupnorm_14": dict(N=512, C=512, H=14, W=14, groups=32, eps=1e-5, act=2, dtype=torch.bfloat16),
     # row reductions (shape ours)
     "reduce": dict(rows=32768, cols=8192, dtype=torch.bfloat16),
 }
