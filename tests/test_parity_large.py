@@ -71,6 +71,43 @@ def test_more_than_2_to_31_elements(kop):
     assert_close(x[SAMPLE], kopref.softmax_scale_bias(xs, bias.cpu(), 0.5, threads=None), 2e-2, "large softmax in place")
 
 
+def test_more_than_2_to_31_elements_ragged_rows(kop):
+    """The same for rows that are not whole 16-byte vectors: bf16 [1100000, 1999] (2.2e9 elements): edge elements and
+    aligned vectors of rows on both sides of the 2^31-element boundary (row 1074279), the span kernel's flat indices
+    beyond 2^32 bytes, in-place softmax."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 16 << 30:
+        pytest.skip("needs about 14 GB of free device memory")
+    rows, cols = 1100000, 1999
+    edge = (2 ** 31) // cols
+    sample = [0, 1, 2, edge - 1, edge, edge + 1, rows - 2, rows - 1]
+    g = torch.Generator(device="cuda")
+    g.manual_seed(11)
+    x = torch.empty((rows, cols), dtype=BF16, device="cuda")
+    for r0 in range(0, rows, 100000):
+        r1 = min(rows, r0 + 100000)
+        x[r0:r1] = torch.randn((r1 - r0, cols), generator=g, device="cuda", dtype=torch.float32).to(BF16)
+    assert x.numel() > 2 ** 31
+    xs = x[sample].cpu()
+    bias = torch.randn(cols, generator=g, device="cuda", dtype=torch.float32) * 0.1
+    v, i = kop.kop_reduce_rows(x, "max")
+    rv, ri = kopref.reduce_rows(xs, "max", threads=None)
+    assert np.array_equal(to_f64(v[sample]), rv) and np.array_equal(i[sample].cpu().numpy(), ri)
+    v, _ = kop.kop_reduce_rows(x, "sum")
+    assert_close(v[sample], kopref.reduce_rows(xs, "sum", threads=None)[0], 1e-3, "large ragged sum")
+    lab = torch.randint(0, cols, (rows,), generator=g, device="cuda").to(torch.int32)
+    loss, mean, bad = kop.kop_ce_loss_rowwise(x, lab)
+    rl, _, _ = kopref.ce_loss_rowwise(xs, lab[sample].cpu(), threads=None)
+    assert_close(loss[sample], rl, 2e-5, "large ragged ce loss")
+    assert int(bad) == 0 and abs(float(mean) - float(loss.double().mean())) < 1e-4
+    y = kop.kop_bias_act(x, bias, "silu")
+    assert_close(y[sample], kopref.bias_act(xs, bias.cpu(), "silu", threads=None), 2e-2, "large ragged bias_act")
+    del y
+    torch.cuda.empty_cache()
+    kop.kop_softmax_scale_bias(x, bias, 0.5, out=x)
+    assert_close(x[sample], kopref.softmax_scale_bias(xs, bias.cpu(), 0.5, threads=None), 2e-2, "large ragged softmax in place")
+
+
 def test_more_than_2_to_31_elements_images(kop):
     free, _ = torch.cuda.mem_get_info()
     if free < 30 << 30:
