@@ -159,9 +159,34 @@ pool2d_tile_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift,
                                      act_of(f[4 * q + 2], sc, sf, relu), act_of(f[4 * q + 3], sc, sf, relu));
         }
     } else {
-        for (int idx = threadIdx.x; idx < n_in; idx += kPoolThreads) {
-            const int r = idx / W, cc = idx - r * W;
+        // rows that are not whole vectors (odd widths, bases off a boundary): the run as head elements up to the first
+        // 16-byte boundary, aligned vectors whose elements may continue in the next row, and tail elements
+        int head = (int)(((16u - (unsigned)(reinterpret_cast<uintptr_t>(xp) & 15u)) & 15u) / (unsigned)sizeof(T));
+        if (head > n_in) head = n_in;
+        const int nv = (n_in - head) / E, tail0 = head + nv * E;
+        const float inv_w = 1.0f / (float)W;
+        for (int k = threadIdx.x; k < head + (n_in - tail0); k += kPoolThreads) {
+            const int idx = k < head ? k : tail0 + (k - head);
+            const int r = div_small(idx, W, inv_w), cc = idx - r * W;
             tile[(top + r) * Ws + lead + cc] = act_of(Elem<T>::load1(xp + idx), sc, sf, relu);
+        }
+        const T* xm = xp + head;
+#pragma unroll 2
+        for (int v = threadIdx.x; v < nv; v += kPoolThreads) {
+            float f[E];
+            Elem<T>::unpack(ld_stream(xm + (int64_t)v * E), f);
+            const int idx = head + v * E;
+            const int r = div_small(idx, W, inv_w);
+            int cc = idx - r * W;
+            float* dst = tile + (top + r) * Ws + lead + cc;
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                *dst++ = act_of(f[e], sc, sf, relu);
+                if (++cc == W) {
+                    cc = 0;
+                    dst += Ws - W;
+                }
+            }
         }
     }
     __syncthreads();
