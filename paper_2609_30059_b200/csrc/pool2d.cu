@@ -386,6 +386,159 @@ pool2d_strip_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift,
     }
 }
 
+// ---- the strip walk for stride-2 windows on rows of any width and alignment -----------------------------------
+// Widths that are not whole 8-column segments (55, 27, 147, 71, 35: the pooling layers of AlexNet-, SqueezeNet- and
+// Inception-style networks, 3 x 3 / stride 2 without padding) start every row at another offset from a 16-byte
+// boundary. A thread still owns four outputs and the nine (eight) input columns under them, but fetches them as the
+// aligned 16-byte vectors that cover them (three for fp32, two for 16-bit data) and picks its elements by the
+// offset, which is the same for all threads of a row, so the selection is a warp-uniform switch over register
+// moves. Every thread loads its own halo column: no shuffles, so threads past the end leave and short bands stop.
+// The first and last 16 bytes of the tensor are read element by element where a whole vector would cross its end.
+template <typename T>
+__device__ __forceinline__ Vec16 window_vector(uintptr_t q, uintptr_t xb, uintptr_t xe)
+{
+    if (q >= xb && q + 16 <= xe) {
+        const uint4 t = __ldg(reinterpret_cast<const uint4*>(q));
+        return Vec16{{t.x, t.y, t.z, t.w}};
+    }
+    Vec16 v{{0u, 0u, 0u, 0u}};
+    constexpr int E = Elem<T>::kPerVec;
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+        const uintptr_t a = q + e * sizeof(T);
+        if (a >= xb && a + sizeof(T) <= xe) {
+            if constexpr (sizeof(T) == 4) v.w[e] = *reinterpret_cast<const uint32_t*>(a);
+            else v.w[e / 2] |= (uint32_t)(*reinterpret_cast<const unsigned short*>(a)) << (16 * (e & 1));
+        }
+    }
+    return v;
+}
+
+// The nine elements that start at p, widened: r[0 .. 8].
+template <typename T>
+__device__ __forceinline__ void window9(const T* p, uintptr_t xb, uintptr_t xe, float (&r)[9])
+{
+    const uintptr_t addr = reinterpret_cast<uintptr_t>(p), base = addr & ~(uintptr_t)15;
+    const int s = (int)((addr - base) / sizeof(T));
+    if constexpr (sizeof(T) == 4) {
+        const Vec16 a = window_vector<T>(base, xb, xe), b = window_vector<T>(base + 16, xb, xe),
+                    c = window_vector<T>(base + 32, xb, xe);
+        const uint32_t w[12] = {a.w[0], a.w[1], a.w[2], a.w[3], b.w[0], b.w[1], b.w[2], b.w[3], c.w[0], c.w[1], c.w[2], c.w[3]};
+        switch (s) {
+        case 0:
+#pragma unroll
+            for (int e = 0; e < 9; ++e) r[e] = __uint_as_float(w[e]);
+            break;
+        case 1:
+#pragma unroll
+            for (int e = 0; e < 9; ++e) r[e] = __uint_as_float(w[e + 1]);
+            break;
+        case 2:
+#pragma unroll
+            for (int e = 0; e < 9; ++e) r[e] = __uint_as_float(w[e + 2]);
+            break;
+        default:
+#pragma unroll
+            for (int e = 0; e < 9; ++e) r[e] = __uint_as_float(w[e + 3]);
+            break;
+        }
+    } else {
+        const Vec16 a = window_vector<T>(base, xb, xe), b = window_vector<T>(base + 16, xb, xe);
+        const uint32_t w[8] = {a.w[0], a.w[1], a.w[2], a.w[3], b.w[0], b.w[1], b.w[2], b.w[3]};
+        uint32_t u[5];
+        switch (s >> 1) {
+        case 0:
+#pragma unroll
+            for (int i = 0; i < 5; ++i) u[i] = w[i];
+            break;
+        case 1:
+#pragma unroll
+            for (int i = 0; i < 5; ++i) u[i] = w[i + 1];
+            break;
+        case 2:
+#pragma unroll
+            for (int i = 0; i < 5; ++i) u[i] = w[i + 2];
+            break;
+        default:
+#pragma unroll
+            for (int i = 0; i < 5; ++i) u[i] = w[i + 3];
+            break;
+        }
+        if (s & 1) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) u[i] = __funnelshift_r(u[i], u[i + 1], 16);
+            u[4] >>= 16;
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float2 f;
+            Elem<T>::unpack_pair(u[i], f);
+            r[2 * i] = f.x;
+            r[2 * i + 1] = f.y;
+        }
+        float2 f;
+        Elem<T>::unpack_pair(u[4], f);
+        r[8] = f.x;
+    }
+}
+
+// P: padding (0 or 1, both directions); KS 3 with either, KS 2 without padding.
+template <typename T, int MODE, int KS, int P>
+__global__ void __launch_bounds__(256)
+pool2d_strip_any_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift, T* __restrict__ y, int64_t strips,
+                        int64_t x_elems, int C, int H, int W, int OH, int OW, int segs, int bands, int band_rows,
+                        int relu_flag, float inv_area)
+{
+    const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= strips) return;
+    const int seg = (int)(g % segs);
+    const int64_t rest = g / segs;
+    const int band = (int)(rest % bands);
+    const int64_t plane = rest / bands;
+    const int c = (int)(plane % C);
+    const float sc = scale.p != nullptr ? scale.at(c) : 1.0f;
+    const float sf = shift.p != nullptr ? shift.at(c) : 0.0f;
+    const float relu = relu_flag ? 0.0f : -INFINITY;
+    const float pad = MODE == 0 ? -INFINITY : 0.0f;
+    const uintptr_t xb = reinterpret_cast<uintptr_t>(x), xe = xb + (uintptr_t)x_elems * sizeof(T);
+    const int oh0 = band * band_rows, oh1 = min(OH, oh0 + band_rows);
+    const T* col = x + plane * H * (int64_t)W + (seg * 8 - P);        // this strip's first column (the halo with padding), row 0
+    T* out = y + (plane * OH + oh0) * (int64_t)OW + seg * 4;
+    const int nout = min(4, OW - seg * 4);
+
+    // horizontal windows of input row i for this thread's four outputs
+    auto hrow = [&](int i, float (&h)[4]) {
+        const bool row_ok = i >= 0 && i < H;
+        float v[9];
+        window9<T>(col + (int64_t)min(max(i, 0), H - 1) * W, xb, xe, v);
+#pragma unroll
+        for (int e = 0; e < 9; ++e) v[e] = row_ok ? act_of(v[e], sc, sf, relu) : pad;
+        if (P == 1 && seg == 0) v[0] = pad;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            h[j] = pool_op<T, MODE>(v[2 * j], v[2 * j + 1]);
+            if (KS == 3) h[j] = pool_op<T, MODE>(h[j], v[2 * j + 2]);
+        }
+    };
+    float carry[4];
+    if (KS == 3) hrow(2 * oh0 - P, carry);
+    for (int oh = oh0; oh < oh1; ++oh, out += OW) {
+        const int i1 = 2 * oh - P + (KS == 3 ? 1 : 0);
+        float a[4], b[4];
+        hrow(i1, a);
+        hrow(i1 + 1, b);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float r = pool_op<T, MODE>(a[j], b[j]);
+            if (KS == 3) {
+                r = pool_op<T, MODE>(carry[j], r);
+                carry[j] = b[j];
+            }
+            if (j < nout) Elem<T>::store1(out + j, MODE == 1 ? r * inv_area : r);
+        }
+    }
+}
+
 // ---- the same strip walk for 3x3 windows at stride 1 (pad 1): eight outputs per thread and row ----------------
 // A thread owns eight columns and produces the eight outputs above them: per input row one vector load, the left
 // and right halo values from the neighbour lanes by shuffle (the first / last lane of a warp loads its own; at the
@@ -1227,6 +1380,36 @@ kop_status_t launch_pool(const void* xv, ParamVec scale, ParamVec shift, void* y
             }
 #undef KOP_STRIP
             return launch_status();
+        }
+    }
+    // the same windows (and 3 x 3 without padding) on rows of any width and alignment, planes beyond the small-plane kernels
+    {
+        const bool k3p0 = kh == 3 && kw == 3 && ph == 0 && pw == 0;
+        // with padding the last window of an odd width would need a padded column on the far side too: even widths only.
+        // Planes from 256 elements (fp32 / bf16 TB/s against the runs-of-planes kernel: 17 x 17 3.2 / 1.6 to 3.7 / 1.9,
+        // 28 x 28 3.2 / 1.8 to 4.0 / 2.0; 13 x 13 and 15 x 15 fp32 3.1 / 3.2 to 2.7 / 2.8)
+        if ((k3p0 || (k3 && W % 2 == 0)) && sh == 2 && sw == 2 && (int64_t)H * W >= 256) {
+            const int segs = (OW + 3) / 4;
+            int band_rows = OH;
+            const int64_t want = 64LL * 32 * sm_count();
+            while (band_rows > 4 && planes * segs * ((OH + band_rows - 1) / band_rows) < want) band_rows = (band_rows + 1) / 2;
+            const int bands = (OH + band_rows - 1) / band_rows;
+            const int64_t strips = planes * segs * bands;
+            const int64_t blocks = (strips + 255) / 256;
+            if (blocks <= 0x7FFFFFFFLL) {
+#define KOP_STRIP_ANY(MODE, KS, P)                                                                     \
+    pool2d_strip_any_kernel<T, MODE, KS, P><<<(unsigned)blocks, 256, 0, stream>>>(                     \
+        x, scale, shift, y, strips, planes * H * W, (int)C, H, W, OH, OW, segs, bands, band_rows, relu, inv_area)
+                if (mode == 0) {
+                    if (k3p0) KOP_STRIP_ANY(0, 3, 0);
+                    else KOP_STRIP_ANY(0, 3, 1);
+                } else {
+                    if (k3p0) KOP_STRIP_ANY(1, 3, 0);
+                    else KOP_STRIP_ANY(1, 3, 1);
+                }
+#undef KOP_STRIP_ANY
+                return launch_status();
+            }
         }
     }
     // 2 x 2 / stride 2 without padding on anything the strip kernel does not take: a thread per output, no tile

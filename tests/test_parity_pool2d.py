@@ -95,6 +95,18 @@ POOL_CASES = [
     (1, 2, 224, 224, (224, 224), (1, 1), (0, 0), F32),
     (70, 3, 2, 2, (2, 2), (1, 1), (0, 0), F32),
     (33, 7, 1, 1, (1, 1), (1, 1), (0, 0), BF16),
+    # 3 x 3 / stride 2 on rows that are not whole 8-column segments: the strip walk with aligned window loads, every
+    # offset of a row from a 16-byte boundary (odd widths), a ragged last group of outputs, one band and several, a
+    # bottom padding row (odd height with padding), planes from 256 elements
+    (2, 3, 55, 55, (3, 3), (2, 2), (0, 0), F32),
+    (3, 5, 27, 27, (3, 3), (2, 2), (0, 0), BF16),
+    (1, 2, 147, 147, (3, 3), (2, 2), (0, 0), torch.float16),
+    (2, 3, 35, 71, (3, 3), (2, 2), (0, 0), F32),
+    (5, 7, 17, 17, (3, 3), (2, 2), (0, 0), BF16),
+    (2, 2, 111, 109, (3, 3), (2, 2), (0, 0), BF16),
+    (2, 3, 61, 60, (3, 3), (2, 2), (1, 1), F32),
+    (3, 4, 30, 30, (3, 3), (2, 2), (1, 1), torch.float16),
+    (2, 5, 16, 18, (3, 3), (2, 2), (1, 1), BF16),
 ]
 
 
@@ -118,6 +130,23 @@ def test_pool2d_parity(kop, N, C, H, W, kernel, stride, padding, dtype, seed):
             if mode == "max" and not affine:
                 assert np.array_equal(y.t.cpu().to(torch.float64).numpy(), ref), what + " (selection is exact)"
             y.check(what)
+
+
+@pytest.mark.parametrize("dtype", [F32, BF16])
+def test_pool2d_window_loads_at_the_tensor_ends(kop, dtype):
+    """The aligned window loads of the any-width strip kernel where a whole 16-byte vector would cross the tensor's first
+    or last byte: x starts one, two and three elements after a 16-byte boundary inside a larger buffer."""
+    N, C, H, W = 2, 3, 33, 37
+    x, scale, shift = synth.bn_pool_inputs(N, C, H, W, dtype, 4, "cuda")
+    ref = kopref.affine_relu_pool2d(host(x), host(scale), host(shift), (3, 3), (2, 2), (0, 0), "max", True, threads=None)
+    n = x.numel()
+    for off in (1, 2, 3, 5):
+        buf = torch.full((n + 16,), float("nan"), dtype=dtype, device="cuda")
+        buf[off:off + n] = x.reshape(-1)
+        y = Guarded((N, C, 16, 18), dtype)
+        kop.kop_affine_relu_pool2d(buf[off:off + n].view(N, C, H, W), scale, shift, (3, 3), (2, 2), (0, 0), "max", True, out=y.t)
+        assert_close(y.t, ref, tol_of(dtype), f"pool2d window loads, offset {off}")
+        y.check("pool2d window loads")
 
 
 def test_pool2d_full_config_seed0(kop):
