@@ -857,6 +857,51 @@ pool2d_k2s2_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift, T* _
     }
 }
 
+// The same for K x K windows at stride K without padding (K = 3, 4): K * K element loads an output; consecutive threads
+// take consecutive outputs, so the K loads of an input row by a warp cover a contiguous run between them.
+template <typename T, int MODE, int K>
+__global__ void __launch_bounds__(256)
+pool2d_kksk_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift, T* __restrict__ y, int total, MagicDiv by_c,
+                   int H, int W, MagicDiv by_oplane, MagicDiv by_ow, float relu_floor, float inv_area)
+{
+    constexpr int U = 2;                                     // outputs per thread
+    const bool identity = scale.p == nullptr && relu_floor == -INFINITY;
+    const int o0 = (int)blockIdx.x * (U * 256) + (int)threadIdx.x;
+    float v[U][K * K];
+    int pl[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const int o = o0 + u * 256;
+        pl[u] = 0;
+        if (o < total) {
+            const int p = by_oplane.div(o), r = o - p * by_oplane.d;
+            const int oi = by_ow.div(r), oj = r - oi * by_ow.d;
+            pl[u] = p;
+            const T* top = x + ((int64_t)p * H + K * oi) * W + K * oj;
+#pragma unroll
+            for (int di = 0; di < K; ++di)
+#pragma unroll
+                for (int dj = 0; dj < K; ++dj) v[u][di * K + dj] = Elem<T>::load1(top + (int64_t)di * W + dj);
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const int o = o0 + u * 256;
+        if (o < total) {
+            if (!identity) {
+                const int c = pl[u] - by_c.div(pl[u]) * by_c.d;
+                const float sc = scale.p != nullptr ? scale.at(c) : 1.0f, sf = shift.p != nullptr ? shift.at(c) : 0.0f;
+#pragma unroll
+                for (int e = 0; e < K * K; ++e) v[u][e] = act_of(v[u][e], sc, sf, relu_floor);
+            }
+            float res = v[u][0];
+#pragma unroll
+            for (int e = 1; e < K * K; ++e) res = MODE == 0 ? max_keep_nan(res, v[u][e]) : res + v[u][e];
+            Elem<T>::store1(y + o, MODE == 0 ? res : res * inv_area);
+        }
+    }
+}
+
 // The same for widths that are a multiple of four: a thread takes two adjacent outputs at a time, one load of four
 // elements per row (16 bytes of fp32, 8 of 16-bit data) and one store of the pair, which halves the index arithmetic
 // and the memory instructions per output (what bounded the 16-bit path above).
@@ -1444,6 +1489,22 @@ kop_status_t launch_pool(const void* xv, ParamVec scale, ParamVec shift, void* y
         if (mode == 0) { if (pair) KOP_K2S2(0, true); else KOP_K2S2(0, false); }
         else { if (pair) KOP_K2S2(1, true); else KOP_K2S2(1, false); }
 #undef KOP_K2S2
+        return launch_status();
+    }
+    // K x K / stride K without padding, K = 3 or 4: a thread per output as well (same index limits)
+    if (kh == kw && sh == kh && sw == kw && (kh == 3 || kh == 4) && ph == 0 && pw == 0 && planes * OH * OW < (1LL << 31) - 1024 &&
+        planes < (1LL << 24) && planes * C < (1LL << 40) && planes * OH * OW * std::max((int64_t)OH * OW, (int64_t)1) < (1LL << 40)) {
+        const int total = (int)(planes * OH * OW);
+        const MagicDiv by_oplane{((1ULL << 40) + (uint64_t)(OH * OW) - 1) / (uint64_t)(OH * OW), OH * OW};
+        const MagicDiv by_ow{((1ULL << 40) + (uint64_t)OW - 1) / (uint64_t)OW, OW};
+        const MagicDiv by_c{((1ULL << 40) + (uint64_t)C - 1) / (uint64_t)C, (int)C};
+        const unsigned blocks = (unsigned)((total + 511) / 512);
+        const float floor_v = relu ? 0.0f : -INFINITY;
+#define KOP_KKSK(M, K) \
+    pool2d_kksk_kernel<T, M, K><<<blocks, 256, 0, stream>>>(x, scale, shift, y, total, by_c, H, W, by_oplane, by_ow, floor_v, inv_area)
+        if (mode == 0) { if (kh == 3) KOP_KKSK(0, 3); else KOP_KKSK(0, 4); }
+        else { if (kh == 3) KOP_KKSK(1, 3); else KOP_KKSK(1, 4); }
+#undef KOP_KKSK
         return launch_status();
     }
     // 3x3 / stride 1 / pad 1 over rows of whole, aligned 8-column segments: the stride-1 strip kernel

@@ -107,6 +107,13 @@ POOL_CASES = [
     (2, 3, 61, 60, (3, 3), (2, 2), (1, 1), F32),
     (3, 4, 30, 30, (3, 3), (2, 2), (1, 1), torch.float16),
     (2, 5, 16, 18, (3, 3), (2, 2), (1, 1), BF16),
+    # K x K windows at stride K without padding (K = 3, 4): a thread per output; sizes that leave unread rows / columns
+    (2, 3, 113, 113, (3, 3), (3, 3), (0, 0), F32),
+    (3, 5, 27, 28, (3, 3), (3, 3), (0, 0), BF16),
+    (2, 4, 56, 56, (4, 4), (4, 4), (0, 0), torch.float16),
+    (5, 7, 9, 10, (4, 4), (4, 4), (0, 0), F32),
+    (1, 2, 256, 256, (3, 3), (3, 3), (0, 0), BF16),
+    (70, 9, 4, 4, (4, 4), (4, 4), (0, 0), BF16),
 ]
 
 
