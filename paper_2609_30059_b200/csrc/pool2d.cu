@@ -482,13 +482,15 @@ __device__ __forceinline__ void window9(const T* p, uintptr_t xb, uintptr_t xe, 
     }
 }
 
-// P: padding (0 or 1, both directions); KS 3 with either, KS 2 without padding.
-template <typename T, int MODE, int KS, int P>
+// 3 x 3 windows; ST: stride 1 or 2; P: padding 0 or 1 (both directions). A thread's nine elements start at column
+// 4 ST seg - P; with padding the columns from W on are padding too (the last window of a row reaches one).
+template <typename T, int MODE, int ST, int P>
 __global__ void __launch_bounds__(256)
 pool2d_strip_any_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift, T* __restrict__ y, int64_t strips,
                         int64_t x_elems, int C, int H, int W, int OH, int OW, int segs, int bands, int band_rows,
                         int relu_flag, float inv_area)
 {
+    constexpr int KS = 3;
     const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (g >= strips) return;
     const int seg = (int)(g % segs);
@@ -502,9 +504,11 @@ pool2d_strip_any_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift,
     const float pad = MODE == 0 ? -INFINITY : 0.0f;
     const uintptr_t xb = reinterpret_cast<uintptr_t>(x), xe = xb + (uintptr_t)x_elems * sizeof(T);
     const int oh0 = band * band_rows, oh1 = min(OH, oh0 + band_rows);
-    const T* col = x + plane * H * (int64_t)W + (seg * 8 - P);        // this strip's first column (the halo with padding), row 0
+    const int c0 = seg * 4 * ST - P;                                  // this strip's first column (the halo with padding)
+    const T* col = x + plane * H * (int64_t)W + c0;
     T* out = y + (plane * OH + oh0) * (int64_t)OW + seg * 4;
     const int nout = min(4, OW - seg * 4);
+    const int nvalid = W - c0;                                        // elements of the nine that are image columns
 
     // horizontal windows of input row i for this thread's four outputs
     auto hrow = [&](int i, float (&h)[4]) {
@@ -512,30 +516,27 @@ pool2d_strip_any_kernel(const T* __restrict__ x, ParamVec scale, ParamVec shift,
         float v[9];
         window9<T>(col + (int64_t)min(max(i, 0), H - 1) * W, xb, xe, v);
 #pragma unroll
-        for (int e = 0; e < 9; ++e) v[e] = row_ok ? act_of(v[e], sc, sf, relu) : pad;
+        for (int e = 0; e < 9; ++e) v[e] = (row_ok && (P == 0 || e < nvalid)) ? act_of(v[e], sc, sf, relu) : pad;
         if (P == 1 && seg == 0) v[0] = pad;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            h[j] = pool_op<T, MODE>(v[2 * j], v[2 * j + 1]);
-            if (KS == 3) h[j] = pool_op<T, MODE>(h[j], v[2 * j + 2]);
-        }
+        for (int j = 0; j < 4; ++j)
+            h[j] = pool_op<T, MODE>(pool_op<T, MODE>(v[ST * j], v[ST * j + 1]), v[ST * j + 2]);
     };
-    float carry[4];
-    if (KS == 3) hrow(2 * oh0 - P, carry);
+    float hs[KS][4];
+#pragma unroll
+    for (int i = 0; i < KS - ST; ++i) hrow(ST * oh0 - P + i, hs[i]);
     for (int oh = oh0; oh < oh1; ++oh, out += OW) {
-        const int i1 = 2 * oh - P + (KS == 3 ? 1 : 0);
-        float a[4], b[4];
-        hrow(i1, a);
-        hrow(i1 + 1, b);
+#pragma unroll
+        for (int i = KS - ST; i < KS; ++i) hrow(ST * oh - P + i, hs[i]);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            float r = pool_op<T, MODE>(a[j], b[j]);
-            if (KS == 3) {
-                r = pool_op<T, MODE>(carry[j], r);
-                carry[j] = b[j];
-            }
+            const float r = pool_op<T, MODE>(pool_op<T, MODE>(hs[0][j], hs[1][j]), hs[2][j]);
             if (j < nout) Elem<T>::store1(out + j, MODE == 1 ? r * inv_area : r);
         }
+#pragma unroll
+        for (int i = 0; i < KS - ST; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) hs[i][j] = hs[i + ST][j];
     }
 }
 
@@ -1427,13 +1428,17 @@ kop_status_t launch_pool(const void* xv, ParamVec scale, ParamVec shift, void* y
             return launch_status();
         }
     }
-    // the same windows (and 3 x 3 without padding) on rows of any width and alignment, planes beyond the small-plane kernels
+    // 3 x 3 windows at stride 2 (with or without padding) or stride 1 (with padding) on rows of any width and alignment
+    // that the aligned strip kernels do not take.
+    // Planes from 256 elements (fp32 / bf16 TB/s against the runs-of-planes kernel: 17 x 17 3.2 / 1.6 to 3.7 / 1.9,
+    // 28 x 28 3.2 / 1.8 to 4.0 / 2.0; 13 x 13 and 15 x 15 fp32 3.1 / 3.2 to 2.7 / 2.8)
     {
         const bool k3p0 = kh == 3 && kw == 3 && ph == 0 && pw == 0;
-        // with padding the last window of an odd width would need a padded column on the far side too: even widths only.
-        // Planes from 256 elements (fp32 / bf16 TB/s against the runs-of-planes kernel: 17 x 17 3.2 / 1.6 to 3.7 / 1.9,
-        // 28 x 28 3.2 / 1.8 to 4.0 / 2.0; 13 x 13 and 15 x 15 fp32 3.1 / 3.2 to 2.7 / 2.8)
-        if ((k3p0 || (k3 && W % 2 == 0)) && sh == 2 && sw == 2 && (int64_t)H * W >= 256) {
+        // at stride 1 only odd widths (fp32 / bf16: 57 x 57 2.6 / 1.4 to 3.4 / 1.7, 35 x 35 3.1 / 1.5 to 3.3 / 1.6, 17 x 17
+        // 2.7 / 1.3 to 3.0 / 1.3; even widths that are not whole segments are faster out of the shared-memory walk:
+        // 28 x 28 3.8 / 2.3 against 2.9 / 1.4 here)
+        if (((k3p0 || k3) && sh == 2 && sw == 2 && (int64_t)H * W >= 256) ||
+            (k3 && sh == 1 && sw == 1 && W % 2 == 1 && (int64_t)H * W >= 256)) {
             const int segs = (OW + 3) / 4;
             int band_rows = OH;
             const int64_t want = 64LL * 32 * sm_count();
@@ -1442,16 +1447,18 @@ kop_status_t launch_pool(const void* xv, ParamVec scale, ParamVec shift, void* y
             const int64_t strips = planes * segs * bands;
             const int64_t blocks = (strips + 255) / 256;
             if (blocks <= 0x7FFFFFFFLL) {
-#define KOP_STRIP_ANY(MODE, KS, P)                                                                     \
-    pool2d_strip_any_kernel<T, MODE, KS, P><<<(unsigned)blocks, 256, 0, stream>>>(                     \
+#define KOP_STRIP_ANY(MODE, ST, P)                                                                     \
+    pool2d_strip_any_kernel<T, MODE, ST, P><<<(unsigned)blocks, 256, 0, stream>>>(                     \
         x, scale, shift, y, strips, planes * H * W, (int)C, H, W, OH, OW, segs, bands, band_rows, relu, inv_area)
-                if (mode == 0) {
-                    if (k3p0) KOP_STRIP_ANY(0, 3, 0);
-                    else KOP_STRIP_ANY(0, 3, 1);
-                } else {
-                    if (k3p0) KOP_STRIP_ANY(1, 3, 0);
-                    else KOP_STRIP_ANY(1, 3, 1);
-                }
+#define KOP_STRIP_ANY_M(MODE)                         \
+    do {                                              \
+        if (sh == 1) KOP_STRIP_ANY(MODE, 1, 1);       \
+        else if (k3p0) KOP_STRIP_ANY(MODE, 2, 0);     \
+        else KOP_STRIP_ANY(MODE, 2, 1);               \
+    } while (0)
+                if (mode == 0) KOP_STRIP_ANY_M(0);
+                else KOP_STRIP_ANY_M(1);
+#undef KOP_STRIP_ANY_M
 #undef KOP_STRIP_ANY
                 return launch_status();
             }

@@ -107,6 +107,11 @@ POOL_CASES = [
     (2, 3, 61, 60, (3, 3), (2, 2), (1, 1), F32),
     (3, 4, 30, 30, (3, 3), (2, 2), (1, 1), torch.float16),
     (2, 5, 16, 18, (3, 3), (2, 2), (1, 1), BF16),
+    (2, 3, 57, 57, (3, 3), (2, 2), (1, 1), F32),                   # padded odd width: a padding column on the far side too
+    (3, 2, 27, 33, (3, 3), (2, 2), (1, 1), BF16),
+    (2, 3, 35, 35, (3, 3), (1, 1), (1, 1), F32),                   # stride 1 on odd widths: the same kernel
+    (3, 5, 17, 17, (3, 3), (1, 1), (1, 1), BF16),
+    (1, 2, 66, 57, (3, 3), (1, 1), (1, 1), torch.float16),
     # K x K windows at stride K without padding (K = 3, 4): a thread per output; sizes that leave unread rows / columns
     (2, 3, 113, 113, (3, 3), (3, 3), (0, 0), F32),
     (3, 5, 27, 28, (3, 3), (3, 3), (0, 0), BF16),
