@@ -255,3 +255,104 @@ def test_fuzz_image_kernels(kop):
             y, _, _ = kop.kop_groupnorm_act_ex(xg, g16, be16, groups, 1e-5, act)
             assert_close(y, kopref.groupnorm_act(host(xg), host(g16), host(be16), groups, 1e-5, act)[0], tol, "groupnorm_ex y " + what)
     assert kop.kop_groupnorm_wait_timeouts() == 0
+
+
+def rehome(rng, t, off, pad):
+    """A copy of the 2-D tensor t whose first element sits `off` elements after a 16-byte boundary and whose rows are
+    `pad` elements apart beyond their length (pad = 0: contiguous); surrounded by NaN so that a stray read shows."""
+    rows, cols = t.shape
+    stride = cols + pad
+    buf = torch.full((rows * stride + 32,), float("nan"), dtype=t.dtype, device=t.device)
+    view = buf[off:off + rows * stride].view(rows, stride)[:, :cols]
+    view.copy_(t)
+    return view
+
+
+def test_fuzz_rows_off_the_vector_grid(kop):
+    """Rows that are not whole aligned 16-byte vectors, input and output at the same random offset from a boundary and
+    with the same random row pitch (the head / vectors / tail split of the softmax, cross-entropy, reduction and
+    bias + activation kernels), in place as well; nothing outside the output rows may change."""
+    rng = np.random.default_rng(197_50257)
+    for it in range(150):
+        dtype = (F32, BF16, F16)[int(rng.integers(0, 3))]
+        tol = tol_of(dtype)
+        rows = pick_len(rng, 40)
+        cols = pick_len(rng, 2600) if rng.integers(0, 4) else int(rng.integers(8000, 20000))
+        off = int(rng.integers(0, 8))
+        pad = int(rng.integers(0, 2)) * int(rng.integers(1, 12))
+        seed = int(rng.integers(0, 1 << 30))
+        what = f"it={it} rows={rows} cols={cols} off={off} pad={pad} {dtype}"
+        x, bias = synth.softmax_inputs(rows, cols, dtype, seed, "cuda")
+        xs = rehome(rng, x, off, pad)
+        use_bias = bool(rng.integers(0, 2))
+        b, hb = (bias, host(bias)) if use_bias else (None, None)
+        log_out = bool(rng.integers(0, 2))
+        out = rehome(rng, torch.full_like(x, 7.0), off, pad)
+        frame = out.untyped_storage()                       # the whole buffer, to check the pitch gaps afterwards
+        kop.kop_softmax_opts(xs, b, 0.5, log_out, 0, out=out)
+        ref = kopref.softmax_opts(host(x), hb, 0.5, log_out, 0)
+        assert_close(out, ref, tol, "softmax " + what)
+        if pad:
+            gaps = torch.empty(0, dtype=dtype, device="cuda").set_(frame)[off:off + rows * (cols + pad)].view(rows, cols + pad)[:, cols:]
+            assert bool(torch.isnan(gaps).all()), "softmax wrote between rows " + what
+        xi = rehome(rng, x, off, pad)
+        kop.kop_softmax_scale_bias(xi, b, 0.5, out=xi)
+        assert_close(xi, kopref.softmax_scale_bias(host(x), hb, 0.5), tol, "softmax in place " + what)
+        # reductions and cross-entropy read only
+        op = ("sum", "max", "min", "logsumexp", "mean")[int(rng.integers(0, 5))]
+        v, i = kop.kop_reduce_rows(xs, op)
+        rv, ri = kopref.reduce_rows(host(x), op)
+        if op in ("max", "min"):
+            assert np.array_equal(to_f64(v), rv) and np.array_equal(i.cpu().numpy(), ri), f"reduce {op} " + what
+        else:
+            mag = np.maximum(1.0, host(x).double().abs().sum(dim=1).numpy()) / (cols if op == "mean" else 1.0)
+            bound = 1e-5 * (mag if op != "logsumexp" else np.maximum(1.0, np.abs(rv)))
+            assert np.all(np.abs(to_f64(v) - rv) <= bound), f"reduce {op} " + what
+        z, lab = synth.ce_inputs(rows, cols, dtype, seed, "cuda")
+        loss, mean, bad = kop.kop_ce_loss_rowwise(rehome(rng, z, off, pad), lab)
+        rl, rmean, rbad = kopref.ce_loss_rowwise(host(z), host(lab))
+        assert_close(loss, rl, max(tol, 2e-5), "ce loss " + what)
+        # bias + activation and the chain: contiguous tensors take the span kernel, pitched ones the element-wise one
+        act = ("silu", "gelu_tanh", "relu", "tanh")[int(rng.integers(0, 4))]
+        out = rehome(rng, torch.full_like(x, 7.0), off, pad)
+        kop.kop_bias_act(xs, b, act, out=out)
+        assert_close(out, kopref.bias_act(host(x), hb, act), tol, f"bias_act {act} " + what)
+        r, _ = synth.softmax_inputs(rows, cols, dtype, seed + 1, "cuda")
+        rs_ = rehome(rng, r, off, pad)
+        kop.kop_epilogue_chain(xs, b, rs_, 0.7, 1.5, -1.0, 2.0, act, out=rs_)
+        assert_close(rs_, kopref.epilogue_chain(host(x), hb, host(r), 0.7, 1.5, -1.0, 2.0, act), tol, f"chain {act} " + what)
+
+
+def test_fuzz_images_off_the_vector_grid(kop):
+    """GroupNorm chunks in registers and the any-width pooling strips on tensors whose first element sits at a random offset
+    from a 16-byte boundary, input and output alike."""
+    rng = np.random.default_rng(55_27_13)
+    for it in range(80):
+        dtype = (F32, BF16, F16)[int(rng.integers(0, 3))]
+        tol = tol_of(dtype)
+        N, H, W = int(rng.integers(1, 4)), int(rng.integers(3, 60)), int(rng.integers(3, 60))
+        groups = int(rng.choice([1, 2, 4, 8]))
+        C = groups * int(rng.integers(1, 7))
+        off = int(rng.integers(0, 8))
+        seed = int(rng.integers(0, 1 << 30))
+        what = f"it={it} N={N} C={C} H={H} W={W} G={groups} off={off} {dtype}"
+        x, gamma, beta = synth.groupnorm_inputs(N, C, H, W, dtype, seed, "cuda")
+        n = x.numel()
+        xb = torch.full((n + 32,), float("nan"), dtype=dtype, device="cuda")
+        xb[off:off + n] = x.reshape(-1)
+        xv = xb[off:off + n].view(N, C, H, W)
+        yb = torch.full((n + 32,), 5.0, dtype=dtype, device="cuda")
+        yv = yb[off:off + n].view(N, C, H, W)
+        act = int(rng.integers(0, 3))
+        kop.kop_groupnorm_act(xv, gamma, beta, groups, 1e-5, act, out=yv)
+        ry, rm, rr = kopref.groupnorm_act(host(x), host(gamma), host(beta), groups, 1e-5, act)
+        assert_close(yv, ry, tol, "groupnorm " + what)
+        assert bool((yb[:off] == 5.0).all()) and bool((yb[off + n:] == 5.0).all()), "groupnorm wrote outside " + what
+        st = int(rng.integers(1, 3))
+        pd = int(rng.integers(0, 2))
+        if H + 2 * pd >= 3 and W + 2 * pd >= 3:
+            _, scale, shift = synth.bn_pool_inputs(N, C, H, W, dtype, seed, "cuda")
+            mode = "max" if rng.integers(0, 2) else "avg"
+            y = kop.kop_affine_relu_pool2d(xv, scale, shift, (3, 3), (st, st), (pd, pd), mode, True)
+            ref = kopref.affine_relu_pool2d(host(x), host(scale), host(shift), (3, 3), (st, st), (pd, pd), mode, True)
+            assert_close(y, ref, tol, f"pool2d 3x3 s={st} p={pd} {mode} " + what)
