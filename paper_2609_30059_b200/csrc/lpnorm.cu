@@ -23,23 +23,47 @@ __device__ __forceinline__ float inv_norm(float s, float eps, float* norm)
     return n != n ? n : 1.0f / fmaxf(n, eps);
 }
 
-template <typename T, int L, int P>
+// kRagged (all three vector kernels): rows that are not whole aligned vectors; `nvec` then carries the row length in
+// elements, a row is split into head elements up to the first 16-byte boundary, whole vectors and tail elements, and the
+// edge elements go to the row's lanes (one or two each) or one to a thread. x and y rows sit at the same offset from a
+// boundary.
+template <typename T, int L, int P, bool kRagged = false>
 __global__ void __launch_bounds__(256)
 lpnorm_group_kernel(const T* __restrict__ x, T* __restrict__ y, float* __restrict__ norm_out, int64_t rows, int nvec,
                     int64_t x_stride, int64_t y_stride, float eps)
 {
     constexpr int E = Elem<T>::kPerVec, Q = E / 2, VPL = 4;
+    constexpr int KE = kRagged ? (2 * (E - 1) + L - 1) / L : 1;      // edge elements a lane holds at most
     const int lane = threadIdx.x & 31, sub = lane & (L - 1);
     const int64_t row = ((int64_t)blockIdx.x * 8 + (threadIdx.x >> 5)) * (32 / L) + lane / L;
     const bool live = row < rows;
     const int64_t r = live ? row : 0;
     const T* xr = x + r * x_stride;
+    T* yr = y + r * y_stride;
+    int edge_col[KE];                                        // this lane's edge columns (-1: none) and their values
+    float ev[KE];
+#pragma unroll
+    for (int q = 0; q < KE; ++q) edge_col[q] = -1, ev[q] = 0.0f;
+    const T* xm = xr;                                        // first whole vector of the row
+    T* ym = yr;
+    if constexpr (kRagged) {
+        const RowSplit<T> sp = row_split<T>(xr, nvec);
+#pragma unroll
+        for (int q = 0; q < KE; ++q)
+            if (live && sub + q * L < sp.edges()) {
+                edge_col[q] = sp.edge_col(sub + q * L);
+                ev[q] = Elem<T>::load1(xr + edge_col[q]);
+            }
+        nvec = sp.nvec;
+        xm += sp.head;
+        ym += sp.head;
+    }
     Vec16 raw[VPL];
 #pragma unroll
     for (int k = 0; k < VPL; ++k) {
         const int v = k * L + sub;
         raw[k] = Vec16{{0u, 0u, 0u, 0u}};
-        if (live && v < nvec) raw[k] = ld_stream(xr + (int64_t)v * E);
+        if (live && v < nvec) raw[k] = ld_stream(xm + (int64_t)v * E);
     }
     float2 val[VPL][Q];
     float2 acc = make_float2(0.0f, 0.0f);
@@ -50,6 +74,10 @@ lpnorm_group_kernel(const T* __restrict__ x, T* __restrict__ y, float* __restric
         for (int q = 0; q < Q; ++q) acc = accumulate<P>(acc, val[k][q]);
     }
     float s = acc.x + acc.y;
+    if constexpr (kRagged) {
+#pragma unroll
+        for (int q = 0; q < KE; ++q) s = P == 1 ? s + fabsf(ev[q]) : fmaf(ev[q], ev[q], s);
+    }
 #pragma unroll
     for (int o = L / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
     float n;
@@ -63,12 +91,17 @@ lpnorm_group_kernel(const T* __restrict__ x, T* __restrict__ y, float* __restric
             float2 o[Q];
 #pragma unroll
             for (int q = 0; q < Q; ++q) o[q] = __fmul2_rn(val[k][q], inv2);
-            st_stream(y + r * y_stride + (int64_t)v * E, Elem<T>::pack2(o));
+            st_stream(ym + (int64_t)v * E, Elem<T>::pack2(o));
         }
+    }
+    if constexpr (kRagged) {
+#pragma unroll
+        for (int q = 0; q < KE; ++q)
+            if (edge_col[q] >= 0) Elem<T>::store1(yr + edge_col[q], ev[q] * inv);
     }
 }
 
-template <typename T, int VPT, int P>
+template <typename T, int VPT, int P, bool kRagged = false>
 __global__ void __launch_bounds__(max_threads_for(VPT * Elem<T>::kPerVec))
 lpnorm_block_kernel(const T* __restrict__ x, T* __restrict__ y, float* __restrict__ norm_out, int nvec, int64_t x_stride,
                     int64_t y_stride, float eps)
@@ -78,12 +111,26 @@ lpnorm_block_kernel(const T* __restrict__ x, T* __restrict__ y, float* __restric
     const int64_t row = blockIdx.x;
     const T* xr = x + row * x_stride;
     T* yr = y + row * y_stride;
+    const T* xm = xr;
+    T* ym = yr;
+    int edge_col = -1;
+    float ev = 0.0f;
+    if constexpr (kRagged) {
+        const RowSplit<T> sp = row_split<T>(xr, nvec);
+        if ((int)threadIdx.x < sp.edges()) {
+            edge_col = sp.edge_col(threadIdx.x);
+            ev = Elem<T>::load1(xr + edge_col);
+        }
+        nvec = sp.nvec;
+        xm += sp.head;
+        ym += sp.head;
+    }
     Vec16 raw[VPT];
 #pragma unroll
     for (int k = 0; k < VPT; ++k) {
         const int v = k * blockDim.x + threadIdx.x;
         raw[k] = Vec16{{0u, 0u, 0u, 0u}};
-        if (v < nvec) raw[k] = ld_stream(xr + (int64_t)v * E);
+        if (v < nvec) raw[k] = ld_stream(xm + (int64_t)v * E);
     }
     float2 val[VPT][Q];
     float2 acc = make_float2(0.0f, 0.0f);
@@ -93,8 +140,10 @@ lpnorm_block_kernel(const T* __restrict__ x, T* __restrict__ y, float* __restric
 #pragma unroll
         for (int q = 0; q < Q; ++q) acc = accumulate<P>(acc, val[k][q]);
     }
+    float part = acc.x + acc.y;
+    if constexpr (kRagged) part = P == 1 ? part + fabsf(ev) : fmaf(ev, ev, part);
     float n;
-    const float inv = inv_norm<P>(block_sum(acc.x + acc.y, red), eps, &n);
+    const float inv = inv_norm<P>(block_sum(part, red), eps, &n);
     if (threadIdx.x == 0 && norm_out != nullptr) norm_out[row] = n;
     const float2 inv2 = make_float2(inv, inv);
 #pragma unroll
@@ -104,12 +153,15 @@ lpnorm_block_kernel(const T* __restrict__ x, T* __restrict__ y, float* __restric
             float2 o[Q];
 #pragma unroll
             for (int q = 0; q < Q; ++q) o[q] = __fmul2_rn(val[k][q], inv2);
-            st_stream(yr + (int64_t)v * E, Elem<T>::pack2(o));
+            st_stream(ym + (int64_t)v * E, Elem<T>::pack2(o));
         }
+    }
+    if constexpr (kRagged) {
+        if (edge_col >= 0) Elem<T>::store1(yr + edge_col, ev * inv);
     }
 }
 
-template <typename T, int P>
+template <typename T, int P, bool kRagged = false>
 __global__ void __launch_bounds__(512)
 lpnorm_long_kernel(const T* __restrict__ x, T* __restrict__ y, float* __restrict__ norm_out, int nvec, int64_t x_stride,
                    int64_t y_stride, float eps)
@@ -119,6 +171,20 @@ lpnorm_long_kernel(const T* __restrict__ x, T* __restrict__ y, float* __restrict
     const int64_t row = blockIdx.x;
     const T* xr = x + row * x_stride;
     T* yr = y + row * y_stride;
+    int edge_col = -1;
+    float ev = 0.0f;
+    T* edge_dst = yr;
+    if constexpr (kRagged) {
+        const RowSplit<T> sp = row_split<T>(xr, nvec);
+        if ((int)threadIdx.x < sp.edges()) {
+            edge_col = sp.edge_col(threadIdx.x);
+            ev = Elem<T>::load1(xr + edge_col);
+            edge_dst = yr + edge_col;
+        }
+        nvec = sp.nvec;
+        xr += sp.head;
+        yr += sp.head;
+    }
     const int step = U * blockDim.x;
     const int nbatch = (nvec + step - 1) / step;
     const uint64_t keep = l2_policy_keep(), drop = l2_policy_drop();
@@ -139,10 +205,15 @@ lpnorm_long_kernel(const T* __restrict__ x, T* __restrict__ y, float* __restrict
             for (int q = 0; q < Q; ++q) acc = accumulate<P>(acc, val[q]);
         }
     }
+    float part = acc.x + acc.y;
+    if constexpr (kRagged) part = P == 1 ? part + fabsf(ev) : fmaf(ev, ev, part);
     float n;
-    const float inv = inv_norm<P>(block_sum(acc.x + acc.y, red), eps, &n);
+    const float inv = inv_norm<P>(block_sum(part, red), eps, &n);
     if (threadIdx.x == 0 && norm_out != nullptr) norm_out[row] = n;
     const float2 inv2 = make_float2(inv, inv);
+    if constexpr (kRagged) {
+        if (edge_col >= 0) Elem<T>::store1(edge_dst, ev * inv);
+    }
     // backwards: the end of the row is what the first sweep left in the L2; y[v] is written by the thread that
     // read x[v], after every thread has finished the first sweep (the barrier in block_sum)
     for (int b = nbatch - 1; b >= 0; --b) {
@@ -231,6 +302,42 @@ kop_status_t launch_lpnorm(const void* xv, void* yv, float* norm_out, int64_t ro
     }
     if (vec && nvec64 <= 0x7FFFFFFF) {
         lpnorm_long_kernel<T, P><<<(unsigned)rows, 512, 0, stream>>>(x, y, norm_out, (int)nvec64, xs, ys, eps);
+        return launch_status();
+    }
+    // rows that are not whole aligned vectors, x and y rows at the same offset from a 16-byte boundary: head elements,
+    // aligned vectors, tail elements in the same three kernels
+    const bool ragged = !vec && (reinterpret_cast<uintptr_t>(x) - reinterpret_cast<uintptr_t>(y)) % 16 == 0 &&
+                        ((xs - ys) * (int64_t)sizeof(T)) % 16 == 0 && cols <= 0x7FFFFFFFLL;
+    if (ragged && nvec64 <= 128) {
+        const int lanes = nvec64 > 64 ? 32 : nvec64 > 32 ? 16 : 8;
+        const int64_t rows_per_cta = 8 * (32 / lanes);
+        const int64_t ctas = (rows + rows_per_cta - 1) / rows_per_cta;
+        if (ctas > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
+#define KOP_LP_RAG(L) lpnorm_group_kernel<T, L, P, true><<<(unsigned)ctas, 256, 0, stream>>>(x, y, norm_out, rows, (int)cols, xs, ys, eps)
+        if (lanes == 32) KOP_LP_RAG(32);
+        else if (lanes == 16) KOP_LP_RAG(16);
+        else KOP_LP_RAG(8);
+#undef KOP_LP_RAG
+        return launch_status();
+    }
+    if (ragged && cols <= kMaxRegisterRow) {
+        const int nvec = (int)nvec64;
+        int vals = 32;
+        if (cols <= 1024) vals = 16;
+        if ((nvec + vals / E - 1) / (vals / E) > max_threads_for(vals)) vals = 64;
+        const int vpt = vals / E;
+        const int threads = ((nvec + vpt - 1) / vpt + 31) / 32 * 32;
+#define KOP_LP_BLOCK_RAG(V) lpnorm_block_kernel<T, V, P, true><<<(unsigned)rows, threads, 0, stream>>>(x, y, norm_out, (int)cols, xs, ys, eps)
+        switch (vals) {
+        case 16: KOP_LP_BLOCK_RAG(16 / E); break;
+        case 32: KOP_LP_BLOCK_RAG(32 / E); break;
+        default: KOP_LP_BLOCK_RAG(64 / E); break;
+        }
+#undef KOP_LP_BLOCK_RAG
+        return launch_status();
+    }
+    if (ragged) {
+        lpnorm_long_kernel<T, P, true><<<(unsigned)rows, 512, 0, stream>>>(x, y, norm_out, (int)cols, xs, ys, eps);
         return launch_status();
     }
     lpnorm_scalar_kernel<T, P><<<(unsigned)rows, 256, 0, stream>>>(x, y, norm_out, cols, xs, ys, eps);

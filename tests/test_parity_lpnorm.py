@@ -16,7 +16,10 @@ SEEDS = synth.SEEDS
 F32, BF16, F16 = torch.float32, torch.bfloat16, torch.float16
 SHAPES = [(2048, 4096, BF16), (300, 4096, F32), (1031, 64, BF16), (517, 128, F32), (259, 520, F16), (65, 1000, F32),
           (33, 1001, F32), (17, 16384, BF16), (9, 20480, F32), (5, 40008, BF16), (3, 20481, BF16), (7, 1, F32),
-          (131, 768, BF16), (67, 1024, F16)]
+          (131, 768, BF16), (67, 1024, F16),
+          # rows that are not whole aligned vectors: edge elements around the aligned vectors in all three kernels
+          (700, 197, BF16), (300, 77, F32), (64, 1001, F32), (41, 4097, BF16), (9, 20011, BF16), (5, 70001, F32),
+          (130, 7, torch.float16), (50, 3, F32), (33, 2051, torch.float16)]
 
 
 @pytest.fixture(scope="module")
@@ -82,3 +85,23 @@ def test_lp_normalize_options_and_special_values(kop):
     t = x[:8].contiguous().view(1, -1)
     _, fn = kop.kop_lp_normalize_rows(t, 2)
     assert abs(float(fn[0]) - float(torch.linalg.matrix_norm(x[:8].double()))) <= 1e-5 * float(fn[0])
+
+
+def test_lp_normalize_rows_off_the_vector_grid(kop):
+    """x and y one element off a 16-byte boundary alike (the split kernels), in place, and at different offsets (the
+    element-wise kernel); nothing outside y may change."""
+    for dtype, (rows, cols) in ((BF16, (300, 197)), (F32, (64, 1001)), (torch.float16, (5, 20011))):
+        x, _ = synth.softmax_inputs(rows, cols, dtype, 3, "cuda")
+        n = rows * cols
+        ry, rn = kopref.lp_normalize_rows(host(x), 2, 1e-12, threads=None)
+        xo = torch.zeros(n + 16, dtype=dtype, device="cuda")
+        xo[1:n + 1] = x.reshape(-1)
+        for yoff in (1, 2):
+            yo = torch.full((n + 16,), 9.0, dtype=dtype, device="cuda")
+            _, norms = kop.kop_lp_normalize_rows(xo[1:n + 1].view(rows, cols), 2, 1e-12, out=yo[yoff:n + yoff].view(rows, cols))
+            assert_close(yo[yoff:n + yoff].view(rows, cols), ry, tol_of(dtype), f"lp_normalize off the grid, y offset {yoff}")
+            assert np.all(np.abs(to_f64(norms) - rn) <= 1e-5 * np.maximum(1e-30, np.abs(rn)))
+            assert bool((yo[:yoff] == 9.0).all()) and bool((yo[n + yoff:] == 9.0).all())
+        xi = xo[1:n + 1].view(rows, cols)
+        kop.kop_lp_normalize_rows(xi, 2, 1e-12, out=xi)
+        assert_close(xi, ry, tol_of(dtype), "lp_normalize off the grid, in place")
