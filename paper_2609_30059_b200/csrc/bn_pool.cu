@@ -104,7 +104,8 @@ struct BnRaw {
 template <typename T, typename PT, int VB, int L>
 __global__ void __launch_bounds__(256)
 bn_plane_group_kernel(const T* __restrict__ x, const PT* __restrict__ scale, const PT* __restrict__ shift,
-                      T* __restrict__ y, float* __restrict__ pooled, int64_t planes, int plane, int C, float inv_plane)
+                      T* __restrict__ y, float* __restrict__ pooled, int64_t planes, int plane, int C, float inv_plane,
+                      int64_t p_first = 0)                   // index of plane 0 in the tensor (its channel is p_first mod C)
 {
     constexpr int EV = VB / (int)sizeof(T);
     constexpr int U = VB >= 16 ? 4 : (VB == 8 ? 8 : 16);
@@ -114,7 +115,7 @@ bn_plane_group_kernel(const T* __restrict__ x, const PT* __restrict__ scale, con
     const bool live = p < planes;
     float sc = 1.0f, sh = 0.0f;
     if (live) {
-        const int c = (int)(p % C);
+        const int c = (int)((p_first + p) % C);
         sc = param1(scale, c);
         sh = param1(shift, c);
     }
@@ -198,6 +199,80 @@ bn_plane_group_kernel(const T* __restrict__ x, const PT* __restrict__ scale, con
     if (live && sub == 0) pooled[p] = sum * inv_plane;
 }
 
+// ---- planes that are not whole vectors, bundled -----------------------------------------------------------------
+// A 7 x 7 plane is 196 bytes of fp32 or 98 of bf16: nothing wider than one element divides it, and element accesses
+// are bound by the L1 (7 x 7 fp32 4.4 TB/s, bf16 2.1; the head of every ResNet). B consecutive planes (2, 4 or 8)
+// together are a whole number of 16-byte vectors, so a team of L lanes takes such a bundle: 16-byte loads and stores
+// over the bundle, every vector's elements in at most two planes (scale / shift picked per element between the two),
+// the activations parked in shared memory as fp32, and after a warp barrier one lane per plane adds its plane's
+// values in index order.
+__device__ __forceinline__ int bn_div_small(int i, int d, float inv_d)
+{
+    int q = (int)((float)i * inv_d);
+    const int r = i - q * d;
+    q += (r >= d) ? 1 : 0;
+    q -= (r < 0) ? 1 : 0;
+    return q;
+}
+
+template <typename T, typename PT, int L>
+__global__ void __launch_bounds__(256)
+bn_bundle_kernel(const T* __restrict__ x, const PT* __restrict__ scale, const PT* __restrict__ shift,
+                 T* __restrict__ y, float* __restrict__ pooled, int64_t bundles, int B, int plane, int nvec, int C,
+                 float inv_plane, float inv_plane_f, int tile_floats)
+{
+    constexpr int E = Elem<T>::kPerVec, NV = 8;
+    extern __shared__ __align__(16) float bn_tile[];
+    const int sub = threadIdx.x & (L - 1), team = threadIdx.x / L;
+    const int64_t b = (int64_t)blockIdx.x * (blockDim.x / L) + team;
+    const bool live = b < bundles;
+    float* tile = bn_tile + team * tile_floats;
+    const int64_t p0 = (live ? b : 0) * B;
+    const T* xb = x + p0 * plane;
+    T* yb = y + p0 * plane;
+    const int c_p0 = (int)(p0 % C);
+    const int n = live ? nvec : 0;
+    Vec16 raw[NV];
+#pragma unroll
+    for (int k = 0; k < NV; ++k) {
+        const int v = k * L + sub;
+        if (v < n) raw[k] = ld_stream(xb + (int64_t)v * E);
+    }
+#pragma unroll
+    for (int k = 0; k < NV; ++k) {
+        const int v = k * L + sub;
+        if (v < n) {
+            const int i0 = v * E;
+            const int pl = bn_div_small(i0, plane, inv_plane_f);
+            const int left = plane - (i0 - pl * plane);              // elements of this vector in plane pl
+            int c = c_p0 + pl;
+            while (c >= C) c -= C;
+            const float sc0 = param1(scale, c), sh0 = param1(shift, c);
+            float sc1 = sc0, sh1 = sh0;
+            if (left < E) {
+                const int c1 = c + 1 == C ? 0 : c + 1;
+                sc1 = param1(scale, c1);
+                sh1 = param1(shift, c1);
+            }
+            float f[E];
+            Elem<T>::unpack(raw[k], f);
+#pragma unroll
+            for (int e = 0; e < E; ++e) f[e] = relu_keep_nan(fmaf(f[e], e < left ? sc0 : sc1, e < left ? sh0 : sh1));
+            float4* dst = reinterpret_cast<float4*>(tile + i0);
+#pragma unroll
+            for (int q = 0; q < E / 4; ++q) dst[q] = make_float4(f[4 * q], f[4 * q + 1], f[4 * q + 2], f[4 * q + 3]);
+            st_stream(yb + i0, Elem<T>::pack(f));
+        }
+    }
+    __syncwarp();
+    if (live && sub < B) {
+        const float* t = tile + sub * plane;
+        float s = 0.0f;
+        for (int j = 0; j < plane; ++j) s += t[j];
+        pooled[p0 + sub] = s * inv_plane;
+    }
+}
+
 // Large planes that cannot be vectorised: one CTA per plane, scalar loads.
 template <typename T, typename PT>
 __global__ void __launch_bounds__(256)
@@ -237,12 +312,45 @@ kop_status_t launch_bn(const void* xv, const void* scalev, const void* shiftv, v
     // planes of at most 1024 elements: lanes per plane. (A warp per plane, and for planes that are not whole vectors
     // runs of planes copied flat through shared memory, were here before: fp32 28 x 28 / 14 x 14 / 7 x 7 planes 5.4 / 5.1 /
     // 3.2 TB/s, bf16 3.8 / 2.6 / 1.8; now 6.1 / 6.3 / 4.0 and 5.8 / 5.5 / 1.9.)
+    // planes that nothing wider than four bytes divides, in bundles of 4 or 8 (7 x 7: 49 vectors a bundle for every data
+    // type; fp32 / bf16 TB/s 4.4 / 2.1 from the lanes-per-plane kernel, 5.6 / 3.1 here). Planes that 8-byte accesses
+    // divide stay there (bf16 14 x 14 and 10 x 10: 6.1 / 5.4 against 2.9 / 3.4 in bundles of two).
+    if (plane <= 256 && plane >= E && aligned_to(x, 16) && aligned_to(y, 16) && (plane * sizeof(T)) % 8 != 0) {
+        const int pbytes = (int)plane * (int)sizeof(T);
+        int B = 2;
+        while ((B * pbytes) % 16 != 0) B *= 2;                       // at most 8: a plane is a whole number of elements
+        const int nvec = B * pbytes / 16;
+        const int64_t bundles = planes / B, rest = planes - bundles * B;
+        const int L = nvec <= 64 ? 8 : 16;
+        const int tile_floats = (B * (int)plane + 3) / 4 * 4;
+        int threads = 256;                                           // the teams' tiles stay within the default 48 KB
+        while (threads > 32 && (size_t)(threads / L) * tile_floats * sizeof(float) > 46 * 1024) threads /= 2;
+        const int teams = threads / L;
+        const int64_t ctas = (bundles + teams - 1) / teams;
+        const size_t smem = (size_t)teams * tile_floats * sizeof(float);
+        if (nvec <= 128 && bundles > 0 && ctas <= 0x7FFFFFFFLL && smem <= 46 * 1024) {
+            const float inv_plane_f = 1.0f / (float)plane;
+            if (L == 8)
+                bn_bundle_kernel<T, PT, 8><<<(unsigned)ctas, threads, smem, stream>>>(x, scale, shift, y, pooled, bundles, B, (int)plane, nvec, (int)C, inv_plane, inv_plane_f, tile_floats);
+            else
+                bn_bundle_kernel<T, PT, 16><<<(unsigned)ctas, threads, smem, stream>>>(x, scale, shift, y, pooled, bundles, B, (int)plane, nvec, (int)C, inv_plane, inv_plane_f, tile_floats);
+            if (rest > 0) {
+                // the planes after the last whole bundle: lanes per plane with element accesses
+                const int64_t pf = bundles * B;
+                bn_plane_group_kernel<T, PT, (int)sizeof(T), 8><<<(unsigned)((rest + 31) / 32), 256, 0, stream>>>(
+                    x + pf * plane, scale, shift, y + pf * plane, pooled + pf, rest, (int)plane, (int)C, inv_plane, pf);
+            }
+            return launch_status();
+        }
+    }
     if (plane <= 1024 && planes <= 0x7FFFFFFFLL * 8) {
         const int pbytes = (int)plane * (int)sizeof(T);
         const int vb = (pbytes % 16 == 0 && aligned_to(x, 16) && aligned_to(y, 16)) ? 16
                        : (pbytes % 8 == 0 && aligned_to(x, 8) && aligned_to(y, 8)) ? 8
                        : (pbytes % 4 == 0 && aligned_to(x, 4) && aligned_to(y, 4)) ? 4 : (int)sizeof(T);
-        const int units = pbytes / vb, per_lane = vb >= 16 ? 4 : (vb == 8 ? 8 : 16);
+        // loads a lane: 64 bytes in flight with 16- and 8-byte units; eight narrower ones, so that more lanes share a plane
+        // and a warp's load covers longer runs (7 x 7 fp32 / bf16 planes: 4.4 / 2.1 TB/s with sixteen, 5.0 / 2.6 with eight)
+        const int units = pbytes / vb, per_lane = vb >= 16 ? 4 : 8;
         int L = 2;
         while (L < 32 && L * per_lane < units) L *= 2;
         const int per_cta = 8 * (32 / L);

@@ -313,13 +313,13 @@ def test_layernorm_options(kop):
 BN_SHAPES = [
     (8, 256, 56, 56, F32),     # benchmark plane
     (3, 5, 56, 56, BF16),
-    (4, 16, 7, 7, F32),        # small odd plane: 4-byte loads
+    (4, 16, 7, 7, F32),        # small odd plane: bundles of four planes
     (4, 16, 14, 14, F32),      # small plane: 16-byte loads
     (2, 3, 112, 112, F32),     # multi-trip plane
     (2, 7, 33, 35, F32),       # large odd plane: scalar CTA
     (5, 3, 1, 1, F32),
     (2, 8, 64, 64, BF16),
-    (16, 2048, 7, 7, BF16),    # 98-byte planes: single-element loads, four lanes a plane
+    (16, 2048, 7, 7, BF16),    # 98-byte planes: bundles of eight
     (3, 5, 7, 7, BF16),
     (3, 5, 14, 14, BF16),      # 392-byte planes: 8-byte loads
     (2, 3, 5, 9, torch.float16),
@@ -327,6 +327,16 @@ BN_SHAPES = [
     (2, 3, 31, 31, F32),       # 961-element planes, four per run
     (7, 9, 3, 3, F32),
     (2, 1100, 1, 1, BF16),     # one element per plane, runs of 1024 planes
+    # planes that are not whole vectors in bundles of 2, 4 or 8: planes left over after the last bundle, vectors that
+    # straddle two planes and two channels, channel indices that wrap inside a bundle, 16 lanes a bundle
+    (3, 5, 7, 7, F32),         # 15 planes: three bundles of four and three planes left over
+    (1, 3, 7, 7, BF16),        # fewer planes than a bundle of eight: the lanes-per-plane kernel alone
+    (5, 2, 7, 7, torch.float16),   # C = 2: the channel wraps four times inside a bundle
+    (2, 9, 9, 9, F32),         # 81 vectors a bundle
+    (3, 7, 9, 11, BF16),       # 198-byte planes: bundles of eight, 99 vectors each, 16 lanes a bundle
+    (4, 6, 5, 5, F32),
+    (2, 11, 3, 3, BF16),       # 9-element planes, eight a bundle
+    (3, 1, 13, 13, torch.float16),
 ]
 
 
