@@ -95,6 +95,12 @@ POOL_CASES = [
     (1, 2, 224, 224, (224, 224), (1, 1), (0, 0), F32),
     (70, 3, 2, 2, (2, 2), (1, 1), (0, 0), F32),
     (33, 7, 1, 1, (1, 1), (1, 1), (0, 0), BF16),
+    # global pooling of planes that nothing wider than four bytes divides
+    (2, 9, 9, 9, (9, 9), (1, 1), (0, 0), F32),
+    (4, 6, 5, 5, (5, 5), (1, 1), (0, 0), torch.float16),
+    (5, 2, 7, 7, (7, 7), (1, 1), (0, 0), BF16),
+    (1, 3, 7, 7, (7, 7), (1, 1), (0, 0), F32),
+    (3, 7, 9, 11, (9, 11), (1, 1), (0, 0), BF16),
     # 3 x 3 / stride 2 on rows that are not whole 8-column segments: the strip walk with aligned window loads, every
     # offset of a row from a 16-byte boundary (odd widths), a ragged last group of outputs, one band and several, a
     # bottom padding row (odd height with padding), planes from 256 elements
