@@ -920,8 +920,10 @@ constexpr size_t kGnStageLimit = 200 * 1024;     // leaves room for the static r
 static_assert(kGnStageLimit <= (size_t)kGnMaxParts * kGnCopyVecs * 16, "one barrier per 32 KB part");
 constexpr int kMaxDevices = 64;
 
-// beyond 40 KB (more than ten warps a team) the staged kernel is ahead: bf16 chunks of 49 KB 4.7 against 4.1 TB/s
-constexpr int64_t kGnRegMaxBytes = 40 * 1024;
+// beyond 40 KB (more than ten warps a team) the staged kernel is ahead: bf16 chunks of 49 KB 4.7 against 4.1 TB/s; where
+// the staged kernel cannot take the chunk (planes that are not whole vectors) the register kernel goes on to its limit
+// of sixteen warps a team, 64 KB (the alternative is the scalar kernel at 0.8 TB/s)
+constexpr int64_t kGnRegMaxBytes = 40 * 1024, kGnRegMaxBytesUnstaged = 64 * 1024;
 
 // Launches the register kernel when the chunk fits a team; false when it does not.
 template <typename T, typename PT, int VB, bool kStraddle>
@@ -965,7 +967,8 @@ bool launch_gn_reg(const T* x, const PT* gamma, const PT* beta, T* y, float* mea
 {
     constexpr int esz = (int)sizeof(T);
     const int64_t bytes = chunk_elems * esz;
-    if (bytes > kGnRegMaxBytes) return false;
+    const bool staged_ok = aligned_to(x, 16) && aligned_to(y, 16) && plane % Elem<T>::kPerVec == 0;
+    if (bytes > (staged_ok ? kGnRegMaxBytes : kGnRegMaxBytesUnstaged)) return false;
     int vb = 16;
     while (vb > esz && (bytes % vb != 0 || !aligned_to(x, vb) || !aligned_to(y, vb) || vb / esz > plane)) vb >>= 1;
 #define KOP_GN_REG(VB)                                                                                                \

@@ -70,6 +70,9 @@ GN_SHAPES = [
     (7, 24, 10, 10, 12, BF16, 0),      # 25 units of 16 bytes: 8 lanes, four units a lane at most
     (3, 20, 32, 32, 2, F32, 2),        # 40 KB: ten warps a chunk, the longest register chunk
     (2, 22, 32, 32, 2, F32, 0),        # 44 KB: the first staged chunk
+    (2, 256, 14, 14, 2, BF16, 2),      # 49 KB of planes that are not whole vectors: thirteen warps a chunk in registers
+    (2, 330, 7, 7, 1, F32, 1),         # 63 KB, sixteen warps; one channel more would be the scalar kernel
+    (2, 340, 7, 7, 1, F32, 1),         # 65 KB: the scalar kernel
     (6, 40, 7, 7, 1, F32, 0),          # groups == 1, chunk of 1960
 ]
 
