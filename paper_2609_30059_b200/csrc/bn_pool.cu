@@ -215,13 +215,13 @@ __device__ __forceinline__ int bn_div_small(int i, int d, float inv_d)
     return q;
 }
 
-template <typename T, typename PT, int L>
+template <typename T, typename PT, int L, int NV>
 __global__ void __launch_bounds__(256)
 bn_bundle_kernel(const T* __restrict__ x, const PT* __restrict__ scale, const PT* __restrict__ shift,
                  T* __restrict__ y, float* __restrict__ pooled, int64_t bundles, int B, int plane, int nvec, int C,
                  float inv_plane, float inv_plane_f, int tile_floats)
 {
-    constexpr int E = Elem<T>::kPerVec, NV = 8;
+    constexpr int E = Elem<T>::kPerVec;
     extern __shared__ __align__(16) float bn_tile[];
     const int sub = threadIdx.x & (L - 1), team = threadIdx.x / L;
     const int64_t b = (int64_t)blockIdx.x * (blockDim.x / L) + team;
@@ -321,7 +321,11 @@ kop_status_t launch_bn(const void* xv, const void* scalev, const void* shiftv, v
         while ((B * pbytes) % 16 != 0) B *= 2;                       // at most 8: a plane is a whole number of elements
         const int nvec = B * pbytes / 16;
         const int64_t bundles = planes / B, rest = planes - bundles * B;
-        const int L = nvec <= 64 ? 8 : 16;
+        // fp32: eight lanes a bundle, eight vectors a lane. 16-bit data: sixteen lanes, four vectors a lane, 46 registers
+        // instead of 64 (bf16 7 x 7 with eight lanes: warps active 46 %, long-scoreboard stalls first, 3.1 TB/s; 4.2 this
+        // way; fp32 the other way round, 5.6 against 5.1). Beyond 64 vectors a bundle: sixteen lanes, eight vectors.
+        const bool wide = sizeof(T) == 2 || nvec > 64;
+        const int L = wide ? 16 : 8;
         const int tile_floats = (B * (int)plane + 3) / 4 * 4;
         int threads = 256;                                           // the teams' tiles stay within the default 48 KB
         while (threads > 32 && (size_t)(threads / L) * tile_floats * sizeof(float) > 46 * 1024) threads /= 2;
@@ -330,10 +334,12 @@ kop_status_t launch_bn(const void* xv, const void* scalev, const void* shiftv, v
         const size_t smem = (size_t)teams * tile_floats * sizeof(float);
         if (nvec <= 128 && bundles > 0 && ctas <= 0x7FFFFFFFLL && smem <= 46 * 1024) {
             const float inv_plane_f = 1.0f / (float)plane;
-            if (L == 8)
-                bn_bundle_kernel<T, PT, 8><<<(unsigned)ctas, threads, smem, stream>>>(x, scale, shift, y, pooled, bundles, B, (int)plane, nvec, (int)C, inv_plane, inv_plane_f, tile_floats);
-            else
-                bn_bundle_kernel<T, PT, 16><<<(unsigned)ctas, threads, smem, stream>>>(x, scale, shift, y, pooled, bundles, B, (int)plane, nvec, (int)C, inv_plane, inv_plane_f, tile_floats);
+#define KOP_BN_BUNDLE(LL, NVV) \
+    bn_bundle_kernel<T, PT, LL, NVV><<<(unsigned)ctas, threads, smem, stream>>>(x, scale, shift, y, pooled, bundles, B, (int)plane, nvec, (int)C, inv_plane, inv_plane_f, tile_floats)
+            if (!wide) KOP_BN_BUNDLE(8, 8);
+            else if (nvec <= 64) KOP_BN_BUNDLE(16, 4);
+            else KOP_BN_BUNDLE(16, 8);
+#undef KOP_BN_BUNDLE
             if (rest > 0) {
                 // the planes after the last whole bundle: lanes per plane with element accesses
                 const int64_t pf = bundles * B;
