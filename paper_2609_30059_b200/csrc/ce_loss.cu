@@ -416,7 +416,10 @@ kop_status_t launch_ce(const void* zv, const int32_t* labels, float* loss, float
     const int64_t nvec64 = vocab / E;
     if (vocab * (int64_t)sizeof(T) <= 16384) {
         const int nvec = (int)nvec64;
-        const int lanes = nvec >= 512 ? 32 : nvec >= 256 ? 16 : nvec >= 128 ? 8 : 4;
+        // up to 32 vectors a lane (eight batches): bf16 rows of 4096 classes 4.7 TB/s with 16 a lane, 5.8 with 32 (5.7 with
+        // 64, 4.9 with 128); fp32 rows of 2048 classes 4.5 / 5.8 / 5.9 / 5.2
+        int lanes = 4;
+        while (lanes < 32 && lanes * 32 < nvec) lanes *= 2;
         const int64_t rows_per_cta = 8 * (32 / lanes);
         const unsigned grid = (unsigned)((rows + rows_per_cta - 1) / rows_per_cta);
 #define KOP_CE_G(L, SM) ce_group_kernel<T, L, kOpts, SM><<<grid, 256, 0, stream>>>(z, labels, loss, mean_loss, bad, ws, rows, stride, vocab, opts)
