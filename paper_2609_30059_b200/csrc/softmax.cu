@@ -93,7 +93,7 @@ softmax_warp_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __r
         for (int q = 0; q < E / 4; ++q) {
             float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
             if constexpr (kRagged) {
-                if (bias != nullptr && v < nvec) {
+                if (kBias && v < nvec) {
                     const int j = head + v * E + 4 * q;
                     b = make_float4(param1(bias, j), param1(bias, j + 1), param1(bias, j + 2), param1(bias, j + 3));
                 }
@@ -116,7 +116,7 @@ softmax_warp_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __r
 #pragma unroll
         for (int q = 0; q < KE; ++q) {
             if (edge_col[q] >= 0) {
-                const float b = bias != nullptr ? param1(bias, edge_col[q]) * kLog2e : 0.0f;
+                const float b = kBias ? param1(bias, edge_col[q]) * kLog2e : 0.0f;
                 te[q] = fmaf(Elem<T>::load1(xr - head + edge_col[q]), s2, b);
             }
             m = fmaxf(m, te[q]);
@@ -179,7 +179,8 @@ __device__ __forceinline__ int64_t last_visible(const SmOpts& o, int64_t row)
 // general form tests both at run time.
 // kRagged: rows that are not whole aligned vectors, split as in the warp kernel (opts.cols carries the row length),
 // one edge element to a thread.
-template <typename T, typename PT, int VPT, bool kOpts, bool kPlain, bool kLog = false, bool kRagged = false>
+template <typename T, typename PT, int VPT, bool kOpts, bool kPlain, bool kLog = false, bool kRagged = false,
+          bool kRagBias = false>                             // kRagBias: ragged rows with a bias (its element loads compiled in)
 __global__ void __launch_bounds__(max_threads_for(VPT * Elem<T>::kPerVec))
 softmax_block_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __restrict__ y,
                      int nvec, int64_t x_stride, int64_t y_stride, float scale, SmOpts opts)
@@ -222,7 +223,7 @@ softmax_block_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __
         for (int q = 0; q < E / 4; ++q) {
             float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
             if constexpr (kRagged) {
-                if (bias != nullptr && v < nvec) {
+                if (kRagBias && v < nvec) {
                     const int j = head + v * E + 4 * q;
                     b = make_float4(param1(bias, j), param1(bias, j + 1), param1(bias, j + 2), param1(bias, j + 3));
                 }
@@ -242,7 +243,7 @@ softmax_block_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __
     float te = -INFINITY;                                    // this thread's edge element
     if constexpr (kRagged) {
         if (edge_col >= 0) {
-            const float b = bias != nullptr ? param1(bias, edge_col) * kLog2e : 0.0f;
+            const float b = kRagBias ? param1(bias, edge_col) * kLog2e : 0.0f;
             te = fmaf(Elem<T>::load1(xr - head + edge_col), s2, b);
         }
         m = fmaxf(m, te);
@@ -552,6 +553,23 @@ kop_status_t launch_softmax(const void* xv, const void* biasv, void* yv, int64_t
         // slower than the form that tests the pointer at run time (bf16 8192 columns, fp32 bias: 5.1 to 4.5), so rows
         // with a bias keep that form
         const bool full = nvec % vpt == 0 && nvec / vpt == threads;
+        if (!full && bias == nullptr && (!with_opts || log_only)) {
+            // rows that do not fill the CTA exactly, without a bias: the split-row variant, which has no bias code at all
+            // (the general form keeps the bias loads as predicated-off instructions: fp32 rows of 1000 columns 5.2 TB/s
+            // there, 6.4 here)
+#define KOP_SM_BLOCK_NB(V)                                                                                                         \
+    do {                                                                                                                          \
+        if (log_only) softmax_block_kernel<T, PT, V, false, false, true, true, false><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, 0, xs, ys, scale, opts); \
+        else softmax_block_kernel<T, PT, V, false, false, false, true, false><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, 0, xs, ys, scale, opts); \
+    } while (0)
+            switch (vpt * E) {
+            case 16: KOP_SM_BLOCK_NB(16 / E); break;
+            case 32: KOP_SM_BLOCK_NB(32 / E); break;
+            default: KOP_SM_BLOCK_NB(64 / E); break;
+            }
+#undef KOP_SM_BLOCK_NB
+            return launch_status();
+        }
 #define KOP_SM_BLOCK_L(V, O, P) \
     softmax_block_kernel<T, PT, V, O, P><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, nvec, xs, ys, scale, opts)
 #define KOP_SM_BLOCK(V)                                                          \
@@ -600,16 +618,24 @@ kop_status_t launch_softmax(const void* xv, const void* biasv, void* yv, int64_t
         const int64_t ctas = (rows + rows_per_cta - 1) / rows_per_cta;
         if (ctas > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
         const unsigned grid = (unsigned)ctas;
-#define KOP_SM_RAG(V, L)                                                                                               \
+#define KOP_SM_RAG_B(V, L, B)                                                                                          \
     do {                                                                                                               \
-        if (log_only) softmax_warp_kernel<T, PT, V, false, false, L, true, false, true><<<grid, 256, 0, stream>>>(x, bias, y, rows, (int)cols, xs, ys, scale); \
-        else softmax_warp_kernel<T, PT, V, false, false, L, false, false, true><<<grid, 256, 0, stream>>>(x, bias, y, rows, (int)cols, xs, ys, scale); \
+        if (log_only) softmax_warp_kernel<T, PT, V, false, B, L, true, false, true><<<grid, 256, 0, stream>>>(x, bias, y, rows, (int)cols, xs, ys, scale); \
+        else softmax_warp_kernel<T, PT, V, false, B, L, false, false, true><<<grid, 256, 0, stream>>>(x, bias, y, rows, (int)cols, xs, ys, scale); \
+    } while (0)
+    // the bias as a compile-time variant: tested at run time its element loads stay in the code as predicated-off
+    // instructions (1.6 load instructions an element on rows without a bias)
+#define KOP_SM_RAG(V, L)                        \
+    do {                                        \
+        if (bias != nullptr) KOP_SM_RAG_B(V, L, true); \
+        else KOP_SM_RAG_B(V, L, false);         \
     } while (0)
         if (lanes == 8 && vp == 2) KOP_SM_RAG(2, 8);
         else if (lanes == 8) KOP_SM_RAG(4, 8);
         else if (vp == 2) KOP_SM_RAG(2, 32);
         else KOP_SM_RAG(4, 32);
 #undef KOP_SM_RAG
+#undef KOP_SM_RAG_B
         return launch_status();
     }
     if (ragged && cols <= kMaxRegisterRow && cols * (int64_t)sizeof(T) <= 32768) {
@@ -617,10 +643,15 @@ kop_status_t launch_softmax(const void* xv, const void* biasv, void* yv, int64_t
         int vpt = (cols >= 2048 ? 32 : 16) / E;
         while (vpt * E < 64 && (nvec + vpt - 1) / vpt > max_threads_for(vpt * E)) vpt *= 2;
         const int threads = ((nvec + vpt - 1) / vpt + 31) / 32 * 32;
-#define KOP_SM_BLOCK_RAG(V)                                                                                                       \
+#define KOP_SM_BLOCK_RAG_B(V, B)                                                                                                  \
     do {                                                                                                                          \
-        if (log_only) softmax_block_kernel<T, PT, V, false, false, true, true><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, 0, xs, ys, scale, opts); \
-        else softmax_block_kernel<T, PT, V, false, false, false, true><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, 0, xs, ys, scale, opts); \
+        if (log_only) softmax_block_kernel<T, PT, V, false, false, true, true, B><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, 0, xs, ys, scale, opts); \
+        else softmax_block_kernel<T, PT, V, false, false, false, true, B><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, 0, xs, ys, scale, opts); \
+    } while (0)
+#define KOP_SM_BLOCK_RAG(V)                              \
+    do {                                                 \
+        if (bias != nullptr) KOP_SM_BLOCK_RAG_B(V, true); \
+        else KOP_SM_BLOCK_RAG_B(V, false);               \
     } while (0)
         switch (vpt * E) {
         case 16: KOP_SM_BLOCK_RAG(16 / E); break;
@@ -628,6 +659,7 @@ kop_status_t launch_softmax(const void* xv, const void* biasv, void* yv, int64_t
         default: KOP_SM_BLOCK_RAG(64 / E); break;
         }
 #undef KOP_SM_BLOCK_RAG
+#undef KOP_SM_BLOCK_RAG_B
         return launch_status();
     }
     if (ragged) {
