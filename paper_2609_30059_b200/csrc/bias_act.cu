@@ -48,7 +48,9 @@ __device__ __forceinline__ float act_dev(float u, float alpha)
 
 // kFlat: rows shorter than a tile; the CTA takes U * blockDim.x vectors in row-major order across rows
 // (nvec_total = rows * nvec). Otherwise a CTA is one tile of one row.
-template <typename T, typename PT, int ACT, bool kFlat>
+// kBias: a bias is present (a compile-time variant: tested at run time, its loads and adds stay in the code of the
+// activation-only call as predicated-off instructions)
+template <typename T, typename PT, int ACT, bool kFlat, bool kBias>
 __global__ void __launch_bounds__(256)
 bias_act_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __restrict__ y, int nvec,
                 int tiles_per_row, int64_t nvec_total, int64_t x_stride, int64_t y_stride, float alpha)
@@ -85,7 +87,7 @@ bias_act_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __restr
         if (live[k]) {
             float f[E];
             Elem<T>::unpack(raw[k], f);
-            if (bias != nullptr) {
+            if (kBias) {
 #pragma unroll
                 for (int q = 0; q < E / 4; ++q) {
                     const float4 b = ldg_p4(bias + (int64_t)v[k] * E + 4 * q);
@@ -368,12 +370,14 @@ kop_status_t launch_bias_act_a(const T* x, const PT* bias, T* y, int64_t rows, i
         if (nvec < 128 || ((int64_t)tiles * 4 * threads - nvec) * 4 > nvec) {
             const int64_t total = rows * nvec, grid = (total + 1023) / 1024;
             if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
-            bias_act_kernel<T, PT, ACT, true><<<(unsigned)grid, 256, 0, stream>>>(x, bias, y, nvec, 1, total, xs, ys, alpha);
+            if (bias != nullptr) bias_act_kernel<T, PT, ACT, true, true><<<(unsigned)grid, 256, 0, stream>>>(x, bias, y, nvec, 1, total, xs, ys, alpha);
+            else bias_act_kernel<T, PT, ACT, true, false><<<(unsigned)grid, 256, 0, stream>>>(x, bias, y, nvec, 1, total, xs, ys, alpha);
             return launch_status();
         }
         const int64_t grid = rows * tiles;
         if (grid > 0x7FFFFFFFLL) return KOP_ERR_BAD_SHAPE;
-        bias_act_kernel<T, PT, ACT, false><<<(unsigned)grid, threads, 0, stream>>>(x, bias, y, nvec, tiles, 0, xs, ys, alpha);
+        if (bias != nullptr) bias_act_kernel<T, PT, ACT, false, true><<<(unsigned)grid, threads, 0, stream>>>(x, bias, y, nvec, tiles, 0, xs, ys, alpha);
+        else bias_act_kernel<T, PT, ACT, false, false><<<(unsigned)grid, threads, 0, stream>>>(x, bias, y, nvec, tiles, 0, xs, ys, alpha);
         return launch_status();
     }
     if (launch_span<T, PT, ACT, false>(x, bias, static_cast<const T*>(nullptr), y, rows, cols, xs, 0, ys,
