@@ -180,7 +180,7 @@ __device__ __forceinline__ int64_t last_visible(const SmOpts& o, int64_t row)
 // kRagged: rows that are not whole aligned vectors, split as in the warp kernel (opts.cols carries the row length),
 // one edge element to a thread.
 template <typename T, typename PT, int VPT, bool kOpts, bool kPlain, bool kLog = false, bool kRagged = false,
-          bool kRagBias = false>                             // kRagBias: ragged rows with a bias (its element loads compiled in)
+          bool kRagBias = false>                             // kRagBias: ragged or kOpts rows with a bias (its loads compiled in)
 __global__ void __launch_bounds__(max_threads_for(VPT * Elem<T>::kPerVec))
 softmax_block_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __restrict__ y,
                      int nvec, int64_t x_stride, int64_t y_stride, float scale, SmOpts opts)
@@ -228,7 +228,9 @@ softmax_block_kernel(const T* __restrict__ x, const PT* __restrict__ bias, T* __
                     b = make_float4(param1(bias, j), param1(bias, j + 1), param1(bias, j + 2), param1(bias, j + 3));
                 }
             } else {
-                if (!kPlain && bias != nullptr && v < nvec) b = ldg_p4(bias + (int64_t)v * E + 4 * q);
+                // the causal / log form tests the bias at compile time (kRagBias); the plain general form at run time,
+                // where a compile-time variant measured slower on rows with a bias
+                if (!kPlain && (!kOpts || kRagBias) && bias != nullptr && v < nvec) b = ldg_p4(bias + (int64_t)v * E + 4 * q);
             }
             const float bb[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
@@ -574,7 +576,8 @@ kop_status_t launch_softmax(const void* xv, const void* biasv, void* yv, int64_t
     softmax_block_kernel<T, PT, V, O, P><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, nvec, xs, ys, scale, opts)
 #define KOP_SM_BLOCK(V)                                                          \
     do {                                                                         \
-        if (with_opts && !log_only) KOP_SM_BLOCK_L(V, true, false);              \
+        if (with_opts && !log_only && bias != nullptr) softmax_block_kernel<T, PT, V, true, false, false, false, true><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, nvec, xs, ys, scale, opts); \
+        else if (with_opts && !log_only) KOP_SM_BLOCK_L(V, true, false);         \
         else if (log_only && full && bias == nullptr) softmax_block_kernel<T, PT, V, false, true, true><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, nvec, xs, ys, scale, opts); \
         else if (log_only) softmax_block_kernel<T, PT, V, false, false, true><<<(unsigned)rows, threads, 0, stream>>>(x, bias, y, nvec, xs, ys, scale, opts); \
         else if (full && bias == nullptr) KOP_SM_BLOCK_L(V, false, true);        \
@@ -722,8 +725,9 @@ extern "C" kop_status_t kop_softmax_opts(const void* x, const float* bias, void*
                                          int64_t x_row_stride, int64_t y_row_stride, float scale, int log_output,
                                          int64_t causal_period, kop_dtype_t dtype, kop_stream_t stream)
 {
-    return kop::softmax_entry(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale, true, log_output, causal_period,
-                              dtype, KOP_F32, stream);
+    // no option set: the kernels of kop_softmax_scale_bias
+    return kop::softmax_entry(x, bias, y, rows, cols, x_row_stride, y_row_stride, scale,
+                              log_output != 0 || causal_period != 0, log_output, causal_period, dtype, KOP_F32, stream);
 }
 
 extern "C" kop_status_t kop_softmax_ex(const void* x, const void* bias, void* y, int64_t rows, int64_t cols,
